@@ -1,0 +1,659 @@
+/*
+ * CPU oracle for the imitation-step hot path.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, scalar restatement of what one control step computes outside
+ * the physics solver in the paper's training loop (Figure 2: reward and dones,
+ * masked reset, observation building, policy inference), written to be checked
+ * against the paper by eye.  It is not part of the product: only the tests,
+ * the smoke check and the benchmark's CPU-baseline leg call it, and it shares
+ * no code with the CUDA library.
+ *
+ * Precision: every quantity that is compared within a tolerance (observations,
+ * rewards, error terms, policy means, Gaussian draws) is computed in fp64.
+ * Every quantity that is compared bit for bit (the per-env time, keyframe
+ * index, flags, reset clip id and phase, Philox words) is computed with single
+ * IEEE fp32 operations or integers, so that any conforming fp32 implementation
+ * reproduces it exactly.  Build with -ffp-contract=off.
+ *
+ * Conventions (the paper fixes only the quaternion order, Figure 3a): right
+ * handed, z up, metres / seconds / radians, unit Hamilton quaternions stored
+ * w,x,y,z, R(q)v = q v q*, parent[0] = -1, parent[j] < j.
+ *
+ * Every function below has at least one pin in tests/ that does not restate
+ * its formula (closed forms, invariants, brute force with 3x3 matrices, the
+ * paper's Figure 5 constants, published Philox known answers).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_MAX_BODIES 32
+#define ORC_N_TERMS 7
+#define ORC_STREAM_RESET 0u
+#define ORC_STREAM_ACTION 1u
+
+#ifndef M_PI
+#define M_PI 3.14159265358979323846
+#endif
+
+/* ------------------------------------------------------------------------ */
+/* Philox4x32-10 (Salmon et al. 2011): counter-based generator the method    */
+/* draws its reset phases and action noise from.                             */
+/* ------------------------------------------------------------------------ */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+        uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Quaternion algebra, fp64.                                                 */
+/* ------------------------------------------------------------------------ */
+void orc_quat_mul(const double a[4], const double b[4], double out[4])
+{
+    double w = a[0]*b[0] - a[1]*b[1] - a[2]*b[2] - a[3]*b[3];
+    double x = a[0]*b[1] + a[1]*b[0] + a[2]*b[3] - a[3]*b[2];
+    double y = a[0]*b[2] - a[1]*b[3] + a[2]*b[0] + a[3]*b[1];
+    double z = a[0]*b[3] + a[1]*b[2] - a[2]*b[1] + a[3]*b[0];
+    out[0] = w; out[1] = x; out[2] = y; out[3] = z;
+}
+
+static void quat_conj(const double a[4], double out[4])
+{
+    out[0] = a[0]; out[1] = -a[1]; out[2] = -a[2]; out[3] = -a[3];
+}
+
+/* R(q) v = q (0,v) q*  written out as the product of the three quaternions. */
+void orc_quat_rotate(const double q[4], const double v[3], double out[3])
+{
+    double p[4] = {0.0, v[0], v[1], v[2]}, qc[4], t[4], r[4];
+    quat_conj(q, qc);
+    orc_quat_mul(q, p, t);
+    orc_quat_mul(t, qc, r);
+    out[0] = r[1]; out[1] = r[2]; out[2] = r[3];
+}
+
+static void quat_rotate_inv(const double q[4], const double v[3], double out[3])
+{
+    double qc[4];
+    quat_conj(q, qc);
+    orc_quat_rotate(qc, v, out);
+}
+
+static void quat_normalize(double q[4])
+{
+    double n = sqrt(q[0]*q[0] + q[1]*q[1] + q[2]*q[2] + q[3]*q[3]);
+    if (n > 0.0) { q[0] /= n; q[1] /= n; q[2] /= n; q[3] /= n; }
+    else { q[0] = 1.0; q[1] = q[2] = q[3] = 0.0; }
+}
+
+/* Half-angle rotation vector of a unit quaternion on the shortest arc:
+ * log(q) = v/|v| * atan2(|v|, w), with q negated first when w < 0. */
+void orc_quat_log(const double q_in[4], double out[3])
+{
+    double q[4] = {q_in[0], q_in[1], q_in[2], q_in[3]};
+    if (q[0] < 0.0) { q[0] = -q[0]; q[1] = -q[1]; q[2] = -q[2]; q[3] = -q[3]; }
+    double n = sqrt(q[1]*q[1] + q[2]*q[2] + q[3]*q[3]);
+    if (n < 1e-12) { out[0] = out[1] = out[2] = 0.0; return; }
+    double h = atan2(n, q[0]);
+    out[0] = q[1] / n * h; out[1] = q[2] / n * h; out[2] = q[3] / n * h;
+}
+
+/* Rotation angle in [0, pi] of a unit quaternion: 2 atan2(|v|, |w|). */
+double orc_geodesic_angle(const double q[4])
+{
+    double n = sqrt(q[1]*q[1] + q[2]*q[2] + q[3]*q[3]);
+    return 2.0 * atan2(n, fabs(q[0]));
+}
+
+/* Angle of the rotation taking frame a to frame b: theta(a* b). */
+static double rel_angle(const double a[4], const double b[4])
+{
+    double ac[4], r[4];
+    quat_conj(a, ac);
+    orc_quat_mul(ac, b, r);
+    return orc_geodesic_angle(r);
+}
+
+/* Shortest-arc spherical interpolation; normalised lerp when nearly equal. */
+void orc_slerp(const double q0[4], const double q1_in[4], double alpha, double out[4])
+{
+    double q1[4] = {q1_in[0], q1_in[1], q1_in[2], q1_in[3]};
+    double d = q0[0]*q1[0] + q0[1]*q1[1] + q0[2]*q1[2] + q0[3]*q1[3];
+    if (d < 0.0) { d = -d; for (int i = 0; i < 4; ++i) q1[i] = -q1[i]; }
+    double s0, s1;
+    if (d > 1.0 - 1e-6) { s0 = 1.0 - alpha; s1 = alpha; }
+    else {
+        double theta = acos(d), s = sin(theta);
+        s0 = sin((1.0 - alpha) * theta) / s;
+        s1 = sin(alpha * theta) / s;
+    }
+    for (int i = 0; i < 4; ++i) out[i] = s0 * q0[i] + s1 * q1[i];
+    quat_normalize(out);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Skeleton and clip library.                                                */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int J;
+    int parent[ORC_MAX_BODIES];
+    double offset[ORC_MAX_BODIES][3];
+    double mass[ORC_MAX_BODIES];
+    int n_ee;
+    int ee[ORC_MAX_BODIES];
+} orc_skeleton;
+
+typedef struct {
+    int C, J;
+    int *K;            /* keyframes per clip */
+    float *fps;        /* fp32, as given */
+    float *dur;        /* D_c = (K_c - 1) / fps_c, one fp32 division */
+    int64_t *start;    /* first frame of each clip in the packed tables */
+    double *root;      /* [sum K][3] */
+    double *quat;      /* [sum K][J][4], renormalised */
+} orc_clips;
+
+orc_skeleton *orc_skeleton_create(int J, const int32_t *parents, const float *offsets,
+                                  const float *masses, const int32_t *ee_ids, int n_ee)
+{
+    if (J < 1 || J > ORC_MAX_BODIES || parents[0] != -1) return NULL;
+    orc_skeleton *s = (orc_skeleton *)calloc(1, sizeof(*s));
+    s->J = J;
+    for (int j = 0; j < J; ++j) {
+        if (j > 0 && (parents[j] < 0 || parents[j] >= j)) { free(s); return NULL; }
+        s->parent[j] = parents[j];
+        for (int c = 0; c < 3; ++c) s->offset[j][c] = (double)offsets[3*j + c];
+        s->mass[j] = masses ? (double)masses[j] : 1.0;
+    }
+    if (ee_ids && n_ee > 0) {
+        s->n_ee = n_ee;
+        for (int i = 0; i < n_ee; ++i) s->ee[i] = ee_ids[i];
+    } else {            /* default end-effectors: bodies without children */
+        int has_child[ORC_MAX_BODIES] = {0};
+        for (int j = 1; j < J; ++j) has_child[parents[j]] = 1;
+        for (int j = 0; j < J; ++j) if (!has_child[j]) s->ee[s->n_ee++] = j;
+    }
+    return s;
+}
+
+void orc_skeleton_destroy(orc_skeleton *s) { free(s); }
+
+orc_clips *orc_clips_create(const orc_skeleton *skel, int C, const int32_t *n_frames,
+                            const float *fps, const float *root_pos, const float *local_quat)
+{
+    orc_clips *c = (orc_clips *)calloc(1, sizeof(*c));
+    int J = skel->J;
+    c->C = C; c->J = J;
+    c->K = (int *)malloc(sizeof(int) * C);
+    c->fps = (float *)malloc(sizeof(float) * C);
+    c->dur = (float *)malloc(sizeof(float) * C);
+    c->start = (int64_t *)malloc(sizeof(int64_t) * C);
+    int64_t total = 0;
+    for (int i = 0; i < C; ++i) {
+        c->K[i] = n_frames[i];
+        c->fps[i] = fps[i];
+        c->dur[i] = (float)(n_frames[i] - 1) / fps[i];
+        c->start[i] = total;
+        total += n_frames[i];
+    }
+    c->root = (double *)malloc(sizeof(double) * total * 3);
+    c->quat = (double *)malloc(sizeof(double) * total * J * 4);
+    for (int64_t i = 0; i < total * 3; ++i) c->root[i] = (double)root_pos[i];
+    for (int64_t i = 0; i < total * J; ++i) {
+        double q[4] = {local_quat[4*i], local_quat[4*i+1], local_quat[4*i+2], local_quat[4*i+3]};
+        quat_normalize(q);
+        memcpy(c->quat + 4*i, q, sizeof(q));
+    }
+    return c;
+}
+
+void orc_clips_destroy(orc_clips *c)
+{
+    if (!c) return;
+    free(c->K); free(c->fps); free(c->dur); free(c->start); free(c->root); free(c->quat); free(c);
+}
+
+float orc_clip_duration(const orc_clips *c, int clip) { return c->dur[clip]; }
+
+/* ------------------------------------------------------------------------ */
+/* Step a1: keyframe index and blend factor at time t.                       */
+/* f = fl32(t * fps); k = min(floor(f), K-2); alpha = f - k in [0,1].        */
+/* ------------------------------------------------------------------------ */
+void orc_lookup_index(float t, float fps, int K, int32_t *k_out, double *alpha_out)
+{
+    volatile float f = t * fps;           /* one fp32 multiply, round to nearest */
+    int k = (int)floorf(f);
+    if (k > K - 2) k = K - 2;
+    if (k < 0) k = 0;
+    double a = (double)f - (double)k;
+    if (a < 0.0) a = 0.0;
+    if (a > 1.0) a = 1.0;
+    *k_out = k; *alpha_out = a;
+}
+
+/* Reference character state at (clip, t): steps a1 + a2. */
+typedef struct {
+    double ql[ORC_MAX_BODIES][4];   /* local (parent-relative) rotations   */
+    double wl[ORC_MAX_BODIES][3];   /* joint angular velocity, child frame  */
+    double p[ORC_MAX_BODIES][3];    /* world positions                      */
+    double q[ORC_MAX_BODIES][4];    /* world rotations                      */
+    double v[ORC_MAX_BODIES][3];    /* world linear velocities              */
+    double w[ORC_MAX_BODIES][3];    /* world angular velocities             */
+    double com[3];
+} orc_ref;
+
+static void cross3(const double a[3], const double b[3], double out[3])
+{
+    out[0] = a[1]*b[2] - a[2]*b[1];
+    out[1] = a[2]*b[0] - a[0]*b[2];
+    out[2] = a[0]*b[1] - a[1]*b[0];
+}
+
+static void center_of_mass(const orc_skeleton *s, double p[][3], double com[3])
+{
+    double m = 0.0;
+    com[0] = com[1] = com[2] = 0.0;
+    for (int j = 0; j < s->J; ++j) {
+        m += s->mass[j];
+        for (int c = 0; c < 3; ++c) com[c] += s->mass[j] * p[j][c];
+    }
+    for (int c = 0; c < 3; ++c) com[c] /= m;
+}
+
+void orc_reference_state(const orc_skeleton *s, const orc_clips *cl, int clip, float t, orc_ref *r)
+{
+    int J = s->J, K = cl->K[clip], k;
+    double alpha, fps = (double)cl->fps[clip];
+    orc_lookup_index(t, cl->fps[clip], K, &k, &alpha);
+    const double *P0 = cl->root + 3 * (cl->start[clip] + k), *P1 = P0 + 3;
+    const double *Q0 = cl->quat + 4 * (int64_t)J * (cl->start[clip] + k), *Q1 = Q0 + 4 * J;
+
+    /* a1: slerp each joint, lerp the root, finite-difference velocities */
+    for (int j = 0; j < J; ++j) {
+        double q0c[4], rel[4], lg[3];
+        orc_slerp(Q0 + 4*j, Q1 + 4*j, alpha, r->ql[j]);
+        quat_conj(Q0 + 4*j, q0c);
+        orc_quat_mul(q0c, Q1 + 4*j, rel);
+        orc_quat_log(rel, lg);
+        for (int c = 0; c < 3; ++c) r->wl[j][c] = 2.0 * lg[c] * fps;
+    }
+    /* a2: forward kinematics with velocity propagation */
+    for (int c = 0; c < 3; ++c) {
+        r->p[0][c] = (1.0 - alpha) * P0[c] + alpha * P1[c];
+        r->v[0][c] = (P1[c] - P0[c]) * fps;
+    }
+    memcpy(r->q[0], r->ql[0], sizeof(double) * 4);
+    orc_quat_rotate(r->q[0], r->wl[0], r->w[0]);
+    for (int j = 1; j < J; ++j) {
+        int a = s->parent[j];
+        double arm[3], wj[3], wxr[3];
+        orc_quat_mul(r->q[a], r->ql[j], r->q[j]);
+        orc_quat_rotate(r->q[a], s->offset[j], arm);
+        orc_quat_rotate(r->q[j], r->wl[j], wj);
+        cross3(r->w[a], arm, wxr);
+        for (int c = 0; c < 3; ++c) {
+            r->p[j][c] = r->p[a][c] + arm[c];
+            r->w[j][c] = r->w[a][c] + wj[c];
+            r->v[j][c] = r->v[a][c] + wxr[c];
+        }
+    }
+    center_of_mass(s, r->p, r->com);
+}
+
+/* Flat export of orc_reference_state for the tests. */
+void orc_reference_state_flat(const orc_skeleton *s, const orc_clips *cl, int clip, float t,
+                              double *p, double *q, double *v, double *w,
+                              double *ql, double *wl, double *com)
+{
+    orc_ref r;
+    orc_reference_state(s, cl, clip, t, &r);
+    for (int j = 0; j < s->J; ++j) {
+        for (int c = 0; c < 3; ++c) {
+            p[3*j+c] = r.p[j][c]; v[3*j+c] = r.v[j][c]; w[3*j+c] = r.w[j][c]; wl[3*j+c] = r.wl[j][c];
+        }
+        for (int c = 0; c < 4; ++c) { q[4*j+c] = r.q[j][c]; ql[4*j+c] = r.ql[j][c]; }
+    }
+    for (int c = 0; c < 3; ++c) com[c] = r.com[c];
+}
+
+/* ------------------------------------------------------------------------ */
+/* Environment configuration (mirrors what a caller of the method chooses).  */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t mode;                   /* 0 multiplicative, 1 additive */
+    float a[ORC_N_TERMS];           /* additive coefficients */
+    float w[ORC_N_TERMS];           /* error scales; order: pose, vel, ee_pos, ee_rot, com, body_pos, body_vel */
+    float h_min;                    /* terminate when root height < h_min */
+    float r_min;                    /* terminate when reward < r_min (-inf: off) */
+} orc_reward_config;
+
+typedef struct {
+    float dt;
+    uint32_t seed_lo, seed_hi;
+    orc_reward_config reward;
+    int32_t write_back_reset;
+} orc_env_config;
+
+/* Body state of one env, fp64 working copy. */
+typedef struct {
+    double p[ORC_MAX_BODIES][3], q[ORC_MAX_BODIES][4], v[ORC_MAX_BODIES][3], w[ORC_MAX_BODIES][3];
+} orc_body_state;
+
+/* Step a3: the seven error terms between a simulated state and the reference
+ * (Section 6.1 names pose, velocity, COM, end-effector position/orientation;
+ * Figure 5 adds whole-body position and velocity sums). */
+static void error_terms(const orc_skeleton *s, const orc_body_state *x, const orc_ref *r, double e[ORC_N_TERMS])
+{
+    int J = s->J;
+    for (int k = 0; k < ORC_N_TERMS; ++k) e[k] = 0.0;
+    for (int j = 0; j < J; ++j) {
+        int a = s->parent[j];
+        double ql_sim[4], wl_sim[3], dw[3];
+        if (a < 0) {
+            memcpy(ql_sim, x->q[j], sizeof(ql_sim));
+            dw[0] = x->w[j][0]; dw[1] = x->w[j][1]; dw[2] = x->w[j][2];
+        } else {
+            double qc[4];
+            quat_conj(x->q[a], qc);
+            orc_quat_mul(qc, x->q[j], ql_sim);
+            for (int c = 0; c < 3; ++c) dw[c] = x->w[j][c] - x->w[a][c];
+        }
+        quat_rotate_inv(x->q[j], dw, wl_sim);
+        double th = rel_angle(r->ql[j], ql_sim);
+        e[0] += th * th;
+        for (int c = 0; c < 3; ++c) {
+            double d = wl_sim[c] - r->wl[j][c];
+            e[1] += d * d;
+            double dp = x->p[j][c] - r->p[j][c];
+            e[5] += dp * dp;
+            double dv = x->v[j][c] - r->v[j][c];
+            e[6] += dv * dv;
+        }
+    }
+    for (int i = 0; i < s->n_ee; ++i) {
+        int b = s->ee[i];
+        for (int c = 0; c < 3; ++c) {
+            double d = x->p[b][c] - r->p[b][c];
+            e[2] += d * d;
+        }
+        double th = rel_angle(r->q[b], x->q[b]);
+        e[3] += th * th;
+    }
+    double com_sim[3];
+    center_of_mass(s, (double (*)[3])x->p, com_sim);
+    for (int c = 0; c < 3; ++c) {
+        double d = com_sim[c] - r->com[c];
+        e[4] += d * d;
+    }
+}
+
+/* Reward from the error terms: prod_k exp(-w_k e_k) = exp(-sum_k w_k e_k)
+ * (Section 6.1) or sum_k a_k exp(-w_k e_k) (Figure 5). */
+double orc_reward(const orc_reward_config *rc, const double e[ORC_N_TERMS])
+{
+    if (rc->mode == 0) {
+        double s = 0.0;
+        for (int k = 0; k < ORC_N_TERMS; ++k) s += (double)rc->w[k] * e[k];
+        return exp(-s);
+    }
+    double r = 0.0;
+    for (int k = 0; k < ORC_N_TERMS; ++k) r += (double)rc->a[k] * exp(-(double)rc->w[k] * e[k]);
+    return r;
+}
+
+/* Step a5: uniform reset draw for env id `env` at step `step`. */
+void orc_reset_draw(const orc_clips *cl, const orc_env_config *cfg, uint32_t env, uint32_t step,
+                    int32_t *clip_out, float *t_out)
+{
+    uint32_t ctr[4] = {env, step, ORC_STREAM_RESET, 0u}, key[2] = {cfg->seed_lo, cfg->seed_hi}, x[4];
+    orc_philox4x32_10(ctr, key, x);
+    int32_t clip = (int32_t)(((uint64_t)x[0] * (uint64_t)(uint32_t)cl->C) >> 32);
+    float u = (float)(x[1] >> 8) * 5.9604644775390625e-08f;       /* 2^-24, exact */
+    volatile float span = cl->dur[clip] - cfg->dt;                  /* one fp32 subtract */
+    if (span < 0.0f) span = 0.0f;
+    volatile float t = u * span;                                    /* one fp32 multiply */
+    *clip_out = clip; *t_out = t;
+}
+
+static void ref_to_state(const orc_skeleton *s, const orc_ref *r, orc_body_state *x)
+{
+    memcpy(x->p, r->p, sizeof(double) * 3 * s->J);
+    memcpy(x->q, r->q, sizeof(double) * 4 * s->J);
+    memcpy(x->v, r->v, sizeof(double) * 3 * s->J);
+    memcpy(x->w, r->w, sizeof(double) * 3 * s->J);
+}
+
+/* Step a6: heading-local observation of state x at (clip, t), D = 24J + 1. */
+static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg,
+                      const orc_body_state *x, int clip, float t, double *obs)
+{
+    int J = s->J;
+    const double ex[3] = {1.0, 0.0, 0.0}, ez[3] = {0.0, 0.0, 1.0};
+    double hx[3];
+    orc_quat_rotate(x->q[0], ex, hx);
+    double psi = 0.0;
+    if (sqrt(hx[0]*hx[0] + hx[1]*hx[1]) >= 1e-6) psi = atan2(hx[1], hx[0]);
+    double qh_inv[4] = {cos(0.5 * psi), 0.0, 0.0, -sin(0.5 * psi)};   /* rotation by -psi about z */
+    double origin[3] = {x->p[0][0], x->p[0][1], 0.0};
+
+    for (int j = 0; j < J; ++j) {
+        double *o = obs + 15 * j, d[3], ql[4];
+        for (int c = 0; c < 3; ++c) d[c] = x->p[j][c] - origin[c];
+        orc_quat_rotate(qh_inv, d, o + 0);
+        orc_quat_mul(qh_inv, x->q[j], ql);
+        orc_quat_rotate(ql, ex, o + 3);
+        orc_quat_rotate(ql, ez, o + 6);
+        orc_quat_rotate(qh_inv, x->v[j], o + 9);
+        orc_quat_rotate(qh_inv, x->w[j], o + 12);
+    }
+    obs[15 * J] = (double)t / (double)cl->dur[clip];
+
+    volatile float t_next = t + cfg->dt;                 /* one fp32 add */
+    float t_tgt = t_next < cl->dur[clip] ? t_next : cl->dur[clip];
+    orc_ref tgt;
+    orc_reference_state(s, cl, clip, t_tgt, &tgt);
+    for (int j = 0; j < J; ++j) {
+        double *o = obs + 15 * J + 1 + 9 * j, d[3], ql[4];
+        for (int c = 0; c < 3; ++c) d[c] = tgt.p[j][c] - origin[c];
+        orc_quat_rotate(qh_inv, d, o + 0);
+        orc_quat_mul(qh_inv, tgt.q[j], ql);
+        orc_quat_rotate(ql, ex, o + 3);
+        orc_quat_rotate(ql, ez, o + 6);
+    }
+}
+
+static void load_sim(const orc_skeleton *s, const float *pos, const float *quat, const float *lin,
+                     const float *ang, int64_t stride, int64_t i, orc_body_state *x)
+{
+    for (int j = 0; j < s->J; ++j) {
+        for (int c = 0; c < 3; ++c) {
+            x->p[j][c] = (double)pos[(3*j+c) * stride + i];
+            x->v[j][c] = (double)lin[(3*j+c) * stride + i];
+            x->w[j][c] = (double)ang[(3*j+c) * stride + i];
+        }
+        for (int c = 0; c < 4; ++c) x->q[j][c] = (double)quat[(4*j+c) * stride + i];
+    }
+}
+
+static void store_sim(const orc_skeleton *s, const orc_body_state *x, float *pos, float *quat,
+                      float *lin, float *ang, int64_t stride, int64_t i)
+{
+    for (int j = 0; j < s->J; ++j) {
+        for (int c = 0; c < 3; ++c) {
+            pos[(3*j+c) * stride + i] = (float)x->p[j][c];
+            lin[(3*j+c) * stride + i] = (float)x->v[j][c];
+            ang[(3*j+c) * stride + i] = (float)x->w[j][c];
+        }
+        for (int c = 0; c < 4; ++c) quat[(4*j+c) * stride + i] = (float)x->q[j][c];
+    }
+}
+
+/* Step 0: every env is reset (counter step 0) and its first observation is
+ * built from the reference state; no reward. */
+void orc_env_reset_all(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg,
+                       int n, const uint32_t *env_ids, uint32_t step,
+                       int32_t *clip_id, float *t, int32_t *ep_len,
+                       double *obs, int64_t ld_obs, int n_threads)
+{
+    if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for num_threads(n_threads) schedule(static)
+    for (int i = 0; i < n; ++i) {
+        orc_ref r;
+        orc_body_state x;
+        orc_reset_draw(cl, cfg, env_ids[i], step, &clip_id[i], &t[i]);
+        ep_len[i] = 0;
+        orc_reference_state(s, cl, clip_id[i], t[i], &r);
+        ref_to_state(s, &r, &x);
+        build_obs(s, cl, cfg, &x, clip_id[i], t[i], obs + (int64_t)i * ld_obs);
+    }
+}
+
+/* One control step for n envs (Figure 2's post-physics phase, in its order:
+ * reward and dones, masked reset, observation).  State arrays are updated in
+ * place.  sim arrays are structure-of-arrays: component c of env i at
+ * c*comp_stride + i.  terms may be NULL. */
+void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg,
+                  int n, const uint32_t *env_ids, uint32_t step,
+                  int32_t *clip_id, float *t, int32_t *ep_len,
+                  float *pos, float *quat, float *linvel, float *angvel, int64_t comp_stride,
+                  double *obs, int64_t ld_obs, double *reward, uint8_t *flags, double *terms,
+                  int n_threads)
+{
+    if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for num_threads(n_threads) schedule(static)
+    for (int i = 0; i < n; ++i) {
+        orc_ref r;
+        orc_body_state x;
+        double e[ORC_N_TERMS];
+        int clip = clip_id[i];
+
+        volatile float t1 = t[i] + cfg->dt;                         /* a0 */
+        orc_reference_state(s, cl, clip, t1, &r);                    /* a1, a2 */
+        load_sim(s, pos, quat, linvel, angvel, comp_stride, i, &x);
+        error_terms(s, &x, &r, e);                                   /* a3 */
+        double rew = orc_reward(&cfg->reward, e);
+        reward[i] = rew;
+        if (terms) for (int k = 0; k < ORC_N_TERMS; ++k) terms[(int64_t)k * n + i] = e[k];
+
+        /* a4: flags.  Root height is compared as the fp32 input value. */
+        float root_z = pos[2 * comp_stride + i];
+        int terminated = (root_z < cfg->reward.h_min) || (rew < (double)cfg->reward.r_min);
+        volatile float t2 = t1 + cfg->dt;
+        int truncated = t2 > cl->dur[clip];
+        flags[i] = (uint8_t)(terminated | (truncated << 1));
+
+        float t_cur = t1;
+        if (flags[i]) {                                              /* a5 */
+            orc_reset_draw(cl, cfg, env_ids[i], step, &clip, &t_cur);
+            ep_len[i] = 0;
+            orc_reference_state(s, cl, clip, t_cur, &r);
+            ref_to_state(s, &r, &x);
+            if (cfg->write_back_reset) store_sim(s, &x, pos, quat, linvel, angvel, comp_stride, i);
+        } else {
+            ep_len[i] += 1;
+        }
+        clip_id[i] = clip;
+        t[i] = t_cur;
+        build_obs(s, cl, cfg, &x, clip, t_cur, obs + (int64_t)i * ld_obs);   /* a6 */
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Step e: policy MLP forward and Gaussian action sampling.                  */
+/* ------------------------------------------------------------------------ */
+
+/* Standard normals for env `env` at step `step`: Philox block i gives four
+ * words; (x0,x1) and (x2,x3) each feed one Box-Muller pair. */
+void orc_action_noise(uint32_t seed_lo, uint32_t seed_hi, uint32_t env, uint32_t step, int A, double *z)
+{
+    uint32_t key[2] = {seed_lo, seed_hi};
+    for (int blk = 0; 4 * blk < A; ++blk) {
+        uint32_t ctr[4] = {env, step, ORC_STREAM_ACTION, (uint32_t)blk}, x[4];
+        orc_philox4x32_10(ctr, key, x);
+        for (int h = 0; h < 2; ++h) {
+            double u1 = ((double)(x[2*h] >> 8) + 1.0) * 5.9604644775390625e-08;
+            double u2 = (double)(x[2*h+1] >> 8) * 5.9604644775390625e-08;
+            double rad = sqrt(-2.0 * log(u1));
+            double zc = rad * cos(2.0 * M_PI * u2), zs = rad * sin(2.0 * M_PI * u2);
+            if (4*blk + 2*h < A) z[4*blk + 2*h] = zc;
+            if (4*blk + 2*h + 1 < A) z[4*blk + 2*h + 1] = zs;
+        }
+    }
+}
+
+/* h_{l+1} = relu(W_l h_l + b_l), last layer linear -> mean; a = mean + sigma z.
+ * Weights W_l are [dims[l+1]][dims[l]] fp32 values (bf16 weights widened
+ * exactly by the caller); accumulation in fp64, activations never rounded. */
+void orc_policy_forward(int n_layers, const int32_t *dims, const float *const *W, const float *const *b,
+                        double sigma, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
+                        int n, const uint32_t *env_ids, const double *obs, int64_t ld_obs,
+                        double *mean, double *action, double *logp, double *z_out, int n_threads)
+{
+    int maxd = 0, A = dims[n_layers];
+    for (int l = 0; l <= n_layers; ++l) if (dims[l] > maxd) maxd = dims[l];
+    if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for num_threads(n_threads) schedule(static)
+    for (int i = 0; i < n; ++i) {
+        double *h0 = (double *)malloc(sizeof(double) * maxd), *h1 = (double *)malloc(sizeof(double) * maxd);
+        double *z = (double *)malloc(sizeof(double) * (A + 4));
+        for (int k = 0; k < dims[0]; ++k) h0[k] = obs[(int64_t)i * ld_obs + k];
+        for (int l = 0; l < n_layers; ++l) {
+            int in = dims[l], out = dims[l+1];
+            for (int o = 0; o < out; ++o) {
+                double acc = (double)b[l][o];
+                const float *w = W[l] + (int64_t)o * in;
+                for (int k = 0; k < in; ++k) acc += (double)w[k] * h0[k];
+                if (l < n_layers - 1 && acc < 0.0) acc = 0.0;
+                h1[o] = acc;
+            }
+            double *tmp = h0; h0 = h1; h1 = tmp;
+        }
+        orc_action_noise(seed_lo, seed_hi, env_ids[i], step, A, z);
+        double zz = 0.0;
+        for (int o = 0; o < A; ++o) {
+            mean[(int64_t)i * A + o] = h0[o];
+            action[(int64_t)i * A + o] = h0[o] + sigma * z[o];
+            if (z_out) z_out[(int64_t)i * A + o] = z[o];
+            zz += z[o] * z[o];
+        }
+        if (logp) logp[i] = -0.5 * zz - (double)A * log(sigma) - 0.5 * (double)A * log(2.0 * M_PI);
+        free(h0); free(h1); free(z);
+    }
+}
+
+/* Error terms and reward of one explicit (state, reference) pair; lets the
+ * tests feed hand-made states. */
+void orc_error_terms_flat(const orc_skeleton *s, const orc_clips *cl, int clip, float t,
+                          const double *p, const double *q, const double *v, const double *w, double *e)
+{
+    orc_ref r;
+    orc_body_state x;
+    orc_reference_state(s, cl, clip, t, &r);
+    for (int j = 0; j < s->J; ++j) {
+        for (int c = 0; c < 3; ++c) { x.p[j][c] = p[3*j+c]; x.v[j][c] = v[3*j+c]; x.w[j][c] = w[3*j+c]; }
+        for (int c = 0; c < 4; ++c) x.q[j][c] = q[4*j+c];
+    }
+    error_terms(s, &x, &r, e);
+}
+
+int orc_openmp_enabled(void)
+{
+#ifdef _OPENMP
+    return 1;
+#else
+    return 0;
+#endif
+}

@@ -1,0 +1,282 @@
+"""ctypes front end of the CPU oracle (oracle/im_oracle.c).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import
+this module.  It compiles the C file with gcc on first use and shares nothing
+with the CUDA library or its Python binding.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "im_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_LIB = os.path.join(_OUT_DIR, "libim_oracle.so")
+N_TERMS = 7
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle: gcc -O2, OpenMP over envs, no FMA contraction."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC",
+                               "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class RewardConfig(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("a", C.c_float * N_TERMS), ("w", C.c_float * N_TERMS),
+                ("h_min", C.c_float), ("r_min", C.c_float)]
+
+
+class EnvConfig(C.Structure):
+    _fields_ = [("dt", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32),
+                ("reward", RewardConfig), ("write_back_reset", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        vp, i32, u32, i64, f32, f64 = C.c_void_p, C.c_int32, C.c_uint32, C.c_int64, C.c_float, C.c_double
+        L.orc_philox4x32_10.argtypes = [vp, vp, vp]
+        L.orc_quat_mul.argtypes = [vp, vp, vp]
+        L.orc_quat_rotate.argtypes = [vp, vp, vp]
+        L.orc_quat_log.argtypes = [vp, vp]
+        L.orc_geodesic_angle.argtypes = [vp]
+        L.orc_geodesic_angle.restype = f64
+        L.orc_slerp.argtypes = [vp, vp, f64, vp]
+        L.orc_skeleton_create.argtypes = [i32, vp, vp, vp, vp, i32]
+        L.orc_skeleton_create.restype = vp
+        L.orc_skeleton_destroy.argtypes = [vp]
+        L.orc_clips_create.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.orc_clips_create.restype = vp
+        L.orc_clips_destroy.argtypes = [vp]
+        L.orc_clip_duration.argtypes = [vp, i32]
+        L.orc_clip_duration.restype = f32
+        L.orc_lookup_index.argtypes = [f32, f32, i32, vp, vp]
+        L.orc_reference_state_flat.argtypes = [vp, vp, i32, f32] + [vp] * 7
+        L.orc_reward.argtypes = [vp, vp]
+        L.orc_reward.restype = f64
+        L.orc_reset_draw.argtypes = [vp, vp, u32, u32, vp, vp]
+        L.orc_env_reset_all.argtypes = [vp, vp, vp, i32, vp, u32, vp, vp, vp, vp, i64, i32]
+        L.orc_env_step.argtypes = [vp, vp, vp, i32, vp, u32, vp, vp, vp, vp, vp, vp, vp, i64,
+                                   vp, i64, vp, vp, vp, i32]
+        L.orc_action_noise.argtypes = [u32, u32, u32, u32, i32, vp]
+        L.orc_policy_forward.argtypes = [i32, vp, vp, vp, f64, u32, u32, u32, i32, vp, vp, i64,
+                                         vp, vp, vp, vp, i32]
+        L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
+        L.orc_openmp_enabled.restype = i32
+        _lib = L
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f64(x) -> np.ndarray:
+    return np.ascontiguousarray(x, np.float64)
+
+
+# ---------------------------------------------------------------- small pieces
+def philox(ctr: Sequence[int], key: Sequence[int]) -> np.ndarray:
+    c = np.asarray(ctr, np.uint32)
+    k = np.asarray(key, np.uint32)
+    out = np.empty(4, np.uint32)
+    lib().orc_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def quat_mul(a, b) -> np.ndarray:
+    a, b, out = _f64(a), _f64(b), np.empty(4)
+    lib().orc_quat_mul(_p(a), _p(b), _p(out))
+    return out
+
+
+def quat_rotate(q, v) -> np.ndarray:
+    q, v, out = _f64(q), _f64(v), np.empty(3)
+    lib().orc_quat_rotate(_p(q), _p(v), _p(out))
+    return out
+
+
+def quat_log(q) -> np.ndarray:
+    q, out = _f64(q), np.empty(3)
+    lib().orc_quat_log(_p(q), _p(out))
+    return out
+
+
+def geodesic_angle(q) -> float:
+    q = _f64(q)
+    return float(lib().orc_geodesic_angle(_p(q)))
+
+
+def slerp(q0, q1, alpha: float) -> np.ndarray:
+    q0, q1, out = _f64(q0), _f64(q1), np.empty(4)
+    lib().orc_slerp(_p(q0), _p(q1), float(alpha), _p(out))
+    return out
+
+
+def lookup_index(t: float, fps: float, K: int):
+    k = np.zeros(1, np.int32)
+    a = np.zeros(1, np.float64)
+    lib().orc_lookup_index(np.float32(t), np.float32(fps), int(K), _p(k), _p(a))
+    return int(k[0]), float(a[0])
+
+
+def action_noise(seed: int, env: int, step: int, A: int) -> np.ndarray:
+    z = np.zeros(A + 4)
+    lib().orc_action_noise(seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF, env, step, A, _p(z))
+    return z[:A]
+
+
+def make_env_config(dt: float, seed: int, reward: dict, h_min: float, r_min: float = -np.inf,
+                    write_back_reset: bool = False) -> EnvConfig:
+    rc = RewardConfig(mode=int(reward["mode"]), h_min=np.float32(h_min), r_min=np.float32(r_min))
+    for k in range(N_TERMS):
+        rc.a[k] = reward["a"][k]
+        rc.w[k] = reward["w"][k]
+    return EnvConfig(dt=np.float32(dt), seed_lo=seed & 0xFFFFFFFF, seed_hi=(seed >> 32) & 0xFFFFFFFF,
+                     reward=rc, write_back_reset=int(write_back_reset))
+
+
+def reward_from_terms(reward: dict, e) -> float:
+    cfg = make_env_config(1.0 / 30, 0, reward, 0.0)
+    e = _f64(e)
+    return float(lib().orc_reward(C.byref(cfg.reward), _p(e)))
+
+
+# ---------------------------------------------------------------- handles
+class Skeleton:
+    def __init__(self, parents, offsets, masses=None, ee_ids=None):
+        self.parents = np.ascontiguousarray(parents, np.int32)
+        self.J = int(self.parents.shape[0])
+        off = np.ascontiguousarray(offsets, np.float32)
+        m = None if masses is None else np.ascontiguousarray(masses, np.float32)
+        ee = None if ee_ids is None else np.ascontiguousarray(ee_ids, np.int32)
+        self.h = lib().orc_skeleton_create(self.J, _p(self.parents), _p(off), _p(m), _p(ee),
+                                           0 if ee is None else int(ee.shape[0]))
+        if not self.h:
+            raise ValueError("invalid skeleton")
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib().orc_skeleton_destroy(self.h)
+            self.h = None
+
+
+class Clips:
+    def __init__(self, skel: Skeleton, n_frames, fps, root_pos, local_quat):
+        self.skel = skel
+        self.n_frames = np.ascontiguousarray(n_frames, np.int32)
+        self.fps = np.ascontiguousarray(fps, np.float32)
+        self.C = int(self.n_frames.shape[0])
+        rp = np.ascontiguousarray(root_pos, np.float32)
+        lq = np.ascontiguousarray(local_quat, np.float32)
+        assert rp.shape == (int(self.n_frames.sum()), 3)
+        assert lq.shape == (int(self.n_frames.sum()), skel.J, 4)
+        self.h = lib().orc_clips_create(skel.h, self.C, _p(self.n_frames), _p(self.fps), _p(rp), _p(lq))
+
+    def duration(self, clip: int) -> np.float32:
+        return np.float32(lib().orc_clip_duration(self.h, int(clip)))
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib().orc_clips_destroy(self.h)
+            self.h = None
+
+
+def reference_state(skel: Skeleton, clips: Clips, clip: int, t: float) -> dict:
+    J = skel.J
+    out = dict(p=np.empty((J, 3)), q=np.empty((J, 4)), v=np.empty((J, 3)), w=np.empty((J, 3)),
+               ql=np.empty((J, 4)), wl=np.empty((J, 3)), com=np.empty(3))
+    lib().orc_reference_state_flat(skel.h, clips.h, int(clip), np.float32(t), _p(out["p"]), _p(out["q"]),
+                                   _p(out["v"]), _p(out["w"]), _p(out["ql"]), _p(out["wl"]), _p(out["com"]))
+    return out
+
+
+def error_terms(skel: Skeleton, clips: Clips, clip: int, t: float, p, q, v, w) -> np.ndarray:
+    e = np.empty(N_TERMS)
+    p, q, v, w = _f64(p), _f64(q), _f64(v), _f64(w)
+    lib().orc_error_terms_flat(skel.h, clips.h, int(clip), np.float32(t), _p(p), _p(q), _p(v), _p(w), _p(e))
+    return e
+
+
+def reset_draw(clips: Clips, cfg: EnvConfig, env: int, step: int):
+    c = np.zeros(1, np.int32)
+    t = np.zeros(1, np.float32)
+    lib().orc_reset_draw(clips.h, C.byref(cfg), env, step, _p(c), _p(t))
+    return int(c[0]), np.float32(t[0])
+
+
+class Env:
+    """Per-env state (clip id, time, episode length) plus the step functions."""
+
+    def __init__(self, skel: Skeleton, clips: Clips, cfg: EnvConfig, n_envs: int,
+                 env_ids: Optional[np.ndarray] = None, n_threads: Optional[int] = None):
+        self.skel, self.clips, self.cfg, self.n = skel, clips, cfg, int(n_envs)
+        self.env_ids = (np.arange(n_envs, dtype=np.uint32) if env_ids is None
+                        else np.ascontiguousarray(env_ids, np.uint32))
+        self.clip_id = np.zeros(self.n, np.int32)
+        self.t = np.zeros(self.n, np.float32)
+        self.ep_len = np.zeros(self.n, np.int32)
+        self.D = 24 * skel.J + 1
+        self.n_threads = int(n_threads or os.cpu_count() or 1)
+
+    def reset_all(self, step: int = 0) -> np.ndarray:
+        obs = np.zeros((self.n, self.D))
+        lib().orc_env_reset_all(self.skel.h, self.clips.h, C.byref(self.cfg), self.n, _p(self.env_ids), step,
+                                _p(self.clip_id), _p(self.t), _p(self.ep_len), _p(obs), self.D,
+                                self.n_threads)
+        return obs
+
+    def step(self, step: int, sim: np.ndarray, want_terms: bool = True) -> dict:
+        """sim: fp32 [13J, n] (positions, quaternions, linear, angular velocities)."""
+        J = self.skel.J
+        assert sim.dtype == np.float32 and sim.shape == (13 * J, self.n) and sim.flags.c_contiguous
+        pos, quat, lin, ang = sim[0:3 * J], sim[3 * J:7 * J], sim[7 * J:10 * J], sim[10 * J:13 * J]
+        obs = np.zeros((self.n, self.D))
+        reward = np.zeros(self.n)
+        flags = np.zeros(self.n, np.uint8)
+        terms = np.zeros((N_TERMS, self.n)) if want_terms else None
+        lib().orc_env_step(self.skel.h, self.clips.h, C.byref(self.cfg), self.n, _p(self.env_ids), step,
+                           _p(self.clip_id), _p(self.t), _p(self.ep_len),
+                           _p(pos), _p(quat), _p(lin), _p(ang), self.n,
+                           _p(obs), self.D, _p(reward), _p(flags), _p(terms), self.n_threads)
+        return dict(obs=obs, reward=reward, flags=flags, terms=terms)
+
+
+def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarray,
+                   env_ids: Optional[np.ndarray] = None, n_threads: Optional[int] = None) -> dict:
+    """obs: fp64 [n, >=dims[0]].  W[l]: fp32 [dims[l+1], dims[l]] (bf16 weights widened exactly)."""
+    nl = len(dims) - 1
+    n = obs.shape[0]
+    obs = _f64(obs)
+    A = int(dims[-1])
+    ids = np.arange(n, dtype=np.uint32) if env_ids is None else np.ascontiguousarray(env_ids, np.uint32)
+    Wc = [np.ascontiguousarray(w, np.float32) for w in W]
+    bc = [np.ascontiguousarray(x, np.float32) for x in b]
+    for l in range(nl):
+        assert Wc[l].shape == (dims[l + 1], dims[l]) and bc[l].shape == (dims[l + 1],)
+    Wp = (C.c_void_p * nl)(*[w.ctypes.data for w in Wc])
+    bp = (C.c_void_p * nl)(*[x.ctypes.data for x in bc])
+    d = np.asarray(dims, np.int32)
+    mean = np.zeros((n, A))
+    action = np.zeros((n, A))
+    logp = np.zeros(n)
+    z = np.zeros((n, A))
+    lib().orc_policy_forward(nl, _p(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), float(sigma),
+                             seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF, step, n, _p(ids),
+                             _p(obs), obs.shape[1], _p(mean), _p(action), _p(logp), _p(z),
+                             int(n_threads or os.cpu_count() or 1))
+    return dict(mean=mean, action=action, logp=logp, z=z)
