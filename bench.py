@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the imitation-step hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole path over all envs of the workload: policy
+forward + Gaussian sampling on the current observations, then the fused env
+step (reference lookup/FK, reward, flags, masked reset, next observation) on
+that step's simulated body states.  Prints one JSON line (rank 0).
+
+`--impl reference` times the CPU oracle on a bounded sample of the same
+workload on the host cores (a deliberately plain program: a baseline, not a
+target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_09821_b200 import workloads as W  # noqa: E402
+
+DEFAULT_WORKLOAD = "cfg4_65536_smpl24"
+METRIC = "env-steps/s (obs+reward+reset+policy fwd)"
+UNIT = "env-steps/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def env_bytes_per_env(J: int) -> int:
+    """Algorithmic HBM bytes of the env kernel per env-step: body states in, observation row,
+    reward, flags out, per-env state read + written."""
+    return 13 * J * 4 + (24 * J + 1) * 4 + 4 + 1 + 24
+
+
+def mlp_flops_per_env(dims) -> int:
+    return sum(2 * a * b for a, b in zip(dims[:-1], dims[1:]))
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2])); power.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w_max=float(max(power)),
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def oracle_leg(wl: W.Workload, skel, lib, pol, n_sample: int, steps: int, warmup: int, budget_s: float):
+    """Times the oracle as it stands on `n_sample` envs of the workload; returns env-steps/s."""
+    from oracle import oracle as O
+    n = min(n_sample, wl.n_envs)
+    osk = O.Skeleton(skel["parents"], skel["offsets"], skel["masses"])
+    ocl = O.Clips(osk, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    cfg = O.make_env_config(wl.dt, wl.seed, W.REWARD_MULT, wl.h_min)
+    cores = os.cpu_count() or 1
+    env = O.Env(osk, ocl, cfg, n, n_threads=cores)
+    state = dict(obs=env.reset_all(0), t=0.0, done=0)
+    t_start = time.perf_counter()
+
+    def consume(s, sim):
+        sim = np.ascontiguousarray(sim.numpy())
+        if state["t"] > budget_s and state["done"] >= 1:
+            raise StopIteration
+        t0 = time.perf_counter()
+        O.policy_forward(pol["dims"], pol["W"], pol["b"], wl.sigma_action, wl.seed, s, state["obs"],
+                         n_threads=cores)
+        out = env.step(s, sim, want_terms=False)
+        dt = time.perf_counter() - t0
+        state["obs"] = out["obs"]
+        if s > warmup:
+            state["t"] += dt
+            state["done"] += 1
+
+    try:
+        W.rollout_inputs(wl, skel, lib, lambda: (env.clip_id, env.t), consume, steps=warmup + steps)
+    except StopIteration:
+        pass
+    done = max(state["done"], 1)
+    return dict(value=n * done / max(state["t"], 1e-9), cores=cores, steps=done, n=n,
+                ms_per_step=1e3 * state["t"] / done, wall_s=time.perf_counter() - t_start)
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
+    ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of one CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = W.WORKLOADS[args.workload]
+    K = args.steps if args.steps is not None else wl.steps
+    Wm = max(args.warmup, 0)
+    skel, lib, pol = W.build_scene(wl)
+    J, D = skel["J"], wl.obs_dim
+    config = dict(workload=wl.name, n_envs_per_gpu=wl.n_envs, bodies=J, obs_dim=D, mlp=list(wl.mlp_dims),
+                  mlp_dtype=wl.mlp_dtype, clips=wl.n_clips, reward="multiplicative")
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        res = oracle_leg(wl, skel, lib, pol, n_sample=2048, steps=K, warmup=Wm, budget_s=60.0)
+        sample = "first %d envs of %s, %d steps" % (res["n"], wl.name, res["steps"])
+        line = dict(metric=METRIC, value=res["value"], unit=UNIT, n_gpus=0, steps=res["steps"], warmup=Wm,
+                    ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="f64", data="synthetic", impl="reference", config=config,
+                    cpu_baseline=dict(value=res["value"], unit=UNIT, cores=res["cores"], kind="oracle", sample=sample),
+                    e2e=dict(value=res["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+        print(json.dumps(line))
+        return
+
+    import torch
+    from paper_2609_09821_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.load()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    n = wl.n_envs                              # weak scaling: every rank runs the whole workload's env count
+    env_base = rank * n
+    ld = B.padded_ld(D)
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+
+    g_skel = B.Skeleton(skel["parents"], skel["offsets"], skel["masses"])
+    g_clips = B.Clips(g_skel, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    cfg = B.make_env_config(n, wl.dt, wl.seed, W.REWARD_MULT, wl.h_min, ld, env_id_base=env_base)
+    env = B.Env(g_skel, g_clips, cfg, stream=stream)
+    Wg = pol["W_bf16"] if pol["dtype"] == "bf16" else pol["W"]
+    policy = B.Policy(pol["dims"], Wg, pol["b"], pol["dtype"], wl.sigma_action, wl.seed, n, env_id_base=env_base,
+                      stream=stream)
+    A = wl.act_dim
+    obs = env.new_obs()
+    reward = torch.empty(n, device=dev)
+    flags = torch.empty(n, dtype=torch.uint8, device=dev)
+    mean = torch.empty((n, A), device=dev)
+    action = torch.empty((n, A), device=dev)
+
+    # ---- inputs: one pre-pass of the rollout fixes every env's (clip, time) per step; the simulator
+    # ---- stand-in writes each step's body states straight into HBM
+    total = Wm + K
+    n_buf = min(total, 96)                     # bound device memory; longer runs cycle through the buffers
+    env.reset_all(obs, 0)
+
+    def get_state():
+        c, t, _ = env.get_state()
+        return c, t
+
+    def consume(s, sim):
+        policy.forward(s, obs, mean, action)
+        env.step(s, sim, obs, reward, flags)
+
+    sims = W.rollout_inputs(wl, skel, lib, get_state, consume, steps=n_buf, env_base=env_base, device=str(dev))
+    torch.cuda.synchronize()
+    if env.device_status() or policy.device_status():
+        raise SystemExit("device status word set during the input pre-pass")
+
+    def run_steps(first, count):
+        for i in range(count):
+            s = first + i
+            policy.forward(s, obs, mean, action)
+            env.step(s, sims[(s - 1) % n_buf], obs, reward, flags)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    env.reset_all(obs, 0)
+    run_steps(1, Wm)
+    torch.cuda.synchronize()
+    graph = None
+    launches_per_replay = None
+    if not args.no_graph:
+        c0, t0, l0 = env.get_state()
+        obs0 = obs.clone()
+        before = B.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            run_steps(Wm + 1, K)
+        launches_per_replay = B.launch_count() - before
+        env.set_state(c0, t0, l0)
+        obs.copy_(obs0)
+        torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    before = B.launch_count()
+    ev0.record(stream)
+    if graph is not None:
+        graph.replay()
+    else:
+        run_steps(Wm + 1, K)
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = launches_per_replay if graph is not None else B.launch_count() - before
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+
+    # ---- per-call breakdown (stream launches with events around each call) for the rooflines
+    env.reset_all(obs, 0)
+    run_steps(1, Wm)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    torch.cuda.synchronize()
+    for i in range(K):
+        s = Wm + 1 + i
+        evs[i][0].record(stream)
+        policy.forward(s, obs, mean, action)
+        evs[i][1].record(stream)
+        env.step(s, sims[(s - 1) % n_buf], obs, reward, flags)
+        evs[i][2].record(stream)
+    torch.cuda.synchronize()
+    t_pol = float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e-3
+    t_env = float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e-3
+
+    # ---- end to end through the host-buffer entry point: pinned host inputs, results read back
+    e2e = None
+    if not args.no_e2e:
+        host_sims = [s.cpu().pin_memory() for s in sims]
+        act_h = torch.empty((n, A)).pin_memory()
+        rew_h = torch.empty(n).pin_memory()
+        fl_h = torch.empty(n, dtype=torch.uint8).pin_memory()
+        env.reset_all_host(0)
+        for s in range(1, Wm + 1):
+            B.step_host(env, policy, s, host_sims[(s - 1) % n_buf], act_h, rew_h, fl_h)
+        barrier()
+        t0 = time.perf_counter()
+        for s in range(Wm + 1, Wm + K + 1):
+            B.step_host(env, policy, s, host_sims[(s - 1) % n_buf], act_h, rew_h, fl_h)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            tmax = torch.tensor([e2e_s], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            e2e_s = float(tmax.item())
+        e2e = dict(value=world * n * K / e2e_s, unit=UNIT, h2d_bytes_per_step=13 * J * n * 4,
+                   d2h_bytes_per_step=n * (A * 4 + 4 + 1), ms_per_step=1e3 * e2e_s / K,
+                   timer="host clock around K calls that each wait for the stream")
+        del host_sims
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops = mlp_flops_per_env(wl.mlp_dims) * n
+    env_bytes = env_bytes_per_env(J) * n
+    tf = flops / t_pol / 1e12
+    gbs = env_bytes / t_env / 1e9
+    tensor_peak = peaks["bf16_tflops_sustained"]
+    roofline = dict(bound="tensor", kernel="policy forward (convert + GEMM chain + sampling)", achieved=tf,
+                    peak=tensor_peak, unit="TFLOP/s", frac=tf / tensor_peak, traffic=None,
+                    peak_source="%s bf16 sustained" % peaks["source"], seconds_per_launch=t_pol)
+    roofline_env = dict(bound="hbm", kernel="env_step_kernel", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=gbs / peaks["hbm_gbs"], traffic=None, peak_source="%s copy" % peaks["source"],
+                        seconds_per_launch=t_env, algorithmic_bytes=env_bytes)
+    if wl.mlp_dtype != "bf16":
+        roofline["bound"] = "alu"
+        roofline["peak_source"] = "fp32 SIMT path: tensor peak shown for scale only"
+    config.update(launch="cuda_graph" if graph is not None else "stream",
+                  l2="every step reads its own %.0f MB body-state buffer and rewrites the %.0f MB observation "
+                     "buffer (%d distinct step buffers)" % (13 * J * n * 4 / 1e6, n * ld * 4 / 1e6, n_buf),
+                  ld_obs=ld, parallelism="envs sharded across GPUs, no collective" if world > 1 else "single GPU")
+    line = dict(metric=METRIC, value=world * n * K / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=Wm,
+                ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16" if wl.mlp_dtype == "bf16" else "f32", data="synthetic", config=config,
+                clocks=clocks, gpu_launches=int(launches), roofline=roofline, roofline_env=roofline_env,
+                breakdown_ms=dict(policy_forward=t_pol * 1e3, env_step=t_env * 1e3))
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        res = oracle_leg(wl, skel, lib, pol, n_sample=2048, steps=64, warmup=1, budget_s=15.0)
+        line["cpu_baseline"] = dict(value=res["value"], unit=UNIT, cores=res["cores"], kind="oracle",
+                                    sample="first %d envs of %s, %d steps" % (res["n"], wl.name, res["steps"]))
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

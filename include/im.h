@@ -1,0 +1,242 @@
+/*
+ * im.h -- C ABI of the B200 imitation-step library.
+ *
+ * The library implements, for N environments at once, everything a
+ * DeepMimic-style training loop does per control step outside the physics
+ * solver (paper Figure 2: policy inference, then the post-physics phase --
+ * reward and dones, masked reset, observation building).  The simulated body
+ * states are an input; physics is not part of this library.
+ *
+ * Conventions: right handed, z up, metres / seconds / radians.  Quaternions
+ * are unit Hamilton quaternions stored w,x,y,z (paper Figure 3a), R(q)v = qvq*.
+ * Bodies are ordered so that parent[0] = -1 and parent[j] < j.
+ *
+ * Pointer kinds: every pointer is marked HOST or DEVICE.  Set-up calls take
+ * HOST pointers, copy what they need, and keep no reference.  Per-step calls
+ * take DEVICE pointers that the caller owns; the library only enqueues work on
+ * the CUDA stream given at creation and holds no reference once the call
+ * returns.  Per-step calls never synchronise, never read device data on the
+ * host, never branch on device data and never allocate (paper Section 4.2:
+ * no CPU access on the rollout step; reset is unconditional with a device-side
+ * mask), so a sequence of them can be captured in a CUDA graph (Section 2.2).
+ *
+ * Errors: a call that returns a negative status has had no effect.  Anomalies
+ * found on the device (a non-finite quaternion, a wait that ran out) set bits
+ * in a sticky status word, the kernel carries on with a defined fallback and
+ * never traps; read the word with im_poll_device_status.
+ */
+#ifndef IM_H_
+#define IM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)   /* the entry points below are the library's only exports */
+#endif
+
+typedef int32_t im_status;
+#define IM_OK                  0
+#define IM_ERR_INVALID_ARG    (-1)  /* null pointer, size out of range, misaligned buffer   */
+#define IM_ERR_BAD_TOPOLOGY   (-2)  /* parent[0] != -1, parent[j] >= j, J > IM_MAX_BODIES   */
+#define IM_ERR_BAD_QUAT       (-3)  /* keyframe quaternion non-finite or |q| off 1 by > 1e-3 */
+#define IM_ERR_ALLOC          (-4)  /* device or host allocation failed                      */
+#define IM_ERR_CUDA           (-5)  /* a CUDA runtime or driver call failed                  */
+#define IM_ERR_UNSUPPORTED    (-6)  /* layer sizes / device the kernels do not cover         */
+
+/* bits of the sticky device status word */
+#define IM_DEV_BAD_SIM_QUAT    1u   /* a simulated quaternion had zero or non-finite norm; identity used */
+#define IM_DEV_WAIT_TIMEOUT    2u   /* a bounded wait inside a kernel ran out; that tile's output is invalid */
+#define IM_DEV_BAD_STATE       4u   /* a per-env clip id was out of range; clamped */
+
+#define IM_MAX_BODIES   32
+#define IM_N_TERMS       7          /* pose, vel, ee_pos, ee_rot, com, body_pos, body_vel */
+#define IM_MAX_LAYERS    8
+
+#define IM_FLAG_TERMINATED 1u
+#define IM_FLAG_TRUNCATED  2u
+
+typedef struct im_skeleton im_skeleton;
+typedef struct im_clips    im_clips;
+typedef struct im_env      im_env;
+typedef struct im_policy   im_policy;
+
+const char *im_status_string(im_status s);
+
+/* ---- skeleton -------------------------------------------------------------
+ * The articulated character the reference motion is played on (forward
+ * kinematics of step (a): q[j] = q[parent] * q_local[j],
+ * p[j] = p[parent] + R(q[parent]) offset[j]).
+ *   J         number of bodies, 1..IM_MAX_BODIES
+ *   parents   HOST [J]      parent[0] = -1, parent[j] < j
+ *   offsets   HOST [J][3]   body origin in the parent's frame, metres (offsets[0] ignored)
+ *   masses    HOST [J] or NULL (all 1): weights of the centre of mass, which is the
+ *             mass-weighted mean of the body origins
+ *   ee_ids    HOST [n_ee] or NULL: end-effector bodies; NULL/0 selects every body without children
+ * Returns a host-side handle; free with im_destroy_skeleton. */
+im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *offsets,
+                             const float *masses, const int32_t *ee_ids, int32_t n_ee,
+                             im_skeleton **out);
+void im_destroy_skeleton(im_skeleton *s);
+
+/* ---- reference motion clips -----------------------------------------------
+ * A library of C keyframed clips (the paper's reference motions, Section 6.2).
+ * Frame k of clip c holds the root position and one local (parent-relative)
+ * quaternion per body.  Between keyframes the library interpolates: shortest
+ * arc slerp per joint, lerp for the root.
+ *   n_frames   HOST [C]            K_c >= 2
+ *   fps        HOST [C]            > 0; clip duration D_c = (K_c - 1) / fps_c (one fp32 division)
+ *   root_pos   HOST [sum K][3]
+ *   local_quat HOST [sum K][J][4]  w,x,y,z; must be finite with | |q| - 1 | <= 1e-3; used as given (the
+ *                                 interpolation and velocity formulas do not depend on the small scale error)
+ * The table is copied to the current CUDA device in rows padded to 16 bytes
+ * ([x y z 0 | q_0 | q_1 ...]); free with im_destroy_clips. */
+im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_frames, const float *fps,
+                        const float *root_pos, const float *local_quat, im_clips **out);
+void im_destroy_clips(im_clips *c);
+
+/* ---- environment ----------------------------------------------------------
+ * Reward (paper Section 6.1 and Figure 5) from seven error terms e_k between
+ * the simulated character and the reference at the env's time:
+ *   0 pose      sum over joints of the squared geodesic angle between reference and simulated
+ *               local rotations (rad^2), root included
+ *   1 vel       sum over joints of |difference of child-frame joint angular velocities|^2
+ *   2 ee_pos    sum over end-effectors of |world position difference|^2
+ *   3 ee_rot    sum over end-effectors of the squared geodesic angle of the world rotations
+ *   4 com       |centre-of-mass difference|^2
+ *   5 body_pos  sum over bodies of |world position difference|^2      (Figure 5 pose_err)
+ *   6 body_vel  sum over bodies of |world linear velocity difference|^2 (Figure 5 vel_err)
+ * mode 0: r = prod_k exp(-w_k e_k) (Section 6.1);  mode 1: r = sum_k a_k exp(-w_k e_k) (Figure 5). */
+typedef struct {
+    int32_t mode;
+    float a[IM_N_TERMS];
+    float w[IM_N_TERMS];
+    float h_min;      /* terminated if simulated root height (z) < h_min                        */
+    float r_min;      /* ... or reward < r_min; -INFINITY switches the reward test off          */
+} im_reward_config;
+
+typedef struct {
+    int32_t n_envs;           /* N >= 1                                                             */
+    uint32_t env_id_base;     /* env i draws random numbers as env id env_id_base + i, so a batch   */
+                              /* split across devices reproduces the unsplit run                    */
+    float dt;                 /* control interval, 0 < dt <= shortest clip duration                 */
+    uint64_t seed;            /* Philox key                                                         */
+    im_reward_config reward;
+    int32_t ld_obs;           /* row stride of obs buffers in floats: >= 24J+1 and a multiple of 4; */
+                              /* columns [24J+1, ld_obs) are written as zeros                       */
+    int32_t write_back_reset; /* non-zero: a reset env's reference state is also stored into the    */
+                              /* caller's body-state arrays (masked store)                          */
+} im_env_config;
+
+/* Simulated body states, DEVICE, structure of arrays: component c of env e at
+ * base[c * comp_stride + e]; per body 3 position rows (x,y,z), 4 quaternion
+ * rows (w,x,y,z), 3 linear and 3 angular velocity rows (world frame), so pos,
+ * linvel, angvel have 3J rows and quat 4J rows.  comp_stride >= N.  Each base
+ * pointer and comp_stride*4 must be multiples of 16 bytes. */
+typedef struct {
+    float *pos;
+    float *quat;
+    float *linvel;
+    float *angvel;
+    int64_t comp_stride;
+} im_body_state;
+
+/* Creates the per-env state (clip id, time, episode length) on the current
+ * device.  cuda_stream is a cudaStream_t (NULL = legacy default stream); every
+ * later call on this handle enqueues there.  skel and clips must outlive it. */
+im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im_env_config *cfg,
+                        void *cuda_stream, im_env **out);
+void im_env_destroy(im_env *e);
+
+/* Step 0: every env is reset with Philox counter (env id, step, 0, 0) to a
+ * uniform clip and a uniform start time in [0, D_clip - dt), and its first
+ * observation is built from the reference state.
+ *   obs_out DEVICE [N][ld_obs] */
+im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out);
+
+/* One control step (post-physics phase of Figure 2), in this order per env:
+ * t += dt; reference lookup + slerp + forward kinematics at t; error terms and
+ * reward; flags (terminated: root height / reward test; truncated: t + dt
+ * would pass the clip end); masked reset with Philox counter (env id, step,
+ * 0, 0) -- only flagged envs change clip/time, the others count one more
+ * step; observation of the (possibly reset) state in the character's heading
+ * frame plus the reference pose one control interval ahead.
+ *   sim        DEVICE, see im_body_state (read; written only for reset envs if write_back_reset)
+ *   obs_out    DEVICE [N][ld_obs]; row: J x (pos3, tangent3, normal3, linvel3, angvel3), phase t/D,
+ *              J x (target pos3, tangent3, normal3), zero padding
+ *   reward_out DEVICE [N]
+ *   flags_out  DEVICE [N] bytes: IM_FLAG_TERMINATED | IM_FLAG_TRUNCATED
+ *   terms_out  DEVICE [IM_N_TERMS][N] or NULL: the seven error terms */
+im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim,
+                      float *obs_out, float *reward_out, uint8_t *flags_out, float *terms_out);
+
+/* Copies the per-env state to / from DEVICE arrays of N elements (stream
+ * ordered); with the step number this is all that is needed to resume a
+ * rollout bit-exactly.  Any pointer may be NULL to skip that array. */
+im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_len);
+im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, const int32_t *ep_len);
+
+/* ---- policy ---------------------------------------------------------------
+ * Multi-layer perceptron h_{l+1} = relu(W_l h_l + b_l), last layer linear,
+ * giving the mean of a Gaussian with fixed standard deviation sigma (paper
+ * Figure 2 `policy(obs)`; Table 4 initial log-std).  action = mean + sigma z
+ * with z standard normal from Philox counter (env id, step, 1, block) and
+ * Box-Muller: block i feeds z[4i..4i+3].
+ *   dims    HOST [n_layers + 1]: input width, hidden widths, action width
+ *   W       HOST [n_layers] pointers, W[l] is [dims[l+1]][dims[l]] row-major,
+ *           float (dtype 0) or bf16 bit patterns as uint16 (dtype 1)
+ *   b       HOST [n_layers] pointers to float [dims[l+1]]
+ * dtype 0 runs fp32 SIMT kernels.  dtype 1 runs the tensor-core path: bf16
+ * operands (observations and hidden activations are rounded to bf16), fp32
+ * accumulation; it needs n_layers >= 2 and hidden widths that are multiples of 64. */
+typedef struct {
+    int32_t n_layers;
+    int32_t dims[IM_MAX_LAYERS + 1];
+    int32_t dtype;
+    float sigma;
+    uint64_t seed;
+    uint32_t env_id_base;
+    int32_t max_batch;       /* largest n a forward call will pass; sizes the activation buffers */
+    int32_t impl;            /* 0: default for dtype; 1: force the SIMT kernels (debug cross-check) */
+} im_policy_config;
+
+im_status im_load_policy(const im_policy_config *cfg, const void *const *W, const float *const *b,
+                         void *cuda_stream, im_policy **out);
+void im_destroy_policy(im_policy *p);
+
+/*   obs        DEVICE [n][ld_obs] float, ld_obs >= dims[0], multiple of 4, 16-byte aligned
+ *   mean_out   DEVICE [n][A]     action_out DEVICE [n][A]     logp_out DEVICE [n] or NULL
+ * logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi. */
+im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
+                            float *mean_out, float *action_out, float *logp_out);
+
+/* ---- whole step from host buffers ------------------------------------------
+ * Convenience for callers whose simulator lives in host memory: copies one
+ * step's body states HOST -> device, runs im_policy_forward on the current
+ * observation and then im_env_step, and copies action, reward and flags back,
+ * all on the env's stream, then waits for the stream.  The first call
+ * allocates the device staging buffers (so it is not capturable).  Call
+ * im_env_reset_all_host first.  sim_host is [13J][N] (pos rows, quat rows,
+ * linvel rows, angvel rows); pinned memory gives the copies full speed.
+ *   action_host HOST [N][A]   reward_host HOST [N]   flags_host HOST [N] */
+im_status im_env_reset_all_host(im_env *e, uint32_t step);
+im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_host,
+                       float *action_host, float *reward_host, uint8_t *flags_host);
+
+/* Reads the sticky device status word of an env or a policy handle (exactly
+ * one of them non-NULL).  This is the only call besides the *_host ones that
+ * waits for the stream. */
+im_status im_poll_device_status(im_env *e, im_policy *p, uint32_t *out);
+
+/* Number of kernel launches the library has enqueued since it was loaded. */
+uint64_t im_launch_count(void);
+
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
+#ifdef __cplusplus
+}
+#endif
+#endif /* IM_H_ */

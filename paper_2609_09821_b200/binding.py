@@ -1,0 +1,272 @@
+"""Thin ctypes binding over the C-ABI CUDA library (include/im.h).
+
+Argument marshalling only: every step of the path runs in the library's
+kernels.  torch supplies device memory and the CUDA stream.  The shared object
+is loaded on first use; if it is missing the calls raise -- there is no
+fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "_build", "libim_b200.so")
+N_TERMS = 7
+MAX_LAYERS = 8
+
+EXPORTS = [
+    "im_status_string", "im_create_skeleton", "im_destroy_skeleton", "im_load_clips", "im_destroy_clips",
+    "im_env_create", "im_env_destroy", "im_env_reset_all", "im_env_step", "im_env_get_state",
+    "im_env_set_state", "im_load_policy", "im_destroy_policy", "im_policy_forward",
+    "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
+]
+
+
+class RewardConfig(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("a", C.c_float * N_TERMS), ("w", C.c_float * N_TERMS),
+                ("h_min", C.c_float), ("r_min", C.c_float)]
+
+
+class EnvConfig(C.Structure):
+    _fields_ = [("n_envs", C.c_int32), ("env_id_base", C.c_uint32), ("dt", C.c_float), ("seed", C.c_uint64),
+                ("reward", RewardConfig), ("ld_obs", C.c_int32), ("write_back_reset", C.c_int32)]
+
+
+class BodyState(C.Structure):
+    _fields_ = [("pos", C.c_void_p), ("quat", C.c_void_p), ("linvel", C.c_void_p), ("angvel", C.c_void_p),
+                ("comp_stride", C.c_int64)]
+
+
+class PolicyConfig(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("dims", C.c_int32 * (MAX_LAYERS + 1)), ("dtype", C.c_int32),
+                ("sigma", C.c_float), ("seed", C.c_uint64), ("env_id_base", C.c_uint32),
+                ("max_batch", C.c_int32), ("impl", C.c_int32)]
+
+
+class ImError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__("%s: %s (status %d)" % (what, _lib.im_status_string(status).decode(), status))
+        self.status = status
+
+
+_lib = None
+
+
+def load():
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library not built: %s is missing (run python -m paper_2609_09821_b200.build)"
+                               % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        vp, i32, u32, u64 = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64
+        L.im_status_string.argtypes = [i32]
+        L.im_status_string.restype = C.c_char_p
+        L.im_create_skeleton.argtypes = [i32, vp, vp, vp, vp, i32, C.POINTER(vp)]
+        L.im_destroy_skeleton.argtypes = [vp]
+        L.im_load_clips.argtypes = [vp, i32, vp, vp, vp, vp, C.POINTER(vp)]
+        L.im_destroy_clips.argtypes = [vp]
+        L.im_env_create.argtypes = [vp, vp, C.POINTER(EnvConfig), vp, C.POINTER(vp)]
+        L.im_env_destroy.argtypes = [vp]
+        L.im_env_reset_all.argtypes = [vp, u32, vp]
+        L.im_env_step.argtypes = [vp, u32, C.POINTER(BodyState), vp, vp, vp, vp]
+        L.im_env_get_state.argtypes = [vp, vp, vp, vp]
+        L.im_env_set_state.argtypes = [vp, vp, vp, vp]
+        L.im_load_policy.argtypes = [C.POINTER(PolicyConfig), vp, vp, vp, C.POINTER(vp)]
+        L.im_destroy_policy.argtypes = [vp]
+        L.im_policy_forward.argtypes = [vp, u32, i32, vp, i32, vp, vp, vp]
+        L.im_env_reset_all_host.argtypes = [vp, u32]
+        L.im_step_host.argtypes = [vp, vp, u32, vp, vp, vp, vp]
+        L.im_poll_device_status.argtypes = [vp, vp, C.POINTER(u32)]
+        L.im_launch_count.restype = u64
+        for name in EXPORTS:
+            if name not in ("im_status_string", "im_launch_count") and not name.startswith("im_destroy") \
+                    and name != "im_env_destroy":
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise ImError(status, what)
+
+
+def _np(a, dtype):
+    return None if a is None else np.ascontiguousarray(a, dtype)
+
+
+def _ptr(a):
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data_as(C.c_void_p)
+    return C.c_void_p(a.data_ptr())          # torch tensor
+
+
+def launch_count() -> int:
+    return int(load().im_launch_count())
+
+
+class Skeleton:
+    def __init__(self, parents, offsets, masses=None, ee_ids=None):
+        L = load()
+        par = _np(parents, np.int32)
+        off = _np(offsets, np.float32)
+        m = _np(masses, np.float32)
+        ee = _np(ee_ids, np.int32)
+        self.J = int(par.shape[0])
+        self.h = C.c_void_p()
+        _check(L.im_create_skeleton(self.J, _ptr(par), _ptr(off), _ptr(m), _ptr(ee),
+                                    0 if ee is None else int(ee.shape[0]), C.byref(self.h)), "im_create_skeleton")
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.im_destroy_skeleton(self.h)
+            self.h = None
+
+
+class Clips:
+    def __init__(self, skel: Skeleton, n_frames, fps, root_pos, local_quat):
+        L = load()
+        self.skel = skel
+        nf = _np(n_frames, np.int32)
+        f = _np(fps, np.float32)
+        rp = _np(root_pos, np.float32)
+        lq = _np(local_quat, np.float32)
+        self.C = int(nf.shape[0])
+        total = int(nf.sum())
+        if rp.shape != (total, 3) or lq.shape != (total, skel.J, 4) or f.shape != (self.C,):
+            raise ValueError("clip arrays have inconsistent shapes")
+        self.h = C.c_void_p()
+        _check(L.im_load_clips(skel.h, self.C, _ptr(nf), _ptr(f), _ptr(rp), _ptr(lq), C.byref(self.h)),
+               "im_load_clips")
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.im_destroy_clips(self.h)
+            self.h = None
+
+
+def make_env_config(n_envs: int, dt: float, seed: int, reward: dict, h_min: float, ld_obs: int,
+                    r_min: float = -np.inf, env_id_base: int = 0, write_back_reset: bool = False) -> EnvConfig:
+    rc = RewardConfig(mode=int(reward["mode"]), h_min=np.float32(h_min), r_min=np.float32(r_min))
+    for k in range(N_TERMS):
+        rc.a[k] = reward["a"][k]
+        rc.w[k] = reward["w"][k]
+    return EnvConfig(n_envs=int(n_envs), env_id_base=int(env_id_base), dt=np.float32(dt), seed=int(seed),
+                     reward=rc, ld_obs=int(ld_obs), write_back_reset=int(write_back_reset))
+
+
+def padded_ld(D: int, multiple: int = 64) -> int:
+    """Row stride that keeps rows 16-byte aligned and a whole number of GEMM K tiles."""
+    return (D + multiple - 1) // multiple * multiple
+
+
+class Env:
+    """Per-env state plus the step calls; all tensors are torch CUDA tensors owned by the caller."""
+
+    def __init__(self, skel: Skeleton, clips: Clips, cfg: EnvConfig, stream=None):
+        import torch
+        L = load()
+        self.skel, self.clips, self.cfg = skel, clips, cfg
+        self.n, self.J, self.D, self.ld_obs = cfg.n_envs, skel.J, 24 * skel.J + 1, cfg.ld_obs
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.h = C.c_void_p()
+        _check(L.im_env_create(skel.h, clips.h, C.byref(cfg), C.c_void_p(self.stream.cuda_stream), C.byref(self.h)),
+               "im_env_create")
+
+    def new_obs(self):
+        import torch
+        return torch.empty((self.n, self.ld_obs), dtype=torch.float32, device="cuda")
+
+    def reset_all(self, obs_out, step: int = 0):
+        _check(load().im_env_reset_all(self.h, step, _ptr(obs_out)), "im_env_reset_all")
+
+    def step(self, step: int, sim, obs_out, reward_out, flags_out, terms_out=None):
+        """sim: CUDA fp32 tensor [13J, stride>=n] (pos, quat, linvel, angvel rows)."""
+        J = self.J
+        stride = sim.stride(0)
+        base = sim.data_ptr()
+        bs = BodyState(base, base + 3 * J * stride * 4, base + 7 * J * stride * 4, base + 10 * J * stride * 4, stride)
+        _check(load().im_env_step(self.h, step, C.byref(bs), _ptr(obs_out), _ptr(reward_out), _ptr(flags_out),
+                                  _ptr(terms_out)), "im_env_step")
+
+    def get_state(self):
+        import torch
+        c = torch.empty(self.n, dtype=torch.int32, device="cuda")
+        t = torch.empty(self.n, dtype=torch.float32, device="cuda")
+        l = torch.empty(self.n, dtype=torch.int32, device="cuda")
+        with torch.cuda.stream(self.stream):
+            _check(load().im_env_get_state(self.h, _ptr(c), _ptr(t), _ptr(l)), "im_env_get_state")
+        self.stream.synchronize()
+        return c, t, l
+
+    def set_state(self, clip_id=None, t=None, ep_len=None):
+        _check(load().im_env_set_state(self.h, _ptr(clip_id), _ptr(t), _ptr(ep_len)), "im_env_set_state")
+        self.stream.synchronize()
+
+    def reset_all_host(self, step: int = 0):
+        _check(load().im_env_reset_all_host(self.h, step), "im_env_reset_all_host")
+
+    def device_status(self) -> int:
+        out = C.c_uint32(0)
+        _check(load().im_poll_device_status(self.h, None, C.byref(out)), "im_poll_device_status")
+        return int(out.value)
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.im_env_destroy(self.h)
+            self.h = None
+
+
+class Policy:
+    def __init__(self, dims: Sequence[int], W, b, dtype: str, sigma: float, seed: int, max_batch: int,
+                 env_id_base: int = 0, impl: int = 0, stream=None):
+        """W[l]: numpy [dims[l+1], dims[l]], float32 (dtype 'f32') or uint16 bf16 bit patterns ('bf16')."""
+        import torch
+        L = load()
+        nl = len(dims) - 1
+        cfg = PolicyConfig(n_layers=nl, dtype=1 if dtype == "bf16" else 0, sigma=np.float32(sigma), seed=int(seed),
+                           env_id_base=int(env_id_base), max_batch=int(max_batch), impl=int(impl))
+        for i, d in enumerate(dims):
+            cfg.dims[i] = int(d)
+        wt = np.uint16 if dtype == "bf16" else np.float32
+        Wc = [_np(w, wt) for w in W]
+        bc = [_np(x, np.float32) for x in b]
+        for l in range(nl):
+            if Wc[l].shape != (dims[l + 1], dims[l]) or bc[l].shape != (dims[l + 1],):
+                raise ValueError("layer %d has the wrong shape" % l)
+        Wp = (C.c_void_p * nl)(*[w.ctypes.data for w in Wc])
+        bp = (C.c_void_p * nl)(*[x.ctypes.data for x in bc])
+        self.dims, self.A, self.max_batch = tuple(dims), int(dims[-1]), int(max_batch)
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.h = C.c_void_p()
+        _check(L.im_load_policy(C.byref(cfg), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p),
+                                C.c_void_p(self.stream.cuda_stream), C.byref(self.h)), "im_load_policy")
+
+    def forward(self, step: int, obs, mean_out, action_out, logp_out=None, n: Optional[int] = None):
+        n = obs.shape[0] if n is None else n
+        _check(load().im_policy_forward(self.h, step, n, _ptr(obs), obs.stride(0), _ptr(mean_out),
+                                        _ptr(action_out), _ptr(logp_out)), "im_policy_forward")
+
+    def device_status(self) -> int:
+        out = C.c_uint32(0)
+        _check(load().im_poll_device_status(None, self.h, C.byref(out)), "im_poll_device_status")
+        return int(out.value)
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.im_destroy_policy(self.h)
+            self.h = None
+
+
+def step_host(env: Env, policy: Policy, step: int, sim_host, action_host, reward_host, flags_host):
+    """One whole step from host buffers (numpy arrays or pinned CPU torch tensors)."""
+    _check(load().im_step_host(env.h, policy.h, step, _ptr(sim_host), _ptr(action_host), _ptr(reward_host),
+                               _ptr(flags_host)), "im_step_host")

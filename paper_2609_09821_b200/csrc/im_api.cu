@@ -1,0 +1,425 @@
+// C-ABI entry points: validation, uploads, handle management, kernel launches.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "im_internal.h"
+#include "mlp.h"
+
+namespace im {
+std::atomic<uint64_t> g_launches{0};
+}
+
+using namespace im;
+
+#define IM_CUDA(call)                                  \
+    do {                                               \
+        cudaError_t e__ = (call);                      \
+        if (e__ != cudaSuccess) return IM_ERR_CUDA;    \
+    } while (0)
+
+extern "C" {
+
+const char *im_status_string(im_status s)
+{
+    switch (s) {
+    case IM_OK: return "ok";
+    case IM_ERR_INVALID_ARG: return "invalid argument";
+    case IM_ERR_BAD_TOPOLOGY: return "bad skeleton topology";
+    case IM_ERR_BAD_QUAT: return "keyframe quaternion is not a finite unit quaternion";
+    case IM_ERR_ALLOC: return "allocation failed";
+    case IM_ERR_CUDA: return "CUDA call failed";
+    case IM_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown status";
+    }
+}
+
+uint64_t im_launch_count(void) { return g_launches.load(); }
+
+/* ------------------------------------------------------------------ skeleton */
+im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *offsets, const float *masses,
+                             const int32_t *ee_ids, int32_t n_ee, im_skeleton **out)
+{
+    if (!out || !parents || !offsets) return IM_ERR_INVALID_ARG;
+    if (J < 1 || J > IM_MAX_BODIES || parents[0] != -1) return IM_ERR_BAD_TOPOLOGY;
+    for (int j = 1; j < J; ++j)
+        if (parents[j] < 0 || parents[j] >= j) return IM_ERR_BAD_TOPOLOGY;
+    if (ee_ids && n_ee > 0) {
+        if (n_ee > J) return IM_ERR_INVALID_ARG;
+        for (int i = 0; i < n_ee; ++i)
+            if (ee_ids[i] < 0 || ee_ids[i] >= J) return IM_ERR_INVALID_ARG;
+    }
+    double msum = 0.0;
+    for (int j = 0; j < J; ++j) {
+        const double m = masses ? (double)masses[j] : 1.0;
+        if (!(m > 0.0) || !std::isfinite(m)) return IM_ERR_INVALID_ARG;
+        for (int c = 0; c < 3; ++c)
+            if (!std::isfinite(offsets[3 * j + c])) return IM_ERR_INVALID_ARG;
+        msum += m;
+    }
+    im_skeleton *s = new (std::nothrow) im_skeleton();
+    if (!s) return IM_ERR_ALLOC;
+    std::memset(s, 0, sizeof(*s));
+    SkelDev &d = s->dev;
+    d.J = J;
+    for (int j = 0; j < J; ++j) {
+        d.parent[j] = parents[j];
+        for (int c = 0; c < 3; ++c) d.off[j][c] = j == 0 ? 0.0f : offsets[3 * j + c];
+        d.mass_frac[j] = (float)((masses ? (double)masses[j] : 1.0) / msum);
+        // ancestor chain root .. j
+        int depth = 0;
+        for (int a = j; a > 0; a = parents[a]) ++depth;
+        d.depth[j] = (uint8_t)depth;
+        int a = j;
+        for (int k = depth; k >= 0; --k) { d.chain[j][k] = (uint8_t)a; a = a > 0 ? parents[a] : 0; }
+    }
+    if (ee_ids && n_ee > 0) {
+        for (int i = 0; i < n_ee; ++i) d.ee_mask |= 1u << ee_ids[i];
+    } else {
+        uint32_t has_child = 0;
+        for (int j = 1; j < J; ++j) has_child |= 1u << parents[j];
+        d.ee_mask = ~has_child & (J == 32 ? 0xffffffffu : ((1u << J) - 1u));
+    }
+    s->n_ee = __builtin_popcount(d.ee_mask);
+    *out = s;
+    return IM_OK;
+}
+
+void im_destroy_skeleton(im_skeleton *s) { delete s; }
+
+/* ------------------------------------------------------------------ clips */
+im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_frames, const float *fps,
+                        const float *root_pos, const float *local_quat, im_clips **out)
+{
+    if (!skel || !out || !n_frames || !fps || !root_pos || !local_quat || C < 1) return IM_ERR_INVALID_ARG;
+    const int J = skel->dev.J;
+    int64_t rows = 0;
+    for (int c = 0; c < C; ++c) {
+        if (n_frames[c] < 2 || !(fps[c] > 0.0f) || !std::isfinite(fps[c])) return IM_ERR_INVALID_ARG;
+        rows += n_frames[c];
+    }
+    if (rows > 0x7fffffff) return IM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < rows * J; ++i) {
+        const float *q = local_quat + 4 * i;
+        const double n2 = (double)q[0] * q[0] + (double)q[1] * q[1] + (double)q[2] * q[2] + (double)q[3] * q[3];
+        if (!std::isfinite(n2) || std::fabs(std::sqrt(n2) - 1.0) > 1e-3) return IM_ERR_BAD_QUAT;
+    }
+    for (int64_t i = 0; i < rows * 3; ++i)
+        if (!std::isfinite(root_pos[i])) return IM_ERR_INVALID_ARG;
+
+    im_clips *cl = new (std::nothrow) im_clips();
+    if (!cl) return IM_ERR_ALLOC;
+    cl->C = C; cl->J = J; cl->rows = rows; cl->d_frames = nullptr; cl->d_meta = nullptr;
+    cl->meta.resize(C);
+    cl->min_dur = INFINITY;
+    int32_t start = 0;
+    for (int c = 0; c < C; ++c) {
+        cl->meta[c] = {n_frames[c], fps[c], (float)(n_frames[c] - 1) / fps[c], start};
+        cl->min_dur = std::fmin(cl->min_dur, cl->meta[c].dur);
+        start += n_frames[c];
+    }
+    // Packed rows of (1 + J) float4: (x, y, z, 0), q_0 .. q_{J-1}.  Quaternions are stored as
+    // given: every formula that consumes them is invariant to their (<= 1e-3) scale error.
+    const size_t RS = (size_t)J + 1;
+    std::vector<float4> host((size_t)rows * RS);
+    for (int64_t r = 0; r < rows; ++r) {
+        host[r * RS] = make_float4(root_pos[3 * r], root_pos[3 * r + 1], root_pos[3 * r + 2], 0.0f);
+        for (int j = 0; j < J; ++j) {
+            const float *q = local_quat + 4 * (r * J + j);
+            host[r * RS + 1 + j] = make_float4(q[0], q[1], q[2], q[3]);
+        }
+    }
+    cudaGetDevice(&cl->device);
+    if (cudaMalloc(&cl->d_frames, host.size() * sizeof(float4)) != cudaSuccess ||
+        cudaMalloc(&cl->d_meta, C * sizeof(ClipMeta)) != cudaSuccess) {
+        im_destroy_clips(cl);
+        return IM_ERR_ALLOC;
+    }
+    if (cudaMemcpy(cl->d_frames, host.data(), host.size() * sizeof(float4), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(cl->d_meta, cl->meta.data(), C * sizeof(ClipMeta), cudaMemcpyHostToDevice) != cudaSuccess) {
+        im_destroy_clips(cl);
+        return IM_ERR_CUDA;
+    }
+    *out = cl;
+    return IM_OK;
+}
+
+void im_destroy_clips(im_clips *c)
+{
+    if (!c) return;
+    cudaFree(c->d_frames);
+    cudaFree(c->d_meta);
+    delete c;
+}
+
+/* ------------------------------------------------------------------ env */
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im_env_config *cfg,
+                        void *cuda_stream, im_env **out)
+{
+    if (!skel || !clips || !cfg || !out) return IM_ERR_INVALID_ARG;
+    const int J = skel->dev.J, D = 24 * J + 1;
+    if (clips->J != J || cfg->n_envs < 1) return IM_ERR_INVALID_ARG;
+    if (cfg->ld_obs < D || (cfg->ld_obs & 3)) return IM_ERR_INVALID_ARG;
+    if (!(cfg->dt > 0.0f) || !(cfg->dt <= clips->min_dur)) return IM_ERR_INVALID_ARG;
+    if (cfg->reward.mode != 0 && cfg->reward.mode != 1) return IM_ERR_INVALID_ARG;
+    for (int k = 0; k < IM_N_TERMS; ++k)
+        if (!std::isfinite(cfg->reward.w[k]) || !std::isfinite(cfg->reward.a[k]) || cfg->reward.w[k] < 0.0f)
+            return IM_ERR_INVALID_ARG;
+    if (std::isnan(cfg->reward.h_min) || std::isnan(cfg->reward.r_min)) return IM_ERR_INVALID_ARG;
+
+    im_env *e = new (std::nothrow) im_env();
+    if (!e) return IM_ERR_ALLOC;
+    std::memset(e, 0, sizeof(*e));
+    e->skel = skel; e->clips = clips; e->cfg = *cfg; e->stream = (cudaStream_t)cuda_stream; e->D = D;
+    e->smem_bytes = env_kernel_smem_bytes(J);
+    int dev = 0, max_smem = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if ((int)e->smem_bytes > max_smem) { delete e; return IM_ERR_UNSUPPORTED; }
+    if (env_kernel_prepare(J, e->smem_bytes) != cudaSuccess) { delete e; return IM_ERR_CUDA; }
+    const size_t n = (size_t)cfg->n_envs;
+    if (cudaMalloc(&e->d_clip_id, n * 4) != cudaSuccess || cudaMalloc(&e->d_t, n * 4) != cudaSuccess ||
+        cudaMalloc(&e->d_ep_len, n * 4) != cudaSuccess || cudaMalloc(&e->d_status, 4) != cudaSuccess) {
+        im_env_destroy(e);
+        return IM_ERR_ALLOC;
+    }
+    cudaMemsetAsync(e->d_clip_id, 0, n * 4, e->stream);
+    cudaMemsetAsync(e->d_t, 0, n * 4, e->stream);
+    cudaMemsetAsync(e->d_ep_len, 0, n * 4, e->stream);
+    cudaMemsetAsync(e->d_status, 0, 4, e->stream);
+    *out = e;
+    return IM_OK;
+}
+
+void im_env_destroy(im_env *e)
+{
+    if (!e) return;
+    cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status);
+    cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
+    cudaFree(e->d_action); cudaFree(e->d_flags);
+    delete e;
+}
+
+static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
+{
+    std::memset(&p, 0, sizeof(p));
+    p.sk = e->skel->dev;
+    p.frames = e->clips->d_frames;
+    p.meta = e->clips->d_meta;
+    p.C = e->clips->C;
+    p.N = e->cfg.n_envs;
+    p.env_id_base = e->cfg.env_id_base;
+    p.dt = e->cfg.dt;
+    p.seed_lo = (uint32_t)e->cfg.seed;
+    p.seed_hi = (uint32_t)(e->cfg.seed >> 32);
+    p.reward = e->cfg.reward;
+    p.ld_obs = e->cfg.ld_obs;
+    p.write_back = e->cfg.write_back_reset;
+    p.step = step;
+    p.clip_id = e->d_clip_id;
+    p.t = e->d_t;
+    p.ep_len = e->d_ep_len;
+    p.status = e->d_status;
+}
+
+im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out)
+{
+    if (!e || !obs_out || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
+    EnvKernelParams p;
+    fill_params(e, step, p);
+    p.obs = obs_out;
+    IM_CUDA(launch_env_kernel(p, true, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float *obs_out, float *reward_out,
+                      uint8_t *flags_out, float *terms_out)
+{
+    if (!e || !sim || !obs_out || !reward_out || !flags_out) return IM_ERR_INVALID_ARG;
+    if (!sim->pos || !sim->quat || !sim->linvel || !sim->angvel || sim->comp_stride < e->cfg.n_envs)
+        return IM_ERR_INVALID_ARG;
+    if (!aligned16(obs_out) || !aligned16(sim->pos) || !aligned16(sim->quat) || !aligned16(sim->linvel) ||
+        !aligned16(sim->angvel) || (sim->comp_stride & 3))
+        return IM_ERR_INVALID_ARG;
+    EnvKernelParams p;
+    fill_params(e, step, p);
+    p.pos = sim->pos; p.quat = sim->quat; p.lin = sim->linvel; p.ang = sim->angvel;
+    p.stride = sim->comp_stride;
+    p.obs = obs_out; p.reward_out = reward_out; p.flags_out = flags_out; p.terms_out = terms_out;
+    IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_len)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    const size_t b = (size_t)e->cfg.n_envs * 4;
+    if (clip_id) IM_CUDA(cudaMemcpyAsync(clip_id, e->d_clip_id, b, cudaMemcpyDeviceToDevice, e->stream));
+    if (t) IM_CUDA(cudaMemcpyAsync(t, e->d_t, b, cudaMemcpyDeviceToDevice, e->stream));
+    if (ep_len) IM_CUDA(cudaMemcpyAsync(ep_len, e->d_ep_len, b, cudaMemcpyDeviceToDevice, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, const int32_t *ep_len)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    const size_t b = (size_t)e->cfg.n_envs * 4;
+    if (clip_id) IM_CUDA(cudaMemcpyAsync(e->d_clip_id, clip_id, b, cudaMemcpyDeviceToDevice, e->stream));
+    if (t) IM_CUDA(cudaMemcpyAsync(e->d_t, t, b, cudaMemcpyDeviceToDevice, e->stream));
+    if (ep_len) IM_CUDA(cudaMemcpyAsync(e->d_ep_len, ep_len, b, cudaMemcpyDeviceToDevice, e->stream));
+    return IM_OK;
+}
+
+/* ------------------------------------------------------------------ policy */
+im_status im_load_policy(const im_policy_config *cfg, const void *const *W, const float *const *b,
+                         void *cuda_stream, im_policy **out)
+{
+    if (!cfg || !W || !b || !out) return IM_ERR_INVALID_ARG;
+    const int nl = cfg->n_layers;
+    if (nl < 1 || nl > IM_MAX_LAYERS || cfg->max_batch < 1) return IM_ERR_INVALID_ARG;
+    if (cfg->dtype != 0 && cfg->dtype != 1) return IM_ERR_INVALID_ARG;
+    if (!(cfg->sigma > 0.0f) || !std::isfinite(cfg->sigma)) return IM_ERR_INVALID_ARG;
+    int max_hidden = 1;
+    for (int l = 0; l <= nl; ++l) {
+        if (cfg->dims[l] < 1) return IM_ERR_INVALID_ARG;
+        if (l > 0 && l < nl) max_hidden = cfg->dims[l] > max_hidden ? cfg->dims[l] : max_hidden;
+    }
+    for (int l = 0; l < nl; ++l)
+        if (!W[l] || !b[l]) return IM_ERR_INVALID_ARG;
+
+    im_policy *p = new (std::nothrow) im_policy();
+    if (!p) return IM_ERR_ALLOC;
+    std::memset(p, 0, sizeof(*p));
+    p->cfg = *cfg; p->stream = (cudaStream_t)cuda_stream; p->nl = nl;
+    p->tensor_path = cfg->dtype == 1 && cfg->impl == 0;
+    if (cudaMalloc(&p->d_status, 4) != cudaSuccess) { im_destroy_policy(p); return IM_ERR_ALLOC; }
+    cudaMemsetAsync(p->d_status, 0, 4, p->stream);
+    if (p->tensor_path) {
+        const im_status s = tc_policy_create(p, W, b);
+        if (s != IM_OK) { im_destroy_policy(p); return s; }
+        *out = p;
+        return IM_OK;
+    }
+    const size_t esz = cfg->dtype == 1 ? 2 : 4;
+    for (int l = 0; l < nl; ++l) {
+        const size_t wn = (size_t)cfg->dims[l] * cfg->dims[l + 1];
+        if (cudaMalloc(&p->d_W[l], wn * esz) != cudaSuccess ||
+            cudaMalloc(&p->d_b[l], (size_t)cfg->dims[l + 1] * 4) != cudaSuccess) {
+            im_destroy_policy(p);
+            return IM_ERR_ALLOC;
+        }
+        if (cudaMemcpy(p->d_W[l], W[l], wn * esz, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(p->d_b[l], b[l], (size_t)cfg->dims[l + 1] * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+            im_destroy_policy(p);
+            return IM_ERR_CUDA;
+        }
+    }
+    p->act_ld = max_hidden;
+    for (int i = 0; i < 2; ++i)
+        if (cudaMalloc(&p->d_act[i], (size_t)cfg->max_batch * max_hidden * 4) != cudaSuccess) {
+            im_destroy_policy(p);
+            return IM_ERR_ALLOC;
+        }
+    *out = p;
+    return IM_OK;
+}
+
+void im_destroy_policy(im_policy *p)
+{
+    if (!p) return;
+    if (p->tc) tc_policy_destroy(p);
+    for (int l = 0; l < IM_MAX_LAYERS; ++l) { cudaFree(p->d_W[l]); cudaFree(p->d_b[l]); }
+    cudaFree(p->d_act[0]); cudaFree(p->d_act[1]); cudaFree(p->d_status);
+    delete p;
+}
+
+im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
+                            float *mean_out, float *action_out, float *logp_out)
+{
+    if (!p || !obs || !mean_out || !action_out) return IM_ERR_INVALID_ARG;
+    if (n < 1 || n > p->cfg.max_batch || ld_obs < p->cfg.dims[0] || (ld_obs & 3) || !aligned16(obs))
+        return IM_ERR_INVALID_ARG;
+    if (p->tensor_path) return tc_policy_forward(p, step, n, obs, ld_obs, mean_out, action_out, logp_out);
+    const float *in = obs;
+    int ld_in = ld_obs;
+    const int A = p->cfg.dims[p->nl];
+    for (int l = 0; l < p->nl; ++l) {
+        const bool last = l == p->nl - 1;
+        float *outp = last ? mean_out : p->d_act[l & 1];
+        const int ldc = last ? A : p->act_ld;
+        IM_CUDA(launch_linear_simt(in, ld_in, p->d_W[l], p->cfg.dtype == 1, p->d_b[l], outp, ldc, n,
+                                   p->cfg.dims[l + 1], p->cfg.dims[l], !last, p->stream));
+        in = outp;
+        ld_in = ldc;
+    }
+    IM_CUDA(launch_sample(mean_out, action_out, logp_out, n, A, p->cfg.sigma, p->cfg.seed, step,
+                          p->cfg.env_id_base, p->stream));
+    return IM_OK;
+}
+
+/* ------------------------------------------------------------------ host-buffer step */
+static im_status ensure_staging(im_env *e, int A)
+{
+    const size_t n = (size_t)e->cfg.n_envs, J = (size_t)e->skel->dev.J;
+    if (!e->d_sim) {
+        if (cudaMalloc(&e->d_sim, 13 * J * n * 4) != cudaSuccess ||
+            cudaMalloc(&e->d_obs, n * (size_t)e->cfg.ld_obs * 4) != cudaSuccess ||
+            cudaMalloc(&e->d_reward, n * 4) != cudaSuccess || cudaMalloc(&e->d_flags, n) != cudaSuccess)
+            return IM_ERR_ALLOC;
+    }
+    if (A > e->staged_A) {
+        cudaFree(e->d_mean); cudaFree(e->d_action);
+        e->d_mean = e->d_action = nullptr;
+        if (cudaMalloc(&e->d_mean, n * (size_t)A * 4) != cudaSuccess ||
+            cudaMalloc(&e->d_action, n * (size_t)A * 4) != cudaSuccess)
+            return IM_ERR_ALLOC;
+        e->staged_A = A;
+    }
+    return IM_OK;
+}
+
+im_status im_env_reset_all_host(im_env *e, uint32_t step)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    const im_status s = ensure_staging(e, 0);
+    if (s != IM_OK) return s;
+    return im_env_reset_all(e, step, e->d_obs);
+}
+
+im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_host, float *action_host,
+                       float *reward_host, uint8_t *flags_host)
+{
+    if (!e || !p || !sim_host || !action_host || !reward_host || !flags_host) return IM_ERR_INVALID_ARG;
+    if (p->stream != e->stream || p->cfg.max_batch < e->cfg.n_envs || p->cfg.dims[0] != e->D) return IM_ERR_INVALID_ARG;
+    const int A = p->cfg.dims[p->nl];
+    if (!e->d_obs) return IM_ERR_INVALID_ARG;          // im_env_reset_all_host has not run
+    im_status s = ensure_staging(e, A);
+    if (s != IM_OK) return s;
+    const size_t n = (size_t)e->cfg.n_envs, J = (size_t)e->skel->dev.J;
+    IM_CUDA(cudaMemcpyAsync(e->d_sim, sim_host, 13 * J * n * 4, cudaMemcpyHostToDevice, e->stream));
+    s = im_policy_forward(p, step, (int32_t)n, e->d_obs, e->cfg.ld_obs, e->d_mean, e->d_action, nullptr);
+    if (s != IM_OK) return s;
+    im_body_state sim = {e->d_sim, e->d_sim + 3 * J * n, e->d_sim + 7 * J * n, e->d_sim + 10 * J * n, (int64_t)n};
+    s = im_env_step(e, step, &sim, e->d_obs, e->d_reward, e->d_flags, nullptr);
+    if (s != IM_OK) return s;
+    IM_CUDA(cudaMemcpyAsync(action_host, e->d_action, n * (size_t)A * 4, cudaMemcpyDeviceToHost, e->stream));
+    IM_CUDA(cudaMemcpyAsync(reward_host, e->d_reward, n * 4, cudaMemcpyDeviceToHost, e->stream));
+    IM_CUDA(cudaMemcpyAsync(flags_host, e->d_flags, n, cudaMemcpyDeviceToHost, e->stream));
+    IM_CUDA(cudaStreamSynchronize(e->stream));
+    return IM_OK;
+}
+
+im_status im_poll_device_status(im_env *e, im_policy *p, uint32_t *out)
+{
+    if (!out || (!e && !p) || (e && p)) return IM_ERR_INVALID_ARG;
+    cudaStream_t st = e ? e->stream : p->stream;
+    const uint32_t *src = e ? e->d_status : p->d_status;
+    IM_CUDA(cudaMemcpyAsync(out, src, 4, cudaMemcpyDeviceToHost, st));
+    IM_CUDA(cudaStreamSynchronize(st));
+    return IM_OK;
+}
+
+}  // extern "C"

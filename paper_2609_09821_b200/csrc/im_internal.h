@@ -1,0 +1,101 @@
+// Host-side definitions shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <atomic>
+#include <vector>
+
+#include "../../include/im.h"
+
+namespace im {
+
+extern std::atomic<uint64_t> g_launches;   // kernels enqueued by this library
+
+// Per-clip metadata, one 16-byte record so a thread fetches it with one load.
+struct ClipMeta {
+    int32_t K;        // keyframes
+    float fps;
+    float dur;        // (K-1)/fps, fp32 division
+    int32_t start;    // first row of the clip in the packed keyframe table
+};
+
+// Skeleton as the kernels see it (passed by value inside the kernel parameters).
+struct SkelDev {
+    int32_t J;
+    uint32_t ee_mask;
+    int32_t parent[IM_MAX_BODIES];
+    float off[IM_MAX_BODIES][3];
+    float mass_frac[IM_MAX_BODIES];                    // m_j / sum m
+    uint8_t depth[IM_MAX_BODIES];                      // number of ancestors
+    uint8_t chain[IM_MAX_BODIES][IM_MAX_BODIES];       // chain[j][0..depth[j]] = root .. j
+};
+
+struct EnvKernelParams {
+    SkelDev sk;
+    // clip library
+    const float4 *frames;     // [rows][1+J] float4: (x,y,z,0), q_0 .. q_{J-1}
+    const ClipMeta *meta;     // [C]
+    int32_t C;
+    // configuration
+    int32_t N;
+    uint32_t env_id_base;
+    float dt;
+    uint32_t seed_lo, seed_hi;
+    im_reward_config reward;
+    int32_t ld_obs;
+    int32_t write_back;
+    uint32_t step;
+    // per-env state
+    int32_t *clip_id;
+    float *t;
+    int32_t *ep_len;
+    // per-step I/O
+    float *pos, *quat, *lin, *ang;
+    long long stride;
+    float *obs;
+    float *reward_out;
+    uint8_t *flags_out;
+    float *terms_out;
+    uint32_t *status;
+};
+
+}  // namespace im
+
+struct im_skeleton {
+    im::SkelDev dev;
+    int32_t n_ee;
+};
+
+struct im_clips {
+    int32_t C, J;
+    int64_t rows;
+    float4 *d_frames;
+    im::ClipMeta *d_meta;
+    std::vector<im::ClipMeta> meta;
+    float min_dur;
+    int device;
+};
+
+struct im_env {
+    const im_skeleton *skel;
+    const im_clips *clips;
+    im_env_config cfg;
+    cudaStream_t stream;
+    int32_t *d_clip_id;
+    float *d_t;
+    int32_t *d_ep_len;
+    uint32_t *d_status;
+    int D;                 // 24J + 1
+    size_t smem_bytes;
+    // staging for the *_host entry points (allocated on first use)
+    float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
+    uint8_t *d_flags;
+    int staged_A;
+};
+
+// Launchers implemented in the kernel translation units.
+namespace im {
+size_t env_kernel_smem_bytes(int J);
+cudaError_t env_kernel_prepare(int J, size_t smem);
+cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
+}  // namespace im

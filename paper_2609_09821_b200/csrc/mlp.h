@@ -1,0 +1,32 @@
+// Policy-side declarations shared by the MLP translation units and the API glue.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/im.h"
+
+struct im_policy {
+    im_policy_config cfg;
+    cudaStream_t stream;
+    int nl;
+    bool tensor_path;                 // bf16 tcgen05 chain (else fp32 SIMT layers)
+    void *d_W[IM_MAX_LAYERS];         // SIMT path: weights as given ([out][in], float or bf16)
+    float *d_b[IM_MAX_LAYERS];
+    float *d_act[2];                  // SIMT path: fp32 activations, [max_batch][max hidden]
+    int act_ld;
+    uint32_t *d_status;
+    struct im_policy_tc *tc;          // tensor path state (weights padded for the GEMM tiles, bf16 activations, tensor maps)
+};
+
+namespace im {
+cudaError_t launch_linear_simt(const float *A, int lda, const void *W, bool w_bf16, const float *bias, float *C,
+                               int ldc, int M, int N, int K, bool relu, cudaStream_t stream);
+cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, int A, float sigma,
+                          uint64_t seed, uint32_t step, uint32_t env_id_base, cudaStream_t stream);
+
+// Tensor-core path (mlp_tc.cu).
+im_status tc_policy_create(im_policy *p, const void *const *W, const float *const *b);
+void tc_policy_destroy(im_policy *p);
+im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
+                            float *mean_out, float *action_out, float *logp_out);
+}  // namespace im

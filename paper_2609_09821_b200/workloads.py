@@ -203,7 +203,7 @@ def analytic_pose(lib: dict, clip_id: np.ndarray, tau: np.ndarray):
 
 
 def _kinematics(skel: dict, root_p: np.ndarray, q_l: np.ndarray):
-    """World positions [n,J,3] and rotations [n,J,4] of every body."""
+    """World positions [n,J,3] and rotations [n,J,4] of every body (numpy, small inputs)."""
     J = skel["J"]
     par = skel["parents"]
     off = skel["offsets"].astype(np.float64)
@@ -218,42 +218,126 @@ def _kinematics(skel: dict, root_p: np.ndarray, q_l: np.ndarray):
     return p, q
 
 
-def synth_sim_state(skel: dict, lib: dict, clip_id: np.ndarray, t: np.ndarray, step: int,
-                    wl: Workload, seed: Optional[int] = None, env_base: int = 0) -> np.ndarray:
-    """Stand-in for the simulator: body states of n envs as one fp32 array [13J, n].
+# ---- the simulator stand-in proper, in torch so that it runs on whichever device holds the
+# ---- rollout (a few million env-steps per benchmark run would take minutes in numpy)
+def _t_qmul(a, b):
+    import torch
+    aw, ax, ay, az = a.unbind(-1)
+    bw, bx, by, bz = b.unbind(-1)
+    return torch.stack([aw * bw - ax * bx - ay * by - az * bz,
+                        aw * bx + ax * bw + ay * bz - az * by,
+                        aw * by - ax * bz + ay * bw + az * bx,
+                        aw * bz + ax * by - ay * bx + az * bw], dim=-1)
 
-    Rows: 3J positions (x,y,z per body), 4J quaternions (w,x,y,z per body),
-    3J linear velocities, 3J angular velocities (world frame); element (c, e)
-    at c*n + e.  State = analytic motion at each env's time plus joint-rotation
-    noise N(0, sigma_q) rad, root noise N(0, sigma_root) m, and velocities from
-    a central finite difference of the noise-free motion over 1/fps plus
-    N(0, sigma_vel) per component.
+
+def _t_qrot(q, v):
+    import torch
+    w, u = q[..., :1], q[..., 1:]
+    t = 2.0 * torch.linalg.cross(u, v)
+    return v + w * t + torch.linalg.cross(u, t)
+
+
+def _t_qexp_half(r):
+    import torch
+    ang = torch.linalg.norm(r, dim=-1, keepdim=True)
+    half = 0.5 * ang
+    k = torch.where(ang > 1e-12, torch.sin(half) / ang.clamp_min(1e-300), torch.full_like(ang, 0.5))
+    return torch.cat([torch.cos(half), k * r], dim=-1)
+
+
+def _t_qlog_rotvec(q):
+    import torch
+    q = torch.where(q[..., :1] < 0, -q, q)
+    n = torch.linalg.norm(q[..., 1:], dim=-1, keepdim=True)
+    ang = 2.0 * torch.atan2(n, q[..., :1])
+    k = torch.where(n > 1e-12, ang / n.clamp_min(1e-300), torch.full_like(n, 2.0))
+    return k * q[..., 1:]
+
+
+def _motion_coeffs(lib: dict, device):
+    """[C, J, 2H, 3] table so that r = coeffs . [sin(w_m tau), cos(w_m tau)] (angle addition)."""
+    import torch
+    key = "_coef_%s" % (device,)
+    if key not in lib:
+        amp, phi = lib["amp"], lib["phi"]                      # [C,J,H,3]
+        coef = np.concatenate([amp * np.cos(phi), amp * np.sin(phi)], axis=2)
+        lib[key] = torch.from_numpy(coef).to(device)
+    return lib[key]
+
+
+def _t_analytic_pose(lib: dict, clip_id, tau):
+    import torch
+    coef = _motion_coeffs(lib, tau.device)
+    m = torch.arange(1, N_HARM + 1, dtype=torch.float64, device=tau.device)
+    arg = (2.0 * math.pi * 0.5) * tau[:, None] * m[None, :]
+    basis = torch.cat([torch.sin(arg), torch.cos(arg)], dim=1)                 # [n, 2H]
+    r = torch.einsum("njkc,nk->njc", coef[clip_id], basis)
+    q = _t_qexp_half(r)
+    p = torch.stack([tau, torch.zeros_like(tau), ROOT_HEIGHT + 0.05 * torch.sin(2.0 * math.pi * tau)], dim=-1)
+    return p, q
+
+
+def _t_kinematics(skel: dict, root_p, q_l):
+    import torch
+    J = skel["J"]
+    par = skel["parents"]
+    off = torch.from_numpy(skel["offsets"].astype(np.float64)).to(q_l.device)
+    p = [root_p]
+    q = [q_l[:, 0]]
+    for j in range(1, J):
+        a = int(par[j])
+        q.append(_t_qmul(q[a], q_l[:, j]))
+        p.append(p[a] + _t_qrot(q[a], off[j].expand_as(p[a])))
+    return torch.stack(p, dim=1), torch.stack(q, dim=1)
+
+
+def synth_sim_state_torch(skel: dict, lib: dict, clip_id, t, step: int, wl: Workload,
+                          seed: Optional[int] = None, env_base: int = 0):
+    """Stand-in for the simulator: body states of n envs as one fp32 tensor [13J, n].
+
+    clip_id (int64) and t (float64) are torch tensors; the result lives on their
+    device.  Rows: 3J positions (x,y,z per body), 4J quaternions (w,x,y,z per
+    body), 3J linear velocities, 3J angular velocities (world frame); element
+    (c, e) at c*n + e.  State = analytic motion at each env's time plus
+    joint-rotation noise N(0, sigma_q) rad, root noise N(0, sigma_root) m, and
+    velocities from a central finite difference of the noise-free motion over
+    1/fps plus N(0, sigma_vel) per component.  The noise is seeded per (seed,
+    step, env_base) on the device in use.
     """
+    import torch
     seed = wl.seed if seed is None else seed
+    dev = t.device
     n = clip_id.shape[0]
     J = skel["J"]
-    g = _rng(seed, 18, step, env_base)
-    tau = t.astype(np.float64)
-    cid = clip_id.astype(np.int64)
+    g = torch.Generator(device=dev)
+    g.manual_seed((int(seed) * 1000003 + int(step)) * 1000003 + int(env_base) + 18)
+    tau = t.to(torch.float64)
+    cid = clip_id.to(torch.int64)
     h = 1.0 / wl.fps
-    p0, q0 = analytic_pose(lib, cid, tau)
-    pa, qa = analytic_pose(lib, cid, tau - 0.5 * h)
-    pb, qb = analytic_pose(lib, cid, tau + 0.5 * h)
-    Pa, Qa = _kinematics(skel, pa, qa)
-    Pb, Qb = _kinematics(skel, pb, qb)
-    lin = (Pb - Pa) / h
-    ang = _qlog_rotvec(_qmul(Qb, _qconj(Qa))) / h
-    qn = _qmul(q0, _qexp_half(g.standard_normal((n, J, 3)) * wl.sigma_q))
-    pn = p0 + g.standard_normal((n, 3)) * wl.sigma_root
-    P, Q = _kinematics(skel, pn, qn)
-    lin = lin + g.standard_normal((n, J, 3)) * wl.sigma_vel
-    ang = ang + g.standard_normal((n, J, 3)) * wl.sigma_vel
-    out = np.empty((13 * J, n), np.float32)
-    out[0:3 * J] = P.reshape(n, 3 * J).T
-    out[3 * J:7 * J] = Q.reshape(n, 4 * J).T
+    tau3 = torch.cat([tau - 0.5 * h, tau + 0.5 * h, tau])
+    p3, q3 = _t_analytic_pose(lib, cid.repeat(3), tau3)
+    noise = torch.randn((n, 9 * J + 3), generator=g, device=dev, dtype=torch.float64)
+    q3[2 * n:] = _t_qmul(q3[2 * n:], _t_qexp_half(noise[:, :3 * J].reshape(n, J, 3) * wl.sigma_q))
+    p3[2 * n:] += noise[:, 3 * J:3 * J + 3] * wl.sigma_root
+    P3, Q3 = _t_kinematics(skel, p3, q3)
+    lin = (P3[n:2 * n] - P3[:n]) / h + noise[:, 3 * J + 3:6 * J + 3].reshape(n, J, 3) * wl.sigma_vel
+    ang = _t_qlog_rotvec(_t_qmul(Q3[n:2 * n], Q3[:n] * Q3.new_tensor([1.0, -1.0, -1.0, -1.0]))) / h
+    ang = ang + noise[:, 6 * J + 3:].reshape(n, J, 3) * wl.sigma_vel
+    out = torch.empty((13 * J, n), dtype=torch.float32, device=dev)
+    out[0:3 * J] = P3[2 * n:].reshape(n, 3 * J).T
+    out[3 * J:7 * J] = Q3[2 * n:].reshape(n, 4 * J).T
     out[7 * J:10 * J] = lin.reshape(n, 3 * J).T
     out[10 * J:13 * J] = ang.reshape(n, 3 * J).T
     return out
+
+
+def synth_sim_state(skel: dict, lib: dict, clip_id: np.ndarray, t: np.ndarray, step: int,
+                    wl: Workload, seed: Optional[int] = None, env_base: int = 0) -> np.ndarray:
+    """numpy front end of synth_sim_state_torch (runs on the CPU)."""
+    import torch
+    out = synth_sim_state_torch(skel, lib, torch.from_numpy(np.ascontiguousarray(clip_id, np.int64)),
+                                torch.from_numpy(np.ascontiguousarray(t, np.float64)), step, wl, seed, env_base)
+    return out.numpy()
 
 
 def split_sim(sim: np.ndarray, J: int):
@@ -300,19 +384,23 @@ def build_scene(wl: Workload) -> Tuple[dict, dict, dict]:
 
 
 def rollout_inputs(wl: Workload, skel: dict, lib: dict,
-                   get_state: Callable[[], Tuple[np.ndarray, np.ndarray]],
-                   consume: Callable[[int, np.ndarray], None],
-                   steps: Optional[int] = None, env_base: int = 0) -> List[np.ndarray]:
+                   get_state: Callable[[], Tuple["np.ndarray", "np.ndarray"]],
+                   consume: Callable[[int, "object"], None],
+                   steps: Optional[int] = None, env_base: int = 0, device: str = "cpu") -> list:
     """Generate the per-step simulator states of a rollout.
 
-    Before step s the driver reports each env's (clip id, time); the simulator
-    stand-in produces the state one control interval later; the driver then
-    consumes it (which may reset some envs).  Returns the list of state arrays.
+    Before step s the driver reports each env's (clip id, time) as numpy arrays
+    or torch tensors; the simulator stand-in produces the state one control
+    interval later as a torch fp32 tensor [13J, n] on `device`; the driver then
+    consumes it (which may reset some envs).  Returns the list of state tensors.
     """
+    import torch
     sims = []
     for s in range(1, (wl.steps if steps is None else steps) + 1):
         cid, t = get_state()
-        sim = synth_sim_state(skel, lib, cid, t.astype(np.float64) + wl.dt, s, wl, env_base=env_base)
+        cid = torch.as_tensor(cid).to(device=device, dtype=torch.int64)
+        t = torch.as_tensor(t).to(device=device, dtype=torch.float64)
+        sim = synth_sim_state_torch(skel, lib, cid, t + wl.dt, s, wl, env_base=env_base)
         consume(s, sim)
         sims.append(sim)
     return sims

@@ -1,0 +1,234 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded inputs,
+through the C ABI.  Small cases span several 32-env tiles plus a ragged tail;
+full-size cases run the launch configuration the benchmark times."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2609_09821_b200 import binding as B
+from paper_2609_09821_b200 import workloads as W
+from tests.parity import Pair, Scene, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def scenes():
+    cache = {}
+
+    def get(name):
+        if name not in cache:
+            cache[name] = Scene(W.WORKLOADS[name])
+        return cache[name]
+    return get
+
+
+def test_library_is_loaded_and_launches_kernels(scenes):
+    before = B.launch_count()
+    p = Pair(scenes("cfg1_tiny64"), 64)
+    p.rollout(steps=1)
+    assert B.launch_count() >= before + 2 + 4
+
+
+# ---------------------------------------------------------------- the five configurations
+def test_cfg1_tiny_fp32_full(scenes):
+    p = Pair(scenes("cfg1_tiny64"), 64)
+    p.rollout()                                   # 10 steps, every env, fp32 policy
+
+
+@pytest.mark.parametrize("reward", [W.REWARD_FIG5, W.REWARD_ADD4], ids=["fig5", "add4"])
+def test_cfg1_additive_rewards(scenes, reward):
+    p = Pair(scenes("cfg1_tiny64"), 64, reward=reward, with_policy=False)
+    h = p.rollout(steps=4)
+    assert np.mean([x["reward"].mean() for x in h]) > 0.01      # not a vacuous all-zero comparison
+
+
+@pytest.mark.parametrize("n", [1, 31, 33, 77, 1000])
+def test_ragged_batches(scenes, n):
+    p = Pair(scenes("cfg2_4096"), n, policy_impl=1)
+    p.rollout(steps=3)
+
+
+def test_cfg2_reduced(scenes):
+    p = Pair(scenes("cfg2_4096"), 1024 + 17)
+    p.rollout(steps=6)
+
+
+def test_cfg3_library_reduced(scenes):
+    p = Pair(scenes("cfg3_16384_lib32"), 2048 + 5, with_policy=False)
+    h = p.rollout(steps=8)
+    assert len({int(c) for c in p.o_env.clip_id}) > 16            # many clips in play
+
+
+def test_cfg4_smpl_reduced(scenes):
+    p = Pair(scenes("cfg4_65536_smpl24"), 640 + 3)
+    p.rollout(steps=4)
+
+
+def test_cfg5_reset_heavy_reduced(scenes):
+    p = Pair(scenes("cfg5_reset_heavy"), 2048 + 9, write_back=True)
+    h = p.rollout(steps=10, policy_every=5)
+    rate = np.mean([(x["flags"] != 0).mean() for x in h])
+    assert 0.08 < rate < 0.4
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_other_seeds(scenes, seed):
+    wl = W.WORKLOADS["cfg3_16384_lib32"]
+    p = Pair(scenes("cfg3_16384_lib32"), 512, seed=seed, with_policy=False)
+    p.rollout(steps=4)
+
+
+@pytest.mark.parametrize("name", ["cfg2_4096", "cfg3_16384_lib32", "cfg4_65536_smpl24", "cfg5_reset_heavy"])
+def test_full_size(scenes, name):
+    """Full env count in the benchmark's launch configuration; every env's observation, reward,
+    flags and state against the oracle, the policy on a sample of envs."""
+    wl = W.WORKLOADS[name]
+    p = Pair(scenes(name), wl.n_envs, policy_sample=192, want_terms=False)
+    p.rollout(steps=3, device="cuda")
+
+
+# ---------------------------------------------------------------- edge cases
+def test_reward_threshold_termination(scenes):
+    """Figure 5's done rule: root height < 0.55 or reward < 0.15."""
+    p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.15, with_policy=False)
+    h = p.rollout(steps=5)
+    assert any((x["flags"] & 1).any() for x in h)
+
+
+def test_all_reset_and_none_reset(scenes):
+    for h_min in (10.0, -10.0):
+        p = Pair(scenes("cfg1_tiny64"), 64, h_min=h_min, with_policy=False, write_back=True)
+        h = p.rollout(steps=3)
+        assert all(((x["flags"] & 1) == (1 if h_min > 0 else 0)).all() for x in h)
+
+
+def test_min_ld_obs_and_padded_component_stride(scenes):
+    p = Pair(scenes("cfg1_tiny64"), 50, ld_obs=364, stride_pad=14, with_policy=False)
+    p.rollout(steps=3)
+
+
+def test_single_body_and_max_bodies():
+    for J in (1, 2, 32):
+        wl = W.Workload("edge_J%d" % J, 40, "custom", 2, (5, 9), 3, (24 * J + 1, 64, 8), "f32")
+        rng = np.random.default_rng(J)
+        parents = np.array([-1] + [int(rng.integers(max(0, j - 3), j)) for j in range(1, J)], np.int32)
+        if J == 32:
+            parents = np.arange(-1, 31, dtype=np.int32)           # one 32-link chain: deepest possible
+        offsets = rng.uniform(-0.3, 0.3, (J, 3)).astype(np.float32)
+        offsets[0] = 0
+        has_child = np.zeros(J, bool)
+        has_child[parents[1:]] = True
+        skel = dict(kind="custom", J=J, parents=parents, offsets=offsets,
+                    masses=rng.uniform(1, 3, J).astype(np.float32), ee_ids=np.nonzero(~has_child)[0].astype(np.int32))
+        lib = W.make_clip_library(J, 2, (5, 9), 30.0, seed=J)
+        pol = W.make_policy_weights(wl.mlp_dims, "f32", seed=J)
+        p = Pair(Scene(wl, skel, lib, pol), 40)
+        p.rollout(steps=3)
+
+
+def test_sharded_envs_reproduce_the_unsplit_batch(scenes):
+    sc = scenes("cfg5_reset_heavy")
+    whole = Pair(sc, 96, with_policy=True)
+    whole.reset_all()
+    obs_whole = whole.obs_g.clone()
+    parts = [Pair(sc, 48, env_base=0), Pair(sc, 48, env_base=48)]
+    for q in parts:
+        q.reset_all()
+    assert torch.equal(torch.cat([q.obs_g for q in parts]), obs_whole)
+    sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(whole.o_env.clip_id.astype(np.int64)),
+                                  torch.from_numpy(whole.o_env.t.astype(np.float64)) + sc.wl.dt, 1, sc.wl)
+    whole.policy_step(1)
+    whole.env_step(1, sim)
+    for k, q in enumerate(parts):
+        q.policy_step(1)
+        q.env_step(1, sim[:, 48 * k:48 * (k + 1)].contiguous())
+    assert torch.equal(torch.cat([q.obs_g for q in parts]), whole.obs_g)
+    assert torch.equal(torch.cat([q.action_g for q in parts]), whole.action_g)
+    assert torch.equal(torch.cat([q.flags_g for q in parts]), whole.flags_g)
+
+
+def test_deterministic_and_resumable(scenes):
+    sc = scenes("cfg5_reset_heavy")
+    a = Pair(sc, 300, with_policy=False)
+    hist = []
+    sims = []
+    a.reset_all()
+
+    def consume(s, sim):
+        sims.append(sim)
+        a.env_step(s, sim)
+        hist.append((a.obs_g.clone(), a.reward_g.clone(), a.flags_g.clone(), a.g_env.get_state()))
+
+    W.rollout_inputs(sc.wl, sc.skel, sc.lib, lambda: (a.o_env.clip_id, a.o_env.t), consume, steps=6)
+    # second env resumes at step 4 from the saved state and must reproduce steps 4..6 bit for bit
+    b = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(300, sc.wl.dt, sc.wl.seed, W.REWARD_MULT, sc.wl.h_min,
+                                                       a.ld_obs))
+    c, t, l = hist[2][3]
+    b.set_state(c, t, l)
+    obs = b.new_obs()
+    rew = torch.empty(300, device="cuda")
+    fl = torch.empty(300, dtype=torch.uint8, device="cuda")
+    for s in (4, 5, 6):
+        b.step(s, sims[s - 1].cuda(), obs, rew, fl)
+        torch.cuda.synchronize()
+        assert torch.equal(obs, hist[s - 1][0]) and torch.equal(rew, hist[s - 1][1]) and torch.equal(fl, hist[s - 1][2])
+
+
+def test_bad_simulated_quaternion_sets_status_not_a_fault(scenes):
+    sc = scenes("cfg1_tiny64")
+    p = Pair(sc, 64, with_policy=False)
+    p.reset_all()
+    sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                  torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, 1, sc.wl).cuda()
+    sim[3 * 15 + 4 * 3:3 * 15 + 4 * 3 + 4, 5] = 0.0            # body 3 of env 5: zero quaternion
+    sim[3 * 15 + 4 * 7, 9] = float("nan")
+    p.g_env.step(1, sim, p.obs_g, p.reward_g, p.flags_g, None)
+    assert p.g_env.device_status() & 1
+    ok = np.ones(64, bool)
+    ok[[5, 9]] = False
+    assert torch.isfinite(p.obs_g[torch.from_numpy(ok).cuda()]).all()
+    assert torch.isfinite(p.obs_g[5]).all()
+
+
+def test_host_buffer_step_matches_device_step(scenes):
+    sc = scenes("cfg2_4096")
+    n = 500
+    p = Pair(sc, n)
+    p.reset_all()
+    env2 = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, sc.wl.dt, sc.wl.seed, W.REWARD_MULT, sc.wl.h_min, p.ld_obs))
+    env2.reset_all_host(0)
+    act = torch.empty((n, p.A)).pin_memory()
+    rew = torch.empty(n).pin_memory()
+    fl = torch.empty(n, dtype=torch.uint8).pin_memory()
+    for s in (1, 2):
+        sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                      torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, s, sc.wl)
+        p.policy_step(s)
+        p.env_step(s, sim)
+        B.step_host(env2, p.policy, s, sim.contiguous().pin_memory(), act, rew, fl)
+        assert torch.equal(act, p.action_g.cpu()) and torch.equal(rew, p.reward_g.cpu()) and torch.equal(fl, p.flags_g.cpu())
+
+
+def test_reset_draws_bit_exact_over_many_counters(scenes):
+    sc = scenes("cfg3_16384_lib32")
+    n = 100000
+    p = Pair(sc, n, seed=0xDEADBEEFCAFE, with_policy=False)
+    p.o_env.reset_all(0)
+    obs = torch.empty((n, p.ld_obs), device="cuda")
+    p.g_env.reset_all(obs, 0)
+    p.check_state("100k resets")
+
+
+def test_invalid_arguments_are_rejected(scenes):
+    sc = scenes("cfg1_tiny64")
+    with pytest.raises(B.ImError):
+        B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, sc.wl.dt, 0, W.REWARD_MULT, 0.3, 360))     # ld_obs < D
+    with pytest.raises(B.ImError):
+        B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, 100.0, 0, W.REWARD_MULT, 0.3, 384))        # dt > clip
+    env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, sc.wl.dt, 0, W.REWARD_MULT, 0.3, 384))
+    obs = torch.empty((64, 384), device="cuda")
+    sim = torch.zeros((13 * 15, 60), device="cuda")                                                   # stride < N
+    with pytest.raises(B.ImError):
+        env.step(1, sim, obs, torch.empty(64, device="cuda"), torch.empty(64, dtype=torch.uint8, device="cuda"))

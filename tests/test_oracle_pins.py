@@ -421,6 +421,7 @@ def _rollout(name, n, steps, reward=W.REWARD_MULT, **cfg_kw):
 
     def consume(s, sim):
         before = (env.clip_id.copy(), env.t.copy(), env.ep_len.copy())
+        sim = sim.numpy()
         out = env.step(s, sim)
         hist.append(dict(before=before, after=(env.clip_id.copy(), env.t.copy(), env.ep_len.copy()),
                          sim=sim, **out))
