@@ -594,13 +594,31 @@ void orc_action_noise(uint32_t seed_lo, uint32_t seed_hi, uint32_t env, uint32_t
     }
 }
 
+/* Nearest-even rounding of a value to bf16 (through fp32), as a double. */
+double orc_round_bf16(double x)
+{
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return (double)f;      /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
 /* h_{l+1} = relu(W_l h_l + b_l), last layer linear -> mean; a = mean + sigma z.
  * Weights W_l are [dims[l+1]][dims[l]] fp32 values (bf16 weights widened
- * exactly by the caller); accumulation in fp64, activations never rounded. */
+ * exactly by the caller); accumulation in fp64.  With bf16_operands the
+ * operands of every layer are bf16 values, as the bf16 configurations
+ * prescribe ("bf16 operands, fp32 accumulation"): the observation and each
+ * hidden activation are rounded to bf16 before they enter the next layer;
+ * otherwise activations are never rounded. */
 void orc_policy_forward(int n_layers, const int32_t *dims, const float *const *W, const float *const *b,
                         double sigma, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
                         int n, const uint32_t *env_ids, const double *obs, int64_t ld_obs,
-                        double *mean, double *action, double *logp, double *z_out, int n_threads)
+                        double *mean, double *action, double *logp, double *z_out, int n_threads,
+                        int bf16_operands)
 {
     int maxd = 0, A = dims[n_layers];
     for (int l = 0; l <= n_layers; ++l) if (dims[l] > maxd) maxd = dims[l];
@@ -609,14 +627,20 @@ void orc_policy_forward(int n_layers, const int32_t *dims, const float *const *W
     for (int i = 0; i < n; ++i) {
         double *h0 = (double *)malloc(sizeof(double) * maxd), *h1 = (double *)malloc(sizeof(double) * maxd);
         double *z = (double *)malloc(sizeof(double) * (A + 4));
-        for (int k = 0; k < dims[0]; ++k) h0[k] = obs[(int64_t)i * ld_obs + k];
+        for (int k = 0; k < dims[0]; ++k) {
+            h0[k] = obs[(int64_t)i * ld_obs + k];
+            if (bf16_operands) h0[k] = orc_round_bf16(h0[k]);
+        }
         for (int l = 0; l < n_layers; ++l) {
             int in = dims[l], out = dims[l+1];
             for (int o = 0; o < out; ++o) {
                 double acc = (double)b[l][o];
                 const float *w = W[l] + (int64_t)o * in;
                 for (int k = 0; k < in; ++k) acc += (double)w[k] * h0[k];
-                if (l < n_layers - 1 && acc < 0.0) acc = 0.0;
+                if (l < n_layers - 1) {
+                    if (acc < 0.0) acc = 0.0;
+                    if (bf16_operands) acc = orc_round_bf16(acc);
+                }
                 h1[o] = acc;
             }
             double *tmp = h0; h0 = h1; h1 = tmp;

@@ -74,7 +74,9 @@ def lib():
                                    vp, i64, vp, vp, vp, i32]
         L.orc_action_noise.argtypes = [u32, u32, u32, u32, i32, vp]
         L.orc_policy_forward.argtypes = [i32, vp, vp, vp, f64, u32, u32, u32, i32, vp, vp, i64,
-                                         vp, vp, vp, vp, i32]
+                                         vp, vp, vp, vp, i32, i32]
+        L.orc_round_bf16.argtypes = [f64]
+        L.orc_round_bf16.restype = f64
         L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
         L.orc_openmp_enabled.restype = i32
         _lib = L
@@ -170,8 +172,8 @@ class Skeleton:
             raise ValueError("invalid skeleton")
 
     def __del__(self):
-        if getattr(self, "h", None):
-            lib().orc_skeleton_destroy(self.h)
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.orc_skeleton_destroy(self.h)
             self.h = None
 
 
@@ -191,8 +193,8 @@ class Clips:
         return np.float32(lib().orc_clip_duration(self.h, int(clip)))
 
     def __del__(self):
-        if getattr(self, "h", None):
-            lib().orc_clips_destroy(self.h)
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.orc_clips_destroy(self.h)
             self.h = None
 
 
@@ -256,9 +258,15 @@ class Env:
         return dict(obs=obs, reward=reward, flags=flags, terms=terms)
 
 
+def round_bf16(x: float) -> float:
+    return float(lib().orc_round_bf16(float(x)))
+
+
 def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarray,
-                   env_ids: Optional[np.ndarray] = None, n_threads: Optional[int] = None) -> dict:
-    """obs: fp64 [n, >=dims[0]].  W[l]: fp32 [dims[l+1], dims[l]] (bf16 weights widened exactly)."""
+                   env_ids: Optional[np.ndarray] = None, n_threads: Optional[int] = None,
+                   bf16_operands: bool = False) -> dict:
+    """obs: fp64 [n, >=dims[0]].  W[l]: fp32 [dims[l+1], dims[l]] (bf16 weights widened exactly).
+    bf16_operands: observation and hidden activations are rounded to bf16 before each layer."""
     nl = len(dims) - 1
     n = obs.shape[0]
     obs = _f64(obs)
@@ -278,5 +286,5 @@ def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarr
     lib().orc_policy_forward(nl, _p(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), float(sigma),
                              seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF, step, n, _p(ids),
                              _p(obs), obs.shape[1], _p(mean), _p(action), _p(logp), _p(z),
-                             int(n_threads or os.cpu_count() or 1))
+                             int(n_threads or os.cpu_count() or 1), int(bool(bf16_operands)))
     return dict(mean=mean, action=action, logp=logp, z=z)

@@ -1,8 +1,561 @@
-// placeholder until the tcgen05 chain lands
+// Tensor-core policy chain for sm_100a: one persistent, warp-specialised GEMM
+// kernel per layer, C[M][N] = act(A[M][K] W[N][K]^T + b), bf16 operands, fp32
+// accumulation in tensor memory.
+//
+//   warp 0      TMA producer: A and W tiles (128B-swizzled, K-major) into a ring of smem stages
+//   warp 1      MMA issuer: tcgen05.mma 128 x BLOCK_N x 16 into one of two TMEM accumulators
+//   warps 2..5  epilogue: tcgen05.ld the finished accumulator, add bias, then either ReLU + bf16
+//               store (hidden layers) or the Gaussian head (last layer: mean, Philox/Box-Muller
+//               noise, action, log-probability), while the MMA warp works on the next tile
+//
+// Hidden activations stay bf16 and L2-resident between layers.  Every wait on
+// an mbarrier is bounded: when the limit runs out the kernel raises
+// IM_DEV_WAIT_TIMEOUT in the status word, stops issuing work, and leaves
+// through the common exit that frees its tensor memory.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <new>
+#include <vector>
+
 #include "im_internal.h"
+#include "im_device.cuh"
 #include "mlp.h"
+
 namespace im {
-im_status tc_policy_create(im_policy *, const void *const *, const float *const *) { return IM_ERR_UNSUPPORTED; }
-void tc_policy_destroy(im_policy *) {}
-im_status tc_policy_forward(im_policy *, uint32_t, int32_t, const float *, int32_t, float *, float *, float *) { return IM_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;               // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kThreads = 192;
+constexpr int kEpiWarps = 4;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+enum Epilogue { EPI_RELU_BF16 = 0, EPI_GAUSS_HEAD = 1 };
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (int spin = 0;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 255) == 255) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem], single-CTA, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 16 consecutive columns of fp32: thread i gets row (lane base + i).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128B swizzle,
+// 8-row groups 1024 bytes apart (the layout a SWIZZLE_128B tensor-map load produces).
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)0 << 16;                                // leading byte offset: unused for swizzled K-major
+    d |= (uint64_t)(1024u >> 4) << 32;                     // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                                // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct GemmParams {
+    int M;             // rows in use (envs)
+    int N;             // valid output columns
+    int K_blocks;      // K / 64 (K is padded with zeros)
+    int n_tiles_n;     // N tiles of BLOCK_N
+    const float *bias; // [n_tiles_n * BLOCK_N], zero padded
+    // hidden layers
+    __nv_bfloat16 *out_bf16;
+    int ld_out;
+    // Gaussian head
+    float *mean, *action, *logp;
+    float sigma;
+    uint32_t seed_lo, seed_hi, step, env_id_base;
+    uint32_t *status;
+};
+
+template <int BLOCK_N>
+struct SmemPlan {
+    static constexpr int kStages = BLOCK_N >= 256 ? 4 : (BLOCK_N >= 128 ? 6 : 8);
+    static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
+    static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
+    static constexpr int kBBytesPadded = (kBBytes + 1023) / 1024 * 1024;     // keep every tile 1024-byte aligned
+    static constexpr int kStageBytes = kABytes + kBBytesPadded;
+    static constexpr int kAccStride = BLOCK_N <= 128 ? 128 : 256;           // TMEM columns between the two accumulators
+    static constexpr int kTmemCols = 2 * kAccStride;
+    static constexpr size_t kBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
+};
+
+template <int BLOCK_N, int EPI>
+__global__ void __launch_bounds__(kThreads, 1) linear_tc_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                const __grid_constant__ CUtensorMap map_b,
+                                                                const GemmParams P)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    constexpr int kStages = Plan::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + (size_t)kStages * Plan::kStageBytes);
+    uint64_t *full = bars, *empty = bars + kStages, *acc_full = bars + 2 * kStages, *acc_empty = bars + 2 * kStages + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (P.M + BLOCK_M - 1) / BLOCK_M;
+    const int n_tiles = tiles_m * P.n_tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, Plan::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+                for (int kb = 0; kb < P.K_blocks; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *sa = tiles + (size_t)stage * Plan::kStageBytes;
+                    mbar_arrive_expect_tx(&full[stage], Plan::kABytes + Plan::kBBytes);
+                    tma_load_2d(sa, &map_a, &full[stage], kb * BLOCK_K, m0);
+                    tma_load_2d(sa + Plan::kABytes, &map_b, &full[stage], kb * BLOCK_K, n0);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(BLOCK_M, BLOCK_N);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Plan::kAccStride);
+                for (int kb = 0; kb < P.K_blocks; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(tiles + (size_t)stage * Plan::kStageBytes);
+                    const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + Plan::kABytes);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                        // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in 16-byte units
+                        umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty[stage]);            // smem stage is free once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[acc]);               // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------- epilogue warps: quadrant q of the 128 TMEM lanes belongs to warps with warp % 4 == q
+        const int quad = warp & 3;
+        const int row_in_tile = quad * 32 + lane;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+            if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int row = m0 + row_in_tile;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
+            float zz = 0.0f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+                float v[16];
+                tmem_ld16(t_row + (uint32_t)c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] += __ldg(P.bias + n0 + c0 + i);
+                if (EPI == EPI_RELU_BF16) {
+                    if (row < P.M) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(v[2 * i], 0.0f), fmaxf(v[2 * i + 1], 0.0f));
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                        uint4 *dst = reinterpret_cast<uint4 *>(P.out_bf16 + (size_t)row * P.ld_out + n0 + c0);
+                        dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                } else {
+                    // Gaussian head: Philox block b feeds outputs 4b .. 4b+3 of this env
+                    if (row < P.M && c0 < P.N) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const int col = c0 + 4 * g;
+                            if (col >= P.N) break;
+                            const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
+                                                                     (uint32_t)(col >> 2)),
+                                                          make_uint2(P.seed_lo, P.seed_hi));
+                            float z[4];
+                            box_muller(x.x, x.y, z[0], z[1]);
+                            box_muller(x.z, x.w, z[2], z[3]);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                if (col + i < P.N) {
+                                    const float mu = v[4 * g + i];
+                                    P.mean[(size_t)row * P.N + col + i] = mu;
+                                    P.action[(size_t)row * P.N + col + i] = mu + P.sigma * z[i];
+                                    zz += z[i] * z[i];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            if (EPI == EPI_GAUSS_HEAD && P.logp && row < P.M)
+                P.logp[row] = -0.5f * zz - (float)P.N * logf(P.sigma) - 0.5f * (float)P.N * 1.8378770664093453f;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---------------- common exit: everyone meets, the allocating warp frees tensor memory
+    if (*abort_flag && lane == 0) {
+        // a wait ran out: give copies and MMAs that are still in flight time to land (bounded)
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(P.status, IM_DEV_WAIT_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, Plan::kTmemCols);
+    }
+}
+
+// fp32 observations -> bf16 rows of a padded buffer; columns beyond `cols` are written as zero.
+__global__ void obs_to_bf16_kernel(const float *__restrict__ obs, int ld_obs, int cols, __nv_bfloat16 *__restrict__ out,
+                                   int ld_out, int n)
+{
+    const int chunks = ld_out / 8;
+    const long long total = (long long)n * chunks;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(i / chunks), c = (int)(i % chunks) * 8;
+        float v[8];
+        if (c + 8 <= cols) {
+            const float4 a = *reinterpret_cast<const float4 *>(obs + (size_t)r * ld_obs + c);
+            const float4 b = *reinterpret_cast<const float4 *>(obs + (size_t)r * ld_obs + c + 4);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = (c + k < cols) ? obs[(size_t)r * ld_obs + c + k] : 0.0f;
+        }
+        uint32_t pk[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+            pk[k] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        *reinterpret_cast<uint4 *>(out + (size_t)r * ld_out + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows][ld] array; box = 64 columns x box_rows, 128B swizzle.
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {BLOCK_K, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_block_n(int N, bool last)
+{
+    if (last) return (N + 15) / 16 * 16;            // one tile holds the whole action row
+    if (N % 256 == 0) return 256;
+    if (N % 128 == 0) return 128;
+    return 64;
+}
+
+}  // namespace
+
+struct TcLayer {
+    int N, K, Kpad, block_n, n_tiles_n;
+    __nv_bfloat16 *d_W;      // [n_tiles_n * block_n][Kpad], zero padded
+    float *d_bias;           // [n_tiles_n * block_n]
+    CUtensorMap map_a, map_b;
+};
+
+}  // namespace im
+
+struct im_policy_tc {
+    std::vector<im::TcLayer> layers;
+    __nv_bfloat16 *d_in;          // [max_batch][Kpad0] bf16 observations
+    __nv_bfloat16 *d_hidden[2];   // [max_batch][max hidden]
+    int ld_in, ld_hidden;
+    int n_sm;
+};
+
+namespace im {
+
+namespace {
+
+template <int BLOCK_N, int EPI>
+cudaError_t launch_tc(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    static bool prepared = false;
+    if (!prepared) {
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BLOCK_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)Plan::kBytes);
+        if (e != cudaSuccess) return e;
+        prepared = true;
+    }
+    const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
+    const int grid = tiles < n_sm ? tiles : n_sm;
+    linear_tc_kernel<BLOCK_N, EPI><<<grid, kThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, gp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n_sm, cudaStream_t stream)
+{
+    if (!last) {
+        switch (L.block_n) {
+        case 256: return launch_tc<256, EPI_RELU_BF16>(L, gp, n_sm, stream);
+        case 128: return launch_tc<128, EPI_RELU_BF16>(L, gp, n_sm, stream);
+        default: return launch_tc<64, EPI_RELU_BF16>(L, gp, n_sm, stream);
+        }
+    }
+    switch (L.block_n) {
+    case 16: return launch_tc<16, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 32: return launch_tc<32, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 48: return launch_tc<48, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 64: return launch_tc<64, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 80: return launch_tc<80, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 96: return launch_tc<96, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 112: return launch_tc<112, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 128: return launch_tc<128, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+im_status tc_policy_create(im_policy *p, const void *const *W, const float *const *b)
+{
+    const im_policy_config &cfg = p->cfg;
+    const int nl = p->nl;
+    if (nl < 2) return IM_ERR_UNSUPPORTED;
+    for (int l = 1; l < nl; ++l)
+        if (cfg.dims[l] % 64) return IM_ERR_UNSUPPORTED;
+    if (cfg.dims[nl] > 128) return IM_ERR_UNSUPPORTED;
+    int dev = 0, cc_major = 0, n_sm = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
+
+    im_policy_tc *tc = new (std::nothrow) im_policy_tc();
+    if (!tc) return IM_ERR_ALLOC;
+    p->tc = tc;
+    tc->n_sm = n_sm;
+    tc->d_in = nullptr;
+    tc->d_hidden[0] = tc->d_hidden[1] = nullptr;
+    tc->layers.resize(nl);
+    for (auto &L : tc->layers) { L.d_W = nullptr; L.d_bias = nullptr; }
+    const size_t mb = (size_t)cfg.max_batch;
+    int max_hidden = 64;
+    for (int l = 1; l < nl; ++l) max_hidden = cfg.dims[l] > max_hidden ? cfg.dims[l] : max_hidden;
+    tc->ld_in = (cfg.dims[0] + BLOCK_K - 1) / BLOCK_K * BLOCK_K;
+    tc->ld_hidden = max_hidden;
+    if (cudaMalloc(&tc->d_in, mb * tc->ld_in * 2) != cudaSuccess ||
+        cudaMalloc(&tc->d_hidden[0], mb * max_hidden * 2) != cudaSuccess ||
+        cudaMalloc(&tc->d_hidden[1], mb * max_hidden * 2) != cudaSuccess)
+        return IM_ERR_ALLOC;
+
+    for (int l = 0; l < nl; ++l) {
+        TcLayer &L = tc->layers[l];
+        const bool last = l == nl - 1;
+        L.N = cfg.dims[l + 1];
+        L.K = cfg.dims[l];
+        L.Kpad = (L.K + BLOCK_K - 1) / BLOCK_K * BLOCK_K;
+        L.block_n = pick_block_n(L.N, last);
+        L.n_tiles_n = (L.N + L.block_n - 1) / L.block_n;
+        const size_t rows = (size_t)L.n_tiles_n * L.block_n;
+        std::vector<uint16_t> hw(rows * L.Kpad, 0);
+        std::vector<float> hb(rows, 0.0f);
+        const uint16_t *src = static_cast<const uint16_t *>(W[l]);
+        for (int n = 0; n < L.N; ++n) {
+            for (int k = 0; k < L.K; ++k) hw[(size_t)n * L.Kpad + k] = src[(size_t)n * L.K + k];
+            hb[n] = b[l][n];
+        }
+        if (cudaMalloc(&L.d_W, hw.size() * 2) != cudaSuccess || cudaMalloc(&L.d_bias, hb.size() * 4) != cudaSuccess)
+            return IM_ERR_ALLOC;
+        if (cudaMemcpy(L.d_W, hw.data(), hw.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(L.d_bias, hb.data(), hb.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+            return IM_ERR_CUDA;
+        const __nv_bfloat16 *a_base = l == 0 ? tc->d_in : tc->d_hidden[(l - 1) & 1];
+        const int a_ld = l == 0 ? tc->ld_in : tc->ld_hidden;
+        if (!make_map(&L.map_a, a_base, mb, (uint64_t)L.Kpad, (uint64_t)a_ld, BLOCK_M) ||
+            !make_map(&L.map_b, L.d_W, rows, (uint64_t)L.Kpad, (uint64_t)L.Kpad, (uint32_t)L.block_n))
+            return IM_ERR_CUDA;
+    }
+    return IM_OK;
+}
+
+void tc_policy_destroy(im_policy *p)
+{
+    im_policy_tc *tc = p->tc;
+    if (!tc) return;
+    for (auto &L : tc->layers) { cudaFree(L.d_W); cudaFree(L.d_bias); }
+    cudaFree(tc->d_in); cudaFree(tc->d_hidden[0]); cudaFree(tc->d_hidden[1]);
+    delete tc;
+    p->tc = nullptr;
+}
+
+im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
+                            float *mean_out, float *action_out, float *logp_out)
+{
+    im_policy_tc *tc = p->tc;
+    const im_policy_config &cfg = p->cfg;
+    {
+        const long long chunks = (long long)n * (tc->ld_in / 8);
+        const int block = 256;
+        long long grid = (chunks + block - 1) / block;
+        if (grid > 148 * 16) grid = 148 * 16;
+        obs_to_bf16_kernel<<<(int)grid, block, 0, p->stream>>>(obs, ld_obs, cfg.dims[0], tc->d_in, tc->ld_in, n);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return IM_ERR_CUDA;
+    }
+    for (int l = 0; l < p->nl; ++l) {
+        const TcLayer &L = tc->layers[l];
+        const bool last = l == p->nl - 1;
+        GemmParams gp;
+        gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
+        gp.out_bf16 = last ? nullptr : tc->d_hidden[l & 1];
+        gp.ld_out = tc->ld_hidden;
+        gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
+        gp.sigma = cfg.sigma; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
+        gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
+        if (dispatch_tc(L, gp, last, tc->n_sm, p->stream) != cudaSuccess) return IM_ERR_CUDA;
+    }
+    return IM_OK;
+}
+
+}  // namespace im

@@ -4,8 +4,13 @@ library on the same seeded inputs and compares them element by element.
 Tolerances (fp32 path vs fp64 oracle): observations, rewards and error terms
 |g - o| <= 1e-5 + 1e-4 |o|; flags, clip ids, time bit patterns and episode
 lengths exact; policy means |g - o| <= tol (|o| + rms of that output over the
-batch) with tol 2e-2 for bf16 operands and 1e-4 for fp32; action noise
-(action - mean) |g - o| <= 1e-5 + 1e-4 |o|.
+batch) with tol 1e-4 for the fp32 policy and 2e-2 for the bf16 policy, where
+the oracle takes the same operand precision (observation and hidden
+activations rounded to bf16, exact accumulation); against the oracle with
+unrounded activations the bf16 policy must have 99.9 % of its means within
+2e-2 and all within 6e-2 (operand rounding alone reaches 2.5e-2 on rare
+envs with large activations); action noise (action - mean) |g - o| <= 1e-5 +
+1e-4 |o|.
 """
 from __future__ import annotations
 
@@ -65,7 +70,7 @@ class Pair:
 
     def __init__(self, scene: Scene, n: int, reward=W.REWARD_MULT, seed=None, h_min=None, r_min=-np.inf,
                  write_back=False, env_base=0, ld_obs=None, stride_pad=0, with_policy=True, policy_impl=0,
-                 policy_sample=None, want_terms=True):
+                 policy_sample=None, want_terms=True, obs_atol=OBS_ATOL):
         wl = scene.wl
         self.scene, self.wl, self.n, self.J = scene, wl, n, scene.J
         self.seed = wl.seed if seed is None else seed
@@ -73,7 +78,8 @@ class Pair:
         self.r_min = r_min
         self.D = 24 * self.J + 1
         self.ld_obs = ld_obs or B.padded_ld(self.D)
-        self.stride = n + stride_pad
+        self.stride = (n + stride_pad + 3) // 4 * 4        # rows of the body-state arrays stay 16-byte aligned
+        self.obs_atol = obs_atol
         self.write_back = write_back
         self.want_terms = want_terms
         ids = np.arange(env_base, env_base + n, dtype=np.uint32)
@@ -113,7 +119,7 @@ class Pair:
 
     def check_obs(self, what):
         g = self.obs_g.cpu().numpy()
-        assert_close(g[:, :self.D], self.obs_o, what=what + " obs")
+        assert_close(g[:, :self.D], self.obs_o, atol=self.obs_atol, what=what + " obs")
         assert np.all(g[:, self.D:] == 0.0), what + " obs padding must be zero"
         self.max_err["obs"] = max(self.max_err["obs"], float(np.abs(g[:, :self.D] - self.obs_o).max()))
 
@@ -128,11 +134,20 @@ class Pair:
         pol = self.scene.pol
         self.policy.forward(s, self.obs_g, self.mean_g, self.action_g, self.logp_g)
         idx = self.sample
+        bf16 = pol["dtype"] == "bf16"
         o = O.policy_forward(pol["dims"], pol["W"], pol["b"], self.wl.sigma_action, self.seed, s,
-                             self.obs_o[idx], env_ids=self.ids[idx])
+                             self.obs_o[idx], env_ids=self.ids[idx], bf16_operands=bf16)
         mg = self.mean_g.cpu().numpy()[idx]
         ag = self.action_g.cpu().numpy()[idx]
         assert_mean_close(mg, o["mean"], self.mean_tol, what="step %d" % s)
+        if bf16:
+            plain = O.policy_forward(pol["dims"], pol["W"], pol["b"], self.wl.sigma_action, self.seed, s,
+                                     self.obs_o[idx], env_ids=self.ids[idx])["mean"]
+            rms = np.sqrt(np.mean(np.square(plain), axis=0, keepdims=True))
+            rel = np.abs(mg - plain) / (np.abs(plain) + rms)
+            assert np.mean(rel <= 2e-2) >= 0.999 and rel.max() <= 6e-2, \
+                "step %d: vs unrounded oracle: %.4f within 2e-2, max %.3g" % (s, np.mean(rel <= 2e-2), rel.max())
+            self.max_err["mean_vs_plain"] = max(self.max_err.get("mean_vs_plain", 0.0), float(rel.max()))
         noise_o = self.wl.sigma_action * o["z"]
         assert_close(ag.astype(np.float64) - mg.astype(np.float64), noise_o, atol=1e-5, rtol=1e-4,
                      what="step %d action noise" % s)
@@ -169,7 +184,7 @@ class Pair:
         self.check_state(what)
         self.check_obs(what)
         if self.write_back:
-            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, what=what + " written-back states")
+            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, atol=self.obs_atol, what=what + " written-back states")
         assert self.g_env.device_status() == 0
         self.max_err["reward"] = max(self.max_err["reward"], float(np.abs(rg - o["reward"]).max()))
         return dict(oracle=o, flags=fg, reward=rg)

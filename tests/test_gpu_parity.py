@@ -91,10 +91,12 @@ def test_full_size(scenes, name):
 
 # ---------------------------------------------------------------- edge cases
 def test_reward_threshold_termination(scenes):
-    """Figure 5's done rule: root height < 0.55 or reward < 0.15."""
-    p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.15, with_policy=False)
+    """Figure 5's done rule (root height or reward below a threshold); the reward threshold is set
+    near the median reward of this workload so that both outcomes occur."""
+    p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.74, with_policy=False)
     h = p.rollout(steps=5)
-    assert any((x["flags"] & 1).any() for x in h)
+    frac = np.mean([(x["flags"] & 1).mean() for x in h])
+    assert 0.05 < frac < 0.95
 
 
 def test_all_reset_and_none_reset(scenes):
@@ -124,7 +126,9 @@ def test_single_body_and_max_bodies():
                     masses=rng.uniform(1, 3, J).astype(np.float32), ee_ids=np.nonzero(~has_child)[0].astype(np.int32))
         lib = W.make_clip_library(J, 2, (5, 9), 30.0, seed=J)
         pol = W.make_policy_weights(wl.mlp_dims, "f32", seed=J)
-        p = Pair(Scene(wl, skel, lib, pol), 40)
+        # fp32 rounding of the propagated velocities grows linearly with the chain depth: a 32-link
+        # chain at these joint speeds (|w| up to ~30 rad/s) is allowed 31 * 2^-24 * 30 * 4 ~ 2e-4
+        p = Pair(Scene(wl, skel, lib, pol), 40, obs_atol=2e-4 if J == 32 else 1e-5)
         p.rollout(steps=3)
 
 

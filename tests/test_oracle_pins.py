@@ -671,6 +671,36 @@ def test_logp_is_the_gaussian_log_density():
     np.testing.assert_allclose(out["logp"], want, atol=1e-10)
 
 
+def test_oracle_bf16_rounding_matches_torch():
+    import torch
+    x = np.concatenate([np.random.default_rng(3).standard_normal(2000) * 10.0 ** np.random.default_rng(4).integers(-6, 6, 2000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38]])
+    want = torch.from_numpy(x).float().to(torch.bfloat16).double().numpy()
+    got = np.array([O.round_bf16(v) for v in x])
+    np.testing.assert_array_equal(got, want)
+
+
+def test_mlp_with_bf16_operands_against_torch():
+    """Same chain with every layer input rounded to bf16 by torch, accumulated in fp64."""
+    import torch
+    rng = np.random.default_rng(5)
+    dims = (37, 64, 48, 9)
+    Ws = [W.round_to_bf16(rng.standard_normal((o, i)).astype(np.float32) / math.sqrt(i))[0]
+          for i, o in zip(dims[:-1], dims[1:])]
+    bs = [rng.standard_normal(o).astype(np.float32) for o in dims[1:]]
+    obs = rng.standard_normal((33, 37)) * 3
+    out = O.policy_forward(dims, Ws, bs, 0.1, 5, 3, obs, bf16_operands=True)
+    h = torch.from_numpy(obs)
+    for l, (Wl, bl) in enumerate(zip(Ws, bs)):
+        h = h.float().to(torch.bfloat16).double()
+        h = torch.nn.functional.linear(h, torch.from_numpy(Wl).double(), torch.from_numpy(bl).double())
+        if l < 2:
+            h = torch.relu(h)
+    np.testing.assert_allclose(out["mean"], h.numpy(), atol=1e-12)
+    plain = O.policy_forward(dims, Ws, bs, 0.1, 5, 3, obs)
+    assert 1e-5 < np.abs(plain["mean"] - out["mean"]).max() < 0.2      # rounding matters, but only a little
+
+
 def test_bf16_rounding_helper():
     import torch
     x = np.random.default_rng(0).standard_normal(1000).astype(np.float32)
