@@ -22,14 +22,23 @@ from paper_2609_09821_b200 import binding as B
 from paper_2609_09821_b200 import workloads as W
 
 OBS_ATOL, OBS_RTOL = 1e-5, 1e-4
+# fp32 slack of velocity-derived entries.  A body's world velocity is a sum of up to depth+1
+# rotated joint velocities; in fp32 each rotated term and each partial sum carries a rounding
+# error of a few ulp of ITS magnitude, whatever the (possibly cancelled) result is.  With S the
+# largest velocity entry of the env's observation, those entries are allowed an extra
+# 2^-20 S (16 ulp-units of S; 1.9e-5 at S = 20 rad/s).  Positions, orientations, phase,
+# targets and the reward keep the plain tolerance.
+VEL_SLACK = 2.0 ** -20
 
 
-def assert_close(got, want, atol=OBS_ATOL, rtol=OBS_RTOL, what=""):
+def assert_close(got, want, atol=OBS_ATOL, rtol=OBS_RTOL, what="", slack=None):
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape, (what, got.shape, want.shape)
     err = np.abs(got - want)
     lim = atol + rtol * np.abs(want)
+    if slack is not None:
+        lim = lim + slack
     bad = ~(err <= lim)                   # NaN counts as bad
     if bad.any():
         i = np.unravel_index(np.argmax(np.where(bad, err - lim, -np.inf)), err.shape)
@@ -105,7 +114,9 @@ class Pair:
             self.logp_g = torch.empty(n, device="cuda")
             self.sample = np.arange(n) if policy_sample is None or policy_sample >= n else \
                 np.sort(np.random.default_rng(1).choice(n, policy_sample, replace=False))
-            self.mean_tol = 2e-2 if pol["dtype"] == "bf16" else 1e-4
+            # the SIMT cross-check path keeps fp32 activations even with bf16 weights
+            self.bf16_ops = pol["dtype"] == "bf16" and policy_impl == 0
+            self.mean_tol = 2e-2 if self.bf16_ops else 1e-4
         self.obs_o = None
         self.max_err = dict(obs=0.0, reward=0.0)
 
@@ -117,9 +128,17 @@ class Pair:
                                       err_msg=what + " time bit patterns")
         np.testing.assert_array_equal(l.cpu().numpy(), self.o_env.ep_len, err_msg=what + " episode lengths")
 
+    def vel_scale(self):
+        """Largest velocity entry of each env's (oracle) observation."""
+        body = self.obs_o[:, :15 * self.J].reshape(self.n, self.J, 15)
+        return np.abs(body[:, :, 9:15]).max(axis=(1, 2))
+
     def check_obs(self, what):
         g = self.obs_g.cpu().numpy()
-        assert_close(g[:, :self.D], self.obs_o, atol=self.obs_atol, what=what + " obs")
+        slack = np.zeros((self.n, self.J, 15))
+        slack[:, :, 9:15] = (VEL_SLACK * self.vel_scale())[:, None, None]
+        slack = np.concatenate([slack.reshape(self.n, -1), np.zeros((self.n, self.D - 15 * self.J))], axis=1)
+        assert_close(g[:, :self.D], self.obs_o, atol=self.obs_atol, what=what + " obs", slack=slack)
         assert np.all(g[:, self.D:] == 0.0), what + " obs padding must be zero"
         self.max_err["obs"] = max(self.max_err["obs"], float(np.abs(g[:, :self.D] - self.obs_o).max()))
 
@@ -134,7 +153,7 @@ class Pair:
         pol = self.scene.pol
         self.policy.forward(s, self.obs_g, self.mean_g, self.action_g, self.logp_g)
         idx = self.sample
-        bf16 = pol["dtype"] == "bf16"
+        bf16 = self.bf16_ops
         o = O.policy_forward(pol["dims"], pol["W"], pol["b"], self.wl.sigma_action, self.seed, s,
                              self.obs_o[idx], env_ids=self.ids[idx], bf16_operands=bf16)
         mg = self.mean_g.cpu().numpy()[idx]
@@ -145,7 +164,8 @@ class Pair:
                                      self.obs_o[idx], env_ids=self.ids[idx])["mean"]
             rms = np.sqrt(np.mean(np.square(plain), axis=0, keepdims=True))
             rel = np.abs(mg - plain) / (np.abs(plain) + rms)
-            assert np.mean(rel <= 2e-2) >= 0.999 and rel.max() <= 6e-2, \
+            frac_ok = np.mean(rel <= 2e-2) >= 0.999 or len(idx) < 64      # a fraction needs a population
+            assert frac_ok and rel.max() <= 6e-2, \
                 "step %d: vs unrounded oracle: %.4f within 2e-2, max %.3g" % (s, np.mean(rel <= 2e-2), rel.max())
             self.max_err["mean_vs_plain"] = max(self.max_err.get("mean_vs_plain", 0.0), float(rel.max()))
         noise_o = self.wl.sigma_action * o["z"]
@@ -162,6 +182,7 @@ class Pair:
         sim_g[:, :self.n] = sim.to("cuda")
         if self.stride > self.n:
             sim_g[:, self.n:] = float("nan")
+        sim_vel_scale = np.abs(sim_np[7 * self.J:]).max(axis=0)      # largest simulated velocity per env
         o = self.o_env.step(s, sim_np, want_terms=self.want_terms)
         self.g_env.step(s, sim_g, self.obs_g, self.reward_g, self.flags_g, self.terms_g)
         self.obs_o = o["obs"]
@@ -180,11 +201,18 @@ class Pair:
             np.testing.assert_array_equal(fg, o["flags"], err_msg=what + " flags")
         assert_close(rg, o["reward"], what=what + " reward")
         if self.want_terms:
-            assert_close(self.terms_g.cpu().numpy(), o["terms"], what=what + " error terms")
+            # d(sum of squares) = 2 sqrt(J e) d(velocity) for the two velocity terms
+            slack = np.zeros_like(o["terms"])
+            for k in (1, 6):
+                slack[k] = 2.0 * np.sqrt(self.J * o["terms"][k]) * VEL_SLACK * sim_vel_scale
+            assert_close(self.terms_g.cpu().numpy(), o["terms"], what=what + " error terms", slack=slack)
         self.check_state(what)
         self.check_obs(what)
         if self.write_back:
-            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, atol=self.obs_atol, what=what + " written-back states")
+            wb_slack = np.zeros_like(sim_np, dtype=np.float64)
+            wb_slack[7 * self.J:] = VEL_SLACK * np.abs(sim_np[7 * self.J:]).max(axis=0)
+            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, atol=self.obs_atol, slack=wb_slack,
+                         what=what + " written-back states")
         assert self.g_env.device_status() == 0
         self.max_err["reward"] = max(self.max_err["reward"], float(np.abs(rg - o["reward"]).max()))
         return dict(oracle=o, flags=fg, reward=rg)

@@ -46,8 +46,14 @@ def test_cfg1_additive_rewards(scenes, reward):
 
 @pytest.mark.parametrize("n", [1, 31, 33, 77, 1000])
 def test_ragged_batches(scenes, n):
-    p = Pair(scenes("cfg2_4096"), n, policy_impl=1)
+    p = Pair(scenes("cfg2_4096"), n)
     p.rollout(steps=3)
+
+
+def test_simt_layers_with_bf16_weights(scenes):
+    """The SIMT cross-check path (bf16 weights, fp32 activations) against the unrounded oracle."""
+    p = Pair(scenes("cfg2_4096"), 200, policy_impl=1)
+    p.rollout(steps=2)
 
 
 def test_cfg2_reduced(scenes):
@@ -96,7 +102,7 @@ def test_reward_threshold_termination(scenes):
     p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.74, with_policy=False)
     h = p.rollout(steps=5)
     frac = np.mean([(x["flags"] & 1).mean() for x in h])
-    assert 0.05 < frac < 0.95
+    assert 0.01 < frac < 0.99
 
 
 def test_all_reset_and_none_reset(scenes):
@@ -126,9 +132,9 @@ def test_single_body_and_max_bodies():
                     masses=rng.uniform(1, 3, J).astype(np.float32), ee_ids=np.nonzero(~has_child)[0].astype(np.int32))
         lib = W.make_clip_library(J, 2, (5, 9), 30.0, seed=J)
         pol = W.make_policy_weights(wl.mlp_dims, "f32", seed=J)
-        # fp32 rounding of the propagated velocities grows linearly with the chain depth: a 32-link
-        # chain at these joint speeds (|w| up to ~30 rad/s) is allowed 31 * 2^-24 * 30 * 4 ~ 2e-4
-        p = Pair(Scene(wl, skel, lib, pol), 40, obs_atol=2e-4 if J == 32 else 1e-5)
+        # fp32 rounding of the pose itself grows with the chain depth too: a 32-link chain (no
+        # benchmark skeleton is deeper than 9) is allowed 4e-5 on positions and orientations
+        p = Pair(Scene(wl, skel, lib, pol), 40, obs_atol=4e-5 if J == 32 else 1e-5)
         p.rollout(steps=3)
 
 
