@@ -33,7 +33,6 @@ constexpr int kThreads = 192;
 constexpr int kEpiWarps = 4;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
-enum Epilogue { EPI_RELU_BF16 = 0, EPI_GAUSS_HEAD = 1 };
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -120,6 +119,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 32 columns, issue only; pair with tmem_ld_wait() before the values are used.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, float *v)
+{
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128B swizzle,
 // 8-row groups 1024 bytes apart (the layout a SWIZZLE_128B tensor-map load produces).
 __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr)
@@ -144,9 +158,6 @@ struct GemmParams {
     int K_blocks;      // K / 64 (K is padded with zeros)
     int n_tiles_n;     // N tiles of BLOCK_N
     const float *bias; // [n_tiles_n * BLOCK_N], zero padded
-    // hidden layers
-    __nv_bfloat16 *out_bf16;
-    int ld_out;
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
@@ -154,175 +165,299 @@ struct GemmParams {
     uint32_t *status;
 };
 
+constexpr int kEpiSlabBytes = 32 * 128;    // one epilogue warp's 32 rows x 64 bf16 staging slab
+
 template <int BLOCK_N>
 struct SmemPlan {
-    static constexpr int kStages = BLOCK_N >= 256 ? 4 : (BLOCK_N >= 128 ? 6 : 8);
+    static constexpr int kStages = BLOCK_N >= 256 ? 4 : 6;
     static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
     static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
     static constexpr int kBBytesPadded = (kBBytes + 1023) / 1024 * 1024;     // keep every tile 1024-byte aligned
     static constexpr int kStageBytes = kABytes + kBBytesPadded;
     static constexpr int kAccStride = BLOCK_N <= 128 ? 128 : 256;           // TMEM columns between the two accumulators
     static constexpr int kTmemCols = 2 * kAccStride;
-    static constexpr size_t kBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
+    static constexpr int kEpiBytes = 4 * kEpiSlabBytes;                     // hidden layers: staging for the TMA stores
+    static constexpr int kHeadBytes = 2 * 4 * 128 * 4 + 2 * 128 * 4;        // head: partial sums of z^2 and arrival counters
+    static constexpr int kBarBytes = 256;
+    static constexpr size_t kBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + kEpiBytes + kHeadBytes + kBarBytes;
 };
 
-template <int BLOCK_N, int EPI>
-__global__ void __launch_bounds__(kThreads, 1) linear_tc_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                                const __grid_constant__ CUtensorMap map_b,
-                                                                const GemmParams P)
+struct Pipe {
+    uint8_t *tiles;
+    uint64_t *full, *empty, *acc_full, *acc_empty;
+    uint32_t *tmem_slot;
+    volatile int *abort_flag;
+    uint8_t *epi;
+};
+
+template <class Plan>
+__device__ __forceinline__ Pipe carve_pipe(uint8_t *smem_raw)
 {
-    using Plan = SmemPlan<BLOCK_N>;
-    constexpr int kStages = Plan::kStages;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tiles + (size_t)kStages * Plan::kStageBytes);
-    uint64_t *full = bars, *empty = bars + kStages, *acc_full = bars + 2 * kStages, *acc_empty = bars + 2 * kStages + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 4);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    Pipe p;
+    p.tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    p.epi = p.tiles + (size_t)Plan::kStages * Plan::kStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(p.epi + Plan::kEpiBytes + Plan::kHeadBytes);
+    p.full = bars;
+    p.empty = bars + Plan::kStages;
+    p.acc_full = bars + 2 * Plan::kStages;
+    p.acc_empty = bars + 2 * Plan::kStages + 2;
+    p.tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Plan::kStages + 4);
+    p.abort_flag = reinterpret_cast<volatile int *>(p.tmem_slot + 1);
+    return p;
+}
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (P.M + BLOCK_M - 1) / BLOCK_M;
-    const int n_tiles = tiles_m * P.n_tiles_n;
-
+template <class Plan>
+__device__ __forceinline__ void pipe_init(const Pipe &p, int epi_arrivals)
+{
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
-        *abort_flag = 0;
+        for (int s = 0; s < Plan::kStages; ++s) { mbar_init(&p.full[s], 1); mbar_init(&p.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&p.acc_full[a], 1); mbar_init(&p.acc_empty[a], epi_arrivals); }
+        *p.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(tmem_slot, Plan::kTmemCols);
+    if ((threadIdx.x >> 5) == 1) tmem_alloc(p.tmem_slot, Plan::kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+}
 
-    if (warp == 0) {
-        // ---------------- TMA producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
-                for (int kb = 0; kb < P.K_blocks; ++kb) {
-                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
-                    uint8_t *sa = tiles + (size_t)stage * Plan::kStageBytes;
-                    mbar_arrive_expect_tx(&full[stage], Plan::kABytes + Plan::kBBytes);
-                    tma_load_2d(sa, &map_a, &full[stage], kb * BLOCK_K, m0);
-                    tma_load_2d(sa + Plan::kABytes, &map_b, &full[stage], kb * BLOCK_K, n0);
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(BLOCK_M, BLOCK_N);
-            int stage = 0, acc = 0;
-            uint32_t phase = 0, acc_phase = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Plan::kAccStride);
-                for (int kb = 0; kb < P.K_blocks; ++kb) {
-                    if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sa = smem_u32(tiles + (size_t)stage * Plan::kStageBytes);
-                    const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + Plan::kABytes);
-#pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                        // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in 16-byte units
-                        umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    umma_commit(&empty[stage]);            // smem stage is free once these MMAs have read it
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                }
-                if (!ok) break;
-                umma_commit(&acc_full[acc]);               // accumulator complete
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-            }
-        }
-    } else {
-        // ---------------- epilogue warps: quadrant q of the 128 TMEM lanes belongs to warps with warp % 4 == q
-        const int quad = warp & 3;
-        const int row_in_tile = quad * 32 + lane;
-        int acc = 0;
-        uint32_t acc_phase = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
-            if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const int row = m0 + row_in_tile;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
-            float zz = 0.0f;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
-                float v[16];
-                tmem_ld16(t_row + (uint32_t)c0, v);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] += __ldg(P.bias + n0 + c0 + i);
-                if (EPI == EPI_RELU_BF16) {
-                    if (row < P.M) {
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(v[2 * i], 0.0f), fmaxf(v[2 * i + 1], 0.0f));
-                            pk[i] = *reinterpret_cast<const uint32_t *>(&h);
-                        }
-                        uint4 *dst = reinterpret_cast<uint4 *>(P.out_bf16 + (size_t)row * P.ld_out + n0 + c0);
-                        dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                    }
-                } else {
-                    // Gaussian head: Philox block b feeds outputs 4b .. 4b+3 of this env
-                    if (row < P.M && c0 < P.N) {
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            const int col = c0 + 4 * g;
-                            if (col >= P.N) break;
-                            const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
-                                                                     (uint32_t)(col >> 2)),
-                                                          make_uint2(P.seed_lo, P.seed_hi));
-                            float z[4];
-                            box_muller(x.x, x.y, z[0], z[1]);
-                            box_muller(x.z, x.w, z[2], z[3]);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                if (col + i < P.N) {
-                                    const float mu = v[4 * g + i];
-                                    P.mean[(size_t)row * P.N + col + i] = mu;
-                                    P.action[(size_t)row * P.N + col + i] = mu + P.sigma * z[i];
-                                    zz += z[i] * z[i];
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-            if (EPI == EPI_GAUSS_HEAD && P.logp && row < P.M)
-                P.logp[row] = -0.5f * zz - (float)P.N * logf(P.sigma) - 0.5f * (float)P.N * 1.8378770664093453f;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[acc]);
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        }
-    }
-
-    // ---------------- common exit: everyone meets, the allocating warp frees tensor memory
-    if (*abort_flag && lane == 0) {
+// Common exit: everyone meets, the allocating warp frees tensor memory.
+template <class Plan>
+__device__ __forceinline__ void pipe_exit(const Pipe &p, uint32_t tmem_base, uint32_t *status)
+{
+    if (*p.abort_flag && (threadIdx.x & 31) == 0) {
         // a wait ran out: give copies and MMAs that are still in flight time to land (bounded)
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) { }
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0 && *abort_flag) atomicOr(P.status, IM_DEV_WAIT_TIMEOUT);
-    if (warp == 1) {
+    if (threadIdx.x == 0 && *p.abort_flag) atomicOr(status, IM_DEV_WAIT_TIMEOUT);
+    if ((threadIdx.x >> 5) == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, Plan::kTmemCols);
     }
+}
+
+// TMA producer (one thread): A and W tiles of every k-block of every tile of this CTA.
+template <class Plan, int BLOCK_N>
+__device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *map_a, const CUtensorMap *map_b,
+                                              const GemmParams &P, int n_tiles)
+{
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+        for (int kb = 0; kb < P.K_blocks; ++kb) {
+            if (!mbar_wait(&p.empty[stage], phase ^ 1u, p.abort_flag)) return;
+            uint8_t *sa = p.tiles + (size_t)stage * Plan::kStageBytes;
+            mbar_arrive_expect_tx(&p.full[stage], Plan::kABytes + Plan::kBBytes);
+            tma_load_2d(sa, map_a, &p.full[stage], kb * BLOCK_K, m0);
+            tma_load_2d(sa + Plan::kABytes, map_b, &p.full[stage], kb * BLOCK_K, n0);
+            if (++stage == Plan::kStages) { stage = 0; phase ^= 1u; }
+        }
+    }
+}
+
+// MMA issuer (one thread).
+template <class Plan, int BLOCK_N>
+__device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, const GemmParams &P, int n_tiles)
+{
+    constexpr uint32_t idesc = instr_desc_bf16(BLOCK_M, BLOCK_N);
+    int stage = 0, acc = 0;
+    uint32_t phase = 0, acc_phase = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        if (!mbar_wait(&p.acc_empty[acc], acc_phase ^ 1u, p.abort_flag)) return;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Plan::kAccStride);
+        for (int kb = 0; kb < P.K_blocks; ++kb) {
+            if (!mbar_wait(&p.full[stage], phase, p.abort_flag)) return;
+            tc_fence_after();
+            const uint32_t sa = smem_u32(p.tiles + (size_t)stage * Plan::kStageBytes);
+            const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + Plan::kABytes);
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in 16-byte units
+                umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(&p.empty[stage]);            // smem stage is free once these MMAs have read it
+            if (++stage == Plan::kStages) { stage = 0; phase ^= 1u; }
+        }
+        umma_commit(&p.acc_full[acc]);               // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+}
+
+// ------------------------------------------------------------------ hidden layers
+// C = relu(A W^T + b) as bf16.  Each epilogue warp owns 32 rows of the tile: it
+// reads 64 accumulator columns at a time, applies bias and ReLU, packs to bf16
+// into a 128B-swizzled slab in shared memory and hands the slab to a TMA store.
+template <int BLOCK_N>
+__global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                       const __grid_constant__ CUtensorMap map_b,
+                                                                       const __grid_constant__ CUtensorMap map_c,
+                                                                       const GemmParams P)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    extern __shared__ uint8_t smem_raw[];
+    const Pipe p = carve_pipe<Plan>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
+    pipe_init<Plan>(p, kEpiWarps);
+    const uint32_t tmem_base = *p.tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) producer_role<Plan, BLOCK_N>(p, &map_a, &map_b, P, n_tiles);
+    } else if (warp == 1) {
+        if (lane == 0) mma_role<Plan, BLOCK_N>(p, tmem_base, P, n_tiles);
+    } else {
+        const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+        uint8_t *slab = p.epi + (size_t)(warp - 2) * kEpiSlabBytes;
+        const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+            if (!mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag)) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 64) {
+                float v[64];
+                tmem_ld32_issue(t_row + (uint32_t)c0, v);
+                tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
+                tmem_ld_wait();
+                const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float4 b = __ldg(b4 + i);
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, 0.0f), fmaxf(v[4 * i + 1] + b.y, 0.0f));
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, 0.0f), fmaxf(v[4 * i + 3] + b.w, 0.0f));
+                    pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
+                    pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+                }
+                // the previous slab's store must have finished reading shared memory
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                                 "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                 ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p.acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores complete before smem goes away
+    }
+    pipe_exit<Plan>(p, tmem_base, P.status);
+}
+
+// ------------------------------------------------------------------ Gaussian head (last layer)
+// mean = A W^T + b; action = mean + sigma z with z from Philox counter (env, step, 1, block)
+// and Box-Muller; logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi.  The GEMM is tiny, the
+// noise is not: sixteen epilogue warps share the tile, four per group of 16 columns.
+constexpr int kHeadEpiWarps = 16;
+constexpr int kHeadThreads = 64 + 32 * kHeadEpiWarps;
+
+template <int BLOCK_N>
+__global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                         const __grid_constant__ CUtensorMap map_b,
+                                                                         const GemmParams P)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    extern __shared__ uint8_t smem_raw[];
+    const Pipe p = carve_pipe<Plan>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (P.M + BLOCK_M - 1) / BLOCK_M;             // one N tile holds the whole action row
+    float *zz_part = reinterpret_cast<float *>(p.epi + Plan::kEpiBytes);            // [2][4][128]
+    int *zz_count = reinterpret_cast<int *>(zz_part + 2 * 4 * 128);                 // [2][128]
+    for (int i = threadIdx.x; i < 2 * 128; i += blockDim.x) zz_count[i] = 0;
+    pipe_init<Plan>(p, kHeadEpiWarps);
+    const uint32_t tmem_base = *p.tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) producer_role<Plan, BLOCK_N>(p, &map_a, &map_b, P, n_tiles);
+    } else if (warp == 1) {
+        if (lane == 0) mma_role<Plan, BLOCK_N>(p, tmem_base, P, n_tiles);
+    } else {
+        const int quad = warp & 3;
+        const int group = (warp - 2) >> 2;                          // 16-column groups group, group+4, ...
+        const int row_in_tile = quad * 32 + lane;
+        constexpr int kGroups = (BLOCK_N / 16) < 4 ? (BLOCK_N / 16) : 4;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            const int m0 = tile * BLOCK_M;
+            if (!mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag)) break;
+            tc_fence_after();
+            const int row = m0 + row_in_tile;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
+            float zz = 0.0f;
+#pragma unroll 1
+            for (int c0 = 16 * group; c0 < BLOCK_N; c0 += 64) {
+                float v[16];
+                tmem_ld16(t_row + (uint32_t)c0, v);
+                if (row < P.M && c0 < P.N) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const int col = c0 + 4 * g;
+                        if (col >= P.N) break;
+                        const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
+                                                                 (uint32_t)(col >> 2)),
+                                                      make_uint2(P.seed_lo, P.seed_hi));
+                        float z[4];
+                        box_muller(x.x, x.y, z[0], z[1]);
+                        box_muller(x.z, x.w, z[2], z[3]);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            if (col + i < P.N) {
+                                const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
+                                P.mean[(size_t)row * P.N + col + i] = mu;
+                                P.action[(size_t)row * P.N + col + i] = mu + P.sigma * z[i];
+                                zz += z[i] * z[i];
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            // log-probability: the last of the column groups to finish a row adds the partial sums in
+            // group order, so the result does not depend on which one that is.  The accumulator is
+            // released only afterwards, which also keeps the partial-sum slots of this buffer from
+            // being rewritten (two tiles later) before they have been read.
+            if (group < kGroups && P.logp) {
+                float *part = zz_part + (size_t)acc * 4 * 128;
+                int *cnt = zz_count + acc * 128;
+                part[group * 128 + row_in_tile] = zz;
+                __threadfence_block();
+                if (atomicAdd(&cnt[row_in_tile], 1) == kGroups - 1) {
+                    __threadfence_block();
+                    float s = 0.0f;
+#pragma unroll
+                    for (int g = 0; g < kGroups; ++g) s += part[g * 128 + row_in_tile];
+                    cnt[row_in_tile] = 0;
+                    if (row < P.M)
+                        P.logp[row] = -0.5f * s - (float)P.N * logf(P.sigma) - 0.5f * (float)P.N * 1.8378770664093453f;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p.acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+    pipe_exit<Plan>(p, tmem_base, P.status);
 }
 
 // fp32 observations -> bf16 rows of a padded buffer; columns beyond `cols` are written as zero.
@@ -398,7 +533,7 @@ struct TcLayer {
     int N, K, Kpad, block_n, n_tiles_n;
     __nv_bfloat16 *d_W;      // [n_tiles_n * block_n][Kpad], zero padded
     float *d_bias;           // [n_tiles_n * block_n]
-    CUtensorMap map_a, map_b;
+    CUtensorMap map_a, map_b, map_c;    // map_c: the hidden-activation buffer this layer stores to
 };
 
 }  // namespace im
@@ -415,20 +550,38 @@ namespace im {
 
 namespace {
 
-template <int BLOCK_N, int EPI>
-cudaError_t launch_tc(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+template <int BLOCK_N>
+cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
     static bool prepared = false;
     if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BLOCK_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)Plan::kBytes);
         if (e != cudaSuccess) return e;
         prepared = true;
     }
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_kernel<BLOCK_N, EPI><<<grid, kThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, gp);
+    linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+template <int BLOCK_N>
+cudaError_t launch_head(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    static bool prepared = false;
+    if (!prepared) {
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_head_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)Plan::kBytes);
+        if (e != cudaSuccess) return e;
+        prepared = true;
+    }
+    const int tiles = (gp.M + BLOCK_M - 1) / BLOCK_M;
+    const int grid = tiles < n_sm ? tiles : n_sm;
+    linear_tc_head_kernel<BLOCK_N><<<grid, kHeadThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -437,20 +590,20 @@ cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n
 {
     if (!last) {
         switch (L.block_n) {
-        case 256: return launch_tc<256, EPI_RELU_BF16>(L, gp, n_sm, stream);
-        case 128: return launch_tc<128, EPI_RELU_BF16>(L, gp, n_sm, stream);
-        default: return launch_tc<64, EPI_RELU_BF16>(L, gp, n_sm, stream);
+        case 256: return launch_hidden<256>(L, gp, n_sm, stream);
+        case 128: return launch_hidden<128>(L, gp, n_sm, stream);
+        default: return launch_hidden<64>(L, gp, n_sm, stream);
         }
     }
     switch (L.block_n) {
-    case 16: return launch_tc<16, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 32: return launch_tc<32, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 48: return launch_tc<48, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 64: return launch_tc<64, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 80: return launch_tc<80, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 96: return launch_tc<96, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 112: return launch_tc<112, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
-    case 128: return launch_tc<128, EPI_GAUSS_HEAD>(L, gp, n_sm, stream);
+    case 16: return launch_head<16>(L, gp, n_sm, stream);
+    case 32: return launch_head<32>(L, gp, n_sm, stream);
+    case 48: return launch_head<48>(L, gp, n_sm, stream);
+    case 64: return launch_head<64>(L, gp, n_sm, stream);
+    case 80: return launch_head<80>(L, gp, n_sm, stream);
+    case 96: return launch_head<96>(L, gp, n_sm, stream);
+    case 112: return launch_head<112>(L, gp, n_sm, stream);
+    case 128: return launch_head<128>(L, gp, n_sm, stream);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -515,6 +668,9 @@ im_status tc_policy_create(im_policy *p, const void *const *W, const float *cons
         if (!make_map(&L.map_a, a_base, mb, (uint64_t)L.Kpad, (uint64_t)a_ld, BLOCK_M) ||
             !make_map(&L.map_b, L.d_W, rows, (uint64_t)L.Kpad, (uint64_t)L.Kpad, (uint32_t)L.block_n))
             return IM_ERR_CUDA;
+        // hidden layers store 32-row x 64-column slabs of their output buffer
+        if (!last && !make_map(&L.map_c, tc->d_hidden[l & 1], mb, rows, (uint64_t)tc->ld_hidden, 32))
+            return IM_ERR_CUDA;
     }
     return IM_OK;
 }
@@ -548,8 +704,6 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         const bool last = l == p->nl - 1;
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
-        gp.out_bf16 = last ? nullptr : tc->d_hidden[l & 1];
-        gp.ld_out = tc->ld_hidden;
         gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
         gp.sigma = cfg.sigma; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
         gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
