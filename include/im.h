@@ -190,7 +190,8 @@ im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, co
  *   b       HOST [n_layers] pointers to float [dims[l+1]]
  * dtype 0 runs fp32 SIMT kernels.  dtype 1 runs the tensor-core path: bf16
  * operands (observations and hidden activations are rounded to bf16), fp32
- * accumulation; it needs n_layers >= 2 and hidden widths that are multiples of 64. */
+ * accumulation; it needs n_layers >= 2, hidden widths that are multiples of 64 and an action
+ * width of at most 80. */
 typedef struct {
     int32_t n_layers;
     int32_t dims[IM_MAX_LAYERS + 1];
@@ -208,6 +209,7 @@ void im_destroy_policy(im_policy *p);
 
 /*   obs        DEVICE [n][ld_obs] float, ld_obs >= dims[0], multiple of 4, 16-byte aligned
  *   mean_out   DEVICE [n][A]     action_out DEVICE [n][A]     logp_out DEVICE [n] or NULL
+ *              (mean_out and action_out 16-byte aligned on the tensor-core path)
  * logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi. */
 im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out);

@@ -342,7 +342,10 @@ im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
     if (!p || !obs || !mean_out || !action_out) return IM_ERR_INVALID_ARG;
     if (n < 1 || n > p->cfg.max_batch || ld_obs < p->cfg.dims[0] || (ld_obs & 3) || !aligned16(obs))
         return IM_ERR_INVALID_ARG;
-    if (p->tensor_path) return tc_policy_forward(p, step, n, obs, ld_obs, mean_out, action_out, logp_out);
+    if (p->tensor_path) {
+        if (!aligned16(mean_out) || !aligned16(action_out)) return IM_ERR_INVALID_ARG;
+        return tc_policy_forward(p, step, n, obs, ld_obs, mean_out, action_out, logp_out);
+    }
     const float *in = obs;
     int ld_in = ld_obs;
     const int A = p->cfg.dims[p->nl];

@@ -157,6 +157,7 @@ struct GemmParams {
     int N;             // valid output columns
     int K_blocks;      // K / 64 (K is padded with zeros)
     int n_tiles_n;     // N tiles of BLOCK_N
+    int stages;        // depth of the operand ring in shared memory
     const float *bias; // [n_tiles_n * BLOCK_N], zero padded
     // Gaussian head
     float *mean, *action, *logp;
@@ -167,22 +168,34 @@ struct GemmParams {
 
 constexpr int kEpiSlabBytes = 32 * 128;    // one epilogue warp's 32 rows x 64 bf16 staging slab
 
+constexpr size_t kSmemLimit = 232448;       // opt-in shared memory per block on this architecture (227 KB)
+
 template <int BLOCK_N>
 struct SmemPlan {
-    static constexpr int kStages = BLOCK_N >= 256 ? 4 : 6;
     static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
     static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
     static constexpr int kBBytesPadded = (kBBytes + 1023) / 1024 * 1024;     // keep every tile 1024-byte aligned
     static constexpr int kStageBytes = kABytes + kBBytesPadded;
     static constexpr int kAccStride = BLOCK_N <= 128 ? 128 : 256;           // TMEM columns between the two accumulators
     static constexpr int kTmemCols = 2 * kAccStride;
-    static constexpr int kEpiBytes = 4 * kEpiSlabBytes;                     // hidden layers: staging for the TMA stores
-    static constexpr int kHeadBytes = 2 * 4 * 128 * 4 + 2 * 128 * 4;        // head: partial sums of z^2 and arrival counters
     static constexpr int kBarBytes = 256;
-    static constexpr size_t kBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + kEpiBytes + kHeadBytes + kBarBytes;
+    static constexpr int kMaxStages = 8;
+    // hidden layers: two staging slabs per epilogue warp for the TMA stores
+    static constexpr int kHiddenEpiBytes = 4 * 2 * kEpiSlabBytes;
+    // head: [2 accumulators][mean, action][128 rows][A] floats laid out as in global memory,
+    // partial sums of z^2 [2][4][128], band counters [2][4]
+    __host__ __device__ static constexpr int head_epi_bytes(int A) { return (2 * 2 * 128 * A * 4 + 2 * 4 * 128 * 4 + 64 + 1023) / 1024 * 1024; }
+    __host__ __device__ static constexpr int stages_for(int epi_bytes)
+    {
+        const int room = (int)kSmemLimit - 1024 - kBarBytes - epi_bytes;
+        const int s = room / kStageBytes;
+        return s > kMaxStages ? kMaxStages : s;
+    }
+    __host__ __device__ static constexpr size_t bytes(int stages, int epi_bytes) { return 1024 + (size_t)stages * kStageBytes + epi_bytes + kBarBytes; }
 };
 
 struct Pipe {
+    int stages;
     uint8_t *tiles;
     uint64_t *full, *empty, *acc_full, *acc_empty;
     uint32_t *tmem_slot;
@@ -191,17 +204,18 @@ struct Pipe {
 };
 
 template <class Plan>
-__device__ __forceinline__ Pipe carve_pipe(uint8_t *smem_raw)
+__device__ __forceinline__ Pipe carve_pipe(uint8_t *smem_raw, int stages, int epi_bytes)
 {
     Pipe p;
+    p.stages = stages;
     p.tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    p.epi = p.tiles + (size_t)Plan::kStages * Plan::kStageBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(p.epi + Plan::kEpiBytes + Plan::kHeadBytes);
+    p.epi = p.tiles + (size_t)stages * Plan::kStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(p.epi + epi_bytes);
     p.full = bars;
-    p.empty = bars + Plan::kStages;
-    p.acc_full = bars + 2 * Plan::kStages;
-    p.acc_empty = bars + 2 * Plan::kStages + 2;
-    p.tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Plan::kStages + 4);
+    p.empty = bars + Plan::kMaxStages;
+    p.acc_full = bars + 2 * Plan::kMaxStages;
+    p.acc_empty = bars + 2 * Plan::kMaxStages + 2;
+    p.tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Plan::kMaxStages + 4);
     p.abort_flag = reinterpret_cast<volatile int *>(p.tmem_slot + 1);
     return p;
 }
@@ -210,7 +224,7 @@ template <class Plan>
 __device__ __forceinline__ void pipe_init(const Pipe &p, int epi_arrivals)
 {
     if (threadIdx.x == 0) {
-        for (int s = 0; s < Plan::kStages; ++s) { mbar_init(&p.full[s], 1); mbar_init(&p.empty[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&p.full[s], 1); mbar_init(&p.empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&p.acc_full[a], 1); mbar_init(&p.acc_empty[a], epi_arrivals); }
         *p.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -254,7 +268,7 @@ __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *
             mbar_arrive_expect_tx(&p.full[stage], Plan::kABytes + Plan::kBBytes);
             tma_load_2d(sa, map_a, &p.full[stage], kb * BLOCK_K, m0);
             tma_load_2d(sa + Plan::kABytes, map_b, &p.full[stage], kb * BLOCK_K, n0);
-            if (++stage == Plan::kStages) { stage = 0; phase ^= 1u; }
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
     }
 }
@@ -281,7 +295,7 @@ __device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, cons
                 umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
             }
             umma_commit(&p.empty[stage]);            // smem stage is free once these MMAs have read it
-            if (++stage == Plan::kStages) { stage = 0; phase ^= 1u; }
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
         umma_commit(&p.acc_full[acc]);               // accumulator complete
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -300,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
 {
     using Plan = SmemPlan<BLOCK_N>;
     extern __shared__ uint8_t smem_raw[];
-    const Pipe p = carve_pipe<Plan>(smem_raw);
+    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::kHiddenEpiBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
     pipe_init<Plan>(p, kEpiWarps);
@@ -312,8 +326,8 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
         if (lane == 0) mma_role<Plan, BLOCK_N>(p, tmem_base, P, n_tiles);
     } else {
         const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
-        uint8_t *slab = p.epi + (size_t)(warp - 2) * kEpiSlabBytes;
-        const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
+        uint8_t *slabs = p.epi + (size_t)(warp - 2) * 2 * kEpiSlabBytes;       // two slabs, used alternately
+        int which = 0;
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -337,9 +351,11 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
                     pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
                     pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
                 }
-                // the previous slab's store must have finished reading shared memory
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                // the store issued two slabs ago (same buffer) must have finished reading shared memory
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 __syncwarp();
+                uint8_t *slab = slabs + which * kEpiSlabBytes;
+                const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
@@ -353,6 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
                                  ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
+                which ^= 1;
             }
             tc_fence_before();
             __syncwarp();
@@ -378,12 +395,17 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
 {
     using Plan = SmemPlan<BLOCK_N>;
     extern __shared__ uint8_t smem_raw[];
-    const Pipe p = carve_pipe<Plan>(smem_raw);
+    const int A = P.N;
+    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::head_epi_bytes(A));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = (P.M + BLOCK_M - 1) / BLOCK_M;             // one N tile holds the whole action row
-    float *zz_part = reinterpret_cast<float *>(p.epi + Plan::kEpiBytes);            // [2][4][128]
-    int *zz_count = reinterpret_cast<int *>(zz_part + 2 * 4 * 128);                 // [2][128]
-    for (int i = threadIdx.x; i < 2 * 128; i += blockDim.x) zz_count[i] = 0;
+    const int out_floats = 128 * A;
+    // staging: per accumulator buffer the tile's mean and action rows laid out exactly as in global
+    // memory ([128][A], dense), so a 32-row band leaves as one contiguous copy
+    float *out_tiles = reinterpret_cast<float *>(p.epi);                            // [2][2][128 * A]
+    float *zz_part = out_tiles + 2 * 2 * out_floats;                                // [2][4][128]
+    int *band_count = reinterpret_cast<int *>(zz_part + 2 * 4 * 128);               // [2][4]
+    if (threadIdx.x < 8) band_count[threadIdx.x] = 0;
     pipe_init<Plan>(p, kHeadEpiWarps);
     const uint32_t tmem_base = *p.tmem_slot;
 
@@ -392,10 +414,11 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
     } else if (warp == 1) {
         if (lane == 0) mma_role<Plan, BLOCK_N>(p, tmem_base, P, n_tiles);
     } else {
-        const int quad = warp & 3;
+        const int quad = warp & 3;                                  // 32-row band of the tile (TMEM lane quadrant)
         const int group = (warp - 2) >> 2;                          // 16-column groups group, group+4, ...
         const int row_in_tile = quad * 32 + lane;
         constexpr int kGroups = (BLOCK_N / 16) < 4 ? (BLOCK_N / 16) : 4;
+        const float logp_const = -(float)A * logf(P.sigma) - 0.5f * (float)A * 1.8378770664093453f;
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -404,52 +427,74 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
             tc_fence_after();
             const int row = m0 + row_in_tile;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
+            float *s_mean = out_tiles + (size_t)acc * 2 * out_floats;
+            float *s_act = s_mean + out_floats;
             float zz = 0.0f;
+            if (group < kGroups) {
 #pragma unroll 1
-            for (int c0 = 16 * group; c0 < BLOCK_N; c0 += 64) {
-                float v[16];
-                tmem_ld16(t_row + (uint32_t)c0, v);
-                if (row < P.M && c0 < P.N) {
+                for (int c0 = 16 * group; c0 < BLOCK_N; c0 += 64) {
+                    float v[16];
+                    tmem_ld16(t_row + (uint32_t)c0, v);
+                    if (c0 < A) {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const int col = c0 + 4 * g;
-                        if (col >= P.N) break;
-                        const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
-                                                                 (uint32_t)(col >> 2)),
-                                                      make_uint2(P.seed_lo, P.seed_hi));
-                        float z[4];
-                        box_muller(x.x, x.y, z[0], z[1]);
-                        box_muller(x.z, x.w, z[2], z[3]);
+                        for (int g = 0; g < 4; ++g) {
+                            const int col = c0 + 4 * g;
+                            if (col >= A) break;
+                            const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
+                                                                     (uint32_t)(col >> 2)),
+                                                          make_uint2(P.seed_lo, P.seed_hi));
+                            float z[4];
+                            box_muller(x.x, x.y, z[0], z[1]);
+                            box_muller(x.z, x.w, z[2], z[3]);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            if (col + i < P.N) {
-                                const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
-                                P.mean[(size_t)row * P.N + col + i] = mu;
-                                P.action[(size_t)row * P.N + col + i] = mu + P.sigma * z[i];
-                                zz += z[i] * z[i];
+                            for (int i = 0; i < 4; ++i) {
+                                if (col + i < A) {
+                                    const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
+                                    s_mean[row_in_tile * A + col + i] = mu;
+                                    s_act[row_in_tile * A + col + i] = mu + P.sigma * z[i];
+                                    zz += z[i] * z[i];
+                                }
                             }
                         }
                     }
                 }
+                zz_part[(acc * 4 + group) * 128 + row_in_tile] = zz;
             }
             tc_fence_before();
-            // log-probability: the last of the column groups to finish a row adds the partial sums in
-            // group order, so the result does not depend on which one that is.  The accumulator is
-            // released only afterwards, which also keeps the partial-sum slots of this buffer from
-            // being rewritten (two tiles later) before they have been read.
-            if (group < kGroups && P.logp) {
-                float *part = zz_part + (size_t)acc * 4 * 128;
-                int *cnt = zz_count + acc * 128;
-                part[group * 128 + row_in_tile] = zz;
+            // The last of the column-group warps to finish a 32-row band sums that band's partial z^2
+            // in group order (so the result does not depend on which warp that is) and copies the
+            // band's mean and action rows out as contiguous 16-byte stores.  The accumulator buffer,
+            // and with it this staging buffer, is released only afterwards.
+            if (group < kGroups) {
                 __threadfence_block();
-                if (atomicAdd(&cnt[row_in_tile], 1) == kGroups - 1) {
+                __syncwarp();
+                int prev = 0;
+                if (lane == 0) prev = atomicAdd(&band_count[acc * 4 + quad], 1);
+                prev = __shfl_sync(0xffffffffu, prev, 0);
+                if (prev == kGroups - 1) {
                     __threadfence_block();
-                    float s = 0.0f;
+                    if (lane == 0) band_count[acc * 4 + quad] = 0;
+                    const int band_row0 = m0 + quad * 32;
+                    int rows_valid = P.M - band_row0;
+                    rows_valid = rows_valid > 32 ? 32 : rows_valid;
+                    if (rows_valid > 0) {
+                        if (P.logp && lane < rows_valid) {
+                            float sum = 0.0f;
 #pragma unroll
-                    for (int g = 0; g < kGroups; ++g) s += part[g * 128 + row_in_tile];
-                    cnt[row_in_tile] = 0;
-                    if (row < P.M)
-                        P.logp[row] = -0.5f * s - (float)P.N * logf(P.sigma) - 0.5f * (float)P.N * 1.8378770664093453f;
+                            for (int g = 0; g < kGroups; ++g) sum += zz_part[(acc * 4 + g) * 128 + row_in_tile];
+                            P.logp[row] = -0.5f * sum + logp_const;
+                        }
+                        const int count = rows_valid * A;                       // floats, contiguous in global
+                        const float *src_m = s_mean + quad * 32 * A, *src_a = s_act + quad * 32 * A;
+                        float *dst_m = P.mean + (size_t)band_row0 * A, *dst_a = P.action + (size_t)band_row0 * A;
+                        // both sides start on a 16-byte boundary: band offsets are multiples of 32 rows
+                        const int n4 = count >> 2;
+                        for (int i = lane; i < n4; i += 32) {
+                            reinterpret_cast<float4 *>(dst_m)[i] = reinterpret_cast<const float4 *>(src_m)[i];
+                            reinterpret_cast<float4 *>(dst_a)[i] = reinterpret_cast<const float4 *>(src_a)[i];
+                        }
+                        for (int i = 4 * n4 + lane; i < count; i += 32) { dst_m[i] = src_m[i]; dst_a[i] = src_a[i]; }
+                    }
                 }
             }
             __syncwarp();
@@ -551,37 +596,45 @@ namespace im {
 namespace {
 
 template <int BLOCK_N>
-cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
     static bool prepared = false;
     if (!prepared) {
         cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)Plan::kBytes);
+                                             (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         prepared = true;
     }
+    GemmParams gp = gp_in;
+    gp.stages = Plan::stages_for(Plan::kHiddenEpiBytes);
+    const size_t smem = Plan::bytes(gp.stages, Plan::kHiddenEpiBytes);
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
 
 template <int BLOCK_N>
-cudaError_t launch_head(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+cudaError_t launch_head(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
     static bool prepared = false;
     if (!prepared) {
         cudaError_t e = cudaFuncSetAttribute(linear_tc_head_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)Plan::kBytes);
+                                             (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         prepared = true;
     }
+    GemmParams gp = gp_in;
+    const int epi = Plan::head_epi_bytes(gp.N);
+    gp.stages = Plan::stages_for(epi);
+    if (gp.stages < 2) return cudaErrorInvalidValue;
+    const size_t smem = Plan::bytes(gp.stages, epi);
     const int tiles = (gp.M + BLOCK_M - 1) / BLOCK_M;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_head_kernel<BLOCK_N><<<grid, kHeadThreads, Plan::kBytes, stream>>>(L.map_a, L.map_b, gp);
+    linear_tc_head_kernel<BLOCK_N><<<grid, kHeadThreads, smem, stream>>>(L.map_a, L.map_b, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -601,9 +654,6 @@ cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n
     case 48: return launch_head<48>(L, gp, n_sm, stream);
     case 64: return launch_head<64>(L, gp, n_sm, stream);
     case 80: return launch_head<80>(L, gp, n_sm, stream);
-    case 96: return launch_head<96>(L, gp, n_sm, stream);
-    case 112: return launch_head<112>(L, gp, n_sm, stream);
-    case 128: return launch_head<128>(L, gp, n_sm, stream);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -617,7 +667,7 @@ im_status tc_policy_create(im_policy *p, const void *const *W, const float *cons
     if (nl < 2) return IM_ERR_UNSUPPORTED;
     for (int l = 1; l < nl; ++l)
         if (cfg.dims[l] % 64) return IM_ERR_UNSUPPORTED;
-    if (cfg.dims[nl] > 128) return IM_ERR_UNSUPPORTED;
+    if (cfg.dims[nl] > 80) return IM_ERR_UNSUPPORTED;      // staging of the head's output tiles is sized for this
     int dev = 0, cc_major = 0, n_sm = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
