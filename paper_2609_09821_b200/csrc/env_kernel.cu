@@ -2,12 +2,18 @@
 // error terms and reward, flags, masked Philox reset, heading-local
 // observation (the post-physics phase of the paper's Figure 2 as one kernel).
 //
-// Mapping: one CTA handles 32 consecutive envs; warp j handles body j and lane
-// e handles env e of the tile, so every global load of the structure-of-arrays
-// body state is one fully used 128-byte line per warp.  Cross-body data (the
-// kinematic chain, reward partial sums, root heading) goes through shared
-// memory; the observation tile is transposed in shared memory so that rows of
-// the row-major [N][ld_obs] output are written as whole lines.
+// Mapping: one CTA handles 32 consecutive envs; lane e handles env e of the
+// tile and warp c handles kinematic chain c of the skeleton, a root-to-leaf
+// path.  A thread walks its path once per pass, carrying the world transform
+// (and velocities) in registers, so forward kinematics needs no exchange
+// between threads; bodies shared by several paths are recomputed (pose only)
+// and "owned" by one path, which alone loads their simulated state, scores them
+// and writes their observation entries.  Every global load of the
+// structure-of-arrays body state is one fully used 128-byte line per warp.
+// The observation tile [32][D] is assembled in shared memory (row stride 4 x odd:
+// conflict-free 16-byte column writes, 16-byte aligned rows) and written out
+// as whole lines.  Two block-wide barriers per tile: after the reward partial
+// sums, and before the tile is stored.
 #include "im_internal.h"
 #include "im_device.cuh"
 
@@ -16,45 +22,19 @@ namespace im {
 namespace {
 
 constexpr int kTile = 32;          // envs per CTA
-constexpr int kRefComps = 7;       // local quaternion + child-frame joint angular velocity
-constexpr int kTgtComps = 4;       // local quaternion
-constexpr int kSimComps = 7;       // world quaternion + world angular velocity (read by children)
 constexpr int kPartials = 9;       // pose, vel, ee_pos, ee_rot, body_pos, body_vel, weighted com difference (3)
 
-struct Smem {
-    float *ref, *tgt, *rootp, *rootv, *tgt_rootp, *head;   // head: root x, root y, cos, sin
-    int *cur_clip, *mask, *any;
-    float *cur_t;
-    float *simx, *part, *tile;                             // tile aliases simx + part
-};
-
-__host__ __device__ inline size_t smem_floats(int J)
+__host__ __device__ inline int tile_stride(int D)
 {
-    const int D = 24 * J + 1;
-    const size_t fixed = (size_t)J * (kRefComps + kTgtComps) * kTile + 9 * kTile + 4 * kTile + 3 * kTile + kTile;
-    const size_t a = (size_t)J * (kSimComps + kPartials) * kTile;
-    const size_t b = (size_t)kTile * D;
-    return fixed + (a > b ? a : b);
+    int s4 = (D + 3) / 4;
+    if ((s4 & 1) == 0) ++s4;       // stride = 4 x odd floats
+    return 4 * s4;
 }
 
-__device__ __forceinline__ Smem carve(float *base, int J)
+__host__ __device__ inline size_t smem_floats(int J, int n_chains)
 {
-    Smem s;
-    float *p = base;
-    s.ref = p;        p += J * kRefComps * kTile;
-    s.tgt = p;        p += J * kTgtComps * kTile;
-    s.rootp = p;      p += 3 * kTile;
-    s.rootv = p;      p += 3 * kTile;
-    s.tgt_rootp = p;  p += 3 * kTile;
-    s.head = p;       p += 4 * kTile;
-    s.cur_clip = reinterpret_cast<int *>(p);  p += kTile;
-    s.mask = reinterpret_cast<int *>(p);      p += kTile;
-    s.cur_t = p;      p += kTile;
-    s.any = reinterpret_cast<int *>(p);       p += kTile;
-    s.simx = p;
-    s.part = p + J * kSimComps * kTile;
-    s.tile = p;
-    return s;
+    const int D = 24 * J + 1;
+    return (size_t)kTile * tile_stride(D) + (size_t)kPartials * n_chains * kTile;
 }
 
 // Keyframe row and blend factor at `time` (step a1): f = fl32(time * fps),
@@ -75,10 +55,39 @@ __device__ __forceinline__ Quat ld_quat(const float4 *p)
     return {v.x, v.y, v.z, v.w};
 }
 
+// asin(y)^2 / y^2 as a series in u = y^2:  1/2 sum_n (4u)^n / (n^2 C(2n,n)) / u.
+// Eight terms: relative truncation error below 1e-8 for u <= 0.15.
+__device__ __forceinline__ float asin2_over_u(float u)
+{
+    float p = 0.03978244f;                 // n = 8
+    p = fmaf(p, u, 0.04871319f);           // n = 7
+    p = fmaf(p, u, 0.06156806f);           // n = 6
+    p = fmaf(p, u, 0.08126984f);           // n = 5
+    p = fmaf(p, u, 0.11428571f);           // n = 4
+    p = fmaf(p, u, 0.17777778f);           // n = 3
+    p = fmaf(p, u, 0.33333333f);           // n = 2
+    return fmaf(p, u, 1.0f);               // n = 1
+}
+
+// sin(sqrt y) / sqrt y for small y (error below 1e-10 for y <= 0.07).
+__device__ __forceinline__ float sinc_sqrt(float y)
+{
+    float p = -1.9841270e-4f;
+    p = fmaf(p, y, 8.3333333e-3f);
+    p = fmaf(p, y, -1.6666667e-1f);
+    return fmaf(p, y, 1.0f);
+}
+
 // Shortest-arc slerp of one joint plus, if asked, the joint's angular velocity
 // in the child frame, 2 log(q0* q1) fps.  The vector part of q0* q1 is formed
 // from q1 - q0, which avoids the cancellation of the direct product when the
 // keyframes are close and keeps the velocity accurate to ~1e-6 rad/s.
+// Keyframes of a motion clip are close together, so the usual case (angle
+// between the two quaternions below 0.25 rad) is evaluated without
+// trigonometric calls: theta^2 from sin^2 theta by the arcsine series, and
+// sin(a theta)/sin(theta) = a sinc(a theta)/sinc(theta) by short polynomials.
+// Everything is normalised by |q0||q1|, so slightly non-unit keyframes give
+// the same rotation as their normalised versions.
 template <bool VEL>
 __device__ __forceinline__ void slerp_joint(Quat q0, Quat q1, float alpha, float fps, Quat &q, Vec3 &wl)
 {
@@ -86,331 +95,422 @@ __device__ __forceinline__ void slerp_joint(Quat q0, Quat q1, float alpha, float
     if (d < 0.0f) { d = -d; q1 = {-q1.w, -q1.x, -q1.y, -q1.z}; }
     const Quat diff = {q1.w - q0.w, q1.x - q0.x, q1.y - q0.y, q1.z - q0.z};
     const Quat c = qmul(qconj(q0), diff);
-    const float n = sqrtf(c.x * c.x + c.y * c.y + c.z * c.z);
-    const float theta = atan2f(n, d);
-    float s0, s1;
-    if (d > 1.0f - 1e-6f) { s0 = 1.0f - alpha; s1 = alpha; }
-    else {
+    const float n2 = c.x * c.x + c.y * c.y + c.z * c.z;
+    const float m2 = fmaf(d, d, n2);                       // (|q0||q1|)^2
+    const float u = __fdividef(n2, m2);                    // sin^2 theta
+    float s0, s1, vel_scale = 0.0f;
+    if (u <= 0.0625f) {
+        const float x = u * asin2_over_u(u);               // theta^2
+        const float sc = sinc_sqrt(x);
+        float inv = __fdividef(1.0f, sc);                  // theta / sin theta ...
+        inv = inv * fmaf(-sc, inv, 2.0f);                  // ... refined to full precision (Newton step)
+        const float a0 = 1.0f - alpha;
+        s0 = a0 * sinc_sqrt(a0 * a0 * x) * inv;
+        s1 = alpha * sinc_sqrt(alpha * alpha * x) * inv;
+        if (VEL) {
+            float rs = rsqrtf(m2);                         // 1 / (|q0||q1|), one Newton step as well:
+            rs = rs * fmaf(-0.5f * m2, rs * rs, 1.5f);     // the velocity is summed down the chain
+            vel_scale = 2.0f * fps * inv * rs;
+        }
+    } else {
+        const float n = sqrtf(n2);
+        const float theta = atan2f(n, d);
         const float inv = 1.0f / n;
         s0 = sinf((1.0f - alpha) * theta) * inv;
         s1 = sinf(alpha * theta) * inv;
+        vel_scale = 2.0f * theta * fps * inv;
     }
-    Quat r = {s0 * q0.w + s1 * q1.w, s0 * q0.x + s1 * q1.x, s0 * q0.y + s1 * q1.y, s0 * q0.z + s1 * q1.z};
-    const float rn = 1.0f / sqrtf(r.w * r.w + r.x * r.x + r.y * r.y + r.z * r.z);
+    const Quat r = {s0 * q0.w + s1 * q1.w, s0 * q0.x + s1 * q1.x, s0 * q0.y + s1 * q1.y, s0 * q0.z + s1 * q1.z};
+    const float rn = rsqrtf(r.w * r.w + r.x * r.x + r.y * r.y + r.z * r.z);
     q = {r.w * rn, r.x * rn, r.y * rn, r.z * rn};
-    if (VEL) {
-        const float k = (n < 1e-12f) ? 0.0f : 2.0f * theta * fps / n;
-        wl = {k * c.x, k * c.y, k * c.z};
-    }
+    if (VEL) wl = {vel_scale * c.x, vel_scale * c.y, vel_scale * c.z};
 }
 
-// Reference pose of body j's own joint at `time` into shared memory; warp 0
-// also publishes the root position (lerp) and, if asked, the root velocity.
-template <bool VEL, int NC>
-__device__ __forceinline__ void stage_joint(const EnvKernelParams &P, const ClipMeta &cm, float time, int j,
-                                            int lane, float *dst, float *rootp, float *rootv,
-                                            Quat &ql, Vec3 &wl)
+// Squared rotation angle, in [0, pi^2], of the rotation taking frame a to frame b.  Small
+// angles (below 0.8 rad, the usual tracking error) use the arcsine series on sin^2(theta/2).
+__device__ __forceinline__ float rel_angle_sq(Quat a, Quat b)
 {
-    int row;
-    float alpha;
-    lookup(cm, time, row, alpha);
-    const int RS = P.sk.J + 1;
-    const float4 *r0 = P.frames + (size_t)row * RS;
-    const float4 *r1 = r0 + RS;
-    slerp_joint<VEL>(ld_quat(r0 + 1 + j), ld_quat(r1 + 1 + j), alpha, cm.fps, ql, wl);
-    float *o = dst + (j * NC) * kTile + lane;
-    o[0 * kTile] = ql.w; o[1 * kTile] = ql.x; o[2 * kTile] = ql.y; o[3 * kTile] = ql.z;
-    if (VEL) { o[4 * kTile] = wl.x; o[5 * kTile] = wl.y; o[6 * kTile] = wl.z; }
-    if (j == 0) {
-        const float4 a = __ldg(r0), b = __ldg(r1);
-        rootp[0 * kTile + lane] = a.x + alpha * (b.x - a.x);
-        rootp[1 * kTile + lane] = a.y + alpha * (b.y - a.y);
-        rootp[2 * kTile + lane] = a.z + alpha * (b.z - a.z);
+    const Quat r = qmul(qconj(a), b);
+    const float n2 = r.x * r.x + r.y * r.y + r.z * r.z;
+    const float u = __fdividef(n2, fmaf(r.w, r.w, n2));    // sin^2(theta / 2)
+    if (u <= 0.15f) return 4.0f * u * asin2_over_u(u);
+    const float th = 2.0f * atan2f(sqrtf(n2), fabsf(r.w));
+    return th * th;
+}
+
+// World transform (and velocities) carried down a kinematic chain (step a2).
+struct Walk {
+    Quat q;
+    Vec3 p, v, w;
+};
+
+// One link of the chain: interpolate joint b between keyframe rows r0/r1 and
+// compose it onto the running transform.  k == 0 is the root.
+template <bool VEL>
+__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, float alpha,
+                                           float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
+{
+    slerp_joint<VEL>(ld_quat(r0 + 1 + b), ld_quat(r1 + 1 + b), alpha, fps, ql, wl);
+    if (k == 0) {
+        const float4 a = __ldg(r0), c = __ldg(r1);
+        s.q = ql;
+        s.p = {a.x + alpha * (c.x - a.x), a.y + alpha * (c.y - a.y), a.z + alpha * (c.z - a.z)};
         if (VEL) {
-            rootv[0 * kTile + lane] = (b.x - a.x) * cm.fps;
-            rootv[1 * kTile + lane] = (b.y - a.y) * cm.fps;
-            rootv[2 * kTile + lane] = (b.z - a.z) * cm.fps;
+            s.v = {(c.x - a.x) * fps, (c.y - a.y) * fps, (c.z - a.z) * fps};
+            s.w = qrot(ql, wl);
         }
+    } else {
+        const Vec3 arm = qrot(s.q, Vec3{sk.off[b][0], sk.off[b][1], sk.off[b][2]});
+        if (VEL) s.v = s.v + cross(s.w, arm);
+        s.p = s.p + arm;
+        s.q = qmul(s.q, ql);
+        if (VEL) s.w = s.w + qrot(s.q, wl);
     }
 }
 
-// Forward kinematics of body j by walking its ancestor chain root -> j
-// (step a2), with velocity propagation when VEL.
-template <bool VEL, int NC>
-__device__ __forceinline__ void fk_walk(const SkelDev &sk, int j, int lane, const float *src,
-                                        const float *rootp, const float *rootv,
-                                        Quat &q, Vec3 &p, Vec3 &v, Vec3 &w)
+// Heading frame of the character the observation is taken from: origin at the
+// root's (x, y, 0), yaw of the root's rotated x axis (step a6).
+struct Heading {
+    float ox, oy, c, s;
+    __device__ __forceinline__ Vec3 turn(Vec3 a) const { return {c * a.x + s * a.y, c * a.y - s * a.x, a.z}; }
+};
+
+__device__ __forceinline__ Heading make_heading(Quat q_root, Vec3 p_root)
 {
-    const float *r = src + lane;
-    q = {r[0 * kTile], r[1 * kTile], r[2 * kTile], r[3 * kTile]};
-    p = {rootp[0 * kTile + lane], rootp[1 * kTile + lane], rootp[2 * kTile + lane]};
-    if (VEL) {
-        v = {rootv[0 * kTile + lane], rootv[1 * kTile + lane], rootv[2 * kTile + lane]};
-        w = qrot(q, Vec3{r[4 * kTile], r[5 * kTile], r[6 * kTile]});
-    }
-    const int depth = sk.depth[j];
-    for (int d = 1; d <= depth; ++d) {
-        const int b = sk.chain[j][d];
-        const Vec3 arm = qrot(q, Vec3{sk.off[b][0], sk.off[b][1], sk.off[b][2]});
-        if (VEL) v = v + cross(w, arm);
-        p = p + arm;
-        const float *c = src + (b * NC) * kTile + lane;
-        q = qmul(q, Quat{c[0 * kTile], c[1 * kTile], c[2 * kTile], c[3 * kTile]});
-        if (VEL) w = w + qrot(q, Vec3{c[4 * kTile], c[5 * kTile], c[6 * kTile]});
+    const Vec3 h = qcol_x(q_root);
+    const float n2 = h.x * h.x + h.y * h.y;
+    Heading H = {p_root.x, p_root.y, 1.0f, 0.0f};
+    if (n2 >= 1e-12f) { const float inv = rsqrtf(n2); H.c = h.x * inv; H.s = h.y * inv; }
+    return H;
+}
+
+// Stores N consecutive floats at dst, whose offset from a 16-byte boundary is OFF floats,
+// using 16-byte stores for the aligned middle.
+template <int N, int OFF>
+__device__ __forceinline__ void store_run_at(float *dst, const float (&v)[N])
+{
+    constexpr int head = (4 - OFF) & 3;
+    constexpr int mid = (N - head) / 4;
+#pragma unroll
+    for (int i = 0; i < head; ++i) dst[i] = v[i];
+#pragma unroll
+    for (int m = 0; m < mid; ++m)
+        *reinterpret_cast<float4 *>(dst + head + 4 * m) =
+            make_float4(v[head + 4 * m], v[head + 4 * m + 1], v[head + 4 * m + 2], v[head + 4 * m + 3]);
+#pragma unroll
+    for (int i = head + 4 * mid; i < N; ++i) dst[i] = v[i];
+}
+
+template <int N>
+__device__ __forceinline__ void store_run(float *row, int col, const float (&v)[N])
+{
+    float *dst = row + col;
+    switch (col & 3) {          // uniform across the warp
+    case 0: store_run_at<N, 0>(dst, v); break;
+    case 1: store_run_at<N, 1>(dst, v); break;
+    case 2: store_run_at<N, 2>(dst, v); break;
+    default: store_run_at<N, 3>(dst, v); break;
     }
 }
 
-template <bool RESET_ALL>
-__global__ void __launch_bounds__(1024, 1) env_step_kernel(const __grid_constant__ EnvKernelParams P)
+// The 15 observation floats of one body seen from the heading frame.
+__device__ __forceinline__ void body_obs(const Heading &H, Quat q, Vec3 p, Vec3 v, Vec3 w, float *row, int b)
+{
+    const Vec3 pl = H.turn(Vec3{p.x - H.ox, p.y - H.oy, p.z});
+    const Vec3 tn = H.turn(qcol_x(q)), nm = H.turn(qcol_z(q));
+    const Vec3 vl = H.turn(v), wl = H.turn(w);
+    const float o[15] = {pl.x, pl.y, pl.z, tn.x, tn.y, tn.z, nm.x, nm.y, nm.z, vl.x, vl.y, vl.z, wl.x, wl.y, wl.z};
+    store_run<15>(row, 15 * b, o);
+}
+
+struct SimBody {
+    Quat q;
+    Vec3 p, v, w;
+};
+
+__device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
+{
+    const float n2 = q.w * q.w + q.x * q.x + q.y * q.y + q.z * q.z;
+    if (!(n2 > 1e-12f && n2 < 1e12f)) {
+        atomicOr(status, IM_DEV_BAD_SIM_QUAT);
+        return {1, 0, 0, 0};
+    }
+    return q;
+}
+
+__device__ __forceinline__ Quat ld_sim_quat(const EnvKernelParams &P, int b, int e)
+{
+    const size_t st = (size_t)P.stride;
+    return {P.quat[(4 * b + 0) * st + e], P.quat[(4 * b + 1) * st + e], P.quat[(4 * b + 2) * st + e],
+            P.quat[(4 * b + 3) * st + e]};
+}
+__device__ __forceinline__ Vec3 ld_sim_vec(const float *base, const EnvKernelParams &P, int b, int e)
+{
+    const size_t st = (size_t)P.stride;
+    return {base[(3 * b + 0) * st + e], base[(3 * b + 1) * st + e], base[(3 * b + 2) * st + e]};
+}
+
+// MAXT: largest block the instantiation may be launched with (32 threads per chain); skeletons with
+// at most 8 leaves use the variant that leaves the compiler more registers per thread.
+template <bool RESET_ALL, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
     const SkelDev &sk = P.sk;
     const int J = sk.J;
     const int D = 24 * J + 1;
+    const int S = tile_stride(D);
+    const int C = sk.n_chains;
     const int lane = threadIdx.x & 31;
-    const int j = threadIdx.x >> 5;
+    const int c = threadIdx.x >> 5;                 // this thread's chain
     const int env = blockIdx.x * kTile + lane;
     const bool valid = env < P.N;
     const int envc = valid ? env : P.N - 1;
-    const Smem S = carve(smem_raw, J);
+    float *tile = smem_raw;
+    float *part = smem_raw + (size_t)kTile * S;
+    float *row = tile + (size_t)lane * S;
+    const int len = sk.chain_len[c];
+    const int first_own = sk.chain_first_own[c];
+    const int RS = J + 1;
+
+    if (c == 0)
+        for (int i = D; i < S; ++i) row[i] = 0.0f;  // columns between D and the row stride
 
     int clip = 0;
     float t1 = 0.0f;
     ClipMeta cm = {2, 1.0f, 1.0f, 0};
-    Quat ql_ref = {1, 0, 0, 0}, q_sim = {1, 0, 0, 0};
-    Vec3 wl_ref = {0, 0, 0}, p_sim = {0, 0, 0}, v_sim = {0, 0, 0}, w_sim = {0, 0, 0};
+    Heading H = {0.0f, 0.0f, 1.0f, 0.0f};
+    float root_z = 0.0f;
 
-    // ---- phase 1: advance time, stage the reference joint, load the simulated body
+    // ---- pass A: reference at the advanced time, errors against the simulated state,
+    //      observation entries of the simulated bodies
     if (!RESET_ALL) {
         clip = P.clip_id[envc];
         if (clip < 0 || clip >= P.C) {
             clip = min(max(clip, 0), P.C - 1);
-            if (j == 0) atomicOr(P.status, IM_DEV_BAD_STATE);
+            if (c == 0) atomicOr(P.status, IM_DEV_BAD_STATE);
         }
         t1 = __fadd_rn(P.t[envc], P.dt);
         cm = P.meta[clip];
-        stage_joint<true, kRefComps>(P, cm, t1, j, lane, S.ref, S.rootp, S.rootv, ql_ref, wl_ref);
+        int frame;
+        float alpha;
+        lookup(cm, t1, frame, alpha);
+        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
 
-        const size_t st = (size_t)P.stride;
-        p_sim = {P.pos[(3 * j + 0) * st + envc], P.pos[(3 * j + 1) * st + envc], P.pos[(3 * j + 2) * st + envc]};
-        q_sim = {P.quat[(4 * j + 0) * st + envc], P.quat[(4 * j + 1) * st + envc],
-                 P.quat[(4 * j + 2) * st + envc], P.quat[(4 * j + 3) * st + envc]};
-        v_sim = {P.lin[(3 * j + 0) * st + envc], P.lin[(3 * j + 1) * st + envc], P.lin[(3 * j + 2) * st + envc]};
-        w_sim = {P.ang[(3 * j + 0) * st + envc], P.ang[(3 * j + 1) * st + envc], P.ang[(3 * j + 2) * st + envc]};
-        const float n2 = q_sim.w * q_sim.w + q_sim.x * q_sim.x + q_sim.y * q_sim.y + q_sim.z * q_sim.z;
-        if (!(n2 > 1e-12f && n2 < 1e12f)) {
-            q_sim = {1, 0, 0, 0};
-            atomicOr(P.status, IM_DEV_BAD_SIM_QUAT);
+        const Quat q_root = sanitize(ld_sim_quat(P, 0, envc), P.status);
+        const Vec3 p_root = ld_sim_vec(P.pos, P, 0, envc);
+        H = make_heading(q_root, p_root);
+        root_z = p_root.z;
+
+        float acc[kPartials];
+#pragma unroll
+        for (int i = 0; i < kPartials; ++i) acc[i] = 0.0f;
+        Walk s;
+        Quat qa = {1, 0, 0, 0};                      // simulated state of the previous body of the chain
+        Vec3 wa = {0, 0, 0};
+        if (first_own > 0) {
+            const int a = sk.chain[c][first_own - 1];
+            qa = sanitize(ld_sim_quat(P, a, envc), P.status);
+            wa = ld_sim_vec(P.ang, P, a, envc);
         }
-        float *o = S.simx + (j * kSimComps) * kTile + lane;
-        o[0 * kTile] = q_sim.w; o[1 * kTile] = q_sim.x; o[2 * kTile] = q_sim.y; o[3 * kTile] = q_sim.z;
-        o[4 * kTile] = w_sim.x; o[5 * kTile] = w_sim.y; o[6 * kTile] = w_sim.z;
+        for (int k = 0; k < len; ++k) {
+            const int b = sk.chain[c][k];
+            const bool own = k >= first_own;
+            SimBody sim;
+            if (own) {                                // issue the loads before the interpolation math
+                sim.q = ld_sim_quat(P, b, envc);
+                sim.p = ld_sim_vec(P.pos, P, b, envc);
+                sim.v = ld_sim_vec(P.lin, P, b, envc);
+                sim.w = ld_sim_vec(P.ang, P, b, envc);
+            }
+            Quat ql;
+            Vec3 wl;
+            joint_step<true>(sk, r0, r1, alpha, cm.fps, b, k, s, ql, wl);
+            if (own) {
+                sim.q = sanitize(sim.q, P.status);
+                Quat ql_sim = sim.q;
+                Vec3 dw = sim.w;
+                if (b > 0) {
+                    ql_sim = qmul(qconj(qa), sim.q);
+                    dw = sim.w - wa;
+                }
+                const Vec3 wl_sim = qrot_inv(sim.q, dw);
+                const float th_sq = rel_angle_sq(ql, ql_sim);
+                const Vec3 dwl = wl_sim - wl;
+                const Vec3 dp = sim.p - s.p;
+                const Vec3 dv = sim.v - s.v;
+                const float dp2 = dot(dp, dp);
+                acc[0] += th_sq;
+                acc[1] += dot(dwl, dwl);
+                if ((sk.ee_mask >> b) & 1u) {
+                    acc[2] += dp2;
+                    acc[3] += rel_angle_sq(s.q, sim.q);
+                }
+                acc[4] += dp2;
+                acc[5] += dot(dv, dv);
+                const float mf = sk.mass_frac[b];
+                acc[6] += mf * dp.x;
+                acc[7] += mf * dp.y;
+                acc[8] += mf * dp.z;
+                body_obs(H, sim.q, sim.p, sim.v, sim.w, row, b);
+                qa = sim.q;
+                wa = sim.w;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kPartials; ++i) part[(i * C + c) * kTile + lane] = acc[i];
     }
     __syncthreads();
 
-    // ---- phase 2: reference FK, simulated joint-local quantities, per-body error partials
+    // ---- decision: every thread of an env adds the chains' partial sums in chain order and takes
+    //      the same reward, flags and reset draw; chain 0 writes them out
+    int flags = 0;
+    float t_cur = t1;
+    int clip_cur = clip;
     if (!RESET_ALL) {
-        Quat q_ref;
-        Vec3 p_ref, v_ref, w_ref;
-        fk_walk<true, kRefComps>(sk, j, lane, S.ref, S.rootp, S.rootv, q_ref, p_ref, v_ref, w_ref);
-
-        Quat ql_sim = q_sim;
-        Vec3 dw = w_sim;
-        const int a = sk.parent[j];
-        if (a >= 0) {
-            const float *c = S.simx + (a * kSimComps) * kTile + lane;
-            const Quat qa = {c[0 * kTile], c[1 * kTile], c[2 * kTile], c[3 * kTile]};
-            ql_sim = qmul(qconj(qa), q_sim);
-            dw = w_sim - Vec3{c[4 * kTile], c[5 * kTile], c[6 * kTile]};
+        float e[kPartials];
+#pragma unroll
+        for (int i = 0; i < kPartials; ++i) {
+            float a = 0.0f;
+            for (int cc = 0; cc < C; ++cc) a += part[(i * C + cc) * kTile + lane];
+            e[i] = a;
         }
-        const Vec3 wl_sim = qrot_inv(q_sim, dw);
-        const float th = rel_angle(ql_ref, ql_sim);
-        const Vec3 dwl = wl_sim - wl_ref;
-        const Vec3 dp = p_sim - p_ref;
-        const Vec3 dv = v_sim - v_ref;
-        const float dp2 = dot(dp, dp);
-        const bool is_ee = (sk.ee_mask >> j) & 1u;
-        float ee_rot = 0.0f;
-        if (is_ee) { const float th2 = rel_angle(q_ref, q_sim); ee_rot = th2 * th2; }
-        const float mf = sk.mass_frac[j];
-        float *o = S.part + j * kTile + lane;
-        const int ps = J * kTile;
-        o[0 * ps] = th * th;
-        o[1 * ps] = dot(dwl, dwl);
-        o[2 * ps] = is_ee ? dp2 : 0.0f;
-        o[3 * ps] = ee_rot;
-        o[4 * ps] = dp2;
-        o[5 * ps] = dot(dv, dv);
-        o[6 * ps] = mf * dp.x;
-        o[7 * ps] = mf * dp.y;
-        o[8 * ps] = mf * dp.z;
+        // term order of the configuration: pose, vel, ee_pos, ee_rot, com, body_pos, body_vel
+        const float term[IM_N_TERMS] = {e[0], e[1], e[2], e[3], e[6] * e[6] + e[7] * e[7] + e[8] * e[8], e[4], e[5]};
+        float r;
+        if (P.reward.mode == 0) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int k = 0; k < IM_N_TERMS; ++k) sum += P.reward.w[k] * term[k];
+            r = expf(-sum);
+        } else {
+            r = 0.0f;
+#pragma unroll
+            for (int k = 0; k < IM_N_TERMS; ++k) r += P.reward.a[k] * expf(-P.reward.w[k] * term[k]);
+        }
+        const bool terminated = (root_z < P.reward.h_min) || (r < P.reward.r_min);
+        const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
+        flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
+        if (c == 0 && valid) {
+            P.reward_out[env] = r;
+            P.flags_out[env] = (uint8_t)flags;
+            if (P.terms_out) {
+#pragma unroll
+                for (int k = 0; k < IM_N_TERMS; ++k) P.terms_out[(size_t)k * P.N + env] = term[k];
+            }
+        }
     }
-    __syncthreads();
+    const bool reset = RESET_ALL || flags != 0;
+    if (reset) {
+        const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)envc, P.step, IM_STREAM_RESET, 0u),
+                                      make_uint2(P.seed_lo, P.seed_hi));
+        clip_cur = (int)__umulhi(x.x, (uint32_t)P.C);
+        const float u = (float)(x.y >> 8) * 5.9604644775390625e-08f;
+        const float span = fmaxf(__fsub_rn(P.meta[clip_cur].dur, P.dt), 0.0f);
+        t_cur = __fmul_rn(u, span);
+    }
+    if (c == 0 && valid) {
+        P.clip_id[env] = clip_cur;
+        P.t[env] = t_cur;
+        P.ep_len[env] = reset ? 0 : P.ep_len[env] + 1;
+    }
+    const ClipMeta cmc = reset ? P.meta[clip_cur] : cm;
 
-    // ---- phase 3 (warp 0): reduce over bodies, reward, flags, masked reset draw, state update
-    if (j == 0) {
-        int flags = 0;
-        float t_cur = t1;
-        int clip_cur = clip;
-        if (!RESET_ALL) {
-            float e[kPartials];
-            const int ps = J * kTile;
-#pragma unroll
-            for (int k = 0; k < kPartials; ++k) {
-                float acc = 0.0f;
-                for (int b = 0; b < J; ++b) acc += S.part[k * ps + b * kTile + lane];
-                e[k] = acc;
-            }
-            // term order of the configuration: pose, vel, ee_pos, ee_rot, com, body_pos, body_vel
-            const float term[IM_N_TERMS] = {e[0], e[1], e[2], e[3], e[6] * e[6] + e[7] * e[7] + e[8] * e[8], e[4], e[5]};
-            float r;
-            if (P.reward.mode == 0) {
-                float s = 0.0f;
-#pragma unroll
-                for (int k = 0; k < IM_N_TERMS; ++k) s += P.reward.w[k] * term[k];
-                r = expf(-s);
-            } else {
-                r = 0.0f;
-#pragma unroll
-                for (int k = 0; k < IM_N_TERMS; ++k) r += P.reward.a[k] * expf(-P.reward.w[k] * term[k]);
-            }
-            const bool terminated = (p_sim.z < P.reward.h_min) || (r < P.reward.r_min);
-            const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
-            flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
-            if (valid) {
-                P.reward_out[env] = r;
-                P.flags_out[env] = (uint8_t)flags;
-                if (P.terms_out) {
-#pragma unroll
-                    for (int k = 0; k < IM_N_TERMS; ++k) P.terms_out[(size_t)k * P.N + env] = term[k];
+    // ---- pass C (only where an env of this warp was reset): reference state at the new phase
+    //      replaces the simulated one in the observation, and optionally in the caller's arrays
+    if (__any_sync(0xffffffffu, reset)) {
+        int frame;
+        float alpha;
+        lookup(cmc, t_cur, frame, alpha);
+        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
+        Walk s;
+        Heading Hn = H;
+        for (int k = 0; k < len; ++k) {
+            const int b = sk.chain[c][k];
+            Quat ql;
+            Vec3 wl;
+            joint_step<true>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
+            if (k == 0) Hn = make_heading(s.q, s.p);
+            if (k >= first_own && reset) {
+                body_obs(Hn, s.q, s.p, s.v, s.w, row, b);
+                if (!RESET_ALL && P.write_back && valid) {
+                    const size_t st = (size_t)P.stride;
+                    P.pos[(3 * b + 0) * st + env] = s.p.x; P.pos[(3 * b + 1) * st + env] = s.p.y; P.pos[(3 * b + 2) * st + env] = s.p.z;
+                    P.quat[(4 * b + 0) * st + env] = s.q.w; P.quat[(4 * b + 1) * st + env] = s.q.x;
+                    P.quat[(4 * b + 2) * st + env] = s.q.y; P.quat[(4 * b + 3) * st + env] = s.q.z;
+                    P.lin[(3 * b + 0) * st + env] = s.v.x; P.lin[(3 * b + 1) * st + env] = s.v.y; P.lin[(3 * b + 2) * st + env] = s.v.z;
+                    P.ang[(3 * b + 0) * st + env] = s.w.x; P.ang[(3 * b + 1) * st + env] = s.w.y; P.ang[(3 * b + 2) * st + env] = s.w.z;
                 }
             }
         }
-        const bool reset = RESET_ALL || flags != 0;
-        if (reset) {
-            const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)envc, P.step, IM_STREAM_RESET, 0u),
-                                          make_uint2(P.seed_lo, P.seed_hi));
-            clip_cur = (int)__umulhi(x.x, (uint32_t)P.C);
-            const float u = (float)(x.y >> 8) * 5.9604644775390625e-08f;
-            const float span = fmaxf(__fsub_rn(P.meta[clip_cur].dur, P.dt), 0.0f);
-            t_cur = __fmul_rn(u, span);
-        }
-        if (valid) {
-            P.clip_id[env] = clip_cur;
-            P.t[env] = t_cur;
-            P.ep_len[env] = reset ? 0 : P.ep_len[env] + 1;
-        }
-        S.cur_clip[lane] = clip_cur;
-        S.cur_t[lane] = t_cur;
-        S.mask[lane] = reset ? 1 : 0;
-        const unsigned any = __ballot_sync(0xffffffffu, reset);
-        if (lane == 0) *S.any = any != 0u;
+        if (reset) H = Hn;
     }
-    __syncthreads();
 
-    // ---- phase 4: stage the target pose one control interval ahead and, if any env of the
-    //      tile was reset, the reference state at the new phase
-    const int clip_cur = S.cur_clip[lane];
-    const float t_cur = S.cur_t[lane];
-    const bool masked = S.mask[lane] != 0;
-    const bool any_reset = *S.any != 0;
-    const ClipMeta cmc = P.meta[clip_cur];
+    // ---- pass B: reference pose one control interval ahead, seen from the same heading frame
     {
-        Quat qt;
-        Vec3 unused;
+        int frame;
+        float alpha;
         const float t_tgt = fminf(__fadd_rn(t_cur, P.dt), cmc.dur);
-        stage_joint<false, kTgtComps>(P, cmc, t_tgt, j, lane, S.tgt, S.tgt_rootp, nullptr, qt, unused);
-        if (any_reset) {
-            stage_joint<true, kRefComps>(P, cmc, t_cur, j, lane, S.ref, S.rootp, S.rootv, ql_ref, wl_ref);
+        lookup(cmc, t_tgt, frame, alpha);
+        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
+        Walk s;
+        for (int k = 0; k < len; ++k) {
+            const int b = sk.chain[c][k];
+            Quat ql;
+            Vec3 wl;
+            joint_step<false>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
+            if (k >= first_own) {
+                const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
+                const Vec3 tt = H.turn(qcol_x(s.q)), tm = H.turn(qcol_z(s.q));
+                const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
+                store_run<9>(row, 15 * J + 1 + 9 * b, o);
+            }
         }
+        if (c == 0) row[15 * J] = t_cur / cmc.dur;
     }
     __syncthreads();
 
-    // ---- phase 5: target FK; state the observation is built from (simulated, or reference if reset)
-    Quat q_tgt;
-    Vec3 p_tgt, unused_v, unused_w;
-    fk_walk<false, kTgtComps>(sk, j, lane, S.tgt, S.tgt_rootp, nullptr, q_tgt, p_tgt, unused_v, unused_w);
-    Quat qx = q_sim;
-    Vec3 px = p_sim, vx = v_sim, wx = w_sim;
-    if (any_reset) {
-        Quat qn;
-        Vec3 pn, vn, wn;
-        fk_walk<true, kRefComps>(sk, j, lane, S.ref, S.rootp, S.rootv, qn, pn, vn, wn);
-        if (masked) { qx = qn; px = pn; vx = vn; wx = wn; }
-    }
-    if (j == 0) {
-        const Vec3 h = qcol_x(qx);
-        const float n2 = h.x * h.x + h.y * h.y;
-        float hc = 1.0f, hs = 0.0f;
-        if (n2 >= 1e-12f) { const float inv = 1.0f / sqrtf(n2); hc = h.x * inv; hs = h.y * inv; }
-        S.head[0 * kTile + lane] = px.x;
-        S.head[1 * kTile + lane] = px.y;
-        S.head[2 * kTile + lane] = hc;
-        S.head[3 * kTile + lane] = hs;
-    }
-    __syncthreads();
-
-    // ---- phase 6: heading-local observation into the transposed tile
+    // ---- rows of the tile to global memory as 16-byte stores, 512 contiguous bytes per warp store
     {
-        const float ox = S.head[0 * kTile + lane], oy = S.head[1 * kTile + lane];
-        const float hc = S.head[2 * kTile + lane], hs = S.head[3 * kTile + lane];
-        auto turn = [&](Vec3 a) -> Vec3 { return {hc * a.x + hs * a.y, hc * a.y - hs * a.x, a.z}; };
-        float *row = S.tile + (size_t)lane * D;
-        float *o = row + 15 * j;
-        const Vec3 pl = turn(Vec3{px.x - ox, px.y - oy, px.z});
-        const Vec3 tn = turn(qcol_x(qx)), nm = turn(qcol_z(qx));
-        const Vec3 vl = turn(vx), wl = turn(wx);
-        o[0] = pl.x; o[1] = pl.y; o[2] = pl.z;
-        o[3] = tn.x; o[4] = tn.y; o[5] = tn.z;
-        o[6] = nm.x; o[7] = nm.y; o[8] = nm.z;
-        o[9] = vl.x; o[10] = vl.y; o[11] = vl.z;
-        o[12] = wl.x; o[13] = wl.y; o[14] = wl.z;
-        float *g = row + 15 * J + 1 + 9 * j;
-        const Vec3 tp = turn(Vec3{p_tgt.x - ox, p_tgt.y - oy, p_tgt.z});
-        const Vec3 tt = turn(qcol_x(q_tgt)), tm = turn(qcol_z(q_tgt));
-        g[0] = tp.x; g[1] = tp.y; g[2] = tp.z;
-        g[3] = tt.x; g[4] = tt.y; g[5] = tt.z;
-        g[6] = tm.x; g[7] = tm.y; g[8] = tm.z;
-        if (j == 0) row[15 * J] = t_cur / cmc.dur;
-
-        if (!RESET_ALL && P.write_back && masked && valid) {
-            const size_t st = (size_t)P.stride;
-            P.pos[(3 * j + 0) * st + env] = px.x; P.pos[(3 * j + 1) * st + env] = px.y; P.pos[(3 * j + 2) * st + env] = px.z;
-            P.quat[(4 * j + 0) * st + env] = qx.w; P.quat[(4 * j + 1) * st + env] = qx.x;
-            P.quat[(4 * j + 2) * st + env] = qx.y; P.quat[(4 * j + 3) * st + env] = qx.z;
-            P.lin[(3 * j + 0) * st + env] = vx.x; P.lin[(3 * j + 1) * st + env] = vx.y; P.lin[(3 * j + 2) * st + env] = vx.z;
-            P.ang[(3 * j + 0) * st + env] = wx.x; P.ang[(3 * j + 1) * st + env] = wx.y; P.ang[(3 * j + 2) * st + env] = wx.z;
+        const int S4 = S >> 2, ld4 = P.ld_obs >> 2;
+        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
+        for (int r = c; r < kTile; r += C) {
+            const int e = blockIdx.x * kTile + r;
+            if (e >= P.N) break;
+            float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
+            for (int i = lane; i < ld4; i += 32)
+                dst[i] = (i < S4) ? tile4[(size_t)r * S4 + i] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
-    }
-    __syncthreads();
-
-    // ---- phase 7: rows of the tile to global memory, 128 contiguous bytes per warp store
-    for (int r = j; r < kTile; r += J) {
-        const int e = blockIdx.x * kTile + r;
-        if (e >= P.N) break;
-        float *dst = P.obs + (size_t)e * P.ld_obs;
-        const float *src = S.tile + (size_t)r * D;
-        for (int c = lane; c < P.ld_obs; c += 32) dst[c] = (c < D) ? src[c] : 0.0f;
     }
 }
 
 }  // namespace
 
-size_t env_kernel_smem_bytes(int J) { return smem_floats(J) * sizeof(float); }
+size_t env_kernel_smem_bytes(int J, int n_chains) { return smem_floats(J, n_chains) * sizeof(float); }
 
-cudaError_t env_kernel_prepare(int J, size_t smem)
+cudaError_t env_kernel_prepare(size_t smem)
 {
-    (void)J;
-    cudaError_t e = cudaFuncSetAttribute(env_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(env_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool done = false;
+    if (done) return cudaSuccess;
+    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(env_step_kernel<false, 256>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<true, 256>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<false, 1024>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<true, 1024>, attr, (int)smem);
+    done = e == cudaSuccess;
+    return e;
 }
 
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)
 {
-    const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.J);
-    if (reset_all) env_step_kernel<true><<<grid, block, smem, stream>>>(p);
-    else env_step_kernel<false><<<grid, block, smem, stream>>>(p);
+    const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
+    if (block.x <= 256) {
+        if (reset_all) env_step_kernel<true, 256><<<grid, block, smem, stream>>>(p);
+        else env_step_kernel<false, 256><<<grid, block, smem, stream>>>(p);
+    } else {
+        if (reset_all) env_step_kernel<true, 1024><<<grid, block, smem, stream>>>(p);
+        else env_step_kernel<false, 1024><<<grid, block, smem, stream>>>(p);
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }

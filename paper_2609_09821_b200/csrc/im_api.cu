@@ -67,12 +67,24 @@ im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *off
         d.parent[j] = parents[j];
         for (int c = 0; c < 3; ++c) d.off[j][c] = j == 0 ? 0.0f : offsets[3 * j + c];
         d.mass_frac[j] = (float)((masses ? (double)masses[j] : 1.0) / msum);
-        // ancestor chain root .. j
-        int depth = 0;
-        for (int a = j; a > 0; a = parents[a]) ++depth;
-        d.depth[j] = (uint8_t)depth;
-        int a = j;
-        for (int k = depth; k >= 0; --k) { d.chain[j][k] = (uint8_t)a; a = a > 0 ? parents[a] : 0; }
+    }
+    // one root-to-leaf path per leaf; a shared body belongs to the first path that contains it
+    {
+        bool has_child[IM_MAX_BODIES] = {false}, owned[IM_MAX_BODIES] = {false};
+        for (int j = 1; j < J; ++j) has_child[parents[j]] = true;
+        for (int leaf = 0; leaf < J; ++leaf) {
+            if (has_child[leaf]) continue;
+            const int c = d.n_chains++;
+            int depth = 0;
+            for (int a = leaf; a > 0; a = parents[a]) ++depth;
+            d.chain_len[c] = (uint8_t)(depth + 1);
+            int a = leaf;
+            for (int k = depth; k >= 0; --k) { d.chain[c][k] = (uint8_t)a; a = a > 0 ? parents[a] : 0; }
+            int first = 0;
+            while (first <= depth && owned[d.chain[c][first]]) ++first;
+            d.chain_first_own[c] = (uint8_t)first;
+            for (int k = first; k <= depth; ++k) owned[d.chain[c][k]] = true;
+        }
     }
     if (ee_ids && n_ee > 0) {
         for (int i = 0; i < n_ee; ++i) d.ee_mask |= 1u << ee_ids[i];
@@ -174,12 +186,13 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     if (!e) return IM_ERR_ALLOC;
     std::memset(e, 0, sizeof(*e));
     e->skel = skel; e->clips = clips; e->cfg = *cfg; e->stream = (cudaStream_t)cuda_stream; e->D = D;
-    e->smem_bytes = env_kernel_smem_bytes(J);
+    e->smem_bytes = env_kernel_smem_bytes(J, skel->dev.n_chains);
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if ((int)e->smem_bytes > max_smem) { delete e; return IM_ERR_UNSUPPORTED; }
-    if (env_kernel_prepare(J, e->smem_bytes) != cudaSuccess) { delete e; return IM_ERR_CUDA; }
+    // opt in to the device maximum once: environments of different sizes share the kernels
+    if (env_kernel_prepare((size_t)max_smem) != cudaSuccess) { delete e; return IM_ERR_CUDA; }
     const size_t n = (size_t)cfg->n_envs;
     if (cudaMalloc(&e->d_clip_id, n * 4) != cudaSuccess || cudaMalloc(&e->d_t, n * 4) != cudaSuccess ||
         cudaMalloc(&e->d_ep_len, n * 4) != cudaSuccess || cudaMalloc(&e->d_status, 4) != cudaSuccess) {

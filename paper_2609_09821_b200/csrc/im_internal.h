@@ -26,8 +26,12 @@ struct SkelDev {
     int32_t parent[IM_MAX_BODIES];
     float off[IM_MAX_BODIES][3];
     float mass_frac[IM_MAX_BODIES];                    // m_j / sum m
-    uint8_t depth[IM_MAX_BODIES];                      // number of ancestors
-    uint8_t chain[IM_MAX_BODIES][IM_MAX_BODIES];       // chain[j][0..depth[j]] = root .. j
+    // Kinematic chains: one root-to-leaf path per leaf.  A body shared by several paths is owned
+    // by the first of them; within a path the owned bodies are a suffix starting at chain_first_own.
+    int32_t n_chains;
+    uint8_t chain_len[IM_MAX_BODIES];
+    uint8_t chain_first_own[IM_MAX_BODIES];
+    uint8_t chain[IM_MAX_BODIES][IM_MAX_BODIES];       // chain[c][0..chain_len[c]) = root .. leaf
 };
 
 struct EnvKernelParams {
@@ -95,7 +99,7 @@ struct im_env {
 
 // Launchers implemented in the kernel translation units.
 namespace im {
-size_t env_kernel_smem_bytes(int J);
-cudaError_t env_kernel_prepare(int J, size_t smem);
+size_t env_kernel_smem_bytes(int J, int n_chains);
+cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
 }  // namespace im
