@@ -10,10 +10,9 @@
 // and "owned" by one path, which alone loads their simulated state, scores them
 // and writes their observation entries.  Every global load of the
 // structure-of-arrays body state is one fully used 128-byte line per warp.
-// The observation tile [32][D] is assembled in shared memory (row stride 4 x odd:
-// conflict-free 16-byte column writes, 16-byte aligned rows) and written out
-// as whole lines.  Two block-wide barriers per tile: after the reward partial
-// sums, and before the tile is stored.
+// The observation rows of the 32 envs are assembled in shared memory in two
+// halves that reuse the same space (row stride 4 x odd: conflict-free 16-byte
+// column writes, 16-byte aligned rows) and written out as whole lines.
 #include "im_internal.h"
 #include "im_device.cuh"
 
@@ -31,10 +30,15 @@ __host__ __device__ inline int tile_stride(int D)
     return 4 * s4;
 }
 
+// The observation row is staged in two halves; the split is the end of the body blocks rounded
+// up to a multiple of four columns so that both halves start on a 16-byte boundary.
+__host__ __device__ inline int split_col(int J) { return (15 * J + 3) / 4 * 4; }
+
 __host__ __device__ inline size_t smem_floats(int J, int n_chains)
 {
-    const int D = 24 * J + 1;
-    return (size_t)kTile * tile_stride(D) + (size_t)kPartials * n_chains * kTile;
+    const int D = 24 * J + 1, c1 = split_col(J);
+    const int s1 = tile_stride(c1), s2 = tile_stride(D - c1);
+    return (size_t)kTile * (s1 > s2 ? s1 : s2) + (size_t)kPartials * n_chains * kTile;
 }
 
 // Keyframe row and blend factor at `time` (step a1): f = fl32(time * fps),
@@ -147,10 +151,10 @@ struct Walk {
 // One link of the chain: interpolate joint b between keyframe rows r0/r1 and
 // compose it onto the running transform.  k == 0 is the root.
 template <bool VEL>
-__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, float alpha,
-                                           float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
+__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, Quat k0, Quat k1,
+                                           float alpha, float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
 {
-    slerp_joint<VEL>(ld_quat(r0 + 1 + b), ld_quat(r1 + 1 + b), alpha, fps, ql, wl);
+    slerp_joint<VEL>(k0, k1, alpha, fps, ql, wl);
     if (k == 0) {
         const float4 a = __ldg(r0), c = __ldg(r1);
         s.q = ql;
@@ -250,16 +254,27 @@ __device__ __forceinline__ Vec3 ld_sim_vec(const float *base, const EnvKernelPar
     return {base[(3 * b + 0) * st + e], base[(3 * b + 1) * st + e], base[(3 * b + 2) * st + e]};
 }
 
-// MAXT: largest block the instantiation may be launched with (32 threads per chain); skeletons with
-// at most 8 leaves use the variant that leaves the compiler more registers per thread.
-template <bool RESET_ALL, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant__ EnvKernelParams P)
+// Keyframe quaternions of joint b in the two bracketing rows.
+struct KeyPair {
+    float4 a, b;
+};
+__device__ __forceinline__ KeyPair ld_keys(const float4 *r0, const float4 *r1, int b)
 {
-    extern __shared__ __align__(16) float smem_raw[];
+    return {__ldg(r0 + 1 + b), __ldg(r1 + 1 + b)};
+}
+__device__ __forceinline__ Quat as_quat(float4 v) { return {v.x, v.y, v.z, v.w}; }
+
+// Kernel body.  The observation row is assembled in two halves that reuse the same shared
+// memory: columns [0, c1) -- the body blocks and, if 15 J is not a multiple of 4, the phase and
+// the first target floats -- and columns [c1, D) -- the targets.
+template <bool RESET_ALL>
+__device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
+{
     const SkelDev &sk = P.sk;
     const int J = sk.J;
     const int D = 24 * J + 1;
-    const int S = tile_stride(D);
+    const int c1 = split_col(J);                    // multiple of 4
+    const int S1 = tile_stride(c1), S2 = tile_stride(D - c1);
     const int C = sk.n_chains;
     const int lane = threadIdx.x & 31;
     const int c = threadIdx.x >> 5;                 // this thread's chain
@@ -267,14 +282,15 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
     const bool valid = env < P.N;
     const int envc = valid ? env : P.N - 1;
     float *tile = smem_raw;
-    float *part = smem_raw + (size_t)kTile * S;
-    float *row = tile + (size_t)lane * S;
+    float *part = smem_raw + (size_t)kTile * (S1 > S2 ? S1 : S2);
+    float *row1 = tile + (size_t)lane * S1;
+    float *row2 = tile + (size_t)lane * S2;
     const int len = sk.chain_len[c];
     const int first_own = sk.chain_first_own[c];
     const int RS = J + 1;
 
     if (c == 0)
-        for (int i = D; i < S; ++i) row[i] = 0.0f;  // columns between D and the row stride
+        for (int i = 15 * J; i < S1; ++i) row1[i] = 0.0f;   // columns between the body blocks and the stride
 
     int clip = 0;
     float t1 = 0.0f;
@@ -296,6 +312,7 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
         float alpha;
         lookup(cm, t1, frame, alpha);
         const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
+        KeyPair keys = ld_keys(r0, r1, sk.chain[c][0]);
 
         const Quat q_root = sanitize(ld_sim_quat(P, 0, envc), P.status);
         const Vec3 p_root = ld_sim_vec(P.pos, P, 0, envc);
@@ -323,9 +340,11 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
                 sim.v = ld_sim_vec(P.lin, P, b, envc);
                 sim.w = ld_sim_vec(P.ang, P, b, envc);
             }
+            const KeyPair cur = keys;
+            if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);     // next joint's keyframes in flight
             Quat ql;
             Vec3 wl;
-            joint_step<true>(sk, r0, r1, alpha, cm.fps, b, k, s, ql, wl);
+            joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cm.fps, b, k, s, ql, wl);
             if (own) {
                 sim.q = sanitize(sim.q, P.status);
                 Quat ql_sim = sim.q;
@@ -352,7 +371,7 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
                 acc[6] += mf * dp.x;
                 acc[7] += mf * dp.y;
                 acc[8] += mf * dp.z;
-                body_obs(H, sim.q, sim.p, sim.v, sim.w, row, b);
+                body_obs(H, sim.q, sim.p, sim.v, sim.w, row1, b);
                 qa = sim.q;
                 wa = sim.w;
             }
@@ -423,16 +442,19 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
         float alpha;
         lookup(cmc, t_cur, frame, alpha);
         const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
+        KeyPair keys = ld_keys(r0, r1, sk.chain[c][0]);
         Walk s;
         Heading Hn = H;
         for (int k = 0; k < len; ++k) {
             const int b = sk.chain[c][k];
+            const KeyPair cur = keys;
+            if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);
             Quat ql;
             Vec3 wl;
-            joint_step<true>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
+            joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, b, k, s, ql, wl);
             if (k == 0) Hn = make_heading(s.q, s.p);
             if (k >= first_own && reset) {
-                body_obs(Hn, s.q, s.p, s.v, s.w, row, b);
+                body_obs(Hn, s.q, s.p, s.v, s.w, row1, b);
                 if (!RESET_ALL && P.write_back && valid) {
                     const size_t st = (size_t)P.stride;
                     P.pos[(3 * b + 0) * st + env] = s.p.x; P.pos[(3 * b + 1) * st + env] = s.p.y; P.pos[(3 * b + 2) * st + env] = s.p.z;
@@ -446,42 +468,99 @@ __global__ void __launch_bounds__(MAXT, 1) env_step_kernel(const __grid_constant
         if (reset) H = Hn;
     }
 
-    // ---- pass B: reference pose one control interval ahead, seen from the same heading frame
-    {
-        int frame;
-        float alpha;
-        const float t_tgt = fminf(__fadd_rn(t_cur, P.dt), cmc.dur);
-        lookup(cmc, t_tgt, frame, alpha);
-        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
+    // ---- the first half also holds the phase and the first floats of the root's target when 15 J
+    //      is not a multiple of 4: chain 0 interpolates the root one interval ahead for them
+    const float t_tgt = fminf(__fadd_rn(t_cur, P.dt), cmc.dur);
+    int frame_t;
+    float alpha_t;
+    lookup(cmc, t_tgt, frame_t, alpha_t);
+    const float4 *rt0 = P.frames + (size_t)frame_t * RS, *rt1 = rt0 + RS;
+    const float phase = t_cur / cmc.dur;
+    if (c == 0 && 15 * J < c1) {
         Walk s;
-        for (int k = 0; k < len; ++k) {
-            const int b = sk.chain[c][k];
-            Quat ql;
-            Vec3 wl;
-            joint_step<false>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
-            if (k >= first_own) {
-                const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
-                const Vec3 tt = H.turn(qcol_x(s.q)), tm = H.turn(qcol_z(s.q));
-                const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
-                store_run<9>(row, 15 * J + 1 + 9 * b, o);
-            }
-        }
-        if (c == 0) row[15 * J] = t_cur / cmc.dur;
+        Quat ql;
+        Vec3 wl;
+        const KeyPair kp = ld_keys(rt0, rt1, 0);
+        joint_step<false>(sk, rt0, rt1, as_quat(kp.a), as_quat(kp.b), alpha_t, cmc.fps, 0, 0, s, ql, wl);
+        const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
+        row1[15 * J] = phase;
+        if (15 * J + 1 < c1) row1[15 * J + 1] = tp.x;
+        if (15 * J + 2 < c1) row1[15 * J + 2] = tp.y;
     }
     __syncthreads();
 
-    // ---- rows of the tile to global memory as 16-byte stores, 512 contiguous bytes per warp store
+    // ---- first half of the rows to global memory, 16-byte stores, 512 contiguous bytes per warp store
     {
-        const int S4 = S >> 2, ld4 = P.ld_obs >> 2;
+        const int n4 = c1 >> 2, S4 = S1 >> 2;
         const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
         for (int r = c; r < kTile; r += C) {
             const int e = blockIdx.x * kTile + r;
             if (e >= P.N) break;
             float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
-            for (int i = lane; i < ld4; i += 32)
-                dst[i] = (i < S4) ? tile4[(size_t)r * S4 + i] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (int i = lane; i < n4; i += 32) dst[i] = tile4[(size_t)r * S4 + i];
         }
     }
+    __syncthreads();
+
+    // ---- pass B: reference pose one control interval ahead, seen from the same heading frame,
+    //      into the second half (which reuses the shared memory of the first)
+    {
+        if (c == 0) {
+            for (int i = D - c1; i < S2; ++i) row2[i] = 0.0f;
+            if (15 * J >= c1) row2[15 * J - c1] = phase;
+        }
+        KeyPair keys = ld_keys(rt0, rt1, sk.chain[c][0]);
+        Walk s;
+        for (int k = 0; k < len; ++k) {
+            const int b = sk.chain[c][k];
+            const KeyPair cur = keys;
+            if (k + 1 < len) keys = ld_keys(rt0, rt1, sk.chain[c][k + 1]);
+            Quat ql;
+            Vec3 wl;
+            joint_step<false>(sk, rt0, rt1, as_quat(cur.a), as_quat(cur.b), alpha_t, cmc.fps, b, k, s, ql, wl);
+            if (k >= first_own) {
+                const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
+                const Vec3 tt = H.turn(qcol_x(s.q)), tm = H.turn(qcol_z(s.q));
+                const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
+                const int col = 15 * J + 1 + 9 * b;
+                if (col >= c1) {
+                    store_run<9>(row2, col - c1, o);
+                } else {                          // the root's block straddles the split
+#pragma unroll
+                    for (int i = 0; i < 9; ++i)
+                        if (col + i >= c1) row2[col + i - c1] = o[i];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    {
+        const int n4 = c1 >> 2, S4 = S2 >> 2, ld4 = P.ld_obs >> 2;
+        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
+        for (int r = c; r < kTile; r += C) {
+            const int e = blockIdx.x * kTile + r;
+            if (e >= P.N) break;
+            float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
+            for (int i = n4 + lane; i < ld4; i += 32)
+                dst[i] = (i - n4 < S4) ? tile4[(size_t)r * S4 + i - n4] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+    }
+}
+
+// Two instantiations per mode: skeletons with at most 8 leaves (blocks of up to 256 threads) get a
+// register budget that lets four blocks share an SM; wider trees fall back to 64 registers.
+template <bool RESET_ALL>
+__global__ void __maxnreg__(96) env_step_kernel_small(const __grid_constant__ EnvKernelParams P)
+{
+    extern __shared__ __align__(16) float smem_raw[];
+    env_step_body<RESET_ALL>(P, smem_raw);
+}
+
+template <bool RESET_ALL>
+__global__ void __launch_bounds__(1024, 1) env_step_kernel_wide(const __grid_constant__ EnvKernelParams P)
+{
+    extern __shared__ __align__(16) float smem_raw[];
+    env_step_body<RESET_ALL>(P, smem_raw);
 }
 
 }  // namespace
@@ -493,10 +572,10 @@ cudaError_t env_kernel_prepare(size_t smem)
     static bool done = false;
     if (done) return cudaSuccess;
     const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(env_step_kernel<false, 256>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<true, 256>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<false, 1024>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel<true, 1024>, attr, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(env_step_kernel_small<false>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_small<true>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<false>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<true>, attr, (int)smem);
     done = e == cudaSuccess;
     return e;
 }
@@ -505,11 +584,11 @@ cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t s
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
     if (block.x <= 256) {
-        if (reset_all) env_step_kernel<true, 256><<<grid, block, smem, stream>>>(p);
-        else env_step_kernel<false, 256><<<grid, block, smem, stream>>>(p);
+        if (reset_all) env_step_kernel_small<true><<<grid, block, smem, stream>>>(p);
+        else env_step_kernel_small<false><<<grid, block, smem, stream>>>(p);
     } else {
-        if (reset_all) env_step_kernel<true, 1024><<<grid, block, smem, stream>>>(p);
-        else env_step_kernel<false, 1024><<<grid, block, smem, stream>>>(p);
+        if (reset_all) env_step_kernel_wide<true><<<grid, block, smem, stream>>>(p);
+        else env_step_kernel_wide<false><<<grid, block, smem, stream>>>(p);
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
