@@ -235,6 +235,37 @@ im_status im_poll_device_status(im_env *e, im_policy *p, uint32_t *out);
 /* Number of kernel launches the library has enqueued since it was loaded. */
 uint64_t im_launch_count(void);
 
+/* ---- allocation-free policy forward ------------------------------------------
+ * (The paper has no counterpart of this call; it exists for deployment.)
+ * For callers that may not allocate device memory when they need an action: a
+ * control loop that cannot afford an allocation's device-wide stall, a process
+ * whose memory was all handed out at start-up, a plug-in living inside another
+ * program's allocator.  The fp32 policy chain of im_policy_forward (same
+ * kernels, same results) runs on weights the CALLER keeps in device memory,
+ * and the only memory the library adds -- the hidden activations -- is a fixed
+ * array inside the library image, IM_NOALLOC_SCRATCH_BYTES per GPU that loads
+ * the library, held until the process exits.  The call allocates and frees
+ * nothing and needs no handle.
+ *   dims        HOST [n_layers + 1]
+ *   W, b        HOST arrays of n_layers DEVICE pointers: W[l] float [dims[l+1]][dims[l]], b[l] float [dims[l+1]]
+ *   obs         DEVICE [n][ld_obs] float       mean_out, action_out DEVICE [n][A]    logp_out DEVICE [n] or NULL
+ *   cuda_stream cudaStream_t the work is enqueued on
+ * Limits: n <= IM_NOALLOC_MAX_BATCH and hidden widths <= IM_NOALLOC_MAX_WIDTH; beyond them the call
+ * returns IM_ERR_UNSUPPORTED and does nothing.
+ * The first call on each device looks up the array's device address (a query, not an allocation);
+ * make that first call outside any stream capture, with the device that will run it current.
+ * All calls on a device share the one array: it keeps whatever the last call left (nothing in it
+ * needs clearing, every value read is written first by the same call), and two calls whose work
+ * overlaps on the GPU -- different streams, or replays of graphs containing it -- race on it.
+ * Run them on one stream. */
+#define IM_NOALLOC_MAX_BATCH  1024
+#define IM_NOALLOC_MAX_WIDTH  1024
+#define IM_NOALLOC_SCRATCH_BYTES (2u * IM_NOALLOC_MAX_BATCH * IM_NOALLOC_MAX_WIDTH * 4u)   /* 8 MiB */
+im_status im_policy_forward_noalloc(int32_t n_layers, const int32_t *dims, const float *const *W,
+                                    const float *const *b, float sigma, uint64_t seed, uint32_t env_id_base,
+                                    uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
+                                    float *mean_out, float *action_out, float *logp_out, void *cuda_stream);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

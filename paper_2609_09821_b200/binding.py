@@ -23,6 +23,7 @@ EXPORTS = [
     "im_env_create", "im_env_destroy", "im_env_reset_all", "im_env_step", "im_env_get_state",
     "im_env_set_state", "im_load_policy", "im_destroy_policy", "im_policy_forward",
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
+    "im_policy_forward_noalloc",
 ]
 
 
@@ -84,6 +85,7 @@ def load():
         L.im_step_host.argtypes = [vp, vp, u32, vp, vp, vp, vp]
         L.im_poll_device_status.argtypes = [vp, vp, C.POINTER(u32)]
         L.im_launch_count.restype = u64
+        L.im_policy_forward_noalloc.argtypes = [i32, vp, vp, vp, C.c_float, u64, u32, u32, i32, vp, i32, vp, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("im_status_string", "im_launch_count") and not name.startswith("im_destroy") \
                     and name != "im_env_destroy":
@@ -270,3 +272,29 @@ def step_host(env: Env, policy: Policy, step: int, sim_host, action_host, reward
     """One whole step from host buffers (numpy arrays or pinned CPU torch tensors)."""
     _check(load().im_step_host(env.h, policy.h, step, _ptr(sim_host), _ptr(action_host), _ptr(reward_host),
                                _ptr(flags_host)), "im_step_host")
+
+
+NOALLOC_MAX_BATCH = 1024
+NOALLOC_MAX_WIDTH = 1024
+
+
+def policy_forward_noalloc(dims: Sequence[int], W_dev, b_dev, sigma: float, seed: int, step: int, obs,
+                           mean_out, action_out, logp_out=None, env_id_base: int = 0, n: Optional[int] = None,
+                           stream=None):
+    """fp32 policy forward that allocates nothing: for callers that cannot call cudaMalloc when they
+    need an action (latency-bound control loops, processes with a fixed memory budget).  W_dev and
+    b_dev are lists of CUDA float32 tensors the caller owns; the hidden activations live in a fixed
+    8 MiB array inside the library, shared by all calls on the device, so calls must not overlap on
+    the GPU.  At most NOALLOC_MAX_BATCH rows and hidden widths up to NOALLOC_MAX_WIDTH."""
+    import torch
+    L = load()
+    nl = len(dims) - 1
+    d = np.asarray(dims, np.int32)
+    Wp = (C.c_void_p * nl)(*[w.data_ptr() for w in W_dev])
+    bp = (C.c_void_p * nl)(*[x.data_ptr() for x in b_dev])
+    st = stream if stream is not None else torch.cuda.current_stream()
+    n = obs.shape[0] if n is None else n
+    _check(L.im_policy_forward_noalloc(nl, _ptr(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p),
+                                       C.c_float(sigma), int(seed), int(env_id_base), int(step), int(n),
+                                       _ptr(obs), obs.stride(0), _ptr(mean_out), _ptr(action_out),
+                                       _ptr(logp_out), C.c_void_p(st.cuda_stream)), "im_policy_forward_noalloc")
