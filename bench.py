@@ -202,6 +202,16 @@ def main():
     policy = B.Policy(pol["dims"], Wg, pol["b"], pol["dtype"], wl.sigma_action, wl.seed, n, env_id_base=env_base,
                       stream=stream)
     A = wl.act_dim
+    staged = pol["dtype"] == "bf16"            # env writes bf16 rows straight into the policy's input buffer
+    if staged:
+        env.attach_policy(policy)
+
+    def policy_forward(s):
+        if staged:
+            policy.forward_staged(s, n, mean, action)
+        else:
+            policy.forward(s, obs, mean, action)
+
     obs = env.new_obs()
     reward = torch.empty(n, device=dev)
     flags = torch.empty(n, dtype=torch.uint8, device=dev)
@@ -219,7 +229,7 @@ def main():
         return c, t
 
     def consume(s, sim):
-        policy.forward(s, obs, mean, action)
+        policy_forward(s)
         env.step(s, sim, obs, reward, flags)
 
     sims = W.rollout_inputs(wl, skel, lib, get_state, consume, steps=n_buf, env_base=env_base, device=str(dev))
@@ -230,7 +240,7 @@ def main():
     def run_steps(first, count):
         for i in range(count):
             s = first + i
-            policy.forward(s, obs, mean, action)
+            policy_forward(s)
             env.step(s, sims[(s - 1) % n_buf], obs, reward, flags)
 
     def barrier():
@@ -283,7 +293,7 @@ def main():
     for i in range(K):
         s = Wm + 1 + i
         evs[i][0].record(stream)
-        policy.forward(s, obs, mean, action)
+        policy_forward(s)
         evs[i][1].record(stream)
         env.step(s, sims[(s - 1) % n_buf], obs, reward, flags)
         evs[i][2].record(stream)
@@ -327,7 +337,7 @@ def main():
     tf = flops / t_pol / 1e12
     gbs = env_bytes / t_env / 1e9
     tensor_peak = peaks["bf16_tflops_sustained"]
-    roofline = dict(bound="tensor", kernel="policy forward (convert + GEMM chain + sampling)", achieved=tf,
+    roofline = dict(bound="tensor", kernel="policy forward (GEMM chain + Gaussian head)", achieved=tf,
                     peak=tensor_peak, unit="TFLOP/s", frac=tf / tensor_peak, traffic=None,
                     peak_source="%s bf16 sustained" % peaks["source"], seconds_per_launch=t_pol)
     roofline_env = dict(bound="hbm", kernel="env_step_kernel", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",

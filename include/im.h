@@ -214,6 +214,20 @@ void im_destroy_policy(im_policy *p);
 im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out);
 
+/* ---- env -> policy staging ----------------------------------------------------
+ * The tensor-core policy consumes bf16 observations.  An env attached to such a
+ * policy writes, besides the fp32 rows the caller asked for, the same rows
+ * rounded to bf16 (nearest even) straight into the policy's input staging
+ * buffer during im_env_reset_all / im_env_step, and im_policy_forward_staged
+ * then runs the policy on rows [0, n) of that buffer -- the same result as
+ * im_policy_forward on the fp32 rows, without the conversion pass over the
+ * observations.  Requirements: tensor-core policy, same stream, policy input
+ * width 24J+1, max_batch >= N, and ld_obs equal to 24J+1 rounded up to a
+ * multiple of 64.  Passing NULL detaches. */
+im_status im_env_attach_policy(im_env *e, im_policy *p);
+im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n,
+                                   float *mean_out, float *action_out, float *logp_out);
+
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current

@@ -23,7 +23,7 @@ EXPORTS = [
     "im_env_create", "im_env_destroy", "im_env_reset_all", "im_env_step", "im_env_get_state",
     "im_env_set_state", "im_load_policy", "im_destroy_policy", "im_policy_forward",
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
-    "im_policy_forward_noalloc",
+    "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
 ]
 
 
@@ -85,6 +85,8 @@ def load():
         L.im_step_host.argtypes = [vp, vp, u32, vp, vp, vp, vp]
         L.im_poll_device_status.argtypes = [vp, vp, C.POINTER(u32)]
         L.im_launch_count.restype = u64
+        L.im_env_attach_policy.argtypes = [vp, vp]
+        L.im_policy_forward_staged.argtypes = [vp, u32, i32, vp, vp, vp]
         L.im_policy_forward_noalloc.argtypes = [i32, vp, vp, vp, C.c_float, u64, u32, u32, i32, vp, i32, vp, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("im_status_string", "im_launch_count") and not name.startswith("im_destroy") \
@@ -213,6 +215,10 @@ class Env:
         _check(load().im_env_set_state(self.h, _ptr(clip_id), _ptr(t), _ptr(ep_len)), "im_env_set_state")
         self.stream.synchronize()
 
+    def attach_policy(self, policy):
+        """The env also writes bf16 observation rows into the policy's input staging buffer."""
+        _check(load().im_env_attach_policy(self.h, None if policy is None else policy.h), "im_env_attach_policy")
+
     def reset_all_host(self, step: int = 0):
         _check(load().im_env_reset_all_host(self.h, step), "im_env_reset_all_host")
 
@@ -256,6 +262,11 @@ class Policy:
         n = obs.shape[0] if n is None else n
         _check(load().im_policy_forward(self.h, step, n, _ptr(obs), obs.stride(0), _ptr(mean_out),
                                         _ptr(action_out), _ptr(logp_out)), "im_policy_forward")
+
+    def forward_staged(self, step: int, n: int, mean_out, action_out, logp_out=None):
+        """Forward on the bf16 rows an attached env left in the input staging buffer."""
+        _check(load().im_policy_forward_staged(self.h, step, n, _ptr(mean_out), _ptr(action_out), _ptr(logp_out)),
+               "im_policy_forward_staged")
 
     def device_status(self) -> int:
         out = C.c_uint32(0)

@@ -13,12 +13,21 @@
 // The observation rows of the 32 envs are assembled in shared memory in two
 // halves that reuse the same space (row stride 4 x odd: conflict-free 16-byte
 // column writes, 16-byte aligned rows) and written out as whole lines.
+#include <cuda_bf16.h>
+
 #include "im_internal.h"
 #include "im_device.cuh"
 
 namespace im {
 
 namespace {
+
+// Four floats rounded to bf16 (nearest even), packed in column order.
+__device__ __forceinline__ uint2 pack_bf16x4(float4 v)
+{
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    return make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
+}
 
 constexpr int kTile = 32;          // envs per CTA
 constexpr int kPartials = 9;       // pose, vel, ee_pos, ee_rot, body_pos, body_vel, weighted com difference (3)
@@ -497,7 +506,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             const int e = blockIdx.x * kTile + r;
             if (e >= P.N) break;
             float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
-            for (int i = lane; i < n4; i += 32) dst[i] = tile4[(size_t)r * S4 + i];
+            uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
+            for (int i = lane; i < n4; i += 32) {
+                const float4 v = tile4[(size_t)r * S4 + i];
+                dst[i] = v;
+                if (dst16) dst16[i] = pack_bf16x4(v);
+            }
         }
     }
     __syncthreads();
@@ -541,8 +555,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             const int e = blockIdx.x * kTile + r;
             if (e >= P.N) break;
             float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
-            for (int i = n4 + lane; i < ld4; i += 32)
-                dst[i] = (i - n4 < S4) ? tile4[(size_t)r * S4 + i - n4] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
+            for (int i = n4 + lane; i < ld4; i += 32) {
+                const float4 v = (i - n4 < S4) ? tile4[(size_t)r * S4 + i - n4] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                dst[i] = v;
+                if (dst16) dst16[i] = pack_bf16x4(v);
+            }
         }
     }
 }

@@ -236,6 +236,7 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.t = e->d_t;
     p.ep_len = e->d_ep_len;
     p.status = e->d_status;
+    p.obs_bf16 = e->d_obs_bf16;
 }
 
 im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out)
@@ -263,6 +264,19 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float 
     p.stride = sim->comp_stride;
     p.obs = obs_out; p.reward_out = reward_out; p.flags_out = flags_out; p.terms_out = terms_out;
     IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_attach_policy(im_env *e, im_policy *p)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    if (!p) { e->d_obs_bf16 = nullptr; return IM_OK; }
+    if (!p->tensor_path) return IM_ERR_UNSUPPORTED;
+    int32_t ld = 0;
+    void *buf = tc_policy_input(p, &ld);
+    if (ld != e->cfg.ld_obs || p->cfg.dims[0] != e->D || p->cfg.max_batch < e->cfg.n_envs || p->stream != e->stream)
+        return IM_ERR_INVALID_ARG;
+    e->d_obs_bf16 = static_cast<uint16_t *>(buf);
     return IM_OK;
 }
 
@@ -376,6 +390,15 @@ im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
     return IM_OK;
 }
 
+im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n, float *mean_out, float *action_out,
+                                   float *logp_out)
+{
+    if (!p || !mean_out || !action_out) return IM_ERR_INVALID_ARG;
+    if (!p->tensor_path) return IM_ERR_UNSUPPORTED;
+    if (n < 1 || n > p->cfg.max_batch || !aligned16(mean_out) || !aligned16(action_out)) return IM_ERR_INVALID_ARG;
+    return tc_policy_forward(p, step, n, nullptr, 0, mean_out, action_out, logp_out);
+}
+
 /* ------------------------------------------------------------------ host-buffer step */
 static im_status ensure_staging(im_env *e, int A)
 {
@@ -416,7 +439,11 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     if (s != IM_OK) return s;
     const size_t n = (size_t)e->cfg.n_envs, J = (size_t)e->skel->dev.J;
     IM_CUDA(cudaMemcpyAsync(e->d_sim, sim_host, 13 * J * n * 4, cudaMemcpyHostToDevice, e->stream));
-    s = im_policy_forward(p, step, (int32_t)n, e->d_obs, e->cfg.ld_obs, e->d_mean, e->d_action, nullptr);
+    int32_t ld_in = 0;
+    if (e->d_obs_bf16 && p->tensor_path && e->d_obs_bf16 == tc_policy_input(p, &ld_in))
+        s = im_policy_forward_staged(p, step, (int32_t)n, e->d_mean, e->d_action, nullptr);
+    else
+        s = im_policy_forward(p, step, (int32_t)n, e->d_obs, e->cfg.ld_obs, e->d_mean, e->d_action, nullptr);
     if (s != IM_OK) return s;
     im_body_state sim = {e->d_sim, e->d_sim + 3 * J * n, e->d_sim + 7 * J * n, e->d_sim + 10 * J * n, (int64_t)n};
     s = im_env_step(e, step, &sim, e->d_obs, e->d_reward, e->d_flags, nullptr);

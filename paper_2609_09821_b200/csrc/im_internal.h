@@ -57,6 +57,7 @@ struct EnvKernelParams {
     float *pos, *quat, *lin, *ang;
     long long stride;
     float *obs;
+    uint16_t *obs_bf16;       // optional bf16 copy of the observation rows (same row stride), or null
     float *reward_out;
     uint8_t *flags_out;
     float *terms_out;
@@ -91,6 +92,7 @@ struct im_env {
     uint32_t *d_status;
     int D;                 // 24J + 1
     size_t smem_bytes;
+    uint16_t *d_obs_bf16;  // attached policy's bf16 input rows (null when detached)
     // staging for the *_host entry points (allocated on first use)
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
     uint8_t *d_flags;

@@ -735,12 +735,19 @@ void tc_policy_destroy(im_policy *p)
     p->tc = nullptr;
 }
 
+void *tc_policy_input(im_policy *p, int32_t *ld)
+{
+    *ld = p->tc->ld_in;
+    return p->tc->d_in;
+}
+
+// obs == nullptr: the bf16 input buffer has already been filled (by an attached environment).
 im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out)
 {
     im_policy_tc *tc = p->tc;
     const im_policy_config &cfg = p->cfg;
-    {
+    if (obs) {
         const long long chunks = (long long)n * (tc->ld_in / 8);
         const int block = 256;
         long long grid = (chunks + block - 1) / block;

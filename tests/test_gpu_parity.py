@@ -221,6 +221,28 @@ def test_host_buffer_step_matches_device_step(scenes):
         assert torch.equal(act, p.action_g.cpu()) and torch.equal(rew, p.reward_g.cpu()) and torch.equal(fl, p.flags_g.cpu())
 
 
+def test_staged_policy_input_matches_the_conversion_pass(scenes):
+    """An env attached to a tensor-core policy leaves bf16 observation rows in the policy's input
+    buffer; the policy run on them must equal the policy run on the fp32 rows bit for bit."""
+    sc = scenes("cfg4_65536_smpl24")
+    n = 700
+    p = Pair(sc, n)
+    p.g_env.attach_policy(p.policy)
+    p.reset_all()
+    mean2 = torch.empty_like(p.mean_g)
+    act2 = torch.empty_like(p.action_g)
+    logp2 = torch.empty_like(p.logp_g)
+    for s in (1, 2, 3):
+        p.policy_step(s)                                              # fp32 rows through the conversion pass
+        p.policy.forward_staged(s, n, mean2, act2, logp2)              # bf16 rows written by the env kernel
+        torch.cuda.synchronize()
+        assert torch.equal(mean2, p.mean_g) and torch.equal(act2, p.action_g) and torch.equal(logp2, p.logp_g)
+        sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                      torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, s, sc.wl)
+        p.env_step(s, sim)
+    p.g_env.attach_policy(None)
+
+
 def test_reset_draws_bit_exact_over_many_counters(scenes):
     sc = scenes("cfg3_16384_lib32")
     n = 100000
