@@ -232,8 +232,10 @@ im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n,
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current
  * observation and then im_env_step, and copies action, reward and flags back,
- * all on the env's stream, then waits for the stream.  The first call
- * allocates the device staging buffers (so it is not capturable).  Call
+ * then waits until everything has arrived.  The upload runs beside the policy
+ * forward and the actions travel back beside the env step (two internal copy
+ * streams); the kernels run on the env's stream.  The first call allocates the
+ * device staging buffers and the copy streams (so it is not capturable).  Call
  * im_env_reset_all_host first.  sim_host is [13J][N] (pos rows, quat rows,
  * linvel rows, angvel rows); pinned memory gives the copies full speed.
  *   action_host HOST [N][A]   reward_host HOST [N]   flags_host HOST [N] */

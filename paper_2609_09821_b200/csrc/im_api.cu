@@ -213,6 +213,10 @@ void im_env_destroy(im_env *e)
     cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status);
     cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
     cudaFree(e->d_action); cudaFree(e->d_flags);
+    if (e->h2d_stream) cudaStreamDestroy(e->h2d_stream);
+    if (e->d2h_stream) cudaStreamDestroy(e->d2h_stream);
+    if (e->ev_h2d) cudaEventDestroy(e->ev_h2d);
+    if (e->ev_policy) cudaEventDestroy(e->ev_policy);
     delete e;
 }
 
@@ -408,6 +412,11 @@ static im_status ensure_staging(im_env *e, int A)
             cudaMalloc(&e->d_obs, n * (size_t)e->cfg.ld_obs * 4) != cudaSuccess ||
             cudaMalloc(&e->d_reward, n * 4) != cudaSuccess || cudaMalloc(&e->d_flags, n) != cudaSuccess)
             return IM_ERR_ALLOC;
+        if (cudaStreamCreateWithFlags(&e->h2d_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&e->d2h_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e->ev_h2d, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e->ev_policy, cudaEventDisableTiming) != cudaSuccess)
+            return IM_ERR_CUDA;
     }
     if (A > e->staged_A) {
         cudaFree(e->d_mean); cudaFree(e->d_action);
@@ -438,20 +447,28 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     im_status s = ensure_staging(e, A);
     if (s != IM_OK) return s;
     const size_t n = (size_t)e->cfg.n_envs, J = (size_t)e->skel->dev.J;
-    IM_CUDA(cudaMemcpyAsync(e->d_sim, sim_host, 13 * J * n * 4, cudaMemcpyHostToDevice, e->stream));
+    // The body states are needed by the env step only: their upload runs on a copy stream beside
+    // the policy forward, and the actions travel back beside the env step (PCIe is full duplex).
+    // The previous call waited for all three streams, so the staging buffers are free.
+    IM_CUDA(cudaMemcpyAsync(e->d_sim, sim_host, 13 * J * n * 4, cudaMemcpyHostToDevice, e->h2d_stream));
+    IM_CUDA(cudaEventRecord(e->ev_h2d, e->h2d_stream));
     int32_t ld_in = 0;
     if (e->d_obs_bf16 && p->tensor_path && e->d_obs_bf16 == tc_policy_input(p, &ld_in))
         s = im_policy_forward_staged(p, step, (int32_t)n, e->d_mean, e->d_action, nullptr);
     else
         s = im_policy_forward(p, step, (int32_t)n, e->d_obs, e->cfg.ld_obs, e->d_mean, e->d_action, nullptr);
     if (s != IM_OK) return s;
+    IM_CUDA(cudaEventRecord(e->ev_policy, e->stream));
+    IM_CUDA(cudaStreamWaitEvent(e->d2h_stream, e->ev_policy, 0));
+    IM_CUDA(cudaMemcpyAsync(action_host, e->d_action, n * (size_t)A * 4, cudaMemcpyDeviceToHost, e->d2h_stream));
+    IM_CUDA(cudaStreamWaitEvent(e->stream, e->ev_h2d, 0));
     im_body_state sim = {e->d_sim, e->d_sim + 3 * J * n, e->d_sim + 7 * J * n, e->d_sim + 10 * J * n, (int64_t)n};
     s = im_env_step(e, step, &sim, e->d_obs, e->d_reward, e->d_flags, nullptr);
     if (s != IM_OK) return s;
-    IM_CUDA(cudaMemcpyAsync(action_host, e->d_action, n * (size_t)A * 4, cudaMemcpyDeviceToHost, e->stream));
     IM_CUDA(cudaMemcpyAsync(reward_host, e->d_reward, n * 4, cudaMemcpyDeviceToHost, e->stream));
     IM_CUDA(cudaMemcpyAsync(flags_host, e->d_flags, n, cudaMemcpyDeviceToHost, e->stream));
     IM_CUDA(cudaStreamSynchronize(e->stream));
+    IM_CUDA(cudaStreamSynchronize(e->d2h_stream));
     return IM_OK;
 }
 

@@ -97,6 +97,8 @@ struct im_env {
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
     uint8_t *d_flags;
     int staged_A;
+    cudaStream_t h2d_stream, d2h_stream;   // copies of the host-buffer step run beside the kernels
+    cudaEvent_t ev_h2d, ev_policy;
 };
 
 // Launchers implemented in the kernel translation units.
