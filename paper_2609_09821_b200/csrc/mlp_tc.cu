@@ -381,6 +381,236 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
     pipe_exit<Plan>(p, tmem_base, P.status);
 }
 
+// ------------------------------------------------------------------ hidden layers, CTA pairs
+// The single-CTA kernel above is limited by shared-memory bandwidth: per 64-deep k-block the
+// tensor core reads A (16 KB) and W (32 KB) while TMA writes as much.  Here two CTAs of a cluster
+// (one TPC) compute a 256 x 256 tile together with tcgen05.mma.cta_group::2: each holds its own 128
+// rows of A and HALF of the W tile (128 of the 256 output columns' rows), the tensor cores exchange
+// the W halves between the two SMs, and each CTA accumulates its 128 rows x 256 columns in its own
+// tensor memory.  Per SM that is 32 KB per k-block instead of 48 KB, and a six-deep ring.
+//   rank 0 ("leader"): its MMA thread issues for the pair; its full[] barriers collect the
+//     transaction bytes of BOTH CTAs' TMA loads; its acc_empty[] barriers collect both epilogues.
+//   both ranks: own TMA producer (own A rows, own W half), own epilogue (own accumulator rows),
+//     own empty[] / acc_full[] barriers, which the leader's commits reach by multicast.
+// No load is multicast; the only multicast is the commit's mbarrier arrive.
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * BLOCK_M * BLOCK_K * 2;             // A 128x64 + W half 128x64, bf16
+constexpr int kPairTmemCols = 512;                                     // two 256-column accumulators
+constexpr size_t kPairSmemBytes = 1024 + (size_t)kPairStages * kPairStageBytes + 4 * 2 * kEpiSlabBytes + 256;
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose completion is signalled on a barrier that may live
+// in the peer CTA (cluster address).
+// Tensor memory of a CTA pair: one warp of EACH CTA issues the allocation, both get the same base.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t *dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives, once the pair's MMAs so far have completed, on the barrier at this offset in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(both) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                             const __grid_constant__ CUtensorMap map_c, const GemmParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *epi = tiles + (size_t)kPairStages * kPairStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(epi + 4 * 2 * kEpiSlabBytes);
+    uint64_t *full = bars, *empty = bars + kPairStages, *acc_full = bars + 2 * kPairStages,
+             *acc_empty = bars + 2 * kPairStages + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kPairStages + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int tiles_m = (P.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M);
+    const int n_tiles = tiles_m * P.n_tiles_n;                       // 256 x 256 tiles
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(tmem_slot, kPairTmemCols);         // one warp of each CTA, collectively
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                              // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0 && rank == 1) {
+        // the pair's MMAs address the accumulator at the same tensor-memory address in both CTAs
+        uint32_t leader_base;
+        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(leader_base) : "r"(map_to_rank(smem_u32(tmem_slot), 0)) : "memory");
+        if (leader_base != tmem_base) *abort_flag = 1;
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both ranks): own A rows and own half of W, signalled to the leader
+        if (lane == 0 && !*abort_flag) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int tile = pair; tile < n_tiles; tile += n_pairs) {
+                const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+                const int n0 = (tile % P.n_tiles_n) * 256 + (int)rank * 128;
+                bool ok = true;
+                for (int kb = 0; kb < P.K_blocks; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *sa = tiles + (size_t)stage * kPairStageBytes;
+                    const uint32_t leader_full = map_to_rank(smem_u32(&full[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * kPairStageBytes);
+                    tma_load_2d_pair(sa, &map_a, leader_full, kb * BLOCK_K, m0);
+                    tma_load_2d_pair(sa + BLOCK_M * BLOCK_K * 2, &map_b, leader_full, kb * BLOCK_K, n0);
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader only)
+        if (lane == 0 && rank == 0 && !*abort_flag) {
+            constexpr uint32_t idesc = instr_desc_bf16(2 * BLOCK_M, 256);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
+                for (int kb = 0; kb < P.K_blocks; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(tiles + (size_t)stage * kPairStageBytes);
+                    const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + BLOCK_M * BLOCK_K * 2);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(&empty[stage]);          // both CTAs' stages are free once these MMAs have read them
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit_pair(&acc_full[acc]);             // both CTAs' accumulators complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------- epilogue warps (both ranks): own 128 rows x 256 columns
+        const int quad = warp & 3;
+        uint8_t *slabs = epi + (size_t)(warp - 2) * 2 * kEpiSlabBytes;
+        int which = 0;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        if (!*abort_flag)
+        for (int tile = pair; tile < n_tiles; tile += n_pairs) {
+            const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+            const int n0 = (tile % P.n_tiles_n) * 256;
+            if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 64) {
+                float v[64];
+                tmem_ld32_issue(t_row + (uint32_t)c0, v);
+                tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
+                tmem_ld_wait();
+                const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float4 b = __ldg(b4 + i);
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, 0.0f), fmaxf(v[4 * i + 1] + b.y, 0.0f));
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, 0.0f), fmaxf(v[4 * i + 3] + b.w, 0.0f));
+                    pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
+                    pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+                }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                uint8_t *slab = slabs + which * kEpiSlabBytes;
+                const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                                 "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                 ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                which ^= 1;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[acc]), 0));   // the leader's barrier
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+
+    // ---------------- common exit: both CTAs meet (the peer's shared memory and barriers stay alive
+    // until the leader is done with them), then each frees its tensor memory
+    if (*abort_flag && lane == 0) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(P.status, IM_DEV_WAIT_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kPairTmemCols);
+    }
+}
+
 // ------------------------------------------------------------------ Gaussian head (last layer)
 // mean = A W^T + b; action = mean + sigma z with z from Philox counter (env, step, 1, block)
 // and Box-Muller; logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi.  The GEMM is tiny, the
@@ -579,6 +809,7 @@ struct TcLayer {
     __nv_bfloat16 *d_W;      // [n_tiles_n * block_n][Kpad], zero padded
     float *d_bias;           // [n_tiles_n * block_n]
     CUtensorMap map_a, map_b, map_c;    // map_c: the hidden-activation buffer this layer stores to
+    CUtensorMap map_b2;                 // W in 128-row boxes: one CTA's half of a 256-column tile
 };
 
 }  // namespace im
@@ -594,6 +825,8 @@ struct im_policy_tc {
 namespace im {
 
 namespace {
+
+bool g_use_pairs = true;
 
 template <int BLOCK_N>
 cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
@@ -612,6 +845,23 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
     const int grid = tiles < n_sm ? tiles : n_sm;
     linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+// 256-wide layers with enough rows to fill the machine run on CTA pairs.
+cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
+{
+    static bool prepared = false;
+    if (!prepared) {
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kPairSmemBytes);
+        if (e != cudaSuccess) return e;
+        prepared = true;
+    }
+    const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
+    const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
+    linear_tc_hidden_pair_kernel<<<2 * pairs, kThreads, kPairSmemBytes, stream>>>(L.map_a, L.map_b2, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -642,6 +892,7 @@ cudaError_t launch_head(const TcLayer &L, const GemmParams &gp_in, int n_sm, cud
 cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n_sm, cudaStream_t stream)
 {
     if (!last) {
+        if (L.block_n == 256 && g_use_pairs) return launch_hidden_pair(L, gp, n_sm, stream);
         switch (L.block_n) {
         case 256: return launch_hidden<256>(L, gp, n_sm, stream);
         case 128: return launch_hidden<128>(L, gp, n_sm, stream);
@@ -717,6 +968,8 @@ im_status tc_policy_create(im_policy *p, const void *const *W, const float *cons
         const int a_ld = l == 0 ? tc->ld_in : tc->ld_hidden;
         if (!make_map(&L.map_a, a_base, mb, (uint64_t)L.Kpad, (uint64_t)a_ld, BLOCK_M) ||
             !make_map(&L.map_b, L.d_W, rows, (uint64_t)L.Kpad, (uint64_t)L.Kpad, (uint32_t)L.block_n))
+            return IM_ERR_CUDA;
+        if (!last && L.block_n == 256 && !make_map(&L.map_b2, L.d_W, rows, (uint64_t)L.Kpad, (uint64_t)L.Kpad, 128))
             return IM_ERR_CUDA;
         // hidden layers store 32-row x 64-column slabs of their output buffer
         if (!last && !make_map(&L.map_c, tc->d_hidden[l & 1], mb, rows, (uint64_t)tc->ld_hidden, 32))
