@@ -200,7 +200,8 @@ typedef struct {
     uint64_t seed;
     uint32_t env_id_base;
     int32_t max_batch;       /* largest n a forward call will pass; sizes the activation buffers */
-    int32_t impl;            /* 0: default for dtype; 1: force the SIMT kernels (debug cross-check) */
+    int32_t impl;            /* 0: default for dtype; 1: force the SIMT kernels (debug cross-check);    */
+                             /* 2: tensor path with CTA-pair GEMMs even for small batches (tests)         */
 } im_policy_config;
 
 im_status im_load_policy(const im_policy_config *cfg, const void *const *W, const float *const *b,

@@ -325,7 +325,7 @@ im_status im_load_policy(const im_policy_config *cfg, const void *const *W, cons
     if (!p) return IM_ERR_ALLOC;
     std::memset(p, 0, sizeof(*p));
     p->cfg = *cfg; p->stream = (cudaStream_t)cuda_stream; p->nl = nl;
-    p->tensor_path = cfg->dtype == 1 && cfg->impl == 0;
+    p->tensor_path = cfg->dtype == 1 && cfg->impl != 1;
     if (cudaMalloc(&p->d_status, 4) != cudaSuccess) { im_destroy_policy(p); return IM_ERR_ALLOC; }
     cudaMemsetAsync(p->d_status, 0, 4, p->stream);
     if (p->tensor_path) {

@@ -123,7 +123,7 @@ class Pair:
             self.sample = np.arange(n) if policy_sample is None or policy_sample >= n else \
                 np.sort(np.random.default_rng(1).choice(n, policy_sample, replace=False))
             # the SIMT cross-check path keeps fp32 activations even with bf16 weights
-            self.bf16_ops = pol["dtype"] == "bf16" and policy_impl == 0
+            self.bf16_ops = pol["dtype"] == "bf16" and policy_impl != 1
             self.mean_tol = 2e-2 if self.bf16_ops else 1e-4
         self.obs_o = None
         self.max_err = dict(obs=0.0, reward=0.0)

@@ -50,6 +50,13 @@ def test_ragged_batches(scenes, n):
     p.rollout(steps=3)
 
 
+@pytest.mark.parametrize("name,n", [("cfg2_4096", 1000), ("cfg4_65536_smpl24", 700), ("cfg5_reset_heavy", 257)])
+def test_cta_pair_gemm_on_small_batches(scenes, name, n):
+    """The cta_group::2 kernel (normally chosen only for many tiles) forced on a ragged small batch."""
+    p = Pair(scenes(name), n, policy_impl=2)
+    p.rollout(steps=2)
+
+
 def test_simt_layers_with_bf16_weights(scenes):
     """The SIMT cross-check path (bf16 weights, fp32 activations) against the unrounded oracle."""
     p = Pair(scenes("cfg2_4096"), 200, policy_impl=1)
