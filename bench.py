@@ -44,6 +44,14 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per step from the committed ncu captures
+# (profiles/*_cfg4_65536_smpl24.md): the four policy kernels, and the env step kernel.
+NCU_TRAFFIC_BYTES = {
+    "cfg4_65536_smpl24": dict(policy=(85.2 + 81.5 + 136.3 + 90.9 + 135.3 + 35.9 + 67.2 + 3.7) * 1e6,
+                              env=(89.3 + 202.1) * 1e6),
+}
+
+
 def env_bytes_per_env(J: int) -> int:
     """Algorithmic HBM bytes of the env kernel per env-step: body states in, observation row,
     reward, flags out, per-env state read + written."""
@@ -68,7 +76,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -158,7 +166,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     wl = W.WORKLOADS[args.workload]
-    K = args.steps if args.steps is not None else wl.steps
+    # default: eight rollouts of the workload's horizon, so that the timed region is long enough
+    # (~0.1 s at the largest config) for clock samples to fall inside it
+    K = args.steps if args.steps is not None else 8 * wl.steps
     Wm = max(args.warmup, 0)
     skel, lib, pol = W.build_scene(wl)
     J, D = skel["J"], wl.obs_dim
@@ -304,17 +314,18 @@ def main():
     # ---- end to end through the host-buffer entry point: pinned host inputs, results read back
     e2e = None
     if not args.no_e2e:
-        host_sims = [s.cpu().pin_memory() for s in sims]
+        n_host = min(n_buf, 16)                    # bound pinned memory; the host buffers are cycled
+        host_sims = [s.cpu().pin_memory() for s in sims[:n_host]]
         act_h = torch.empty((n, A)).pin_memory()
         rew_h = torch.empty(n).pin_memory()
         fl_h = torch.empty(n, dtype=torch.uint8).pin_memory()
         env.reset_all_host(0)
         for s in range(1, Wm + 1):
-            B.step_host(env, policy, s, host_sims[(s - 1) % n_buf], act_h, rew_h, fl_h)
+            B.step_host(env, policy, s, host_sims[(s - 1) % n_host], act_h, rew_h, fl_h)
         barrier()
         t0 = time.perf_counter()
         for s in range(Wm + 1, Wm + K + 1):
-            B.step_host(env, policy, s, host_sims[(s - 1) % n_buf], act_h, rew_h, fl_h)
+            B.step_host(env, policy, s, host_sims[(s - 1) % n_host], act_h, rew_h, fl_h)
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
         if world > 1:
@@ -337,11 +348,12 @@ def main():
     tf = flops / t_pol / 1e12
     gbs = env_bytes / t_env / 1e9
     tensor_peak = peaks["bf16_tflops_sustained"]
+    traffic = NCU_TRAFFIC_BYTES.get(wl.name, {})
     roofline = dict(bound="tensor", kernel="policy forward (GEMM chain + Gaussian head)", achieved=tf,
-                    peak=tensor_peak, unit="TFLOP/s", frac=tf / tensor_peak, traffic=None,
+                    peak=tensor_peak, unit="TFLOP/s", frac=tf / tensor_peak, traffic=traffic.get("policy"),
                     peak_source="%s bf16 sustained" % peaks["source"], seconds_per_launch=t_pol)
     roofline_env = dict(bound="hbm", kernel="env_step_kernel", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=gbs / peaks["hbm_gbs"], traffic=None, peak_source="%s copy" % peaks["source"],
+                        frac=gbs / peaks["hbm_gbs"], traffic=traffic.get("env"), peak_source="%s copy" % peaks["source"],
                         seconds_per_launch=t_env, algorithmic_bytes=env_bytes)
     if wl.mlp_dtype != "bf16":
         roofline["bound"] = "alu"
