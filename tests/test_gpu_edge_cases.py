@@ -1,0 +1,104 @@
+"""GPU parity on shapes and settings off the benchmark configurations: odd policy widths and
+depths, control intervals that do not match the keyframe rate, clips of different rates and of
+the minimum length, explicit end-effectors, uniform masses, zero reward weights."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2609_09821_b200 import binding as B
+from paper_2609_09821_b200 import workloads as W
+from tests.parity import Pair, Scene
+
+pytestmark = pytest.mark.gpu
+
+
+def _scene(name, mlp_dims, mlp_dtype="bf16", skeleton="humanoid15", n_clips=3, frames=(20, 40), dt=1.0 / 30.0,
+           fps=None, seed=5, masses=True, ee_ids=None, **kw):
+    wl = W.Workload(name, 256, skeleton, n_clips, frames, 4, tuple(mlp_dims), mlp_dtype, dt=dt, seed=seed, **kw)
+    skel = W.make_skeleton(skeleton, seed)
+    lib = W.make_clip_library(skel["J"], n_clips, frames, 30.0, seed)
+    if fps is not None:
+        lib["fps"] = np.asarray(fps, np.float32)
+    pol = W.make_policy_weights(mlp_dims, mlp_dtype, seed)
+    sc = Scene.__new__(Scene)
+    sc.wl, sc.skel, sc.lib, sc.pol, sc.J = wl, skel, lib, pol, skel["J"]
+    m = skel["masses"] if masses else None
+    sc.o_skel = O.Skeleton(skel["parents"], skel["offsets"], m, ee_ids)
+    sc.o_clips = O.Clips(sc.o_skel, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    sc.g_skel = B.Skeleton(skel["parents"], skel["offsets"], m, ee_ids)
+    sc.g_clips = B.Clips(sc.g_skel, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    return sc
+
+
+@pytest.mark.parametrize("dims", [
+    (361, 64, 28),                       # one narrow hidden layer: 64-column tiles
+    (361, 128, 192, 8),                  # 128- and 64-column tiles
+    (361, 256, 64, 64, 64, 64, 64, 5),   # seven layers
+    (361, 512, 80),                      # widest action the Gaussian head takes
+    (361, 1024, 1),                      # a single output
+], ids=lambda d: "x".join(map(str, d)))
+def test_policy_shapes_on_the_tensor_path(dims):
+    sc = _scene("edge_policy", dims)
+    p = Pair(sc, 300)
+    p.rollout(steps=2)
+
+
+def test_unsupported_policy_shapes_are_rejected():
+    pol = W.make_policy_weights((361, 100, 28), "bf16", 0)           # hidden width not a multiple of 64
+    with pytest.raises(B.ImError) as e:
+        B.Policy(pol["dims"], pol["W_bf16"], pol["b"], "bf16", 0.1, 0, 64)
+    assert e.value.status == -6
+    pol = W.make_policy_weights((361, 128, 96), "bf16", 0)           # action wider than the head's staging
+    with pytest.raises(B.ImError) as e:
+        B.Policy(pol["dims"], pol["W_bf16"], pol["b"], "bf16", 0.1, 0, 64)
+    assert e.value.status == -6
+    pol = W.make_policy_weights((361, 28), "bf16", 0)                # a single layer has no hidden GEMM
+    with pytest.raises(B.ImError) as e:
+        B.Policy(pol["dims"], pol["W_bf16"], pol["b"], "bf16", 0.1, 0, 64)
+    assert e.value.status == -6
+
+
+@pytest.mark.parametrize("dt", [1.0 / 60.0, 0.05, 1.0 / 30.0 + 1e-4])
+def test_control_interval_off_the_keyframe_rate(dt):
+    sc = _scene("edge_dt", (361, 64, 28), "f32", dt=dt)
+    p = Pair(sc, 200, with_policy=False)
+    p.rollout(steps=6)
+
+
+def test_clips_of_different_rates():
+    sc = _scene("edge_fps", (361, 64, 28), "f32", n_clips=4, frames=(12, 30), fps=[24.0, 30.0, 60.0, 120.0],
+                dt=1.0 / 120.0)
+    p = Pair(sc, 200, with_policy=False)
+    h = p.rollout(steps=8)
+    assert any((x["flags"] & 2).any() for x in h)        # the short, fast clips truncate within a few steps
+
+
+def test_two_keyframe_clips_reset_every_step():
+    sc = _scene("edge_k2", (361, 64, 28), "f32", n_clips=2, frames=(2, 2))
+    p = Pair(sc, 100, with_policy=False)
+    h = p.rollout(steps=3)
+    assert all((x["flags"] & 2).all() for x in h)        # D = dt: the next step would always pass the end
+    assert np.all(p.o_env.t == 0.0)
+
+
+def test_uniform_masses_explicit_end_effectors_and_zero_weights():
+    zero = dict(mode=0, a=[0.0] * 7, w=[0.0] * 7)
+    sc = _scene("edge_skel", (361, 64, 28), "f32", masses=False, ee_ids=[3, 6, 9])
+    p = Pair(sc, 150, reward=zero, with_policy=False)
+    h = p.rollout(steps=2)
+    assert all(np.all(x["reward"] == 1.0) for x in h)     # exp(-0) exactly
+    p = Pair(sc, 150, reward=W.REWARD_ADD4, with_policy=False)
+    p.rollout(steps=2)
+
+
+def test_smpl_skeleton_with_fp32_policy():
+    sc = _scene("edge_smpl_f32", (577, 96, 40, 69), "f32", skeleton="smpl24")
+    p = Pair(sc, 130)
+    p.rollout(steps=2)
+
+
+def test_zero_envs_is_an_error():
+    sc = _scene("edge_zero", (361, 64, 28), "f32")
+    with pytest.raises(B.ImError):
+        B.Env(sc.g_skel, sc.g_clips, B.make_env_config(0, 1 / 30, 0, W.REWARD_MULT, 0.3, 384))
