@@ -251,16 +251,17 @@ __device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
     return q;
 }
 
-__device__ __forceinline__ Quat ld_sim_quat(const EnvKernelParams &P, int b, int e)
+// Body-state loads: `col` points at this thread's env in row 0 of the array, so a component is
+// one per-thread pointer plus a warp-uniform row offset.
+__device__ __forceinline__ Quat ld_sim_quat(const float *col, size_t st, int b)
 {
-    const size_t st = (size_t)P.stride;
-    return {P.quat[(4 * b + 0) * st + e], P.quat[(4 * b + 1) * st + e], P.quat[(4 * b + 2) * st + e],
-            P.quat[(4 * b + 3) * st + e]};
+    const float *p = col + (size_t)(4 * b) * st;
+    return {p[0], p[st], p[2 * st], p[3 * st]};
 }
-__device__ __forceinline__ Vec3 ld_sim_vec(const float *base, const EnvKernelParams &P, int b, int e)
+__device__ __forceinline__ Vec3 ld_sim_vec(const float *col, size_t st, int b)
 {
-    const size_t st = (size_t)P.stride;
-    return {base[(3 * b + 0) * st + e], base[(3 * b + 1) * st + e], base[(3 * b + 2) * st + e]};
+    const float *p = col + (size_t)(3 * b) * st;
+    return {p[0], p[st], p[2 * st]};
 }
 
 // Keyframe quaternions of joint b in the two bracketing rows.
@@ -323,8 +324,10 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
         KeyPair keys = ld_keys(r0, r1, sk.chain[c][0]);
 
-        const Quat q_root = sanitize(ld_sim_quat(P, 0, envc), P.status);
-        const Vec3 p_root = ld_sim_vec(P.pos, P, 0, envc);
+        const size_t st = (size_t)P.stride;
+        const float *pos_e = P.pos + envc, *quat_e = P.quat + envc, *lin_e = P.lin + envc, *ang_e = P.ang + envc;
+        const Quat q_root = sanitize(ld_sim_quat(quat_e, st, 0), P.status);
+        const Vec3 p_root = ld_sim_vec(pos_e, st, 0);
         H = make_heading(q_root, p_root);
         root_z = p_root.z;
 
@@ -336,18 +339,18 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         Vec3 wa = {0, 0, 0};
         if (first_own > 0) {
             const int a = sk.chain[c][first_own - 1];
-            qa = sanitize(ld_sim_quat(P, a, envc), P.status);
-            wa = ld_sim_vec(P.ang, P, a, envc);
+            qa = sanitize(ld_sim_quat(quat_e, st, a), P.status);
+            wa = ld_sim_vec(ang_e, st, a);
         }
         for (int k = 0; k < len; ++k) {
             const int b = sk.chain[c][k];
             const bool own = k >= first_own;
             SimBody sim;
             if (own) {                                // issue the loads before the interpolation math
-                sim.q = ld_sim_quat(P, b, envc);
-                sim.p = ld_sim_vec(P.pos, P, b, envc);
-                sim.v = ld_sim_vec(P.lin, P, b, envc);
-                sim.w = ld_sim_vec(P.ang, P, b, envc);
+                sim.q = ld_sim_quat(quat_e, st, b);
+                sim.p = ld_sim_vec(pos_e, st, b);
+                sim.v = ld_sim_vec(lin_e, st, b);
+                sim.w = ld_sim_vec(ang_e, st, b);
             }
             const KeyPair cur = keys;
             if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);     // next joint's keyframes in flight
