@@ -193,6 +193,61 @@ def test_deterministic_and_resumable(scenes):
         assert torch.equal(obs, hist[s - 1][0]) and torch.equal(rew, hist[s - 1][1]) and torch.equal(fl, hist[s - 1][2])
 
 
+def test_steps_are_capturable_and_replay_bit_exact(scenes):
+    """Per-step calls only enqueue work: a CUDA graph of a whole rollout replays to the same bits."""
+    sc = scenes("cfg2_4096")
+    n, steps = 600, 5
+    p = Pair(sc, n)
+    p.g_env.attach_policy(p.policy)
+    p.reset_all()
+    c0, t0, l0 = p.g_env.get_state()
+    obs0 = p.obs_g.clone()
+    sims = []
+
+    def consume(s, sim):
+        sims.append(sim.cuda())
+        p.policy.forward_staged(s, n, p.mean_g, p.action_g, p.logp_g)
+        p.env_step(s, sim)
+
+    W.rollout_inputs(sc.wl, sc.skel, sc.lib, lambda: (p.o_env.clip_id, p.o_env.t), consume, steps=steps)
+    want = (p.obs_g.clone(), p.reward_g.clone(), p.flags_g.clone(), p.action_g.clone(), p.g_env.get_state())
+    # same rollout again as one captured graph, from the same initial state
+    stream = p.g_env.stream
+    p.g_env.set_state(c0, t0, l0)
+    p.g_env.reset_all(p.obs_g, 0)            # refills the policy's staged input as well
+    assert torch.equal(p.obs_g, obs0)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    env2 = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, sc.wl.dt, sc.wl.seed, W.REWARD_MULT, sc.wl.h_min, p.ld_obs),
+                 stream=side)
+    pol2 = B.Policy(sc.pol["dims"], sc.pol["W_bf16"], sc.pol["b"], "bf16", sc.wl.sigma_action, sc.wl.seed, n, stream=side)
+    env2.attach_policy(pol2)
+    obs = env2.new_obs()
+    rew = torch.empty(n, device="cuda")
+    fl = torch.empty(n, dtype=torch.uint8, device="cuda")
+    mean = torch.empty((n, p.A), device="cuda")
+    act = torch.empty((n, p.A), device="cuda")
+    with torch.cuda.stream(side):
+        env2.reset_all(obs, 0)
+    side.synchronize()
+    with torch.cuda.graph(g, stream=side):
+        for s in range(1, steps + 1):
+            pol2.forward_staged(s, n, mean, act)
+            env2.step(s, sims[s - 1], obs, rew, fl)
+    for _ in range(2):                        # replaying twice from the same state gives the same result
+        env2.set_state(c0, t0, l0)
+        with torch.cuda.stream(side):
+            env2.reset_all(obs, 0)
+        side.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        c, t, l = env2.get_state()
+        assert torch.equal(obs, want[0]) and torch.equal(rew, want[1]) and torch.equal(fl, want[2])
+        assert torch.equal(act, want[3])
+        assert torch.equal(c, want[4][0]) and torch.equal(t, want[4][1]) and torch.equal(l, want[4][2])
+
+
 def test_bad_simulated_quaternion_sets_status_not_a_fault(scenes):
     sc = scenes("cfg1_tiny64")
     p = Pair(sc, 64, with_policy=False)
