@@ -21,7 +21,8 @@
  *
  * Every function below has at least one pin in tests/ that does not restate
  * its formula (closed forms, invariants, brute force with 3x3 matrices, the
- * paper's Figure 5 constants, published Philox known answers).
+ * paper's Figure 5 constants, published Philox known answers; for the advantage
+ * estimator: the discounted-sum form of its definition and geometric series).
  */
 #include <math.h>
 #include <stdint.h>
@@ -671,6 +672,42 @@ void orc_error_terms_flat(const orc_skeleton *s, const orc_clips *cl, int clip, 
         for (int c = 0; c < 4; ++c) x.q[j][c] = q[4*j+c];
     }
     error_terms(s, &x, &r, e);
+}
+
+/* ------------------------------------------------------------------------
+ * Generalised advantage estimation over one rollout of T control steps (the
+ * estimator whose discount factor and parameter lambda the paper's Table of
+ * training hyper-parameters lists; the rollout loop of the paper's training-loop
+ * figure stores reward, terminated and truncated per step for it).
+ *
+ *   done_t  = terminated_t or truncated_t            (flags bit 0 / bit 1)
+ *   r'_t    = r_t + gamma V_t   if bootstrap_truncated and truncated_t and not terminated_t
+ *           = r_t               otherwise
+ *   delta_t = r'_t + gamma V_{t+1} (1 - done_t) - V_t
+ *   A_t     = delta_t + gamma lambda (1 - done_t) A_{t+1},      A_T = 0
+ *   R_t     = A_t + V_t
+ *
+ * Arrays are [T][ld] (value: [T+1][ld]; row T is the value of the observation after the last
+ * step), env index fastest.  fp32 inputs, fp64 arithmetic and outputs. */
+void orc_gae(int T, int N, int64_t ld, const float *reward, const float *value, const uint8_t *flags,
+             double gamma, double lambda, int bootstrap_truncated, double *adv, double *ret)
+{
+    for (int e = 0; e < N; ++e) {
+        double a_next = 0.0;
+        for (int t = T - 1; t >= 0; --t) {
+            const int64_t i = (int64_t)t * ld + e;
+            const int terminated = flags[i] & 1, truncated = (flags[i] >> 1) & 1;
+            const double live = (terminated || truncated) ? 0.0 : 1.0;
+            const double v = (double)value[i], v_next = (double)value[i + ld];
+            double r = (double)reward[i];
+            if (bootstrap_truncated && truncated && !terminated) r += gamma * v;
+            const double delta = r + gamma * v_next * live - v;
+            const double a = delta + gamma * lambda * live * a_next;
+            adv[i] = a;
+            ret[i] = a + v;
+            a_next = a;
+        }
+    }
 }
 
 int orc_openmp_enabled(void)

@@ -79,6 +79,7 @@ def lib():
         L.orc_round_bf16.restype = f64
         L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
         L.orc_openmp_enabled.restype = i32
+        L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
 
@@ -288,3 +289,18 @@ def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarr
                              _p(obs), obs.shape[1], _p(mean), _p(action), _p(logp), _p(z),
                              int(n_threads or os.cpu_count() or 1), int(bool(bf16_operands)))
     return dict(mean=mean, action=action, logp=logp, z=z)
+
+
+def gae(reward: np.ndarray, value: np.ndarray, flags: np.ndarray, gamma: float, lam: float,
+        bootstrap_truncated: bool = True):
+    """reward [T, N] fp32, value [T+1, N] fp32, flags [T, N] uint8 -> (advantage, return) fp64 [T, N]."""
+    reward = np.ascontiguousarray(reward, np.float32)
+    value = np.ascontiguousarray(value, np.float32)
+    flags = np.ascontiguousarray(flags, np.uint8)
+    T, N = reward.shape
+    assert value.shape == (T + 1, N) and flags.shape == (T, N)
+    adv = np.zeros((T, N))
+    ret = np.zeros((T, N))
+    lib().orc_gae(T, N, N, _p(reward), _p(value), _p(flags), float(gamma), float(lam),
+                  int(bool(bootstrap_truncated)), _p(adv), _p(ret))
+    return adv, ret

@@ -411,3 +411,18 @@ def shard_envs(n_total: int, world_size: int, rank: int) -> Tuple[int, int]:
     base, rem = divmod(n_total, world_size)
     first = rank * base + min(rank, rem)
     return first, base + (1 if rank < rem else 0)
+
+
+# ----------------------------------------------------------------------------
+# Rollout signals for the advantage estimator
+# ----------------------------------------------------------------------------
+def make_rollout_signals(T: int, N: int, seed: int = 0, p_term: float = 0.01, p_trunc: float = 0.01):
+    """Seeded stand-ins for one rollout's per-step signals, time-major [T][N]: rewards U[0, 1) (the range
+    of the imitation reward), critic outputs N(0, 3^2) for T + 1 observations, and flag bytes (bit 0
+    terminated, bit 1 truncated) with the given per-step rates."""
+    g = _rng(seed, 64, T, N)
+    reward = g.random((T, N), dtype=np.float32)
+    value = (3.0 * g.standard_normal((T + 1, N), dtype=np.float32)).astype(np.float32)
+    flags = (g.random((T, N), dtype=np.float32) < p_term).astype(np.uint8)
+    flags |= (g.random((T, N), dtype=np.float32) < p_trunc).astype(np.uint8) << 1
+    return reward, value, flags
