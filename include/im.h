@@ -229,6 +229,44 @@ im_status im_env_attach_policy(im_env *e, im_policy *p);
 im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n,
                                    float *mean_out, float *action_out, float *logp_out);
 
+/* ---- rollout-side plumbing: value head and advantage estimation ------------------
+ * (The paper's training loop, its Figure 2, stores obs, action, reward, terminated and
+ * truncated per step and hands the storage to the PPO update; its hyper-parameter table
+ * lists the discount factor and the GAE parameter.  The storage itself is plain device
+ * memory: callers pass pointers into their [T][N] arrays to the per-step calls.)
+ *
+ * Value head: a critic is an im_policy (any output width, normally 1) read without
+ * sampling.  im_policy_forward with action_out == NULL (and logp_out == NULL) does the
+ * same thing; these two are the named form.
+ *   value_out  DEVICE [n][dims[last]] (16-byte aligned on the tensor-core path)
+ * im_value_forward_staged runs on the bf16 observation rows an attached environment has
+ * written into the staging buffer of `src` (the actor the env is attached to; NULL: the
+ * critic's own buffer).  Both must be tensor-core policies with the same input width,
+ * created on the same stream; src->max_batch >= n. */
+im_status im_value_forward(im_policy *critic, int32_t n, const float *obs, int32_t ld_obs, float *value_out);
+im_status im_value_forward_staged(im_policy *critic, im_policy *src, int32_t n, float *value_out);
+
+/* Generalised advantage estimation (Schulman et al. 2016) over T control steps of N envs:
+ *   done_t  = flags_t != 0        (the flag bytes im_env_step writes)
+ *   r'_t    = r_t + gamma V_t     if bootstrap_truncated and step t is truncated, not terminated
+ *   delta_t = r'_t + gamma V_{t+1} (1 - done_t) - V_t
+ *   A_t     = delta_t + gamma lambda (1 - done_t) A_{t+1},  A_T = 0        R_t = A_t + V_t
+ * All arrays DEVICE, time-major with row stride ld >= N elements, env index fastest:
+ *   reward [T][ld] float   value [T+1][ld] float (row T: value of the observation after the
+ *   last step)   flags [T][ld] uint8   advantage, returns [T][ld] float (written; padding
+ *   columns are not touched).
+ * fp32 arithmetic; chunks of the horizon are folded in parallel, so results differ from the
+ * plain backward recursion by rounding only.  Asynchronous on cuda_stream, allocates nothing,
+ * capturable.  gamma and lambda must lie in [0, 1] (IM_ERR_INVALID_ARG otherwise). */
+typedef struct {
+    float gamma, lambda;
+    int32_t bootstrap_truncated;
+} im_gae_config;
+
+im_status im_gae(const im_gae_config *cfg, int32_t T, int32_t N, int64_t ld, const float *reward,
+                 const float *value, const uint8_t *flags, float *advantage, float *returns,
+                 void *cuda_stream);
+
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current

@@ -24,6 +24,7 @@ EXPORTS = [
     "im_env_set_state", "im_load_policy", "im_destroy_policy", "im_policy_forward",
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
+    "im_value_forward", "im_value_forward_staged", "im_gae",
 ]
 
 
@@ -40,6 +41,10 @@ class EnvConfig(C.Structure):
 class BodyState(C.Structure):
     _fields_ = [("pos", C.c_void_p), ("quat", C.c_void_p), ("linvel", C.c_void_p), ("angvel", C.c_void_p),
                 ("comp_stride", C.c_int64)]
+
+
+class GaeConfig(C.Structure):
+    _fields_ = [("gamma", C.c_float), ("lam", C.c_float), ("bootstrap_truncated", C.c_int32)]
 
 
 class PolicyConfig(C.Structure):
@@ -88,6 +93,9 @@ def load():
         L.im_env_attach_policy.argtypes = [vp, vp]
         L.im_policy_forward_staged.argtypes = [vp, u32, i32, vp, vp, vp]
         L.im_policy_forward_noalloc.argtypes = [i32, vp, vp, vp, C.c_float, u64, u32, u32, i32, vp, i32, vp, vp, vp, vp]
+        L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
+        L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
+        L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("im_status_string", "im_launch_count") and not name.startswith("im_destroy") \
                     and name != "im_env_destroy":
@@ -268,6 +276,16 @@ class Policy:
         _check(load().im_policy_forward_staged(self.h, step, n, _ptr(mean_out), _ptr(action_out), _ptr(logp_out)),
                "im_policy_forward_staged")
 
+    def value_forward(self, obs, value_out, n: Optional[int] = None):
+        """This network read as a critic: writes only its outputs ([n, dims[-1]]), draws no noise."""
+        n = obs.shape[0] if n is None else n
+        _check(load().im_value_forward(self.h, n, _ptr(obs), obs.stride(0), _ptr(value_out)), "im_value_forward")
+
+    def value_forward_staged(self, n: int, value_out, src: Optional["Policy"] = None):
+        """Critic forward on the bf16 rows an env attached to `src` (default: this policy) has staged."""
+        _check(load().im_value_forward_staged(self.h, src.h if src is not None else None, n, _ptr(value_out)),
+               "im_value_forward_staged")
+
     def device_status(self) -> int:
         out = C.c_uint32(0)
         _check(load().im_poll_device_status(None, self.h, C.byref(out)), "im_poll_device_status")
@@ -283,6 +301,22 @@ def step_host(env: Env, policy: Policy, step: int, sim_host, action_host, reward
     """One whole step from host buffers (numpy arrays or pinned CPU torch tensors)."""
     _check(load().im_step_host(env.h, policy.h, step, _ptr(sim_host), _ptr(action_host), _ptr(reward_host),
                                _ptr(flags_host)), "im_step_host")
+
+
+def gae(reward, value, flags, advantage, returns, gamma: float, lam: float, bootstrap_truncated: bool = True,
+        stream=None):
+    """Generalised advantage estimation over a rollout.  CUDA tensors, time-major: reward, flags (uint8),
+    advantage, returns [T, N] and value [T + 1, N], all with the same row stride."""
+    import torch
+    T, N = reward.shape
+    ld = reward.stride(0) if T > 1 else max(N, value.stride(0))
+    for a, rows in ((value, T + 1), (flags, T), (advantage, T), (returns, T)):
+        if a.shape != (rows, N) or (rows > 1 and a.stride(0) != ld) or a.stride(1) != 1:
+            raise ValueError("rollout arrays must be [T, N] (value [T + 1, N]) with one common row stride")
+    cfg = GaeConfig(np.float32(gamma), np.float32(lam), int(bool(bootstrap_truncated)))
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().im_gae(C.byref(cfg), T, N, ld, _ptr(reward), _ptr(value), _ptr(flags), _ptr(advantage),
+                         _ptr(returns), C.c_void_p(st.cuda_stream)), "im_gae")
 
 
 NOALLOC_MAX_BATCH = 1024

@@ -370,7 +370,7 @@ void im_destroy_policy(im_policy *p)
 im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out)
 {
-    if (!p || !obs || !mean_out || !action_out) return IM_ERR_INVALID_ARG;
+    if (!p || !obs || !mean_out || (!action_out && logp_out)) return IM_ERR_INVALID_ARG;
     if (n < 1 || n > p->cfg.max_batch || ld_obs < p->cfg.dims[0] || (ld_obs & 3) || !aligned16(obs))
         return IM_ERR_INVALID_ARG;
     if (p->tensor_path) {
@@ -389,8 +389,9 @@ im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         in = outp;
         ld_in = ldc;
     }
-    IM_CUDA(launch_sample(mean_out, action_out, logp_out, n, A, p->cfg.sigma, p->cfg.seed, step,
-                          p->cfg.env_id_base, p->stream));
+    if (action_out)
+        IM_CUDA(launch_sample(mean_out, action_out, logp_out, n, A, p->cfg.sigma, p->cfg.seed, step,
+                              p->cfg.env_id_base, p->stream));
     return IM_OK;
 }
 
@@ -401,6 +402,21 @@ im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n, float
     if (!p->tensor_path) return IM_ERR_UNSUPPORTED;
     if (n < 1 || n > p->cfg.max_batch || !aligned16(mean_out) || !aligned16(action_out)) return IM_ERR_INVALID_ARG;
     return tc_policy_forward(p, step, n, nullptr, 0, mean_out, action_out, logp_out);
+}
+
+/* ------------------------------------------------------------------ value head */
+im_status im_value_forward(im_policy *critic, int32_t n, const float *obs, int32_t ld_obs, float *value_out)
+{
+    return im_policy_forward(critic, 0u, n, obs, ld_obs, value_out, nullptr, nullptr);
+}
+
+im_status im_value_forward_staged(im_policy *critic, im_policy *src, int32_t n, float *value_out)
+{
+    if (!critic || !value_out) return IM_ERR_INVALID_ARG;
+    if (!critic->tensor_path || (src && !src->tensor_path)) return IM_ERR_UNSUPPORTED;
+    if (n < 1 || n > critic->cfg.max_batch || !aligned16(value_out)) return IM_ERR_INVALID_ARG;
+    if (src && src->stream != critic->stream) return IM_ERR_INVALID_ARG;
+    return tc_policy_forward(critic, 0u, n, nullptr, 0, value_out, nullptr, nullptr, src);
 }
 
 /* ------------------------------------------------------------------ host-buffer step */

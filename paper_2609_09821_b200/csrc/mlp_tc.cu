@@ -648,7 +648,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
         const int group = (warp - 2) >> 2;                          // 16-column groups group, group+4, ...
         const int row_in_tile = quad * 32 + lane;
         constexpr int kGroups = (BLOCK_N / 16) < 4 ? (BLOCK_N / 16) : 4;
-        const float logp_const = -(float)A * logf(P.sigma) - 0.5f * (float)A * 1.8378770664093453f;
+        const bool sample = P.action != nullptr;                     // a value head reads only the mean
+        const float logp_const = sample ? -(float)A * logf(P.sigma) - 0.5f * (float)A * 1.8378770664093453f : 0.0f;
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -670,18 +671,20 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
                         for (int g = 0; g < 4; ++g) {
                             const int col = c0 + 4 * g;
                             if (col >= A) break;
-                            const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step, IM_STREAM_ACTION,
-                                                                     (uint32_t)(col >> 2)),
-                                                          make_uint2(P.seed_lo, P.seed_hi));
-                            float z[4];
-                            box_muller(x.x, x.y, z[0], z[1]);
-                            box_muller(x.z, x.w, z[2], z[3]);
+                            float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                            if (sample) {
+                                const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)row, P.step,
+                                                                         IM_STREAM_ACTION, (uint32_t)(col >> 2)),
+                                                              make_uint2(P.seed_lo, P.seed_hi));
+                                box_muller(x.x, x.y, z[0], z[1]);
+                                box_muller(x.z, x.w, z[2], z[3]);
+                            }
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 if (col + i < A) {
                                     const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
                                     s_mean[row_in_tile * A + col + i] = mu;
-                                    s_act[row_in_tile * A + col + i] = mu + P.sigma * z[i];
+                                    if (sample) s_act[row_in_tile * A + col + i] = mu + P.sigma * z[i];
                                     zz += z[i] * z[i];
                                 }
                             }
@@ -716,14 +719,18 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
                         }
                         const int count = rows_valid * A;                       // floats, contiguous in global
                         const float *src_m = s_mean + quad * 32 * A, *src_a = s_act + quad * 32 * A;
-                        float *dst_m = P.mean + (size_t)band_row0 * A, *dst_a = P.action + (size_t)band_row0 * A;
+                        float *dst_m = P.mean + (size_t)band_row0 * A;
+                        float *dst_a = sample ? P.action + (size_t)band_row0 * A : nullptr;
                         // both sides start on a 16-byte boundary: band offsets are multiples of 32 rows
                         const int n4 = count >> 2;
                         for (int i = lane; i < n4; i += 32) {
                             reinterpret_cast<float4 *>(dst_m)[i] = reinterpret_cast<const float4 *>(src_m)[i];
-                            reinterpret_cast<float4 *>(dst_a)[i] = reinterpret_cast<const float4 *>(src_a)[i];
+                            if (sample) reinterpret_cast<float4 *>(dst_a)[i] = reinterpret_cast<const float4 *>(src_a)[i];
                         }
-                        for (int i = 4 * n4 + lane; i < count; i += 32) { dst_m[i] = src_m[i]; dst_a[i] = src_a[i]; }
+                        for (int i = 4 * n4 + lane; i < count; i += 32) {
+                            dst_m[i] = src_m[i];
+                            if (sample) dst_a[i] = src_a[i];
+                        }
                     }
                 }
             }
@@ -820,6 +827,8 @@ struct im_policy_tc {
     __nv_bfloat16 *d_hidden[2];   // [max_batch][max hidden]
     int ld_in, ld_hidden;
     int n_sm;
+    const __nv_bfloat16 *ext_in;  // another policy's input buffer the first layer last read from (or null)
+    CUtensorMap map_a_ext;        // first-layer operand map over ext_in
 };
 
 namespace im {
@@ -934,6 +943,7 @@ im_status tc_policy_create(im_policy *p, const void *const *W, const float *cons
     p->tc = tc;
     tc->n_sm = n_sm;
     tc->d_in = nullptr;
+    tc->ext_in = nullptr;
     tc->d_hidden[0] = tc->d_hidden[1] = nullptr;
     tc->layers.resize(nl);
     for (auto &L : tc->layers) { L.d_W = nullptr; L.d_bias = nullptr; }
@@ -998,12 +1008,27 @@ void *tc_policy_input(im_policy *p, int32_t *ld)
     return p->tc->d_in;
 }
 
-// obs == nullptr: the bf16 input buffer has already been filled (by an attached environment).
+// obs == nullptr: the bf16 input buffer has already been filled (by an attached environment); it is
+// this policy's own buffer, or that of `src` (same input width), whose rows the first layer then reads
+// through a tensor map built on first use.  action_out == nullptr: no sampling, only the mean is written.
 im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
-                            float *mean_out, float *action_out, float *logp_out)
+                            float *mean_out, float *action_out, float *logp_out, im_policy *src)
 {
     im_policy_tc *tc = p->tc;
     const im_policy_config &cfg = p->cfg;
+    const bool external = !obs && src && src != p;
+    if (external) {
+        im_policy_tc *st = src->tc;
+        if (!st || st->ld_in != tc->ld_in || src->cfg.dims[0] != cfg.dims[0] || src->cfg.max_batch < n)
+            return IM_ERR_INVALID_ARG;
+        if (tc->ext_in != st->d_in) {
+            const TcLayer &L0 = tc->layers[0];
+            if (!make_map(&tc->map_a_ext, st->d_in, (uint64_t)src->cfg.max_batch, (uint64_t)L0.Kpad, (uint64_t)st->ld_in,
+                          BLOCK_M))
+                return IM_ERR_CUDA;
+            tc->ext_in = st->d_in;
+        }
+    }
     if (obs) {
         const long long chunks = (long long)n * (tc->ld_in / 8);
         const int block = 256;
@@ -1014,7 +1039,8 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         if (cudaGetLastError() != cudaSuccess) return IM_ERR_CUDA;
     }
     for (int l = 0; l < p->nl; ++l) {
-        const TcLayer &L = tc->layers[l];
+        TcLayer L = tc->layers[l];
+        if (l == 0 && external) L.map_a = tc->map_a_ext;
         const bool last = l == p->nl - 1;
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;

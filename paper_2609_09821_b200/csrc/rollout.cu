@@ -1,0 +1,133 @@
+// Generalised advantage estimation over one rollout (the estimator behind the paper's
+// "discount factor" and "GAE parameter" hyper-parameters), time-major arrays, env index fastest.
+//
+//   done_t  = flags_t != 0 (bit 0 terminated, bit 1 truncated)
+//   r'_t    = r_t + gamma V_t   on a step that is truncated but not terminated (if configured)
+//   delta_t = r'_t + gamma V_{t+1} (1 - done_t) - V_t
+//   A_t     = delta_t + gamma lambda (1 - done_t) A_{t+1},  A_T = 0;      R_t = A_t + V_t
+//
+// The recursion is a chain of affine maps A_t = delta_t + c_t A_{t+1}, and affine maps compose, so
+// the horizon is cut into chunks of 8 steps that run in parallel: lane = env (every load and store
+// is one full 128-byte line per warp), warp = chunk.  A thread loads its chunk (25 independent
+// loads in flight: the kernel is a pure stream over 17 bytes per env-step), folds it into one map
+// (a, b), the maps of the later chunks are folded in shared memory, and the thread then replays its
+// chunk from the now known A at the chunk's end.  Horizons longer than one CTA's window
+// (chunks x 8 steps) are walked window by window from the end, carrying A across in shared memory.
+#include "im_internal.h"
+
+namespace im {
+
+namespace {
+
+constexpr int kChunk = 8;          // steps per thread
+constexpr int kMaxChunks = 16;     // chunks (warps) per CTA
+
+struct GaeParams {
+    const float *reward, *value;
+    const uint8_t *flags;
+    float *adv, *ret;
+    long long ld;
+    int T, N;
+    float gamma, gl;               // gl = gamma * lambda
+    int bootstrap;
+    int chunks;                    // warps per CTA
+};
+
+__global__ void __launch_bounds__(32 * kMaxChunks) gae_kernel(const GaeParams P)
+{
+    __shared__ float s_a[kMaxChunks][32], s_b[kMaxChunks][32], s_carry[32];
+    const int lane = threadIdx.x, g = threadIdx.y, G = P.chunks;
+    const int env = blockIdx.x * 32 + lane;
+    const bool valid = env < P.N;
+    const int e = valid ? env : P.N - 1;
+    const int window = G * kChunk;
+    const int n_windows = (P.T + window - 1) / window;
+    if (g == 0) s_carry[lane] = 0.0f;                       // A_T = 0
+
+    for (int w = n_windows - 1; w >= 0; --w) {
+        const int t0 = w * window + g * kChunk;             // this thread's steps: [t0, t0 + n)
+        int n = P.T - t0;
+        n = n < 0 ? 0 : (n > kChunk ? kChunk : n);
+        float delta[kChunk], c[kChunk], v[kChunk + 1];
+        v[kChunk] = 0.0f;
+        {
+            float r[kChunk];
+            uint8_t f[kChunk];
+            const size_t base = (size_t)t0 * (size_t)P.ld + (size_t)e;
+#pragma unroll
+            for (int i = 0; i < kChunk; ++i) {
+                const bool in = i < n;
+                const size_t idx = base + (size_t)i * (size_t)P.ld;
+                r[i] = in ? __ldg(P.reward + idx) : 0.0f;
+                f[i] = in ? __ldg(P.flags + idx) : (uint8_t)1;
+                v[i] = in ? __ldg(P.value + idx) : 0.0f;
+            }
+#pragma unroll
+            for (int i = kChunk; i >= 1; --i)               // value row after the chunk's last step
+                if (i == n) v[i] = __ldg(P.value + base + (size_t)i * (size_t)P.ld);
+#pragma unroll
+            for (int i = 0; i < kChunk; ++i) {
+                const bool live = f[i] == 0;
+                float ri = r[i];
+                if (P.bootstrap && (f[i] & 3) == 2) ri = fmaf(P.gamma, v[i], ri);
+                const float vn = (i < n) ? v[i + 1] : 0.0f;
+                delta[i] = (live ? fmaf(P.gamma, vn, ri) : ri) - v[i];
+                c[i] = live ? P.gl : 0.0f;
+                if (i >= n) { delta[i] = 0.0f; c[i] = 1.0f; }            // identity map beyond the horizon
+            }
+        }
+        // fold the chunk: A_{t0} = a + b A_{t0+n}
+        float a = 0.0f, b = 1.0f;
+#pragma unroll
+        for (int i = kChunk - 1; i >= 0; --i) {
+            a = fmaf(c[i], a, delta[i]);
+            b = c[i] * b;
+        }
+        s_a[g][lane] = a;
+        s_b[g][lane] = b;
+        __syncthreads();
+        // A at the end of this chunk: the later chunks of the window applied to the window's carry
+        float x = s_carry[lane];
+        for (int h = G - 1; h > g; --h) x = fmaf(s_b[h][lane], x, s_a[h][lane]);
+        __syncthreads();                                    // every thread has read the carry
+        if (g == 0) s_carry[lane] = fmaf(b, x, a);          // A at the start of the window
+        // replay the chunk
+        const size_t base = (size_t)t0 * (size_t)P.ld + (size_t)env;
+#pragma unroll
+        for (int i = kChunk - 1; i >= 0; --i) {
+            x = fmaf(c[i], x, delta[i]);
+            if (valid && i < n) {
+                const size_t idx = base + (size_t)i * (size_t)P.ld;
+                P.adv[idx] = x;
+                P.ret[idx] = x + v[i];
+            }
+        }
+        // the carry written above is read only after the next window's first barrier
+    }
+}
+
+}  // namespace
+
+}  // namespace im
+
+extern "C" im_status im_gae(const im_gae_config *cfg, int32_t T, int32_t N, int64_t ld, const float *reward,
+                            const float *value, const uint8_t *flags, float *advantage, float *returns,
+                            void *cuda_stream)
+{
+    using namespace im;
+    if (!cfg || !reward || !value || !flags || !advantage || !returns) return IM_ERR_INVALID_ARG;
+    if (T < 1 || N < 1 || ld < N) return IM_ERR_INVALID_ARG;
+    if (!(cfg->gamma >= 0.0f && cfg->gamma <= 1.0f) || !(cfg->lambda >= 0.0f && cfg->lambda <= 1.0f))
+        return IM_ERR_INVALID_ARG;
+    GaeParams p;
+    p.reward = reward; p.value = value; p.flags = flags; p.adv = advantage; p.ret = returns;
+    p.ld = ld; p.T = T; p.N = N;
+    p.gamma = cfg->gamma; p.gl = cfg->gamma * cfg->lambda;
+    p.bootstrap = cfg->bootstrap_truncated ? 1 : 0;
+    int chunks = (T + kChunk - 1) / kChunk;
+    p.chunks = chunks > kMaxChunks ? kMaxChunks : chunks;
+    const dim3 grid((unsigned)((N + 31) / 32)), block(32, (unsigned)p.chunks);
+    gae_kernel<<<grid, block, 0, (cudaStream_t)cuda_stream>>>(p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
