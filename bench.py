@@ -160,6 +160,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of one CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-rollout-extras", action="store_true",
+                    help="skip the separate timing of the value head and the advantage estimator")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -311,6 +313,52 @@ def main():
     t_pol = float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e-3
     t_env = float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e-3
 
+    # ---- rollout-side calls, timed on their own (not part of the metric): critic forward on the rows the
+    # ---- env staged for the actor, and the advantage estimator over one rollout of wl.steps steps.  The
+    # ---- estimator's 17 B per env-step fit in L2, so a 256 MB buffer is read before every launch (reading
+    # ---- leaves clean lines behind: a written buffer's write-back would be charged to the kernel).
+    extras = None
+    if not args.no_rollout_extras and rank == 0:
+        reps = 20
+        T = wl.steps
+        r_np, v_np, f_np = W.make_rollout_signals(T, n, wl.seed)
+        r_d, v_d, f_d = (torch.from_numpy(a).to(dev) for a in (r_np, v_np, f_np))
+        adv_d, ret_d = torch.empty((T, n), device=dev), torch.empty((T, n), device=dev)
+        flush = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
+        t_gae = []
+        for i in range(3 + reps):
+            flush.sum()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            B.gae(r_d, v_d, f_d, adv_d, ret_d, 0.99, 0.95, True, stream=stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                t_gae.append(a.elapsed_time(b) * 1e-3)
+        t_gae = float(np.median(t_gae))
+        gae_bytes = T * n * 17 + n * 4
+        extras = dict(gae=dict(T=T, seconds_per_launch=t_gae, algorithmic_bytes=gae_bytes,
+                               achieved_gbs=gae_bytes / t_gae / 1e9, l2="256 MB read before every launch"))
+        if staged:
+            cdims = tuple(wl.mlp_dims[:-1]) + (1,)
+            cw = W.make_policy_weights(cdims, "bf16", wl.seed + 1)
+            critic = B.Policy(cdims, cw["W_bf16"], cw["b"], "bf16", 1.0, wl.seed, n, stream=stream)
+            value = torch.empty((n, 1), device=dev)
+            t_v = []
+            for i in range(3 + reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                critic.value_forward_staged(n, value, src=policy)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    t_v.append(a.elapsed_time(b) * 1e-3)
+            t_v = float(np.median(t_v))
+            cflops = mlp_flops_per_env(cdims) * n
+            extras["value_head"] = dict(dims=list(cdims), seconds_per_launch=t_v, achieved_tflops=cflops / t_v / 1e12)
+            del critic
+        del flush
+
     # ---- end to end through the host-buffer entry point: pinned host inputs, results read back
     e2e = None
     if not args.no_e2e:
@@ -369,6 +417,11 @@ def main():
                 breakdown_ms=dict(policy_forward=t_pol * 1e3, env_step=t_env * 1e3))
     if e2e is not None:
         line["e2e"] = e2e
+    if extras is not None:
+        extras["gae"]["frac_of_hbm_peak"] = extras["gae"]["achieved_gbs"] / peaks["hbm_gbs"]
+        if "value_head" in extras:
+            extras["value_head"]["frac_of_tensor_peak"] = extras["value_head"]["achieved_tflops"] / tensor_peak
+        line["rollout_extras"] = extras
     if not args.no_cpu_baseline:
         res = oracle_leg(wl, skel, lib, pol, n_sample=2048, steps=64, warmup=1, budget_s=15.0)
         line["cpu_baseline"] = dict(value=res["value"], unit=UNIT, cores=res["cores"], kind="oracle",

@@ -13,6 +13,9 @@
 // (a, b), the maps of the later chunks are folded in shared memory, and the thread then replays its
 // chunk from the now known A at the chunk's end.  Horizons longer than one CTA's window
 // (chunks x 8 steps) are walked window by window from the end, carrying A across in shared memory.
+// One env per lane is deliberate: with four envs per lane and 16-byte accesses the grid is four
+// times smaller and the kernel, which lives on the number of loads in flight, was 15-35 % slower
+// at every size from 16 k to 1 M envs (measured: 2.9 TB/s at 65536 x 32, 5.6 TB/s at 1 M x 32).
 #include "im_internal.h"
 
 namespace im {

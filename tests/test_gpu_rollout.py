@@ -45,7 +45,9 @@ def run_gae(reward, value, flags, gamma, lam, bootstrap=True, ld=None):
 
 
 @pytest.mark.parametrize("T,N,ld", [(32, 4096 + 17, None), (1, 5, None), (8, 33, 48), (7, 100, None), (13, 64, 64),
-                                     (129, 70, 96), (200, 257, None), (300, 31, None)])
+                                     (129, 70, 96), (200, 257, None), (300, 31, None),
+                                     # aligned row strides and env counts that are multiples of four
+                                     (32, 4096 + 16, None), (200, 256, 320), (1, 4, None), (9, 132, 136)])
 @pytest.mark.parametrize("gamma,lam,bootstrap", [(0.99, 0.95, True), (0.98, 0.99, False)])
 def test_gae_matches_oracle(T, N, ld, gamma, lam, bootstrap):
     """Horizons that are not a multiple of the 8-step chunk, several 128-step windows, ragged env
@@ -171,3 +173,61 @@ def test_value_head_on_rows_staged_by_the_env():
     bad = B.Policy(other["dims"], other["W_bf16"], other["b"], "bf16", 1.0, 0, n)
     with pytest.raises(B.ImError):
         bad.value_forward_staged(n, v_staged, src=p.policy)
+
+
+# ---------------------------------------------------------------- whole rollout into storage
+@pytest.mark.parametrize("staged", [False, True], ids=["fp32-rows", "staged-bf16-rows"])
+def test_collect_fills_storage_like_the_separate_calls(staged):
+    """T steps collected straight into time-major storage: every stored signal against the oracle
+    stage by stage, and the advantages against the oracle's estimator fed the stored signals."""
+    from paper_2609_09821_b200 import rollout as R
+    from tests.parity import assert_close
+    wl = W.WORKLOADS["cfg3_16384_lib32"]
+    sc = Scene(wl)
+    n, T, gamma, lam = 512, 6, 0.99, 0.95
+    ld = B.padded_ld(wl.obs_dim)
+    pol = sc.pol
+    cw = critic_weights(wl.obs_dim, "bf16")
+    o_env = O.Env(sc.o_skel, sc.o_clips, O.make_env_config(wl.dt, 0, W.REWARD_MULT, 0.8), n)
+    g_env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, wl.dt, 0, W.REWARD_MULT, 0.8, ld))
+    actor = B.Policy(pol["dims"], pol["W_bf16"], pol["b"], "bf16", wl.sigma_action, 0, n)
+    critic = B.Policy(cw["dims"], cw["W_bf16"], cw["b"], "bf16", 1.0, 0, n)
+    if staged:
+        g_env.attach_policy(actor)
+    # oracle pass: fixes the simulator states of every step
+    obs_o = [o_env.reset_all(0)]
+    sims, reward_o, flags_o = {}, [], []
+    for t in range(T):
+        s = 1 + t
+        sim = W.synth_sim_state(sc.skel, sc.lib, o_env.clip_id, o_env.t.astype(np.float64) + wl.dt, s, wl)
+        sims[s] = torch.from_numpy(np.ascontiguousarray(sim)).cuda()
+        out = o_env.step(s, sim, want_terms=False)
+        obs_o.append(out["obs"]); reward_o.append(out["reward"]); flags_o.append(out["flags"])
+    st = R.RolloutStorage(T, n, pol["dims"][-1], ld, keep_obs=True)
+    g_env.reset_all(st.obs_row(0), 0)
+    R.collect(g_env, actor, critic, st, lambda s: sims[s], 1, gamma, lam, True, staged=staged)
+    torch.cuda.synchronize()
+    assert g_env.device_status() == 0 and actor.device_status() == 0 and critic.device_status() == 0
+    flags = st.flags.cpu().numpy()
+    np.testing.assert_array_equal(flags, np.stack(flags_o))
+    assert (flags != 0).any()                                     # h_min = 0.8 ends some episodes
+    assert_close(st.reward.cpu().numpy(), np.stack(reward_o), what="stored rewards")
+    for t in range(T + 1):
+        got = st.obs[t, :, :wl.obs_dim].cpu().numpy()
+        assert np.abs(got - obs_o[t]).max() < 1e-3                # loose here; the env parity tests hold the real bar
+    for t in (0, T - 1):
+        want = O.policy_forward(pol["dims"], pol["W"], pol["b"], wl.sigma_action, 0, 1 + t, obs_o[t],
+                                bf16_operands=True)
+        assert_mean_close(st.mean[t].cpu().numpy(), want["mean"], 2e-2, "stored means")
+        assert_close(st.logp[t].cpu().numpy(), want["logp"], atol=1e-3, rtol=1e-5, what="stored logp")
+        assert_close((st.action[t] - st.mean[t]).cpu().numpy(), wl.sigma_action * want["z"], atol=1e-5, rtol=1e-4,
+                     what="stored action noise")
+    for t in (0, T):
+        want = O.policy_forward(cw["dims"], cw["W"], cw["b"], 1.0, 0, 0, obs_o[t], bf16_operands=True)["mean"]
+        assert_mean_close(st.value[t].cpu().numpy()[:, None], want, 2e-2, "stored values")
+    reward, value = st.reward.cpu().numpy(), st.value.cpu().numpy()
+    adv_o, ret_o = O.gae(reward, value, flags, gamma, lam, True)
+    tol = gae_tolerance(T, gamma, lam, reward, value, adv_o)
+    assert np.abs(st.advantage.cpu().numpy() - adv_o).max() <= tol
+    assert np.abs(st.returns.cpu().numpy() - ret_o).max() <= tol
+    g_env.attach_policy(None)
