@@ -209,9 +209,11 @@ im_status im_load_policy(const im_policy_config *cfg, const void *const *W, cons
 void im_destroy_policy(im_policy *p);
 
 /*   obs        DEVICE [n][ld_obs] float, ld_obs >= dims[0], multiple of 4, 16-byte aligned
- *   mean_out   DEVICE [n][A]     action_out DEVICE [n][A]     logp_out DEVICE [n] or NULL
+ *   mean_out   DEVICE [n][A]     action_out DEVICE [n][A] or NULL     logp_out DEVICE [n] or NULL
  *              (mean_out and action_out 16-byte aligned on the tensor-core path)
- * logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi. */
+ * logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi.
+ * action_out == NULL (logp_out must then be NULL too, else IM_ERR_INVALID_ARG) evaluates the
+ * mean only: no noise is drawn. */
 im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out);
 

@@ -33,6 +33,7 @@
 #define ORC_N_TERMS 7
 #define ORC_STREAM_RESET 0u
 #define ORC_STREAM_ACTION 1u
+#define ORC_STREAM_RESET_NOISE 2u
 
 #ifndef M_PI
 #define M_PI 3.14159265358979323846
@@ -274,6 +275,8 @@ static void center_of_mass(const orc_skeleton *s, double p[][3], double com[3])
     for (int c = 0; c < 3; ++c) com[c] /= m;
 }
 
+static void forward_kinematics(const orc_skeleton *s, orc_ref *r);
+
 void orc_reference_state(const orc_skeleton *s, const orc_clips *cl, int clip, float t, orc_ref *r)
 {
     int J = s->J, K = cl->K[clip], k;
@@ -291,11 +294,18 @@ void orc_reference_state(const orc_skeleton *s, const orc_clips *cl, int clip, f
         orc_quat_log(rel, lg);
         for (int c = 0; c < 3; ++c) r->wl[j][c] = 2.0 * lg[c] * fps;
     }
-    /* a2: forward kinematics with velocity propagation */
     for (int c = 0; c < 3; ++c) {
         r->p[0][c] = (1.0 - alpha) * P0[c] + alpha * P1[c];
         r->v[0][c] = (P1[c] - P0[c]) * fps;
     }
+    forward_kinematics(s, r);
+}
+
+/* a2: forward kinematics with velocity propagation from the local rotations ql, the joint
+ * angular velocities wl and the root's position and linear velocity (p[0], v[0]). */
+static void forward_kinematics(const orc_skeleton *s, orc_ref *r)
+{
+    int J = s->J;
     memcpy(r->q[0], r->ql[0], sizeof(double) * 4);
     orc_quat_rotate(r->q[0], r->wl[0], r->w[0]);
     for (int j = 1; j < J; ++j) {
@@ -346,6 +356,8 @@ typedef struct {
     uint32_t seed_lo, seed_hi;
     orc_reward_config reward;
     int32_t write_back_reset;
+    int32_t grace_steps;            /* no early termination while fewer than this many steps of the episode are done */
+    float reset_noise_std;          /* motion randomisation of the state an env is reset to (0: off) */
 } orc_env_config;
 
 /* Body state of one env, fp64 working copy. */
@@ -427,6 +439,62 @@ void orc_reset_draw(const orc_clips *cl, const orc_env_config *cfg, uint32_t env
     if (span < 0.0f) span = 0.0f;
     volatile float t = u * span;                                    /* one fp32 multiply */
     *clip_out = clip; *t_out = t;
+}
+
+/* Four standard normals from one Philox block: (x0,x1) and (x2,x3) each feed one Box-Muller pair. */
+static void normal4(const uint32_t ctr[4], const uint32_t key[2], double z[4])
+{
+    uint32_t x[4];
+    orc_philox4x32_10(ctr, key, x);
+    for (int h = 0; h < 2; ++h) {
+        double u1 = ((double)(x[2*h] >> 8) + 1.0) * 5.9604644775390625e-08;
+        double u2 = (double)(x[2*h+1] >> 8) * 5.9604644775390625e-08;
+        double rad = sqrt(-2.0 * log(u1));
+        z[2*h] = rad * cos(2.0 * M_PI * u2);
+        z[2*h+1] = rad * sin(2.0 * M_PI * u2);
+    }
+}
+
+/* Motion randomisation of a reset state (the hyper-parameter "motion randomization std" of the
+ * paper's configuration table; the paper does not say what is perturbed -- reading: every joint's
+ * local rotation is turned by a rotation vector n ~ N(0, std^2 I) given in the joint's own frame,
+ * ql' = ql exp(n/2), and the root position is shifted by N(0, std^2 I); local joint velocities and
+ * the root's linear velocity are kept, and the world state follows by forward kinematics).
+ * Joint j draws from Philox counter (env, step, 2, j), the root shift from (env, step, 2, J);
+ * the first three normals of a block are used. */
+void orc_reset_noise(const orc_skeleton *s, const orc_env_config *cfg, uint32_t env, uint32_t step, orc_ref *r)
+{
+    double std = (double)cfg->reset_noise_std, z[4];
+    uint32_t key[2] = {cfg->seed_lo, cfg->seed_hi};
+    if (!(std > 0.0)) return;
+    for (int j = 0; j <= s->J; ++j) {
+        uint32_t ctr[4] = {env, step, ORC_STREAM_RESET_NOISE, (uint32_t)j};
+        normal4(ctr, key, z);
+        if (j == s->J) {
+            for (int c = 0; c < 3; ++c) r->p[0][c] += std * z[c];
+        } else {
+            double n[3] = {std * z[0], std * z[1], std * z[2]};
+            double th = sqrt(n[0]*n[0] + n[1]*n[1] + n[2]*n[2]);
+            double k = th > 1e-12 ? sin(0.5 * th) / th : 0.5;
+            double dq[4] = {cos(0.5 * th), k * n[0], k * n[1], k * n[2]}, out[4];
+            orc_quat_mul(r->ql[j], dq, out);
+            memcpy(r->ql[j], out, sizeof(out));
+        }
+    }
+    forward_kinematics(s, r);
+}
+
+/* Flat export for the tests: the randomised reset state of (clip, t). */
+void orc_reset_state_flat(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg, uint32_t env,
+                          uint32_t step, int clip, float t, double *p, double *q, double *v, double *w, double *ql)
+{
+    orc_ref r;
+    orc_reference_state(s, cl, clip, t, &r);
+    orc_reset_noise(s, cfg, env, step, &r);
+    for (int j = 0; j < s->J; ++j) {
+        for (int c = 0; c < 3; ++c) { p[3*j+c] = r.p[j][c]; v[3*j+c] = r.v[j][c]; w[3*j+c] = r.w[j][c]; }
+        for (int c = 0; c < 4; ++c) { q[4*j+c] = r.q[j][c]; ql[4*j+c] = r.ql[j][c]; }
+    }
 }
 
 static void ref_to_state(const orc_skeleton *s, const orc_ref *r, orc_body_state *x)
@@ -517,6 +585,7 @@ void orc_env_reset_all(const orc_skeleton *s, const orc_clips *cl, const orc_env
         orc_reset_draw(cl, cfg, env_ids[i], step, &clip_id[i], &t[i]);
         ep_len[i] = 0;
         orc_reference_state(s, cl, clip_id[i], t[i], &r);
+        orc_reset_noise(s, cfg, env_ids[i], step, &r);
         ref_to_state(s, &r, &x);
         build_obs(s, cl, cfg, &x, clip_id[i], t[i], obs + (int64_t)i * ld_obs);
     }
@@ -552,6 +621,7 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
         /* a4: flags.  Root height is compared as the fp32 input value. */
         float root_z = pos[2 * comp_stride + i];
         int terminated = (root_z < cfg->reward.h_min) || (rew < (double)cfg->reward.r_min);
+        if (ep_len[i] < cfg->grace_steps) terminated = 0;           /* early-termination grace steps */
         volatile float t2 = t1 + cfg->dt;
         int truncated = t2 > cl->dur[clip];
         flags[i] = (uint8_t)(terminated | (truncated << 1));
@@ -561,6 +631,7 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
             orc_reset_draw(cl, cfg, env_ids[i], step, &clip, &t_cur);
             ep_len[i] = 0;
             orc_reference_state(s, cl, clip, t_cur, &r);
+            orc_reset_noise(s, cfg, env_ids[i], step, &r);
             ref_to_state(s, &r, &x);
             if (cfg->write_back_reset) store_sim(s, &x, pos, quat, linvel, angvel, comp_stride, i);
         } else {

@@ -38,7 +38,8 @@ class RewardConfig(C.Structure):
 
 class EnvConfig(C.Structure):
     _fields_ = [("dt", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32),
-                ("reward", RewardConfig), ("write_back_reset", C.c_int32)]
+                ("reward", RewardConfig), ("write_back_reset", C.c_int32), ("grace_steps", C.c_int32),
+                ("reset_noise_std", C.c_float)]
 
 
 _lib = None
@@ -79,6 +80,7 @@ def lib():
         L.orc_round_bf16.restype = f64
         L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
         L.orc_openmp_enabled.restype = i32
+        L.orc_reset_state_flat.argtypes = [vp, vp, vp, u32, u32, i32, f32, vp, vp, vp, vp, vp]
         L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
@@ -144,13 +146,14 @@ def action_noise(seed: int, env: int, step: int, A: int) -> np.ndarray:
 
 
 def make_env_config(dt: float, seed: int, reward: dict, h_min: float, r_min: float = -np.inf,
-                    write_back_reset: bool = False) -> EnvConfig:
+                    write_back_reset: bool = False, grace_steps: int = 0, reset_noise_std: float = 0.0) -> EnvConfig:
     rc = RewardConfig(mode=int(reward["mode"]), h_min=np.float32(h_min), r_min=np.float32(r_min))
     for k in range(N_TERMS):
         rc.a[k] = reward["a"][k]
         rc.w[k] = reward["w"][k]
     return EnvConfig(dt=np.float32(dt), seed_lo=seed & 0xFFFFFFFF, seed_hi=(seed >> 32) & 0xFFFFFFFF,
-                     reward=rc, write_back_reset=int(write_back_reset))
+                     reward=rc, write_back_reset=int(write_back_reset), grace_steps=int(grace_steps),
+                     reset_noise_std=np.float32(reset_noise_std))
 
 
 def reward_from_terms(reward: dict, e) -> float:
@@ -304,3 +307,12 @@ def gae(reward: np.ndarray, value: np.ndarray, flags: np.ndarray, gamma: float, 
     lib().orc_gae(T, N, N, _p(reward), _p(value), _p(flags), float(gamma), float(lam),
                   int(bool(bootstrap_truncated)), _p(adv), _p(ret))
     return adv, ret
+
+
+def reset_state(skel: Skeleton, clips: Clips, cfg: EnvConfig, env: int, step: int, clip: int, t: float) -> dict:
+    """State an env reset at (clip, t) with counter (env, step) starts from (motion randomisation applied)."""
+    J = skel.J
+    out = {k: np.zeros((J, n)) for k, n in (("p", 3), ("q", 4), ("v", 3), ("w", 3), ("ql", 4))}
+    lib().orc_reset_state_flat(skel.h, clips.h, C.byref(cfg), env, step, clip, np.float32(t),
+                               _p(out["p"]), _p(out["q"]), _p(out["v"]), _p(out["w"]), _p(out["ql"]))
+    return out

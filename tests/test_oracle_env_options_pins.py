@@ -1,0 +1,153 @@
+"""Pins for the oracle's optional env semantics: early-termination grace steps and motion
+randomisation of the reset state (both named in the paper's hyper-parameter table, both off by
+default).  None of the checks restates the oracle's code path: they use the counter layout with an
+independently written Box-Muller, rigid-body invariants, moments of the normal distribution, and
+episode-length bookkeeping.
+"""
+import math
+
+import numpy as np
+
+from oracle import oracle as O
+from paper_2609_09821_b200 import workloads as W
+
+
+def _scene(kind="humanoid15", n_clips=3, frames=(40, 60)):
+    skel = W.make_skeleton(kind, 0)
+    lib = W.make_clip_library(skel["J"], n_clips, frames, 30.0, 0)
+    o_skel = O.Skeleton(skel["parents"], skel["offsets"], skel["masses"])
+    o_clips = O.Clips(o_skel, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    return skel, lib, o_skel, o_clips
+
+
+def _qmul(a, b):
+    w1, x1, y1, z1 = a
+    w2, x2, y2, z2 = b
+    return np.array([w1 * w2 - x1 * x2 - y1 * y2 - z1 * z2, w1 * x2 + x1 * w2 + y1 * z2 - z1 * y2,
+                     w1 * y2 - x1 * z2 + y1 * w2 + z1 * x2, w1 * z2 + x1 * y2 - y1 * x2 + z1 * w2])
+
+
+def _normals(seed, env, step, block):
+    """First three Box-Muller normals of Philox block (env, step, 2, block), written out here."""
+    x = O.philox([env, step, 2, block], [seed & 0xFFFFFFFF, seed >> 32])
+    u1 = (float(x[0] >> 8) + 1.0) * 2.0 ** -24
+    u2 = float(x[1] >> 8) * 2.0 ** -24
+    u3 = (float(x[2] >> 8) + 1.0) * 2.0 ** -24
+    u4 = float(x[3] >> 8) * 2.0 ** -24
+    r1, r2 = math.sqrt(-2 * math.log(u1)), math.sqrt(-2 * math.log(u3))
+    return np.array([r1 * math.cos(2 * math.pi * u2), r1 * math.sin(2 * math.pi * u2), r2 * math.cos(2 * math.pi * u4)])
+
+
+def test_zero_std_leaves_the_reference_state():
+    skel, lib, o_skel, o_clips = _scene()
+    cfg = O.make_env_config(1 / 30, 5, W.REWARD_MULT, 0.3)
+    ref = O.reference_state(o_skel, o_clips, 1, 0.4)
+    got = O.reset_state(o_skel, o_clips, cfg, 7, 3, 1, 0.4)
+    for k in ("p", "q", "v", "w"):
+        np.testing.assert_array_equal(got[k], ref[k])
+
+
+def test_noise_uses_the_stated_counters_and_rotates_in_the_joint_frame():
+    skel, lib, o_skel, o_clips = _scene()
+    std, seed, env, step = 0.05, 0x1234ABCD5678, 11, 4
+    cfg = O.make_env_config(1 / 30, seed, W.REWARD_MULT, 0.3, reset_noise_std=std)
+    ref = O.reference_state(o_skel, o_clips, 2, 0.7)
+    got = O.reset_state(o_skel, o_clips, cfg, env, step, 2, 0.7)
+    J = skel["J"]
+    for j in range(J):
+        n = std * _normals(seed, env, step, j)
+        th = np.linalg.norm(n)
+        dq = np.concatenate([[math.cos(th / 2)], math.sin(th / 2) * n / th])
+        np.testing.assert_allclose(got["ql"][j], _qmul(ref["ql"][j], dq), atol=1e-12)
+    np.testing.assert_allclose(got["p"][0], ref["p"][0] + std * _normals(seed, env, step, J), atol=1e-12)
+    # another env or step draws other numbers
+    other = O.reset_state(o_skel, o_clips, cfg, env + 1, step, 2, 0.7)
+    assert np.abs(other["ql"] - got["ql"]).max() > 1e-4
+    other = O.reset_state(o_skel, o_clips, cfg, env, step + 1, 2, 0.7)
+    assert np.abs(other["ql"] - got["ql"]).max() > 1e-4
+
+
+def test_randomised_state_is_a_rigid_pose_of_the_same_skeleton():
+    """Bone lengths are kept, world rotations are the products of the local ones, and the velocity of
+    a child origin is the parent's plus omega x arm."""
+    skel, lib, o_skel, o_clips = _scene("smpl24")
+    cfg = O.make_env_config(1 / 30, 9, W.REWARD_MULT, 0.3, reset_noise_std=0.2)
+    st = O.reset_state(o_skel, o_clips, cfg, 3, 8, 0, 0.31)
+    par = skel["parents"]
+    for j in range(1, skel["J"]):
+        a = par[j]
+        arm = st["p"][j] - st["p"][a]
+        np.testing.assert_allclose(np.linalg.norm(arm), np.linalg.norm(skel["offsets"][j]), atol=1e-6)
+        np.testing.assert_allclose(st["q"][j], _qmul(st["q"][a], st["ql"][j]), atol=1e-12)
+        np.testing.assert_allclose(st["v"][j], st["v"][a] + np.cross(st["w"][a], arm), atol=1e-10)
+    np.testing.assert_allclose(np.linalg.norm(st["q"], axis=1), 1.0, atol=1e-12)
+
+
+def test_noise_moments():
+    """Over many envs: joint rotation angles have E|n|^2 = 3 std^2, the root shift has mean 0 and
+    variance std^2 per axis, and two joints are uncorrelated."""
+    skel, lib, o_skel, o_clips = _scene()
+    std = 0.02                                            # the paper's baseline value
+    cfg = O.make_env_config(1 / 30, 1, W.REWARD_MULT, 0.3, reset_noise_std=std)
+    ref = O.reference_state(o_skel, o_clips, 0, 0.5)
+    ang2, shift, n3, n5 = [], [], [], []
+    for env in range(3000):
+        st = O.reset_state(o_skel, o_clips, cfg, env, 1, 0, 0.5)
+        rel = np.array([_qmul(ref["ql"][j] * [1, -1, -1, -1], st["ql"][j]) for j in range(skel["J"])])
+        rv = 2 * rel[:, 1:] / np.maximum(rel[:, :1], 1e-9)            # small angles: n ~ 2 vec / w
+        ang2.append((rv ** 2).sum(axis=1))
+        n3.append(rv[3, 0]); n5.append(rv[5, 0])
+        shift.append(st["p"][0] - ref["p"][0])
+    ang2, shift = np.array(ang2), np.array(shift)
+    np.testing.assert_allclose(ang2.mean(), 3 * std ** 2, rtol=0.03)
+    np.testing.assert_allclose(shift.std(axis=0), std, rtol=0.05)
+    assert np.abs(shift.mean(axis=0)).max() < 4 * std / math.sqrt(3000)
+    assert abs(np.corrcoef(n3, n5)[0, 1]) < 0.08
+
+
+def test_reset_env_observes_and_writes_back_the_randomised_state():
+    skel, lib, o_skel, o_clips = _scene()
+    wl = W.WORKLOADS["cfg1_tiny64"]
+    n, J = 32, skel["J"]
+    cfg = O.make_env_config(wl.dt, 3, W.REWARD_MULT, 10.0, write_back_reset=True, reset_noise_std=0.05)   # h_min 10: all reset
+    env = O.Env(o_skel, o_clips, cfg, n)
+    env.reset_all(0)
+    sim = W.synth_sim_state(skel, lib, env.clip_id, env.t.astype(np.float64) + wl.dt, 1, wl)
+    out = env.step(1, sim)
+    assert (out["flags"] & 1).all()
+    for e in (0, 17, 31):
+        st = O.reset_state(o_skel, o_clips, cfg, e, 1, int(env.clip_id[e]), float(env.t[e]))
+        pos, quat, lin, ang = W.split_sim(sim, J)
+        np.testing.assert_allclose(pos[:, e].reshape(J, 3), st["p"], atol=1e-6)
+        np.testing.assert_allclose(quat[:, e].reshape(J, 4), st["q"], atol=1e-6)
+        np.testing.assert_allclose(lin[:, e].reshape(J, 3), st["v"], atol=1e-5)
+        np.testing.assert_allclose(ang[:, e].reshape(J, 3), st["w"], atol=1e-5)
+        # the root's observed position is (0, 0, z) in its own heading frame, z of the shifted root
+        np.testing.assert_allclose(out["obs"][e, :3], [0.0, 0.0, st["p"][0][2]], atol=1e-12)
+
+
+def test_grace_steps_delay_early_termination_but_not_truncation():
+    skel, lib, o_skel, o_clips = _scene(n_clips=2, frames=(12, 12))          # 11 intervals: truncation comes early
+    wl = W.WORKLOADS["cfg1_tiny64"]
+    n, G = 16, 3
+    cfg = O.make_env_config(wl.dt, 2, W.REWARD_MULT, 10.0, grace_steps=G)     # h_min 10: every step would terminate
+    env = O.Env(o_skel, o_clips, cfg, n)
+    env.reset_all(0)
+    lens = [env.ep_len.copy()]
+    for s in range(1, 14):
+        before = env.ep_len.copy()
+        sim = W.synth_sim_state(skel, lib, env.clip_id, env.t.astype(np.float64) + wl.dt, s, wl)
+        out = env.step(s, sim)
+        term, trunc = out["flags"] & 1, out["flags"] >> 1
+        np.testing.assert_array_equal(term, (before >= G).astype(np.uint8))
+        # truncation is decided by the clock alone
+        assert ((trunc == 1) | (term == 1) == (env.ep_len == 0)).all()
+        lens.append(env.ep_len.copy())
+    lens = np.array(lens)
+    assert lens.max() == G                               # an episode never survives G + 1 steps here
+    assert (np.diff(lens, axis=0)[lens[1:] > 0] == 1).all()
+    # G = 0 is the old behaviour: everything terminates at once
+    env0 = O.Env(o_skel, o_clips, O.make_env_config(wl.dt, 2, W.REWARD_MULT, 10.0), n)
+    env0.reset_all(0)
+    sim = W.synth_sim_state(skel, lib, env0.clip_id, env0.t.astype(np.float64) + wl.dt, 1, wl)
+    assert (env0.step(1, sim)["flags"] & 1).all()
