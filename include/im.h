@@ -128,6 +128,19 @@ typedef struct {
                               /* columns [24J+1, ld_obs) are written as zeros                       */
     int32_t write_back_reset; /* non-zero: a reset env's reference state is also stored into the    */
                               /* caller's body-state arrays (masked store)                          */
+    /* Optional semantics named in the paper's hyper-parameter table; 0 switches them off.         */
+    int32_t grace_steps;      /* early-termination grace steps: the terminated flag is suppressed   */
+                              /* while the episode has completed fewer than this many steps         */
+                              /* (truncation at the clip end is not affected)                       */
+    float reset_noise_std;    /* motion randomisation: an env is reset to the reference state with  */
+                              /* every joint turned, in its own frame, by a rotation vector         */
+                              /* n ~ N(0, std^2 I) (q_local' = q_local exp(n/2), radians) and the   */
+                              /* root shifted by N(0, std^2 I) metres; velocities of the joints and */
+                              /* of the root are kept and the world state follows by forward        */
+                              /* kinematics.  Joint j draws from Philox counter (env id, step, 2,   */
+                              /* j), the root shift from (env id, step, 2, J); Box-Muller as for    */
+                              /* the actions, first three normals of the block.  The observation    */
+                              /* targets stay those of the unperturbed reference.                   */
 } im_env_config;
 
 /* Simulated body states, DEVICE, structure of arrays: component c of env e at

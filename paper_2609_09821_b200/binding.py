@@ -35,7 +35,8 @@ class RewardConfig(C.Structure):
 
 class EnvConfig(C.Structure):
     _fields_ = [("n_envs", C.c_int32), ("env_id_base", C.c_uint32), ("dt", C.c_float), ("seed", C.c_uint64),
-                ("reward", RewardConfig), ("ld_obs", C.c_int32), ("write_back_reset", C.c_int32)]
+                ("reward", RewardConfig), ("ld_obs", C.c_int32), ("write_back_reset", C.c_int32),
+                ("grace_steps", C.c_int32), ("reset_noise_std", C.c_float)]
 
 
 class BodyState(C.Structure):
@@ -166,13 +167,15 @@ class Clips:
 
 
 def make_env_config(n_envs: int, dt: float, seed: int, reward: dict, h_min: float, ld_obs: int,
-                    r_min: float = -np.inf, env_id_base: int = 0, write_back_reset: bool = False) -> EnvConfig:
+                    r_min: float = -np.inf, env_id_base: int = 0, write_back_reset: bool = False,
+                    grace_steps: int = 0, reset_noise_std: float = 0.0) -> EnvConfig:
     rc = RewardConfig(mode=int(reward["mode"]), h_min=np.float32(h_min), r_min=np.float32(r_min))
     for k in range(N_TERMS):
         rc.a[k] = reward["a"][k]
         rc.w[k] = reward["w"][k]
     return EnvConfig(n_envs=int(n_envs), env_id_base=int(env_id_base), dt=np.float32(dt), seed=int(seed),
-                     reward=rc, ld_obs=int(ld_obs), write_back_reset=int(write_back_reset))
+                     reward=rc, ld_obs=int(ld_obs), write_back_reset=int(write_back_reset),
+                     grace_steps=int(grace_steps), reset_noise_std=np.float32(reset_noise_std))
 
 
 def padded_ld(D: int, multiple: int = 64) -> int:

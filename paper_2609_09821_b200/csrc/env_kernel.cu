@@ -160,10 +160,9 @@ struct Walk {
 // One link of the chain: interpolate joint b between keyframe rows r0/r1 and
 // compose it onto the running transform.  k == 0 is the root.
 template <bool VEL>
-__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, Quat k0, Quat k1,
-                                           float alpha, float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
+__device__ __forceinline__ void joint_compose(const SkelDev &sk, const float4 *r0, const float4 *r1, float alpha,
+                                              float fps, int b, int k, Walk &s, Quat ql, Vec3 wl)
 {
-    slerp_joint<VEL>(k0, k1, alpha, fps, ql, wl);
     if (k == 0) {
         const float4 a = __ldg(r0), c = __ldg(r1);
         s.q = ql;
@@ -179,6 +178,41 @@ __device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, 
         s.q = qmul(s.q, ql);
         if (VEL) s.w = s.w + qrot(s.q, wl);
     }
+}
+
+template <bool VEL>
+__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, Quat k0, Quat k1,
+                                           float alpha, float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
+{
+    slerp_joint<VEL>(k0, k1, alpha, fps, ql, wl);
+    joint_compose<VEL>(sk, r0, r1, alpha, fps, b, k, s, ql, wl);
+}
+
+// Motion randomisation of a reset state: three standard normals of Philox counter
+// (env id, step, 2, block), scaled by the configured standard deviation.
+__device__ __forceinline__ Vec3 reset_noise_vec(const EnvKernelParams &P, int env, int block)
+{
+    const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)env, P.step, IM_STREAM_RESET_NOISE, (uint32_t)block),
+                                  make_uint2(P.seed_lo, P.seed_hi));
+    float z0, z1, z2, z3;
+    box_muller(x.x, x.y, z0, z1);
+    box_muller(x.z, x.w, z2, z3);
+    return {P.reset_noise_std * z0, P.reset_noise_std * z1, P.reset_noise_std * z2};
+}
+// ... as the rotation exp(n / 2) applied to joint `b` in its own frame (block b) ...
+__device__ __forceinline__ Quat reset_noise_quat(const EnvKernelParams &P, int env, int b)
+{
+    const Vec3 n = reset_noise_vec(P, env, b);
+    const float th = sqrtf(dot(n, n));
+    float sn, cs;
+    sincosf(0.5f * th, &sn, &cs);
+    const float k = th > 1e-12f ? sn / th : 0.5f;
+    return {cs, k * n.x, k * n.y, k * n.z};
+}
+// ... and as the shift of the root position (block J).
+__device__ __forceinline__ Vec3 reset_noise_shift(const EnvKernelParams &P, int env, int J)
+{
+    return reset_noise_vec(P, env, J);
 }
 
 // Heading frame of the character the observation is taken from: origin at the
@@ -277,7 +311,9 @@ __device__ __forceinline__ Quat as_quat(float4 v) { return {v.x, v.y, v.z, v.w};
 // Kernel body.  The observation row is assembled in two halves that reuse the same shared
 // memory: columns [0, c1) -- the body blocks and, if 15 J is not a multiple of 4, the phase and
 // the first target floats -- and columns [c1, D) -- the targets.
-template <bool RESET_ALL>
+// OPT compiles in the optional semantics (grace steps, motion randomisation); envs that use neither run
+// the instantiation without them.
+template <bool RESET_ALL, bool OPT>
 __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
 {
     const SkelDev &sk = P.sk;
@@ -419,7 +455,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
 #pragma unroll
             for (int k = 0; k < IM_N_TERMS; ++k) r += P.reward.a[k] * expf(-P.reward.w[k] * term[k]);
         }
-        const bool terminated = (root_z < P.reward.h_min) || (r < P.reward.r_min);
+        bool terminated = (root_z < P.reward.h_min) || (r < P.reward.r_min);
+        if (OPT && P.ep_len[envc] < P.grace_steps) terminated = false;
         const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
         flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
         if (c == 0 && valid) {
@@ -463,7 +500,16 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);
             Quat ql;
             Vec3 wl;
-            joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, b, k, s, ql, wl);
+            if (OPT && P.reset_noise_std > 0.0f) {
+                // motion randomisation: the joint turns by a small random rotation in its own frame and
+                // the root is shifted; every chain that walks a shared body draws the same numbers
+                slerp_joint<true>(as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, ql, wl);
+                ql = qmul(ql, reset_noise_quat(P, envc, b));
+                joint_compose<true>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
+                if (k == 0) s.p = s.p + reset_noise_shift(P, envc, sk.J);
+            } else {
+                joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, b, k, s, ql, wl);
+            }
             if (k == 0) Hn = make_heading(s.q, s.p);
             if (k >= first_own && reset) {
                 body_obs(Hn, s.q, s.p, s.v, s.w, row1, b);
@@ -570,18 +616,34 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
 
 // Two instantiations per mode: skeletons with at most 8 leaves (blocks of up to 256 threads) get a
 // register budget that lets four blocks share an SM; wider trees fall back to 64 registers.
-template <bool RESET_ALL>
+template <bool RESET_ALL, bool OPT>
 __global__ void __maxnreg__(96) env_step_kernel_small(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
-    env_step_body<RESET_ALL>(P, smem_raw);
+    env_step_body<RESET_ALL, OPT>(P, smem_raw);
 }
 
-template <bool RESET_ALL>
+template <bool RESET_ALL, bool OPT>
 __global__ void __launch_bounds__(1024, 1) env_step_kernel_wide(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
-    env_step_body<RESET_ALL>(P, smem_raw);
+    env_step_body<RESET_ALL, OPT>(P, smem_raw);
+}
+
+template <bool RESET_ALL, bool OPT>
+cudaError_t prepare_one(size_t smem)
+{
+    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(env_step_kernel_small<RESET_ALL, OPT>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<RESET_ALL, OPT>, attr, (int)smem);
+    return e;
+}
+
+template <bool RESET_ALL, bool OPT>
+void launch_one(const EnvKernelParams &p, dim3 grid, dim3 block, size_t smem, cudaStream_t stream)
+{
+    if (block.x <= 256) env_step_kernel_small<RESET_ALL, OPT><<<grid, block, smem, stream>>>(p);
+    else env_step_kernel_wide<RESET_ALL, OPT><<<grid, block, smem, stream>>>(p);
 }
 
 }  // namespace
@@ -592,11 +654,10 @@ cudaError_t env_kernel_prepare(size_t smem)
 {
     static bool done = false;
     if (done) return cudaSuccess;
-    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(env_step_kernel_small<false>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_small<true>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<false>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<true>, attr, (int)smem);
+    cudaError_t e = prepare_one<false, false>(smem);
+    if (e == cudaSuccess) e = prepare_one<true, false>(smem);
+    if (e == cudaSuccess) e = prepare_one<false, true>(smem);
+    if (e == cudaSuccess) e = prepare_one<true, true>(smem);
     done = e == cudaSuccess;
     return e;
 }
@@ -604,12 +665,13 @@ cudaError_t env_kernel_prepare(size_t smem)
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
-    if (block.x <= 256) {
-        if (reset_all) env_step_kernel_small<true><<<grid, block, smem, stream>>>(p);
-        else env_step_kernel_small<false><<<grid, block, smem, stream>>>(p);
+    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f;
+    if (opt) {
+        if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
+        else launch_one<false, true>(p, grid, block, smem, stream);
     } else {
-        if (reset_all) env_step_kernel_wide<true><<<grid, block, smem, stream>>>(p);
-        else env_step_kernel_wide<false><<<grid, block, smem, stream>>>(p);
+        if (reset_all) launch_one<true, false>(p, grid, block, smem, stream);
+        else launch_one<false, false>(p, grid, block, smem, stream);
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();

@@ -181,6 +181,8 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
         if (!std::isfinite(cfg->reward.w[k]) || !std::isfinite(cfg->reward.a[k]) || cfg->reward.w[k] < 0.0f)
             return IM_ERR_INVALID_ARG;
     if (std::isnan(cfg->reward.h_min) || std::isnan(cfg->reward.r_min)) return IM_ERR_INVALID_ARG;
+    if (cfg->grace_steps < 0 || !(cfg->reset_noise_std >= 0.0f) || !std::isfinite(cfg->reset_noise_std))
+        return IM_ERR_INVALID_ARG;
 
     im_env *e = new (std::nothrow) im_env();
     if (!e) return IM_ERR_ALLOC;
@@ -235,6 +237,8 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.reward = e->cfg.reward;
     p.ld_obs = e->cfg.ld_obs;
     p.write_back = e->cfg.write_back_reset;
+    p.grace_steps = e->cfg.grace_steps;
+    p.reset_noise_std = e->cfg.reset_noise_std;
     p.step = step;
     p.clip_id = e->d_clip_id;
     p.t = e->d_t;

@@ -8,6 +8,7 @@ namespace im {
 
 #define IM_STREAM_RESET 0u
 #define IM_STREAM_ACTION 1u
+#define IM_STREAM_RESET_NOISE 2u
 
 struct Quat { float w, x, y, z; };
 struct Vec3 { float x, y, z; };

@@ -48,6 +48,8 @@ struct EnvKernelParams {
     im_reward_config reward;
     int32_t ld_obs;
     int32_t write_back;
+    int32_t grace_steps;
+    float reset_noise_std;
     uint32_t step;
     // per-env state
     int32_t *clip_id;

@@ -87,7 +87,7 @@ class Pair:
 
     def __init__(self, scene: Scene, n: int, reward=W.REWARD_MULT, seed=None, h_min=None, r_min=-np.inf,
                  write_back=False, env_base=0, ld_obs=None, stride_pad=0, with_policy=True, policy_impl=0,
-                 policy_sample=None, want_terms=True, obs_atol=OBS_ATOL):
+                 policy_sample=None, want_terms=True, obs_atol=OBS_ATOL, grace_steps=0, reset_noise_std=0.0):
         wl = scene.wl
         self.scene, self.wl, self.n, self.J = scene, wl, n, scene.J
         self.seed = wl.seed if seed is None else seed
@@ -102,10 +102,11 @@ class Pair:
         ids = np.arange(env_base, env_base + n, dtype=np.uint32)
         self.ids = ids
         self.o_env = O.Env(scene.o_skel, scene.o_clips,
-                           O.make_env_config(wl.dt, self.seed, reward, self.h_min, r_min, write_back), n, ids)
+                           O.make_env_config(wl.dt, self.seed, reward, self.h_min, r_min, write_back, grace_steps,
+                                             reset_noise_std), n, ids)
         self.g_env = B.Env(scene.g_skel, scene.g_clips,
                            B.make_env_config(n, wl.dt, self.seed, reward, self.h_min, self.ld_obs, r_min,
-                                             env_base, write_back))
+                                             env_base, write_back, grace_steps, reset_noise_std))
         self.obs_g = torch.full((n, self.ld_obs), float("nan"), device="cuda")
         self.reward_g = torch.empty(n, device="cuda")
         self.flags_g = torch.empty(n, dtype=torch.uint8, device="cuda")

@@ -102,3 +102,40 @@ def test_zero_envs_is_an_error():
     sc = _scene("edge_zero", (361, 64, 28), "f32")
     with pytest.raises(B.ImError):
         B.Env(sc.g_skel, sc.g_clips, B.make_env_config(0, 1 / 30, 0, W.REWARD_MULT, 0.3, 384))
+
+
+# ---------------------------------------------------------------- optional env semantics
+@pytest.mark.parametrize("skeleton,dims", [("humanoid15", (361, 64, 28)), ("smpl24", (577, 64, 69))])
+def test_motion_randomisation_of_reset_states(skeleton, dims):
+    """Reset envs start from the randomised reference state: observation and written-back body
+    states against the oracle, with terminations frequent enough that many envs reset each step."""
+    sc = _scene("edge_noise_" + skeleton, dims, "f32", skeleton=skeleton, sigma_root=0.05)
+    p = Pair(sc, 300, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, reset_noise_std=0.05, seed=77)
+    h = p.rollout(steps=6)
+    frac = np.mean([(x["flags"] != 0).mean() for x in h])
+    assert 0.2 < frac < 0.9                                # resets and survivors both well represented
+    # the randomisation is there: the same rollout without it observes different reset states
+    q = Pair(sc, 300, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, seed=77)
+    q.reset_all()
+    p2 = Pair(sc, 300, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, reset_noise_std=0.05, seed=77)
+    p2.reset_all()
+    assert np.abs(p2.obs_o - q.obs_o).max() > 1e-2
+
+
+def test_grace_steps_hold_off_termination():
+    sc = _scene("edge_grace", (361, 64, 28), "f32", n_clips=2, frames=(12, 14))
+    p = Pair(sc, 200, h_min=10.0, with_policy=False, grace_steps=3)          # h_min 10: the height test always fires
+    h = p.rollout(steps=12)
+    term = np.array([(x["flags"] & 1) for x in h])
+    trunc = np.array([(x["flags"] >> 1) for x in h])
+    assert not term[:3].any() and term[3:].any()           # nothing terminates in the first three steps
+    assert trunc.any()                                     # the 11- to 13-interval clips still truncate
+    _, _, ep = p.g_env.get_state()
+    assert int(ep.max()) <= 3
+
+
+def test_env_options_are_validated():
+    sc = _scene("edge_opts", (361, 64, 28), "f32")
+    for kw in (dict(grace_steps=-1), dict(reset_noise_std=-0.1), dict(reset_noise_std=float("nan"))):
+        with pytest.raises(B.ImError):
+            B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, 1 / 30, 0, W.REWARD_MULT, 0.3, 384, **kw))
