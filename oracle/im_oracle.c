@@ -358,7 +358,43 @@ typedef struct {
     int32_t write_back_reset;
     int32_t grace_steps;            /* no early termination while fewer than this many steps of the episode are done */
     float reset_noise_std;          /* motion randomisation of the state an env is reset to (0: off) */
+    /* adaptive episode initialisation: B phase bins per clip with a cumulative table over the C*B
+     * (clip, bin) pairs; n_bins = 0 keeps the uniform draw */
+    int32_t n_bins;
+    const uint64_t *reset_cdf;      /* [C*B] exclusive upper thresholds in [0, 2^32], see orc_reset_cdf */
+    uint32_t *stat_starts;          /* [C*B] episodes started in the bin (or NULL) */
+    uint32_t *stat_failures;        /* [C*B] early terminations that happened in the bin (or NULL) */
 } orc_env_config;
+
+/* Cumulative table of a weight table w[n] >= 0 (not all zero): T_i = floor(2^32 (w_0 + .. + w_i) / total)
+ * with the sums taken in order in fp64, T_{n-1} = 2^32.  A 32-bit uniform word x selects the smallest
+ * i with x < T_i, so bin i is drawn with probability (T_i - T_{i-1}) / 2^32 and a bin of weight 0 never. */
+int orc_reset_cdf(int n, const float *w, uint64_t *T)
+{
+    double total = 0.0, cum = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (!(w[i] >= 0.0f) || isinf(w[i])) return -1;
+        total += (double)w[i];
+    }
+    if (!(total > 0.0)) return -1;
+    for (int i = 0; i < n; ++i) {
+        cum += (double)w[i];
+        T[i] = (uint64_t)floor(cum / total * 4294967296.0);
+    }
+    T[n - 1] = 4294967296ull;
+    return 0;
+}
+
+/* Phase bin of time t in a clip whose start times span [0, span]: floor(t / (span / B)) in single
+ * fp32 operations, clamped to B - 1 (times past the last start time fall in the last bin). */
+static int phase_bin(float t, float span, int B)
+{
+    volatile float width = span / (float)B;
+    if (!(width > 0.0f)) return 0;
+    volatile float f = t / width;
+    int b = (int)floorf(f);
+    return b < 0 ? 0 : (b > B - 1 ? B - 1 : b);
+}
 
 /* Body state of one env, fp64 working copy. */
 typedef struct {
@@ -433,8 +469,26 @@ void orc_reset_draw(const orc_clips *cl, const orc_env_config *cfg, uint32_t env
 {
     uint32_t ctr[4] = {env, step, ORC_STREAM_RESET, 0u}, key[2] = {cfg->seed_lo, cfg->seed_hi}, x[4];
     orc_philox4x32_10(ctr, key, x);
-    int32_t clip = (int32_t)(((uint64_t)x[0] * (uint64_t)(uint32_t)cl->C) >> 32);
     float u = (float)(x[1] >> 8) * 5.9604644775390625e-08f;       /* 2^-24, exact */
+    if (cfg->n_bins > 0) {
+        /* adaptive initialisation: (clip, bin) from the cumulative table, then uniform inside the bin */
+        int B = cfg->n_bins, n = cl->C * B, i = 0;
+        while (i < n - 1 && !((uint64_t)x[0] < cfg->reset_cdf[i])) ++i;
+        int32_t clip = i / B, b = i % B;
+        volatile float span = cl->dur[clip] - cfg->dt;
+        if (span < 0.0f) span = 0.0f;
+        volatile float width = span / (float)B;
+        volatile float pos = (float)b + u;
+        volatile float t = pos * width;
+        if (t > span) t = span;
+        *clip_out = clip; *t_out = t;
+        if (cfg->stat_starts) {
+#pragma omp atomic
+            cfg->stat_starts[i] += 1u;
+        }
+        return;
+    }
+    int32_t clip = (int32_t)(((uint64_t)x[0] * (uint64_t)(uint32_t)cl->C) >> 32);
     volatile float span = cl->dur[clip] - cfg->dt;                  /* one fp32 subtract */
     if (span < 0.0f) span = 0.0f;
     volatile float t = u * span;                                    /* one fp32 multiply */
@@ -622,6 +676,13 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
         float root_z = pos[2 * comp_stride + i];
         int terminated = (root_z < cfg->reward.h_min) || (rew < (double)cfg->reward.r_min);
         if (ep_len[i] < cfg->grace_steps) terminated = 0;           /* early-termination grace steps */
+        if (terminated && cfg->n_bins > 0 && cfg->stat_failures) {  /* where the episode failed */
+            volatile float span = cl->dur[clip] - cfg->dt;
+            if (span < 0.0f) span = 0.0f;
+            int b = phase_bin(t1, span, cfg->n_bins);
+#pragma omp atomic
+            cfg->stat_failures[clip * cfg->n_bins + b] += 1u;
+        }
         volatile float t2 = t1 + cfg->dt;
         int truncated = t2 > cl->dur[clip];
         flags[i] = (uint8_t)(terminated | (truncated << 1));

@@ -39,7 +39,8 @@ class RewardConfig(C.Structure):
 class EnvConfig(C.Structure):
     _fields_ = [("dt", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32),
                 ("reward", RewardConfig), ("write_back_reset", C.c_int32), ("grace_steps", C.c_int32),
-                ("reset_noise_std", C.c_float)]
+                ("reset_noise_std", C.c_float), ("n_bins", C.c_int32), ("reset_cdf", C.c_void_p),
+                ("stat_starts", C.c_void_p), ("stat_failures", C.c_void_p)]
 
 
 _lib = None
@@ -81,6 +82,8 @@ def lib():
         L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
         L.orc_openmp_enabled.restype = i32
         L.orc_reset_state_flat.argtypes = [vp, vp, vp, u32, u32, i32, f32, vp, vp, vp, vp, vp]
+        L.orc_reset_cdf.argtypes = [i32, vp, vp]
+        L.orc_reset_cdf.restype = i32
         L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
@@ -239,6 +242,18 @@ class Env:
         self.D = 24 * skel.J + 1
         self.n_threads = int(n_threads or os.cpu_count() or 1)
 
+    def set_reset_bins(self, n_bins: int, weights) -> None:
+        """Adaptive episode initialisation: weights [C, n_bins] over (clip, phase bin)."""
+        w = np.ascontiguousarray(weights, np.float32)
+        assert w.shape == (self.clips.C, n_bins)
+        self.reset_cdf = reset_cdf(w.ravel())
+        self.stat_starts = np.zeros(w.size, np.uint32)
+        self.stat_failures = np.zeros(w.size, np.uint32)
+        self.cfg.n_bins = int(n_bins)
+        self.cfg.reset_cdf = self.reset_cdf.ctypes.data
+        self.cfg.stat_starts = self.stat_starts.ctypes.data
+        self.cfg.stat_failures = self.stat_failures.ctypes.data
+
     def reset_all(self, step: int = 0) -> np.ndarray:
         obs = np.zeros((self.n, self.D))
         lib().orc_env_reset_all(self.skel.h, self.clips.h, C.byref(self.cfg), self.n, _p(self.env_ids), step,
@@ -316,3 +331,12 @@ def reset_state(skel: Skeleton, clips: Clips, cfg: EnvConfig, env: int, step: in
     lib().orc_reset_state_flat(skel.h, clips.h, C.byref(cfg), env, step, clip, np.float32(t),
                                _p(out["p"]), _p(out["q"]), _p(out["v"]), _p(out["w"]), _p(out["ql"]))
     return out
+
+
+def reset_cdf(weights) -> np.ndarray:
+    """Cumulative thresholds (uint64, in [0, 2^32]) of a flat weight table."""
+    w = np.ascontiguousarray(weights, np.float32).ravel()
+    T = np.zeros(w.size, np.uint64)
+    if lib().orc_reset_cdf(w.size, _p(w), _p(T)) != 0:
+        raise ValueError("weights must be finite, non-negative and not all zero")
+    return T

@@ -151,3 +151,85 @@ def test_grace_steps_delay_early_termination_but_not_truncation():
     env0.reset_all(0)
     sim = W.synth_sim_state(skel, lib, env0.clip_id, env0.t.astype(np.float64) + wl.dt, 1, wl)
     assert (env0.step(1, sim)["flags"] & 1).all()
+
+
+# ---------------------------------------------------------------- adaptive episode initialisation
+def test_cumulative_table_closed_forms():
+    np.testing.assert_array_equal(O.reset_cdf([1, 1, 2]), [2 ** 30, 2 ** 31, 2 ** 32])
+    np.testing.assert_array_equal(O.reset_cdf([0, 3, 0, 1, 0]), [0, 3 * 2 ** 30, 3 * 2 ** 30, 2 ** 32, 2 ** 32])
+    np.testing.assert_array_equal(O.reset_cdf([5.0]), [2 ** 32])
+    T = O.reset_cdf(np.ones(7))
+    np.testing.assert_array_equal(T[:-1], [(k * 2 ** 32) // 7 for k in range(1, 7)])
+    for bad in ([0, 0], [1, -1], [np.nan, 1], [np.inf, 1]):
+        try:
+            O.reset_cdf(bad)
+        except ValueError:
+            continue
+        raise AssertionError("accepted %r" % (bad,))
+
+
+def _binned_env(weights, n=4000, seed=11, frames=(40, 60), h_min=0.3):
+    skel, lib, o_skel, o_clips = _scene(n_clips=3, frames=frames)
+    cfg = O.make_env_config(1 / 30, seed, W.REWARD_MULT, h_min)
+    env = O.Env(o_skel, o_clips, cfg, n)
+    env.set_reset_bins(np.asarray(weights).shape[1], weights)
+    return skel, lib, o_clips, env
+
+
+def test_binned_draws_follow_the_weights_and_stay_inside_their_bin():
+    import scipy.stats
+    w = np.array([[1, 0, 2, 1], [0, 0, 0, 4], [3, 1, 0, 0]], np.float32)
+    skel, lib, o_clips, env = _binned_env(w, n=20000)
+    env.reset_all(0)
+    B = w.shape[1]
+    span = np.array([o_clips.duration(c) for c in range(3)], np.float64) - 1 / 30
+    b = np.minimum(np.floor(env.t / (span[env.clip_id] / B) * (1 + 1e-9)).astype(int), B - 1)
+    counts = np.zeros_like(w)
+    np.add.at(counts, (env.clip_id, b), 1)
+    assert (counts[w == 0] == 0).all()                                   # weight 0 is never drawn
+    expect = w / w.sum() * env.n
+    chi2 = ((counts - expect)[w > 0] ** 2 / expect[w > 0]).sum()
+    assert chi2 < scipy.stats.chi2.ppf(0.999, (w > 0).sum() - 1)
+    # uniform inside a bin: position within the bin against U(0, 1)
+    sel = (env.clip_id == 1)
+    frac = env.t[sel] / (span[1] / B) - 3
+    assert frac.min() >= -1e-6 and frac.max() <= 1 + 1e-6
+    assert scipy.stats.kstest(np.clip(frac, 0, 1), "uniform").pvalue > 1e-3
+    assert (env.t <= span[env.clip_id] + 1e-9).all()
+    np.testing.assert_array_equal(env.stat_starts.reshape(w.shape), counts.astype(np.uint32))
+
+
+def test_one_equal_bin_per_clip_is_the_uniform_distribution_over_clips():
+    import scipy.stats
+    skel, lib, o_clips, env = _binned_env(np.ones((3, 1), np.float32), n=30000)
+    env.reset_all(0)
+    counts = np.bincount(env.clip_id, minlength=3)
+    assert scipy.stats.chisquare(counts).pvalue > 1e-3
+    span = np.array([o_clips.duration(c) for c in range(3)], np.float64) - 1 / 30
+    assert scipy.stats.kstest(env.t / span[env.clip_id], "uniform").pvalue > 1e-3
+
+
+def test_failure_and_start_counts_add_up():
+    wl = W.WORKLOADS["cfg1_tiny64"]
+    B = 5
+    skel, lib, o_clips, env = _binned_env(np.ones((3, B), np.float32), n=600, h_min=W.ROOT_HEIGHT)
+    env.reset_all(0)
+    n_term = n_reset = 0
+    fail_bins = np.zeros((3, B), np.int64)
+    span = np.array([o_clips.duration(c) for c in range(3)], np.float64) - wl.dt
+    for s in range(1, 9):
+        clip_before = env.clip_id.copy()
+        t1 = (env.t + np.float32(wl.dt)).astype(np.float64)
+        sim = W.synth_sim_state(skel, lib, env.clip_id, env.t.astype(np.float64) + wl.dt, s, wl)
+        out = env.step(s, sim, want_terms=False)
+        term = (out["flags"] & 1) == 1
+        n_term += int(term.sum())
+        n_reset += int((out["flags"] != 0).sum())
+        pos = t1 / (span[clip_before] / B)
+        safe = term & (np.abs(pos - np.round(pos)) > 1e-4)               # away from bin edges the bin is unambiguous
+        np.add.at(fail_bins, (clip_before[safe], np.minimum(np.floor(pos[safe]).astype(int), B - 1)), 1)
+        assert safe.sum() >= term.sum() - 2
+    assert n_term > 100
+    assert int(env.stat_failures.sum()) == n_term
+    assert int(env.stat_starts.sum()) == env.n + n_reset
+    assert np.abs(env.stat_failures.reshape(3, B).astype(np.int64) - fail_bins).sum() <= 16
