@@ -191,6 +191,31 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim,
 im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_len);
 im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, const int32_t *ep_len);
 
+/* ---- adaptive episode initialisation --------------------------------------
+ * (The paper trains "with early termination and adaptive episode-initialization
+ * sampling", Section 6, without giving the rule; this is the mechanism such rules
+ * need, kept on the device: a weighted reset distribution and failure counts.)
+ * Each clip's start times [0, D_c - dt] are cut into n_bins equal phase bins.
+ * A reset draws the pair (clip, bin) with probability proportional to its weight
+ * and the start time uniformly inside the bin:
+ *   T_i = floor(2^32 (w_0 + ... + w_i) / sum w)   (sums in order, fp64; T_last = 2^32)
+ *   i   = smallest index with x0 < T_i, clip = i / n_bins, b = i % n_bins
+ *   t   = min(fl32(fl32(b + u) * fl32(span / n_bins)), span),  span = max(D_clip - dt, 0)
+ * with x0 and u = (x1 >> 8) 2^-24 from the same Philox block as the uniform draw,
+ * every operation a single fp32 one.  A bin of weight 0 is never drawn.
+ *   weights  HOST [C][n_bins], finite, >= 0, not all zero.  n_bins = 0 restores the
+ *            uniform draw (weights ignored).
+ * Changing n_bins reallocates the tables and clears the counts; the call waits for
+ * the env's stream (not capturable).  Counts, per (clip, bin): `starts`, episodes begun
+ * there by a reset (im_env_reset_all included); `failures`, early terminations
+ * (IM_FLAG_TERMINATED) whose time fell there, bin = min(floor(t / (span / n_bins)),
+ * n_bins - 1).  Integer atomics, so the counts do not depend on execution order.
+ * im_env_get_reset_stats copies them to DEVICE arrays of C * n_bins uint32 (either may
+ * be NULL), stream-ordered, and zeroes them afterwards if clear != 0;
+ * IM_ERR_UNSUPPORTED while n_bins == 0. */
+im_status im_env_set_reset_bins(im_env *e, int32_t n_bins, const float *weights);
+im_status im_env_get_reset_stats(im_env *e, uint32_t *starts, uint32_t *failures, int32_t clear);
+
 /* ---- policy ---------------------------------------------------------------
  * Multi-layer perceptron h_{l+1} = relu(W_l h_l + b_l), last layer linear,
  * giving the mean of a Gaussian with fixed standard deviation sigma (paper

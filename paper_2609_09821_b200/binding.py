@@ -24,7 +24,7 @@ EXPORTS = [
     "im_env_set_state", "im_load_policy", "im_destroy_policy", "im_policy_forward",
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
-    "im_value_forward", "im_value_forward_staged", "im_gae",
+    "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
 ]
 
 
@@ -94,6 +94,8 @@ def load():
         L.im_env_attach_policy.argtypes = [vp, vp]
         L.im_policy_forward_staged.argtypes = [vp, u32, i32, vp, vp, vp]
         L.im_policy_forward_noalloc.argtypes = [i32, vp, vp, vp, C.c_float, u64, u32, u32, i32, vp, i32, vp, vp, vp, vp]
+        L.im_env_set_reset_bins.argtypes = [vp, i32, vp]
+        L.im_env_get_reset_stats.argtypes = [vp, vp, vp, i32]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
@@ -192,6 +194,7 @@ class Env:
         self.skel, self.clips, self.cfg = skel, clips, cfg
         self.n, self.J, self.D, self.ld_obs = cfg.n_envs, skel.J, 24 * skel.J + 1, cfg.ld_obs
         self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.n_bins = 0
         self.h = C.c_void_p()
         _check(L.im_env_create(skel.h, clips.h, C.byref(cfg), C.c_void_p(self.stream.cuda_stream), C.byref(self.h)),
                "im_env_create")
@@ -225,6 +228,25 @@ class Env:
     def set_state(self, clip_id=None, t=None, ep_len=None):
         _check(load().im_env_set_state(self.h, _ptr(clip_id), _ptr(t), _ptr(ep_len)), "im_env_set_state")
         self.stream.synchronize()
+
+    def set_reset_bins(self, n_bins: int, weights=None):
+        """Adaptive episode initialisation: weights [C, n_bins] over (clip, phase bin); 0 bins: uniform."""
+        w = None if weights is None else _np(weights, np.float32)
+        if w is not None and w.shape != (self.clips.C, n_bins):
+            raise ValueError("weights must be [n_clips, n_bins]")
+        _check(load().im_env_set_reset_bins(self.h, int(n_bins), _ptr(w)), "im_env_set_reset_bins")
+        self.n_bins = int(n_bins)
+
+    def reset_stats(self, clear: bool = False):
+        """(starts, failures) per (clip, phase bin) as CUDA int32 tensors [C, n_bins] (uint32 counts)."""
+        import torch
+        with torch.cuda.stream(self.stream):
+            starts = torch.empty((self.clips.C, self.n_bins), dtype=torch.int32, device="cuda")
+            failures = torch.empty_like(starts)
+            _check(load().im_env_get_reset_stats(self.h, _ptr(starts), _ptr(failures), int(clear)),
+                   "im_env_get_reset_stats")
+        self.stream.synchronize()
+        return starts, failures
 
     def attach_policy(self, policy):
         """The env also writes bf16 observation rows into the policy's input staging buffer."""

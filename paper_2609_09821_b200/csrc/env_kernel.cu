@@ -215,6 +215,16 @@ __device__ __forceinline__ Vec3 reset_noise_shift(const EnvKernelParams &P, int 
     return reset_noise_vec(P, env, J);
 }
 
+// Phase bin of time t in a clip whose start times span [0, span]: floor(t / (span / B)) in single
+// fp32 operations, clamped to B - 1.
+__device__ __forceinline__ int phase_bin(float t, float span, int B)
+{
+    const float width = __fdiv_rn(span, (float)B);
+    if (!(width > 0.0f)) return 0;
+    const int b = (int)floorf(__fdiv_rn(t, width));
+    return min(max(b, 0), B - 1);
+}
+
 // Heading frame of the character the observation is taken from: origin at the
 // root's (x, y, 0), yaw of the root's rotated x axis (step a6).
 struct Heading {
@@ -311,7 +321,7 @@ __device__ __forceinline__ Quat as_quat(float4 v) { return {v.x, v.y, v.z, v.w};
 // Kernel body.  The observation row is assembled in two halves that reuse the same shared
 // memory: columns [0, c1) -- the body blocks and, if 15 J is not a multiple of 4, the phase and
 // the first target floats -- and columns [c1, D) -- the targets.
-// OPT compiles in the optional semantics (grace steps, motion randomisation); envs that use neither run
+// OPT compiles in the optional semantics (grace steps, motion randomisation, adaptive initialisation); envs that use none run
 // the instantiation without them.
 template <bool RESET_ALL, bool OPT>
 __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
@@ -457,6 +467,11 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
         bool terminated = (root_z < P.reward.h_min) || (r < P.reward.r_min);
         if (OPT && P.ep_len[envc] < P.grace_steps) terminated = false;
+        if (OPT && P.n_bins > 0 && terminated && c == 0 && valid) {
+            // adaptive initialisation statistics: the (clip, phase bin) the episode failed in
+            const float span = fmaxf(__fsub_rn(cm.dur, P.dt), 0.0f);
+            atomicAdd(P.stat_failures + clip * P.n_bins + phase_bin(t1, span, P.n_bins), 1u);
+        }
         const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
         flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
         if (c == 0 && valid) {
@@ -472,10 +487,26 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     if (reset) {
         const uint4 x = philox4x32_10(make_uint4(P.env_id_base + (uint32_t)envc, P.step, IM_STREAM_RESET, 0u),
                                       make_uint2(P.seed_lo, P.seed_hi));
-        clip_cur = (int)__umulhi(x.x, (uint32_t)P.C);
         const float u = (float)(x.y >> 8) * 5.9604644775390625e-08f;
-        const float span = fmaxf(__fsub_rn(P.meta[clip_cur].dur, P.dt), 0.0f);
-        t_cur = __fmul_rn(u, span);
+        if (OPT && P.n_bins > 0) {
+            // weighted (clip, phase bin) from the cumulative table: smallest i with x < T_i
+            const int B = P.n_bins;
+            int lo = 0, hi = P.C * B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if ((unsigned long long)x.x < __ldg(P.reset_cdf + mid)) hi = mid;
+                else lo = mid + 1;
+            }
+            clip_cur = lo / B;
+            const float span = fmaxf(__fsub_rn(P.meta[clip_cur].dur, P.dt), 0.0f);
+            const float width = __fdiv_rn(span, (float)B);
+            t_cur = fminf(__fmul_rn(__fadd_rn((float)(lo - clip_cur * B), u), width), span);
+            if (c == 0 && valid) atomicAdd(P.stat_starts + lo, 1u);
+        } else {
+            clip_cur = (int)__umulhi(x.x, (uint32_t)P.C);
+            const float span = fmaxf(__fsub_rn(P.meta[clip_cur].dur, P.dt), 0.0f);
+            t_cur = __fmul_rn(u, span);
+        }
     }
     if (c == 0 && valid) {
         P.clip_id[env] = clip_cur;
@@ -665,7 +696,7 @@ cudaError_t env_kernel_prepare(size_t smem)
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
-    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f;
+    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0;
     if (opt) {
         if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
         else launch_one<false, true>(p, grid, block, smem, stream);

@@ -215,6 +215,7 @@ void im_env_destroy(im_env *e)
     cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status);
     cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
     cudaFree(e->d_action); cudaFree(e->d_flags);
+    cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
     if (e->h2d_stream) cudaStreamDestroy(e->h2d_stream);
     if (e->d2h_stream) cudaStreamDestroy(e->d2h_stream);
     if (e->ev_h2d) cudaEventDestroy(e->ev_h2d);
@@ -239,6 +240,10 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.write_back = e->cfg.write_back_reset;
     p.grace_steps = e->cfg.grace_steps;
     p.reset_noise_std = e->cfg.reset_noise_std;
+    p.n_bins = e->n_bins;
+    p.reset_cdf = e->d_reset_cdf;
+    p.stat_starts = e->d_stat_starts;
+    p.stat_failures = e->d_stat_failures;
     p.step = step;
     p.clip_id = e->d_clip_id;
     p.t = e->d_t;
@@ -406,6 +411,72 @@ im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n, float
     if (!p->tensor_path) return IM_ERR_UNSUPPORTED;
     if (n < 1 || n > p->cfg.max_batch || !aligned16(mean_out) || !aligned16(action_out)) return IM_ERR_INVALID_ARG;
     return tc_policy_forward(p, step, n, nullptr, 0, mean_out, action_out, logp_out);
+}
+
+/* ------------------------------------------------------------------ adaptive episode initialisation */
+im_status im_env_set_reset_bins(im_env *e, int32_t n_bins, const float *weights)
+{
+    if (!e || n_bins < 0 || (n_bins > 0 && !weights)) return IM_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)e->clips->C * n_bins;
+    if (n > (1 << 26)) return IM_ERR_INVALID_ARG;
+    std::vector<unsigned long long> T;
+    try {
+        T.resize((size_t)n);
+    } catch (const std::bad_alloc &) {
+        return IM_ERR_ALLOC;
+    }
+    if (n_bins > 0) {
+        // T_i = floor(2^32 (w_0 + .. + w_i) / total), sums in order in fp64, last entry 2^32
+        double total = 0.0, cum = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            if (!(weights[i] >= 0.0f) || std::isinf(weights[i])) return IM_ERR_INVALID_ARG;
+            total += (double)weights[i];
+        }
+        if (!(total > 0.0)) return IM_ERR_INVALID_ARG;
+        for (int64_t i = 0; i < n; ++i) {
+            cum += (double)weights[i];
+            T[(size_t)i] = (unsigned long long)std::floor(cum / total * 4294967296.0);
+        }
+        T[(size_t)n - 1] = 4294967296ull;
+    }
+    if (n_bins != e->n_bins) {
+        // kernels enqueued earlier may still read the old tables
+        IM_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
+        e->d_reset_cdf = nullptr; e->d_stat_starts = e->d_stat_failures = nullptr;
+        e->n_bins = 0;
+        if (n_bins > 0) {
+            if (cudaMalloc(&e->d_reset_cdf, (size_t)n * 8) != cudaSuccess ||
+                cudaMalloc(&e->d_stat_starts, (size_t)n * 4) != cudaSuccess ||
+                cudaMalloc(&e->d_stat_failures, (size_t)n * 4) != cudaSuccess) {
+                cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
+                e->d_reset_cdf = nullptr; e->d_stat_starts = e->d_stat_failures = nullptr;
+                return IM_ERR_ALLOC;
+            }
+            e->n_bins = n_bins;
+            IM_CUDA(cudaMemsetAsync(e->d_stat_starts, 0, (size_t)n * 4, e->stream));
+            IM_CUDA(cudaMemsetAsync(e->d_stat_failures, 0, (size_t)n * 4, e->stream));
+        }
+    }
+    if (n_bins > 0) {
+        IM_CUDA(cudaMemcpyAsync(e->d_reset_cdf, T.data(), (size_t)n * 8, cudaMemcpyHostToDevice, e->stream));
+        IM_CUDA(cudaStreamSynchronize(e->stream));      // T is a local
+    }
+    return IM_OK;
+}
+
+im_status im_env_get_reset_stats(im_env *e, uint32_t *starts, uint32_t *failures, int32_t clear)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    if (e->n_bins <= 0) return IM_ERR_UNSUPPORTED;
+    const size_t bytes = (size_t)e->clips->C * e->n_bins * 4;
+    if (starts) IM_CUDA(cudaMemcpyAsync(starts, e->d_stat_starts, bytes, cudaMemcpyDeviceToDevice, e->stream));
+    if (failures) IM_CUDA(cudaMemcpyAsync(failures, e->d_stat_failures, bytes, cudaMemcpyDeviceToDevice, e->stream));
+    if (clear) {
+        IM_CUDA(cudaMemsetAsync(e->d_stat_starts, 0, bytes, e->stream));
+        IM_CUDA(cudaMemsetAsync(e->d_stat_failures, 0, bytes, e->stream));
+    }
+    return IM_OK;
 }
 
 /* ------------------------------------------------------------------ value head */

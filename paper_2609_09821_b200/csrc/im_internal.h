@@ -50,6 +50,9 @@ struct EnvKernelParams {
     int32_t write_back;
     int32_t grace_steps;
     float reset_noise_std;
+    int32_t n_bins;                          // adaptive initialisation: phase bins per clip (0: uniform draw)
+    const unsigned long long *reset_cdf;     // [C * n_bins] exclusive upper thresholds in [0, 2^32]
+    uint32_t *stat_starts, *stat_failures;   // [C * n_bins]
     uint32_t step;
     // per-env state
     int32_t *clip_id;
@@ -95,6 +98,9 @@ struct im_env {
     int D;                 // 24J + 1
     size_t smem_bytes;
     uint16_t *d_obs_bf16;  // attached policy's bf16 input rows (null when detached)
+    int32_t n_bins;        // adaptive initialisation (0: off)
+    unsigned long long *d_reset_cdf;
+    uint32_t *d_stat_starts, *d_stat_failures;
     // staging for the *_host entry points (allocated on first use)
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
     uint8_t *d_flags;

@@ -139,3 +139,45 @@ def test_env_options_are_validated():
     for kw in (dict(grace_steps=-1), dict(reset_noise_std=-0.1), dict(reset_noise_std=float("nan"))):
         with pytest.raises(B.ImError):
             B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, 1 / 30, 0, W.REWARD_MULT, 0.3, 384, **kw))
+
+
+def test_adaptive_initialisation_draws_and_counts_match_the_oracle():
+    """Weighted (clip, phase bin) resets: clip ids, start times (bit patterns) and the start/failure
+    counts against the oracle over a rollout with frequent terminations; then new weights mid-run."""
+    sc = _scene("edge_bins", (361, 64, 28), "f32", n_clips=4, frames=(20, 45), sigma_root=0.05)
+    n, B_ = 500, 6
+    g = np.random.default_rng(3)
+    w = g.uniform(0.0, 1.0, (4, B_)).astype(np.float32)
+    w[1, :] = 0.0                                        # a clip that is never started
+    w[2, 3] = 0.0
+    p = Pair(sc, n, h_min=W.ROOT_HEIGHT, with_policy=False, seed=21, grace_steps=1)
+    p.o_env.set_reset_bins(B_, w)
+    p.g_env.set_reset_bins(B_, w)
+    h = p.rollout(steps=5)                               # Pair checks clip ids and time bit patterns every step
+    assert sum(int((x["flags"] & 1).sum()) for x in h) > 200
+    starts, failures = p.g_env.reset_stats()
+    np.testing.assert_array_equal(starts.cpu().numpy().ravel(), p.o_env.stat_starts.view(np.int32))
+    np.testing.assert_array_equal(failures.cpu().numpy().ravel(), p.o_env.stat_failures.view(np.int32))
+    assert starts[1].sum() == 0 and starts[2, 3] == 0 and int(starts.sum()) > n
+    # new weights, same bin count: tables are replaced, counts go on
+    w2 = np.ones((4, B_), np.float32)
+    p.o_env.set_reset_bins(B_, w2)
+    p.o_env.stat_starts[:] = starts.cpu().numpy().ravel().view(np.uint32)
+    p.o_env.stat_failures[:] = failures.cpu().numpy().ravel().view(np.uint32)
+    p.g_env.set_reset_bins(B_, w2)
+    sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                  torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, 6, sc.wl)
+    p.env_step(6, sim)
+    starts, failures = p.g_env.reset_stats(clear=True)
+    np.testing.assert_array_equal(starts.cpu().numpy().ravel(), p.o_env.stat_starts.view(np.int32))
+    np.testing.assert_array_equal(failures.cpu().numpy().ravel(), p.o_env.stat_failures.view(np.int32))
+    assert starts[1].sum() > 0
+    z, _ = p.g_env.reset_stats()
+    assert int(z.sum()) == 0
+    # back to the uniform draw
+    p.g_env.set_reset_bins(0)
+    with pytest.raises(B.ImError):
+        p.g_env.reset_stats()
+    for bad in (np.zeros((4, B_)), -np.ones((4, B_)), np.full((4, B_), np.nan)):
+        with pytest.raises(B.ImError):
+            p.g_env.set_reset_bins(B_, bad)
