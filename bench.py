@@ -182,7 +182,7 @@ def main():
             return
         res = oracle_leg(wl, skel, lib, pol, n_sample=2048, steps=K, warmup=Wm, budget_s=60.0)
         sample = "first %d envs of %s, %d steps" % (res["n"], wl.name, res["steps"])
-        line = dict(metric=METRIC, value=res["value"], unit=UNIT, n_gpus=0, steps=res["steps"], warmup=Wm,
+        line = dict(metric=METRIC, value=res["value"], unit=UNIT, n_gpus=args.gpus, steps=res["steps"], warmup=Wm,
                     ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="f64", data="synthetic", impl="reference", config=config,
                     cpu_baseline=dict(value=res["value"], unit=UNIT, cores=res["cores"], kind="oracle", sample=sample),
