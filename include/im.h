@@ -185,6 +185,32 @@ im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out);
 im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim,
                       float *obs_out, float *reward_out, uint8_t *flags_out, float *terms_out);
 
+/* The same step on a simulator's own arrays (array of structures), read where they
+ * are (the paper's Section 4.2: post-physics kernels take simulator state from the
+ * GPU-resident arrays, no host copy).  Element (env e, body j, component c) of an
+ * array is base[e * env_stride + j * body_stride + c]; strides in floats, so arrays
+ * with a leading world body (point base at body 1), or spatial velocities stored as
+ * six floats per body (point linvel and angvel into the same array, body_stride 6),
+ * are described without copying.  pos, linvel, angvel have 3 components, quat 4
+ * (w,x,y,z).  DEVICE; no alignment requirement.
+ * One gather kernel transposes the records into component rows inside the library
+ * (first call allocates that buffer: not capturable), then the env kernel runs as in
+ * im_env_step -- results are identical to im_env_step on the transposed data.  With
+ * write_back_reset, the states of reset envs are scattered back into the caller's
+ * arrays. */
+typedef struct {
+    float *base;
+    int64_t env_stride;
+    int32_t body_stride;
+} im_aos_array;
+
+typedef struct {
+    im_aos_array pos, quat, linvel, angvel;
+} im_body_state_aos;
+
+im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim,
+                          float *obs_out, float *reward_out, uint8_t *flags_out, float *terms_out);
+
 /* Copies the per-env state to / from DEVICE arrays of N elements (stream
  * ordered); with the step number this is all that is needed to resume a
  * rollout bit-exactly.  Any pointer may be NULL to skip that array. */

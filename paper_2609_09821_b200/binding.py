@@ -25,6 +25,7 @@ EXPORTS = [
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
+    "im_env_step_aos",
 ]
 
 
@@ -37,6 +38,14 @@ class EnvConfig(C.Structure):
     _fields_ = [("n_envs", C.c_int32), ("env_id_base", C.c_uint32), ("dt", C.c_float), ("seed", C.c_uint64),
                 ("reward", RewardConfig), ("ld_obs", C.c_int32), ("write_back_reset", C.c_int32),
                 ("grace_steps", C.c_int32), ("reset_noise_std", C.c_float)]
+
+
+class AosArray(C.Structure):
+    _fields_ = [("base", C.c_void_p), ("env_stride", C.c_int64), ("body_stride", C.c_int32)]
+
+
+class BodyStateAos(C.Structure):
+    _fields_ = [("pos", AosArray), ("quat", AosArray), ("linvel", AosArray), ("angvel", AosArray)]
 
 
 class BodyState(C.Structure):
@@ -82,6 +91,7 @@ def load():
         L.im_env_destroy.argtypes = [vp]
         L.im_env_reset_all.argtypes = [vp, u32, vp]
         L.im_env_step.argtypes = [vp, u32, C.POINTER(BodyState), vp, vp, vp, vp]
+        L.im_env_step_aos.argtypes = [vp, u32, C.POINTER(BodyStateAos), vp, vp, vp, vp]
         L.im_env_get_state.argtypes = [vp, vp, vp, vp]
         L.im_env_set_state.argtypes = [vp, vp, vp, vp]
         L.im_load_policy.argtypes = [C.POINTER(PolicyConfig), vp, vp, vp, C.POINTER(vp)]
@@ -214,6 +224,17 @@ class Env:
         bs = BodyState(base, base + 3 * J * stride * 4, base + 7 * J * stride * 4, base + 10 * J * stride * 4, stride)
         _check(load().im_env_step(self.h, step, C.byref(bs), _ptr(obs_out), _ptr(reward_out), _ptr(flags_out),
                                   _ptr(terms_out)), "im_env_step")
+
+    def step_aos(self, step: int, pos, quat, linvel, angvel, obs_out, reward_out, flags_out, terms_out=None):
+        """One step on simulator-native arrays: CUDA float32 tensors (or views) indexed [env, body, component];
+        any strides along env and body, components contiguous."""
+        def arr(t, comps):
+            if t.dim() != 3 or t.shape[0] != self.n or t.shape[1] != self.J or t.shape[2] != comps or t.stride(2) != 1:
+                raise ValueError("expected a [%d, %d, %d] view with contiguous components" % (self.n, self.J, comps))
+            return AosArray(t.data_ptr(), t.stride(0), t.stride(1))
+        sim = BodyStateAos(arr(pos, 3), arr(quat, 4), arr(linvel, 3), arr(angvel, 3))
+        _check(load().im_env_step_aos(self.h, step, C.byref(sim), _ptr(obs_out), _ptr(reward_out), _ptr(flags_out),
+                                      _ptr(terms_out)), "im_env_step_aos")
 
     def get_state(self):
         import torch

@@ -62,12 +62,6 @@ __device__ __forceinline__ void lookup(const ClipMeta &m, float time, int &row, 
     row = m.start + k;
 }
 
-__device__ __forceinline__ Quat ld_quat(const float4 *p)
-{
-    const float4 v = __ldg(p);
-    return {v.x, v.y, v.z, v.w};
-}
-
 // asin(y)^2 / y^2 as a series in u = y^2:  1/2 sum_n (4u)^n / (n^2 C(2n,n)) / u.
 // Eight terms: relative truncation error below 1e-8 for u <= 0.15.
 __device__ __forceinline__ float asin2_over_u(float u)

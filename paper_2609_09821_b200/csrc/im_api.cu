@@ -216,6 +216,7 @@ void im_env_destroy(im_env *e)
     cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
     cudaFree(e->d_action); cudaFree(e->d_flags);
     cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
+    cudaFree(e->d_aos_sim);
     if (e->h2d_stream) cudaStreamDestroy(e->h2d_stream);
     if (e->d2h_stream) cudaStreamDestroy(e->d2h_stream);
     if (e->ev_h2d) cudaEventDestroy(e->ev_h2d);
@@ -277,6 +278,33 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float 
     p.stride = sim->comp_stride;
     p.obs = obs_out; p.reward_out = reward_out; p.flags_out = flags_out; p.terms_out = terms_out;
     IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim, float *obs_out, float *reward_out,
+                          uint8_t *flags_out, float *terms_out)
+{
+    if (!e || !sim || !obs_out || !reward_out || !flags_out || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
+    const int J = e->skel->dev.J, N = e->cfg.n_envs;
+    const im_aos_array *arr[4] = {&sim->pos, &sim->quat, &sim->linvel, &sim->angvel};
+    for (int i = 0; i < 4; ++i) {
+        const int comps = i == 1 ? 4 : 3;
+        if (!arr[i]->base || arr[i]->body_stride < comps ||
+            arr[i]->env_stride < (int64_t)(J - 1) * arr[i]->body_stride + comps)
+            return IM_ERR_INVALID_ARG;
+    }
+    const int64_t stride = ((int64_t)N + 3) / 4 * 4;
+    if (!e->d_aos_sim) {
+        if (aos_adapter_prepare() != cudaSuccess) return IM_ERR_CUDA;
+        if (cudaMalloc(&e->d_aos_sim, (size_t)13 * J * stride * sizeof(float)) != cudaSuccess) return IM_ERR_ALLOC;
+    }
+    IM_CUDA(launch_aos_gather(*sim, J, N, e->d_aos_sim, stride, e->stream));
+    im_body_state rows = {e->d_aos_sim, e->d_aos_sim + 3 * J * stride, e->d_aos_sim + 7 * J * stride,
+                          e->d_aos_sim + 10 * J * stride, stride};
+    const im_status s = im_env_step(e, step, &rows, obs_out, reward_out, flags_out, terms_out);
+    if (s != IM_OK) return s;
+    if (e->cfg.write_back_reset)
+        IM_CUDA(launch_aos_scatter_reset(*sim, J, N, e->d_aos_sim, stride, flags_out, e->stream));
     return IM_OK;
 }
 

@@ -102,6 +102,7 @@ struct im_env {
     unsigned long long *d_reset_cdf;
     uint32_t *d_stat_starts, *d_stat_failures;
     // staging for the *_host entry points (allocated on first use)
+    float *d_aos_sim;      // component rows gathered from array-of-structures inputs (allocated on first use)
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
     uint8_t *d_flags;
     int staged_A;
@@ -114,4 +115,9 @@ namespace im {
 size_t env_kernel_smem_bytes(int J, int n_chains);
 cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
+// simulator-native (array of structures) body states <-> component rows [13 J][stride]
+cudaError_t aos_adapter_prepare();
+cudaError_t launch_aos_gather(const im_body_state_aos &sim, int J, int N, float *soa, long long stride, cudaStream_t stream);
+cudaError_t launch_aos_scatter_reset(const im_body_state_aos &sim, int J, int N, const float *soa, long long stride,
+                                     const uint8_t *flags, cudaStream_t stream);
 }  // namespace im

@@ -181,7 +181,7 @@ struct SmemPlan {
     static constexpr int kBarBytes = 256;
     static constexpr int kMaxStages = 8;
     // hidden layers: two staging slabs per epilogue warp for the TMA stores
-    static constexpr int kHiddenEpiBytes = 4 * 2 * kEpiSlabBytes;
+    static constexpr __host__ __device__ int hidden_epi_bytes() { return 4 * 2 * kEpiSlabBytes; }
     // head: [2 accumulators][mean, action][128 rows][A] floats laid out as in global memory,
     // partial sums of z^2 [2][4][128], band counters [2][4]
     __host__ __device__ static constexpr int head_epi_bytes(int A) { return (2 * 2 * 128 * A * 4 + 2 * 4 * 128 * 4 + 64 + 1023) / 1024 * 1024; }
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
 {
     using Plan = SmemPlan<BLOCK_N>;
     extern __shared__ uint8_t smem_raw[];
-    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::kHiddenEpiBytes);
+    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::hidden_epi_bytes());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
     pipe_init<Plan>(p, kEpiWarps);
@@ -847,8 +847,8 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
         prepared = true;
     }
     GemmParams gp = gp_in;
-    gp.stages = Plan::stages_for(Plan::kHiddenEpiBytes);
-    const size_t smem = Plan::bytes(gp.stages, Plan::kHiddenEpiBytes);
+    gp.stages = Plan::stages_for(Plan::hidden_epi_bytes());
+    const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
     const int grid = tiles < n_sm ? tiles : n_sm;
     linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);

@@ -181,3 +181,55 @@ def test_adaptive_initialisation_draws_and_counts_match_the_oracle():
     for bad in (np.zeros((4, B_)), -np.ones((4, B_)), np.full((4, B_), np.nan)):
         with pytest.raises(B.ImError):
             p.g_env.set_reset_bins(B_, bad)
+
+
+# ---------------------------------------------------------------- simulator-native input arrays
+@pytest.mark.parametrize("skeleton,dims,n", [("humanoid15", (361, 64, 28), 333), ("smpl24", (577, 64, 69), 200)])
+def test_step_on_array_of_structures_inputs(skeleton, dims, n):
+    """Body states laid out as a physics engine keeps them -- [env][body][component] with a leading world
+    body and angular|linear velocity stored as six floats -- give bit for bit what the component-row
+    layout gives (which the other tests hold against the oracle), and reset envs are written back."""
+    sc = _scene("edge_aos_" + skeleton, dims, "f32", skeleton=skeleton, sigma_root=0.05)
+    J = sc.J
+    p = Pair(sc, n, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, seed=9)
+    p.reset_all()
+    ld = p.ld_obs
+    env2 = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, sc.wl.dt, 9, W.REWARD_MULT, W.ROOT_HEIGHT, ld,
+                                                           write_back_reset=True))
+    obs2 = torch.empty((n, ld), device="cuda")
+    env2.reset_all(obs2, 0)
+    rew2 = torch.empty(n, device="cuda")
+    fl2 = torch.empty(n, dtype=torch.uint8, device="cuda")
+    terms2 = torch.empty((7, n), device="cuda")
+    for s in (1, 2, 3):
+        sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                      torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, s, sc.wl).cuda()
+        xpos = torch.full((n, J + 1, 3), 7.0, device="cuda")
+        xquat = torch.full((n, J + 1, 4), 7.0, device="cuda")
+        cvel = torch.full((n, J + 1, 6), 7.0, device="cuda")
+        xpos[:, 1:] = sim[0:3 * J].reshape(J, 3, n).permute(2, 0, 1)
+        xquat[:, 1:] = sim[3 * J:7 * J].reshape(J, 4, n).permute(2, 0, 1)
+        cvel[:, 1:, 3:] = sim[7 * J:10 * J].reshape(J, 3, n).permute(2, 0, 1)
+        cvel[:, 1:, :3] = sim[10 * J:13 * J].reshape(J, 3, n).permute(2, 0, 1)
+        env2.step_aos(s, xpos[:, 1:], xquat[:, 1:], cvel[:, 1:, 3:], cvel[:, 1:, :3], obs2, rew2, fl2, terms2)
+        out = p.env_step(s, sim)                                       # component rows, checked against the oracle
+        torch.cuda.synchronize()
+        assert torch.equal(obs2, p.obs_g) and torch.equal(rew2, p.reward_g) and torch.equal(fl2, p.flags_g)
+        assert torch.equal(terms2, p.terms_g)
+        reset = torch.from_numpy(out["flags"] != 0).cuda()
+        assert 0 < int(reset.sum()) < n
+        # reset envs: the reference state arrived in the simulator's arrays; the others and the world body are untouched
+        sim_back = torch.cat([xpos[:, 1:].permute(1, 2, 0).reshape(3 * J, n), xquat[:, 1:].permute(1, 2, 0).reshape(4 * J, n),
+                              cvel[:, 1:, 3:].permute(1, 2, 0).reshape(3 * J, n),
+                              cvel[:, 1:, :3].permute(1, 2, 0).reshape(3 * J, n)])
+        assert torch.equal(sim_back[:, ~reset], sim[:, ~reset])
+        assert not torch.equal(sim_back[:, reset], sim[:, reset])
+        assert (xpos[:, 0] == 7.0).all() and (xquat[:, 0] == 7.0).all() and (cvel[:, 0] == 7.0).all()
+        c2, t2, _ = env2.get_state()
+        ref = O.reference_state(sc.o_skel, sc.o_clips, int(c2[reset][0]), float(t2[reset][0]))
+        e0 = int(torch.nonzero(reset)[0])
+        np.testing.assert_allclose(xpos[e0, 1:].cpu().numpy(), ref["p"], atol=1e-5)
+        np.testing.assert_allclose(cvel[e0, 1:, :3].cpu().numpy(), ref["w"], atol=1e-4)
+    bad = torch.zeros((n, J, 3), device="cuda")
+    with pytest.raises(ValueError):
+        env2.step_aos(4, bad[:, :, :2], xquat[:, 1:], bad, bad, obs2, rew2, fl2)
