@@ -747,11 +747,31 @@ double orc_round_bf16(double x)
  * prescribe ("bf16 operands, fp32 accumulation"): the observation and each
  * hidden activation are rounded to bf16 before they enter the next layer;
  * otherwise activations are never rounded. */
+void orc_policy_forward_std(int n_layers, const int32_t *dims, const float *const *W, const float *const *b,
+                            double sigma, const float *log_std, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
+                            int n, const uint32_t *env_ids, const double *obs, int64_t ld_obs,
+                            double *mean, double *action, double *logp, double *z_out, int n_threads,
+                            int bf16_operands);
+
 void orc_policy_forward(int n_layers, const int32_t *dims, const float *const *W, const float *const *b,
                         double sigma, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
                         int n, const uint32_t *env_ids, const double *obs, int64_t ld_obs,
                         double *mean, double *action, double *logp, double *z_out, int n_threads,
                         int bf16_operands)
+{
+    orc_policy_forward_std(n_layers, dims, W, b, sigma, NULL, seed_lo, seed_hi, step, n, env_ids, obs, ld_obs,
+                           mean, action, logp, z_out, n_threads, bf16_operands);
+}
+
+/* The same with a state-independent standard deviation per action dimension, sigma_i =
+ * exp(log_std[i]) (the "policy log std" parameter of the paper's hyper-parameter table);
+ * log_std == NULL uses the scalar sigma for every dimension.
+ * a_i = mean_i + sigma_i z_i;  logp = -0.5 sum z^2 - sum_i ln sigma_i - (A/2) ln 2 pi. */
+void orc_policy_forward_std(int n_layers, const int32_t *dims, const float *const *W, const float *const *b,
+                            double sigma, const float *log_std, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
+                            int n, const uint32_t *env_ids, const double *obs, int64_t ld_obs,
+                            double *mean, double *action, double *logp, double *z_out, int n_threads,
+                            int bf16_operands)
 {
     int maxd = 0, A = dims[n_layers];
     for (int l = 0; l <= n_layers; ++l) if (dims[l] > maxd) maxd = dims[l];
@@ -782,11 +802,13 @@ void orc_policy_forward(int n_layers, const int32_t *dims, const float *const *W
         double zz = 0.0;
         for (int o = 0; o < A; ++o) {
             mean[(int64_t)i * A + o] = h0[o];
-            action[(int64_t)i * A + o] = h0[o] + sigma * z[o];
+            action[(int64_t)i * A + o] = h0[o] + (log_std ? exp((double)log_std[o]) : sigma) * z[o];
             if (z_out) z_out[(int64_t)i * A + o] = z[o];
             zz += z[o] * z[o];
         }
-        if (logp) logp[i] = -0.5 * zz - (double)A * log(sigma) - 0.5 * (double)A * log(2.0 * M_PI);
+        double sum_log = (double)A * log(sigma);
+        if (log_std) { sum_log = 0.0; for (int o = 0; o < A; ++o) sum_log += (double)log_std[o]; }
+        if (logp) logp[i] = -0.5 * zz - sum_log - 0.5 * (double)A * log(2.0 * M_PI);
         free(h0); free(h1); free(z);
     }
 }

@@ -77,6 +77,8 @@ def lib():
         L.orc_action_noise.argtypes = [u32, u32, u32, u32, i32, vp]
         L.orc_policy_forward.argtypes = [i32, vp, vp, vp, f64, u32, u32, u32, i32, vp, vp, i64,
                                          vp, vp, vp, vp, i32, i32]
+        L.orc_policy_forward_std.argtypes = [i32, vp, vp, vp, f64, vp, u32, u32, u32, i32, vp, vp, i64,
+                                             vp, vp, vp, vp, i32, i32]
         L.orc_round_bf16.argtypes = [f64]
         L.orc_round_bf16.restype = f64
         L.orc_error_terms_flat.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp, vp]
@@ -283,9 +285,10 @@ def round_bf16(x: float) -> float:
 
 def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarray,
                    env_ids: Optional[np.ndarray] = None, n_threads: Optional[int] = None,
-                   bf16_operands: bool = False) -> dict:
+                   bf16_operands: bool = False, log_std: Optional[np.ndarray] = None) -> dict:
     """obs: fp64 [n, >=dims[0]].  W[l]: fp32 [dims[l+1], dims[l]] (bf16 weights widened exactly).
-    bf16_operands: observation and hidden activations are rounded to bf16 before each layer."""
+    bf16_operands: observation and hidden activations are rounded to bf16 before each layer.
+    log_std: fp32 [A], per-dimension standard deviation exp(log_std) instead of the scalar sigma."""
     nl = len(dims) - 1
     n = obs.shape[0]
     obs = _f64(obs)
@@ -302,7 +305,9 @@ def policy_forward(dims, W, b, sigma: float, seed: int, step: int, obs: np.ndarr
     action = np.zeros((n, A))
     logp = np.zeros(n)
     z = np.zeros((n, A))
-    lib().orc_policy_forward(nl, _p(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), float(sigma),
+    ls = None if log_std is None else np.ascontiguousarray(log_std, np.float32)
+    assert ls is None or ls.shape == (A,)
+    lib().orc_policy_forward_std(nl, _p(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), float(sigma), _p(ls),
                              seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF, step, n, _p(ids),
                              _p(obs), obs.shape[1], _p(mean), _p(action), _p(logp), _p(z),
                              int(n_threads or os.cpu_count() or 1), int(bool(bf16_operands)))

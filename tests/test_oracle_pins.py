@@ -669,6 +669,15 @@ def test_logp_is_the_gaussian_log_density():
     out = O.policy_forward(dims, Ws, bs, 0.3, 9, 2, rng.standard_normal((7, 8)))
     want = scipy.stats.norm.logpdf(out["action"], loc=out["mean"], scale=0.3).sum(axis=1)
     np.testing.assert_allclose(out["logp"], want, atol=1e-10)
+    # one standard deviation per action dimension, exp(log_std)
+    log_std = np.array([-2.0, -1.5, 0.0, 0.3, -0.7], np.float32)
+    out2 = O.policy_forward(dims, Ws, bs, 0.3, 9, 2, rng.standard_normal((7, 8)), log_std=log_std)
+    want2 = scipy.stats.norm.logpdf(out2["action"], loc=out2["mean"], scale=np.exp(log_std.astype(np.float64))).sum(axis=1)
+    np.testing.assert_allclose(out2["logp"], want2, atol=1e-10)
+    np.testing.assert_allclose(out2["action"] - out2["mean"], np.exp(log_std.astype(np.float64)) * out2["z"], atol=1e-14)
+    same = O.policy_forward(dims, Ws, bs, 0.3, 9, 2, np.zeros((3, 8)), log_std=np.full(5, math.log(0.3), np.float32))
+    ref = O.policy_forward(dims, Ws, bs, 0.3, 9, 2, np.zeros((3, 8)))
+    np.testing.assert_allclose(same["action"], ref["action"], atol=1e-7)      # log 0.3 is rounded to fp32
 
 
 def test_oracle_bf16_rounding_matches_torch():
