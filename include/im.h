@@ -277,6 +277,15 @@ im_status im_load_policy(const im_policy_config *cfg, const void *const *W, cons
                          void *cuda_stream, im_policy **out);
 void im_destroy_policy(im_policy *p);
 
+/* One standard deviation per action dimension, sigma_i = exp(log_std[i]) (the learnable,
+ * state-independent "policy log std" of the paper's hyper-parameter table): afterwards
+ * action_i = mean_i + sigma_i z_i and logp = -0.5 sum z^2 - sum_i log_std[i] - (A/2) ln 2 pi.
+ *   log_std  DEVICE [A]; copied (stream-ordered) into the policy, so an optimiser can hand
+ *            over its updated parameter between rollouts without touching the host.
+ *            NULL returns to the scalar sigma of the configuration (waits for the stream).
+ * The first call allocates the A floats. */
+im_status im_policy_set_log_std(im_policy *p, const float *log_std);
+
 /*   obs        DEVICE [n][ld_obs] float, ld_obs >= dims[0], multiple of 4, 16-byte aligned
  *   mean_out   DEVICE [n][A]     action_out DEVICE [n][A] or NULL     logp_out DEVICE [n] or NULL
  *              (mean_out and action_out 16-byte aligned on the tensor-core path)

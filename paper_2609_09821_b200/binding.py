@@ -25,7 +25,7 @@ EXPORTS = [
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
-    "im_env_step_aos",
+    "im_env_step_aos", "im_policy_set_log_std",
 ]
 
 
@@ -106,6 +106,7 @@ def load():
         L.im_policy_forward_noalloc.argtypes = [i32, vp, vp, vp, C.c_float, u64, u32, u32, i32, vp, i32, vp, vp, vp, vp]
         L.im_env_set_reset_bins.argtypes = [vp, i32, vp]
         L.im_env_get_reset_stats.argtypes = [vp, vp, vp, i32]
+        L.im_policy_set_log_std.argtypes = [vp, vp]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
@@ -321,6 +322,12 @@ class Policy:
         """Forward on the bf16 rows an attached env left in the input staging buffer."""
         _check(load().im_policy_forward_staged(self.h, step, n, _ptr(mean_out), _ptr(action_out), _ptr(logp_out)),
                "im_policy_forward_staged")
+
+    def set_log_std(self, log_std):
+        """Per-dimension standard deviation exp(log_std): CUDA float32 tensor [A], or None for the scalar sigma."""
+        if log_std is not None and (tuple(log_std.shape) != (self.A,) or not log_std.is_contiguous()):
+            raise ValueError("log_std must be a contiguous [A] tensor")
+        _check(load().im_policy_set_log_std(self.h, _ptr(log_std)), "im_policy_set_log_std")
 
     def value_forward(self, obs, value_out, n: Optional[int] = None):
         """This network read as a critic: writes only its outputs ([n, dims[-1]]), draws no noise."""

@@ -400,8 +400,23 @@ void im_destroy_policy(im_policy *p)
     if (!p) return;
     if (p->tc) tc_policy_destroy(p);
     for (int l = 0; l < IM_MAX_LAYERS; ++l) { cudaFree(p->d_W[l]); cudaFree(p->d_b[l]); }
-    cudaFree(p->d_act[0]); cudaFree(p->d_act[1]); cudaFree(p->d_status);
+    cudaFree(p->d_act[0]); cudaFree(p->d_act[1]); cudaFree(p->d_status); cudaFree(p->d_log_std);
     delete p;
+}
+
+im_status im_policy_set_log_std(im_policy *p, const float *log_std)
+{
+    if (!p) return IM_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)p->cfg.dims[p->nl] * sizeof(float);
+    if (!log_std) {                                     // back to the scalar sigma of the configuration
+        IM_CUDA(cudaStreamSynchronize(p->stream));      // kernels in flight may still read the array
+        cudaFree(p->d_log_std);
+        p->d_log_std = nullptr;
+        return IM_OK;
+    }
+    if (!p->d_log_std && cudaMalloc(&p->d_log_std, bytes) != cudaSuccess) return IM_ERR_ALLOC;
+    IM_CUDA(cudaMemcpyAsync(p->d_log_std, log_std, bytes, cudaMemcpyDeviceToDevice, p->stream));
+    return IM_OK;
 }
 
 im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
@@ -427,7 +442,7 @@ im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         ld_in = ldc;
     }
     if (action_out)
-        IM_CUDA(launch_sample(mean_out, action_out, logp_out, n, A, p->cfg.sigma, p->cfg.seed, step,
+        IM_CUDA(launch_sample(mean_out, action_out, logp_out, n, A, p->cfg.sigma, p->d_log_std, p->cfg.seed, step,
                               p->cfg.env_id_base, p->stream));
     return IM_OK;
 }

@@ -15,13 +15,14 @@ struct im_policy {
     float *d_act[2];                  // SIMT path: fp32 activations, [max_batch][max hidden]
     int act_ld;
     uint32_t *d_status;
+    float *d_log_std;                 // [A] per-dimension ln(sigma) once im_policy_set_log_std has been called, else null
     struct im_policy_tc *tc;          // tensor path state (weights padded for the GEMM tiles, bf16 activations, tensor maps)
 };
 
 namespace im {
 cudaError_t launch_linear_simt(const float *A, int lda, const void *W, bool w_bf16, const float *bias, float *C,
                                int ldc, int M, int N, int K, bool relu, cudaStream_t stream);
-cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, int A, float sigma,
+cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, int A, float sigma, const float *log_std,
                           uint64_t seed, uint32_t step, uint32_t env_id_base, cudaStream_t stream);
 
 // Tensor-core path (mlp_tc.cu).

@@ -67,12 +67,16 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const float *__restric
 // action = mean + sigma z, z from Philox counter (env id, step, 1, block) and
 // Box-Muller; logp = -0.5 sum z^2 - A ln sigma - (A/2) ln 2 pi.  One thread per env.
 __global__ void sample_kernel(const float *__restrict__ mean, float *__restrict__ action, float *__restrict__ logp,
-                              int n, int A, float sigma, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
-                              uint32_t env_id_base)
+                              int n, int A, float sigma, const float *__restrict__ log_std, uint32_t seed_lo,
+                              uint32_t seed_hi, uint32_t step, uint32_t env_id_base)
 {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n) return;
-    float zz = 0.0f;
+    float zz = 0.0f, sum_log = (float)A * logf(sigma);
+    if (log_std) {
+        sum_log = 0.0f;
+        for (int i = 0; i < A; ++i) sum_log += __ldg(log_std + i);
+    }
     for (int blk = 0; 4 * blk < A; ++blk) {
         const uint4 x = philox4x32_10(make_uint4(env_id_base + (uint32_t)e, step, IM_STREAM_ACTION, (uint32_t)blk),
                                       make_uint2(seed_lo, seed_hi));
@@ -83,12 +87,13 @@ __global__ void sample_kernel(const float *__restrict__ mean, float *__restrict_
         for (int i = 0; i < 4; ++i) {
             const int o = 4 * blk + i;
             if (o < A) {
-                action[(size_t)e * A + o] = mean[(size_t)e * A + o] + sigma * z[i];
+                const float sg = log_std ? expf(__ldg(log_std + o)) : sigma;
+                action[(size_t)e * A + o] = mean[(size_t)e * A + o] + sg * z[i];
                 zz += z[i] * z[i];
             }
         }
     }
-    if (logp) logp[e] = -0.5f * zz - (float)A * logf(sigma) - 0.5f * (float)A * 1.8378770664093453f;
+    if (logp) logp[e] = -0.5f * zz - sum_log - 0.5f * (float)A * 1.8378770664093453f;
 }
 
 }  // namespace
@@ -110,10 +115,10 @@ cudaError_t launch_linear_simt(const float *A, int lda, const void *W, bool w_bf
     return cudaGetLastError();
 }
 
-cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, int A, float sigma,
+cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, int A, float sigma, const float *log_std,
                           uint64_t seed, uint32_t step, uint32_t env_id_base, cudaStream_t stream)
 {
-    sample_kernel<<<(n + 127) / 128, 128, 0, stream>>>(mean, action, logp, n, A, sigma, (uint32_t)seed,
+    sample_kernel<<<(n + 127) / 128, 128, 0, stream>>>(mean, action, logp, n, A, sigma, log_std, (uint32_t)seed,
                                                        (uint32_t)(seed >> 32), step, env_id_base);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();

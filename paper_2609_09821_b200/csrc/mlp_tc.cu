@@ -162,6 +162,7 @@ struct GemmParams {
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
+    const float *log_std;   // [N] per-column ln(sigma), or null: the scalar sigma for every column
     uint32_t seed_lo, seed_hi, step, env_id_base;
     uint32_t *status;
 };
@@ -649,7 +650,15 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
         const int row_in_tile = quad * 32 + lane;
         constexpr int kGroups = (BLOCK_N / 16) < 4 ? (BLOCK_N / 16) : 4;
         const bool sample = P.action != nullptr;                     // a value head reads only the mean
-        const float logp_const = sample ? -(float)A * logf(P.sigma) - 0.5f * (float)A * 1.8378770664093453f : 0.0f;
+        float logp_const = 0.0f;
+        if (sample) {
+            float sum_log = (float)A * logf(P.sigma);
+            if (P.log_std) {                                         // same order in every thread
+                sum_log = 0.0f;
+                for (int i = 0; i < A; ++i) sum_log += __ldg(P.log_std + i);
+            }
+            logp_const = -sum_log - 0.5f * (float)A * 1.8378770664093453f;
+        }
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -684,7 +693,10 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
                                 if (col + i < A) {
                                     const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
                                     s_mean[row_in_tile * A + col + i] = mu;
-                                    if (sample) s_act[row_in_tile * A + col + i] = mu + P.sigma * z[i];
+                                    if (sample) {
+                                        const float sg = P.log_std ? expf(__ldg(P.log_std + col + i)) : P.sigma;
+                                        s_act[row_in_tile * A + col + i] = mu + sg * z[i];
+                                    }
                                     zz += z[i] * z[i];
                                 }
                             }
@@ -1045,7 +1057,7 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
         gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
-        gp.sigma = cfg.sigma; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
+        gp.sigma = cfg.sigma; gp.log_std = p->d_log_std; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
         gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
         if (dispatch_tc(L, gp, last, tc->n_sm, cfg.impl == 2, p->stream) != cudaSuccess) return IM_ERR_CUDA;
     }

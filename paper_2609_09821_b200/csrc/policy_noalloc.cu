@@ -81,7 +81,7 @@ extern "C" im_status im_policy_forward_noalloc(int32_t n_layers, const int32_t *
         in = outp;
         ld_in = ldc;
     }
-    if (im::launch_sample(mean_out, action_out, logp_out, n, A, sigma, seed, step, env_id_base, stream) != cudaSuccess)
+    if (im::launch_sample(mean_out, action_out, logp_out, n, A, sigma, nullptr, seed, step, env_id_base, stream) != cudaSuccess)
         return IM_ERR_CUDA;
     return IM_OK;
 }

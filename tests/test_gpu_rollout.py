@@ -231,3 +231,36 @@ def test_collect_fills_storage_like_the_separate_calls(staged):
     assert np.abs(st.advantage.cpu().numpy() - adv_o).max() <= tol
     assert np.abs(st.returns.cpu().numpy() - ret_o).max() <= tol
     g_env.attach_policy(None)
+
+
+# ---------------------------------------------------------------- per-dimension standard deviation
+@pytest.mark.parametrize("dtype,dims", [("f32", (361, 64, 28)), ("bf16", (361, 128, 28)), ("bf16", (577, 256, 69))])
+def test_per_dimension_log_std(dtype, dims):
+    from tests.parity import assert_close
+    n, seed, step = 500, 0xABCDEF12345, 7
+    pw = W.make_policy_weights(dims, dtype, 3)
+    A = dims[-1]
+    g = np.random.default_rng(5)
+    obs = g.standard_normal((n, dims[0])).astype(np.float32)
+    log_std = g.uniform(-2.5, 0.5, A).astype(np.float32)          # around the paper's initial values (-2.0, -1.5)
+    pol = B.Policy(dims, pw["W_bf16"] if dtype == "bf16" else pw["W"], pw["b"], dtype, 0.1, seed, n)
+    ld = B.padded_ld(dims[0])
+    obs_g = torch.zeros((n, ld), device="cuda")
+    obs_g[:, :dims[0]] = torch.from_numpy(obs).cuda()
+    mean, act, logp = (torch.empty((n, A), device="cuda"), torch.empty((n, A), device="cuda"), torch.empty(n, device="cuda"))
+    pol.set_log_std(torch.from_numpy(log_std).cuda())
+    pol.forward(step, obs_g, mean, act, logp)
+    torch.cuda.synchronize()
+    want = O.policy_forward(dims, pw["W"], pw["b"], 0.1, seed, step, obs.astype(np.float64),
+                            bf16_operands=dtype == "bf16", log_std=log_std)
+    assert_mean_close(mean.cpu().numpy(), want["mean"], 2e-2 if dtype == "bf16" else 1e-4, "means")
+    noise = (act - mean).cpu().numpy().astype(np.float64)
+    assert_close(noise, np.exp(log_std.astype(np.float64)) * want["z"], atol=1e-5, rtol=1e-4, what="per-dimension noise")
+    assert_close(logp.cpu().numpy(), want["logp"], atol=1e-3, rtol=1e-5, what="logp")
+    # back to the scalar sigma
+    pol.set_log_std(None)
+    pol.forward(step, obs_g, mean, act, logp)
+    torch.cuda.synchronize()
+    assert_close((act - mean).cpu().numpy(), 0.1 * want["z"], atol=1e-5, rtol=1e-4, what="scalar noise")
+    with pytest.raises(ValueError):
+        pol.set_log_std(torch.zeros(A + 1, device="cuda"))
