@@ -864,6 +864,94 @@ void orc_gae(int T, int N, int64_t ld, const float *reward, const float *value, 
     }
 }
 
+/* ------------------------------------------------------------------------
+ * PPO minibatch loss and its gradients with respect to the network outputs (the paper's
+ * hyper-parameter table lists the ratio clip, the value-loss and entropy coefficients and the KL
+ * threshold; the objective is the clipped surrogate of Schulman et al. 2017 as the usual on-policy
+ * runners implement it).  For sample i of M, action dimension k of A, sigma_k = exp(log_std_k):
+ *
+ *   logp_i   = -1/2 sum_k ((a_ik - mu_ik) / sigma_k)^2 - sum_k log_std_k - A/2 ln 2 pi
+ *   r_i      = exp(logp_i - logp_old_i),      Ahat_i = (adv_i - adv_mean) adv_rstd
+ *   surr_i   = -min(r_i Ahat_i, clip(r_i, 1 - eps, 1 + eps) Ahat_i)
+ *   vl_i     = (V_i - R_i)^2, or with value clipping max((V_i - R_i)^2, (Vc_i - R_i)^2),
+ *              Vc_i = Vold_i + clip(V_i - Vold_i, -eps, eps)
+ *   H        = sum_k (log_std_k + 1/2 ln(2 pi e))                 (entropy, the same for every sample)
+ *   L        = mean_i surr_i + c_v mean_i vl_i - c_e H
+ *   kl_i     = sum_k [log_std_k - log_std_old_k + (sigma_old_k^2 + (mu_old_ik - mu_ik)^2) / (2 sigma_k^2) - 1/2]
+ *
+ * Outputs: dL/dmu [M][A], dL/dlog_std [A], dL/dV [M], and summary = {L, mean surr, mean vl, H,
+ * mean kl, fraction of samples with |r - 1| > eps}.  The branch of min / max that is active decides
+ * the gradient (on a tie both branches have the same derivative here). */
+typedef struct {
+    float clip, value_coef, entropy_coef;
+    int32_t clip_value_loss;
+} orc_ppo_config;
+
+void orc_ppo_loss(const orc_ppo_config *cfg, int64_t M, int A, const float *mean, const float *log_std,
+                  const float *action, const float *logp_old, const float *mean_old, const float *log_std_old,
+                  const float *adv, double adv_mean, double adv_rstd, const float *value, const float *value_old,
+                  const float *returns, double *d_mean, double *d_log_std, double *d_value, double *summary)
+{
+    const double eps = (double)cfg->clip, cv = (double)cfg->value_coef, ce = (double)cfg->entropy_coef;
+    double sum_log = 0.0, H = 0.0, s_surr = 0.0, s_vl = 0.0, s_kl = 0.0, s_clip = 0.0;
+    for (int k = 0; k < A; ++k) {
+        sum_log += (double)log_std[k];
+        H += (double)log_std[k] + 0.5 * log(2.0 * M_PI * exp(1.0));
+        d_log_std[k] = -ce;
+    }
+    for (int64_t i = 0; i < M; ++i) {
+        double zz = 0.0, kl = 0.0;
+        for (int k = 0; k < A; ++k) {
+            double sg = exp((double)log_std[k]), so = exp((double)log_std_old[k]);
+            double z = ((double)action[i * A + k] - (double)mean[i * A + k]) / sg;
+            double dm = (double)mean_old[i * A + k] - (double)mean[i * A + k];
+            zz += z * z;
+            kl += (double)log_std[k] - (double)log_std_old[k] + (so * so + dm * dm) / (2.0 * sg * sg) - 0.5;
+        }
+        double logp = -0.5 * zz - sum_log - 0.5 * (double)A * log(2.0 * M_PI);
+        double r = exp(logp - (double)logp_old[i]);
+        double ah = ((double)adv[i] - adv_mean) * adv_rstd;
+        double rc = r < 1.0 - eps ? 1.0 - eps : (r > 1.0 + eps ? 1.0 + eps : r);
+        double s1 = r * ah, s2 = rc * ah;
+        double g_r = s1 <= s2 ? -ah : 0.0;                 /* d surr / d r */
+        s_surr += -(s1 <= s2 ? s1 : s2);
+        s_clip += fabs(r - 1.0) > eps ? 1.0 : 0.0;
+        s_kl += kl;
+        for (int k = 0; k < A; ++k) {
+            double sg = exp((double)log_std[k]);
+            double z = ((double)action[i * A + k] - (double)mean[i * A + k]) / sg;
+            d_mean[i * A + k] = g_r * r * z / sg / (double)M;            /* dlogp/dmu = z / sigma */
+            d_log_std[k] += g_r * r * (z * z - 1.0) / (double)M;         /* dlogp/dlog_std = z^2 - 1 */
+        }
+        double v = (double)value[i], R = (double)returns[i], e1 = v - R, vl = e1 * e1, gv = 2.0 * e1;
+        if (cfg->clip_value_loss) {
+            double d = v - (double)value_old[i];
+            double dc = d < -eps ? -eps : (d > eps ? eps : d);
+            double e2 = (double)value_old[i] + dc - R;
+            if (e2 * e2 > vl) { vl = e2 * e2; gv = (d == dc) ? 2.0 * e2 : 0.0; }
+        }
+        s_vl += vl;
+        d_value[i] = cv * gv / (double)M;
+    }
+    summary[1] = s_surr / (double)M;
+    summary[2] = s_vl / (double)M;
+    summary[3] = H;
+    summary[4] = s_kl / (double)M;
+    summary[5] = s_clip / (double)M;
+    summary[0] = summary[1] + cv * summary[2] - ce * H;
+}
+
+/* Mean and 1 / (std + 1e-8) of n values, std with the n - 1 divisor (advantage normalisation). */
+void orc_moments(const float *x, int64_t n, double *mean_out, double *rstd_out)
+{
+    double s = 0.0, q = 0.0;
+    for (int64_t i = 0; i < n; ++i) s += (double)x[i];
+    double m = s / (double)n;
+    for (int64_t i = 0; i < n; ++i) q += ((double)x[i] - m) * ((double)x[i] - m);
+    *mean_out = m;
+    *rstd_out = 1.0 / (sqrt(n > 1 ? q / (double)(n - 1) : 0.0) + 1e-8);
+}
+
 int orc_openmp_enabled(void)
 {
 #ifdef _OPENMP

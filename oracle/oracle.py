@@ -86,6 +86,8 @@ def lib():
         L.orc_reset_state_flat.argtypes = [vp, vp, vp, u32, u32, i32, f32, vp, vp, vp, vp, vp]
         L.orc_reset_cdf.argtypes = [i32, vp, vp]
         L.orc_reset_cdf.restype = i32
+        L.orc_ppo_loss.argtypes = [vp, i64, i32] + [vp] * 7 + [f64, f64] + [vp] * 7
+        L.orc_moments.argtypes = [vp, i64, vp, vp]
         L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
@@ -345,3 +347,31 @@ def reset_cdf(weights) -> np.ndarray:
     if lib().orc_reset_cdf(w.size, _p(w), _p(T)) != 0:
         raise ValueError("weights must be finite, non-negative and not all zero")
     return T
+
+
+class PpoConfig(C.Structure):
+    _fields_ = [("clip", C.c_float), ("value_coef", C.c_float), ("entropy_coef", C.c_float),
+                ("clip_value_loss", C.c_int32)]
+
+
+def moments(x) -> tuple:
+    """(mean, 1 / (std + 1e-8)) with the n - 1 divisor."""
+    x = np.ascontiguousarray(x, np.float32).ravel()
+    m, r = C.c_double(), C.c_double()
+    lib().orc_moments(_p(x), x.size, C.byref(m), C.byref(r))
+    return m.value, r.value
+
+
+def ppo_loss(batch: dict, clip: float, value_coef: float, entropy_coef: float, clip_value_loss: bool,
+             adv_mean: float = 0.0, adv_rstd: float = 1.0) -> dict:
+    """batch: mean, action, mean_old [M, A]; log_std, log_std_old [A]; logp_old, advantage, value,
+    value_old, returns [M] (all read as fp32).  Returns d_mean, d_log_std, d_value, summary (fp64)."""
+    f = {k: np.ascontiguousarray(v, np.float32) for k, v in batch.items()}
+    M, A = f["mean"].shape
+    cfg = PpoConfig(np.float32(clip), np.float32(value_coef), np.float32(entropy_coef), int(bool(clip_value_loss)))
+    out = dict(d_mean=np.zeros((M, A)), d_log_std=np.zeros(A), d_value=np.zeros(M), summary=np.zeros(6))
+    lib().orc_ppo_loss(C.byref(cfg), M, A, _p(f["mean"]), _p(f["log_std"]), _p(f["action"]), _p(f["logp_old"]),
+                       _p(f["mean_old"]), _p(f["log_std_old"]), _p(f["advantage"]), float(adv_mean), float(adv_rstd),
+                       _p(f["value"]), _p(f["value_old"]), _p(f["returns"]), _p(out["d_mean"]),
+                       _p(out["d_log_std"]), _p(out["d_value"]), _p(out["summary"]))
+    return out

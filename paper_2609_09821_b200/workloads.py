@@ -426,3 +426,29 @@ def make_rollout_signals(T: int, N: int, seed: int = 0, p_term: float = 0.01, p_
     flags = (g.random((T, N), dtype=np.float32) < p_term).astype(np.uint8)
     flags |= (g.random((T, N), dtype=np.float32) < p_trunc).astype(np.uint8) << 1
     return reward, value, flags
+
+
+# ----------------------------------------------------------------------------
+# One PPO minibatch for the loss kernel
+# ----------------------------------------------------------------------------
+def make_ppo_batch(M: int, A: int, seed: int = 0, drift: float = 0.05) -> dict:
+    """Seeded stand-in for a minibatch some epochs into an update: the behaviour policy's means and
+    log-stds, actions sampled from it with their log-probabilities, and a current policy that has
+    drifted by `drift` (so a share of the probability ratios sits outside a 0.2 clip range);
+    advantages N(0, 1) * 2 + 0.3, returns and values N(0, 3^2) with values near their old ones."""
+    g = _rng(seed, 65, M, A)
+    f32 = np.float32
+    mean_old = g.standard_normal((M, A), dtype=f32)
+    log_std_old = g.uniform(-2.0, -0.5, A).astype(f32)
+    z = g.standard_normal((M, A), dtype=f32)
+    action = (mean_old + np.exp(log_std_old) * z).astype(f32)
+    logp_old = (-0.5 * (z.astype(np.float64) ** 2).sum(1) - log_std_old.astype(np.float64).sum()
+                - 0.5 * A * math.log(2.0 * math.pi)).astype(f32)
+    mean = (mean_old + drift * np.exp(log_std_old) * g.standard_normal((M, A), dtype=f32)).astype(f32)
+    log_std = (log_std_old + 0.02 * g.standard_normal(A, dtype=f32)).astype(f32)
+    value_old = (3.0 * g.standard_normal(M, dtype=f32)).astype(f32)
+    value = (value_old + 0.3 * g.standard_normal(M, dtype=f32)).astype(f32)
+    returns = (value_old + g.standard_normal(M, dtype=f32)).astype(f32)
+    advantage = (2.0 * g.standard_normal(M, dtype=f32) + 0.3).astype(f32)
+    return dict(mean=mean, log_std=log_std, action=action, logp_old=logp_old, mean_old=mean_old,
+                log_std_old=log_std_old, advantage=advantage, value=value, value_old=value_old, returns=returns)
