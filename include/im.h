@@ -347,6 +347,43 @@ im_status im_gae(const im_gae_config *cfg, int32_t T, int32_t N, int64_t ld, con
                  const float *value, const uint8_t *flags, float *advantage, float *returns,
                  void *cuda_stream);
 
+/* ---- PPO minibatch loss -------------------------------------------------------
+ * (The paper's update phase, "update_policy(storage)" in its Figure 2, with the
+ * coefficients of its hyper-parameter table: PPO ratio clip, value-loss and entropy
+ * coefficients; the mean KL below is what its KL threshold is compared with.  This
+ * call covers the part of the update between the forward and the backward GEMMs.)
+ * For sample i of M and action dimension k of A (A <= 128), sigma_k = exp(log_std_k):
+ *   logp_i = -1/2 sum_k ((a_ik - mu_ik)/sigma_k)^2 - sum_k log_std_k - A/2 ln 2 pi
+ *   r_i    = exp(logp_i - logp_old_i),   Ahat_i = (adv_i - adv_mean) adv_rstd
+ *   surr_i = -min(r_i Ahat_i, clip(r_i, 1-clip, 1+clip) Ahat_i)
+ *   vl_i   = (V_i - R_i)^2, or with clip_value_loss max(vl_i, (Vold_i + clip(V_i - Vold_i, -clip, clip) - R_i)^2)
+ *   L      = mean_i surr_i + value_coef mean_i vl_i - entropy_coef sum_k (log_std_k + 1/2 ln(2 pi e))
+ * Inputs, all DEVICE float: mean, action, mean_old [M][A]; log_std, log_std_old [A];
+ * logp_old, advantage, value, value_old (may be NULL without clip_value_loss), returns [M];
+ * adv_moments [2] = (adv_mean, adv_rstd) as im_moments writes them, or NULL for (0, 1).
+ * Outputs, DEVICE: d_mean [M][A] = dL/dmu, d_log_std [A], d_value [M] = dL/dV, and
+ * summary [6] = {L, mean surr, mean vl, entropy, mean KL(old || new), fraction of samples
+ * with |r - 1| > clip}.  fp32 arithmetic, batch sums finished in fp64 in a fixed order
+ * (bit-reproducible).  workspace: DEVICE, im_ppo_workspace_bytes() bytes, 8-byte aligned,
+ * contents irrelevant.  Two launches on cuda_stream; nothing is allocated or read on the host.
+ *
+ * im_moments: out2 = (mean, 1 / (std + 1e-8)) of n floats, std with the n - 1 divisor
+ * (advantage normalisation), accumulated in fp64; same workspace rules. */
+typedef struct {
+    float clip, value_coef, entropy_coef;
+    int32_t clip_value_loss;
+} im_ppo_config;
+
+typedef struct {
+    const float *mean, *log_std, *action, *logp_old, *mean_old, *log_std_old;
+    const float *advantage, *adv_moments, *value, *value_old, *returns;
+} im_ppo_batch;
+
+size_t im_ppo_workspace_bytes(void);
+im_status im_moments(const float *x, int64_t n, float *out2, void *workspace, void *cuda_stream);
+im_status im_ppo_loss(const im_ppo_config *cfg, int64_t M, int32_t A, const im_ppo_batch *batch, float *d_mean,
+                      float *d_log_std, float *d_value, float *summary, void *workspace, void *cuda_stream);
+
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current

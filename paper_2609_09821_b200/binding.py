@@ -25,7 +25,7 @@ EXPORTS = [
     "im_env_reset_all_host", "im_step_host", "im_poll_device_status", "im_launch_count",
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
-    "im_env_step_aos", "im_policy_set_log_std",
+    "im_env_step_aos", "im_policy_set_log_std", "im_ppo_workspace_bytes", "im_moments", "im_ppo_loss",
 ]
 
 
@@ -55,6 +55,16 @@ class BodyState(C.Structure):
 
 class GaeConfig(C.Structure):
     _fields_ = [("gamma", C.c_float), ("lam", C.c_float), ("bootstrap_truncated", C.c_int32)]
+
+
+class PpoConfig(C.Structure):
+    _fields_ = [("clip", C.c_float), ("value_coef", C.c_float), ("entropy_coef", C.c_float),
+                ("clip_value_loss", C.c_int32)]
+
+
+class PpoBatch(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("mean", "log_std", "action", "logp_old", "mean_old", "log_std_old",
+                                          "advantage", "adv_moments", "value", "value_old", "returns")]
 
 
 class PolicyConfig(C.Structure):
@@ -107,11 +117,15 @@ def load():
         L.im_env_set_reset_bins.argtypes = [vp, i32, vp]
         L.im_env_get_reset_stats.argtypes = [vp, vp, vp, i32]
         L.im_policy_set_log_std.argtypes = [vp, vp]
+        L.im_ppo_workspace_bytes.restype = C.c_size_t
+        L.im_moments.argtypes = [vp, C.c_int64, vp, vp, vp]
+        L.im_ppo_loss.argtypes = [C.POINTER(PpoConfig), C.c_int64, i32, C.POINTER(PpoBatch), vp, vp, vp, vp, vp, vp]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
-            if name not in ("im_status_string", "im_launch_count") and not name.startswith("im_destroy") \
+            if name not in ("im_status_string", "im_launch_count", "im_ppo_workspace_bytes") \
+                    and not name.startswith("im_destroy") \
                     and name != "im_env_destroy":
                 getattr(L, name).restype = i32
         _lib = L
@@ -370,6 +384,40 @@ def gae(reward, value, flags, advantage, returns, gamma: float, lam: float, boot
     st = stream if stream is not None else torch.cuda.current_stream()
     _check(load().im_gae(C.byref(cfg), T, N, ld, _ptr(reward), _ptr(value), _ptr(flags), _ptr(advantage),
                          _ptr(returns), C.c_void_p(st.cuda_stream)), "im_gae")
+
+
+def ppo_workspace():
+    """Scratch tensor for moments() and ppo_loss()."""
+    import torch
+    return torch.empty(load().im_ppo_workspace_bytes() // 8, dtype=torch.float64, device="cuda")
+
+
+def moments(x, out2, workspace, stream=None):
+    """out2 <- (mean, 1 / (std + 1e-8)) of the CUDA float32 tensor x (std with the n - 1 divisor)."""
+    import torch
+    st = stream if stream is not None else torch.cuda.current_stream()
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous")
+    _check(load().im_moments(_ptr(x), x.numel(), _ptr(out2), _ptr(workspace), C.c_void_p(st.cuda_stream)), "im_moments")
+
+
+def ppo_loss(batch: dict, d_mean, d_log_std, d_value, summary, workspace, clip: float, value_coef: float,
+             entropy_coef: float, clip_value_loss: bool, adv_moments=None, stream=None):
+    """PPO minibatch loss and output gradients.  batch: contiguous CUDA float32 tensors mean, action,
+    mean_old [M, A]; log_std, log_std_old [A]; logp_old, advantage, value, value_old, returns [M]."""
+    import torch
+    M, A = batch["mean"].shape
+    for k, v in batch.items():
+        if not v.is_contiguous() or v.dtype != torch.float32:
+            raise ValueError("batch[%r] must be a contiguous float32 tensor" % k)
+    b = PpoBatch(**{k: batch[k].data_ptr() for k in ("mean", "log_std", "action", "logp_old", "mean_old",
+                                                      "log_std_old", "advantage", "value", "returns")})
+    b.value_old = batch["value_old"].data_ptr() if batch.get("value_old") is not None else None
+    b.adv_moments = adv_moments.data_ptr() if adv_moments is not None else None
+    cfg = PpoConfig(np.float32(clip), np.float32(value_coef), np.float32(entropy_coef), int(bool(clip_value_loss)))
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().im_ppo_loss(C.byref(cfg), M, A, C.byref(b), _ptr(d_mean), _ptr(d_log_std), _ptr(d_value),
+                              _ptr(summary), _ptr(workspace), C.c_void_p(st.cuda_stream)), "im_ppo_loss")
 
 
 NOALLOC_MAX_BATCH = 1024
