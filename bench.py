@@ -339,6 +339,33 @@ def main():
         gae_bytes = T * n * 17 + n * 4
         extras = dict(gae=dict(T=T, seconds_per_launch=t_gae, algorithmic_bytes=gae_bytes,
                                achieved_gbs=gae_bytes / t_gae / 1e9, l2="256 MB read before every launch"))
+        # PPO minibatch loss: one of four minibatches of the rollout (T * n / 4 samples), moments + loss + finish
+        Mb = T * n // 4
+        pb = {k: torch.from_numpy(v).to(dev) for k, v in W.make_ppo_batch(min(Mb, 65536), A, wl.seed, drift=0.02).items()}
+        reps_rows = (Mb + pb["mean"].shape[0] - 1) // pb["mean"].shape[0]
+        for k in ("mean", "action", "mean_old"):
+            pb[k] = pb[k].repeat(reps_rows, 1)[:Mb].contiguous()
+        for k in ("logp_old", "advantage", "value", "value_old", "returns"):
+            pb[k] = pb[k].repeat(reps_rows)[:Mb].contiguous()
+        ws, mom = B.ppo_workspace(), torch.empty(2, device=dev)
+        outs = [torch.empty((Mb, A), device=dev), torch.empty(A, device=dev), torch.empty(Mb, device=dev),
+                torch.empty(6, device=dev)]
+        t_ppo = []
+        for i in range(3 + reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            B.moments(pb["advantage"], mom, ws, stream=stream)
+            B.ppo_loss(pb, *outs, ws, 0.2, 2.0, 2.5e-4, True, adv_moments=mom, stream=stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                t_ppo.append(a.elapsed_time(b) * 1e-3)
+        t_ppo = float(np.median(t_ppo))
+        ppo_bytes = Mb * ((3 * A + 5) * 4 + (A + 1) * 4 + 4)
+        extras["ppo_loss"] = dict(rows=Mb, A=A, seconds_per_launch=t_ppo, algorithmic_bytes=ppo_bytes,
+                                  achieved_gbs=ppo_bytes / t_ppo / 1e9,
+                                  l2="%.0f MB working set, larger than L2" % (ppo_bytes / 1e6))
+        del pb, outs
         if staged:
             cdims = tuple(wl.mlp_dims[:-1]) + (1,)
             cw = W.make_policy_weights(cdims, "bf16", wl.seed + 1)
@@ -419,6 +446,7 @@ def main():
         line["e2e"] = e2e
     if extras is not None:
         extras["gae"]["frac_of_hbm_peak"] = extras["gae"]["achieved_gbs"] / peaks["hbm_gbs"]
+        extras["ppo_loss"]["frac_of_hbm_peak"] = extras["ppo_loss"]["achieved_gbs"] / peaks["hbm_gbs"]
         if "value_head" in extras:
             extras["value_head"]["frac_of_tensor_peak"] = extras["value_head"]["achieved_tflops"] / tensor_peak
         line["rollout_extras"] = extras

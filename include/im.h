@@ -365,7 +365,10 @@ im_status im_gae(const im_gae_config *cfg, int32_t T, int32_t N, int64_t ld, con
  * summary [6] = {L, mean surr, mean vl, entropy, mean KL(old || new), fraction of samples
  * with |r - 1| > clip}.  fp32 arithmetic, batch sums finished in fp64 in a fixed order
  * (bit-reproducible).  workspace: DEVICE, im_ppo_workspace_bytes() bytes, 8-byte aligned,
- * contents irrelevant.  Two launches on cuda_stream; nothing is allocated or read on the host.
+ * contents irrelevant.  Two or three launches on cuda_stream; nothing is allocated or read on the
+ * host.  When the [M] and [M][A] arrays are 16-byte aligned, whole 32-row tiles travel as bulk
+ * asynchronous copies (the fast path); otherwise, and for the rows after the last full tile, rows
+ * are fetched element by element.  Per-row results do not depend on the path.
  *
  * im_moments: out2 = (mean, 1 / (std + 1e-8)) of n floats, std with the n - 1 divisor
  * (advantage normalisation), accumulated in fp64; same workspace rules. */

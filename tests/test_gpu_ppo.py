@@ -98,6 +98,29 @@ def test_ppo_loss_is_bit_reproducible_and_capturable():
     np.testing.assert_array_equal(out[3].cpu().numpy(), a["summary"])
 
 
+def test_unaligned_arrays_take_the_element_wise_path():
+    """Arrays that start 4 bytes off a 16-byte boundary cannot use bulk copies; same results."""
+    M, A = 3000, 69
+    b = W.make_ppo_batch(M, A, seed=8, drift=0.02)
+    ref = run_gpu(b, 0.2, 2.0, 1e-3, True, False)
+
+    def shifted(v):
+        buf = torch.empty(v.size + 1, device="cuda")
+        buf[1:] = torch.from_numpy(v.ravel()).cuda()
+        return buf[1:].view(*v.shape)
+    t = {k: shifted(v) for k, v in b.items()}
+    assert t["mean"].data_ptr() % 16 == 4
+    ws = B.ppo_workspace()
+    d_mean, d_value = shifted(np.zeros((M, A), np.float32)), shifted(np.zeros(M, np.float32))
+    d_log_std, summary = torch.empty(A, device="cuda"), torch.empty(6, device="cuda")
+    B.ppo_loss(t, d_mean, d_log_std, d_value, summary, ws, 0.2, 2.0, 1e-3, True)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(d_mean.cpu().numpy(), ref["d_mean"])        # same arithmetic per row
+    np.testing.assert_array_equal(d_value.cpu().numpy(), ref["d_value"])
+    np.testing.assert_allclose(d_log_std.cpu().numpy(), ref["d_log_std"], rtol=1e-4, atol=1e-7)   # other summation order
+    np.testing.assert_allclose(summary.cpu().numpy(), ref["summary"], rtol=1e-5)
+
+
 def test_moments_edge_cases():
     ws = B.ppo_workspace()
     out = torch.empty(2, device="cuda")
