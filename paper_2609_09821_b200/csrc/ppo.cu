@@ -569,11 +569,6 @@ im_status im_ppo_loss(const im_ppo_config *cfg, int64_t M, int32_t A, const im_p
             cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
         }
         const size_t smem = 2 * (size_t)stage_floats(A, T) * sizeof(float);
-        int per_sm = (int)((200 * 1024) / (smem + 4096));
-        per_sm = per_sm < 1 ? 1 : (per_sm > 6 ? 6 : per_sm);
-        long long gb = (long long)n_sm * per_sm;
-        grid_bulk = (int)(gb > n_tiles ? n_tiles : gb);
-        if (grid_bulk > kMaxGrid) grid_bulk = kMaxGrid;
         p.row_begin = 0; p.partial_begin = 0;
 #define IM_PPO_BULK(LPR, NI)                                                                                        \
         do {                                                                                                        \
@@ -584,7 +579,14 @@ im_status im_ppo_loss(const im_ppo_config *cfg, int64_t M, int32_t A, const im_p
                     return IM_ERR_CUDA;                                                                             \
                 prepared = true;                                                                                    \
             }                                                                                                       \
-            ppo_loss_bulk_kernel<LPR, NI><<<grid_bulk, 32 * bulk_warps(LPR), smem, st>>>(p, n_tiles, T);                        \
+            int per_sm = 1;   /* persistent grid: as many CTAs as are resident at once */                         \
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ppo_loss_bulk_kernel<LPR, NI>,                   \
+                                                          32 * bulk_warps(LPR), smem);                              \
+            per_sm = per_sm < 1 ? 1 : per_sm;                                                                       \
+            const long long gb = (long long)n_sm * per_sm;                                                          \
+            grid_bulk = (int)(gb > n_tiles ? n_tiles : gb);                                                         \
+            if (grid_bulk > kMaxGrid) grid_bulk = kMaxGrid;                                                         \
+            ppo_loss_bulk_kernel<LPR, NI><<<grid_bulk, 32 * bulk_warps(LPR), smem, st>>>(p, n_tiles, T);            \
         } while (0)
         IM_PPO_DISPATCH(IM_PPO_BULK)
 #undef IM_PPO_BULK
