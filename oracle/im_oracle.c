@@ -952,6 +952,51 @@ void orc_moments(const float *x, int64_t n, double *mean_out, double *rstd_out)
     *rstd_out = 1.0 / (sqrt(n > 1 ? q / (double)(n - 1) : 0.0) + 1e-8);
 }
 
+/* ------------------------------------------------------------------------
+ * Optimiser step of the update (Adam, Kingma & Ba 2015, with bias correction, as in the usual
+ * deep-learning libraries), global-norm gradient clipping and the KL-adaptive learning rate
+ * that the paper's "KL threshold" hyper-parameter belongs to.
+ *
+ *   g      = grad * grad_scale
+ *   m      = b1 m + (1 - b1) g,    v = b2 v + (1 - b2) g^2
+ *   param -= lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)            t = 1, 2, ...
+ *
+ *   grad_scale = min(1, max_norm / (||all grads||_2 + 1e-6))                (norm over every tensor)
+ *
+ *   lr' = max(lr / 1.5, lr_min) if kl > 2 kl_target;  min(lr * 1.5, lr_max) if 0 < kl < kl_target / 2;
+ *         lr otherwise                                                      (the adaptive schedule of
+ *                                                                            common on-policy runners)
+ * fp32 inputs and state, fp64 arithmetic, results rounded to fp32 once. */
+void orc_adam_step(int64_t n, float *param, const float *grad, float *m, float *v, double lr, double b1,
+                   double b2, double eps, int t, double grad_scale)
+{
+    const double c1 = 1.0 - pow(b1, (double)t), c2 = 1.0 - pow(b2, (double)t);
+    for (int64_t i = 0; i < n; ++i) {
+        const double g = (double)grad[i] * grad_scale;
+        const double mi = b1 * (double)m[i] + (1.0 - b1) * g;
+        const double vi = b2 * (double)v[i] + (1.0 - b2) * g * g;
+        m[i] = (float)mi;
+        v[i] = (float)vi;
+        param[i] = (float)((double)param[i] - lr * (mi / c1) / (sqrt(vi / c2) + eps));
+    }
+}
+
+double orc_grad_scale(int n_tensors, const float *const *grads, const int64_t *sizes, double max_norm)
+{
+    double q = 0.0;
+    for (int k = 0; k < n_tensors; ++k)
+        for (int64_t i = 0; i < sizes[k]; ++i) q += (double)grads[k][i] * (double)grads[k][i];
+    const double s = max_norm / (sqrt(q) + 1e-6);
+    return s < 1.0 ? s : 1.0;
+}
+
+double orc_adaptive_lr(double lr, double kl, double kl_target, double lr_min, double lr_max)
+{
+    if (kl > 2.0 * kl_target) { lr = lr / 1.5; return lr > lr_min ? lr : lr_min; }
+    if (kl > 0.0 && kl < 0.5 * kl_target) { lr = lr * 1.5; return lr < lr_max ? lr : lr_max; }
+    return lr;
+}
+
 int orc_openmp_enabled(void)
 {
 #ifdef _OPENMP

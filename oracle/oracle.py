@@ -88,6 +88,11 @@ def lib():
         L.orc_reset_cdf.restype = i32
         L.orc_ppo_loss.argtypes = [vp, i64, i32] + [vp] * 7 + [f64, f64] + [vp] * 7
         L.orc_moments.argtypes = [vp, i64, vp, vp]
+        L.orc_adam_step.argtypes = [i64, vp, vp, vp, vp, f64, f64, f64, f64, i32, f64]
+        L.orc_grad_scale.argtypes = [i32, vp, vp, f64]
+        L.orc_grad_scale.restype = f64
+        L.orc_adaptive_lr.argtypes = [f64] * 5
+        L.orc_adaptive_lr.restype = f64
         L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
@@ -375,3 +380,24 @@ def ppo_loss(batch: dict, clip: float, value_coef: float, entropy_coef: float, c
                        _p(f["value"]), _p(f["value_old"]), _p(f["returns"]), _p(out["d_mean"]),
                        _p(out["d_log_std"]), _p(out["d_value"]), _p(out["summary"]))
     return out
+
+
+def adam_step(param, grad, m, v, lr: float, t: int, b1: float = 0.9, b2: float = 0.999, eps: float = 1e-8,
+              grad_scale: float = 1.0):
+    """In-place Adam step on contiguous fp32 numpy arrays (param, m, v are updated)."""
+    for a in (param, grad, m, v):
+        assert a.dtype == np.float32 and a.flags.c_contiguous and a.size == param.size
+    lib().orc_adam_step(param.size, _p(param), _p(grad), _p(m), _p(v), float(lr), float(b1), float(b2), float(eps),
+                        int(t), float(grad_scale))
+
+
+def grad_scale(grads, max_norm: float) -> float:
+    """min(1, max_norm / (global L2 norm + 1e-6)) over a list of fp32 arrays."""
+    gs = [np.ascontiguousarray(g, np.float32).ravel() for g in grads]
+    ptrs = (C.c_void_p * len(gs))(*[g.ctypes.data for g in gs])
+    sizes = np.asarray([g.size for g in gs], np.int64)
+    return float(lib().orc_grad_scale(len(gs), C.cast(ptrs, C.c_void_p), _p(sizes), float(max_norm)))
+
+
+def adaptive_lr(lr: float, kl: float, kl_target: float, lr_min: float = 1e-5, lr_max: float = 1e-2) -> float:
+    return float(lib().orc_adaptive_lr(float(lr), float(kl), float(kl_target), float(lr_min), float(lr_max)))

@@ -102,3 +102,60 @@ def test_entropy_coefficient_only_moves_log_std():
     ce = float(np.float32(0.01))                         # the coefficient travels as fp32
     np.testing.assert_allclose(c["d_log_std"] - a["d_log_std"], -ce, rtol=1e-9)
     np.testing.assert_allclose(c["summary"][0] - a["summary"][0], -ce * a["summary"][3], rtol=1e-9)
+
+
+# ---------------------------------------------------------------- optimiser step
+def test_adam_matches_torch_optim_over_several_steps():
+    g = np.random.default_rng(0)
+    n = 5000
+    p0 = g.standard_normal(n).astype(np.float32)
+    grads = [(g.standard_normal(n) * 10.0 ** g.uniform(-4, 1, n)).astype(np.float32) for _ in range(6)]
+    p, m, v = p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    tp = torch.nn.Parameter(torch.tensor(p0, dtype=torch.float64))
+    opt = torch.optim.Adam([tp], lr=5e-4, betas=(0.9, 0.999), eps=1e-8)
+    for t, gr in enumerate(grads, 1):
+        O.adam_step(p, gr, m, v, 5e-4, t)
+        tp.grad = torch.tensor(gr, dtype=torch.float64)
+        opt.step()
+        # the oracle stores its state in fp32 between steps: agreement to fp32 rounding
+        np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-6, atol=1e-7)
+    st = opt.state[tp]
+    np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=1e-5, atol=1e-12)
+    np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=1e-5, atol=1e-20)
+
+
+def test_adam_first_step_moves_by_lr_against_the_gradient_sign():
+    grad = np.array([3.0, -0.5, 1e-3, -40.0], np.float32)
+    p, m, v = np.zeros(4, np.float32), np.zeros(4, np.float32), np.zeros(4, np.float32)
+    O.adam_step(p, grad, m, v, 1e-2, 1)
+    np.testing.assert_allclose(p, -1e-2 * np.sign(grad), rtol=1e-4)       # m_hat / sqrt(v_hat) = sign(g) at t = 1
+    np.testing.assert_allclose(m, 0.1 * grad, rtol=1e-6)
+    np.testing.assert_allclose(v, 0.001 * grad.astype(np.float64) ** 2, rtol=1e-6)
+    q, m2, v2 = np.zeros(4, np.float32), np.zeros(4, np.float32), np.zeros(4, np.float32)
+    O.adam_step(q, grad, m2, v2, 1e-2, 1, grad_scale=0.25)               # scaling g leaves the first step unchanged
+    np.testing.assert_allclose(q, p, rtol=1e-4)
+    np.testing.assert_allclose(m2, 0.25 * m, rtol=1e-6)
+
+
+def test_grad_scale_matches_torch_clip_grad_norm():
+    g = np.random.default_rng(1)
+    grads = [g.standard_normal(s).astype(np.float32) * 0.3 for s in ((40, 7), (7,), (300,))]
+    for max_norm in (1.0, 100.0):
+        params = [torch.nn.Parameter(torch.zeros(x.shape, dtype=torch.float64)) for x in grads]
+        for prm, x in zip(params, grads):
+            prm.grad = torch.tensor(x, dtype=torch.float64)
+        total = torch.nn.utils.clip_grad_norm_(params, max_norm)
+        s = O.grad_scale(grads, max_norm)
+        np.testing.assert_allclose(s, min(1.0, max_norm / (total.item() + 1e-6)), rtol=1e-12)
+        np.testing.assert_allclose(params[0].grad.numpy(), grads[0].astype(np.float64) * s, rtol=1e-9)
+    assert O.grad_scale(grads, 100.0) == 1.0
+
+
+def test_adaptive_learning_rate_rule():
+    kl_t = 0.008                                          # the paper's baseline KL threshold
+    assert O.adaptive_lr(1e-3, 0.02, kl_t) == pytest.approx(1e-3 / 1.5)
+    assert O.adaptive_lr(1e-3, 0.003, kl_t) == pytest.approx(1.5e-3)
+    assert O.adaptive_lr(1e-3, 0.008, kl_t) == 1e-3
+    assert O.adaptive_lr(1e-3, 0.0, kl_t) == 1e-3         # no information: unchanged
+    assert O.adaptive_lr(1.2e-5, 1.0, kl_t) == 1e-5       # clamped below
+    assert O.adaptive_lr(9e-3, 1e-6, kl_t) == 1e-2        # clamped above
