@@ -120,8 +120,9 @@ def test_adam_matches_torch_optim_over_several_steps():
         # the oracle stores its state in fp32 between steps: agreement to fp32 rounding
         np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-6, atol=1e-7)
     st = opt.state[tp]
-    np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=1e-5, atol=1e-12)
-    np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=1e-5, atol=1e-20)
+    # state kept in fp32 between steps: errors of one fp32 rounding of the largest summand
+    np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=1e-5, atol=1e-6 * np.abs(m).max())
+    np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=1e-5, atol=1e-6 * np.abs(v).max())
 
 
 def test_adam_first_step_moves_by_lr_against_the_gradient_sign():
