@@ -387,6 +387,40 @@ im_status im_moments(const float *x, int64_t n, float *out2, void *workspace, vo
 im_status im_ppo_loss(const im_ppo_config *cfg, int64_t M, int32_t A, const im_ppo_batch *batch, float *d_mean,
                       float *d_log_std, float *d_value, float *summary, void *workspace, void *cuda_stream);
 
+/* ---- optimiser step -----------------------------------------------------------
+ * (Adam with bias correction as in the common deep-learning libraries; the learning
+ * rate follows the mean KL against the paper's "KL threshold"; the gradient is
+ * clipped by its global norm.  Learning rate and gradient scale are DEVICE scalars,
+ * so a whole update runs without the host reading anything back.)
+ *   g = grad * grad_scale;   m = beta1 m + (1 - beta1) g;   v = beta2 v + (1 - beta2) g^2
+ *   param -= lr (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)          t = 1, 2, ...
+ * im_adam_step: param, grad, m, v DEVICE float [n] (param, m, v updated in place);
+ *   lr DEVICE float [1]; grad_scale DEVICE float [1] or NULL (1).  bf16_out, if not NULL,
+ *   receives the new parameters rounded to bf16 (nearest even) as a [n / cols][cols] matrix
+ *   with row stride ld_bf16 elements -- e.g. a layer's padded weight matrix from
+ *   im_policy_layer_buffers, so the next forward uses the updated weights.
+ * im_grad_scale: scale_out DEVICE float [2] <- (min(1, max_norm / (norm + 1e-6)), norm), norm
+ *   the L2 norm over all n_tensors gradient tensors (HOST arrays of DEVICE pointers and
+ *   sizes, at most 64 tensors); fp64 sums in a fixed order.  workspace as for im_ppo_loss.
+ * im_adaptive_lr: lr <- max(lr / 1.5, lr_min) if kl > 2 kl_target; min(1.5 lr, lr_max) if
+ *   0 < kl < kl_target / 2; unchanged otherwise.  lr, kl DEVICE float [1] (kl is
+ *   summary[4] of im_ppo_loss).
+ * All asynchronous on cuda_stream, no allocation, capturable.
+ * im_policy_layer_buffers: the DEVICE weight matrix of a layer ([dims[l+1]][dims[l]] with
+ *   row stride *ld elements; bf16 on the tensor-core path and for dtype 1, else float) and
+ *   its float bias, for in-place updates by an optimiser running on the policy's stream. */
+typedef struct {
+    float beta1, beta2, eps;
+} im_adam_config;
+
+im_status im_adam_step(const im_adam_config *cfg, int32_t t, int64_t n, float *param, const float *grad, float *m,
+                       float *v, const float *lr, const float *grad_scale, uint16_t *bf16_out, int32_t cols,
+                       int32_t ld_bf16, void *cuda_stream);
+im_status im_grad_scale(int32_t n_tensors, const float *const *grads, const int64_t *sizes, float max_norm,
+                        float *scale_out, void *workspace, void *cuda_stream);
+im_status im_adaptive_lr(float *lr, const float *kl, float kl_target, float lr_min, float lr_max, void *cuda_stream);
+im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t *ld, float **bias);
+
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current

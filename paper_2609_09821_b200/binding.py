@@ -26,6 +26,7 @@ EXPORTS = [
     "im_policy_forward_noalloc", "im_env_attach_policy", "im_policy_forward_staged",
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
     "im_env_step_aos", "im_policy_set_log_std", "im_ppo_workspace_bytes", "im_moments", "im_ppo_loss",
+    "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
 ]
 
 
@@ -65,6 +66,10 @@ class PpoConfig(C.Structure):
 class PpoBatch(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in ("mean", "log_std", "action", "logp_old", "mean_old", "log_std_old",
                                           "advantage", "adv_moments", "value", "value_old", "returns")]
+
+
+class AdamConfig(C.Structure):
+    _fields_ = [("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
 
 
 class PolicyConfig(C.Structure):
@@ -120,6 +125,10 @@ def load():
         L.im_ppo_workspace_bytes.restype = C.c_size_t
         L.im_moments.argtypes = [vp, C.c_int64, vp, vp, vp]
         L.im_ppo_loss.argtypes = [C.POINTER(PpoConfig), C.c_int64, i32, C.POINTER(PpoBatch), vp, vp, vp, vp, vp, vp]
+        L.im_adam_step.argtypes = [C.POINTER(AdamConfig), i32, C.c_int64, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
+        L.im_grad_scale.argtypes = [i32, vp, vp, C.c_float, vp, vp, vp]
+        L.im_adaptive_lr.argtypes = [vp, vp, C.c_float, C.c_float, C.c_float, vp]
+        L.im_policy_layer_buffers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(vp)]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
@@ -343,6 +352,13 @@ class Policy:
             raise ValueError("log_std must be a contiguous [A] tensor")
         _check(load().im_policy_set_log_std(self.h, _ptr(log_std)), "im_policy_set_log_std")
 
+    def layer_buffers(self, layer: int):
+        """(weight pointer, row stride in elements, bias pointer) of a layer on the device."""
+        w, b, ld = C.c_void_p(), C.c_void_p(), C.c_int32()
+        _check(load().im_policy_layer_buffers(self.h, layer, C.byref(w), C.byref(ld), C.byref(b)),
+               "im_policy_layer_buffers")
+        return w.value, int(ld.value), b.value
+
     def value_forward(self, obs, value_out, n: Optional[int] = None):
         """This network read as a critic: writes only its outputs ([n, dims[-1]]), draws no noise."""
         n = obs.shape[0] if n is None else n
@@ -418,6 +434,38 @@ def ppo_loss(batch: dict, d_mean, d_log_std, d_value, summary, workspace, clip: 
     st = stream if stream is not None else torch.cuda.current_stream()
     _check(load().im_ppo_loss(C.byref(cfg), M, A, C.byref(b), _ptr(d_mean), _ptr(d_log_std), _ptr(d_value),
                               _ptr(summary), _ptr(workspace), C.c_void_p(st.cuda_stream)), "im_ppo_loss")
+
+
+def adam_step(param, grad, m, v, lr, t: int, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+              grad_scale=None, bf16_out_ptr: Optional[int] = None, cols: int = 0, ld_bf16: int = 0, stream=None):
+    """Fused Adam step on contiguous CUDA float32 tensors; lr (and grad_scale) are 1-element CUDA tensors."""
+    import torch
+    for a in (param, grad, m, v):
+        if not a.is_contiguous() or a.dtype != torch.float32 or a.numel() != param.numel():
+            raise ValueError("param, grad, m, v must be contiguous float32 tensors of one size")
+    cfg = AdamConfig(np.float32(beta1), np.float32(beta2), np.float32(eps))
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().im_adam_step(C.byref(cfg), int(t), param.numel(), _ptr(param), _ptr(grad), _ptr(m), _ptr(v), _ptr(lr),
+                               _ptr(grad_scale), C.c_void_p(bf16_out_ptr) if bf16_out_ptr else None, int(cols),
+                               int(ld_bf16), C.c_void_p(st.cuda_stream)), "im_adam_step")
+
+
+def grad_scale(grads, max_norm: float, scale_out, workspace, stream=None):
+    """scale_out[0:2] <- (min(1, max_norm / (global L2 norm + 1e-6)), norm) over a list of CUDA float32 tensors."""
+    import torch
+    ptrs = (C.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    sizes = np.asarray([g.numel() for g in grads], np.int64)
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().im_grad_scale(len(grads), C.cast(ptrs, C.c_void_p), _ptr(sizes), C.c_float(max_norm), _ptr(scale_out),
+                                _ptr(workspace), C.c_void_p(st.cuda_stream)), "im_grad_scale")
+
+
+def adaptive_lr(lr, kl, kl_target: float, lr_min: float = 1e-5, lr_max: float = 1e-2, stream=None):
+    """lr (1-element CUDA tensor) follows the mean KL (1-element CUDA tensor or view) against kl_target."""
+    import torch
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().im_adaptive_lr(_ptr(lr), _ptr(kl), C.c_float(kl_target), C.c_float(lr_min), C.c_float(lr_max),
+                                 C.c_void_p(st.cuda_stream)), "im_adaptive_lr")
 
 
 NOALLOC_MAX_BATCH = 1024

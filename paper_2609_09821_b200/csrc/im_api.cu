@@ -404,6 +404,19 @@ void im_destroy_policy(im_policy *p)
     delete p;
 }
 
+im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t *ld, float **bias)
+{
+    if (!p || !W || !ld || !bias || layer < 0 || layer >= p->nl) return IM_ERR_INVALID_ARG;
+    if (p->tensor_path) {
+        tc_policy_layer(p, layer, W, ld, bias);
+    } else {
+        *W = p->d_W[layer];
+        *ld = p->cfg.dims[layer];
+        *bias = p->d_b[layer];
+    }
+    return IM_OK;
+}
+
 im_status im_policy_set_log_std(im_policy *p, const float *log_std)
 {
     if (!p) return IM_ERR_INVALID_ARG;

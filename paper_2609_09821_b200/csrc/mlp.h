@@ -28,6 +28,7 @@ cudaError_t launch_sample(const float *mean, float *action, float *logp, int n, 
 // Tensor-core path (mlp_tc.cu).
 im_status tc_policy_create(im_policy *p, const void *const *W, const float *const *b);
 void tc_policy_destroy(im_policy *p);
+void tc_policy_layer(im_policy *p, int layer, void **W, int32_t *ld, float **bias);
 void *tc_policy_input(im_policy *p, int32_t *ld);     // bf16 [max_batch][ld] staging buffer of the first layer
 im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out, im_policy *src = nullptr);

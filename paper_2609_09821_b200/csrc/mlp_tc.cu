@@ -1014,6 +1014,14 @@ void tc_policy_destroy(im_policy *p)
     p->tc = nullptr;
 }
 
+void tc_policy_layer(im_policy *p, int layer, void **W, int32_t *ld, float **bias)
+{
+    TcLayer &L = p->tc->layers[layer];
+    *W = L.d_W;
+    *ld = L.Kpad;
+    *bias = L.d_bias;
+}
+
 void *tc_policy_input(im_policy *p, int32_t *ld)
 {
     *ld = p->tc->ld_in;

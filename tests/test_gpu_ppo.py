@@ -149,3 +149,82 @@ def test_ppo_loss_rejects_bad_arguments():
         B.ppo_loss(b, *outs, ws, 0.2, 1.0, 0.0, True)                  # value clipping needs the old values
     B.ppo_loss(b, *outs, ws, 0.2, 1.0, 0.0, False)
     torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------- optimiser step
+@pytest.mark.parametrize("n", [1, 37, 4096, 1000003])
+def test_adam_steps_match_oracle(n):
+    g = np.random.default_rng(n)
+    p0 = g.standard_normal(n).astype(np.float32)
+    po, mo, vo = p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    pg, mg, vg = (torch.from_numpy(p0.copy()).cuda(), torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda"))
+    lr = torch.tensor([5e-4], device="cuda")              # the paper's baseline learning rate
+    for t in range(1, 5):
+        grad = (g.standard_normal(n) * 10.0 ** g.uniform(-4, 1, n)).astype(np.float32)
+        scale = 1.0 if t % 2 else 0.37
+        # the coefficients reach the kernel as fp32: the oracle gets the same rounded values
+        O.adam_step(po, grad, mo, vo, float(np.float32(5e-4)), t, b1=float(np.float32(0.9)), b2=float(np.float32(0.999)),
+                    eps=float(np.float32(1e-8)), grad_scale=float(np.float32(scale)))
+        B.adam_step(pg, torch.from_numpy(grad).cuda(), mg, vg, lr, t,
+                    grad_scale=None if t % 2 else torch.tensor([scale], device="cuda"))
+        torch.cuda.synchronize()
+        # one fp32 rounding of each of the few operations: a few ulp of the operands
+        np.testing.assert_allclose(pg.cpu().numpy(), po, rtol=2e-6, atol=2e-9)
+        np.testing.assert_allclose(mg.cpu().numpy(), mo, rtol=1e-5, atol=1e-6 * np.abs(mo).max())
+        np.testing.assert_allclose(vg.cpu().numpy(), vo, rtol=1e-5, atol=1e-6 * np.abs(vo).max())
+        # keep both sides on the same trajectory
+        po, mo, vo = pg.cpu().numpy().copy(), mg.cpu().numpy().copy(), vg.cpu().numpy().copy()
+
+
+def test_grad_scale_and_adaptive_lr_match_oracle():
+    g = np.random.default_rng(2)
+    grads = [g.standard_normal(s).astype(np.float32) * 0.05 for s in (1024 * 577, 1024, 512 * 1024, 69, 1)]
+    ws = B.ppo_workspace()
+    out = torch.empty(2, device="cuda")
+    dev = [torch.from_numpy(x).cuda() for x in grads]
+    for max_norm in (1.0, 1e6):
+        B.grad_scale(dev, max_norm, out, ws)
+        torch.cuda.synchronize()
+        want = O.grad_scale(grads, max_norm)
+        np.testing.assert_allclose(out[0].item(), want, rtol=1e-6)
+        np.testing.assert_allclose(out[1].item(), np.sqrt(sum((x.astype(np.float64) ** 2).sum() for x in grads)), rtol=1e-6)
+    lr = torch.tensor([1e-3], device="cuda")
+    for kl in (0.02, 0.003, 0.008, 0.0, 1.0, 1.0, 1.0):
+        want = O.adaptive_lr(lr.item(), float(np.float32(kl)), 0.008)
+        B.adaptive_lr(lr, torch.tensor([kl], device="cuda"), 0.008)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(lr.item(), want, rtol=1e-6)
+    with pytest.raises(B.ImError):
+        B.grad_scale(dev, -1.0, out, ws)
+
+
+def test_adam_writes_new_weights_into_a_loaded_policy():
+    """The bf16 copy of an Adam step lands in a tensor-core policy's padded weight matrix: the next
+    forward equals a policy loaded with the updated weights."""
+    dims = (361, 128, 28)
+    n = 300
+    pw = W.make_policy_weights(dims, "bf16", 4)
+    pol = B.Policy(dims, pw["W_bf16"], pw["b"], "bf16", 0.1, 0, n)
+    g = np.random.default_rng(6)
+    lr = torch.tensor([1e-2], device="cuda")
+    new_W = []
+    for l in range(2):
+        w_ptr, ld, b_ptr = pol.layer_buffers(l)
+        assert ld == (dims[l] + 63) // 64 * 64
+        master = torch.from_numpy(pw["W"][l].copy()).cuda()                       # fp32 master copy
+        grad = torch.from_numpy(g.standard_normal(pw["W"][l].shape).astype(np.float32)).cuda()
+        m, v = torch.zeros_like(master), torch.zeros_like(master)
+        B.adam_step(master, grad, m, v, lr, 1, bf16_out_ptr=w_ptr, cols=dims[l], ld_bf16=ld)
+        new_W.append(master.cpu().numpy())
+    torch.cuda.synchronize()
+    obs = torch.zeros((n, 384), device="cuda")
+    obs[:, :361] = torch.from_numpy(g.standard_normal((n, 361)).astype(np.float32)).cuda()
+    mean, act = torch.empty((n, 28), device="cuda"), torch.empty((n, 28), device="cuda")
+    pol.forward(1, obs, mean, act)
+    ref_bits = [W.round_to_bf16(x)[1] for x in new_W]
+    ref = B.Policy(dims, ref_bits, pw["b"], "bf16", 0.1, 0, n)
+    mean2, act2 = torch.empty_like(mean), torch.empty_like(act)
+    ref.forward(1, obs, mean2, act2)
+    torch.cuda.synchronize()
+    assert torch.equal(mean, mean2) and torch.equal(act, act2)
+    assert np.abs(new_W[0] - pw["W"][0]).max() > 5e-3                              # the step moved the weights
