@@ -421,6 +421,46 @@ im_status im_grad_scale(int32_t n_tensors, const float *const *grads, const int6
 im_status im_adaptive_lr(float *lr, const float *kl, float kl_target, float lr_min, float lr_max, void *cuda_stream);
 im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t *ld, float **bias);
 
+/* ---- backward-pass building blocks ---------------------------------------------
+ * (The GEMMs and glue kernels of the update's backward pass; the paper runs this
+ * phase through torch.compile.)  With H_l = relu(H_{l-1} W_l^T + b_l) and dZ_l the
+ * gradient at layer l's pre-activation:  dW_l = dZ_l^T H_{l-1},  db_l = column sums of
+ * dZ_l,  dH_{l-1} = dZ_l W_l,  dZ_{l-1} = dH_{l-1} masked by H_{l-1} > 0.
+ * All matrices DEVICE, row-major bf16 bit patterns (uint16) unless stated; ld* are row
+ * strides in elements.  Everything is asynchronous on cuda_stream and allocates nothing.
+ *
+ * im_gemm_bf16: C[M][N] = act(A[M][K] B[N][K]^T + bias[N]) on the tcgen05 kernels of the
+ *   forward path (fp32 accumulation, output rounded to bf16; relu != 0: act = max(., 0)).
+ *   N and K multiples of 64; lda, ldb, ldc multiples of 8; all pointers 16-byte aligned;
+ *   bias float [N] (pass zeros for none); status DEVICE uint32 [1] receives
+ *   IM_DEV_WAIT_TIMEOUT if a bounded wait inside the kernel runs out.
+ * im_gemm_bf16_f32out: C[M][N] float, dense = A[M][K] B[N][K]^T + bias, N <= 80; B and bias
+ *   must hold ceil(N / 16) * 16 rows / floats (the extra ones zero).
+ * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.
+ * im_relu_mask_bf16: dH[r][c] = H[r][c] > 0 ? dH[r][c] : 0 in place; cols, ld_d, ld_h
+ *   multiples of 8, 16-byte aligned pointers.
+ * im_f32_to_bf16_padded: out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
+ * im_bf16_to_f32: out (float, dense [rows][cols]) = in (bf16, row stride ld_in).
+ * im_colsum_f32 / im_colsum_bf16: out[c] = sum_r x[r][c], float [cols]; rows are summed in
+ *   fp32 within slices of 2048 rows and the slices in order in fp64 (bit-reproducible);
+ *   workspace DEVICE, at least ceil(rows / 2048) * cols * 4 bytes. */
+im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                       int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu, uint32_t *status,
+                       void *cuda_stream);
+im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,
+                              int32_t N, int32_t K, const float *bias, uint32_t *status, void *cuda_stream);
+im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int64_t ld_out,
+                            void *cuda_stream);
+im_status im_relu_mask_bf16(uint16_t *dH, int64_t ld_d, const uint16_t *H, int64_t ld_h, int32_t rows, int32_t cols,
+                            void *cuda_stream);
+im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int32_t ld_out,
+                                void *cuda_stream);
+im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream);
+im_status im_colsum_f32(const float *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream);
+im_status im_colsum_bf16(const uint16_t *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream);
+
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one
  * step's body states HOST -> device, runs im_policy_forward on the current

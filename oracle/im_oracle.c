@@ -997,6 +997,72 @@ double orc_adaptive_lr(double lr, double kl, double kl_target, double lr_min, do
     return lr;
 }
 
+/* ------------------------------------------------------------------------
+ * Backward pass of the MLP h_l = relu(W_l h_{l-1} + b_l) (last layer linear) for a batch: given
+ * g = dL/d(output) per sample, the gradients of L with respect to every W_l and b_l by the chain
+ * rule:  gz_L = g;  dW_l = sum_i gz_l,i h_{l-1,i}^T;  db_l = sum_i gz_l,i;
+ *        gh_{l-1} = W_l^T gz_l;  gz_{l-1} = gh_{l-1} where h_{l-1} > 0, else 0.
+ * With bf16_operands the tensors that enter a matrix product are bf16 values, as on the
+ * tensor-core path: the input and every hidden activation (as in orc_policy_forward), the output
+ * gradient, every gh (rounded when it is formed) and the resulting dW; the bias gradient of the
+ * last layer sums the unrounded g.  Sums are exact (fp64).
+ * dW is a flat array, layer after layer, each [dims[l+1]][dims[l]]; db likewise. */
+void orc_mlp_backward(int n_layers, const int32_t *dims, const float *const *W, const float *const *b, int n,
+                      const double *obs, int64_t ld_obs, const double *g_out, double *dW, double *db,
+                      int bf16_operands)
+{
+    int maxd = 0;
+    int64_t w_total = 0, b_total = 0, act_total = 0;
+    for (int l = 0; l <= n_layers; ++l) { if (dims[l] > maxd) maxd = dims[l]; act_total += dims[l]; }
+    for (int l = 0; l < n_layers; ++l) { w_total += (int64_t)dims[l] * dims[l + 1]; b_total += dims[l + 1]; }
+    memset(dW, 0, sizeof(double) * (size_t)w_total);
+    memset(db, 0, sizeof(double) * (size_t)b_total);
+    double *h = (double *)malloc(sizeof(double) * (size_t)act_total);      /* activations of one sample, all layers */
+    double *gz = (double *)malloc(sizeof(double) * (size_t)maxd), *gh = (double *)malloc(sizeof(double) * (size_t)maxd);
+    for (int i = 0; i < n; ++i) {
+        /* forward, keeping every layer's activation */
+        double *h0 = h;
+        for (int k = 0; k < dims[0]; ++k) h0[k] = bf16_operands ? orc_round_bf16(obs[(int64_t)i * ld_obs + k]) : obs[(int64_t)i * ld_obs + k];
+        double *hin = h0;
+        for (int l = 0; l < n_layers; ++l) {
+            double *hout = hin + dims[l];
+            for (int o = 0; o < dims[l + 1]; ++o) {
+                double acc = (double)b[l][o];
+                for (int k = 0; k < dims[l]; ++k) acc += (double)W[l][(int64_t)o * dims[l] + k] * hin[k];
+                if (l < n_layers - 1) { acc = acc > 0.0 ? acc : 0.0; if (bf16_operands) acc = orc_round_bf16(acc); }
+                hout[o] = acc;
+            }
+            hin = hout;
+        }
+        /* backward */
+        const int A = dims[n_layers];
+        for (int o = 0; o < A; ++o) gz[o] = g_out[(int64_t)i * A + o];
+        int64_t w_off = w_total, b_off = b_total;
+        double *hl = h + act_total - A;                                       /* output layer's slot */
+        for (int l = n_layers - 1; l >= 0; --l) {
+            const int N = dims[l + 1], K = dims[l];
+            double *hprev = hl - K;
+            w_off -= (int64_t)N * K; b_off -= N;
+            for (int o = 0; o < N; ++o) db[b_off + o] += gz[o];                /* before operand rounding */
+            if (bf16_operands) for (int o = 0; o < N; ++o) gz[o] = orc_round_bf16(gz[o]);
+            for (int o = 0; o < N; ++o)
+                for (int k = 0; k < K; ++k) dW[w_off + (int64_t)o * K + k] += gz[o] * hprev[k];
+            if (l > 0) {
+                for (int k = 0; k < K; ++k) {
+                    double acc = 0.0;
+                    for (int o = 0; o < N; ++o) acc += (double)W[l][(int64_t)o * K + k] * gz[o];
+                    if (bf16_operands) acc = orc_round_bf16(acc);
+                    gh[k] = hprev[k] > 0.0 ? acc : 0.0;
+                }
+                for (int k = 0; k < K; ++k) gz[k] = gh[k];
+            }
+            hl = hprev;
+        }
+    }
+    if (bf16_operands) for (int64_t j = 0; j < w_total; ++j) dW[j] = orc_round_bf16(dW[j]);
+    free(h); free(gz); free(gh);
+}
+
 int orc_openmp_enabled(void)
 {
 #ifdef _OPENMP

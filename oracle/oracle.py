@@ -93,6 +93,7 @@ def lib():
         L.orc_grad_scale.restype = f64
         L.orc_adaptive_lr.argtypes = [f64] * 5
         L.orc_adaptive_lr.restype = f64
+        L.orc_mlp_backward.argtypes = [i32, vp, vp, vp, i32, vp, i64, vp, vp, vp, i32]
         L.orc_gae.argtypes = [i32, i32, i64, vp, vp, vp, f64, f64, i32, vp, vp]
         _lib = L
     return _lib
@@ -401,3 +402,27 @@ def grad_scale(grads, max_norm: float) -> float:
 
 def adaptive_lr(lr: float, kl: float, kl_target: float, lr_min: float = 1e-5, lr_max: float = 1e-2) -> float:
     return float(lib().orc_adaptive_lr(float(lr), float(kl), float(kl_target), float(lr_min), float(lr_max)))
+
+
+def mlp_backward(dims, W, b, obs: np.ndarray, g_out: np.ndarray, bf16_operands: bool = False):
+    """Gradients (dW list, db list, fp64) of a loss with dL/d(output) = g_out [n, A] for the MLP on obs [n, >=dims[0]]."""
+    nl = len(dims) - 1
+    obs = _f64(obs)
+    g_out = _f64(g_out)
+    n = obs.shape[0]
+    assert g_out.shape == (n, dims[-1])
+    Wc = [np.ascontiguousarray(w, np.float32) for w in W]
+    bc = [np.ascontiguousarray(x, np.float32) for x in b]
+    Wp = (C.c_void_p * nl)(*[w.ctypes.data for w in Wc])
+    bp = (C.c_void_p * nl)(*[x.ctypes.data for x in bc])
+    d = np.asarray(dims, np.int32)
+    dW = np.zeros(sum(int(dims[l]) * int(dims[l + 1]) for l in range(nl)))
+    db = np.zeros(sum(int(dims[l + 1]) for l in range(nl)))
+    lib().orc_mlp_backward(nl, _p(d), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), n, _p(obs), obs.shape[1],
+                           _p(g_out), _p(dW), _p(db), int(bool(bf16_operands)))
+    outW, outb, wo, bo = [], [], 0, 0
+    for l in range(nl):
+        k, m = int(dims[l]), int(dims[l + 1])
+        outW.append(dW[wo:wo + m * k].reshape(m, k)); wo += m * k
+        outb.append(db[bo:bo + m]); bo += m
+    return outW, outb

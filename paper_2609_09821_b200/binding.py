@@ -27,6 +27,8 @@ EXPORTS = [
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
     "im_env_step_aos", "im_policy_set_log_std", "im_ppo_workspace_bytes", "im_moments", "im_ppo_loss",
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
+    "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
+    "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32",
 ]
 
 
@@ -129,6 +131,15 @@ def load():
         L.im_grad_scale.argtypes = [i32, vp, vp, C.c_float, vp, vp, vp]
         L.im_adaptive_lr.argtypes = [vp, vp, C.c_float, C.c_float, C.c_float, vp]
         L.im_policy_layer_buffers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(vp)]
+        i64 = C.c_int64
+        L.im_gemm_bf16.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i32, vp, vp]
+        L.im_gemm_bf16_f32out.argtypes = [vp, i64, vp, i64, vp, i32, i32, i32, vp, vp, vp]
+        L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
+        L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
+        L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_bf16_to_f32.argtypes = [vp, i64, i32, i32, vp, vp]
+        L.im_colsum_f32.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
+        L.im_colsum_bf16.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
@@ -466,6 +477,55 @@ def adaptive_lr(lr, kl, kl_target: float, lr_min: float = 1e-5, lr_max: float = 
     st = stream if stream is not None else torch.cuda.current_stream()
     _check(load().im_adaptive_lr(_ptr(lr), _ptr(kl), C.c_float(kl_target), C.c_float(lr_min), C.c_float(lr_max),
                                  C.c_void_p(st.cuda_stream)), "im_adaptive_lr")
+
+
+# ---- backward-pass building blocks: 2-D CUDA tensors, bf16 as torch.bfloat16, row stride = stride(0)
+def _st(stream):
+    import torch
+    return C.c_void_p((stream if stream is not None else torch.cuda.current_stream()).cuda_stream)
+
+
+def gemm_bf16(A, B, Cout, bias, relu: bool, status, stream=None):
+    """Cout[M, N] (bf16) = act(A[M, K] @ B[N, K].T + bias)."""
+    M, K = A.shape
+    N = B.shape[0]
+    _check(load().im_gemm_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), Cout.stride(0), M, N, K,
+                               _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16")
+
+
+def gemm_bf16_f32out(A, B, Cout, bias, status, stream=None):
+    """Cout[M, N] (float32, dense, N <= 80) = A[M, K] @ B[:N, K].T + bias; B and bias padded to 16 rows."""
+    M, K = A.shape
+    N = Cout.shape[1]
+    _check(load().im_gemm_bf16_f32out(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), M, N, K, _ptr(bias),
+                                      _ptr(status), _st(stream)), "im_gemm_bf16_f32out")
+
+
+def transpose_bf16(x, out, stream=None):
+    _check(load().im_transpose_bf16(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), out.stride(0), _st(stream)),
+           "im_transpose_bf16")
+
+
+def relu_mask_bf16(dH, H, stream=None):
+    _check(load().im_relu_mask_bf16(_ptr(dH), dH.stride(0), _ptr(H), H.stride(0), dH.shape[0], dH.shape[1], _st(stream)),
+           "im_relu_mask_bf16")
+
+
+def f32_to_bf16_padded(x, out, stream=None):
+    _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), out.stride(0),
+                                        _st(stream)), "im_f32_to_bf16_padded")
+
+
+def bf16_to_f32(x, out, stream=None):
+    """out (dense float32 [rows, cols]) = x (bf16 view [rows, cols])."""
+    _check(load().im_bf16_to_f32(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), _st(stream)), "im_bf16_to_f32")
+
+
+def colsum(x, out, workspace, stream=None):
+    import torch
+    fn = load().im_colsum_bf16 if x.dtype == torch.bfloat16 else load().im_colsum_f32
+    _check(fn(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), _ptr(workspace),
+              workspace.numel() * workspace.element_size(), _st(stream)), "im_colsum")
 
 
 NOALLOC_MAX_BATCH = 1024

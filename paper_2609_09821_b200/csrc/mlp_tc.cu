@@ -12,6 +12,8 @@
 // an mbarrier is bounded: when the limit runs out the kernel raises
 // IM_DEV_WAIT_TIMEOUT in the status word, stops issuing work, and leaves
 // through the common exit that frees its tensor memory.
+#include <cmath>
+#include <cstring>
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -159,6 +161,7 @@ struct GemmParams {
     int n_tiles_n;     // N tiles of BLOCK_N
     int stages;        // depth of the operand ring in shared memory
     const float *bias; // [n_tiles_n * BLOCK_N], zero padded
+    float act_floor;   // hidden-layer epilogue: out = max(acc + bias, act_floor); 0 is ReLU, -inf no activation
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
@@ -343,12 +346,13 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
                 tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
                 tmem_ld_wait();
                 const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
+                const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
                 uint32_t pk[32];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float4 b = __ldg(b4 + i);
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, 0.0f), fmaxf(v[4 * i + 1] + b.y, 0.0f));
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, 0.0f), fmaxf(v[4 * i + 3] + b.w, 0.0f));
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, fl), fmaxf(v[4 * i + 1] + b.y, fl));
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, fl), fmaxf(v[4 * i + 3] + b.w, fl));
                     pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
                     pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
                 }
@@ -560,12 +564,13 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
                 tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
                 tmem_ld_wait();
                 const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
+                const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
                 uint32_t pk[32];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float4 b = __ldg(b4 + i);
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, 0.0f), fmaxf(v[4 * i + 1] + b.y, 0.0f));
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, 0.0f), fmaxf(v[4 * i + 3] + b.w, 0.0f));
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, fl), fmaxf(v[4 * i + 1] + b.y, fl));
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, fl), fmaxf(v[4 * i + 3] + b.w, fl));
                     pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
                     pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
                 }
@@ -1064,12 +1069,75 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         const bool last = l == p->nl - 1;
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
+        gp.act_floor = 0.0f;
         gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
         gp.sigma = cfg.sigma; gp.log_std = p->d_log_std; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
         gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
         if (dispatch_tc(L, gp, last, tc->n_sm, cfg.impl == 2, p->stream) != cudaSuccess) return IM_ERR_CUDA;
     }
     return IM_OK;
+}
+
+
+// C[M][N] = act(A[M][K] B[N][K]^T + bias) on the hidden-layer kernels, operands anywhere in device
+// memory: the three tensor maps are encoded for this call and travel as kernel parameters.
+im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int M, int N, int K,
+                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream)
+{
+    static int n_sm = 0;
+    if (!n_sm) {
+        int dev = 0, cc_major = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    }
+    TcLayer L;
+    L.N = N; L.K = K; L.Kpad = K;
+    L.block_n = pick_block_n(N, false);
+    L.n_tiles_n = N / L.block_n;
+    L.d_W = nullptr; L.d_bias = nullptr;
+    if (!make_map(&L.map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_M) ||
+        !make_map(&L.map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)L.block_n) ||
+        !make_map(&L.map_c, C, (uint64_t)M, (uint64_t)N, (uint64_t)ldc, 32))
+        return IM_ERR_CUDA;
+    if (L.block_n == 256 && !make_map(&L.map_b2, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 128)) return IM_ERR_CUDA;
+    GemmParams gp;
+    std::memset(&gp, 0, sizeof(gp));
+    gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
+    gp.act_floor = relu ? 0.0f : -INFINITY;
+    gp.status = status;
+    return dispatch_tc(L, gp, false, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+
+// mean[M][N] (fp32, dense) = A[M][K] B[N][K]^T + bias on the Gaussian-head kernel without sampling.
+// B must hold ceil(N / 16) * 16 rows (rows beyond N zero), bias as many floats.
+im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, int M, int N, int K, const float *bias,
+                       float *mean_out, uint32_t *status, cudaStream_t stream)
+{
+    static int n_sm = 0;
+    if (!n_sm) {
+        int dev = 0, cc_major = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    }
+    TcLayer L;
+    L.N = N; L.K = K; L.Kpad = K;
+    L.block_n = pick_block_n(N, true);
+    L.n_tiles_n = 1;
+    L.d_W = nullptr; L.d_bias = nullptr;
+    if (!make_map(&L.map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_M) ||
+        !make_map(&L.map_b, B, (uint64_t)L.block_n, (uint64_t)K, (uint64_t)ldb, (uint32_t)L.block_n))
+        return IM_ERR_CUDA;
+    GemmParams gp;
+    std::memset(&gp, 0, sizeof(gp));
+    gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = 1; gp.bias = bias;
+    gp.mean = mean_out; gp.sigma = 1.0f;
+    gp.status = status;
+    return dispatch_tc(L, gp, true, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
 
 }  // namespace im

@@ -1,0 +1,243 @@
+// Building blocks of the backward pass of the policy / critic MLP (the paper's update phase):
+// the generic bf16 GEMM entries on the tcgen05 kernels of the forward path, and the small
+// HBM-bound kernels between them.  With activations H_l = relu(H_{l-1} W_l^T + b_l) and dZ_l the
+// gradient at layer l's pre-activation:
+//
+//   dW_l = dZ_l^T H_{l-1}      as a GEMM over the batch dimension: (dZ_l^T)[N][M] x (H_{l-1}^T)[K][M]^T
+//   db_l = column sums of dZ_l
+//   dH_{l-1} = dZ_l W_l        as a GEMM over N: dZ_l[M][N] x (W_l^T)[K][N]^T
+//   dZ_{l-1} = dH_{l-1} where H_{l-1} > 0, else 0
+//
+// Every GEMM is C[M][N] = A[M][K] B[N][K]^T with both operands contiguous along the contraction,
+// the one form the tensor-core kernels implement; the transposed operands are made by
+// transpose_bf16.  Sums over the batch are two-stage and ordered (bit-reproducible).
+#include <cmath>
+#include <cuda_bf16.h>
+
+#include "im_internal.h"
+#include "mlp.h"
+
+namespace im {
+
+namespace {
+
+// out[c][r] = in[r][c] for a [rows][cols] bf16 matrix, 64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *__restrict__ in, long long ld_in, int rows,
+                                                             int cols, __nv_bfloat16 *__restrict__ out, long long ld_out)
+{
+    __shared__ __nv_bfloat16 tile[64][66];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;          // 64 x 4
+    for (int i = ty; i < 64; i += 4) {
+        const int r = r0 + i, c = c0 + tx;
+        tile[i][tx] = (r < rows && c < cols) ? in[(long long)r * ld_in + c] : __float2bfloat16_rn(0.0f);
+    }
+    __syncthreads();
+    for (int i = ty; i < 64; i += 4) {
+        const int c = c0 + i, r = r0 + tx;
+        if (c < cols && r < rows) out[(long long)c * ld_out + r] = tile[tx][i];
+    }
+}
+
+// dH <- dH where H > 0, else 0 (eight bf16 per thread; ld and cols multiples of 8).
+__global__ void __launch_bounds__(256) relu_mask_kernel(__nv_bfloat16 *__restrict__ dH, const __nv_bfloat16 *__restrict__ H,
+                                                        long long ld_d, long long ld_h, int rows, int cols)
+{
+    const int chunks = cols >> 3;
+    const long long total = (long long)rows * chunks;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks;
+        const int c = (int)(i - r * chunks) << 3;
+        uint4 d = *reinterpret_cast<const uint4 *>(dH + r * ld_d + c);
+        const uint4 h = __ldg(reinterpret_cast<const uint4 *>(H + r * ld_h + c));
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
+        uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            // a bf16 is positive when its sign bit is clear and it is not zero
+            const uint32_t lo = hw[k] & 0xffffu, hi = hw[k] >> 16;
+            const bool plo = lo != 0u && !(lo & 0x8000u), phi = hi != 0u && !(hi & 0x8000u);
+            dw[k] = (plo ? dw[k] & 0x0000ffffu : 0u) | (phi ? dw[k] & 0xffff0000u : 0u);
+        }
+        *reinterpret_cast<uint4 *>(dH + r * ld_d + c) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+    }
+}
+
+// out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
+__global__ void __launch_bounds__(256) to_bf16_padded_kernel(const float *__restrict__ in, long long ld_in, int rows, int cols,
+                                                             __nv_bfloat16 *__restrict__ out, int ld_out)
+{
+    const long long total = (long long)rows * ld_out;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / ld_out;
+        const int c = (int)(i - r * ld_out);
+        out[i] = __float2bfloat16_rn(c < cols ? __ldg(in + r * ld_in + c) : 0.0f);
+    }
+}
+
+// out[r][c] (float, dense [rows][cols]) = in[r][c] (bf16, row stride ld_in).
+__global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *__restrict__ in, long long ld_in, int rows,
+                                                          int cols, float *__restrict__ out)
+{
+    const long long total = (long long)rows * cols;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / cols;
+        const int c = (int)(i - r * cols);
+        out[i] = __bfloat162float(in[r * ld_in + c]);
+    }
+}
+
+// Column sums, stage 1: CTA g adds its slice of rows for 256 columns (fp32, rows in order).
+constexpr int kColsumRowsPerCta = 2048;
+template <typename T>
+__device__ __forceinline__ float ld_as_float(const T *p);
+template <>
+__device__ __forceinline__ float ld_as_float<float>(const float *p) { return __ldg(p); }
+template <>
+__device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict__ x, long long ld, long long rows, int cols,
+                                                             float *__restrict__ partial)
+{
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    const long long r0 = (long long)blockIdx.y * kColsumRowsPerCta;
+    long long r1 = r0 + kColsumRowsPerCta;
+    r1 = r1 < rows ? r1 : rows;
+    if (c >= cols) return;
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+    long long r = r0;
+    for (; r + 4 <= r1; r += 4) {                          // four independent chains, combined in a fixed order
+        s0 += ld_as_float(x + r * ld + c);
+        s1 += ld_as_float(x + (r + 1) * ld + c);
+        s2 += ld_as_float(x + (r + 2) * ld + c);
+        s3 += ld_as_float(x + (r + 3) * ld + c);
+    }
+    for (; r < r1; ++r) s0 += ld_as_float(x + r * ld + c);
+    partial[(long long)blockIdx.y * cols + c] = (s0 + s1) + (s2 + s3);
+}
+
+// Stage 2: the slices in order, in fp64.
+__global__ void __launch_bounds__(256) colsum_finish_kernel(const float *__restrict__ partial, int slices, int cols,
+                                                            float *__restrict__ out)
+{
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (c >= cols) return;
+    double s = 0.0;
+    for (int g = 0; g < slices; ++g) s += (double)partial[(long long)g * cols + c];
+    out[c] = (float)s;
+}
+
+bool al16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+im_status colsum(const T *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace, size_t workspace_bytes,
+                 cudaStream_t st)
+{
+    if (!x || !out || !workspace || rows < 1 || cols < 1 || ld < cols) return IM_ERR_INVALID_ARG;
+    const long long slices = (rows + kColsumRowsPerCta - 1) / kColsumRowsPerCta;
+    if ((size_t)slices * (size_t)cols * sizeof(float) > workspace_bytes || slices > 65535) return IM_ERR_INVALID_ARG;
+    const dim3 grid((cols + 255) / 256, (unsigned)slices);
+    colsum_partial_kernel<T><<<grid, 256, 0, st>>>(x, ld, rows, cols, static_cast<float *>(workspace));
+    colsum_finish_kernel<<<(cols + 255) / 256, 256, 0, st>>>(static_cast<const float *>(workspace), (int)slices, cols, out);
+    g_launches.fetch_add(2, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+}  // namespace
+
+}  // namespace im
+
+extern "C" {
+
+im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                       int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu, uint32_t *status,
+                       void *cuda_stream)
+{
+    using namespace im;
+    if (!A || !B || !C || !bias || !status || M < 1 || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
+    if ((N & 63) || (K & 63) || lda < K || ldb < K || ldc < N || (lda & 7) || (ldb & 7) || (ldc & 7)) return IM_ERR_INVALID_ARG;
+    if (!al16(A) || !al16(B) || !al16(C) || !al16(bias)) return IM_ERR_INVALID_ARG;
+    return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream);
+}
+
+im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,
+                              int32_t N, int32_t K, const float *bias, uint32_t *status, void *cuda_stream)
+{
+    using namespace im;
+    if (!A || !B || !C || !bias || !status || M < 1 || N < 1 || N > 80 || K < 64) return IM_ERR_INVALID_ARG;
+    if ((K & 63) || lda < K || ldb < K || (lda & 7) || (ldb & 7)) return IM_ERR_INVALID_ARG;
+    if (!al16(A) || !al16(B) || !al16(C)) return IM_ERR_INVALID_ARG;
+    return tc_gemm_head(A, lda, B, ldb, M, N, K, bias, C, status, (cudaStream_t)cuda_stream);
+}
+
+im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int64_t ld_out,
+                            void *cuda_stream)
+{
+    using namespace im;
+    if (!in || !out || rows < 1 || cols < 1 || ld_in < cols || ld_out < rows) return IM_ERR_INVALID_ARG;
+    const dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+    if (grid.y > 65535) return IM_ERR_INVALID_ARG;
+    transpose_bf16_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const __nv_bfloat16 *>(in), ld_in, rows,
+                                                                       cols, reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+im_status im_relu_mask_bf16(uint16_t *dH, int64_t ld_d, const uint16_t *H, int64_t ld_h, int32_t rows, int32_t cols,
+                            void *cuda_stream)
+{
+    using namespace im;
+    if (!dH || !H || rows < 1 || cols < 8 || (cols & 7) || (ld_d & 7) || (ld_h & 7) || ld_d < cols || ld_h < cols ||
+        !al16(dH) || !al16(H))
+        return IM_ERR_INVALID_ARG;
+    const long long total = (long long)rows * (cols >> 3);
+    long long g = (total + 255) / 256;
+    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
+    relu_mask_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<__nv_bfloat16 *>(dH),
+                                                                  reinterpret_cast<const __nv_bfloat16 *>(H), ld_d, ld_h, rows, cols);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int32_t ld_out,
+                                void *cuda_stream)
+{
+    using namespace im;
+    if (!in || !out || rows < 1 || cols < 1 || ld_in < cols || ld_out < cols) return IM_ERR_INVALID_ARG;
+    const long long total = (long long)rows * ld_out;
+    long long g = (total + 255) / 256;
+    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
+    to_bf16_padded_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(in, ld_in, rows, cols,
+                                                                       reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream)
+{
+    using namespace im;
+    if (!in || !out || rows < 1 || cols < 1 || ld_in < cols) return IM_ERR_INVALID_ARG;
+    const long long total = (long long)rows * cols;
+    long long g = (total + 255) / 256;
+    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
+    bf16_to_f32_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const __nv_bfloat16 *>(in), ld_in, rows,
+                                                                    cols, out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+im_status im_colsum_f32(const float *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream)
+{
+    return im::colsum<float>(x, ld, rows, cols, out, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+im_status im_colsum_bf16(const uint16_t *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream)
+{
+    return im::colsum<__nv_bfloat16>(reinterpret_cast<const __nv_bfloat16 *>(x), ld, rows, cols, out, workspace,
+                                     workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"

@@ -160,3 +160,41 @@ def test_adaptive_learning_rate_rule():
     assert O.adaptive_lr(1e-3, 0.0, kl_t) == 1e-3         # no information: unchanged
     assert O.adaptive_lr(1.2e-5, 1.0, kl_t) == 1e-5       # clamped below
     assert O.adaptive_lr(9e-3, 1e-6, kl_t) == 1e-2        # clamped above
+
+
+# ---------------------------------------------------------------- backward pass of the MLP
+def test_mlp_backward_matches_torch_autograd():
+    g = np.random.default_rng(3)
+    dims = (23, 40, 32, 7)
+    Ws = [g.standard_normal((o, i)).astype(np.float32) / math.sqrt(i) for i, o in zip(dims[:-1], dims[1:])]
+    bs = [g.standard_normal(o).astype(np.float32) * 0.1 for o in dims[1:]]
+    obs = g.standard_normal((50, 23))
+    g_out = g.standard_normal((50, 7))
+    dW, db = O.mlp_backward(dims, Ws, bs, obs, g_out)
+    tW = [torch.tensor(w, dtype=torch.float64, requires_grad=True) for w in Ws]
+    tb = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in bs]
+    h = torch.tensor(obs)
+    for l in range(3):
+        h = torch.nn.functional.linear(h, tW[l], tb[l])
+        if l < 2:
+            h = torch.relu(h)
+    (h * torch.tensor(g_out)).sum().backward()
+    for l in range(3):
+        np.testing.assert_allclose(dW[l], tW[l].grad.numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(db[l], tb[l].grad.numpy(), rtol=1e-10, atol=1e-12)
+    # bf16 weights and operands move the gradients (masks near zero flip), but not far; dW comes out as bf16 values
+    dWb, dbb = O.mlp_backward(dims, [W.round_to_bf16(w)[0] for w in Ws], bs, obs, g_out, bf16_operands=True)
+    for l in range(3):
+        scale = np.abs(dW[l]).max()
+        assert 1e-6 * scale < np.abs(dWb[l] - dW[l]).max() < 0.2 * scale
+        np.testing.assert_array_equal(dWb[l], W.round_to_bf16(dWb[l].astype(np.float32))[0])
+
+
+def test_mlp_backward_single_linear_layer_closed_form():
+    """One layer, no activation: dW = g^T x, db = column sums of g."""
+    g = np.random.default_rng(4)
+    Wm = g.standard_normal((5, 9)).astype(np.float32)
+    x, go = g.standard_normal((13, 9)), g.standard_normal((13, 5))
+    dW, db = O.mlp_backward((9, 5), [Wm], [np.zeros(5, np.float32)], x, go)
+    np.testing.assert_allclose(dW[0], go.T @ x, rtol=1e-12)
+    np.testing.assert_allclose(db[0], go.sum(0), rtol=1e-12)
