@@ -1,0 +1,133 @@
+"""Training-side sequencing of the C-ABI calls for one MLP (actor or critic): forward that keeps
+every layer's activation, backward pass, optimiser step.  Argument marshalling only -- every
+arithmetic step runs in the CUDA library:
+
+    forward    hidden layers  im_gemm_bf16 (bias + ReLU fused, bf16 activations kept per layer)
+               last layer     im_gemm_bf16_f32out (fp32 outputs)
+    backward   dZ_L           im_f32_to_bf16_padded(dL/d output)            db_L  im_colsum_f32
+               per layer      im_transpose_bf16 x 2, im_gemm_bf16 -> dW (bf16), im_bf16_to_f32
+                              im_gemm_bf16 with W^T -> dH, im_relu_mask_bf16 -> dZ_{l-1}, im_colsum_bf16 -> db
+    step       im_grad_scale (global norm), im_adam_step per tensor (writes the bf16 weights in place),
+               im_transpose_bf16 refreshes W^T
+
+Shapes are padded to what the tensor-core kernels take: widths to multiples of 64 (zero padding, which
+the arithmetic leaves zero), batch rows M to a multiple of 64.
+"""
+from __future__ import annotations
+
+from typing import List, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def _pad64(x: int) -> int:
+    return (x + 63) // 64 * 64
+
+
+class MlpTrainer:
+    """fp32 master weights + Adam state + bf16 working copies of one MLP, and its buffers for up to max_rows samples."""
+
+    def __init__(self, dims: Sequence[int], W: List[np.ndarray], b: List[np.ndarray], max_rows: int, stream=None):
+        if max_rows % 64:
+            raise ValueError("max_rows must be a multiple of 64")
+        self.dims = tuple(int(d) for d in dims)
+        self.nl = len(dims) - 1
+        self.Mb = int(max_rows)
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        dev, bf, f32 = "cuda", torch.bfloat16, torch.float32
+        self.Kp = [_pad64(d) for d in self.dims[:-1]]
+        self.Np = [_pad64(d) for d in self.dims[1:]]
+        self.W, self.b, self.Wb, self.WbT = [], [], [], []
+        self.mW, self.vW, self.mb, self.vb, self.dW, self.db, self.dWb = [], [], [], [], [], [], []
+        for l in range(self.nl):
+            N, K = self.dims[l + 1], self.dims[l]
+            w = torch.from_numpy(np.ascontiguousarray(W[l], np.float32)).to(dev)
+            self.W.append(w)
+            bias = torch.zeros(self.Np[l], dtype=f32, device=dev)          # padded: the GEMM epilogue reads whole tiles
+            bias[:N] = torch.from_numpy(np.ascontiguousarray(b[l], np.float32)).to(dev)
+            self.b.append(bias)
+            wb = torch.zeros((self.Np[l], self.Kp[l]), dtype=bf, device=dev)
+            wb[:N, :K] = w.to(bf)
+            self.Wb.append(wb)
+            self.WbT.append(torch.zeros((self.Kp[l], self.Np[l]), dtype=bf, device=dev))
+            self.mW.append(torch.zeros_like(w)); self.vW.append(torch.zeros_like(w))
+            self.mb.append(torch.zeros(N, dtype=f32, device=dev)); self.vb.append(torch.zeros(N, dtype=f32, device=dev))
+            self.dW.append(torch.zeros_like(w)); self.db.append(torch.zeros(N, dtype=f32, device=dev))
+            self.dWb.append(torch.zeros((self.Np[l], self.Kp[l]), dtype=bf, device=dev))
+        Mb = self.Mb
+        self.H = [torch.zeros((Mb, self.Kp[0]), dtype=bf, device=dev)]
+        self.H += [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl - 1)]
+        self.out = torch.zeros((Mb, self.dims[-1]), dtype=f32, device=dev)
+        self.dZ = [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl)]
+        self.dZT = torch.zeros((max(self.Np), Mb), dtype=bf, device=dev)
+        self.HT = torch.zeros((max(self.Kp), Mb), dtype=bf, device=dev)
+        self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.colsum_ws = torch.empty(((Mb + 2047) // 2048) * max(self.Np), dtype=f32, device=dev)
+        self.t = 0
+        with torch.cuda.stream(self.stream):
+            for l in range(self.nl):
+                B.transpose_bf16(self.Wb[l], self.WbT[l], self.stream)
+
+    # -- forward ---------------------------------------------------------------
+    def input_rows(self, M: int) -> torch.Tensor:
+        """bf16 view [M, Kp0] the caller fills with the (zero-padded) observations."""
+        return self.H[0][:M]
+
+    def forward(self, M: int) -> torch.Tensor:
+        """Runs the net on input_rows(M); returns the fp32 outputs [M, dims[-1]] (a view)."""
+        if M < 1 or M > self.Mb:
+            raise ValueError("M out of range")
+        st = self.stream
+        for l in range(self.nl - 1):
+            B.gemm_bf16(self.H[l][:M], self.Wb[l], self.H[l + 1][:M], self.b[l], True, self.status, st)
+        L = self.nl - 1
+        B.gemm_bf16_f32out(self.H[L][:M], self.Wb[L], self.out[:M], self.b[L], self.status, st)
+        return self.out[:M]
+
+    # -- backward --------------------------------------------------------------
+    def backward(self, d_out: torch.Tensor, M: int):
+        """d_out: float32 [M, dims[-1]] = dL/d(outputs) of the forward just run on M rows (M % 64 == 0).
+        Fills self.dW[l] (float32 [N, K]) and self.db[l] (float32 [N])."""
+        if M % 64 or M < 64 or M > self.Mb:
+            raise ValueError("M must be a multiple of 64 within the buffers")
+        st = self.stream
+        L = self.nl - 1
+        B.f32_to_bf16_padded(d_out, self.dZ[L][:M], st)
+        B.colsum(d_out, self.db[L], self.colsum_ws, st)
+        for l in range(L, -1, -1):
+            N, K, Np, Kp = self.dims[l + 1], self.dims[l], self.Np[l], self.Kp[l]
+            dZ = self.dZ[l][:M]
+            dZT, HT = self.dZT[:Np, :M], self.HT[:Kp, :M]
+            B.transpose_bf16(dZ, dZT, st)
+            B.transpose_bf16(self.H[l][:M], HT, st)
+            B.gemm_bf16(dZT, HT, self.dWb[l], self.zeros, False, self.status, st)           # dW = dZ^T H
+            B.bf16_to_f32(self.dWb[l][:N, :K], self.dW[l], st)
+            if l > 0:
+                dH = self.dZ[l - 1][:M]                                                       # [M, Kp] = [M, Np of layer l-1]
+                B.gemm_bf16(dZ, self.WbT[l], dH, self.zeros, False, self.status, st)         # dH = dZ W
+                B.relu_mask_bf16(dH, self.H[l][:M], st)
+                B.colsum(dH[:, :K], self.db[l - 1], self.colsum_ws, st)
+
+    # -- optimiser -------------------------------------------------------------
+    def grads(self) -> List[torch.Tensor]:
+        return self.dW + self.db
+
+    def step(self, lr: torch.Tensor, grad_scale: torch.Tensor = None, beta1=0.9, beta2=0.999, eps=1e-8):
+        """Adam step on every tensor; the bf16 working copies (and their transposes) follow."""
+        self.t += 1
+        st = self.stream
+        for l in range(self.nl):
+            K = self.dims[l]
+            B.adam_step(self.W[l], self.dW[l], self.mW[l], self.vW[l], lr, self.t, beta1, beta2, eps, grad_scale,
+                        bf16_out_ptr=self.Wb[l].data_ptr(), cols=K, ld_bf16=self.Kp[l], stream=st)
+            N = self.dims[l + 1]
+            B.adam_step(self.b[l][:N], self.db[l], self.mb[l], self.vb[l], lr, self.t, beta1, beta2, eps, grad_scale,
+                        stream=st)
+            B.transpose_bf16(self.Wb[l], self.WbT[l], st)
+
+    def device_status(self) -> int:
+        return int(self.status.item())

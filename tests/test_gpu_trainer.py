@@ -1,0 +1,129 @@
+"""GPU parity of the training-side path (forward with kept activations, backward pass, Adam step) of
+one MLP against the CPU oracle, through the C ABI.
+
+Tolerance of the gradients: the oracle takes the kernels' operand precision (bf16 activations, output
+gradients and dH, exact sums, dW rounded to bf16); what is left is fp32 accumulation order, the rare
+bf16 rounding flip of a hidden activation (fp32 versus exact accumulation) and what it does to a ReLU
+mask.  Bound used: |g - o| <= 2e-2 (|o| + rms of the tensor), the policy-mean bar of the forward path.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2609_09821_b200 import binding as B
+from paper_2609_09821_b200 import trainer as T
+from paper_2609_09821_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def close(got, want, tol, what):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    lim = tol * (np.abs(want) + np.sqrt(np.mean(want ** 2)))
+    bad = np.abs(got - want) > lim
+    assert not bad.any(), "%s: %d of %d outside %.0e, worst %.3e" % (what, bad.sum(), bad.size, tol,
+                                                                      (np.abs(got - want) / (lim / tol + 1e-300)).max())
+
+
+def test_building_blocks_against_plain_definitions():
+    g = torch.Generator(device="cuda").manual_seed(1)
+    x = torch.randn((300, 200), device="cuda", generator=g).to(torch.bfloat16)
+    out = torch.zeros((200, 304), dtype=torch.bfloat16, device="cuda")
+    B.transpose_bf16(x, out[:, :300])
+    assert torch.equal(out[:, :300], x.t())
+    h = torch.randn((128, 64), device="cuda", generator=g).to(torch.bfloat16)
+    h[0, :4] = torch.tensor([0.0, -0.0, 1e-30, -1e-30], device="cuda").to(torch.bfloat16)
+    d = torch.randn((128, 64), device="cuda", generator=g).to(torch.bfloat16)
+    want = torch.where(h > 0, d, torch.zeros_like(d))
+    B.relu_mask_bf16(d, h)
+    assert torch.equal(d, want)
+    f = torch.randn((70, 69), device="cuda", generator=g)
+    p = torch.full((70, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    B.f32_to_bf16_padded(f, p)
+    assert torch.equal(p[:, :69], f.to(torch.bfloat16)) and (p[:, 69:] == 0).all()
+    back = torch.empty((70, 69), device="cuda")
+    B.bf16_to_f32(p[:, :69], back)
+    assert torch.equal(back, f.to(torch.bfloat16).float())
+    big = torch.randn((5000, 300), device="cuda", generator=g)
+    ws = torch.empty(3 * 300, device="cuda")
+    cs = torch.empty(300, device="cuda")
+    B.colsum(big, cs, ws)
+    np.testing.assert_allclose(cs.cpu().numpy(), big.double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
+    B.colsum(big.to(torch.bfloat16), cs, ws)
+    np.testing.assert_allclose(cs.cpu().numpy(), big.to(torch.bfloat16).double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
+    with pytest.raises(B.ImError):
+        B.colsum(big, cs, ws[:300])                       # workspace too small for three slices
+
+
+@pytest.mark.parametrize("M,N,K,relu", [(200, 64, 64, True), (1000, 256, 192, False), (4096, 1024, 640, True),
+                                         (130, 128, 1024, False)])
+def test_generic_gemm_against_exact_products(M, N, K, relu):
+    """bf16 operands, exact products summed in fp64, bf16 output: the kernel may differ by the fp32
+    accumulation and one bf16 rounding."""
+    g = np.random.default_rng(M + N)
+    a = W.round_to_bf16(g.standard_normal((M, K)).astype(np.float32))[0]
+    b = W.round_to_bf16((g.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32))[0]
+    bias = g.standard_normal(N).astype(np.float32)
+    want = a.astype(np.float64) @ b.astype(np.float64).T + bias
+    if relu:
+        want = np.maximum(want, 0.0)
+    A_, B_ = torch.from_numpy(a).cuda().to(torch.bfloat16), torch.from_numpy(b).cuda().to(torch.bfloat16)
+    C_ = torch.full((M, N), 9.0, dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gemm_bf16(A_, B_, C_, torch.from_numpy(bias).cuda(), relu, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got = C_.float().cpu().numpy()
+    assert np.abs(got - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3
+    close(got, want, 1e-2, "gemm")
+
+
+@pytest.mark.parametrize("dims,M", [((361, 128, 64, 28), 256), ((577, 256, 128, 69), 640), ((361, 64, 1), 128)])
+def test_forward_backward_and_step_match_oracle(dims, M):
+    pw = W.make_policy_weights(dims, "bf16", 11)
+    g = np.random.default_rng(12)
+    obs = g.standard_normal((M, dims[0])).astype(np.float32)
+    d_out = (g.standard_normal((M, dims[-1])) / M).astype(np.float32)
+    tr = T.MlpTrainer(dims, pw["W"], pw["b"], max_rows=M + 64)
+    rows = tr.input_rows(M)
+    rows.zero_()
+    rows[:, :dims[0]] = torch.from_numpy(obs).cuda().to(torch.bfloat16)
+    out = tr.forward(M)
+    want = O.policy_forward(dims, pw["W"], pw["b"], 1.0, 0, 0, obs.astype(np.float64), bf16_operands=True)["mean"]
+    close(out.cpu().numpy(), want, 2e-2, "training forward")
+    tr.backward(torch.from_numpy(d_out).cuda(), M)
+    torch.cuda.synchronize()
+    assert tr.device_status() == 0
+    dW, db = O.mlp_backward(dims, pw["W"], pw["b"], obs.astype(np.float64), d_out.astype(np.float64), bf16_operands=True)
+    for l in range(len(dims) - 1):
+        close(tr.dW[l].cpu().numpy(), dW[l], 2e-2, "dW[%d]" % l)
+        close(tr.db[l].cpu().numpy(), db[l], 2e-2, "db[%d]" % l)
+    # optimiser step from the kernel's own gradients: new fp32 weights, bf16 copies and transposes
+    grads = [x.cpu().numpy().copy() for x in tr.grads()]
+    ws, sc = B.ppo_workspace(), torch.empty(2, device="cuda")
+    B.grad_scale(tr.grads(), 1e-3, sc, ws)
+    lr = torch.tensor([5e-4], device="cuda")
+    W0 = [w.cpu().numpy().copy() for w in tr.W]
+    b0 = [x.cpu().numpy().copy() for x in tr.b]
+    tr.step(lr, sc)
+    torch.cuda.synchronize()
+    scale = O.grad_scale(grads, 1e-3)
+    np.testing.assert_allclose(sc[0].item(), scale, rtol=1e-5)
+    assert scale < 1.0
+    f = lambda x: float(np.float32(x))
+    for l in range(len(dims) - 1):
+        N, K = dims[l + 1], dims[l]
+        w, m, v = W0[l].copy(), np.zeros_like(W0[l]), np.zeros_like(W0[l])
+        O.adam_step(w, grads[l], m, v, f(5e-4), 1, f(0.9), f(0.999), f(1e-8), f(sc[0].item()))
+        np.testing.assert_allclose(tr.W[l].cpu().numpy(), w, rtol=2e-6, atol=2e-9)
+        assert torch.equal(tr.Wb[l][:N, :K], tr.W[l].to(torch.bfloat16))
+        assert torch.equal(tr.WbT[l], tr.Wb[l].t())
+        assert (tr.Wb[l][N:] == 0).all() and (tr.Wb[l][:, K:] == 0).all()
+        bb, m, v = b0[l][:N].copy(), np.zeros(N, np.float32), np.zeros(N, np.float32)
+        O.adam_step(bb, grads[len(dims) - 1 + l], m, v, f(5e-4), 1, f(0.9), f(0.999), f(1e-8), f(sc[0].item()))
+        np.testing.assert_allclose(tr.b[l][:N].cpu().numpy(), bb, rtol=2e-6, atol=2e-9)
+    # the updated net runs: a second forward differs from the first
+    out2 = tr.forward(M).clone()
+    torch.cuda.synchronize()
+    assert not torch.equal(out2, torch.from_numpy(want.astype(np.float32)).cuda())
