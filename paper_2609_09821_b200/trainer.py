@@ -131,3 +131,57 @@ class MlpTrainer:
 
     def device_status(self) -> int:
         return int(self.status.item())
+
+
+class PpoUpdater:
+    """One PPO minibatch update of an actor and a critic (the paper's `update_policy`), every step a
+    library kernel and nothing read back on the host: forward of both nets on the minibatch, loss
+    and output gradients (im_moments + im_ppo_loss), both backward passes, global-norm clip over all
+    gradient tensors, Adam on every tensor, learning rate adapted from the mean KL.
+    """
+
+    def __init__(self, actor: MlpTrainer, critic: MlpTrainer, log_std: torch.Tensor, lr: float, clip: float = 0.2,
+                 value_coef: float = 2.0, entropy_coef: float = 0.0, clip_value_loss: bool = True,
+                 max_grad_norm: float = 1.0, kl_target: float = 0.008, normalize_advantage: bool = True):
+        if actor.stream != critic.stream or critic.dims[-1] != 1 or actor.Mb != critic.Mb:
+            raise ValueError("actor and critic must share the stream and batch size; the critic has one output")
+        self.actor, self.critic, self.stream = actor, critic, actor.stream
+        self.A, self.Mb = actor.dims[-1], actor.Mb
+        dev, f32 = "cuda", torch.float32
+        self.log_std = log_std.detach().clone().to(dev, f32).contiguous()      # learnable parameter [A]
+        self.m_ls, self.v_ls = torch.zeros_like(self.log_std), torch.zeros_like(self.log_std)
+        self.d_log_std = torch.zeros_like(self.log_std)
+        self.lr = torch.tensor([lr], dtype=f32, device=dev)
+        self.scale = torch.zeros(2, dtype=f32, device=dev)
+        self.moments = torch.zeros(2, dtype=f32, device=dev)
+        self.summary = torch.zeros(6, dtype=f32, device=dev)
+        self.d_mean = torch.zeros((self.Mb, self.A), dtype=f32, device=dev)
+        self.d_value = torch.zeros(self.Mb, dtype=f32, device=dev)
+        self.ws = B.ppo_workspace()
+        self.cfg = dict(clip=clip, value_coef=value_coef, entropy_coef=entropy_coef, clip_value_loss=clip_value_loss)
+        self.max_grad_norm, self.kl_target, self.normalize = max_grad_norm, kl_target, normalize_advantage
+        self.t = 0
+
+    def update(self, M: int, batch: dict):
+        """batch: contiguous CUDA float32 tensors action, mean_old [M, A]; log_std_old [A]; logp_old, advantage,
+        value_old, returns [M].  The minibatch observations must already sit (bf16, zero padded) in
+        actor.input_rows(M) and critic.input_rows(M).  M % 64 == 0."""
+        st = self.stream
+        mean = self.actor.forward(M)
+        value = self.critic.forward(M)
+        b = dict(batch, mean=mean, log_std=self.log_std, value=value.view(M))
+        mom = None
+        if self.normalize:
+            B.moments(batch["advantage"], self.moments, self.ws, st)
+            mom = self.moments
+        B.ppo_loss(b, self.d_mean[:M], self.d_log_std, self.d_value[:M], self.summary, self.ws,
+                   self.cfg["clip"], self.cfg["value_coef"], self.cfg["entropy_coef"], self.cfg["clip_value_loss"],
+                   adv_moments=mom, stream=st)
+        self.actor.backward(self.d_mean[:M], M)
+        self.critic.backward(self.d_value[:M].view(M, 1), M)
+        B.grad_scale(self.actor.grads() + self.critic.grads() + [self.d_log_std], self.max_grad_norm, self.scale, self.ws, st)
+        self.actor.step(self.lr, self.scale[:1])
+        self.critic.step(self.lr, self.scale[:1])
+        self.t += 1
+        B.adam_step(self.log_std, self.d_log_std, self.m_ls, self.v_ls, self.lr, self.t, grad_scale=self.scale[:1], stream=st)
+        B.adaptive_lr(self.lr, self.summary[4:5], self.kl_target, stream=st)

@@ -127,3 +127,53 @@ def test_forward_backward_and_step_match_oracle(dims, M):
     out2 = tr.forward(M).clone()
     torch.cuda.synchronize()
     assert not torch.equal(out2, torch.from_numpy(want.astype(np.float32)).cuda())
+
+
+def test_ppo_update_matches_the_oracle_pipeline_and_improves_the_objective():
+    """One whole minibatch update (both nets, loss, clip, Adam, learning rate) against the same
+    pipeline assembled from oracle functions; then a few more updates on the same minibatch must
+    lower the loss (the update does what an optimiser step is for)."""
+    from tests.test_gpu_trainer import close as _close
+    A, D, M = 28, 361, 512
+    adims, cdims = (D, 128, 64, A), (D, 128, 64, 1)
+    aw, cw = W.make_policy_weights(adims, "bf16", 21), W.make_policy_weights(cdims, "bf16", 22)
+    g = np.random.default_rng(23)
+    obs = g.standard_normal((M, D)).astype(np.float32)
+    actor, critic = T.MlpTrainer(adims, aw["W"], aw["b"], M), T.MlpTrainer(cdims, cw["W"], cw["b"], M)
+    log_std0 = np.full(A, -1.0, np.float32)
+    up = T.PpoUpdater(actor, critic, torch.from_numpy(log_std0), lr=5e-4, clip=0.2, value_coef=2.0, entropy_coef=2.5e-4,
+                      max_grad_norm=1.0, kl_target=0.008)
+    for tr in (actor, critic):
+        rows = tr.input_rows(M)
+        rows.zero_()
+        rows[:, :D] = torch.from_numpy(obs).cuda().to(torch.bfloat16)
+    # behaviour data: the current nets' outputs are the "old" policy, actions sampled around them
+    mean_old = O.policy_forward(adims, aw["W"], aw["b"], 1.0, 0, 0, obs.astype(np.float64), bf16_operands=True)["mean"]
+    value_old = O.policy_forward(cdims, cw["W"], cw["b"], 1.0, 0, 0, obs.astype(np.float64), bf16_operands=True)["mean"][:, 0]
+    z = g.standard_normal((M, A))
+    action = (mean_old + np.exp(-1.0) * z).astype(np.float32)
+    logp_old = (-0.5 * (z ** 2).sum(1) - A * (-1.0) - 0.5 * A * np.log(2 * np.pi)).astype(np.float32)
+    batch_np = dict(action=action, mean_old=mean_old.astype(np.float32), log_std_old=log_std0, logp_old=logp_old,
+                    advantage=(g.standard_normal(M) * 2 + 0.5).astype(np.float32), value_old=value_old.astype(np.float32),
+                    returns=(value_old + g.standard_normal(M)).astype(np.float32))
+    batch = {k: torch.from_numpy(v).cuda() for k, v in batch_np.items()}
+    up.update(M, batch)
+    torch.cuda.synchronize()
+    assert actor.device_status() == 0 and critic.device_status() == 0
+    # oracle pipeline on the same inputs
+    am, ar = O.moments(batch_np["advantage"])
+    ob = dict(batch_np, mean=mean_old.astype(np.float32), log_std=log_std0, value=value_old.astype(np.float32))
+    loss = O.ppo_loss(ob, 0.2, 2.0, 2.5e-4, True, am, ar)
+    s = up.summary.cpu().numpy()
+    np.testing.assert_allclose(s[:4], loss["summary"][:4], rtol=2e-2, atol=2e-3)       # bf16 nets: forward differs by ~1e-2
+    dWa, dba = O.mlp_backward(adims, aw["W"], aw["b"], obs.astype(np.float64), loss["d_mean"], bf16_operands=True)
+    for l in range(3):
+        _close(actor.dW[l].cpu().numpy(), dWa[l], 5e-2, "actor dW[%d] through the whole pipeline" % l)
+    assert 0.0 < up.scale[0].item() <= 1.0 and up.scale[1].item() > 0.0
+    assert up.lr.item() == pytest.approx(5e-4 * 1.5, rel=1e-5)          # KL of the first update is ~0: the rate goes up
+    first = float(s[0])
+    for _ in range(8):
+        up.update(M, batch)
+    torch.cuda.synchronize()
+    assert float(up.summary[0].item()) < first
+    assert np.isfinite(up.log_std.cpu().numpy()).all()
