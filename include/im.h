@@ -434,6 +434,11 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   N and K multiples of 64; lda, ldb, ldc multiples of 8; all pointers 16-byte aligned;
  *   bias float [N] (pass zeros for none); status DEVICE uint32 [1] receives
  *   IM_DEV_WAIT_TIMEOUT if a bounded wait inside the kernel runs out.
+ * im_gemm_bf16_batched: `batches` independent products in one launch, stacked along the rows:
+ *   batch b multiplies A[bM .. bM+M) with B[bN .. bN+N) into C[bM .. bM+M); M a multiple of 128
+ *   when batches > 1.  Used to split the long batch-dimension contraction of dW into slices that
+ *   fill the machine; im_sum_slices_bf16_to_f32 then adds the slices (in order, fp32) into a dense
+ *   float matrix: out[r][c] = sum_s in[s * slice_stride + r * ld_in + c].
  * im_gemm_bf16_f32out: C[M][N] float, dense = A[M][K] B[N][K]^T + bias, N <= 80; B and bias
  *   must hold ceil(N / 16) * 16 rows / floats (the extra ones zero).
  * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.
@@ -447,6 +452,11 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
 im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                        int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu, uint32_t *status,
                        void *cuda_stream);
+im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                               int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
+                               uint32_t *status, void *cuda_stream);
+im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
+                                    int32_t cols, float *out, void *cuda_stream);
 im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,
                               int32_t N, int32_t K, const float *bias, uint32_t *status, void *cuda_stream);
 im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int64_t ld_out,

@@ -28,7 +28,7 @@ EXPORTS = [
     "im_env_step_aos", "im_policy_set_log_std", "im_ppo_workspace_bytes", "im_moments", "im_ppo_loss",
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
-    "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32",
+    "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
 ]
 
 
@@ -133,6 +133,8 @@ def load():
         L.im_policy_layer_buffers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(vp)]
         i64 = C.c_int64
         L.im_gemm_bf16.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i32, vp, vp]
+        L.im_gemm_bf16_batched.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp, i32, vp, vp]
+        L.im_sum_slices_bf16_to_f32.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp]
         L.im_gemm_bf16_f32out.argtypes = [vp, i64, vp, i64, vp, i32, i32, i32, vp, vp, vp]
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
@@ -491,6 +493,21 @@ def gemm_bf16(A, B, Cout, bias, relu: bool, status, stream=None):
     N = B.shape[0]
     _check(load().im_gemm_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), Cout.stride(0), M, N, K,
                                _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16")
+
+
+def gemm_bf16_batched(A, B, Cout, batches: int, bias, relu: bool, status, stream=None):
+    """`batches` stacked products: A [batches * M, K], B [batches * N, K] -> Cout [batches * M, N] (bf16)."""
+    M, K = A.shape[0] // batches, A.shape[1]
+    N = B.shape[0] // batches
+    _check(load().im_gemm_bf16_batched(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), Cout.stride(0), batches,
+                                       M, N, K, _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16_batched")
+
+
+def sum_slices_bf16_to_f32(x, slices: int, rows: int, cols: int, out, stream=None):
+    """out (dense float32 [rows, cols]) = sum of the `slices` row blocks of x ([slices * R, ld] bf16, R = x.shape[0] // slices)."""
+    R = x.shape[0] // slices
+    _check(load().im_sum_slices_bf16_to_f32(_ptr(x), R * x.stride(0), x.stride(0), slices, rows, cols, _ptr(out), _st(stream)),
+           "im_sum_slices_bf16_to_f32")
 
 
 def gemm_bf16_f32out(A, B, Cout, bias, status, stream=None):

@@ -162,6 +162,9 @@ struct GemmParams {
     int stages;        // depth of the operand ring in shared memory
     const float *bias; // [n_tiles_n * BLOCK_N], zero padded
     float act_floor;   // hidden-layer epilogue: out = max(acc + bias, act_floor); 0 is ReLU, -inf no activation
+    // Batched products on the single-CTA hidden kernel: batch b multiplies rows [b a_batch_rows, +M) of A
+    // with rows [b b_batch_rows, +N) of B into rows [b a_batch_rows, +M) of C.  n_batches = 1: plain GEMM.
+    int n_batches, a_batch_rows, b_batch_rows;
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
@@ -264,8 +267,10 @@ __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *
 {
     int stage = 0;
     uint32_t phase = 0;
+    const int tiles_per_batch = n_tiles / P.n_batches;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+        const int b = tile / tiles_per_batch, t = tile - b * tiles_per_batch;
+        const int m0 = b * P.a_batch_rows + (t / P.n_tiles_n) * BLOCK_M, n0 = b * P.b_batch_rows + (t % P.n_tiles_n) * BLOCK_N;
         for (int kb = 0; kb < P.K_blocks; ++kb) {
             if (!mbar_wait(&p.empty[stage], phase ^ 1u, p.abort_flag)) return;
             uint8_t *sa = p.tiles + (size_t)stage * Plan::kStageBytes;
@@ -320,7 +325,8 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
     extern __shared__ uint8_t smem_raw[];
     const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::hidden_epi_bytes());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
+    const int tiles_per_batch = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
+    const int n_tiles = tiles_per_batch * P.n_batches;
     pipe_init<Plan>(p, kEpiWarps);
     const uint32_t tmem_base = *p.tmem_slot;
 
@@ -335,7 +341,8 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-            const int m0 = (tile / P.n_tiles_n) * BLOCK_M, n0 = (tile % P.n_tiles_n) * BLOCK_N;
+            const int bt = tile / tiles_per_batch, tt = tile - bt * tiles_per_batch;
+            const int m0 = bt * P.a_batch_rows + (tt / P.n_tiles_n) * BLOCK_M, n0 = (tt % P.n_tiles_n) * BLOCK_N;
             if (!mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
@@ -866,7 +873,7 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
     GemmParams gp = gp_in;
     gp.stages = Plan::stages_for(Plan::hidden_epi_bytes());
     const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
-    const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n;
+    const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
     linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -921,7 +928,7 @@ cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n
         // balance the machine better (measured: 16384 x 1024 x 384 is 8 % faster single, 16384 x 1024 x 2048
         // 7 % faster paired)
         const int pair_tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
-        if (L.block_n == 256 && (force_pairs || (pair_tiles >= n_sm && gp.K_blocks >= 8)))
+        if (L.block_n == 256 && gp.n_batches == 1 && (force_pairs || (pair_tiles >= n_sm && gp.K_blocks >= 8)))
             return launch_hidden_pair(L, gp, n_sm, stream);
         switch (L.block_n) {
         case 256: return launch_hidden<256>(L, gp, n_sm, stream);
@@ -1070,6 +1077,7 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
         gp.act_floor = 0.0f;
+        gp.n_batches = 1; gp.a_batch_rows = 0; gp.b_batch_rows = 0;
         gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
         gp.sigma = cfg.sigma; gp.log_std = p->d_log_std; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
         gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
@@ -1082,7 +1090,7 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
 // C[M][N] = act(A[M][K] B[N][K]^T + bias) on the hidden-layer kernels, operands anywhere in device
 // memory: the three tensor maps are encoded for this call and travel as kernel parameters.
 im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int M, int N, int K,
-                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream)
+                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches)
 {
     static int n_sm = 0;
     if (!n_sm) {
@@ -1097,15 +1105,17 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
     L.block_n = pick_block_n(N, false);
     L.n_tiles_n = N / L.block_n;
     L.d_W = nullptr; L.d_bias = nullptr;
-    if (!make_map(&L.map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_M) ||
-        !make_map(&L.map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)L.block_n) ||
-        !make_map(&L.map_c, C, (uint64_t)M, (uint64_t)N, (uint64_t)ldc, 32))
+    const uint64_t nb = (uint64_t)batches;
+    if (!make_map(&L.map_a, A, nb * (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_M) ||
+        !make_map(&L.map_b, B, nb * (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)L.block_n) ||
+        !make_map(&L.map_c, C, nb * (uint64_t)M, (uint64_t)N, (uint64_t)ldc, 32))
         return IM_ERR_CUDA;
-    if (L.block_n == 256 && !make_map(&L.map_b2, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 128)) return IM_ERR_CUDA;
+    if (L.block_n == 256 && !make_map(&L.map_b2, B, nb * (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 128)) return IM_ERR_CUDA;
     GemmParams gp;
     std::memset(&gp, 0, sizeof(gp));
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
     gp.act_floor = relu ? 0.0f : -INFINITY;
+    gp.n_batches = batches; gp.a_batch_rows = M; gp.b_batch_rows = N;
     gp.status = status;
     return dispatch_tc(L, gp, false, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
@@ -1136,6 +1146,7 @@ im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, i
     std::memset(&gp, 0, sizeof(gp));
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = 1; gp.bias = bias;
     gp.mean = mean_out; gp.sigma = 1.0f;
+    gp.n_batches = 1;
     gp.status = status;
     return dispatch_tc(L, gp, true, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }

@@ -22,20 +22,56 @@ namespace im {
 namespace {
 
 // out[c][r] = in[r][c] for a [rows][cols] bf16 matrix, 64 x 64 tiles through shared memory.
+// VEC: both matrices allow 16-byte accesses (pointers and row strides multiples of 8 elements): a tile is
+// read and written as 8-element chunks, the transposition happens in the 2-byte shared-memory reads
+// (the 8-element chunks of a tile row are XOR-swizzled by the row group, so a column walk spreads over the banks).
+template <bool VEC>
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *__restrict__ in, long long ld_in, int rows,
                                                              int cols, __nv_bfloat16 *__restrict__ out, long long ld_out)
 {
-    __shared__ __nv_bfloat16 tile[64][66];
+    __shared__ __align__(16) __nv_bfloat16 tile[64][72];
     const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;          // 64 x 4
-    for (int i = ty; i < 64; i += 4) {
-        const int r = r0 + i, c = c0 + tx;
-        tile[i][tx] = (r < rows && c < cols) ? in[(long long)r * ld_in + c] : __float2bfloat16_rn(0.0f);
-    }
-    __syncthreads();
-    for (int i = ty; i < 64; i += 4) {
-        const int c = c0 + i, r = r0 + tx;
-        if (c < cols && r < rows) out[(long long)c * ld_out + r] = tile[tx][i];
+    if (VEC) {
+        // 64 rows x 8 chunks of 8 elements: two chunks per thread
+        for (int q = threadIdx.x; q < 512; q += 256) {
+            const int i = q >> 3, ch = (q & 7) << 3;
+            const int r = r0 + i, c = c0 + ch;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (r < rows && c + 8 <= cols) {
+                v = __ldg(reinterpret_cast<const uint4 *>(in + (long long)r * ld_in + c));
+            } else if (r < rows) {
+                __nv_bfloat16 e[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) e[k] = c + k < cols ? in[(long long)r * ld_in + c + k] : __float2bfloat16_rn(0.0f);
+                v = *reinterpret_cast<const uint4 *>(e);
+            }
+            *reinterpret_cast<uint4 *>(&tile[i][ch ^ (((i >> 3) & 7) << 3)]) = v;        // chunk index swizzled by the row group
+        }
+        __syncthreads();
+        for (int q = threadIdx.x; q < 512; q += 256) {
+            const int j = q >> 3, ch = (q & 7) << 3;          // output row c0 + j, elements r0 + ch .. + 7
+            const int c = c0 + j, r = r0 + ch;
+            if (c >= cols || r >= rows) continue;
+            __nv_bfloat16 e[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) e[k] = tile[ch + k][(((j >> 3) ^ (ch >> 3)) << 3) + (j & 7)];
+            if (r + 8 <= rows) {
+                *reinterpret_cast<uint4 *>(out + (long long)c * ld_out + r) = *reinterpret_cast<const uint4 *>(e);
+            } else {
+                for (int k = 0; k < 8 && r + k < rows; ++k) out[(long long)c * ld_out + r + k] = e[k];
+            }
+        }
+    } else {
+        const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;          // 64 x 4
+        for (int i = ty; i < 64; i += 4) {
+            const int r = r0 + i, c = c0 + tx;
+            tile[i][tx] = (r < rows && c < cols) ? in[(long long)r * ld_in + c] : __float2bfloat16_rn(0.0f);
+        }
+        __syncthreads();
+        for (int i = ty; i < 64; i += 4) {
+            const int c = c0 + i, r = r0 + tx;
+            if (c < cols && r < rows) out[(long long)c * ld_out + r] = tile[tx][i];
+        }
     }
 }
 
@@ -84,6 +120,21 @@ __global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *_
         const long long r = i / cols;
         const int c = (int)(i - r * cols);
         out[i] = __bfloat162float(in[r * ld_in + c]);
+    }
+}
+
+// out[r][c] (float, dense [rows][cols]) = sum over s of in[s][r][c] (bf16 slices `slice_stride` elements
+// apart, row stride ld_in), slices added in order.
+__global__ void __launch_bounds__(256) sum_slices_kernel(const __nv_bfloat16 *__restrict__ in, long long slice_stride,
+                                                         long long ld_in, int slices, int rows, int cols, float *__restrict__ out)
+{
+    const long long total = (long long)rows * cols;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / cols;
+        const int c = (int)(i - r * cols);
+        float acc = 0.0f;
+        for (int k = 0; k < slices; ++k) acc += __bfloat162float(in[k * slice_stride + r * ld_in + c]);
+        out[i] = acc;
     }
 }
 
@@ -161,6 +212,33 @@ im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_
     return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream);
 }
 
+im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                               int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
+                               uint32_t *status, void *cuda_stream)
+{
+    using namespace im;
+    if (!A || !B || !C || !bias || !status || batches < 1 || M < 1 || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
+    if ((N & 63) || (K & 63) || lda < K || ldb < K || ldc < N || (lda & 7) || (ldb & 7) || (ldc & 7)) return IM_ERR_INVALID_ARG;
+    if (batches > 1 && (M & 127)) return IM_ERR_INVALID_ARG;          // 128-row tiles must not straddle two batches
+    if ((int64_t)batches * M > 0x7fffffff || (int64_t)batches * N > 0x7fffffff) return IM_ERR_INVALID_ARG;
+    if (!al16(A) || !al16(B) || !al16(C) || !al16(bias)) return IM_ERR_INVALID_ARG;
+    return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream, batches);
+}
+
+im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
+                                    int32_t cols, float *out, void *cuda_stream)
+{
+    using namespace im;
+    if (!in || !out || slices < 1 || rows < 1 || cols < 1 || ld_in < cols) return IM_ERR_INVALID_ARG;
+    const long long total = (long long)rows * cols;
+    long long g = (total + 255) / 256;
+    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
+    sum_slices_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const __nv_bfloat16 *>(in), slice_stride, ld_in,
+                                                                   slices, rows, cols, out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
 im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,
                               int32_t N, int32_t K, const float *bias, uint32_t *status, void *cuda_stream)
 {
@@ -178,8 +256,11 @@ im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int
     if (!in || !out || rows < 1 || cols < 1 || ld_in < cols || ld_out < rows) return IM_ERR_INVALID_ARG;
     const dim3 grid((cols + 63) / 64, (rows + 63) / 64);
     if (grid.y > 65535) return IM_ERR_INVALID_ARG;
-    transpose_bf16_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const __nv_bfloat16 *>(in), ld_in, rows,
-                                                                       cols, reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    const bool vec = al16(in) && al16(out) && (ld_in & 7) == 0 && (ld_out & 7) == 0;
+    const __nv_bfloat16 *pi = reinterpret_cast<const __nv_bfloat16 *>(in);
+    __nv_bfloat16 *po = reinterpret_cast<__nv_bfloat16 *>(out);
+    if (vec) transpose_bf16_kernel<true><<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(pi, ld_in, rows, cols, po, ld_out);
+    else transpose_bf16_kernel<false><<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(pi, ld_in, rows, cols, po, ld_out);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }

@@ -5,7 +5,8 @@ arithmetic step runs in the CUDA library:
     forward    hidden layers  im_gemm_bf16 (bias + ReLU fused, bf16 activations kept per layer)
                last layer     im_gemm_bf16_f32out (fp32 outputs)
     backward   dZ_L           im_f32_to_bf16_padded(dL/d output)            db_L  im_colsum_f32
-               per layer      im_transpose_bf16 x 2, im_gemm_bf16 -> dW (bf16), im_bf16_to_f32
+               per layer      im_transpose_bf16 (per slice), im_gemm_bf16_batched -> partial dW (bf16),
+                              im_sum_slices_bf16_to_f32 -> dW
                               im_gemm_bf16 with W^T -> dH, im_relu_mask_bf16 -> dZ_{l-1}, im_colsum_bf16 -> db
     step       im_grad_scale (global norm), im_adam_step per tensor (writes the bf16 weights in place),
                im_transpose_bf16 refreshes W^T
@@ -41,7 +42,7 @@ class MlpTrainer:
         self.Kp = [_pad64(d) for d in self.dims[:-1]]
         self.Np = [_pad64(d) for d in self.dims[1:]]
         self.W, self.b, self.Wb, self.WbT = [], [], [], []
-        self.mW, self.vW, self.mb, self.vb, self.dW, self.db, self.dWb = [], [], [], [], [], [], []
+        self.mW, self.vW, self.mb, self.vb, self.dW, self.db = [], [], [], [], [], []
         for l in range(self.nl):
             N, K = self.dims[l + 1], self.dims[l]
             w = torch.from_numpy(np.ascontiguousarray(W[l], np.float32)).to(dev)
@@ -56,13 +57,15 @@ class MlpTrainer:
             self.mW.append(torch.zeros_like(w)); self.vW.append(torch.zeros_like(w))
             self.mb.append(torch.zeros(N, dtype=f32, device=dev)); self.vb.append(torch.zeros(N, dtype=f32, device=dev))
             self.dW.append(torch.zeros_like(w)); self.db.append(torch.zeros(N, dtype=f32, device=dev))
-            self.dWb.append(torch.zeros((self.Np[l], self.Kp[l]), dtype=bf, device=dev))
         Mb = self.Mb
         self.H = [torch.zeros((Mb, self.Kp[0]), dtype=bf, device=dev)]
         self.H += [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl - 1)]
         self.out = torch.zeros((Mb, self.dims[-1]), dtype=f32, device=dev)
         self.dZ = [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl)]
-        self.dZT = torch.zeros((max(self.Np), Mb), dtype=bf, device=dev)
+        self.max_split = 16                                                 # most slices of the batch dimension in a dW GEMM
+        np128 = (max(self.Np) + 127) // 128 * 128
+        self.dWs = torch.zeros((self.max_split * np128, max(self.Kp)), dtype=bf, device=dev)
+        self.dZT = torch.zeros((np128, Mb), dtype=bf, device=dev)
         self.HT = torch.zeros((max(self.Kp), Mb), dtype=bf, device=dev)
         self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -101,11 +104,24 @@ class MlpTrainer:
         for l in range(L, -1, -1):
             N, K, Np, Kp = self.dims[l + 1], self.dims[l], self.Np[l], self.Kp[l]
             dZ = self.dZ[l][:M]
-            dZT, HT = self.dZT[:Np, :M], self.HT[:Kp, :M]
-            B.transpose_bf16(dZ, dZT, st)
-            B.transpose_bf16(self.H[l][:M], HT, st)
-            B.gemm_bf16(dZT, HT, self.dWb[l], self.zeros, False, self.status, st)           # dW = dZ^T H
-            B.bf16_to_f32(self.dWb[l][:N, :K], self.dW[l], st)
+            # dW = dZ^T H contracts over the batch rows: a long sum feeding few output tiles.  The rows are
+            # cut into S slices that run as one batched launch (S times the tiles, enough to fill the
+            # machine) and the S partial products are added afterwards.  Slices sit 128-row aligned in
+            # the stacked operand (rows between Np and the pitch are never read back).
+            Npb = (Np + 127) // 128 * 128
+            tiles = (Npb // 128) * max(1, Kp // 256)
+            S = 1
+            while S < self.max_split and tiles * S < 148 and M % (128 * S) == 0:
+                S *= 2
+            Ms = M // S
+            dZT = self.dZT.view(-1)[:S * Npb * Ms].view(S * Npb, Ms)
+            HT = self.HT.view(-1)[:S * Kp * Ms].view(S * Kp, Ms)
+            for s_ in range(S):
+                B.transpose_bf16(dZ[s_ * Ms:(s_ + 1) * Ms], dZT[s_ * Npb:s_ * Npb + Np], st)
+                B.transpose_bf16(self.H[l][s_ * Ms:(s_ + 1) * Ms], HT[s_ * Kp:(s_ + 1) * Kp], st)
+            dWs = self.dWs.view(-1)[:S * Npb * Kp].view(S * Npb, Kp)
+            B.gemm_bf16_batched(dZT, HT, dWs, S, self.zeros, False, self.status, st)
+            B.sum_slices_bf16_to_f32(dWs, S, N, K, self.dW[l], st)
             if l > 0:
                 dH = self.dZ[l - 1][:M]                                                       # [M, Kp] = [M, Np of layer l-1]
                 B.gemm_bf16(dZ, self.WbT[l], dH, self.zeros, False, self.status, st)         # dH = dZ W

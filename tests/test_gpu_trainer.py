@@ -79,7 +79,29 @@ def test_generic_gemm_against_exact_products(M, N, K, relu):
     close(got, want, 1e-2, "gemm")
 
 
-@pytest.mark.parametrize("dims,M", [((361, 128, 64, 28), 256), ((577, 256, 128, 69), 640), ((361, 64, 1), 128)])
+def test_batched_gemm_and_slice_sum():
+    g = np.random.default_rng(5)
+    S, M, N, K = 3, 128, 192, 256
+    a = W.round_to_bf16(g.standard_normal((S * M, K)).astype(np.float32))[0]
+    b = W.round_to_bf16((g.standard_normal((S * N, K)) / 16).astype(np.float32))[0]
+    A_, B_ = torch.from_numpy(a).cuda().to(torch.bfloat16), torch.from_numpy(b).cuda().to(torch.bfloat16)
+    C_ = torch.zeros((S * M, N), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gemm_bf16_batched(A_, B_, C_, S, torch.zeros(N, device="cuda"), False, status)
+    out = torch.empty((100, 150), device="cuda")
+    B.sum_slices_bf16_to_f32(C_, S, 100, 150, out)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    want = np.stack([a[s * M:(s + 1) * M].astype(np.float64) @ b[s * N:(s + 1) * N].astype(np.float64).T for s in range(S)])
+    got = C_.float().cpu().numpy().reshape(S, M, N)
+    assert np.abs(got - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3
+    np.testing.assert_allclose(out.cpu().numpy(), got[:, :100, :150].sum(0), rtol=1e-6, atol=1e-6)
+    with pytest.raises(B.ImError):
+        B.gemm_bf16_batched(A_[:S * 64], B_, C_, S, torch.zeros(N, device="cuda"), False, status)   # 64-row batches
+
+
+@pytest.mark.parametrize("dims,M", [((361, 128, 64, 28), 256), ((577, 256, 128, 69), 640), ((361, 64, 1), 128),
+                                    ((577, 256, 128, 69), 1024)])       # the last one splits every dW product in four
 def test_forward_backward_and_step_match_oracle(dims, M):
     pw = W.make_policy_weights(dims, "bf16", 11)
     g = np.random.default_rng(12)
