@@ -367,6 +367,41 @@ def main():
                                   l2="%.0f MB working set, larger than L2" % (ppo_bytes / 1e6))
         del pb, outs
         if staged:
+            # one whole PPO minibatch update (actor + critic forward, loss, both backward passes, clip, Adam,
+            # learning rate): 2 * n rows, a sixteenth of the rollout, through paper_2609_09821_b200.trainer
+            from paper_2609_09821_b200 import trainer as TR
+            Mu = 2 * n
+            adims, cdims_u = tuple(wl.mlp_dims), tuple(wl.mlp_dims[:-1]) + (1,)
+            cwu = W.make_policy_weights(cdims_u, "bf16", wl.seed + 1)
+            with torch.cuda.stream(stream):
+                actor_t = TR.MlpTrainer(adims, pol["W"], pol["b"], Mu, stream=stream)
+                critic_t = TR.MlpTrainer(cdims_u, cwu["W"], cwu["b"], Mu, stream=stream)
+                upd = TR.PpoUpdater(actor_t, critic_t, torch.full((A,), -2.0), lr=5e-4, clip=0.2, value_coef=2.0)
+                gen = torch.Generator(device=dev).manual_seed(wl.seed)
+                for tr_ in (actor_t, critic_t):
+                    rows_ = tr_.input_rows(Mu)
+                    rows_.zero_()
+                    rows_[:, :D] = torch.randn((Mu, D), device=dev, generator=gen).to(torch.bfloat16)
+                rnd = lambda *sh: torch.randn(*sh, device=dev, generator=gen)
+                ub = dict(action=rnd(Mu, A) * 0.2, mean_old=rnd(Mu, A) * 0.2, log_std_old=torch.full((A,), -2.0, device=dev),
+                          logp_old=rnd(Mu) + 60.0, advantage=rnd(Mu), value_old=rnd(Mu), returns=rnd(Mu))
+                t_up = []
+                for i in range(2 + 5):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    upd.update(Mu, ub)
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    if i >= 2:
+                        t_up.append(a.elapsed_time(b) * 1e-3)
+            t_up = float(np.median(t_up))
+            up_flops = 3 * (mlp_flops_per_env(adims) + mlp_flops_per_env(cdims_u)) * Mu      # forward + two backward products
+            extras["ppo_update"] = dict(rows=Mu, seconds_per_update=t_up, achieved_tflops=up_flops / t_up / 1e12,
+                                        status=[actor_t.device_status(), critic_t.device_status()],
+                                        note="forward + backward + Adam of actor and critic on one minibatch; "
+                                             "flops = 3 x forward flops")
+            del actor_t, critic_t, upd, ub
+        if staged:
             cdims = tuple(wl.mlp_dims[:-1]) + (1,)
             cw = W.make_policy_weights(cdims, "bf16", wl.seed + 1)
             critic = B.Policy(cdims, cw["W_bf16"], cw["b"], "bf16", 1.0, wl.seed, n, stream=stream)
@@ -447,6 +482,8 @@ def main():
     if extras is not None:
         extras["gae"]["frac_of_hbm_peak"] = extras["gae"]["achieved_gbs"] / peaks["hbm_gbs"]
         extras["ppo_loss"]["frac_of_hbm_peak"] = extras["ppo_loss"]["achieved_gbs"] / peaks["hbm_gbs"]
+        if "ppo_update" in extras:
+            extras["ppo_update"]["frac_of_tensor_peak"] = extras["ppo_update"]["achieved_tflops"] / tensor_peak
         if "value_head" in extras:
             extras["value_head"]["frac_of_tensor_peak"] = extras["value_head"]["achieved_tflops"] / tensor_peak
         line["rollout_extras"] = extras
