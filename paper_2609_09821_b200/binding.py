@@ -29,6 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
+    "im_copy_f32",
 ]
 
 
@@ -139,6 +140,7 @@ def load():
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_copy_f32.argtypes = [vp, vp, i64, vp]
         L.im_bf16_to_f32.argtypes = [vp, i64, i32, i32, vp, vp]
         L.im_colsum_f32.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
         L.im_colsum_bf16.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
@@ -531,6 +533,16 @@ def relu_mask_bf16(dH, H, stream=None):
 def f32_to_bf16_padded(x, out, stream=None):
     _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), out.stride(0),
                                         _st(stream)), "im_f32_to_bf16_padded")
+
+
+def f32_to_bf16_padded_ptr(x, out_ptr: int, ld_out: int, stream=None):
+    """Like f32_to_bf16_padded, into a raw device pointer (a policy's weight matrix from Policy.layer_buffers)."""
+    _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], C.c_void_p(out_ptr), int(ld_out),
+                                        _st(stream)), "im_f32_to_bf16_padded")
+
+
+def copy_f32_ptr(dst_ptr: int, src, stream=None):
+    _check(load().im_copy_f32(C.c_void_p(dst_ptr), _ptr(src), src.numel(), _st(stream)), "im_copy_f32")
 
 
 def bf16_to_f32(x, out, stream=None):

@@ -295,6 +295,13 @@ im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, in
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
 
+im_status im_copy_f32(float *dst, const float *src, int64_t n, void *cuda_stream)
+{
+    if (!dst || !src || n < 1) return IM_ERR_INVALID_ARG;
+    return cudaMemcpyAsync(dst, src, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream) == cudaSuccess
+               ? IM_OK : IM_ERR_CUDA;
+}
+
 im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream)
 {
     using namespace im;

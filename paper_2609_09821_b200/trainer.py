@@ -145,6 +145,17 @@ class MlpTrainer:
                         stream=st)
             B.transpose_bf16(self.Wb[l], self.WbT[l], st)
 
+    def push_to_policy(self, policy: B.Policy):
+        """Writes the current weights into a loaded tensor-core policy of the same shape (bf16 weight rows
+        with the policy's row stride, fp32 biases), so the next rollout acts with the trained network.
+        Stream-ordered, no host copy; the policy must use this trainer's stream."""
+        if tuple(policy.dims) != self.dims:
+            raise ValueError("policy and trainer differ in shape")
+        for l in range(self.nl):
+            w_ptr, ld, b_ptr = policy.layer_buffers(l)
+            B.f32_to_bf16_padded_ptr(self.W[l], w_ptr, ld, self.stream)
+            B.copy_f32_ptr(b_ptr, self.b[l][:self.dims[l + 1]], self.stream)
+
     def device_status(self) -> int:
         return int(self.status.item())
 
@@ -165,6 +176,7 @@ class PpoUpdater:
         self.A, self.Mb = actor.dims[-1], actor.Mb
         dev, f32 = "cuda", torch.float32
         self.log_std = log_std.detach().clone().to(dev, f32).contiguous()      # learnable parameter [A]
+        self.log_std_old = self.log_std.clone()                                # the behaviour policy's, frozen per rollout
         self.m_ls, self.v_ls = torch.zeros_like(self.log_std), torch.zeros_like(self.log_std)
         self.d_log_std = torch.zeros_like(self.log_std)
         self.lr = torch.tensor([lr], dtype=f32, device=dev)
@@ -201,3 +213,30 @@ class PpoUpdater:
         self.t += 1
         B.adam_step(self.log_std, self.d_log_std, self.m_ls, self.v_ls, self.lr, self.t, grad_scale=self.scale[:1], stream=st)
         B.adaptive_lr(self.lr, self.summary[4:5], self.kl_target, stream=st)
+
+
+def update_from_storage(upd: PpoUpdater, storage, epochs: int, n_minibatches: int):
+    """The update phase over one collected rollout: `epochs` passes over `n_minibatches` contiguous blocks
+    of the T * N samples (row t * N + e of the flattened time-major arrays).  Each block's observations
+    are converted into both nets' bf16 input rows by im_f32_to_bf16_padded; everything else is read in
+    place from the storage.  Enqueues only; capturable in a CUDA graph together with the rollout."""
+    T, N, A = storage.T, storage.N, storage.A
+    total = T * N
+    M = total // n_minibatches
+    if total % n_minibatches or M % 64 or M > upd.Mb:
+        raise ValueError("T * N must split into minibatches of a multiple of 64 rows that fit the trainers")
+    if not storage.keep_obs:
+        raise ValueError("the update reads the stored observations")
+    flat = lambda x, *tail: x.view(total, *tail) if tail else x.view(total)
+    obs = storage.obs[:T].view(total, storage.ld_obs)
+    action, mean, logp = flat(storage.action, A), flat(storage.mean, A), flat(storage.logp)
+    adv, ret, val = flat(storage.advantage), flat(storage.returns), storage.value[:T].reshape(total)
+    D = upd.actor.dims[0]
+    st = upd.stream
+    for _ in range(epochs):
+        for k in range(n_minibatches):
+            sl = slice(k * M, (k + 1) * M)
+            for tr in (upd.actor, upd.critic):
+                B.f32_to_bf16_padded(obs[sl, :D], tr.input_rows(M), st)
+            upd.update(M, dict(action=action[sl], mean_old=mean[sl], log_std_old=upd.log_std_old, logp_old=logp[sl],
+                               advantage=adv[sl], value_old=val[sl], returns=ret[sl]))

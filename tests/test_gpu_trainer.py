@@ -199,3 +199,82 @@ def test_ppo_update_matches_the_oracle_pipeline_and_improves_the_objective():
     torch.cuda.synchronize()
     assert float(up.summary[0].item()) < first
     assert np.isfinite(up.log_std.cpu().numpy()).all()
+
+
+def test_whole_training_iteration_runs_from_one_cuda_graph():
+    """Rollout (policy forward, critic, env step into storage), GAE and the PPO update epochs enqueued
+    back to back with no host read in between; the same sequence captured in one CUDA graph and
+    replayed from the same starting state reproduces every number bit for bit."""
+    from paper_2609_09821_b200 import rollout as R
+    wl = W.WORKLOADS["cfg3_16384_lib32"]
+    skel, lib, pol = W.build_scene(wl)
+    n, Tn, A, D = 256, 4, wl.act_dim, wl.obs_dim
+    ld = B.padded_ld(D)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        gs = B.Skeleton(skel["parents"], skel["offsets"], skel["masses"])
+        gc = B.Clips(gs, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+        env = B.Env(gs, gc, B.make_env_config(n, wl.dt, 0, W.REWARD_MULT, W.ROOT_HEIGHT, ld), stream=stream)
+        cdims = tuple(wl.mlp_dims[:-1]) + (1,)
+        cw = W.make_policy_weights(cdims, "bf16", 5)
+        actor_t = T.MlpTrainer(wl.mlp_dims, pol["W"], pol["b"], 256, stream=stream)
+        critic_t = T.MlpTrainer(cdims, cw["W"], cw["b"], 256, stream=stream)
+        upd = T.PpoUpdater(actor_t, critic_t, torch.full((A,), -2.0), lr=5e-4)
+        actor = B.Policy(wl.mlp_dims, pol["W_bf16"], pol["b"], "bf16", 0.1, 0, n, stream=stream)
+        critic = B.Policy(cdims, cw["W_bf16"], cw["b"], "bf16", 1.0, 0, n, stream=stream)
+        actor.set_log_std(upd.log_std)
+        st = R.RolloutStorage(Tn, n, A, ld, keep_obs=True)
+        env.reset_all(st.obs_row(0), 0)
+        c, t, _ = env.get_state()
+        sims = {s: W.synth_sim_state_torch(skel, lib, c.long(), t.double() + wl.dt * s, s, wl) for s in range(1, Tn + 1)}
+        state0 = [x.clone() for x in env.get_state()]
+        obs0 = st.obs_row(0).clone()
+        probe_mean, probe_act = torch.empty((n, A), device="cuda"), torch.empty((n, A), device="cuda")
+        before_mean = torch.empty((n, A), device="cuda")
+        actor.forward(99, st.obs_row(0), before_mean, probe_act)
+
+        def iteration():
+            R.collect(env, actor, critic, st, lambda s: sims[s], 1, 0.99, 0.95)
+            T.update_from_storage(upd, st, epochs=2, n_minibatches=4)
+            actor_t.push_to_policy(actor)                          # the next rollout acts with the trained nets
+            critic_t.push_to_policy(critic)
+            actor.set_log_std(upd.log_std)
+            actor.forward(99, st.obs_row(0), probe_mean, probe_act)
+
+        def snapshot():
+            return [x.clone() for x in (st.advantage, st.returns, st.reward, upd.summary, upd.lr, upd.log_std,
+                                        actor_t.W[0], actor_t.W[-1], critic_t.W[1], actor_t.mW[0], probe_mean)]
+
+        def restore(tr0):
+            env.set_state(*state0)
+            st.obs_row(0).copy_(obs0)
+            for tr, saved in zip((actor_t, critic_t), tr0):
+                for dst, src in zip(tr.W + tr.b + tr.mW + tr.vW + tr.mb + tr.vb + tr.Wb + tr.WbT, saved):
+                    dst.copy_(src)
+                tr.t = 0
+            upd.t = 0
+            upd.lr.fill_(5e-4); upd.log_std.fill_(-2.0); upd.m_ls.zero_(); upd.v_ls.zero_()
+            actor_t.push_to_policy(actor); critic_t.push_to_policy(critic); actor.set_log_std(upd.log_std)
+
+        saved = [[x.clone() for x in tr.W + tr.b + tr.mW + tr.vW + tr.mb + tr.vb + tr.Wb + tr.WbT] for tr in (actor_t, critic_t)]
+        iteration()
+        stream.synchronize()
+        eager = snapshot()
+        assert all(torch.isfinite(x).all() for x in eager)
+        assert not torch.equal(eager[6], saved[0][0])             # the actor's first layer moved
+        assert not torch.equal(eager[10], before_mean)            # and the rollout policy acts differently now
+        # the pushed weights are the trainer's: the policy's means equal the trainer's own forward
+        rows = actor_t.input_rows(n)
+        B.f32_to_bf16_padded(st.obs_row(0)[:, :D], rows, stream)
+        assert torch.equal(actor_t.forward(n), eager[10])
+        restore(saved)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            iteration()
+        restore(saved)                                             # capture itself does not run anything
+        graph.replay()
+        stream.synchronize()
+        for a, b in zip(eager, snapshot()):
+            assert torch.equal(a, b)
+        assert env.device_status() == 0 and actor_t.device_status() == 0 and critic_t.device_status() == 0
