@@ -439,6 +439,11 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   when batches > 1.  Used to split the long batch-dimension contraction of dW into slices that
  *   fill the machine; im_sum_slices_bf16_to_f32 then adds the slices (in order, fp32) into a dense
  *   float matrix: out[r][c] = sum_s in[s * slice_stride + r * ld_in + c].
+ * im_gemm_bf16_tn: the transposed product of two row-major matrices without transposing either:
+ *   C_s[Mo][No] = sum over rows r of slice s of A[r][0..Mo) (x) B[r][0..No), for `slices` equal
+ *   ranges of the R rows (R a multiple of 64 * slices), partial results stacked c_pitch rows apart
+ *   (c_pitch >= Mo, a multiple of 128; rows Mo..c_pitch of a slice are written as zeros).  The
+ *   tensor cores read both operands M/N-major.  No a multiple of 64; zeros: float [No] of zeros.
  * im_gemm_bf16_f32out: C[M][N] float, dense = A[M][K] B[N][K]^T + bias, N <= 80; B and bias
  *   must hold ceil(N / 16) * 16 rows / floats (the extra ones zero).
  * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.
@@ -457,6 +462,9 @@ im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_
 im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                                int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
                                uint32_t *status, void *cuda_stream);
+im_status im_gemm_bf16_tn(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, const float *zeros,
+                          uint32_t *status, void *cuda_stream);
 im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
                                     int32_t cols, float *out, void *cuda_stream);
 im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,

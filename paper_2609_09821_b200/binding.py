@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32",
+    "im_copy_f32", "im_gemm_bf16_tn",
 ]
 
 
@@ -135,6 +135,7 @@ def load():
         i64 = C.c_int64
         L.im_gemm_bf16.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i32, vp, vp]
         L.im_gemm_bf16_batched.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp, i32, vp, vp]
+        L.im_gemm_bf16_tn.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp]
         L.im_sum_slices_bf16_to_f32.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp]
         L.im_gemm_bf16_f32out.argtypes = [vp, i64, vp, i64, vp, i32, i32, i32, vp, vp, vp]
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
@@ -503,6 +504,14 @@ def gemm_bf16_batched(A, B, Cout, batches: int, bias, relu: bool, status, stream
     N = B.shape[0] // batches
     _check(load().im_gemm_bf16_batched(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), Cout.stride(0), batches,
                                        M, N, K, _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16_batched")
+
+
+def gemm_bf16_tn(A, Bm, Cout, slices: int, c_pitch: int, zeros, status, stream=None):
+    """Cout (bf16, [slices * c_pitch, No]): slice s holds A[rows of s].T @ Bm[rows of s]; A [R, Mo], Bm [R, No]."""
+    R, Mo = A.shape
+    No = Bm.shape[1]
+    _check(load().im_gemm_bf16_tn(_ptr(A), A.stride(0), _ptr(Bm), Bm.stride(0), _ptr(Cout), Cout.stride(0), R, Mo, No,
+                                  slices, c_pitch, _ptr(zeros), _ptr(status), _st(stream)), "im_gemm_bf16_tn")
 
 
 def sum_slices_bf16_to_f32(x, slices: int, rows: int, cols: int, out, stream=None):

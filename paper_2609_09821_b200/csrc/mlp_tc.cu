@@ -148,11 +148,27 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr)
     d |= (uint64_t)2 << 61;                                // SWIZZLE_128B
     return d;
 }
+// Operand stored with its M (or N) index contiguous: rows of the shared-memory tile are contraction
+// (K) steps, each row holding 64 consecutive M/N elements (128 bytes, 128B-swizzled).  Eight K rows
+// form a 1024-byte group (stride byte offset); the next block of 64 M/N elements starts
+// `mn_block_bytes` further (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr, uint32_t mn_block_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
+// ... the same with both operands M/N-major (bits 15 and 16).
+__host__ __device__ constexpr uint32_t instr_desc_bf16_mn(int M, int N) { return instr_desc_bf16(M, N) | (1u << 15) | (1u << 16); }
 
 struct GemmParams {
     int M;             // rows in use (envs)
@@ -165,6 +181,7 @@ struct GemmParams {
     // Batched products on the single-CTA hidden kernel: batch b multiplies rows [b a_batch_rows, +M) of A
     // with rows [b b_batch_rows, +N) of B into rows [b a_batch_rows, +M) of C.  n_batches = 1: plain GEMM.
     int n_batches, a_batch_rows, b_batch_rows;
+    int c_batch_rows;  // rows of C between two batches
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
@@ -261,7 +278,7 @@ __device__ __forceinline__ void pipe_exit(const Pipe &p, uint32_t tmem_base, uin
 }
 
 // TMA producer (one thread): A and W tiles of every k-block of every tile of this CTA.
-template <class Plan, int BLOCK_N>
+template <class Plan, int BLOCK_N, bool MN = false>
 __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *map_a, const CUtensorMap *map_b,
                                               const GemmParams &P, int n_tiles)
 {
@@ -270,6 +287,24 @@ __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *
     const int tiles_per_batch = n_tiles / P.n_batches;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int b = tile / tiles_per_batch, t = tile - b * tiles_per_batch;
+        if (MN) {
+            // operands are [contraction rows][M or N columns]: a K block is 64 rows, fetched as boxes of 64 columns;
+            // batch b is the row range starting at b * a_batch_rows of both operands
+            const int mm = (t / P.n_tiles_n) * BLOCK_M, nn = (t % P.n_tiles_n) * BLOCK_N, r0 = b * P.a_batch_rows;
+            for (int kb = 0; kb < P.K_blocks; ++kb) {
+                if (!mbar_wait(&p.empty[stage], phase ^ 1u, p.abort_flag)) return;
+                uint8_t *sa = p.tiles + (size_t)stage * Plan::kStageBytes;
+                mbar_arrive_expect_tx(&p.full[stage], Plan::kABytes + Plan::kBBytes);
+#pragma unroll
+                for (int i = 0; i < BLOCK_M / 64; ++i)
+                    tma_load_2d(sa + i * 8192, map_a, &p.full[stage], mm + 64 * i, r0 + kb * BLOCK_K);
+#pragma unroll
+                for (int i = 0; i < BLOCK_N / 64; ++i)
+                    tma_load_2d(sa + Plan::kABytes + i * 8192, map_b, &p.full[stage], nn + 64 * i, r0 + kb * BLOCK_K);
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
+            continue;
+        }
         const int m0 = b * P.a_batch_rows + (t / P.n_tiles_n) * BLOCK_M, n0 = b * P.b_batch_rows + (t % P.n_tiles_n) * BLOCK_N;
         for (int kb = 0; kb < P.K_blocks; ++kb) {
             if (!mbar_wait(&p.empty[stage], phase ^ 1u, p.abort_flag)) return;
@@ -283,10 +318,10 @@ __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *
 }
 
 // MMA issuer (one thread).
-template <class Plan, int BLOCK_N>
+template <class Plan, int BLOCK_N, bool MN = false>
 __device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, const GemmParams &P, int n_tiles)
 {
-    constexpr uint32_t idesc = instr_desc_bf16(BLOCK_M, BLOCK_N);
+    constexpr uint32_t idesc = MN ? instr_desc_bf16_mn(BLOCK_M, BLOCK_N) : instr_desc_bf16(BLOCK_M, BLOCK_N);
     int stage = 0, acc = 0;
     uint32_t phase = 0, acc_phase = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -297,11 +332,20 @@ __device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, cons
             if (!mbar_wait(&p.full[stage], phase, p.abort_flag)) return;
             tc_fence_after();
             const uint32_t sa = smem_u32(p.tiles + (size_t)stage * Plan::kStageBytes);
-            const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + Plan::kABytes);
+            if (MN) {
+                const uint64_t da = smem_desc_mn_major_sw128(sa, 8192u), db = smem_desc_mn_major_sw128(sa + Plan::kABytes, 8192u);
 #pragma unroll
-            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in 16-byte units
-                umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                    // advancing K by 16 rows = two 1024-byte groups: +128 in 16-byte units
+                    umma_bf16(d_tmem, da + (uint64_t)(128 * k), db + (uint64_t)(128 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                }
+            } else {
+                const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + Plan::kABytes);
+#pragma unroll
+                for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                    // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in 16-byte units
+                    umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                }
             }
             umma_commit(&p.empty[stage]);            // smem stage is free once these MMAs have read it
             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -315,7 +359,7 @@ __device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, cons
 // C = relu(A W^T + b) as bf16.  Each epilogue warp owns 32 rows of the tile: it
 // reads 64 accumulator columns at a time, applies bias and ReLU, packs to bf16
 // into a 128B-swizzled slab in shared memory and hands the slab to a TMA store.
-template <int BLOCK_N>
+template <int BLOCK_N, bool MN = false>
 __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                        const __grid_constant__ CUtensorMap map_b,
                                                                        const __grid_constant__ CUtensorMap map_c,
@@ -331,9 +375,9 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
     const uint32_t tmem_base = *p.tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) producer_role<Plan, BLOCK_N>(p, &map_a, &map_b, P, n_tiles);
+        if (lane == 0) producer_role<Plan, BLOCK_N, MN>(p, &map_a, &map_b, P, n_tiles);
     } else if (warp == 1) {
-        if (lane == 0) mma_role<Plan, BLOCK_N>(p, tmem_base, P, n_tiles);
+        if (lane == 0) mma_role<Plan, BLOCK_N, MN>(p, tmem_base, P, n_tiles);
     } else {
         const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
         uint8_t *slabs = p.epi + (size_t)(warp - 2) * 2 * kEpiSlabBytes;       // two slabs, used alternately
@@ -342,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
             const int bt = tile / tiles_per_batch, tt = tile - bt * tiles_per_batch;
-            const int m0 = bt * P.a_batch_rows + (tt / P.n_tiles_n) * BLOCK_M, n0 = (tt % P.n_tiles_n) * BLOCK_N;
+            const int m0 = bt * P.c_batch_rows + (tt / P.n_tiles_n) * BLOCK_M, n0 = (tt % P.n_tiles_n) * BLOCK_N;
             if (!mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
@@ -881,6 +925,28 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
 }
 
 // 256-wide layers with enough rows to fill the machine run on CTA pairs.
+// The same kernel with both operands stored [contraction rows][M or N columns].
+template <int BLOCK_N>
+cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
+{
+    using Plan = SmemPlan<BLOCK_N>;
+    static bool prepared = false;
+    if (!prepared) {
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        prepared = true;
+    }
+    GemmParams gp = gp_in;
+    gp.stages = Plan::stages_for(Plan::hidden_epi_bytes());
+    const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
+    const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
+    const int grid = tiles < n_sm ? tiles : n_sm;
+    linear_tc_hidden_kernel<BLOCK_N, true><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
 {
     static bool prepared = false;
@@ -1077,7 +1143,7 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         GemmParams gp;
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
         gp.act_floor = 0.0f;
-        gp.n_batches = 1; gp.a_batch_rows = 0; gp.b_batch_rows = 0;
+        gp.n_batches = 1; gp.a_batch_rows = 0; gp.b_batch_rows = 0; gp.c_batch_rows = 0;
         gp.mean = mean_out; gp.action = action_out; gp.logp = logp_out;
         gp.sigma = cfg.sigma; gp.log_std = p->d_log_std; gp.seed_lo = (uint32_t)cfg.seed; gp.seed_hi = (uint32_t)(cfg.seed >> 32);
         gp.step = step; gp.env_id_base = cfg.env_id_base; gp.status = p->d_status;
@@ -1115,11 +1181,50 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
     std::memset(&gp, 0, sizeof(gp));
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
     gp.act_floor = relu ? 0.0f : -INFINITY;
-    gp.n_batches = batches; gp.a_batch_rows = M; gp.b_batch_rows = N;
+    gp.n_batches = batches; gp.a_batch_rows = M; gp.b_batch_rows = N; gp.c_batch_rows = M;
     gp.status = status;
     return dispatch_tc(L, gp, false, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
 
+
+// C_s[Mo][No] = sum over the rows r of slice s of A[r][0..Mo) (x) B[r][0..No)  (bf16, fp32 accumulation):
+// the transposed product A^T B of two row-major matrices over `slices` equal row ranges, the partial
+// results stacked with a pitch of `c_pitch` rows.  Operands are read M/N-major, so no transposed copy
+// of either matrix is needed.
+im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int R, int Mo, int No,
+                     int slices, int c_pitch, const float *bias, uint32_t *status, cudaStream_t stream)
+{
+    static int n_sm = 0;
+    if (!n_sm) {
+        int dev = 0, cc_major = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    }
+    TcLayer L;
+    L.N = No; L.K = R / slices; L.Kpad = L.K;
+    L.block_n = pick_block_n(No, false);
+    L.n_tiles_n = No / L.block_n;
+    L.d_W = nullptr; L.d_bias = nullptr;
+    if (!make_map(&L.map_a, A, (uint64_t)R, (uint64_t)Mo, (uint64_t)lda, 64) ||
+        !make_map(&L.map_b, B, (uint64_t)R, (uint64_t)No, (uint64_t)ldb, 64) ||
+        !make_map(&L.map_c, C, (uint64_t)slices * (uint64_t)c_pitch, (uint64_t)No, (uint64_t)ldc, 32))
+        return IM_ERR_CUDA;
+    GemmParams gp;
+    std::memset(&gp, 0, sizeof(gp));
+    gp.M = Mo; gp.N = No; gp.K_blocks = (R / slices) / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
+    gp.act_floor = -INFINITY;
+    gp.n_batches = slices; gp.a_batch_rows = R / slices; gp.b_batch_rows = 0; gp.c_batch_rows = c_pitch;
+    gp.status = status;
+    cudaError_t e;
+    switch (L.block_n) {
+    case 256: e = launch_hidden_mn<256>(L, gp, n_sm, stream); break;
+    case 128: e = launch_hidden_mn<128>(L, gp, n_sm, stream); break;
+    default: e = launch_hidden_mn<64>(L, gp, n_sm, stream); break;
+    }
+    return e == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
 
 // mean[M][N] (fp32, dense) = A[M][K] B[N][K]^T + bias on the Gaussian-head kernel without sampling.
 // B must hold ceil(N / 16) * 16 rows (rows beyond N zero), bias as many floats.

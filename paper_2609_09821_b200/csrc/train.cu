@@ -225,6 +225,19 @@ im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B
     return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream, batches);
 }
 
+im_status im_gemm_bf16_tn(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
+                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, const float *zeros,
+                          uint32_t *status, void *cuda_stream)
+{
+    using namespace im;
+    if (!A || !B || !C || !zeros || !status || R < 64 || Mo < 1 || No < 64 || slices < 1) return IM_ERR_INVALID_ARG;
+    if ((No & 63) || R % (64 * slices) || lda < Mo || ldb < No || ldc < No || (lda & 7) || (ldb & 7) || (ldc & 7))
+        return IM_ERR_INVALID_ARG;
+    if (c_pitch < Mo || (c_pitch & 127)) return IM_ERR_INVALID_ARG;
+    if (!al16(A) || !al16(B) || !al16(C) || !al16(zeros)) return IM_ERR_INVALID_ARG;
+    return tc_gemm_tn(A, lda, B, ldb, C, ldc, R, Mo, No, slices, c_pitch, zeros, status, (cudaStream_t)cuda_stream);
+}
+
 im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
                                     int32_t cols, float *out, void *cuda_stream)
 {

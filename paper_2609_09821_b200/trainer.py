@@ -5,7 +5,7 @@ arithmetic step runs in the CUDA library:
     forward    hidden layers  im_gemm_bf16 (bias + ReLU fused, bf16 activations kept per layer)
                last layer     im_gemm_bf16_f32out (fp32 outputs)
     backward   dZ_L           im_f32_to_bf16_padded(dL/d output)            db_L  im_colsum_f32
-               per layer      im_transpose_bf16 (per slice), im_gemm_bf16_batched -> partial dW (bf16),
+               per layer      im_gemm_bf16_tn -> partial dW per row slice (bf16, operands read in place),
                               im_sum_slices_bf16_to_f32 -> dW
                               im_gemm_bf16 with W^T -> dH, im_relu_mask_bf16 -> dZ_{l-1}, im_colsum_bf16 -> db
     step       im_grad_scale (global norm), im_adam_step per tensor (writes the bf16 weights in place),
@@ -65,8 +65,6 @@ class MlpTrainer:
         self.max_split = 16                                                 # most slices of the batch dimension in a dW GEMM
         np128 = (max(self.Np) + 127) // 128 * 128
         self.dWs = torch.zeros((self.max_split * np128, max(self.Kp)), dtype=bf, device=dev)
-        self.dZT = torch.zeros((np128, Mb), dtype=bf, device=dev)
-        self.HT = torch.zeros((max(self.Kp), Mb), dtype=bf, device=dev)
         self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.colsum_ws = torch.empty(((Mb + 2047) // 2048) * max(self.Np), dtype=f32, device=dev)
@@ -105,22 +103,16 @@ class MlpTrainer:
             N, K, Np, Kp = self.dims[l + 1], self.dims[l], self.Np[l], self.Kp[l]
             dZ = self.dZ[l][:M]
             # dW = dZ^T H contracts over the batch rows: a long sum feeding few output tiles.  The rows are
-            # cut into S slices that run as one batched launch (S times the tiles, enough to fill the
-            # machine) and the S partial products are added afterwards.  Slices sit 128-row aligned in
-            # the stacked operand (rows between Np and the pitch are never read back).
+            # cut into S slices that run as one launch (S times the tiles, enough to fill the machine)
+            # and the S partial products are added afterwards.  im_gemm_bf16_tn reads dZ and H as they
+            # are (M/N-major tensor-core operands): no transposed copies.
             Npb = (Np + 127) // 128 * 128
             tiles = (Npb // 128) * max(1, Kp // 256)
             S = 1
             while S < self.max_split and tiles * S < 148 and M % (128 * S) == 0:
                 S *= 2
-            Ms = M // S
-            dZT = self.dZT.view(-1)[:S * Npb * Ms].view(S * Npb, Ms)
-            HT = self.HT.view(-1)[:S * Kp * Ms].view(S * Kp, Ms)
-            for s_ in range(S):
-                B.transpose_bf16(dZ[s_ * Ms:(s_ + 1) * Ms], dZT[s_ * Npb:s_ * Npb + Np], st)
-                B.transpose_bf16(self.H[l][s_ * Ms:(s_ + 1) * Ms], HT[s_ * Kp:(s_ + 1) * Kp], st)
             dWs = self.dWs.view(-1)[:S * Npb * Kp].view(S * Npb, Kp)
-            B.gemm_bf16_batched(dZT, HT, dWs, S, self.zeros, False, self.status, st)
+            B.gemm_bf16_tn(dZ, self.H[l][:M], dWs, S, Npb, self.zeros, self.status, st)
             B.sum_slices_bf16_to_f32(dWs, S, N, K, self.dW[l], st)
             if l > 0:
                 dH = self.dZ[l - 1][:M]                                                       # [M, Kp] = [M, Np of layer l-1]

@@ -278,3 +278,27 @@ def test_whole_training_iteration_runs_from_one_cuda_graph():
         for a, b in zip(eager, snapshot()):
             assert torch.equal(a, b)
         assert env.device_status() == 0 and actor_t.device_status() == 0 and critic_t.device_status() == 0
+
+
+@pytest.mark.parametrize("R,Mo,No,slices", [(128, 64, 64, 1), (256, 128, 128, 2), (1024, 200, 256, 4), (512, 69, 512, 2),
+                                             (2048, 1024, 640, 4)])
+def test_transposed_product_reads_both_operands_in_place(R, Mo, No, slices):
+    """A^T B of two row-major bf16 matrices on the tensor cores (operands M/N-major), per row slice."""
+    g = np.random.default_rng(R + Mo)
+    a = W.round_to_bf16(g.standard_normal((R, Mo)).astype(np.float32))[0]
+    b = W.round_to_bf16((g.standard_normal((R, No)) / 8).astype(np.float32))[0]
+    lda = (Mo + 7) // 8 * 8
+    A_ = torch.zeros((R, lda), dtype=torch.bfloat16, device="cuda")
+    A_[:, :Mo] = torch.from_numpy(a).cuda().to(torch.bfloat16)
+    B_ = torch.from_numpy(b).cuda().to(torch.bfloat16)
+    pitch = (Mo + 127) // 128 * 128
+    C_ = torch.full((slices * pitch, No), 5.0, dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gemm_bf16_tn(A_[:, :Mo], B_, C_, slices, pitch, torch.zeros(No, device="cuda"), status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    Rs = R // slices
+    got = C_.float().cpu().numpy().reshape(slices, pitch, No)
+    for s in range(slices):
+        want = a[s * Rs:(s + 1) * Rs].astype(np.float64).T @ b[s * Rs:(s + 1) * Rs].astype(np.float64)
+        assert np.abs(got[s, :Mo] - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3, "slice %d" % s
