@@ -219,7 +219,8 @@ void im_env_destroy(im_env *e)
     cudaFree(e->d_aos_sim);
     if (e->h2d_stream) cudaStreamDestroy(e->h2d_stream);
     if (e->d2h_stream) cudaStreamDestroy(e->d2h_stream);
-    if (e->ev_h2d) cudaEventDestroy(e->ev_h2d);
+    for (int c = 0; c < kHostChunks; ++c)
+        if (e->ev_h2d[c]) cudaEventDestroy(e->ev_h2d[c]);
     if (e->ev_policy) cudaEventDestroy(e->ev_policy);
     delete e;
 }
@@ -277,6 +278,25 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float 
     p.pos = sim->pos; p.quat = sim->quat; p.lin = sim->linvel; p.ang = sim->angvel;
     p.stride = sim->comp_stride;
     p.obs = obs_out; p.reward_out = reward_out; p.flags_out = flags_out; p.terms_out = terms_out;
+    IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+// The env step on envs [first, first + count) only (count a multiple of the kernel's 32-env tile unless
+// it reaches the end): every per-env pointer is advanced, the Philox env ids follow.
+static im_status env_step_range(im_env *e, uint32_t step, const im_body_state *sim, float *obs_out, float *reward_out,
+                                uint8_t *flags_out, int first, int count)
+{
+    EnvKernelParams p;
+    fill_params(e, step, p);
+    p.N = count;
+    p.env_id_base += (uint32_t)first;
+    p.clip_id += first; p.t += first; p.ep_len += first;
+    p.pos = sim->pos + first; p.quat = sim->quat + first; p.lin = sim->linvel + first; p.ang = sim->angvel + first;
+    p.stride = sim->comp_stride;
+    p.obs = obs_out + (size_t)first * e->cfg.ld_obs;
+    if (p.obs_bf16) p.obs_bf16 += (size_t)first * e->cfg.ld_obs;
+    p.reward_out = reward_out + first; p.flags_out = flags_out + first; p.terms_out = nullptr;
     IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
     return IM_OK;
 }
@@ -561,9 +581,10 @@ static im_status ensure_staging(im_env *e, int A)
             return IM_ERR_ALLOC;
         if (cudaStreamCreateWithFlags(&e->h2d_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&e->d2h_stream, cudaStreamNonBlocking) != cudaSuccess ||
-            cudaEventCreateWithFlags(&e->ev_h2d, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&e->ev_policy, cudaEventDisableTiming) != cudaSuccess)
             return IM_ERR_CUDA;
+        for (int c = 0; c < kHostChunks; ++c)
+            if (cudaEventCreateWithFlags(&e->ev_h2d[c], cudaEventDisableTiming) != cudaSuccess) return IM_ERR_CUDA;
     }
     if (A > e->staged_A) {
         cudaFree(e->d_mean); cudaFree(e->d_action);
@@ -597,8 +618,15 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     // The body states are needed by the env step only: their upload runs on a copy stream beside
     // the policy forward, and the actions travel back beside the env step (PCIe is full duplex).
     // The previous call waited for all three streams, so the staging buffers are free.
-    IM_CUDA(cudaMemcpyAsync(e->d_sim, sim_host, 13 * J * n * 4, cudaMemcpyHostToDevice, e->h2d_stream));
-    IM_CUDA(cudaEventRecord(e->ev_h2d, e->h2d_stream));
+    // The upload is cut into env ranges (columns of the [13 J][N] array) so that the env kernel of a range
+    // starts as soon as its columns have arrived and only the last range's kernel is not hidden by the copy.
+    const int chunks = (n >= 4096 && n % (4 * 32) == 0) ? kHostChunks : 1;
+    const size_t nc = n / chunks;
+    for (int c = 0; c < chunks; ++c) {
+        IM_CUDA(cudaMemcpy2DAsync(e->d_sim + c * nc, n * 4, sim_host + c * nc, n * 4, nc * 4, 13 * J, cudaMemcpyHostToDevice,
+                                  e->h2d_stream));
+        IM_CUDA(cudaEventRecord(e->ev_h2d[c], e->h2d_stream));
+    }
     int32_t ld_in = 0;
     if (e->d_obs_bf16 && p->tensor_path && e->d_obs_bf16 == tc_policy_input(p, &ld_in))
         s = im_policy_forward_staged(p, step, (int32_t)n, e->d_mean, e->d_action, nullptr);
@@ -608,10 +636,12 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     IM_CUDA(cudaEventRecord(e->ev_policy, e->stream));
     IM_CUDA(cudaStreamWaitEvent(e->d2h_stream, e->ev_policy, 0));
     IM_CUDA(cudaMemcpyAsync(action_host, e->d_action, n * (size_t)A * 4, cudaMemcpyDeviceToHost, e->d2h_stream));
-    IM_CUDA(cudaStreamWaitEvent(e->stream, e->ev_h2d, 0));
     im_body_state sim = {e->d_sim, e->d_sim + 3 * J * n, e->d_sim + 7 * J * n, e->d_sim + 10 * J * n, (int64_t)n};
-    s = im_env_step(e, step, &sim, e->d_obs, e->d_reward, e->d_flags, nullptr);
-    if (s != IM_OK) return s;
+    for (int c = 0; c < chunks; ++c) {
+        IM_CUDA(cudaStreamWaitEvent(e->stream, e->ev_h2d[c], 0));
+        s = env_step_range(e, step, &sim, e->d_obs, e->d_reward, e->d_flags, (int)(c * nc), (int)nc);
+        if (s != IM_OK) return s;
+    }
     IM_CUDA(cudaMemcpyAsync(reward_host, e->d_reward, n * 4, cudaMemcpyDeviceToHost, e->stream));
     IM_CUDA(cudaMemcpyAsync(flags_host, e->d_flags, n, cudaMemcpyDeviceToHost, e->stream));
     IM_CUDA(cudaStreamSynchronize(e->stream));

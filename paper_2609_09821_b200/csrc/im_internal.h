@@ -86,6 +86,8 @@ struct im_clips {
     int device;
 };
 
+constexpr int kHostChunks = 4;             // env ranges the host-buffer step uploads and launches separately
+
 struct im_env {
     const im_skeleton *skel;
     const im_clips *clips;
@@ -107,7 +109,7 @@ struct im_env {
     uint8_t *d_flags;
     int staged_A;
     cudaStream_t h2d_stream, d2h_stream;   // copies of the host-buffer step run beside the kernels
-    cudaEvent_t ev_h2d, ev_policy;
+    cudaEvent_t ev_h2d[4], ev_policy;      // one upload event per env range of the host-buffer step
 };
 
 // Launchers implemented in the kernel translation units.

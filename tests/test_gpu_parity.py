@@ -264,10 +264,11 @@ def test_bad_simulated_quaternion_sets_status_not_a_fault(scenes):
     assert torch.isfinite(p.obs_g[5]).all()
 
 
-def test_host_buffer_step_matches_device_step(scenes):
+@pytest.mark.parametrize("n", [500, 4224], ids=["one-upload", "four-env-ranges"])
+def test_host_buffer_step_matches_device_step(scenes, n):
+    """From 4096 envs on the upload and the env kernel are split into four env ranges; same results."""
     sc = scenes("cfg2_4096")
-    n = 500
-    p = Pair(sc, n)
+    p = Pair(sc, n, policy_sample=300)
     p.reset_all()
     env2 = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, sc.wl.dt, sc.wl.seed, W.REWARD_MULT, sc.wl.h_min, p.ld_obs))
     env2.reset_all_host(0)
