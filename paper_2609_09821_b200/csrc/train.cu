@@ -138,8 +138,9 @@ __global__ void __launch_bounds__(256) sum_slices_kernel(const __nv_bfloat16 *__
     }
 }
 
-// Column sums, stage 1: CTA g adds its slice of rows for 256 columns (fp32, rows in order).
-constexpr int kColsumRowsPerCta = 2048;
+// Column sums, stage 1: a CTA adds a slice of 256 rows for 64 columns; thread (column, row group g of 4)
+// adds rows g, g + 4, ... in two independent chains, the four groups are then added in order.
+constexpr int kColsumRowsPerCta = 256;
 template <typename T>
 __device__ __forceinline__ float ld_as_float(const T *p);
 template <>
@@ -151,21 +152,88 @@ template <typename T>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict__ x, long long ld, long long rows, int cols,
                                                              float *__restrict__ partial)
 {
-    const int c = blockIdx.x * 256 + threadIdx.x;
+    __shared__ float s_part[4][64];
+    const int cx = threadIdx.x & 63, g = threadIdx.x >> 6;
+    const int c = blockIdx.x * 64 + cx;
     const long long r0 = (long long)blockIdx.y * kColsumRowsPerCta;
     long long r1 = r0 + kColsumRowsPerCta;
     r1 = r1 < rows ? r1 : rows;
-    if (c >= cols) return;
-    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
-    long long r = r0;
-    for (; r + 4 <= r1; r += 4) {                          // four independent chains, combined in a fixed order
-        s0 += ld_as_float(x + r * ld + c);
-        s1 += ld_as_float(x + (r + 1) * ld + c);
-        s2 += ld_as_float(x + (r + 2) * ld + c);
-        s3 += ld_as_float(x + (r + 3) * ld + c);
+    float s0 = 0.0f, s1 = 0.0f;
+    if (c < cols) {
+        long long r = r0 + g;
+        for (; r + 4 < r1; r += 8) {
+            s0 += ld_as_float(x + r * ld + c);
+            s1 += ld_as_float(x + (r + 4) * ld + c);
+        }
+        if (r < r1) s0 += ld_as_float(x + r * ld + c);
     }
-    for (; r < r1; ++r) s0 += ld_as_float(x + r * ld + c);
-    partial[(long long)blockIdx.y * cols + c] = (s0 + s1) + (s2 + s3);
+    s_part[g][cx] = s0 + s1;
+    __syncthreads();
+    if (g == 0 && c < cols)
+        partial[(long long)blockIdx.y * cols + c] = ((s_part[0][cx] + s_part[1][cx]) + s_part[2][cx]) + s_part[3][cx];
+}
+
+// The same for matrices that allow 16-byte row accesses: a thread owns 8 (bf16) or 4 (float) adjacent
+// columns and adds every eighth row of the slice; a CTA covers 32 such column groups and 8 row groups.
+template <typename T>
+struct VecOf;
+template <>
+struct VecOf<float> {
+    static constexpr int kN = 4;
+    static __device__ __forceinline__ void load(const float *p, float (&v)[4])
+    {
+        const float4 x = __ldg(reinterpret_cast<const float4 *>(p));
+        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    }
+};
+template <>
+struct VecOf<__nv_bfloat16> {
+    static constexpr int kN = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&v)[8])
+    {
+        const uint4 x = __ldg(reinterpret_cast<const uint4 *>(p));
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = __uint_as_float(w[k] << 16);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+        }
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const T *__restrict__ x, long long ld, long long rows, int cols,
+                                                                 float *__restrict__ partial)
+{
+    constexpr int V = VecOf<T>::kN;
+    __shared__ float s_part[8][32 * V];
+    const int cg = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const int c = (blockIdx.x * 32 + cg) * V;                     // first of this thread's columns
+    const long long r0 = (long long)blockIdx.y * kColsumRowsPerCta;
+    long long r1 = r0 + kColsumRowsPerCta;
+    r1 = r1 < rows ? r1 : rows;
+    float acc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) acc[k] = 0.0f;
+    if (c < cols) {                                               // cols is a multiple of V here
+        for (long long r = r0 + g; r < r1; r += 8) {
+            float v[V];
+            VecOf<T>::load(x + r * ld + c, v);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] += v[k];
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < V; ++k) s_part[g][cg * V + k] = acc[k];
+    __syncthreads();
+    for (int j = threadIdx.x; j < 32 * V; j += 256) {
+        const int cc = blockIdx.x * 32 * V + j;
+        if (cc >= cols) continue;
+        float t = 0.0f;
+#pragma unroll
+        for (int gg = 0; gg < 8; ++gg) t += s_part[gg][j];
+        partial[(long long)blockIdx.y * cols + cc] = t;
+    }
 }
 
 // Stage 2: the slices in order, in fp64.
@@ -188,8 +256,14 @@ im_status colsum(const T *x, int64_t ld, int64_t rows, int32_t cols, float *out,
     if (!x || !out || !workspace || rows < 1 || cols < 1 || ld < cols) return IM_ERR_INVALID_ARG;
     const long long slices = (rows + kColsumRowsPerCta - 1) / kColsumRowsPerCta;
     if ((size_t)slices * (size_t)cols * sizeof(float) > workspace_bytes || slices > 65535) return IM_ERR_INVALID_ARG;
-    const dim3 grid((cols + 255) / 256, (unsigned)slices);
-    colsum_partial_kernel<T><<<grid, 256, 0, st>>>(x, ld, rows, cols, static_cast<float *>(workspace));
+    constexpr int V = VecOf<T>::kN;
+    if (cols % V == 0 && ld % V == 0 && al16(x)) {
+        const dim3 grid((cols + 32 * V - 1) / (32 * V), (unsigned)slices);
+        colsum_partial_vec_kernel<T><<<grid, 256, 0, st>>>(x, ld, rows, cols, static_cast<float *>(workspace));
+    } else {
+        const dim3 grid((cols + 63) / 64, (unsigned)slices);
+        colsum_partial_kernel<T><<<grid, 256, 0, st>>>(x, ld, rows, cols, static_cast<float *>(workspace));
+    }
     colsum_finish_kernel<<<(cols + 255) / 256, 256, 0, st>>>(static_cast<const float *>(workspace), (int)slices, cols, out);
     g_launches.fetch_add(2, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;

@@ -67,7 +67,7 @@ class MlpTrainer:
         self.dWs = torch.zeros((self.max_split * np128, max(self.Kp)), dtype=bf, device=dev)
         self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.colsum_ws = torch.empty(((Mb + 2047) // 2048) * max(self.Np), dtype=f32, device=dev)
+        self.colsum_ws = torch.empty(((Mb + 255) // 256) * max(self.Np), dtype=f32, device=dev)
         self.t = 0
         with torch.cuda.stream(self.stream):
             for l in range(self.nl):

@@ -46,14 +46,14 @@ def test_building_blocks_against_plain_definitions():
     B.bf16_to_f32(p[:, :69], back)
     assert torch.equal(back, f.to(torch.bfloat16).float())
     big = torch.randn((5000, 300), device="cuda", generator=g)
-    ws = torch.empty(3 * 300, device="cuda")
+    ws = torch.empty(20 * 300, device="cuda")
     cs = torch.empty(300, device="cuda")
     B.colsum(big, cs, ws)
     np.testing.assert_allclose(cs.cpu().numpy(), big.double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
     B.colsum(big.to(torch.bfloat16), cs, ws)
     np.testing.assert_allclose(cs.cpu().numpy(), big.to(torch.bfloat16).double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
     with pytest.raises(B.ImError):
-        B.colsum(big, cs, ws[:300])                       # workspace too small for three slices
+        B.colsum(big, cs, ws[:300])                       # workspace too small for twenty slices
 
 
 @pytest.mark.parametrize("M,N,K,relu", [(200, 64, 64, True), (1000, 256, 192, False), (4096, 1024, 640, True),
