@@ -450,6 +450,10 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  * im_relu_mask_bf16: dH[r][c] = H[r][c] > 0 ? dH[r][c] : 0 in place; cols, ld_d, ld_h
  *   multiples of 8, 16-byte aligned pointers.
  * im_f32_to_bf16_padded: out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
+ * im_gather_rows_f32: out[i][0..cols) = in[idx[i]][0..cols) for i < rows (shuffled minibatches); idx
+ *   DEVICE int32 [rows] with values in [0, n_src); out is float [rows][ld_out], or with to_bf16 != 0
+ *   bf16 [rows][ld_out] with columns cols..ld_out written as zeros.  An index out of range is clamped
+ *   and sets IM_DEV_BAD_STATE in *status (DEVICE uint32).
  * im_copy_f32: dst[0..n) = src[0..n), DEVICE to DEVICE on the stream (e.g. a trained bias vector
  *   into the buffer im_policy_layer_buffers returns).
  * im_bf16_to_f32: out (float, dense [rows][cols]) = in (bf16, row stride ld_in).
@@ -475,6 +479,8 @@ im_status im_relu_mask_bf16(uint16_t *dH, int64_t ld_d, const uint16_t *H, int64
                             void *cuda_stream);
 im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int32_t ld_out,
                                 void *cuda_stream);
+im_status im_gather_rows_f32(const float *in, int64_t ld_in, const int32_t *idx, int64_t n_src, int32_t rows, int32_t cols,
+                             void *out, int32_t ld_out, int32_t to_bf16, uint32_t *status, void *cuda_stream);
 im_status im_copy_f32(float *dst, const float *src, int64_t n, void *cuda_stream);
 im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream);
 im_status im_colsum_f32(const float *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,

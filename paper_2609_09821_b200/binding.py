@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32", "im_gemm_bf16_tn",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32",
 ]
 
 
@@ -141,6 +141,7 @@ def load():
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
         L.im_copy_f32.argtypes = [vp, vp, i64, vp]
         L.im_bf16_to_f32.argtypes = [vp, i64, i32, i32, vp, vp]
         L.im_colsum_f32.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
@@ -548,6 +549,17 @@ def f32_to_bf16_padded_ptr(x, out_ptr: int, ld_out: int, stream=None):
     """Like f32_to_bf16_padded, into a raw device pointer (a policy's weight matrix from Policy.layer_buffers)."""
     _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], C.c_void_p(out_ptr), int(ld_out),
                                         _st(stream)), "im_f32_to_bf16_padded")
+
+
+def gather_rows(x, idx, out, status, stream=None):
+    """out[i] = x[idx[i]] for a float32 [R, cols] source (1-D sources are taken as one column); out float32 with
+    x's width, or bfloat16 [M, ld] zero padded.  idx: int32 CUDA tensor."""
+    import torch
+    x2 = x if x.dim() == 2 else x.view(-1, 1)
+    o2 = out if out.dim() == 2 else out.view(-1, 1)
+    _check(load().im_gather_rows_f32(_ptr(x2), x2.stride(0), _ptr(idx), x2.shape[0], idx.numel(), x2.shape[1], _ptr(o2),
+                                     o2.stride(0), int(out.dtype == torch.bfloat16), _ptr(status), _st(stream)),
+           "im_gather_rows_f32")
 
 
 def copy_f32_ptr(dst_ptr: int, src, stream=None):

@@ -138,6 +138,32 @@ __global__ void __launch_bounds__(256) sum_slices_kernel(const __nv_bfloat16 *__
     }
 }
 
+// Row gather for shuffled minibatches: out[i][0..cols) = in[idx[i]][0..cols), written as float or, with
+// zero padding up to ld_out, as bf16.  A warp copies one row (consecutive lanes, consecutive columns).
+template <bool TO_BF16>
+__global__ void __launch_bounds__(256) gather_rows_kernel(const float *__restrict__ in, long long ld_in,
+                                                          const int32_t *__restrict__ idx, long long n_src, int rows, int cols,
+                                                          void *__restrict__ out, int ld_out, uint32_t *__restrict__ status)
+{
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < rows; i += warps) {
+        long long src = idx[i];
+        if (src < 0 || src >= n_src) {                       // a bad index is clamped and reported, never followed
+            if (lane == 0) atomicOr(status, IM_DEV_BAD_STATE);
+            src = src < 0 ? 0 : n_src - 1;
+        }
+        const float *row = in + src * ld_in;
+        if (TO_BF16) {
+            __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out) + (long long)i * ld_out;
+            for (int c = lane; c < ld_out; c += 32) o[c] = __float2bfloat16_rn(c < cols ? __ldg(row + c) : 0.0f);
+        } else {
+            float *o = static_cast<float *>(out) + (long long)i * ld_out;
+            for (int c = lane; c < cols; c += 32) o[c] = __ldg(row + c);
+        }
+    }
+}
+
 // Column sums, stage 1: a CTA adds a slice of 256 rows for 64 columns; thread (column, row group g of 4)
 // adds rows g, g + 4, ... in two independent chains, the four groups are then added in order.
 constexpr int kColsumRowsPerCta = 256;
@@ -378,6 +404,21 @@ im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, in
     const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
     to_bf16_padded_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(in, ld_in, rows, cols,
                                                                        reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+}
+
+im_status im_gather_rows_f32(const float *in, int64_t ld_in, const int32_t *idx, int64_t n_src, int32_t rows, int32_t cols,
+                             void *out, int32_t ld_out, int32_t to_bf16, uint32_t *status, void *cuda_stream)
+{
+    using namespace im;
+    if (!in || !idx || !out || !status || n_src < 1 || rows < 1 || cols < 1 || ld_in < cols || ld_out < cols)
+        return IM_ERR_INVALID_ARG;
+    long long g = ((long long)rows * 32 + 255) / 256;
+    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (to_bf16) gather_rows_kernel<true><<<grid, 256, 0, st>>>(in, ld_in, idx, n_src, rows, cols, out, ld_out, status);
+    else gather_rows_kernel<false><<<grid, 256, 0, st>>>(in, ld_in, idx, n_src, rows, cols, out, ld_out, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }

@@ -207,11 +207,14 @@ class PpoUpdater:
         B.adaptive_lr(self.lr, self.summary[4:5], self.kl_target, stream=st)
 
 
-def update_from_storage(upd: PpoUpdater, storage, epochs: int, n_minibatches: int):
-    """The update phase over one collected rollout: `epochs` passes over `n_minibatches` contiguous blocks
-    of the T * N samples (row t * N + e of the flattened time-major arrays).  Each block's observations
-    are converted into both nets' bf16 input rows by im_f32_to_bf16_padded; everything else is read in
-    place from the storage.  Enqueues only; capturable in a CUDA graph together with the rollout."""
+def update_from_storage(upd: PpoUpdater, storage, epochs: int, n_minibatches: int, perm: torch.Tensor = None):
+    """The update phase over one collected rollout: `epochs` passes over `n_minibatches` blocks of the
+    T * N samples (row t * N + e of the flattened time-major arrays).
+    perm None: contiguous blocks -- each block's observations are converted into both nets' bf16 input
+    rows by im_f32_to_bf16_padded, everything else is read in place from the storage.
+    perm: int32 CUDA tensor [epochs, T * N], a permutation of the sample indices per epoch (shuffled
+    minibatches): every per-sample array of a block is gathered by im_gather_rows_f32.
+    Enqueues only; capturable in a CUDA graph together with the rollout."""
     T, N, A = storage.T, storage.N, storage.A
     total = T * N
     M = total // n_minibatches
@@ -225,10 +228,27 @@ def update_from_storage(upd: PpoUpdater, storage, epochs: int, n_minibatches: in
     adv, ret, val = flat(storage.advantage), flat(storage.returns), storage.value[:T].reshape(total)
     D = upd.actor.dims[0]
     st = upd.stream
-    for _ in range(epochs):
+    if perm is not None:
+        if perm.dtype != torch.int32 or tuple(perm.shape) != (epochs, total):
+            raise ValueError("perm must be an int32 tensor [epochs, T * N]")
+        if not hasattr(upd, "_gather") or upd._gather["action"].shape[0] < M:
+            f = lambda *sh: torch.empty(*sh, dtype=torch.float32, device="cuda")
+            upd._gather = dict(action=f(M, A), mean_old=f(M, A), logp_old=f(M), advantage=f(M), value_old=f(M), returns=f(M))
+    for ep in range(epochs):
         for k in range(n_minibatches):
             sl = slice(k * M, (k + 1) * M)
-            for tr in (upd.actor, upd.critic):
-                B.f32_to_bf16_padded(obs[sl, :D], tr.input_rows(M), st)
-            upd.update(M, dict(action=action[sl], mean_old=mean[sl], log_std_old=upd.log_std_old, logp_old=logp[sl],
-                               advantage=adv[sl], value_old=val[sl], returns=ret[sl]))
+            if perm is None:
+                for tr in (upd.actor, upd.critic):
+                    B.f32_to_bf16_padded(obs[sl, :D], tr.input_rows(M), st)
+                batch = dict(action=action[sl], mean_old=mean[sl], logp_old=logp[sl], advantage=adv[sl], value_old=val[sl],
+                             returns=ret[sl])
+            else:
+                idx = perm[ep, sl]
+                for tr in (upd.actor, upd.critic):
+                    B.gather_rows(obs[:, :D], idx, tr.input_rows(M), upd.actor.status, st)
+                g = upd._gather
+                for name, src in (("action", action), ("mean_old", mean), ("logp_old", logp), ("advantage", adv),
+                                  ("value_old", val), ("returns", ret)):
+                    B.gather_rows(src, idx, g[name][:M], upd.actor.status, st)
+                batch = {name: g[name][:M] for name in g}
+            upd.update(M, dict(batch, log_std_old=upd.log_std_old))

@@ -302,3 +302,65 @@ def test_transposed_product_reads_both_operands_in_place(R, Mo, No, slices):
     for s in range(slices):
         want = a[s * Rs:(s + 1) * Rs].astype(np.float64).T @ b[s * Rs:(s + 1) * Rs].astype(np.float64)
         assert np.abs(got[s, :Mo] - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3, "slice %d" % s
+
+
+def test_row_gather_is_exact_and_flags_bad_indices():
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn((5000, 361), generator=g).cuda()
+    v = torch.randn(5000, generator=g).cuda()
+    idx = torch.randperm(5000, generator=g)[:1234].to(torch.int32).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((1234, 361), 7.0, device="cuda")
+    B.gather_rows(x, idx, out, status)
+    assert torch.equal(out, x[idx.long()])
+    out1 = torch.empty(1234, device="cuda")
+    B.gather_rows(v, idx, out1, status)
+    assert torch.equal(out1, v[idx.long()])
+    ob = torch.full((1234, 384), 7.0, dtype=torch.bfloat16, device="cuda")
+    B.gather_rows(x, idx, ob, status)
+    assert torch.equal(ob[:, :361], x[idx.long()].to(torch.bfloat16)) and not ob[:, 361:].any()
+    assert int(status.item()) == 0
+    bad = idx.clone(); bad[5] = 5000; bad[9] = -1
+    B.gather_rows(x, bad, out, status)
+    assert int(status.item()) != 0                                   # clamped and reported, nothing read out of range
+    assert torch.equal(out[5], x[4999]) and torch.equal(out[9], x[0]) and torch.equal(out[10], x[idx[10].long()])
+
+
+def test_shuffled_minibatches_equal_contiguous_ones_on_permuted_data():
+    """update_from_storage with a permutation visits sample perm[k] where the contiguous path visits
+    sample k: run on the permutation and on explicitly permuted arrays, the two leave the same bits."""
+    from types import SimpleNamespace
+    dims, cdims, Tn, n = (61, 128, 64, 12), (61, 128, 64, 1), 4, 128
+    A, D, total = dims[-1], dims[0], Tn * n
+    ld = B.padded_ld(D)
+    g = torch.Generator().manual_seed(11)
+    rnd = lambda *sh: torch.randn(*sh, generator=g).cuda()
+    base = SimpleNamespace(T=Tn, N=n, A=A, keep_obs=True, ld_obs=ld, obs=rnd(Tn + 1, n, ld), action=rnd(Tn, n, A),
+                           mean=rnd(Tn, n, A) * 0.1, logp=rnd(Tn, n) - 5.0, advantage=rnd(Tn, n), returns=rnd(Tn, n),
+                           value=rnd(Tn + 1, n))
+    perm = torch.stack([torch.randperm(total, generator=g) for _ in range(2)]).to(torch.int32).cuda()
+
+    def fresh():
+        aw, cw = W.make_policy_weights(dims, "bf16", 2), W.make_policy_weights(cdims, "bf16", 3)
+        return T.PpoUpdater(T.MlpTrainer(dims, aw["W"], aw["b"], 256), T.MlpTrainer(cdims, cw["W"], cw["b"], 256),
+                            torch.full((A,), -1.0), lr=1e-3)
+
+    up1 = fresh()
+    T.update_from_storage(up1, base, epochs=2, n_minibatches=2, perm=perm)
+    up2 = fresh()
+    for ep in range(2):
+        p = perm[ep].long()
+        take = lambda x, *tail: x.reshape(total, *tail)[p].reshape(Tn, n, *tail).contiguous()
+        obs = base.obs.clone(); obs[:Tn] = take(base.obs[:Tn], ld)
+        val = base.value.clone(); val[:Tn] = take(base.value[:Tn])
+        shuffled = SimpleNamespace(T=Tn, N=n, A=A, keep_obs=True, ld_obs=ld, obs=obs, action=take(base.action, A),
+                                   mean=take(base.mean, A), logp=take(base.logp), advantage=take(base.advantage),
+                                   returns=take(base.returns), value=val)
+        T.update_from_storage(up2, shuffled, epochs=1, n_minibatches=2)
+    torch.cuda.synchronize()
+    for a, b in zip(up1.actor.W + up1.critic.W + [up1.log_std, up1.lr, up1.summary],
+                    up2.actor.W + up2.critic.W + [up2.log_std, up2.lr, up2.summary]):
+        assert torch.equal(a, b)
+    assert up1.actor.device_status() == 0
+    with pytest.raises(ValueError):
+        T.update_from_storage(up1, base, epochs=2, n_minibatches=2, perm=perm.long())
