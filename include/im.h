@@ -449,6 +449,13 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.
  * im_relu_mask_bf16: dH[r][c] = H[r][c] > 0 ? dH[r][c] : 0 in place; cols, ld_d, ld_h
  *   multiples of 8, 16-byte aligned pointers.
+ * im_gemm_bf16_dgrad: the backward product through a linear layer fused with what follows it,
+ *   dH[r][c] = (H[r][c] > 0) * sum_k dZ[r][k] Wt[c][k]  as bf16 [M][N] (Wt = the layer's weights transposed,
+ *   bf16 [N][K]; H = the forward activations the ReLU produced, bf16 [M][N], or NULL for no mask), and
+ *   colsum_partial[(r / 32) * ld_partial + c] = the sum of the fp32 values of dH over the 32-row block
+ *   (float [M / 32][ld_partial], or NULL); summing those rows with im_colsum_f32 gives the bias gradient
+ *   of the layer below.  M a multiple of 32; zeros: DEVICE float [N] of zeros; the other rules of
+ *   im_gemm_bf16 apply.
  * im_f32_to_bf16_padded: out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
  * im_gather_rows_f32: out[i][0..cols) = in[idx[i]][0..cols) for i < rows (shuffled minibatches); idx
  *   DEVICE int32 [rows] with values in [0, n_src); out is float [rows][ld_out], or with to_bf16 != 0
@@ -463,6 +470,9 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
 im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                        int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu, uint32_t *status,
                        void *cuda_stream);
+im_status im_gemm_bf16_dgrad(const uint16_t *dZ, int64_t ld_dz, const uint16_t *Wt, int64_t ld_wt, uint16_t *dH, int64_t ld_dh,
+                             int32_t M, int32_t N, int32_t K, const uint16_t *H, int64_t ld_h, float *colsum_partial,
+                             int32_t ld_partial, const float *zeros, uint32_t *status, void *cuda_stream);
 im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                                int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
                                uint32_t *status, void *cuda_stream);

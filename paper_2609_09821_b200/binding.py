@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad",
 ]
 
 
@@ -141,6 +141,7 @@ def load():
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp, vp]
         L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
         L.im_copy_f32.argtypes = [vp, vp, i64, vp]
         L.im_bf16_to_f32.argtypes = [vp, i64, i32, i32, vp, vp]
@@ -549,6 +550,18 @@ def f32_to_bf16_padded_ptr(x, out_ptr: int, ld_out: int, stream=None):
     """Like f32_to_bf16_padded, into a raw device pointer (a policy's weight matrix from Policy.layer_buffers)."""
     _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], C.c_void_p(out_ptr), int(ld_out),
                                         _st(stream)), "im_f32_to_bf16_padded")
+
+
+def gemm_bf16_dgrad(dZ, Wt, dH, H, colsum_partial, zeros, status, stream=None):
+    """dH [M, N] = (H > 0) * (dZ [M, K] @ Wt [N, K]^T) as bf16, and the fp32 column sums of dH per 32-row block into
+    colsum_partial [M / 32, >= N] float32.  H and colsum_partial may be None."""
+    M, K = dZ.shape
+    N = Wt.shape[0]
+    _check(load().im_gemm_bf16_dgrad(_ptr(dZ), dZ.stride(0), _ptr(Wt), Wt.stride(0), _ptr(dH), dH.stride(0), M, N, K,
+                                     _ptr(H) if H is not None else None, H.stride(0) if H is not None else 0,
+                                     _ptr(colsum_partial) if colsum_partial is not None else None,
+                                     colsum_partial.stride(0) if colsum_partial is not None else 0, _ptr(zeros), _ptr(status),
+                                     _st(stream)), "im_gemm_bf16_dgrad")
 
 
 def gather_rows(x, idx, out, status, stream=None):

@@ -33,7 +33,8 @@ void *tc_policy_input(im_policy *p, int32_t *ld);     // bf16 [max_batch][ld] st
 im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float *obs, int32_t ld_obs,
                             float *mean_out, float *action_out, float *logp_out, im_policy *src = nullptr);
 im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int M, int N, int K,
-                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches = 1);
+                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches = 1,
+                  const void *mask = nullptr, int64_t ld_mask = 0, float *colsum_partial = nullptr, int ld_partial = 0);
 im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int R, int Mo, int No,
                      int slices, int c_pitch, const float *bias, uint32_t *status, cudaStream_t stream);
 im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, int M, int N, int K, const float *bias,

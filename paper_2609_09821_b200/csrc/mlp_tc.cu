@@ -182,6 +182,13 @@ struct GemmParams {
     // with rows [b b_batch_rows, +N) of B into rows [b a_batch_rows, +M) of C.  n_batches = 1: plain GEMM.
     int n_batches, a_batch_rows, b_batch_rows;
     int c_batch_rows;  // rows of C between two batches
+    // Backward-pass epilogue (BWD instantiations): output (r, c) is zeroed where mask[r][c] <= 0 (the ReLU of the
+    // forward pass), and the column sums of the masked fp32 values over each 32-row block r / 32 go to
+    // colsum_partial[(r / 32) * ld_partial + c] (M a multiple of 32).  Either may be null.
+    const __nv_bfloat16 *mask;
+    long long ld_mask;
+    float *colsum_partial;
+    int ld_partial;
     // Gaussian head
     float *mean, *action, *logp;
     float sigma;
@@ -355,11 +362,89 @@ __device__ __forceinline__ void mma_role(const Pipe &p, uint32_t tmem_base, cons
     }
 }
 
+// Warp reduce-scatter step: every lane holds 2 C values; afterwards C sums over the lane pair (lane, lane ^ offset),
+// the lower lane keeping the first C columns and the upper lane the second C.
+template <int C>
+__device__ __forceinline__ void reduce_scatter_step(float *v, int lane, int offset)
+{
+    const bool up = (lane & offset) != 0;
+#pragma unroll
+    for (int i = 0; i < C; ++i) {
+        const float keep = up ? v[i + C] : v[i], send = up ? v[i] : v[i + C];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, offset);
+    }
+}
+
+// One epilogue chunk of the hidden-layer kernels: 64 accumulator columns of this thread's row -> bias, floor,
+// (BWD: ReLU mask of the forward activations, column sums over the warp's 32 rows) -> 32 packed bf16 pairs.
+// The forward activations of this thread's row under 64 output columns (8 x 16 bytes); rows past M read as positive.
+__device__ __forceinline__ void load_mask(const GemmParams &P, int row, int col0, uint4 (&mk)[8])
+{
+    if (P.mask && row < P.M) {
+        const uint4 *m4 = reinterpret_cast<const uint4 *>(P.mask + (long long)row * P.ld_mask + col0);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) mk[c] = __ldg(m4 + c);
+    } else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) mk[c] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
+    }
+}
+
+template <bool BWD>
+__device__ __forceinline__ void hidden_chunk(const GemmParams &P, uint32_t t_addr, int row, int col0, int lane,
+                                             const uint4 (&mk)[8], uint32_t (&pk)[32])
+{
+    float v[64];
+    tmem_ld32_issue(t_addr, v);
+    tmem_ld32_issue(t_addr + 32u, v + 32);
+    tmem_ld_wait();
+    const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + col0);
+    const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float4 b = __ldg(b4 + i);
+        v[4 * i] = fmaxf(v[4 * i] + b.x, fl);
+        v[4 * i + 1] = fmaxf(v[4 * i + 1] + b.y, fl);
+        v[4 * i + 2] = fmaxf(v[4 * i + 2] + b.z, fl);
+        v[4 * i + 3] = fmaxf(v[4 * i + 3] + b.w, fl);
+    }
+    if (BWD) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t w[4] = {mk[c].x, mk[c].y, mk[c].z, mk[c].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                // a bf16 is positive when its 16 bits read as a signed integer are
+                if ((int)(short)(w[j] & 0xffffu) <= 0) v[8 * c + 2 * j] = 0.0f;
+                if ((int)(short)(w[j] >> 16) <= 0) v[8 * c + 2 * j + 1] = 0.0f;
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        pk[i] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+    if (BWD) {
+        if (P.colsum_partial) {
+            reduce_scatter_step<32>(v, lane, 16);
+            reduce_scatter_step<16>(v, lane, 8);
+            reduce_scatter_step<8>(v, lane, 4);
+            reduce_scatter_step<4>(v, lane, 2);
+            reduce_scatter_step<2>(v, lane, 1);
+            const int row0 = row - lane;                 // lane now holds columns 2 lane, 2 lane + 1 of the 64
+            if (row0 < P.M)
+                *reinterpret_cast<float2 *>(P.colsum_partial + (long long)(row0 >> 5) * P.ld_partial + col0 + 2 * lane) =
+                    make_float2(v[0], v[1]);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ hidden layers
 // C = relu(A W^T + b) as bf16.  Each epilogue warp owns 32 rows of the tile: it
 // reads 64 accumulator columns at a time, applies bias and ReLU, packs to bf16
 // into a 128B-swizzled slab in shared memory and hands the slab to a TMA store.
-template <int BLOCK_N, bool MN = false>
+template <int BLOCK_N, bool MN = false, bool BWD = false>
 __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                        const __grid_constant__ CUtensorMap map_b,
                                                                        const __grid_constant__ CUtensorMap map_c,
@@ -384,28 +469,36 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
         int which = 0;
         int acc = 0;
         uint32_t acc_phase = 0;
+        // BWD: the mask words of a chunk are fetched one chunk ahead (across tile boundaries), so their
+        // latency hides behind the previous chunk and the wait for the accumulator
+        uint4 mk[8], mk_next[8];
+        if (BWD && (int)blockIdx.x < n_tiles) {
+            const int bt = (int)blockIdx.x / tiles_per_batch, tt = (int)blockIdx.x - bt * tiles_per_batch;
+            load_mask(P, bt * P.c_batch_rows + (tt / P.n_tiles_n) * BLOCK_M + quad * 32 + lane, (tt % P.n_tiles_n) * BLOCK_N, mk);
+        }
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
             const int bt = tile / tiles_per_batch, tt = tile - bt * tiles_per_batch;
             const int m0 = bt * P.c_batch_rows + (tt / P.n_tiles_n) * BLOCK_M, n0 = (tt % P.n_tiles_n) * BLOCK_N;
-            if (!mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag)) break;
+            bool ready = mbar_wait(&p.acc_full[acc], acc_phase, p.abort_flag);
+            if (BWD) ready = __all_sync(0xffffffffu, ready);           // the column sums shuffle across the whole warp
+            if (!ready) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Plan::kAccStride);
 #pragma unroll 1
             for (int c0 = 0; c0 < BLOCK_N; c0 += 64) {
-                float v[64];
-                tmem_ld32_issue(t_row + (uint32_t)c0, v);
-                tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
-                tmem_ld_wait();
-                const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
-                const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
                 uint32_t pk[32];
+                if (BWD) {
+                    if (c0 + 64 < BLOCK_N) load_mask(P, m0 + quad * 32 + lane, n0 + c0 + 64, mk_next);
+                    else if (tile + (int)gridDim.x < n_tiles) {
+                        const int t2 = tile + (int)gridDim.x, bt2 = t2 / tiles_per_batch, tt2 = t2 - bt2 * tiles_per_batch;
+                        load_mask(P, bt2 * P.c_batch_rows + (tt2 / P.n_tiles_n) * BLOCK_M + quad * 32 + lane,
+                                  (tt2 % P.n_tiles_n) * BLOCK_N, mk_next);
+                    }
+                }
+                hidden_chunk<BWD>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
+                if (BWD) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float4 b = __ldg(b4 + i);
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, fl), fmaxf(v[4 * i + 1] + b.y, fl));
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, fl), fmaxf(v[4 * i + 3] + b.w, fl));
-                    pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
-                    pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+                    for (int c = 0; c < 8; ++c) mk[c] = mk_next[c];
                 }
                 // the store issued two slabs ago (same buffer) must have finished reading shared memory
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -507,6 +600,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
                  ::"r"(smem_u32(bar)), "h"(both) : "memory");
 }
 
+template <bool BWD = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                              const __grid_constant__ CUtensorMap map_c, const GemmParams P)
@@ -601,29 +695,33 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
         int which = 0;
         int acc = 0;
         uint32_t acc_phase = 0;
+        uint4 mk[8], mk_next[8];                     // BWD: mask words, fetched one chunk ahead
+        if (BWD && pair < n_tiles)
+            load_mask(P, (pair / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32 + lane, (pair % P.n_tiles_n) * 256, mk);
         if (!*abort_flag)
         for (int tile = pair; tile < n_tiles; tile += n_pairs) {
             const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
             const int n0 = (tile % P.n_tiles_n) * 256;
-            if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) break;
+            bool ready = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
+            if (BWD) ready = __all_sync(0xffffffffu, ready);           // the column sums shuffle across the whole warp
+            if (!ready) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
 #pragma unroll 1
             for (int c0 = 0; c0 < 256; c0 += 64) {
-                float v[64];
-                tmem_ld32_issue(t_row + (uint32_t)c0, v);
-                tmem_ld32_issue(t_row + (uint32_t)c0 + 32u, v + 32);
-                tmem_ld_wait();
-                const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + n0 + c0);
-                const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
                 uint32_t pk[32];
+                if (BWD) {
+                    if (c0 + 64 < 256) load_mask(P, m0 + quad * 32 + lane, n0 + c0 + 64, mk_next);
+                    else if (tile + n_pairs < n_tiles) {
+                        const int t2 = tile + n_pairs;
+                        load_mask(P, (t2 / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32 + lane,
+                                  (t2 % P.n_tiles_n) * 256, mk_next);
+                    }
+                }
+                hidden_chunk<BWD>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
+                if (BWD) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float4 b = __ldg(b4 + i);
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaxf(v[4 * i] + b.x, fl), fmaxf(v[4 * i + 1] + b.y, fl));
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaxf(v[4 * i + 2] + b.z, fl), fmaxf(v[4 * i + 3] + b.w, fl));
-                    pk[2 * i] = *reinterpret_cast<const uint32_t *>(&lo);
-                    pk[2 * i + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+                    for (int c = 0; c < 8; ++c) mk[c] = mk_next[c];
                 }
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 __syncwarp();
@@ -903,13 +1001,13 @@ namespace im {
 
 namespace {
 
-template <int BLOCK_N>
+template <int BLOCK_N, bool BWD = false>
 cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
     static bool prepared = false;
     if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, false, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         prepared = true;
@@ -919,7 +1017,7 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
     const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    linear_tc_hidden_kernel<BLOCK_N, false, BWD><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -947,18 +1045,19 @@ cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm
     return cudaGetLastError();
 }
 
+template <bool BWD>
 cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
 {
     static bool prepared = false;
     if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kPairSmemBytes);
         if (e != cudaSuccess) return e;
         prepared = true;
     }
     const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-    linear_tc_hidden_pair_kernel<<<2 * pairs, kThreads, kPairSmemBytes, stream>>>(L.map_a, L.map_b2, L.map_c, gp);
+    linear_tc_hidden_pair_kernel<BWD><<<2 * pairs, kThreads, kPairSmemBytes, stream>>>(L.map_a, L.map_b2, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -994,12 +1093,13 @@ cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n
         // balance the machine better (measured: 16384 x 1024 x 384 is 8 % faster single, 16384 x 1024 x 2048
         // 7 % faster paired)
         const int pair_tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
+        const bool bwd = gp.mask || gp.colsum_partial;
         if (L.block_n == 256 && gp.n_batches == 1 && (force_pairs || (pair_tiles >= n_sm && gp.K_blocks >= 8)))
-            return launch_hidden_pair(L, gp, n_sm, stream);
+            return bwd ? launch_hidden_pair<true>(L, gp, n_sm, stream) : launch_hidden_pair<false>(L, gp, n_sm, stream);
         switch (L.block_n) {
-        case 256: return launch_hidden<256>(L, gp, n_sm, stream);
-        case 128: return launch_hidden<128>(L, gp, n_sm, stream);
-        default: return launch_hidden<64>(L, gp, n_sm, stream);
+        case 256: return bwd ? launch_hidden<256, true>(L, gp, n_sm, stream) : launch_hidden<256>(L, gp, n_sm, stream);
+        case 128: return bwd ? launch_hidden<128, true>(L, gp, n_sm, stream) : launch_hidden<128>(L, gp, n_sm, stream);
+        default: return bwd ? launch_hidden<64, true>(L, gp, n_sm, stream) : launch_hidden<64>(L, gp, n_sm, stream);
         }
     }
     switch (L.block_n) {
@@ -1141,6 +1241,7 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
         if (l == 0 && external) L.map_a = tc->map_a_ext;
         const bool last = l == p->nl - 1;
         GemmParams gp;
+        std::memset(&gp, 0, sizeof(gp));
         gp.M = n; gp.N = L.N; gp.K_blocks = L.Kpad / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = L.d_bias;
         gp.act_floor = 0.0f;
         gp.n_batches = 1; gp.a_batch_rows = 0; gp.b_batch_rows = 0; gp.c_batch_rows = 0;
@@ -1156,7 +1257,8 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
 // C[M][N] = act(A[M][K] B[N][K]^T + bias) on the hidden-layer kernels, operands anywhere in device
 // memory: the three tensor maps are encoded for this call and travel as kernel parameters.
 im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int M, int N, int K,
-                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches)
+                  const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches, const void *mask,
+                  int64_t ld_mask, float *colsum_partial, int ld_partial)
 {
     static int n_sm = 0;
     if (!n_sm) {
@@ -1182,6 +1284,8 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
     gp.act_floor = relu ? 0.0f : -INFINITY;
     gp.n_batches = batches; gp.a_batch_rows = M; gp.b_batch_rows = N; gp.c_batch_rows = M;
+    gp.mask = static_cast<const __nv_bfloat16 *>(mask); gp.ld_mask = ld_mask;
+    gp.colsum_partial = colsum_partial; gp.ld_partial = ld_partial;
     gp.status = status;
     return dispatch_tc(L, gp, false, n_sm, false, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }

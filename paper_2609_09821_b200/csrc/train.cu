@@ -312,6 +312,20 @@ im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_
     return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream);
 }
 
+im_status im_gemm_bf16_dgrad(const uint16_t *dZ, int64_t ld_dz, const uint16_t *Wt, int64_t ld_wt, uint16_t *dH, int64_t ld_dh,
+                             int32_t M, int32_t N, int32_t K, const uint16_t *H, int64_t ld_h, float *colsum_partial,
+                             int32_t ld_partial, const float *zeros, uint32_t *status, void *cuda_stream)
+{
+    using namespace im;
+    if (!dZ || !Wt || !dH || !zeros || !status || M < 32 || (M & 31) || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
+    if ((N & 63) || (K & 63) || ld_dz < K || ld_wt < K || ld_dh < N || (ld_dz & 7) || (ld_wt & 7) || (ld_dh & 7)) return IM_ERR_INVALID_ARG;
+    if (!al16(dZ) || !al16(Wt) || !al16(dH) || !al16(zeros)) return IM_ERR_INVALID_ARG;
+    if (H && (ld_h < N || (ld_h & 7) || !al16(H))) return IM_ERR_INVALID_ARG;
+    if (colsum_partial && (ld_partial < N || (ld_partial & 1) || (reinterpret_cast<uintptr_t>(colsum_partial) & 7u))) return IM_ERR_INVALID_ARG;
+    return tc_gemm(dZ, ld_dz, Wt, ld_wt, dH, ld_dh, M, N, K, zeros, false, status, (cudaStream_t)cuda_stream, 1, H, ld_h,
+                   colsum_partial, ld_partial);
+}
+
 im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                                int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
                                uint32_t *status, void *cuda_stream)

@@ -68,6 +68,7 @@ class MlpTrainer:
         self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.colsum_ws = torch.empty(((Mb + 255) // 256) * max(self.Np), dtype=f32, device=dev)
+        self.col_partial = torch.empty((Mb // 32, max(self.Np)), dtype=f32, device=dev)   # 32-row column sums of a dH product
         self.t = 0
         with torch.cuda.stream(self.stream):
             for l in range(self.nl):
@@ -116,9 +117,11 @@ class MlpTrainer:
             B.sum_slices_bf16_to_f32(dWs, S, N, K, self.dW[l], st)
             if l > 0:
                 dH = self.dZ[l - 1][:M]                                                       # [M, Kp] = [M, Np of layer l-1]
-                B.gemm_bf16(dZ, self.WbT[l], dH, self.zeros, False, self.status, st)         # dH = dZ W
-                B.relu_mask_bf16(dH, self.H[l][:M], st)
-                B.colsum(dH[:, :K], self.db[l - 1], self.colsum_ws, st)
+                # dH = (H > 0) * (dZ W); the GEMM's epilogue applies the ReLU mask and leaves the column sums of
+                # every 32-row block, which add up to the bias gradient of the layer below
+                part = self.col_partial[:M // 32]
+                B.gemm_bf16_dgrad(dZ, self.WbT[l], dH, self.H[l][:M], part, self.zeros, self.status, st)
+                B.colsum(part[:, :K], self.db[l - 1], self.colsum_ws, st)
 
     # -- optimiser -------------------------------------------------------------
     def grads(self) -> List[torch.Tensor]:

@@ -364,3 +364,30 @@ def test_shuffled_minibatches_equal_contiguous_ones_on_permuted_data():
     assert up1.actor.device_status() == 0
     with pytest.raises(ValueError):
         T.update_from_storage(up1, base, epochs=2, n_minibatches=2, perm=perm.long())
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 64, 64), (320, 128, 192), (1024, 256, 128), (37888 + 64, 512, 1024), (40000 - 32, 1024, 512)])
+def test_dgrad_product_masks_and_sums_in_its_epilogue(M, N, K):
+    """im_gemm_bf16_dgrad against the three separate steps it replaces, in exact arithmetic: small integer
+    operands make every product and sum exact, so the fused output and its 32-row column sums must
+    equal dZ @ Wt^T masked by H > 0 bit for bit (single-CTA and CTA-pair kernels, ragged last tiles)."""
+    g = torch.Generator().manual_seed(M + N)
+    dz = torch.randint(-2, 3, (M, K), generator=g).to(torch.bfloat16).cuda()
+    wt = torch.randint(-2, 3, (N, K), generator=g).to(torch.bfloat16).cuda()
+    h = torch.randint(-1, 3, (M, N), generator=g).clamp(min=0).to(torch.bfloat16).cuda()
+    h[0, :] = 0; h[:, 1] = 0; h[3, 5] = -0.0
+    zeros = torch.zeros(N, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    want = (dz.float() @ wt.float().T) * (h > 0)
+    for use_mask, use_sum in ((True, True), (True, False), (False, True)):
+        out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+        part = torch.full((M // 32, N + 2), 7.0, device="cuda")
+        B.gemm_bf16_dgrad(dz, wt, out, h if use_mask else None, part if use_sum else None, zeros, status)
+        ref = want if use_mask else dz.float() @ wt.float().T
+        assert torch.equal(out.float(), ref.to(torch.bfloat16).float())
+        if use_sum:
+            assert torch.equal(part[:, :N], ref.view(M // 32, 32, N).sum(1))
+            assert (part[:, N:] == 7.0).all()
+        else:
+            assert (part == 7.0).all()
+    assert int(status.item()) == 0
