@@ -212,7 +212,8 @@ struct SmemPlan {
     static constexpr int kBarBytes = 256;
     static constexpr int kMaxStages = 8;
     // hidden layers: two staging slabs per epilogue warp for the TMA stores
-    static constexpr __host__ __device__ int hidden_epi_bytes() { return 4 * 2 * kEpiSlabBytes; }
+    // (backward epilogue: two more per warp for the ReLU mask boxes)
+    static constexpr __host__ __device__ int hidden_epi_bytes(bool bwd = false) { return (bwd ? 2 : 1) * 4 * 2 * kEpiSlabBytes; }
     // head: [2 accumulators][mean, action][128 rows][A] floats laid out as in global memory,
     // partial sums of z^2 [2][4][128], band counters [2][4]
     __host__ __device__ static constexpr int head_epi_bytes(int A) { return (2 * 2 * 128 * A * 4 + 2 * 4 * 128 * 4 + 64 + 1023) / 1024 * 1024; }
@@ -231,6 +232,7 @@ struct Pipe {
     uint64_t *full, *empty, *acc_full, *acc_empty;
     uint32_t *tmem_slot;
     volatile int *abort_flag;
+    uint64_t *mask_bar;      // [4 epilogue warps][2]
     uint8_t *epi;
 };
 
@@ -248,6 +250,7 @@ __device__ __forceinline__ Pipe carve_pipe(uint8_t *smem_raw, int stages, int ep
     p.acc_empty = bars + 2 * Plan::kMaxStages + 2;
     p.tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Plan::kMaxStages + 4);
     p.abort_flag = reinterpret_cast<volatile int *>(p.tmem_slot + 1);
+    p.mask_bar = bars + 2 * Plan::kMaxStages + 5;
     return p;
 }
 
@@ -257,6 +260,7 @@ __device__ __forceinline__ void pipe_init(const Pipe &p, int epi_arrivals)
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&p.full[s], 1); mbar_init(&p.empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&p.acc_full[a], 1); mbar_init(&p.acc_empty[a], epi_arrivals); }
+        for (int i = 0; i < 2 * kEpiWarps; ++i) mbar_init(&p.mask_bar[i], 1);
         *p.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -377,17 +381,26 @@ __device__ __forceinline__ void reduce_scatter_step(float *v, int lane, int offs
 
 // One epilogue chunk of the hidden-layer kernels: 64 accumulator columns of this thread's row -> bias, floor,
 // (BWD: ReLU mask of the forward activations, column sums over the warp's 32 rows) -> 32 packed bf16 pairs.
-// The forward activations of this thread's row under 64 output columns (8 x 16 bytes); rows past M read as positive.
-__device__ __forceinline__ void load_mask(const GemmParams &P, int row, int col0, uint4 (&mk)[8])
+// ReLU mask of the backward epilogue: each epilogue warp keeps two 32-row x 64-column boxes of the forward
+// activations in shared memory (128B-swizzled, like the output slabs), fetched by TMA one chunk ahead.
+__device__ __forceinline__ void mask_issue(const CUtensorMap *map_m, uint8_t *slab, uint64_t *bar, int col0, int row0)
 {
-    if (P.mask && row < P.M) {
-        const uint4 *m4 = reinterpret_cast<const uint4 *>(P.mask + (long long)row * P.ld_mask + col0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the warp's earlier reads of this slab come first
+    mbar_arrive_expect_tx(bar, kEpiSlabBytes);
+    tma_load_2d(slab, map_m, bar, col0, row0);
+}
+__device__ __forceinline__ void mask_read(const uint8_t *slab, int lane, uint4 (&mk)[8])
+{
+    const uint32_t row = smem_u32(slab) + (uint32_t)lane * 128u;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) mk[c] = __ldg(m4 + c);
-    } else {
+    for (int c = 0; c < 8; ++c)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(mk[c].x), "=r"(mk[c].y), "=r"(mk[c].z), "=r"(mk[c].w)
+                     : "r"(row + (uint32_t)((c ^ (lane & 7)) << 4)) : "memory");
+}
+__device__ __forceinline__ void mask_all_positive(uint4 (&mk)[8])
+{
 #pragma unroll
-        for (int c = 0; c < 8; ++c) mk[c] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
-    }
+    for (int c = 0; c < 8; ++c) mk[c] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
 }
 
 template <bool BWD>
@@ -448,11 +461,12 @@ template <int BLOCK_N, bool MN = false, bool BWD = false>
 __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                        const __grid_constant__ CUtensorMap map_b,
                                                                        const __grid_constant__ CUtensorMap map_c,
+                                                                       const __grid_constant__ CUtensorMap map_m,
                                                                        const GemmParams P)
 {
     using Plan = SmemPlan<BLOCK_N>;
     extern __shared__ uint8_t smem_raw[];
-    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::hidden_epi_bytes());
+    const Pipe p = carve_pipe<Plan>(smem_raw, P.stages, Plan::hidden_epi_bytes(BWD));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_per_batch = ((P.M + BLOCK_M - 1) / BLOCK_M) * P.n_tiles_n;
     const int n_tiles = tiles_per_batch * P.n_batches;
@@ -469,12 +483,17 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
         int which = 0;
         int acc = 0;
         uint32_t acc_phase = 0;
-        // BWD: the mask words of a chunk are fetched one chunk ahead (across tile boundaries), so their
-        // latency hides behind the previous chunk and the wait for the accumulator
-        uint4 mk[8], mk_next[8];
-        if (BWD && (int)blockIdx.x < n_tiles) {
+        // BWD: the mask box of a chunk is fetched one chunk ahead (across tile boundaries), so its latency
+        // hides behind the previous chunk and the wait for the accumulator
+        const bool masked = BWD && P.mask != nullptr;
+        uint8_t *mslabs = p.epi + (size_t)(4 + warp - 2) * 2 * kEpiSlabBytes;
+        uint64_t *mbar = p.mask_bar + (warp - 2) * 2;
+        uint32_t ci = 0;                               // chunks consumed by this warp
+        bool bail = false;
+        uint4 mk[8];
+        if (masked && (int)blockIdx.x < n_tiles && lane == 0) {
             const int bt = (int)blockIdx.x / tiles_per_batch, tt = (int)blockIdx.x - bt * tiles_per_batch;
-            load_mask(P, bt * P.c_batch_rows + (tt / P.n_tiles_n) * BLOCK_M + quad * 32 + lane, (tt % P.n_tiles_n) * BLOCK_N, mk);
+            mask_issue(&map_m, mslabs, &mbar[0], (tt % P.n_tiles_n) * BLOCK_N, bt * P.c_batch_rows + (tt / P.n_tiles_n) * BLOCK_M + quad * 32);
         }
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
             const int bt = tile / tiles_per_batch, tt = tile - bt * tiles_per_batch;
@@ -488,18 +507,22 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
             for (int c0 = 0; c0 < BLOCK_N; c0 += 64) {
                 uint32_t pk[32];
                 if (BWD) {
-                    if (c0 + 64 < BLOCK_N) load_mask(P, m0 + quad * 32 + lane, n0 + c0 + 64, mk_next);
-                    else if (tile + (int)gridDim.x < n_tiles) {
-                        const int t2 = tile + (int)gridDim.x, bt2 = t2 / tiles_per_batch, tt2 = t2 - bt2 * tiles_per_batch;
-                        load_mask(P, bt2 * P.c_batch_rows + (tt2 / P.n_tiles_n) * BLOCK_M + quad * 32 + lane,
-                                  (tt2 % P.n_tiles_n) * BLOCK_N, mk_next);
-                    }
+                    if (masked) {
+                        if (lane == 0) {
+                            uint8_t *nslab = mslabs + ((ci + 1u) & 1u) * kEpiSlabBytes;
+                            if (c0 + 64 < BLOCK_N) mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], n0 + c0 + 64, m0 + quad * 32);
+                            else if (tile + (int)gridDim.x < n_tiles) {
+                                const int t2 = tile + (int)gridDim.x, bt2 = t2 / tiles_per_batch, tt2 = t2 - bt2 * tiles_per_batch;
+                                mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], (tt2 % P.n_tiles_n) * BLOCK_N,
+                                           bt2 * P.c_batch_rows + (tt2 / P.n_tiles_n) * BLOCK_M + quad * 32);
+                            }
+                        }
+                        if (!__all_sync(0xffffffffu, mbar_wait(&mbar[ci & 1u], (ci >> 1) & 1u, p.abort_flag))) { bail = true; break; }
+                        mask_read(mslabs + (ci & 1u) * kEpiSlabBytes, lane, mk);
+                        ++ci;
+                    } else mask_all_positive(mk);
                 }
                 hidden_chunk<BWD>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
-                if (BWD) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) mk[c] = mk_next[c];
-                }
                 // the store issued two slabs ago (same buffer) must have finished reading shared memory
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 __syncwarp();
@@ -520,6 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
                 }
                 which ^= 1;
             }
+            if (bail) break;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&p.acc_empty[acc]);
@@ -545,7 +569,11 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
 constexpr int kPairStages = 6;
 constexpr int kPairStageBytes = 2 * BLOCK_M * BLOCK_K * 2;             // A 128x64 + W half 128x64, bf16
 constexpr int kPairTmemCols = 512;                                     // two 256-column accumulators
-constexpr size_t kPairSmemBytes = 1024 + (size_t)kPairStages * kPairStageBytes + 4 * 2 * kEpiSlabBytes + 256;
+constexpr __host__ __device__ int pair_stages(bool bwd) { return bwd ? kPairStages - 1 : kPairStages; }
+constexpr size_t pair_smem_bytes(bool bwd)
+{
+    return 1024 + (size_t)pair_stages(bwd) * kPairStageBytes + (bwd ? 2 : 1) * 4 * 2 * kEpiSlabBytes + 256;
+}
 
 __device__ __forceinline__ uint32_t cluster_rank()
 {
@@ -603,12 +631,15 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
 template <bool BWD = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                             const __grid_constant__ CUtensorMap map_c, const GemmParams P)
+                             const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
+                             const GemmParams P)
 {
+    constexpr int kStages = pair_stages(BWD);        // the backward epilogue's mask boxes take one stage's room
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *epi = tiles + (size_t)kPairStages * kPairStageBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(epi + 4 * 2 * kEpiSlabBytes);
+    uint8_t *epi = tiles + (size_t)kStages * kPairStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(epi + (BWD ? 2 : 1) * 4 * 2 * kEpiSlabBytes);
+    uint64_t *mask_bar = bars + 2 * kPairStages + 5;
     uint64_t *full = bars, *empty = bars + kPairStages, *acc_full = bars + 2 * kPairStages,
              *acc_empty = bars + 2 * kPairStages + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kPairStages + 4);
@@ -621,7 +652,8 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
     const int n_tiles = tiles_m * P.n_tiles_n;                       // 256 x 256 tiles
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int i = 0; i < 2 * kEpiWarps; ++i) mbar_init(&mask_bar[i], 1);
         for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -656,7 +688,7 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
                     if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * kPairStageBytes);
                     tma_load_2d_pair(sa, &map_a, leader_full, kb * BLOCK_K, m0);
                     tma_load_2d_pair(sa + BLOCK_M * BLOCK_K * 2, &map_b, leader_full, kb * BLOCK_K, n0);
-                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
             }
@@ -681,7 +713,7 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
                         umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
                     umma_commit_pair(&empty[stage]);          // both CTAs' stages are free once these MMAs have read them
-                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit_pair(&acc_full[acc]);             // both CTAs' accumulators complete
@@ -695,9 +727,14 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
         int which = 0;
         int acc = 0;
         uint32_t acc_phase = 0;
-        uint4 mk[8], mk_next[8];                     // BWD: mask words, fetched one chunk ahead
-        if (BWD && pair < n_tiles)
-            load_mask(P, (pair / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32 + lane, (pair % P.n_tiles_n) * 256, mk);
+        const bool masked = BWD && P.mask != nullptr;   // BWD: mask boxes, fetched one chunk ahead
+        uint8_t *mslabs = epi + (size_t)(4 + warp - 2) * 2 * kEpiSlabBytes;
+        uint64_t *mbar = mask_bar + (warp - 2) * 2;
+        uint32_t ci = 0;
+        bool bail = false;
+        uint4 mk[8];
+        if (masked && pair < n_tiles && lane == 0 && !*abort_flag)
+            mask_issue(&map_m, mslabs, &mbar[0], (pair % P.n_tiles_n) * 256, (pair / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32);
         if (!*abort_flag)
         for (int tile = pair; tile < n_tiles; tile += n_pairs) {
             const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
@@ -711,18 +748,22 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
             for (int c0 = 0; c0 < 256; c0 += 64) {
                 uint32_t pk[32];
                 if (BWD) {
-                    if (c0 + 64 < 256) load_mask(P, m0 + quad * 32 + lane, n0 + c0 + 64, mk_next);
-                    else if (tile + n_pairs < n_tiles) {
-                        const int t2 = tile + n_pairs;
-                        load_mask(P, (t2 / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32 + lane,
-                                  (t2 % P.n_tiles_n) * 256, mk_next);
-                    }
+                    if (masked) {
+                        if (lane == 0) {
+                            uint8_t *nslab = mslabs + ((ci + 1u) & 1u) * kEpiSlabBytes;
+                            if (c0 + 64 < 256) mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], n0 + c0 + 64, m0 + quad * 32);
+                            else if (tile + n_pairs < n_tiles) {
+                                const int t2 = tile + n_pairs;
+                                mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], (t2 % P.n_tiles_n) * 256,
+                                           (t2 / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32);
+                            }
+                        }
+                        if (!__all_sync(0xffffffffu, mbar_wait(&mbar[ci & 1u], (ci >> 1) & 1u, abort_flag))) { bail = true; break; }
+                        mask_read(mslabs + (ci & 1u) * kEpiSlabBytes, lane, mk);
+                        ++ci;
+                    } else mask_all_positive(mk);
                 }
                 hidden_chunk<BWD>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
-                if (BWD) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) mk[c] = mk_next[c];
-                }
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 __syncwarp();
                 uint8_t *slab = slabs + which * kEpiSlabBytes;
@@ -742,6 +783,7 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
                 }
                 which ^= 1;
             }
+            if (bail) break;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[acc]), 0));   // the leader's barrier
@@ -983,6 +1025,7 @@ struct TcLayer {
     float *d_bias;           // [n_tiles_n * block_n]
     CUtensorMap map_a, map_b, map_c;    // map_c: the hidden-activation buffer this layer stores to
     CUtensorMap map_b2;                 // W in 128-row boxes: one CTA's half of a 256-column tile
+    CUtensorMap map_m;                  // backward epilogue: the forward activations behind the ReLU mask (boxes like map_c)
 };
 
 }  // namespace im
@@ -1013,11 +1056,11 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
         prepared = true;
     }
     GemmParams gp = gp_in;
-    gp.stages = Plan::stages_for(Plan::hidden_epi_bytes());
-    const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
+    gp.stages = Plan::stages_for(Plan::hidden_epi_bytes(BWD));
+    const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes(BWD));
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N, false, BWD><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    linear_tc_hidden_kernel<BLOCK_N, false, BWD><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -1040,7 +1083,7 @@ cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm
     const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N, true><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, gp);
+    linear_tc_hidden_kernel<BLOCK_N, true><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -1051,13 +1094,13 @@ cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm,
     static bool prepared = false;
     if (!prepared) {
         cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kPairSmemBytes);
+                                             (int)pair_smem_bytes(BWD));
         if (e != cudaSuccess) return e;
         prepared = true;
     }
     const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-    linear_tc_hidden_pair_kernel<BWD><<<2 * pairs, kThreads, kPairSmemBytes, stream>>>(L.map_a, L.map_b2, L.map_c, gp);
+    linear_tc_hidden_pair_kernel<BWD><<<2 * pairs, kThreads, pair_smem_bytes(BWD), stream>>>(L.map_a, L.map_b2, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -1178,6 +1221,7 @@ im_status tc_policy_create(im_policy *p, const void *const *W, const float *cons
         // hidden layers store 32-row x 64-column slabs of their output buffer
         if (!last && !make_map(&L.map_c, tc->d_hidden[l & 1], mb, rows, (uint64_t)tc->ld_hidden, 32))
             return IM_ERR_CUDA;
+        L.map_m = L.map_c;               // the forward pass has no mask: a valid placeholder
     }
     return IM_OK;
 }
@@ -1279,6 +1323,8 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
         !make_map(&L.map_c, C, nb * (uint64_t)M, (uint64_t)N, (uint64_t)ldc, 32))
         return IM_ERR_CUDA;
     if (L.block_n == 256 && !make_map(&L.map_b2, B, nb * (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 128)) return IM_ERR_CUDA;
+    L.map_m = L.map_c;
+    if (mask && !make_map(&L.map_m, mask, (uint64_t)M, (uint64_t)N, (uint64_t)ld_mask, 32)) return IM_ERR_CUDA;
     GemmParams gp;
     std::memset(&gp, 0, sizeof(gp));
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
