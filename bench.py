@@ -385,22 +385,30 @@ def main():
                 rnd = lambda *sh: torch.randn(*sh, device=dev, generator=gen)
                 ub = dict(action=rnd(Mu, A) * 0.2, mean_old=rnd(Mu, A) * 0.2, log_std_old=torch.full((A,), -2.0, device=dev),
                           logp_old=rnd(Mu) + 60.0, advantage=rnd(Mu), value_old=rnd(Mu), returns=rnd(Mu))
+                for i in range(2):
+                    upd.update(Mu, ub)
+                stream.synchronize()
+                # the update's ~100 launches are replayed from one CUDA graph, as a training loop would run them
+                up_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(up_graph, stream=stream):
+                    upd.update(Mu, ub)
                 t_up = []
-                for i in range(2 + 5):
+                for i in range(1 + 5):
                     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     a.record(stream)
-                    upd.update(Mu, ub)
+                    up_graph.replay()
                     b.record(stream)
                     torch.cuda.synchronize()
-                    if i >= 2:
+                    if i >= 1:
                         t_up.append(a.elapsed_time(b) * 1e-3)
             t_up = float(np.median(t_up))
             up_flops = 3 * (mlp_flops_per_env(adims) + mlp_flops_per_env(cdims_u)) * Mu      # forward + two backward products
             extras["ppo_update"] = dict(rows=Mu, seconds_per_update=t_up, achieved_tflops=up_flops / t_up / 1e12,
                                         status=[actor_t.device_status(), critic_t.device_status()],
+                                        launch="cuda_graph",
                                         note="forward + backward + Adam of actor and critic on one minibatch; "
                                              "flops = 3 x forward flops")
-            del actor_t, critic_t, upd, ub
+            del up_graph, actor_t, critic_t, upd, ub
         if staged:
             cdims = tuple(wl.mlp_dims[:-1]) + (1,)
             cw = W.make_policy_weights(cdims, "bf16", wl.seed + 1)
