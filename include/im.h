@@ -443,7 +443,8 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   C_s[Mo][No] = sum over rows r of slice s of A[r][0..Mo) (x) B[r][0..No), for `slices` equal
  *   ranges of the R rows (R a multiple of 64 * slices), partial results stacked c_pitch rows apart
  *   (c_pitch >= Mo, a multiple of 128; rows Mo..c_pitch of a slice are written as zeros).  The
- *   tensor cores read both operands M/N-major.  No a multiple of 64; zeros: float [No] of zeros.
+ *   tensor cores read both operands M/N-major.  No a multiple of 64; zeros: DEVICE, non-NULL, kept for
+ *   call compatibility (the product has no bias and the buffer is not read).
  * im_gemm_bf16_f32out: C[M][N] float, dense = A[M][K] B[N][K]^T + bias, N <= 80; B and bias
  *   must hold ceil(N / 16) * 16 rows / floats (the extra ones zero).
  * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.

@@ -411,15 +411,20 @@ __device__ __forceinline__ void hidden_chunk(const GemmParams &P, uint32_t t_add
     tmem_ld32_issue(t_addr, v);
     tmem_ld32_issue(t_addr + 32u, v + 32);
     tmem_ld_wait();
-    const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + col0);
     const float fl = P.act_floor;          // 0: ReLU; -inf: linear output
+    if (P.bias) {
+        const float4 *b4 = reinterpret_cast<const float4 *>(P.bias + col0);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const float4 b = __ldg(b4 + i);
-        v[4 * i] = fmaxf(v[4 * i] + b.x, fl);
-        v[4 * i + 1] = fmaxf(v[4 * i + 1] + b.y, fl);
-        v[4 * i + 2] = fmaxf(v[4 * i + 2] + b.z, fl);
-        v[4 * i + 3] = fmaxf(v[4 * i + 3] + b.w, fl);
+        for (int i = 0; i < 16; ++i) {
+            const float4 b = __ldg(b4 + i);
+            v[4 * i] = fmaxf(v[4 * i] + b.x, fl);
+            v[4 * i + 1] = fmaxf(v[4 * i + 1] + b.y, fl);
+            v[4 * i + 2] = fmaxf(v[4 * i + 2] + b.z, fl);
+            v[4 * i + 3] = fmaxf(v[4 * i + 3] + b.w, fl);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) v[i] = fmaxf(v[i], fl);
     }
     if (BWD) {
 #pragma unroll
@@ -1354,8 +1359,11 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
     }
     TcLayer L;
     L.N = No; L.K = R / slices; L.Kpad = L.K;
-    L.block_n = pick_block_n(No, false);
-    L.n_tiles_n = No / L.block_n;
+    // wide outputs take 256-column tiles even when that leaves a ragged last tile (640 columns: three tiles,
+    // a sixth of the MMAs wasted, against five 128-column tiles at little more than half the tensor-pipe rate);
+    // TMA fills the operand columns past No with zeros and clips the stores
+    L.block_n = No > 256 ? 256 : pick_block_n(No, false);
+    L.n_tiles_n = (No + L.block_n - 1) / L.block_n;
     L.d_W = nullptr; L.d_bias = nullptr;
     if (!make_map(&L.map_a, A, (uint64_t)R, (uint64_t)Mo, (uint64_t)lda, 64) ||
         !make_map(&L.map_b, B, (uint64_t)R, (uint64_t)No, (uint64_t)ldb, 64) ||
@@ -1363,7 +1371,8 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
         return IM_ERR_CUDA;
     GemmParams gp;
     std::memset(&gp, 0, sizeof(gp));
-    gp.M = Mo; gp.N = No; gp.K_blocks = (R / slices) / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
+    gp.M = Mo; gp.N = No; gp.K_blocks = (R / slices) / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = nullptr;    // no bias in this product
+    (void)bias;
     gp.act_floor = -INFINITY;
     gp.n_batches = slices; gp.a_batch_rows = R / slices; gp.b_batch_rows = 0; gp.c_batch_rows = c_pitch;
     gp.status = status;

@@ -281,7 +281,7 @@ def test_whole_training_iteration_runs_from_one_cuda_graph():
 
 
 @pytest.mark.parametrize("R,Mo,No,slices", [(128, 64, 64, 1), (256, 128, 128, 2), (1024, 200, 256, 4), (512, 69, 512, 2),
-                                             (2048, 1024, 640, 4)])
+                                             (2048, 1024, 640, 4), (512, 128, 320, 2)])
 def test_transposed_product_reads_both_operands_in_place(R, Mo, No, slices):
     """A^T B of two row-major bf16 matrices on the tensor cores (operands M/N-major), per row slice."""
     g = np.random.default_rng(R + Mo)
