@@ -111,6 +111,30 @@ __global__ void __launch_bounds__(256) to_bf16_padded_kernel(const float *__rest
     }
 }
 
+// The same with 16-byte stores: a thread converts eight consecutive columns of one row (ld_out a multiple of 8,
+// out 16-byte aligned); its eight loads are 32 consecutive bytes, a warp's one contiguous kilobyte of the row.
+__global__ void __launch_bounds__(256) to_bf16_padded_vec_kernel(const float *__restrict__ in, long long ld_in, int rows, int cols,
+                                                                 __nv_bfloat16 *__restrict__ out, int ld_out)
+{
+    const int gpr = ld_out >> 3;                                   // 8-column groups per row
+    const long long total = (long long)rows * gpr;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / gpr;
+        const int c = (int)(i - r * gpr) << 3;
+        const float *src = in + r * ld_in + c;
+        float v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = c + j < cols ? __ldg(src + j) : 0.0f;
+        uint4 o;
+        __nv_bfloat162 h;
+        h = __floats2bfloat162_rn(v[0], v[1]); o.x = *reinterpret_cast<const uint32_t *>(&h);
+        h = __floats2bfloat162_rn(v[2], v[3]); o.y = *reinterpret_cast<const uint32_t *>(&h);
+        h = __floats2bfloat162_rn(v[4], v[5]); o.z = *reinterpret_cast<const uint32_t *>(&h);
+        h = __floats2bfloat162_rn(v[6], v[7]); o.w = *reinterpret_cast<const uint32_t *>(&h);
+        *reinterpret_cast<uint4 *>(out + r * ld_out + c) = o;
+    }
+}
+
 // out[r][c] (float, dense [rows][cols]) = in[r][c] (bf16, row stride ld_in).
 __global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *__restrict__ in, long long ld_in, int rows,
                                                           int cols, float *__restrict__ out)
@@ -413,11 +437,16 @@ im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, in
 {
     using namespace im;
     if (!in || !out || rows < 1 || cols < 1 || ld_in < cols || ld_out < cols) return IM_ERR_INVALID_ARG;
-    const long long total = (long long)rows * ld_out;
+    const bool vec = (ld_out & 7) == 0 && al16(out);
+    const long long total = vec ? (long long)rows * (ld_out >> 3) : (long long)rows * ld_out;
     long long g = (total + 255) / 256;
     const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
-    to_bf16_padded_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(in, ld_in, rows, cols,
-                                                                       reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    if (vec)
+        to_bf16_padded_vec_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(in, ld_in, rows, cols,
+                                                                               reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
+    else
+        to_bf16_padded_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(in, ld_in, rows, cols,
+                                                                           reinterpret_cast<__nv_bfloat16 *>(out), ld_out);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }

@@ -42,6 +42,13 @@ def test_building_blocks_against_plain_definitions():
     p = torch.full((70, 128), 7.0, dtype=torch.bfloat16, device="cuda")
     B.f32_to_bf16_padded(f, p)
     assert torch.equal(p[:, :69], f.to(torch.bfloat16)) and (p[:, 69:] == 0).all()
+    q = torch.full((70, 124), 7.0, dtype=torch.bfloat16, device="cuda")       # row stride not a multiple of 8: scalar kernel
+    B.f32_to_bf16_padded(f, q)
+    assert torch.equal(q[:, :69], f.to(torch.bfloat16)) and (q[:, 69:] == 0).all()
+    wide = torch.randn((3001, 577), device="cuda", generator=g)
+    pw = torch.full((3001, 640), 7.0, dtype=torch.bfloat16, device="cuda")
+    B.f32_to_bf16_padded(wide, pw)
+    assert torch.equal(pw[:, :577], wide.to(torch.bfloat16)) and (pw[:, 577:] == 0).all()
     back = torch.empty((70, 69), device="cuda")
     B.bf16_to_f32(p[:, :69], back)
     assert torch.equal(back, f.to(torch.bfloat16).float())
