@@ -7,7 +7,8 @@ arithmetic step runs in the CUDA library:
     backward   dZ_L           im_f32_to_bf16_padded(dL/d output)            db_L  im_colsum_f32
                per layer      im_gemm_bf16_tn -> partial dW per row slice (bf16, operands read in place),
                               im_sum_slices_bf16_to_f32 -> dW
-                              im_gemm_bf16 with W^T -> dH, im_relu_mask_bf16 -> dZ_{l-1}, im_colsum_bf16 -> db
+                              im_gemm_bf16_dgrad with W^T -> dZ_{l-1} = (H > 0) * (dZ W) and its 32-row column
+                              sums (both in the product's epilogue), im_colsum_f32 of those -> db_{l-1}
     step       im_grad_scale (global norm), im_adam_step per tensor (writes the bf16 weights in place),
                im_transpose_bf16 refreshes W^T
 
@@ -255,3 +256,34 @@ def update_from_storage(upd: PpoUpdater, storage, epochs: int, n_minibatches: in
                     B.gather_rows(src, idx, g[name][:M], upd.actor.status, st)
                 batch = {name: g[name][:M] for name in g}
             upd.update(M, dict(batch, log_std_old=upd.log_std_old))
+
+
+def _main():
+    """python -m paper_2609_09821_b200.trainer [--rows M] [--passes P] [--dims 577 1024 1024 512 69]:
+    forward + backward of one MLP on M random rows, P times; prints the time of the last pass."""
+    import argparse
+    from . import workloads as W
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--rows", type=int, default=65536)
+    ap.add_argument("--passes", type=int, default=2)
+    ap.add_argument("--dims", type=int, nargs="+", default=[577, 1024, 1024, 512, 69])
+    a = ap.parse_args()
+    dims, M = tuple(a.dims), a.rows
+    w = W.make_policy_weights(dims, "bf16", 1)
+    tr = MlpTrainer(dims, w["W"], w["b"], M)
+    gen = torch.Generator(device="cuda").manual_seed(0)
+    rows = tr.input_rows(M)
+    rows.zero_()
+    rows[:, :dims[0]] = torch.randn((M, dims[0]), device="cuda", generator=gen).to(torch.bfloat16)
+    d_out = torch.randn((M, dims[-1]), device="cuda", generator=gen) / M
+    for _ in range(a.passes):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(tr.stream); tr.forward(M)
+        e[1].record(tr.stream); tr.backward(d_out, M)
+        e[2].record(tr.stream); torch.cuda.synchronize()
+    print("rows %d dims %s: forward %.3f ms, backward %.3f ms, device status %d"
+          % (M, "-".join(map(str, dims)), e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2]), tr.device_status()))
+
+
+if __name__ == "__main__":
+    _main()
