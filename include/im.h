@@ -466,7 +466,7 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   into the buffer im_policy_layer_buffers returns).
  * im_bf16_to_f32: out (float, dense [rows][cols]) = in (bf16, row stride ld_in).
  * im_colsum_f32 / im_colsum_bf16: out[c] = sum_r x[r][c], float [cols]; rows are summed in
- *   fp32 within slices of 256 rows and the slices in order in fp64 (bit-reproducible);
+ *   fp32 within slices of 256 rows and the slices in a fixed order in fp64 (bit-reproducible);
  *   workspace DEVICE, at least ceil(rows / 256) * cols * 4 bytes. */
 im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
                        int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu, uint32_t *status,

@@ -63,9 +63,14 @@ class MlpTrainer:
         self.H += [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl - 1)]
         self.out = torch.zeros((Mb, self.dims[-1]), dtype=f32, device=dev)
         self.dZ = [torch.zeros((Mb, self.Np[l]), dtype=bf, device=dev) for l in range(self.nl)]
-        self.max_split = 16                                                 # most slices of the batch dimension in a dW GEMM
-        np128 = (max(self.Np) + 127) // 128 * 128
-        self.dWs = torch.zeros((self.max_split * np128, max(self.Kp)), dtype=bf, device=dev)
+        self.max_split = 64                                                 # most slices of the batch dimension in a dW GEMM
+        # partial dW products of one layer: room for the most slices _dw_slices can choose
+        need = 0
+        for l in range(self.nl):
+            npb = (self.Np[l] + 127) // 128 * 128
+            s_max = self._dw_slices(l, self.Mb, any_rows=True)     # more rows never favour fewer slices
+            need = max(need, s_max * npb * self.Kp[l])
+        self.dWs = torch.zeros(need, dtype=bf, device=dev)
         self.zeros = torch.zeros(max(self.Kp + self.Np), dtype=f32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.colsum_ws = torch.empty(((Mb + 255) // 256) * max(self.Np), dtype=f32, device=dev)
@@ -74,6 +79,22 @@ class MlpTrainer:
         with torch.cuda.stream(self.stream):
             for l in range(self.nl):
                 B.transpose_bf16(self.Wb[l], self.WbT[l], self.stream)
+
+    def _dw_slices(self, l: int, M: int, any_rows: bool = False) -> int:
+        """Row slices of the dW product of layer l on M rows: dW contracts over the batch (a long sum feeding
+        few output tiles), so the rows are cut into S slices that run as one launch.  S is the power of two
+        (slices of whole 128-row blocks) with the least modelled time: waves of tiles on 148 SMs times rows per
+        slice (5 ns per row and wave, measured on the 1024 x 1024 layer), plus the pass that adds the S
+        partial products (1 ps per element).  any_rows: ignore the divisibility rule (an upper bound for sizing)."""
+        npb = (self.Np[l] + 127) // 128 * 128
+        tiles = (npb // 128) * max(1, (self.Kp[l] + 255) // 256)
+        best, best_cost, S = 1, None, 1
+        while S <= self.max_split and (any_rows or M % (128 * S) == 0):
+            cost = 5e-9 * M * -(-tiles * S // 148) / S + 1e-12 * S * npb * self.Kp[l]
+            if best_cost is None or cost < best_cost * (1.0 - 1e-9):
+                best, best_cost = S, cost
+            S *= 2
+        return best
 
     # -- forward ---------------------------------------------------------------
     def input_rows(self, M: int) -> torch.Tensor:
@@ -104,16 +125,11 @@ class MlpTrainer:
         for l in range(L, -1, -1):
             N, K, Np, Kp = self.dims[l + 1], self.dims[l], self.Np[l], self.Kp[l]
             dZ = self.dZ[l][:M]
-            # dW = dZ^T H contracts over the batch rows: a long sum feeding few output tiles.  The rows are
-            # cut into S slices that run as one launch (S times the tiles, enough to fill the machine)
-            # and the S partial products are added afterwards.  im_gemm_bf16_tn reads dZ and H as they
-            # are (M/N-major tensor-core operands): no transposed copies.
+            # dW = dZ^T H over S row slices in one launch (im_gemm_bf16_tn reads dZ and H as they are, M/N-major
+            # tensor-core operands: no transposed copies); the S partial products are added afterwards
             Npb = (Np + 127) // 128 * 128
-            tiles = (Npb // 128) * max(1, Kp // 256)
-            S = 1
-            while S < self.max_split and tiles * S < 148 and M % (128 * S) == 0:
-                S *= 2
-            dWs = self.dWs.view(-1)[:S * Npb * Kp].view(S * Npb, Kp)
+            S = self._dw_slices(l, M)
+            dWs = self.dWs[:S * Npb * Kp].view(S * Npb, Kp)
             B.gemm_bf16_tn(dZ, self.H[l][:M], dWs, S, Npb, self.zeros, self.status, st)
             B.sum_slices_bf16_to_f32(dWs, S, N, K, self.dW[l], st)
             if l > 0:
