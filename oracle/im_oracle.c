@@ -364,6 +364,15 @@ typedef struct {
     const uint64_t *reset_cdf;      /* [C*B] exclusive upper thresholds in [0, 2^32], see orc_reset_cdf */
     uint32_t *stat_starts;          /* [C*B] episodes started in the bin (or NULL) */
     uint32_t *stat_failures;        /* [C*B] early terminations that happened in the bin (or NULL) */
+    /* extended observation (Section 6: "future reference end-effector frames, and the previous action"), appended
+     * after the 24J+1 entries; zero fields switch it off:
+     *   n_future F > 1: for f = 2..F and each end effector in body order, position (3) and first and third
+     *     rotation column (3 + 3) of the reference at min(t + f dt, D_clip), seen from the observed root's heading frame
+     *   act_dim A > 0: the A entries of prev_action[i] (zeros for an env that was just reset) */
+    int32_t n_future;
+    int32_t act_dim;
+    const float *prev_action;       /* [n][ld_action] */
+    int64_t ld_action;
 } orc_env_config;
 
 /* Cumulative table of a weight table w[n] >= 0 (not all zero): T_i = floor(2^32 (w_0 + .. + w_i) / total)
@@ -561,7 +570,7 @@ static void ref_to_state(const orc_skeleton *s, const orc_ref *r, orc_body_state
 
 /* Step a6: heading-local observation of state x at (clip, t), D = 24J + 1. */
 static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg,
-                      const orc_body_state *x, int clip, float t, double *obs)
+                      const orc_body_state *x, int clip, float t, double *obs, int i, int was_reset)
 {
     int J = s->J;
     const double ex[3] = {1.0, 0.0, 0.0}, ez[3] = {0.0, 0.0, 1.0};
@@ -596,6 +605,30 @@ static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_
         orc_quat_rotate(ql, ex, o + 3);
         orc_quat_rotate(ql, ez, o + 6);
     }
+
+    /* extended entries */
+    double *o = obs + 24 * J + 1;
+    for (int f = 2; f <= cfg->n_future; ++f) {
+        volatile float ahead = (float)f * cfg->dt;          /* one fp32 multiplication, */
+        volatile float t_f = t + ahead;                      /* one fp32 addition        */
+        float t_c = t_f < cl->dur[clip] ? t_f : cl->dur[clip];
+        orc_ref fut;
+        orc_reference_state(s, cl, clip, t_c, &fut);
+        for (int j = 0; j < J; ++j) {
+            int is_ee = 0;
+            for (int k = 0; k < s->n_ee; ++k) is_ee |= (s->ee[k] == j);
+            if (!is_ee) continue;
+            double d[3], ql[4];
+            for (int c = 0; c < 3; ++c) d[c] = fut.p[j][c] - origin[c];
+            orc_quat_rotate(qh_inv, d, o + 0);
+            orc_quat_mul(qh_inv, fut.q[j], ql);
+            orc_quat_rotate(ql, ex, o + 3);
+            orc_quat_rotate(ql, ez, o + 6);
+            o += 9;
+        }
+    }
+    for (int a = 0; a < cfg->act_dim; ++a)
+        *o++ = was_reset ? 0.0 : (double)cfg->prev_action[(int64_t)i * cfg->ld_action + a];
 }
 
 static void load_sim(const orc_skeleton *s, const float *pos, const float *quat, const float *lin,
@@ -641,7 +674,7 @@ void orc_env_reset_all(const orc_skeleton *s, const orc_clips *cl, const orc_env
         orc_reference_state(s, cl, clip_id[i], t[i], &r);
         orc_reset_noise(s, cfg, env_ids[i], step, &r);
         ref_to_state(s, &r, &x);
-        build_obs(s, cl, cfg, &x, clip_id[i], t[i], obs + (int64_t)i * ld_obs);
+        build_obs(s, cl, cfg, &x, clip_id[i], t[i], obs + (int64_t)i * ld_obs, i, 1);
     }
 }
 
@@ -700,7 +733,7 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
         }
         clip_id[i] = clip;
         t[i] = t_cur;
-        build_obs(s, cl, cfg, &x, clip, t_cur, obs + (int64_t)i * ld_obs);   /* a6 */
+        build_obs(s, cl, cfg, &x, clip, t_cur, obs + (int64_t)i * ld_obs, i, flags[i] != 0);   /* a6 */
     }
 }
 

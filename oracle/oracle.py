@@ -40,7 +40,8 @@ class EnvConfig(C.Structure):
     _fields_ = [("dt", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32),
                 ("reward", RewardConfig), ("write_back_reset", C.c_int32), ("grace_steps", C.c_int32),
                 ("reset_noise_std", C.c_float), ("n_bins", C.c_int32), ("reset_cdf", C.c_void_p),
-                ("stat_starts", C.c_void_p), ("stat_failures", C.c_void_p)]
+                ("stat_starts", C.c_void_p), ("stat_failures", C.c_void_p),
+                ("n_future", C.c_int32), ("act_dim", C.c_int32), ("prev_action", C.c_void_p), ("ld_action", C.c_int64)]
 
 
 _lib = None
@@ -183,6 +184,10 @@ class Skeleton:
         off = np.ascontiguousarray(offsets, np.float32)
         m = None if masses is None else np.ascontiguousarray(masses, np.float32)
         ee = None if ee_ids is None else np.ascontiguousarray(ee_ids, np.int32)
+        # end effectors: the given bodies, else the bodies without children
+        self.ee_ids = sorted(int(e) for e in ee) if ee is not None else \
+            [j for j in range(self.J) if j not in set(int(p) for p in self.parents)]
+        self.n_ee = len(self.ee_ids)
         self.h = lib().orc_skeleton_create(self.J, _p(self.parents), _p(off), _p(m), _p(ee),
                                            0 if ee is None else int(ee.shape[0]))
         if not self.h:
@@ -263,6 +268,21 @@ class Env:
         self.cfg.reset_cdf = self.reset_cdf.ctypes.data
         self.cfg.stat_starts = self.stat_starts.ctypes.data
         self.cfg.stat_failures = self.stat_failures.ctypes.data
+
+    def set_obs_extension(self, n_future: int = 1, prev_action: Optional[np.ndarray] = None) -> int:
+        """Extended observation: end-effector targets of reference frames 2 .. n_future, then the previous action
+        (fp32 [n, A]; the array is read by later steps, so the caller updates it in place).  Returns the width."""
+        self.prev_action = None if prev_action is None else prev_action
+        A = 0
+        if prev_action is not None:
+            assert prev_action.dtype == np.float32 and prev_action.shape[0] == self.n and prev_action.flags.c_contiguous
+            A = prev_action.shape[1]
+            self.cfg.prev_action = prev_action.ctypes.data
+            self.cfg.ld_action = A
+        self.cfg.n_future = int(n_future)
+        self.cfg.act_dim = A
+        self.D = 24 * self.skel.J + 1 + (int(n_future) - 1) * 9 * self.skel.n_ee + A
+        return self.D
 
     def reset_all(self, step: int = 0) -> np.ndarray:
         obs = np.zeros((self.n, self.D))
