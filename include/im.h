@@ -222,6 +222,22 @@ im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim
 im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_len);
 im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, const int32_t *ep_len);
 
+/* ---- extended observation ---------------------------------------------------
+ * (Section 6: observations also hold "future reference end-effector frames, and the
+ * previous action"; the paper gives no layout, this one appends to the 24J+1 row.)
+ *   columns [24J+1, 24J+1 + (n_future-1) * 9 * n_ee):  for each further reference frame
+ *       f = 2 .. n_future, at time min(fl32(t + fl32(f * dt)), D_clip), and each end effector
+ *       in body order: position (3), first and third column of the rotation (3 + 3), seen
+ *       from the heading frame of the observed root exactly like the frame-1 targets
+ *   then act_dim columns: prev_action[env][0..act_dim), the action the policy took before
+ *       this step (DEVICE float [n_envs][ld_action], read by every later step: the caller
+ *       keeps it alive and fills it, normally with the policy's action output); zeros for
+ *       an env that this step reset, and after im_env_reset_all.
+ * n_future = 1 and act_dim = 0 restore the 24J+1 layout.  ld_obs must hold the extended
+ * row, else IM_ERR_INVALID_ARG; a policy attached for another width is detached.  Takes
+ * effect with the next launch (host state only).  im_step_host does not support act_dim > 0. */
+im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim, const float *prev_action, int32_t ld_action);
+
 /* ---- adaptive episode initialisation --------------------------------------
  * (The paper trains "with early termination and adaptive episode-initialization
  * sampling", Section 6, without giving the rule; this is the mechanism such rules

@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension",
 ]
 
 
@@ -141,6 +141,7 @@ def load():
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp, vp]
         L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
         L.im_copy_f32.argtypes = [vp, vp, i64, vp]
@@ -188,6 +189,8 @@ class Skeleton:
         m = _np(masses, np.float32)
         ee = _np(ee_ids, np.int32)
         self.J = int(par.shape[0])
+        # end effectors: the given bodies, else the leaves of the tree
+        self.n_ee = int(ee.shape[0]) if ee is not None else self.J - len(set(int(x) for x in par if x >= 0))
         self.h = C.c_void_p()
         _check(L.im_create_skeleton(self.J, _ptr(par), _ptr(off), _ptr(m), _ptr(ee),
                                     0 if ee is None else int(ee.shape[0]), C.byref(self.h)), "im_create_skeleton")
@@ -299,6 +302,19 @@ class Env:
             raise ValueError("weights must be [n_clips, n_bins]")
         _check(load().im_env_set_reset_bins(self.h, int(n_bins), _ptr(w)), "im_env_set_reset_bins")
         self.n_bins = int(n_bins)
+
+    def set_obs_extension(self, n_future: int = 1, prev_action=None):
+        """Extended observation: end-effector targets of reference frames 2 .. n_future and the previous action
+        (a float32 CUDA tensor [n, A] that later steps read; kept alive here).  Returns the observation width."""
+        if prev_action is not None and (prev_action.dim() != 2 or prev_action.shape[0] < self.n or prev_action.stride(1) != 1):
+            raise ValueError("prev_action must be a [n, A] tensor with contiguous rows")
+        A = 0 if prev_action is None else prev_action.shape[1]
+        _check(load().im_env_set_obs_extension(self.h, int(n_future), A, _ptr(prev_action) if A else None,
+                                               prev_action.stride(0) if A else 0), "im_env_set_obs_extension")
+        self._prev_action = prev_action
+        self.n_future = int(n_future)
+        self.D = 24 * self.J + 1 + (int(n_future) - 1) * 9 * self.skel.n_ee + A
+        return self.D
 
     def reset_stats(self, clear: bool = False):
         """(starts, failures) per (clip, phase bin) as CUDA int32 tensors [C, n_bins] (uint32 counts)."""

@@ -43,9 +43,9 @@ __host__ __device__ inline int tile_stride(int D)
 // up to a multiple of four columns so that both halves start on a 16-byte boundary.
 __host__ __device__ inline int split_col(int J) { return (15 * J + 3) / 4 * 4; }
 
-__host__ __device__ inline size_t smem_floats(int J, int n_chains)
+__host__ __device__ inline size_t smem_floats(int J, int n_chains, int extra_cols)
 {
-    const int D = 24 * J + 1, c1 = split_col(J);
+    const int D = 24 * J + 1 + extra_cols, c1 = split_col(J);
     const int s1 = tile_stride(c1), s2 = tile_stride(D - c1);
     return (size_t)kTile * (s1 > s2 ? s1 : s2) + (size_t)kPartials * n_chains * kTile;
 }
@@ -324,7 +324,11 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     const int J = sk.J;
     const int D = 24 * J + 1;
     const int c1 = split_col(J);                    // multiple of 4
-    const int S1 = tile_stride(c1), S2 = tile_stride(D - c1);
+    // extended observation: end-effector targets of further future frames, then the previous action
+    const int n_ee = OPT ? __popc(sk.ee_mask) : 0;
+    const int ext_future = (OPT && P.n_future > 1) ? (P.n_future - 1) * 9 * n_ee : 0;
+    const int D_ext = D + ext_future + (OPT ? P.act_dim : 0);
+    const int S1 = tile_stride(c1), S2 = tile_stride(D_ext - c1);
     const int C = sk.n_chains;
     const int lane = threadIdx.x & 31;
     const int c = threadIdx.x >> 5;                 // this thread's chain
@@ -594,7 +598,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     //      into the second half (which reuses the shared memory of the first)
     {
         if (c == 0) {
-            for (int i = D - c1; i < S2; ++i) row2[i] = 0.0f;
+            for (int i = D_ext - c1; i < S2; ++i) row2[i] = 0.0f;
             if (15 * J >= c1) row2[15 * J - c1] = phase;
         }
         KeyPair keys = ld_keys(rt0, rt1, sk.chain[c][0]);
@@ -619,6 +623,37 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                         if (col + i >= c1) row2[col + i - c1] = o[i];
                 }
             }
+        }
+        if (OPT && D_ext > D) {
+            // frames f = 2 .. n_future of the reference, t + f dt (two fp32 operations, clamped to the clip's end):
+            // every chain walks them again and the owner of an end effector writes its nine entries
+            for (int f = 2; f <= P.n_future; ++f) {
+                const float t_f = fminf(__fadd_rn(t_cur, __fmul_rn((float)f, P.dt)), cmc.dur);
+                int frame_f;
+                float alpha_f;
+                lookup(cmc, t_f, frame_f, alpha_f);
+                const float4 *rf0 = P.frames + (size_t)frame_f * RS, *rf1 = rf0 + RS;
+                Walk sf;
+                for (int k = 0; k < len; ++k) {
+                    const int b = sk.chain[c][k];
+                    const KeyPair kp = ld_keys(rf0, rf1, b);
+                    Quat ql;
+                    Vec3 wl;
+                    joint_step<false>(sk, rf0, rf1, as_quat(kp.a), as_quat(kp.b), alpha_f, cmc.fps, b, k, sf, ql, wl);
+                    if (k >= first_own && ((sk.ee_mask >> b) & 1u)) {
+                        const Vec3 tp = H.turn(Vec3{sf.p.x - H.ox, sf.p.y - H.oy, sf.p.z});
+                        const Vec3 tt = H.turn(qcol_x(sf.q)), tm = H.turn(qcol_z(sf.q));
+                        const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
+                        float *dst = row2 + (D - c1) + ((f - 2) * n_ee + __popc(sk.ee_mask & ((1u << b) - 1u))) * 9;
+#pragma unroll
+                        for (int i = 0; i < 9; ++i) dst[i] = o[i];
+                    }
+                }
+            }
+            // the action the policy took before this step; an env that was just reset has none
+            float *dst = row2 + (D - c1) + ext_future;
+            for (int j = c; j < P.act_dim; j += C)
+                dst[j] = (reset || !valid) ? 0.0f : __ldg(P.prev_action + (size_t)env * P.ld_action + j);
         }
     }
     __syncthreads();
@@ -673,7 +708,7 @@ void launch_one(const EnvKernelParams &p, dim3 grid, dim3 block, size_t smem, cu
 
 }  // namespace
 
-size_t env_kernel_smem_bytes(int J, int n_chains) { return smem_floats(J, n_chains) * sizeof(float); }
+size_t env_kernel_smem_bytes(int J, int n_chains, int extra_cols) { return smem_floats(J, n_chains, extra_cols) * sizeof(float); }
 
 cudaError_t env_kernel_prepare(size_t smem)
 {
@@ -690,7 +725,7 @@ cudaError_t env_kernel_prepare(size_t smem)
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
-    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0;
+    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0 || p.n_future > 1 || p.act_dim > 0;
     if (opt) {
         if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
         else launch_one<false, true>(p, grid, block, smem, stream);

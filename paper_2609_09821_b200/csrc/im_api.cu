@@ -188,7 +188,8 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     if (!e) return IM_ERR_ALLOC;
     std::memset(e, 0, sizeof(*e));
     e->skel = skel; e->clips = clips; e->cfg = *cfg; e->stream = (cudaStream_t)cuda_stream; e->D = D;
-    e->smem_bytes = env_kernel_smem_bytes(J, skel->dev.n_chains);
+    e->smem_bytes = env_kernel_smem_bytes(J, skel->dev.n_chains, 0);
+    e->n_future = 1;
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -246,6 +247,10 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.reset_cdf = e->d_reset_cdf;
     p.stat_starts = e->d_stat_starts;
     p.stat_failures = e->d_stat_failures;
+    p.n_future = e->n_future;
+    p.act_dim = e->act_dim;
+    p.prev_action = e->prev_action;
+    p.ld_action = e->ld_action;
     p.step = step;
     p.clip_id = e->d_clip_id;
     p.t = e->d_t;
@@ -297,6 +302,7 @@ static im_status env_step_range(im_env *e, uint32_t step, const im_body_state *s
     p.obs = obs_out + (size_t)first * e->cfg.ld_obs;
     if (p.obs_bf16) p.obs_bf16 += (size_t)first * e->cfg.ld_obs;
     p.reward_out = reward_out + first; p.flags_out = flags_out + first; p.terms_out = nullptr;
+    if (p.prev_action) p.prev_action += (size_t)first * p.ld_action;
     IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
     return IM_OK;
 }
@@ -490,6 +496,27 @@ im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n, float
 }
 
 /* ------------------------------------------------------------------ adaptive episode initialisation */
+im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim, const float *prev_action, int32_t ld_action)
+{
+    if (!e || n_future < 1 || n_future > 16 || act_dim < 0 || act_dim > 1024) return IM_ERR_INVALID_ARG;
+    if (act_dim > 0 && (!prev_action || ld_action < act_dim)) return IM_ERR_INVALID_ARG;
+    const int J = e->skel->dev.J;
+    const int extra = (n_future - 1) * 9 * e->skel->n_ee + act_dim;
+    const int D = 24 * J + 1 + extra;
+    if (e->cfg.ld_obs < D) return IM_ERR_INVALID_ARG;
+    const size_t smem = env_kernel_smem_bytes(J, e->skel->dev.n_chains, extra);
+    int dev = 0, max_smem = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if ((int64_t)smem > (int64_t)max_smem) return IM_ERR_UNSUPPORTED;
+    e->n_future = n_future; e->act_dim = act_dim; e->prev_action = act_dim > 0 ? prev_action : nullptr;
+    e->ld_action = act_dim > 0 ? ld_action : 0;
+    if (D != e->D) e->d_obs_bf16 = nullptr;            // a policy attached for another width no longer fits
+    e->D = D;
+    e->smem_bytes = smem;
+    return IM_OK;
+}
+
 im_status im_env_set_reset_bins(im_env *e, int32_t n_bins, const float *weights)
 {
     if (!e || n_bins < 0 || (n_bins > 0 && !weights)) return IM_ERR_INVALID_ARG;
@@ -610,6 +637,7 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
 {
     if (!e || !p || !sim_host || !action_host || !reward_host || !flags_host) return IM_ERR_INVALID_ARG;
     if (p->stream != e->stream || p->cfg.max_batch < e->cfg.n_envs || p->cfg.dims[0] != e->D) return IM_ERR_INVALID_ARG;
+    if (e->act_dim > 0) return IM_ERR_UNSUPPORTED;     // the caller-owned previous-action buffer belongs to the device path
     const int A = p->cfg.dims[p->nl];
     if (!e->d_obs) return IM_ERR_INVALID_ARG;          // im_env_reset_all_host has not run
     im_status s = ensure_staging(e, A);

@@ -53,6 +53,11 @@ struct EnvKernelParams {
     int32_t n_bins;                          // adaptive initialisation: phase bins per clip (0: uniform draw)
     const unsigned long long *reset_cdf;     // [C * n_bins] exclusive upper thresholds in [0, 2^32]
     uint32_t *stat_starts, *stat_failures;   // [C * n_bins]
+    // extended observation (0 / null: the 24J+1 layout)
+    int32_t n_future;                        // reference frames ahead whose end-effector targets are observed (>= 1)
+    int32_t act_dim;                         // previous-action entries
+    const float *prev_action;                // [N][ld_action]
+    int32_t ld_action;
     uint32_t step;
     // per-env state
     int32_t *clip_id;
@@ -97,12 +102,14 @@ struct im_env {
     float *d_t;
     int32_t *d_ep_len;
     uint32_t *d_status;
-    int D;                 // 24J + 1
+    int D;                 // observation width: 24J + 1 plus the extension columns
     size_t smem_bytes;
     uint16_t *d_obs_bf16;  // attached policy's bf16 input rows (null when detached)
     int32_t n_bins;        // adaptive initialisation (0: off)
     unsigned long long *d_reset_cdf;
     uint32_t *d_stat_starts, *d_stat_failures;
+    int32_t n_future, act_dim, ld_action;   // extended observation (im_env_set_obs_extension); D is the extended width
+    const float *prev_action;
     // staging for the *_host entry points (allocated on first use)
     float *d_aos_sim;      // component rows gathered from array-of-structures inputs (allocated on first use)
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;
@@ -114,7 +121,7 @@ struct im_env {
 
 // Launchers implemented in the kernel translation units.
 namespace im {
-size_t env_kernel_smem_bytes(int J, int n_chains);
+size_t env_kernel_smem_bytes(int J, int n_chains, int extra_cols);
 cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
 // simulator-native (array of structures) body states <-> component rows [13 J][stride]

@@ -68,6 +68,10 @@ def collect(env: B.Env, actor: B.Policy, critic: Optional[B.Policy], storage: Ro
             actor.forward(s, obs, st.mean[t], st.action[t], st.logp[t])
             if critic is not None:
                 critic.value_forward(obs, st.value[t].unsqueeze(1))
+        if getattr(env, "_prev_action", None) is not None:
+            # extended observation: the next row's previous-action entries are this step's actions (host state
+            # only; the pointer travels with the launch, so a captured graph keeps one per step)
+            env.set_obs_extension(env.n_future, st.action[t])
         env.step(s, sim_of_step(s), st.obs_row(t + 1), st.reward[t], st.flags[t])
     if critic is not None:
         last = st.obs_row(T)

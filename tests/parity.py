@@ -87,13 +87,15 @@ class Pair:
 
     def __init__(self, scene: Scene, n: int, reward=W.REWARD_MULT, seed=None, h_min=None, r_min=-np.inf,
                  write_back=False, env_base=0, ld_obs=None, stride_pad=0, with_policy=True, policy_impl=0,
-                 policy_sample=None, want_terms=True, obs_atol=OBS_ATOL, grace_steps=0, reset_noise_std=0.0):
+                 policy_sample=None, want_terms=True, obs_atol=OBS_ATOL, grace_steps=0, reset_noise_std=0.0,
+                 n_future=1, prev_action_dim=0):
         wl = scene.wl
         self.scene, self.wl, self.n, self.J = scene, wl, n, scene.J
         self.seed = wl.seed if seed is None else seed
         self.h_min = wl.h_min if h_min is None else h_min
         self.r_min = r_min
-        self.D = 24 * self.J + 1
+        # extended observation: end-effector targets of further frames, previous action (with_policy must be off)
+        self.D = 24 * self.J + 1 + (n_future - 1) * 9 * scene.o_skel.n_ee + prev_action_dim
         self.ld_obs = ld_obs or B.padded_ld(self.D)
         self.stride = (n + stride_pad + 3) // 4 * 4        # rows of the body-state arrays stay 16-byte aligned
         self.obs_atol = obs_atol
@@ -107,6 +109,13 @@ class Pair:
         self.g_env = B.Env(scene.g_skel, scene.g_clips,
                            B.make_env_config(n, wl.dt, self.seed, reward, self.h_min, self.ld_obs, r_min,
                                              env_base, write_back, grace_steps, reset_noise_std))
+        self.prev_o = self.prev_g = None
+        if n_future > 1 or prev_action_dim > 0:
+            if prev_action_dim > 0:
+                self.prev_o = np.zeros((n, prev_action_dim), np.float32)
+                self.prev_g = torch.zeros((n, prev_action_dim + 3), device="cuda")[:, :prev_action_dim]   # padded rows
+            assert self.o_env.set_obs_extension(n_future, self.prev_o) == self.D
+            assert self.g_env.set_obs_extension(n_future, self.prev_g) == self.D
         self.obs_g = torch.full((n, self.ld_obs), float("nan"), device="cuda")
         self.reward_g = torch.empty(n, device="cuda")
         self.flags_g = torch.empty(n, dtype=torch.uint8, device="cuda")
@@ -232,6 +241,9 @@ class Pair:
         def consume(s, sim):
             if self.policy is not None and (s - 1) % policy_every == 0:
                 self.policy_step(s)
+            if self.prev_o is not None:                 # stand-in for the policy's action of this step, same on both sides
+                self.prev_o[:] = np.random.default_rng(1000 + s).standard_normal(self.prev_o.shape).astype(np.float32)
+                self.prev_g.copy_(torch.from_numpy(self.prev_o))
             hist.append(self.env_step(s, sim))
 
         W.rollout_inputs(self.wl, self.scene.skel, self.scene.lib,

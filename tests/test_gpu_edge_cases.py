@@ -233,3 +233,41 @@ def test_step_on_array_of_structures_inputs(skeleton, dims, n):
     bad = torch.zeros((n, J, 3), device="cuda")
     with pytest.raises(ValueError):
         env2.step_aos(4, bad[:, :, :2], xquat[:, 1:], bad, bad, obs2, rew2, fl2)
+
+
+@pytest.mark.parametrize("skeleton,dims,n_future,A", [("humanoid15", (361, 64, 28), 3, 28), ("smpl24", (577, 64, 69), 2, 69),
+                                                      ("humanoid15", (361, 64, 28), 4, 0), ("smpl24", (577, 64, 69), 1, 5)])
+def test_extended_observation_future_frames_and_previous_action(skeleton, dims, n_future, A):
+    """End-effector targets of further reference frames and the previous action behind the standard row,
+    against the oracle, with resets frequent enough that cleared and copied action entries both occur and with
+    clips short enough that future frames run into the clip's end."""
+    sc = _scene("edge_ext_" + skeleton, dims, "f32", skeleton=skeleton, n_clips=3, frames=(10, 24), sigma_root=0.05)
+    p = Pair(sc, 333, h_min=W.ROOT_HEIGHT, with_policy=False, n_future=n_future, prev_action_dim=A, seed=21)
+    assert p.D == 24 * sc.J + 1 + (n_future - 1) * 9 * sc.o_skel.n_ee + A
+    h = p.rollout(steps=8)
+    frac = np.mean([(x["flags"] != 0).mean() for x in h])
+    assert 0.1 < frac < 0.95
+    if A:
+        tail = p.obs_g[:, p.D - A:p.D].cpu().numpy()
+        reset = h[-1]["flags"] != 0
+        assert reset.any() and (~reset).any()
+        assert not tail[reset].any() and np.array_equal(tail[~reset], p.prev_o[~reset])
+    # switching the extension off again restores the standard row
+    std = 24 * sc.J + 1
+    assert p.g_env.set_obs_extension(1, None) == std
+    obs = torch.full((p.n, p.ld_obs), float("nan"), device="cuda")
+    p.g_env.reset_all(obs, 0)
+    assert bool((obs[:, std:] == 0).all()) and bool(torch.isfinite(obs).all())
+
+
+def test_extended_observation_is_validated():
+    sc = _scene("edge_ext_bad", (361, 64, 28), "f32")
+    env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, 1 / 30, 0, W.REWARD_MULT, 0.3, 384))
+    act = torch.zeros((64, 28), device="cuda")
+    with pytest.raises(B.ImError):
+        env.set_obs_extension(0, None)                       # at least the standard frame
+    with pytest.raises(B.ImError):
+        env.set_obs_extension(2, act)                        # 361 + 36 + 28 columns do not fit a row stride of 384
+    with pytest.raises(ValueError):
+        env.set_obs_extension(1, act[:32])                   # fewer rows than envs
+    assert env.set_obs_extension(1, act[:, :20]) == 381

@@ -233,6 +233,46 @@ def test_collect_fills_storage_like_the_separate_calls(staged):
     g_env.attach_policy(None)
 
 
+@pytest.mark.parametrize("staged", [False, True], ids=["fp32-rows", "staged-bf16-rows"])
+def test_collect_with_the_extended_observation_feeds_actions_back(staged):
+    """With the observation extension on, the policy's input row is wider (further end-effector frames,
+    previous action) and every step's actions show up in the next row, zeroed where the env was reset."""
+    from paper_2609_09821_b200 import rollout as R
+    wl = W.WORKLOADS["cfg3_16384_lib32"]
+    sc = Scene(wl)
+    n, T, A, F = 256, 4, wl.act_dim, 2
+    D = wl.obs_dim + (F - 1) * 9 * sc.o_skel.n_ee + A
+    ld = B.padded_ld(D)
+    dims = (D, 128, A)
+    pw = W.make_policy_weights(dims, "bf16", 3)
+    g_env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, wl.dt, 0, W.REWARD_MULT, 0.8, ld))
+    st = R.RolloutStorage(T, n, A, ld, keep_obs=True)
+    assert g_env.set_obs_extension(F, st.action[0]) == D
+    actor = B.Policy(dims, pw["W_bf16"], pw["b"], "bf16", 0.1, 0, n)
+    if staged:
+        g_env.attach_policy(actor)
+    g_env.reset_all(st.obs_row(0), 0)
+    c, t, _ = g_env.get_state()
+    sims = {s: W.synth_sim_state_torch(sc.skel, sc.lib, c.long(), t.double() + wl.dt * s, s, wl) for s in range(1, T + 1)}
+    R.collect(g_env, actor, None, st, lambda s: sims[s], 1, 0.99, 0.95, staged=staged)
+    torch.cuda.synchronize()
+    assert g_env.device_status() == 0 and actor.device_status() == 0
+    assert not st.obs[0, :, D - A:D].any()
+    some_reset = False
+    for k in range(T):
+        reset = st.flags[k] != 0
+        some_reset |= bool(reset.any())
+        tail = st.obs[k + 1, :, D - A:D]
+        assert torch.equal(tail[~reset], st.action[k][~reset]) and not tail[reset].any()
+        assert bool((st.obs[k + 1, :, D:] == 0).all())
+    assert some_reset
+    # the policy read the whole extended row: its means match the oracle's on the stored rows
+    want = O.policy_forward(dims, pw["W"], pw["b"], 0.1, 0, T, st.obs[T - 1].cpu().numpy().astype(np.float64),
+                            bf16_operands=True)
+    assert_mean_close(st.mean[T - 1].cpu().numpy(), want["mean"], 2e-2, "means on extended rows")
+    g_env.attach_policy(None)
+
+
 # ---------------------------------------------------------------- per-dimension standard deviation
 @pytest.mark.parametrize("dtype,dims", [("f32", (361, 64, 28)), ("bf16", (361, 128, 28)), ("bf16", (577, 256, 69))])
 def test_per_dimension_log_std(dtype, dims):
