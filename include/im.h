@@ -471,8 +471,8 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   bf16 [N][K]; H = the forward activations the ReLU produced, bf16 [M][N], or NULL for no mask), and
  *   colsum_partial[(r / 32) * ld_partial + c] = the sum of the fp32 values of dH over the 32-row block
  *   (float [M / 32][ld_partial], or NULL); summing those rows with im_colsum_f32 gives the bias gradient
- *   of the layer below.  M a multiple of 32; zeros: DEVICE float [N] of zeros; the other rules of
- *   im_gemm_bf16 apply.
+ *   of the layer below.  M a multiple of 32; zeros: DEVICE, non-NULL, kept for call compatibility (not
+ *   read: the product has no bias); the other rules of im_gemm_bf16 apply.
  * im_f32_to_bf16_padded: out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
  * im_gather_rows_f32: out[i][0..cols) = in[idx[i]][0..cols) for i < rows (shuffled minibatches); idx
  *   DEVICE int32 [rows] with values in [0, n_src); out is float [rows][ld_out], or with to_bf16 != 0

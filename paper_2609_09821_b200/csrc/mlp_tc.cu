@@ -422,7 +422,7 @@ __device__ __forceinline__ void hidden_chunk(const GemmParams &P, uint32_t t_add
             v[4 * i + 2] = fmaxf(v[4 * i + 2] + b.z, fl);
             v[4 * i + 3] = fmaxf(v[4 * i + 3] + b.w, fl);
         }
-    } else {
+    } else if (fl > -INFINITY) {
 #pragma unroll
         for (int i = 0; i < 64; ++i) v[i] = fmaxf(v[i], fl);
     }
@@ -1335,6 +1335,7 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
     gp.M = M; gp.N = N; gp.K_blocks = K / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = bias;
     gp.act_floor = relu ? 0.0f : -INFINITY;
     gp.n_batches = batches; gp.a_batch_rows = M; gp.b_batch_rows = N; gp.c_batch_rows = M;
+    if (mask || colsum_partial) gp.bias = nullptr;         // the backward product has no bias: its epilogue skips the add
     gp.mask = static_cast<const __nv_bfloat16 *>(mask); gp.ld_mask = ld_mask;
     gp.colsum_partial = colsum_partial; gp.ld_partial = ld_partial;
     gp.status = status;
