@@ -14,6 +14,7 @@
 // through the common exit that frees its tensor memory.
 #include <cmath>
 #include <cstring>
+#include <utility>
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -95,6 +96,13 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its
+// predecessor in the stream is still running; dep_wait() returns once that predecessor has completed and its
+// writes are visible, dep_release() lets the successor's blocks be scheduled as SMs free up.  Both are no-ops
+// for a plain launch.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem], single-CTA, bf16 inputs, fp32 accumulate.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
@@ -477,6 +485,8 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
     const int n_tiles = tiles_per_batch * P.n_batches;
     pipe_init<Plan>(p, kEpiWarps);
     const uint32_t tmem_base = *p.tmem_slot;
+    dep_release();
+    dep_wait();                       // nothing before this line touches global memory
 
     if (warp == 0) {
         if (lane == 0) producer_role<Plan, BLOCK_N, MN>(p, &map_a, &map_b, P, n_tiles);
@@ -669,6 +679,8 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
     cluster_sync_all();                                              // both CTAs' barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    dep_release();
+    dep_wait();                       // nothing before this line touches global memory
     if (threadIdx.x == 0 && rank == 1) {
         // the pair's MMAs address the accumulator at the same tensor-memory address in both CTAs
         uint32_t leader_base;
@@ -840,6 +852,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
     if (threadIdx.x < 8) band_count[threadIdx.x] = 0;
     pipe_init<Plan>(p, kHeadEpiWarps);
     const uint32_t tmem_base = *p.tmem_slot;
+    dep_release();
+    dep_wait();                       // nothing before this line touches global memory
 
     if (warp == 0) {
         if (lane == 0) producer_role<Plan, BLOCK_N>(p, &map_a, &map_b, P, n_tiles);
@@ -1049,6 +1063,20 @@ namespace im {
 
 namespace {
 
+// Launch with programmatic stream serialization (see dep_wait): the kernel's prologue overlaps the tail of the
+// kernel before it in the stream.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <int BLOCK_N, bool BWD = false>
 cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
@@ -1065,9 +1093,10 @@ cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, c
     const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes(BWD));
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N, false, BWD><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, L.map_m, gp);
+    const cudaError_t le = launch_pdl(linear_tc_hidden_kernel<BLOCK_N, false, BWD>, dim3(grid), dim3(kThreads), smem, stream,
+                                      L.map_a, L.map_b, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 // 256-wide layers with enough rows to fill the machine run on CTA pairs.
@@ -1105,9 +1134,10 @@ cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm,
     }
     const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-    linear_tc_hidden_pair_kernel<BWD><<<2 * pairs, kThreads, pair_smem_bytes(BWD), stream>>>(L.map_a, L.map_b2, L.map_c, L.map_m, gp);
+    const cudaError_t le = launch_pdl(linear_tc_hidden_pair_kernel<BWD>, dim3(2 * pairs), dim3(kThreads), pair_smem_bytes(BWD), stream,
+                                      L.map_a, L.map_b2, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <int BLOCK_N>
@@ -1128,9 +1158,9 @@ cudaError_t launch_head(const TcLayer &L, const GemmParams &gp_in, int n_sm, cud
     const size_t smem = Plan::bytes(gp.stages, epi);
     const int tiles = (gp.M + BLOCK_M - 1) / BLOCK_M;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_head_kernel<BLOCK_N><<<grid, kHeadThreads, smem, stream>>>(L.map_a, L.map_b, gp);
+    const cudaError_t le = launch_pdl(linear_tc_head_kernel<BLOCK_N>, dim3(grid), dim3(kHeadThreads), smem, stream, L.map_a, L.map_b, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n_sm, bool force_pairs, cudaStream_t stream)
