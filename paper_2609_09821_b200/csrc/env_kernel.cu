@@ -320,6 +320,9 @@ __device__ __forceinline__ Quat as_quat(float4 v) { return {v.x, v.y, v.z, v.w};
 template <bool RESET_ALL, bool OPT>
 __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
 {
+    // a successor launched with programmatic stream serialization (the policy's first GEMM) may be scheduled
+    // onto SMs as this grid drains; it waits for this grid's completion before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const SkelDev &sk = P.sk;
     const int J = sk.J;
     const int D = 24 * J + 1;
