@@ -1117,9 +1117,10 @@ cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm
     const size_t smem = Plan::bytes(gp.stages, Plan::hidden_epi_bytes());
     const int tiles = ((gp.M + BLOCK_M - 1) / BLOCK_M) * gp.n_tiles_n * gp.n_batches;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    linear_tc_hidden_kernel<BLOCK_N, true><<<grid, kThreads, smem, stream>>>(L.map_a, L.map_b, L.map_c, L.map_c, gp);
+    const cudaError_t le = launch_pdl(linear_tc_hidden_kernel<BLOCK_N, true>, dim3(grid), dim3(kThreads), smem, stream,
+                                      L.map_a, L.map_b, L.map_c, L.map_c, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool BWD>

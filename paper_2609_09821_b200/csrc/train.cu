@@ -21,6 +21,11 @@ namespace im {
 
 namespace {
 
+// A tensor-core product launched with programmatic stream serialization right after one of these kernels may set
+// up (barriers, tensor memory) while this grid drains; it still waits for this grid to complete before it reads.
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 // out[c][r] = in[r][c] for a [rows][cols] bf16 matrix, 64 x 64 tiles through shared memory.
 // VEC: both matrices allow 16-byte accesses (pointers and row strides multiples of 8 elements): a tile is
 // read and written as 8-element chunks, the transposition happens in the 2-byte shared-memory reads
@@ -103,6 +108,7 @@ __global__ void __launch_bounds__(256) relu_mask_kernel(__nv_bfloat16 *__restric
 __global__ void __launch_bounds__(256) to_bf16_padded_kernel(const float *__restrict__ in, long long ld_in, int rows, int cols,
                                                              __nv_bfloat16 *__restrict__ out, int ld_out)
 {
+    release_dependents();
     const long long total = (long long)rows * ld_out;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const long long r = i / ld_out;
@@ -116,6 +122,7 @@ __global__ void __launch_bounds__(256) to_bf16_padded_kernel(const float *__rest
 __global__ void __launch_bounds__(256) to_bf16_padded_vec_kernel(const float *__restrict__ in, long long ld_in, int rows, int cols,
                                                                  __nv_bfloat16 *__restrict__ out, int ld_out)
 {
+    release_dependents();
     const int gpr = ld_out >> 3;                                   // 8-column groups per row
     const long long total = (long long)rows * gpr;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
@@ -152,6 +159,7 @@ __global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *_
 __global__ void __launch_bounds__(256) sum_slices_kernel(const __nv_bfloat16 *__restrict__ in, long long slice_stride,
                                                          long long ld_in, int slices, int rows, int cols, float *__restrict__ out)
 {
+    release_dependents();
     const long long total = (long long)rows * cols;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const long long r = i / cols;
@@ -292,6 +300,7 @@ constexpr int kFinishParts = 16;
 __global__ void __launch_bounds__(32 * kFinishParts) colsum_finish_kernel(const float *__restrict__ partial, int slices, int cols,
                                                                           float *__restrict__ out)
 {
+    release_dependents();
     __shared__ double part[kFinishParts][33];
     const int c = blockIdx.x * 32 + threadIdx.x;
     double s = 0.0;
