@@ -269,6 +269,19 @@ class Env:
         self.cfg.stat_starts = self.stat_starts.ctypes.data
         self.cfg.stat_failures = self.stat_failures.ctypes.data
 
+    def adapt_reset_bins(self, floor_weight: float, clear: bool = True) -> np.ndarray:
+        """Adaptive episode initialisation from the failure counts (Section 6 names adaptive sampling after
+        [Won 2019/2020] without the rule; this build's: bins where more episodes ended early are started
+        more often): weight of (clip, bin) i = fl32(fl32(failures_i) + floor_weight), then the cumulative
+        table of those weights replaces the current one; the counts are cleared if asked.  Returns the weights."""
+        w = (self.stat_failures.astype(np.float32) + np.float32(floor_weight)).astype(np.float32)
+        self.reset_cdf = reset_cdf(w)
+        self.cfg.reset_cdf = self.reset_cdf.ctypes.data
+        if clear:
+            self.stat_starts[:] = 0
+            self.stat_failures[:] = 0
+        return w
+
     def set_obs_extension(self, n_future: int = 1, prev_action: Optional[np.ndarray] = None) -> int:
         """Extended observation: end-effector targets of reference frames 2 .. n_future, then the previous action
         (fp32 [n, A]; the array is read by later steps, so the caller updates it in place).  Returns the width."""

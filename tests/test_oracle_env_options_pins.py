@@ -233,3 +233,33 @@ def test_failure_and_start_counts_add_up():
     assert int(env.stat_failures.sum()) == n_term
     assert int(env.stat_starts.sum()) == env.n + n_reset
     assert np.abs(env.stat_failures.reshape(3, B).astype(np.int64) - fail_bins).sum() <= 16
+
+
+def test_adaptation_draws_bins_in_proportion_to_failures_plus_floor():
+    """After adapt_reset_bins the probability of a (clip, bin) is (failures + floor) / sum, to within the
+    2^-32 granularity of the table; a large floor tends to the uniform table; the counts restart."""
+    import scipy.stats
+    B = 4
+    skel, lib, o_clips, env = _binned_env(np.ones((3, B), np.float32), n=30000)
+    fails = np.array([[0, 5, 0, 1], [40, 0, 0, 0], [2, 2, 2, 100]], np.uint32)
+    env.stat_failures[:] = fails.ravel()
+    env.stat_starts[:] = 7
+    floor = 0.5
+    w = env.adapt_reset_bins(floor)
+    assert not env.stat_failures.any() and not env.stat_starts.any()
+    want = (fails.ravel().astype(np.float64) + floor)
+    np.testing.assert_array_equal(w, want.astype(np.float32))
+    T = env.reset_cdf.astype(np.float64)
+    prob = np.diff(np.concatenate([[0.0], T])) / 2.0 ** 32
+    np.testing.assert_allclose(prob, want / want.sum(), atol=2.0 ** -31)
+    # the draws follow it
+    env.reset_all(3)
+    counts = env.stat_starts.astype(np.float64)
+    expect = want / want.sum() * env.n
+    assert ((counts - expect) ** 2 / expect).sum() < scipy.stats.chi2.ppf(0.999, want.size - 1)
+    # keeping the counts, and a floor that swamps them
+    env.stat_failures[:] = fails.ravel()
+    env.adapt_reset_bins(1e9, clear=False)
+    np.testing.assert_array_equal(env.stat_failures, fails.ravel())
+    prob = np.diff(np.concatenate([[0.0], env.reset_cdf.astype(np.float64)])) / 2.0 ** 32
+    np.testing.assert_allclose(prob, 1.0 / want.size, rtol=1e-6)
