@@ -261,6 +261,12 @@ im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim,
  * be NULL), stream-ordered, and zeroes them afterwards if clear != 0;
  * IM_ERR_UNSUPPORTED while n_bins == 0. */
 im_status im_env_set_reset_bins(im_env *e, int32_t n_bins, const float *weights);
+/* The adaptive part, on the device and stream-ordered (capturable): the weight of (clip, bin) i becomes
+ * fl32(fl32(failures_i) + floor_weight) -- bins where more episodes ended early are started more
+ * often, floor_weight > 0 keeps every bin reachable -- and the cumulative table is rebuilt from
+ * those weights by the rule above; clear != 0 zeroes both counts afterwards.  IM_ERR_UNSUPPORTED
+ * while n_bins == 0 or with more than 12288 (clip, bin) pairs. */
+im_status im_env_adapt_reset_bins(im_env *e, float floor_weight, int32_t clear);
 im_status im_env_get_reset_stats(im_env *e, uint32_t *starts, uint32_t *failures, int32_t clear);
 
 /* ---- policy ---------------------------------------------------------------

@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins",
 ]
 
 
@@ -141,6 +141,7 @@ def load():
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
+        L.im_env_adapt_reset_bins.argtypes = [vp, C.c_float, i32]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp, vp]
         L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
@@ -302,6 +303,10 @@ class Env:
             raise ValueError("weights must be [n_clips, n_bins]")
         _check(load().im_env_set_reset_bins(self.h, int(n_bins), _ptr(w)), "im_env_set_reset_bins")
         self.n_bins = int(n_bins)
+
+    def adapt_reset_bins(self, floor_weight: float, clear: bool = True):
+        """Adaptive episode initialisation on the device: bin weights = failure counts + floor_weight."""
+        _check(load().im_env_adapt_reset_bins(self.h, float(floor_weight), int(clear)), "im_env_adapt_reset_bins")
 
     def set_obs_extension(self, n_future: int = 1, prev_action=None):
         """Extended observation: end-effector targets of reference frames 2 .. n_future and the previous action

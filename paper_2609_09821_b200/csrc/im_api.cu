@@ -568,6 +568,16 @@ im_status im_env_set_reset_bins(im_env *e, int32_t n_bins, const float *weights)
     return IM_OK;
 }
 
+im_status im_env_adapt_reset_bins(im_env *e, float floor_weight, int32_t clear)
+{
+    if (!e || !(floor_weight > 0.0f) || std::isinf(floor_weight)) return IM_ERR_INVALID_ARG;
+    if (e->n_bins <= 0) return IM_ERR_UNSUPPORTED;
+    const int64_t n = (int64_t)e->clips->C * e->n_bins;
+    if (n > 12288) return IM_ERR_UNSUPPORTED;
+    IM_CUDA(launch_adapt_reset_cdf(e->d_stat_starts, e->d_stat_failures, (int)n, floor_weight, clear, e->d_reset_cdf, e->stream));
+    return IM_OK;
+}
+
 im_status im_env_get_reset_stats(im_env *e, uint32_t *starts, uint32_t *failures, int32_t clear)
 {
     if (!e) return IM_ERR_INVALID_ARG;

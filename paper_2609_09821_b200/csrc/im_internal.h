@@ -126,6 +126,9 @@ cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
 // simulator-native (array of structures) body states <-> component rows [13 J][stride]
 cudaError_t aos_adapter_prepare();
+// reset-bin weights from the failure counts (rollout.cu); n <= 12288 entries
+cudaError_t launch_adapt_reset_cdf(uint32_t *starts, uint32_t *failures, int n, float floor_weight, int clear,
+                                   unsigned long long *cdf, cudaStream_t stream);
 cudaError_t launch_aos_gather(const im_body_state_aos &sim, int J, int N, float *soa, long long stride, cudaStream_t stream);
 cudaError_t launch_aos_scatter_reset(const im_body_state_aos &sim, int J, int N, const float *soa, long long stride,
                                      const uint8_t *flags, cudaStream_t stream);

@@ -109,7 +109,39 @@ __global__ void __launch_bounds__(32 * kMaxChunks) gae_kernel(const GaeParams P)
     }
 }
 
+// Adaptive episode initialisation: the weight of (clip, bin) i becomes fl32(fl32(failures_i) + floor) and the
+// cumulative table T_i = floor(2^32 (w_0 + .. + w_i) / total) is rebuilt from them, sums in order in fp64
+// (one thread walks the table: it has at most a few thousand entries), T_last = 2^32.
+constexpr int kAdaptMax = 12288;           // entries staged in shared memory
+__global__ void __launch_bounds__(256) adapt_reset_cdf_kernel(uint32_t *__restrict__ starts, uint32_t *__restrict__ failures, int n,
+                                                              float floor_weight, int clear, unsigned long long *__restrict__ cdf)
+{
+    __shared__ float w[kAdaptMax];
+    for (int i = threadIdx.x; i < n; i += blockDim.x) w[i] = __fadd_rn((float)failures[i], floor_weight);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double total = 0.0, cum = 0.0;
+        for (int i = 0; i < n; ++i) total += (double)w[i];
+        for (int i = 0; i < n; ++i) {
+            cum += (double)w[i];
+            cdf[i] = (unsigned long long)floor(cum / total * 4294967296.0);
+        }
+        cdf[n - 1] = 4294967296ull;
+    }
+    if (clear)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) { starts[i] = 0u; failures[i] = 0u; }
+}
+
 }  // namespace
+
+cudaError_t launch_adapt_reset_cdf(uint32_t *starts, uint32_t *failures, int n, float floor_weight, int clear,
+                                   unsigned long long *cdf, cudaStream_t stream)
+{
+    if (n < 1 || n > kAdaptMax) return cudaErrorInvalidValue;
+    adapt_reset_cdf_kernel<<<1, 256, 0, stream>>>(starts, failures, n, floor_weight, clear, cdf);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
 
 }  // namespace im
 

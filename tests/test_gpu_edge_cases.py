@@ -183,6 +183,78 @@ def test_adaptive_initialisation_draws_and_counts_match_the_oracle():
             p.g_env.set_reset_bins(B_, bad)
 
 
+def test_bin_weights_adapted_on_the_device_match_the_oracle():
+    """im_env_adapt_reset_bins rebuilds the reset table from the failure counts without leaving the stream:
+    after it the weighted draws (clip ids, start-time bit patterns, checked by Pair every step) and the
+    restarted counts must keep matching the oracle, eagerly and when the call is replayed from a CUDA graph."""
+    sc = _scene("edge_adapt", (361, 64, 28), "f32", n_clips=4, frames=(20, 45), sigma_root=0.05)
+    n, B_ = 600, 5
+    p = Pair(sc, n, h_min=W.ROOT_HEIGHT, with_policy=False, seed=5)
+    w = np.ones((4, B_), np.float32)
+    p.o_env.set_reset_bins(B_, w)
+    p.g_env.set_reset_bins(B_, w)
+    p.reset_all()
+    step = [0]
+
+    def advance(k):
+        for _ in range(k):
+            step[0] += 1
+            sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                          torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, step[0], sc.wl)
+            p.env_step(step[0], sim)
+
+    advance(4)
+    assert int(p.o_env.stat_failures.sum()) > 100
+    before = p.o_env.reset_cdf.copy()
+    p.o_env.adapt_reset_bins(0.25)
+    p.g_env.adapt_reset_bins(0.25)
+    assert (p.o_env.reset_cdf != before).any()
+    advance(4)                                              # draws from the adapted table, bit for bit
+    starts, failures = p.g_env.reset_stats()
+    np.testing.assert_array_equal(starts.cpu().numpy().ravel(), p.o_env.stat_starts.view(np.int32))
+    np.testing.assert_array_equal(failures.cpu().numpy().ravel(), p.o_env.stat_failures.view(np.int32))
+    assert int(starts.sum()) < 4 * n                        # the counts restarted at the adaptation
+    # keeping the counts
+    p.o_env.adapt_reset_bins(2.0, clear=False)
+    p.g_env.adapt_reset_bins(2.0, clear=False)
+    advance(3)
+    starts, failures = p.g_env.reset_stats()
+    np.testing.assert_array_equal(starts.cpu().numpy().ravel(), p.o_env.stat_starts.view(np.int32))
+    np.testing.assert_array_equal(failures.cpu().numpy().ravel(), p.o_env.stat_failures.view(np.int32))
+    assert p.g_env.device_status() == 0
+    # the call is stream-ordered and capturable: a second env on a side stream adapts from a graph replay
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        g2 = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, sc.wl.dt, 5, W.REWARD_MULT, W.ROOT_HEIGHT, p.ld_obs), stream=stream)
+        g2.set_reset_bins(B_, w)
+        obs2 = torch.empty((n, p.ld_obs), device="cuda")
+        g2.reset_all(obs2, 0)                               # fills the start counts
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            g2.adapt_reset_bins(3.0, clear=True)
+        graph.replay()
+        g2.reset_all(obs2, 7)
+        stream.synchronize()
+        c2, t2, _ = g2.get_state()
+        s2, f2 = g2.reset_stats()
+    o2 = O.Env(sc.o_skel, sc.o_clips, O.make_env_config(sc.wl.dt, 5, W.REWARD_MULT, W.ROOT_HEIGHT), n)
+    o2.set_reset_bins(B_, w)
+    o2.reset_all(0)
+    o2.adapt_reset_bins(3.0, clear=True)
+    o2.reset_all(7)
+    np.testing.assert_array_equal(c2.cpu().numpy(), o2.clip_id)
+    np.testing.assert_array_equal(t2.cpu().numpy().view(np.uint32), o2.t.view(np.uint32))
+    np.testing.assert_array_equal(s2.cpu().numpy().ravel(), o2.stat_starts.view(np.int32))
+    assert int(s2.sum()) == n and int(f2.sum()) == 0
+    for bad in (0.0, -1.0, float("inf"), float("nan")):
+        with pytest.raises(B.ImError):
+            p.g_env.adapt_reset_bins(bad)
+    p.g_env.set_reset_bins(0)
+    with pytest.raises(B.ImError):
+        p.g_env.adapt_reset_bins(1.0)
+
+
 # ---------------------------------------------------------------- simulator-native input arrays
 @pytest.mark.parametrize("skeleton,dims,n", [("humanoid15", (361, 64, 28), 333), ("smpl24", (577, 64, 69), 200)])
 def test_step_on_array_of_structures_inputs(skeleton, dims, n):
