@@ -527,7 +527,7 @@ im_status im_colsum_bf16(const uint16_t *x, int64_t ld, int64_t rows, int32_t co
  * observation and then im_env_step, and copies action, reward and flags back,
  * then waits until everything has arrived.  The upload runs beside the policy
  * forward and the actions travel back beside the env step (two internal copy
- * streams); the kernels run on the env's stream.  From 4096 envs on, the upload
+ * streams); the kernels run on the env's stream.  From 49152 envs on, the upload
  * is cut into four env ranges and each range's env kernel starts when its
  * columns have arrived.  The first call allocates the
  * device staging buffers and the copy streams (so it is not capturable).  Call

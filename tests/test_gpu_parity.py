@@ -264,9 +264,9 @@ def test_bad_simulated_quaternion_sets_status_not_a_fault(scenes):
     assert torch.isfinite(p.obs_g[5]).all()
 
 
-@pytest.mark.parametrize("n", [500, 4224], ids=["one-upload", "four-env-ranges"])
+@pytest.mark.parametrize("n", [500, 49280], ids=["one-upload", "four-env-ranges"])
 def test_host_buffer_step_matches_device_step(scenes, n):
-    """From 4096 envs on the upload and the env kernel are split into four env ranges; same results."""
+    """From 49152 envs on the upload and the env kernel are split into four env ranges; same results."""
     sc = scenes("cfg2_4096")
     p = Pair(sc, n, policy_sample=300)
     p.reset_all()
