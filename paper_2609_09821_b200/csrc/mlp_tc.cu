@@ -584,11 +584,22 @@ __global__ void __launch_bounds__(kThreads, 1) linear_tc_hidden_kernel(const __g
 constexpr int kPairStages = 6;
 constexpr int kPairStageBytes = 2 * BLOCK_M * BLOCK_K * 2;             // A 128x64 + W half 128x64, bf16
 constexpr int kPairTmemCols = 512;                                     // two 256-column accumulators
-constexpr __host__ __device__ int pair_stages(bool bwd) { return bwd ? kPairStages - 1 : kPairStages; }
-constexpr size_t pair_smem_bytes(bool bwd)
+// The backward instantiation (ReLU mask and column sums in the epilogue) runs eight epilogue warps, two per
+// tensor-memory lane quadrant, each owning one half of the tile's columns; every warp cycles through a ring of
+// three 4 KB slabs, each of which first receives a chunk's mask box and is then overwritten with the chunk's
+// output for the TMA store.  The ring takes the room of two operand stages.
+constexpr int kPairEpiWarpsBwd = 8;
+constexpr int kPairRing = 3;
+constexpr __host__ __device__ int pair_epi_warps(bool bwd) { return bwd ? kPairEpiWarpsBwd : kEpiWarps; }
+constexpr __host__ __device__ int pair_threads(bool bwd) { return 64 + 32 * pair_epi_warps(bwd); }
+constexpr __host__ __device__ int pair_stages(bool bwd) { return bwd ? kPairStages - 2 : kPairStages; }
+constexpr __host__ __device__ int pair_epi_bytes(bool bwd)
 {
-    return 1024 + (size_t)pair_stages(bwd) * kPairStageBytes + (bwd ? 2 : 1) * 4 * 2 * kEpiSlabBytes + 256;
+    return bwd ? kPairEpiWarpsBwd * kPairRing * kEpiSlabBytes : kEpiWarps * 2 * kEpiSlabBytes;
 }
+constexpr size_t pair_smem_bytes(bool bwd) { return 1024 + (size_t)pair_stages(bwd) * kPairStageBytes + pair_epi_bytes(bwd) + 512; }
+static_assert(pair_smem_bytes(true) <= kSmemLimit && pair_smem_bytes(false) <= kSmemLimit, "shared memory plan of the pair kernel");
+static_assert((2 * kPairStages + 5 + kPairEpiWarpsBwd * kPairRing) * 8 <= 512, "barrier area of the pair kernel");
 
 __device__ __forceinline__ uint32_t cluster_rank()
 {
@@ -644,16 +655,17 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
 }
 
 template <bool BWD = false>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair_threads(BWD), 1)
 linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                              const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
                              const GemmParams P)
 {
-    constexpr int kStages = pair_stages(BWD);        // the backward epilogue's mask boxes take one stage's room
+    constexpr int kStages = pair_stages(BWD);
+    constexpr int kEpi = pair_epi_warps(BWD);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *epi = tiles + (size_t)kStages * kPairStageBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(epi + (BWD ? 2 : 1) * 4 * 2 * kEpiSlabBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(epi + pair_epi_bytes(BWD));
     uint64_t *mask_bar = bars + 2 * kPairStages + 5;
     uint64_t *full = bars, *empty = bars + kPairStages, *acc_full = bars + 2 * kPairStages,
              *acc_empty = bars + 2 * kPairStages + 2;
@@ -668,8 +680,9 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int i = 0; i < 2 * kEpiWarps; ++i) mbar_init(&mask_bar[i], 1);
-        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpiWarps); }
+        if (BWD)
+            for (int i = 0; i < kPairEpiWarpsBwd * kPairRing; ++i) mbar_init(&mask_bar[i], 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpi); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -739,72 +752,113 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
         }
     } else {
         // ---------------- epilogue warps (both ranks): own 128 rows x 256 columns
-        const int quad = warp & 3;
-        uint8_t *slabs = epi + (size_t)(warp - 2) * 2 * kEpiSlabBytes;
-        int which = 0;
+        const int quad = warp & 3;                     // tensor-memory lanes 32 quad .. 32 quad + 31
         int acc = 0;
         uint32_t acc_phase = 0;
-        const bool masked = BWD && P.mask != nullptr;   // BWD: mask boxes, fetched one chunk ahead
-        uint8_t *mslabs = epi + (size_t)(4 + warp - 2) * 2 * kEpiSlabBytes;
-        uint64_t *mbar = mask_bar + (warp - 2) * 2;
-        uint32_t ci = 0;
-        bool bail = false;
-        uint4 mk[8];
-        if (masked && pair < n_tiles && lane == 0 && !*abort_flag)
-            mask_issue(&map_m, mslabs, &mbar[0], (pair % P.n_tiles_n) * 256, (pair / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32);
-        if (!*abort_flag)
-        for (int tile = pair; tile < n_tiles; tile += n_pairs) {
-            const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
-            const int n0 = (tile % P.n_tiles_n) * 256;
-            bool ready = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
-            if (BWD) ready = __all_sync(0xffffffffu, ready);           // the column sums shuffle across the whole warp
-            if (!ready) break;
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
+        if constexpr (!BWD) {
+            uint8_t *slabs = epi + (size_t)(warp - 2) * 2 * kEpiSlabBytes;
+            int which = 0;
+            uint4 mk[8];                                // unused without the backward epilogue
+            if (!*abort_flag)
+            for (int tile = pair; tile < n_tiles; tile += n_pairs) {
+                const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+                const int n0 = (tile % P.n_tiles_n) * 256;
+                if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
 #pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 64) {
-                uint32_t pk[32];
-                if (BWD) {
-                    if (masked) {
-                        if (lane == 0) {
-                            uint8_t *nslab = mslabs + ((ci + 1u) & 1u) * kEpiSlabBytes;
-                            if (c0 + 64 < 256) mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], n0 + c0 + 64, m0 + quad * 32);
-                            else if (tile + n_pairs < n_tiles) {
-                                const int t2 = tile + n_pairs;
-                                mask_issue(&map_m, nslab, &mbar[(ci + 1u) & 1u], (t2 % P.n_tiles_n) * 256,
-                                           (t2 / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32);
-                            }
-                        }
-                        if (!__all_sync(0xffffffffu, mbar_wait(&mbar[ci & 1u], (ci >> 1) & 1u, abort_flag))) { bail = true; break; }
-                        mask_read(mslabs + (ci & 1u) * kEpiSlabBytes, lane, mk);
-                        ++ci;
-                    } else mask_all_positive(mk);
-                }
-                hidden_chunk<BWD>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                __syncwarp();
-                uint8_t *slab = slabs + which * kEpiSlabBytes;
-                const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
+                for (int c0 = 0; c0 < 256; c0 += 64) {
+                    uint32_t pk[32];
+                    hidden_chunk<false>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                    uint8_t *slab = slabs + which * kEpiSlabBytes;
+                    const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
-                                 "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                                     "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    which ^= 1;
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                 ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
-                which ^= 1;
+                if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[acc]), 0));   // the leader's barrier
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
-            if (bail) break;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[acc]), 0));   // the leader's barrier
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        } else {
+            // warp 2 + e: quadrant (2 + e) & 3, column chunks 2 (e / 4) and 2 (e / 4) + 1 of every tile.  Chunk j of
+            // the warp's sequence uses slab j % 3: mask box in (requested one chunk ahead), output out.
+            const int ew = warp - 2, half = ew >> 2;
+            uint8_t *ring = epi + (size_t)ew * kPairRing * kEpiSlabBytes;
+            uint64_t *mbar = mask_bar + ew * kPairRing;
+            const bool masked = P.mask != nullptr;
+            uint32_t ci = 0;
+            bool bail = false;
+            uint4 mk[8];
+            auto issue_mask = [&](uint32_t j) {
+                const int t2 = pair + (int)(j >> 1) * n_pairs;
+                if (t2 >= n_tiles) return;
+                mask_issue(&map_m, ring + (j % kPairRing) * kEpiSlabBytes, &mbar[j % kPairRing],
+                           (t2 % P.n_tiles_n) * 256 + (2 * half + (int)(j & 1u)) * 64,
+                           (t2 / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M + quad * 32);
+            };
+            if (masked && lane == 0 && !*abort_flag) issue_mask(0u);
+            if (!*abort_flag)
+            for (int tile = pair; tile < n_tiles; tile += n_pairs) {
+                const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+                const int n0 = (tile % P.n_tiles_n) * 256;
+                // (the column sums shuffle across the whole warp: every lane takes the same decision)
+                if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
+#pragma unroll 1
+                for (int j = 0; j < 2; ++j) {
+                    const int c0 = (2 * half + j) * 64;
+                    if (lane == 0) {
+                        // slab (ci + 1) % 3 last held chunk ci - 2: its store must have read it before the next box lands
+                        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        if (masked) issue_mask(ci + 1u);
+                    }
+                    __syncwarp();
+                    uint8_t *slab = ring + (ci % kPairRing) * kEpiSlabBytes;
+                    if (masked) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(&mbar[ci % kPairRing], (ci / kPairRing) & 1u, abort_flag))) { bail = true; break; }
+                        mask_read(slab, lane, mk);
+                    } else mask_all_positive(mk);
+                    uint32_t pk[32];
+                    hidden_chunk<true>(P, t_row + (uint32_t)c0, m0 + quad * 32 + lane, n0 + c0, lane, mk, pk);
+                    // each lane overwrites the 128 bytes it read its own mask words from
+                    const uint32_t slab_row = smem_u32(slab) + (uint32_t)lane * 128u;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t dst = slab_row + (uint32_t)((c ^ (lane & 7)) << 4);      // 128B swizzle
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                                     "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(&map_c), "r"(smem_u32(slab)), "r"(n0 + c0), "r"(m0 + quad * 32) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    ++ci;
+                }
+                if (bail) break;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[acc]), 0));   // the leader's barrier
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -1135,7 +1189,7 @@ cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm,
     }
     const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-    const cudaError_t le = launch_pdl(linear_tc_hidden_pair_kernel<BWD>, dim3(2 * pairs), dim3(kThreads), pair_smem_bytes(BWD), stream,
+    const cudaError_t le = launch_pdl(linear_tc_hidden_pair_kernel<BWD>, dim3(2 * pairs), dim3(pair_threads(BWD)), pair_smem_bytes(BWD), stream,
                                       L.map_a, L.map_b2, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return le != cudaSuccess ? le : cudaGetLastError();
@@ -1173,7 +1227,10 @@ cudaError_t dispatch_tc(const TcLayer &L, const GemmParams &gp, bool last, int n
         // 7 % faster paired)
         const int pair_tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
         const bool bwd = gp.mask || gp.colsum_partial;
-        if (L.block_n == 256 && gp.n_batches == 1 && (force_pairs || (pair_tiles >= n_sm && gp.K_blocks >= 8)))
+        // (the backward epilogue is the longer part of a tile when K is short, and the pair kernel runs it on
+        // eight warps: it takes those products whenever its tiles fill the machine)
+        if (L.block_n == 256 && gp.n_batches == 1 &&
+            (force_pairs || (pair_tiles >= n_sm && gp.K_blocks >= 8) || (bwd && pair_tiles >= n_sm / 2)))
             return bwd ? launch_hidden_pair<true>(L, gp, n_sm, stream) : launch_hidden_pair<false>(L, gp, n_sm, stream);
         switch (L.block_n) {
         case 256: return bwd ? launch_hidden<256, true>(L, gp, n_sm, stream) : launch_hidden<256>(L, gp, n_sm, stream);
