@@ -162,6 +162,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-rollout-extras", action="store_true",
                     help="skip the separate timing of the value head and the advantage estimator")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short device-resident runs of the other benchmark configurations")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -495,6 +497,29 @@ def main():
         if "value_head" in extras:
             extras["value_head"]["frac_of_tensor_peak"] = extras["value_head"]["achieved_tflops"] / tensor_peak
         line["rollout_extras"] = extras
+    if world == 1 and not args.no_other_configs and args.workload == DEFAULT_WORKLOAD and args.steps is None:
+        # the other configurations, device-resident numbers only, each in a process of its own (this one's
+        # buffers are released first); the headline stays the default workload's
+        import subprocess
+        import sys
+        del graph
+        torch.cuda.empty_cache()
+        others = {}
+        for name in sorted(W.WORKLOADS):
+            if name == wl.name:
+                continue
+            cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--warmup", str(max(Wm, 3)),
+                   "--no-cpu-baseline", "--no-e2e", "--no-rollout-extras", "--no-other-configs"]
+            try:
+                out = subprocess.run(cmd, capture_output=True, text=True, timeout=120)
+                d = json.loads(out.stdout.strip().splitlines()[-1])
+                others[name] = dict(value=d["value"], unit=UNIT, ms_per_step=d["ms_per_step"], steps=d["steps"],
+                                    n_envs=d["config"]["n_envs_per_gpu"], dtype=d["dtype"],
+                                    policy_frac_of_tensor_peak=d["roofline"]["frac"] if d["dtype"] == "bf16" else None,
+                                    env_frac_of_hbm_peak=d["roofline_env"]["frac"], sm_mhz=d["clocks"].get("sm_mhz"))
+            except Exception as exc:                     # a side measurement must not take the headline down with it
+                others[name] = dict(error=repr(exc)[:200])
+        line["other_configs"] = others
     if not args.no_cpu_baseline:
         res = oracle_leg(wl, skel, lib, pol, n_sample=2048, steps=64, warmup=1, budget_s=15.0)
         line["cpu_baseline"] = dict(value=res["value"], unit=UNIT, cores=res["cores"], kind="oracle",
