@@ -332,6 +332,25 @@ def test_extended_observation_future_frames_and_previous_action(skeleton, dims, 
     assert bool((obs[:, std:] == 0).all()) and bool(torch.isfinite(obs).all())
 
 
+def test_all_optional_semantics_together():
+    """Grace steps, motion randomisation, weighted initialisation, write-back and the extended observation in one
+    env: the options share the kernel's reset and observation phases, so they are also checked in combination."""
+    sc = _scene("edge_all_opts", (577, 64, 69), "f32", skeleton="smpl24", n_clips=3, frames=(12, 30), sigma_root=0.05)
+    n, B_ = 260, 4
+    p = Pair(sc, n, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, grace_steps=2, reset_noise_std=0.03,
+             n_future=3, prev_action_dim=7, seed=9)
+    w = np.random.default_rng(4).uniform(0.1, 1.0, (3, B_)).astype(np.float32)
+    p.o_env.set_reset_bins(B_, w)
+    p.g_env.set_reset_bins(B_, w)
+    h = p.rollout(steps=7)
+    flags = np.array([x["flags"] for x in h])
+    assert not (flags[:2] & 1).any() and (flags[2:] & 1).any() and (flags >> 1).any()
+    starts, failures = p.g_env.reset_stats()
+    np.testing.assert_array_equal(starts.cpu().numpy().ravel(), p.o_env.stat_starts.view(np.int32))
+    np.testing.assert_array_equal(failures.cpu().numpy().ravel(), p.o_env.stat_failures.view(np.int32))
+    assert p.g_env.device_status() == 0
+
+
 def test_extended_observation_is_validated():
     sc = _scene("edge_ext_bad", (361, 64, 28), "f32")
     env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(64, 1 / 30, 0, W.REWARD_MULT, 0.3, 384))
