@@ -224,7 +224,11 @@ struct SmemPlan {
     static constexpr __host__ __device__ int hidden_epi_bytes(bool bwd = false) { return (bwd ? 2 : 1) * 4 * 2 * kEpiSlabBytes; }
     // head: [2 accumulators][mean, action][128 rows][A] floats laid out as in global memory,
     // partial sums of z^2 [2][4][128], band counters [2][4]
-    __host__ __device__ static constexpr int head_epi_bytes(int A) { return (2 * 2 * 128 * A * 4 + 2 * 4 * 128 * 4 + 64 + 1023) / 1024 * 1024; }
+    // (+ bias and per-column sigma of the tile's columns, 2 x 128 floats)
+    __host__ __device__ static constexpr int head_epi_bytes(int A)
+    {
+        return (2 * 2 * 128 * A * 4 + 2 * 4 * 128 * 4 + 64 + 2 * 128 * 4 + 1023) / 1024 * 1024;
+    }
     __host__ __device__ static constexpr int stages_for(int epi_bytes)
     {
         const int room = (int)kSmemLimit - 1024 - kBarBytes - epi_bytes;
@@ -903,11 +907,20 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
     float *out_tiles = reinterpret_cast<float *>(p.epi);                            // [2][2][128 * A]
     float *zz_part = out_tiles + 2 * 2 * out_floats;                                // [2][4][128]
     int *band_count = reinterpret_cast<int *>(zz_part + 2 * 4 * 128);               // [2][4]
+    float *s_bias = reinterpret_cast<float *>(band_count + 16);                     // [128]: bias of the tile's columns
+    float *s_sigma = s_bias + 128;                                                  // [128]: standard deviation per column
     if (threadIdx.x < 8) band_count[threadIdx.x] = 0;
     pipe_init<Plan>(p, kHeadEpiWarps);
     const uint32_t tmem_base = *p.tmem_slot;
     dep_release();
     dep_wait();                       // nothing before this line touches global memory
+    // the epilogue reads bias and sigma from shared memory as 16-byte words instead of one global load per output
+    if (threadIdx.x < BLOCK_N) {
+        const int cidx = threadIdx.x;
+        s_bias[cidx] = __ldg(P.bias + cidx);
+        s_sigma[cidx] = cidx < A ? (P.log_std ? expf(__ldg(P.log_std + cidx)) : P.sigma) : 0.0f;
+    }
+    __syncthreads();
 
     if (warp == 0) {
         if (lane == 0) producer_role<Plan, BLOCK_N>(p, &map_a, &map_b, P, n_tiles);
@@ -957,15 +970,15 @@ __global__ void __launch_bounds__(kHeadThreads, 1) linear_tc_head_kernel(const _
                                 box_muller(x.x, x.y, z[0], z[1]);
                                 box_muller(x.z, x.w, z[2], z[3]);
                             }
+                            const float4 b4 = *reinterpret_cast<const float4 *>(s_bias + col);
+                            const float4 s4 = *reinterpret_cast<const float4 *>(s_sigma + col);
+                            const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 if (col + i < A) {
-                                    const float mu = v[4 * g + i] + __ldg(P.bias + col + i);
+                                    const float mu = v[4 * g + i] + bb[i];
                                     s_mean[row_in_tile * A + col + i] = mu;
-                                    if (sample) {
-                                        const float sg = P.log_std ? expf(__ldg(P.log_std + col + i)) : P.sigma;
-                                        s_act[row_in_tile * A + col + i] = mu + sg * z[i];
-                                    }
+                                    if (sample) s_act[row_in_tile * A + col + i] = mu + ss[i] * z[i];
                                     zz += z[i] * z[i];
                                 }
                             }
