@@ -429,6 +429,20 @@ def main():
             cflops = mlp_flops_per_env(cdims) * n
             extras["value_head"] = dict(dims=list(cdims), seconds_per_launch=t_v, achieved_tflops=cflops / t_v / 1e12)
             del critic
+            # policy serving: the env step asked for the policy's bf16 rows only (no fp32 observation output);
+            # back-to-back launches over the step buffers, which together exceed L2
+            t_s = []
+            for i in range(3 + reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for j in range(8):
+                    env.step(Wm + K + 1 + 8 * i + j, sims[(8 * i + j) % n_buf], None, reward, flags)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    t_s.append(a.elapsed_time(b) * 1e-3 / 8)
+            extras["env_step_bf16_rows_only"] = dict(seconds_per_launch=float(np.median(t_s)),
+                                                     note="im_env_step with obs_out == NULL while attached to the policy")
         del flush
 
     # ---- end to end through the host-buffer entry point: pinned host inputs, results read back

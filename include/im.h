@@ -326,7 +326,10 @@ im_status im_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
  * im_policy_forward on the fp32 rows, without the conversion pass over the
  * observations.  Requirements: tensor-core policy, same stream, policy input
  * width 24J+1, max_batch >= N, and ld_obs equal to 24J+1 rounded up to a
- * multiple of 64.  Passing NULL detaches. */
+ * multiple of 64.  Passing NULL detaches.  While a policy is attached,
+ * im_env_reset_all and im_env_step accept obs_out == NULL: only the bf16 rows
+ * are written then (a policy-serving loop that never reads the fp32
+ * observation saves their 4 (24J+1) bytes of stores per env). */
 im_status im_env_attach_policy(im_env *e, im_policy *p);
 im_status im_policy_forward_staged(im_policy *p, uint32_t step, int32_t n,
                                    float *mean_out, float *action_out, float *logp_out);

@@ -586,11 +586,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         for (int r = c; r < kTile; r += C) {
             const int e = blockIdx.x * kTile + r;
             if (e >= P.N) break;
-            float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
+            // (a policy-serving loop may ask for the bf16 rows only: obs null)
+            float4 *dst = P.obs ? reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs) : nullptr;
             uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
             for (int i = lane; i < n4; i += 32) {
                 const float4 v = tile4[(size_t)r * S4 + i];
-                dst[i] = v;
+                if (dst) dst[i] = v;
                 if (dst16) dst16[i] = pack_bf16x4(v);
             }
         }
@@ -666,11 +667,11 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         for (int r = c; r < kTile; r += C) {
             const int e = blockIdx.x * kTile + r;
             if (e >= P.N) break;
-            float4 *dst = reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs);
+            float4 *dst = P.obs ? reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs) : nullptr;
             uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
             for (int i = n4 + lane; i < ld4; i += 32) {
                 const float4 v = (i - n4 < S4) ? tile4[(size_t)r * S4 + i - n4] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                dst[i] = v;
+                if (dst) dst[i] = v;
                 if (dst16) dst16[i] = pack_bf16x4(v);
             }
         }

@@ -261,7 +261,8 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
 
 im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out)
 {
-    if (!e || !obs_out || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
+    if (!e || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
+    if (!obs_out && !e->d_obs_bf16) return IM_ERR_INVALID_ARG;      // no fp32 rows only with an attached policy's bf16 rows
     EnvKernelParams p;
     fill_params(e, step, p);
     p.obs = obs_out;
@@ -272,7 +273,8 @@ im_status im_env_reset_all(im_env *e, uint32_t step, float *obs_out)
 im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float *obs_out, float *reward_out,
                       uint8_t *flags_out, float *terms_out)
 {
-    if (!e || !sim || !obs_out || !reward_out || !flags_out) return IM_ERR_INVALID_ARG;
+    if (!e || !sim || !reward_out || !flags_out) return IM_ERR_INVALID_ARG;
+    if (!obs_out && !e->d_obs_bf16) return IM_ERR_INVALID_ARG;      // no fp32 rows only with an attached policy's bf16 rows
     if (!sim->pos || !sim->quat || !sim->linvel || !sim->angvel || sim->comp_stride < e->cfg.n_envs)
         return IM_ERR_INVALID_ARG;
     if (!aligned16(obs_out) || !aligned16(sim->pos) || !aligned16(sim->quat) || !aligned16(sim->linvel) ||

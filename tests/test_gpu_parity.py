@@ -306,6 +306,40 @@ def test_staged_policy_input_matches_the_conversion_pass(scenes):
     p.g_env.attach_policy(None)
 
 
+def test_bf16_rows_only_when_the_fp32_observation_is_not_asked_for(scenes):
+    """With a policy attached obs_out may be NULL: the staged bf16 rows (and everything else the step returns)
+    are the same bits as with the fp32 rows written as well; without a policy NULL is an error."""
+    sc = scenes("cfg3_16384_lib32")
+    wl, n = sc.wl, 1000
+    ld = B.padded_ld(wl.obs_dim)
+    pol = sc.pol
+    outs = []
+    for with_obs in (True, False):
+        env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(n, wl.dt, 3, W.REWARD_MULT, 0.8, ld))
+        policy = B.Policy(pol["dims"], pol["W_bf16"], pol["b"], "bf16", wl.sigma_action, 3, n)
+        env.attach_policy(policy)
+        obs = torch.zeros((n, ld), device="cuda") if with_obs else None
+        rew, fl = torch.empty(n, device="cuda"), torch.empty(n, dtype=torch.uint8, device="cuda")
+        mean, act, logp = torch.empty((n, wl.act_dim), device="cuda"), torch.empty((n, wl.act_dim), device="cuda"), torch.empty(n, device="cuda")
+        env.reset_all(obs, 0)
+        hist = []
+        for s in range(1, 4):
+            c, t, _ = env.get_state()
+            sim = W.synth_sim_state_torch(sc.skel, sc.lib, c.long(), t.double() + wl.dt, s, wl)
+            policy.forward_staged(s, n, mean, act, logp)
+            env.step(s, sim, obs, rew, fl)
+            hist.append((mean.clone(), act.clone(), rew.clone(), fl.clone()))
+        outs.append(hist)
+        env.attach_policy(None)
+        if not with_obs:
+            with pytest.raises(B.ImError):
+                env.step(4, sim, None, rew, fl)              # detached: the fp32 rows are the only output
+    for a, b in zip(*outs):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    assert bool((outs[0][-1][3] != 0).any())
+
+
 def test_reset_draws_bit_exact_over_many_counters(scenes):
     sc = scenes("cfg3_16384_lib32")
     n = 100000
