@@ -658,7 +658,9 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
                  ::"r"(smem_u32(bar)), "h"(both) : "memory");
 }
 
-template <bool BWD = false>
+// MN: both operands are stored [contraction rows][M or N columns] (the transposed product of two row-major
+// matrices, as in the single-CTA kernel's MN instantiation), possibly over several row slices ("batches").
+template <bool BWD = false, bool MN = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair_threads(BWD), 1)
 linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                              const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
@@ -680,7 +682,8 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int tiles_m = (P.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M);
-    const int n_tiles = tiles_m * P.n_tiles_n;                       // 256 x 256 tiles
+    const int tiles_per_batch = tiles_m * P.n_tiles_n;               // 256 x 256 tiles
+    const int n_tiles = tiles_per_batch * (MN ? P.n_batches : 1);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -712,16 +715,27 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
             int stage = 0;
             uint32_t phase = 0;
             for (int tile = pair; tile < n_tiles; tile += n_pairs) {
-                const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
-                const int n0 = (tile % P.n_tiles_n) * 256 + (int)rank * 128;
+                const int bt = MN ? tile / tiles_per_batch : 0, tt = tile - bt * tiles_per_batch;
+                const int m0 = (tt / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+                const int n0 = (tt % P.n_tiles_n) * 256 + (int)rank * 128;
                 bool ok = true;
                 for (int kb = 0; kb < P.K_blocks; ++kb) {
                     if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t *sa = tiles + (size_t)stage * kPairStageBytes;
                     const uint32_t leader_full = map_to_rank(smem_u32(&full[stage]), 0);
                     if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * kPairStageBytes);
-                    tma_load_2d_pair(sa, &map_a, leader_full, kb * BLOCK_K, m0);
-                    tma_load_2d_pair(sa + BLOCK_M * BLOCK_K * 2, &map_b, leader_full, kb * BLOCK_K, n0);
+                    if (MN) {
+                        // a K block is 64 rows of the slice; this CTA's 128 M columns and its 128 N columns as 64-column boxes
+                        const int r = bt * P.a_batch_rows + kb * BLOCK_K;
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            tma_load_2d_pair(sa + i * 8192, &map_a, leader_full, m0 + 64 * i, r);
+                            tma_load_2d_pair(sa + BLOCK_M * BLOCK_K * 2 + i * 8192, &map_b, leader_full, n0 + 64 * i, r);
+                        }
+                    } else {
+                        tma_load_2d_pair(sa, &map_a, leader_full, kb * BLOCK_K, m0);
+                        tma_load_2d_pair(sa + BLOCK_M * BLOCK_K * 2, &map_b, leader_full, kb * BLOCK_K, n0);
+                    }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
@@ -730,7 +744,7 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only)
         if (lane == 0 && rank == 0 && !*abort_flag) {
-            constexpr uint32_t idesc = instr_desc_bf16(2 * BLOCK_M, 256);
+            constexpr uint32_t idesc = MN ? instr_desc_bf16_mn(2 * BLOCK_M, 256) : instr_desc_bf16(2 * BLOCK_M, 256);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -742,10 +756,17 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
                     if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(tiles + (size_t)stage * kPairStageBytes);
-                    const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + BLOCK_M * BLOCK_K * 2);
+                    if (MN) {
+                        const uint64_t da = smem_desc_mn_major_sw128(sa, 8192u), db = smem_desc_mn_major_sw128(sa + BLOCK_M * BLOCK_K * 2, 8192u);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            umma_bf16_pair(d_tmem, da + (uint64_t)(128 * k), db + (uint64_t)(128 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    } else {
+                        const uint64_t da = smem_desc_k_major_sw128(sa), db = smem_desc_k_major_sw128(sa + BLOCK_M * BLOCK_K * 2);
+#pragma unroll
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
                     umma_commit_pair(&empty[stage]);          // both CTAs' stages are free once these MMAs have read them
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -765,8 +786,9 @@ linear_tc_hidden_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __
             uint4 mk[8];                                // unused without the backward epilogue
             if (!*abort_flag)
             for (int tile = pair; tile < n_tiles; tile += n_pairs) {
-                const int m0 = (tile / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
-                const int n0 = (tile % P.n_tiles_n) * 256;
+                const int bt = MN ? tile / tiles_per_batch : 0, tt = tile - bt * tiles_per_batch;
+                const int m0 = bt * P.c_batch_rows + (tt / P.n_tiles_n) * 2 * BLOCK_M + (int)rank * BLOCK_M;
+                const int n0 = (tt % P.n_tiles_n) * 256;
                 if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
@@ -1190,20 +1212,20 @@ cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
-template <bool BWD>
+template <bool BWD, bool MN = false>
 cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
 {
     static bool prepared = false;
     if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD, MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)pair_smem_bytes(BWD));
         if (e != cudaSuccess) return e;
         prepared = true;
     }
-    const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n;
+    const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n * (MN ? gp.n_batches : 1);
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
-    const cudaError_t le = launch_pdl(linear_tc_hidden_pair_kernel<BWD>, dim3(2 * pairs), dim3(pair_threads(BWD)), pair_smem_bytes(BWD), stream,
-                                      L.map_a, L.map_b2, L.map_c, L.map_m, gp);
+    const cudaError_t le = launch_pdl(linear_tc_hidden_pair_kernel<BWD, MN>, dim3(2 * pairs), dim3(pair_threads(BWD)), pair_smem_bytes(BWD), stream,
+                                      L.map_a, MN ? L.map_b : L.map_b2, L.map_c, L.map_m, gp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -1479,6 +1501,13 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
     gp.n_batches = slices; gp.a_batch_rows = R / slices; gp.b_batch_rows = 0; gp.c_batch_rows = c_pitch;
     gp.status = status;
     cudaError_t e;
+    // CTA pairs (256 x 256 tiles, half of the N operand per SM) when the output splits into whole 256-row tiles,
+    // the slices' pitch keeps those tiles apart and there are tiles for most pairs
+    const int pair_tiles = ((Mo + 255) / 256) * L.n_tiles_n * slices;
+    if (L.block_n == 256 && Mo % 256 == 0 && c_pitch % 256 == 0 && pair_tiles >= n_sm / 3 && gp.K_blocks >= 8) {
+        L.map_m = L.map_c;
+        return launch_hidden_pair<false, true>(L, gp, n_sm, stream) == cudaSuccess ? IM_OK : IM_ERR_CUDA;
+    }
     switch (L.block_n) {
     case 256: e = launch_hidden_mn<256>(L, gp, n_sm, stream); break;
     case 128: e = launch_hidden_mn<128>(L, gp, n_sm, stream); break;

@@ -288,9 +288,11 @@ def test_whole_training_iteration_runs_from_one_cuda_graph():
 
 
 @pytest.mark.parametrize("R,Mo,No,slices", [(128, 64, 64, 1), (256, 128, 128, 2), (1024, 200, 256, 4), (512, 69, 512, 2),
-                                             (2048, 1024, 640, 4), (512, 128, 320, 2)])
+                                             (2048, 1024, 640, 4), (512, 128, 320, 2),
+                                             (8192, 1024, 1024, 8), (16384, 512, 640, 16), (4096, 1024, 512, 8)])
 def test_transposed_product_reads_both_operands_in_place(R, Mo, No, slices):
-    """A^T B of two row-major bf16 matrices on the tensor cores (operands M/N-major), per row slice."""
+    """A^T B of two row-major bf16 matrices on the tensor cores (operands M/N-major), per row slice; the last
+    three shapes have enough 256 x 256 tiles for the CTA-pair kernel (one of them with a ragged last tile)."""
     g = np.random.default_rng(R + Mo)
     a = W.round_to_bf16(g.standard_normal((R, Mo)).astype(np.float32))[0]
     b = W.round_to_bf16((g.standard_normal((R, No)) / 8).astype(np.float32))[0]
