@@ -153,13 +153,13 @@ cudaError_t launch_aos_scatter_reset(const im_body_state_aos &sim, int J, int N,
 
 cudaError_t aos_adapter_prepare()
 {
-    static bool done = false;
-    if (done) return cudaSuccess;
-    const int bytes = (int)tile_bytes(IM_MAX_BODIES);      // 53 KB at 32 bodies: above the 48 KB default
-    cudaError_t e = cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(scatter_reset_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    done = e == cudaSuccess;
-    return e;
+    static DeviceOnce once;
+    return once.run([] {
+        const int bytes = (int)tile_bytes(IM_MAX_BODIES);      // 53 KB at 32 bodies: above the 48 KB default
+        cudaError_t e = cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(scatter_reset_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        return e;
+    });
 }
 
 }  // namespace im

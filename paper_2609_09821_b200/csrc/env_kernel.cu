@@ -43,11 +43,65 @@ __host__ __device__ inline int tile_stride(int D)
 // up to a multiple of four columns so that both halves start on a 16-byte boundary.
 __host__ __device__ inline int split_col(int J) { return (15 * J + 3) / 4 * 4; }
 
-__host__ __device__ inline size_t smem_floats(int J, int n_chains, int extra_cols)
+// Shared memory, in floats: the staged half rows, the chains' partial sums, the chains' link records.
+__host__ __device__ inline size_t smem_floats(int J, int n_chains, int n_links, int extra_cols)
 {
     const int D = 24 * J + 1 + extra_cols, c1 = split_col(J);
     const int s1 = tile_stride(c1), s2 = tile_stride(D - c1);
-    return (size_t)kTile * (s1 > s2 ? s1 : s2) + (size_t)kPartials * n_chains * kTile;
+    return (size_t)kTile * (s1 > s2 ? s1 : s2) + (size_t)kPartials * n_chains * kTile + (size_t)8 * n_links;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Clip table.  Row r (one keyframe) holds 2 + 2 J 16-byte words:
+//   [0]        root position (x, y, z, 0)
+//   [1]        root displacement to the next keyframe (0 in a clip's last frame)
+//   [2 + 2 j]  local rotation of joint j, normalised (w, x, y, z)
+//   [3 + 2 j]  (h, |h|^2): h = log(q_j[k]* q_j[k+1]) on the shortest arc, the half-angle rotation
+//              vector that takes this keyframe's rotation to the next one's (0 in the last frame)
+// With h in the table the interpolation of step a1 needs one row instead of two and no inverse
+// trigonometry per step: slerp(q0, q1, alpha) = q0 exp(alpha h), and the joint's angular velocity
+// in the child frame, 2 log(q0* q1) fps, is 2 fps h.  The rows are built on the device, in double
+// precision, when the clips are loaded.
+// ---------------------------------------------------------------------------------------------
+__global__ void clip_table_kernel(const float *__restrict__ root_pos, const float *__restrict__ local_quat,
+                                  const uint8_t *__restrict__ last, long long rows, int J, float4 *__restrict__ frames)
+{
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i >= rows * (J + 1)) return;
+    const long long r = i / (J + 1);
+    const int j = (int)(i - r * (J + 1)) - 1;                  // -1: the root translation
+    float4 *row = frames + r * (2 + 2 * J);
+    const bool has_next = !last[r];
+    if (j < 0) {
+        const float *p = root_pos + 3 * r;
+        row[0] = make_float4(p[0], p[1], p[2], 0.0f);
+        row[1] = has_next ? make_float4((float)((double)p[3] - p[0]), (float)((double)p[4] - p[1]), (float)((double)p[5] - p[2]), 0.0f)
+                          : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        return;
+    }
+    const float *a = local_quat + 4 * (r * J + j);
+    double q0[4] = {a[0], a[1], a[2], a[3]};
+    const double n0 = sqrt(q0[0] * q0[0] + q0[1] * q0[1] + q0[2] * q0[2] + q0[3] * q0[3]);
+    for (int c = 0; c < 4; ++c) q0[c] /= n0;
+    row[2 + 2 * j] = make_float4((float)q0[0], (float)q0[1], (float)q0[2], (float)q0[3]);
+    double h[3] = {0.0, 0.0, 0.0};
+    if (has_next) {
+        const float *bq = a + 4 * J;
+        double q1[4] = {bq[0], bq[1], bq[2], bq[3]};
+        const double n1 = sqrt(q1[0] * q1[0] + q1[1] * q1[1] + q1[2] * q1[2] + q1[3] * q1[3]);
+        for (int c = 0; c < 4; ++c) q1[c] /= n1;
+        // rel = q0* q1, on the shortest arc
+        double w = q0[0] * q1[0] + q0[1] * q1[1] + q0[2] * q1[2] + q0[3] * q1[3];
+        double x = q0[0] * q1[1] - q0[1] * q1[0] - q0[2] * q1[3] + q0[3] * q1[2];
+        double y = q0[0] * q1[2] + q0[1] * q1[3] - q0[2] * q1[0] - q0[3] * q1[1];
+        double z = q0[0] * q1[3] - q0[1] * q1[2] + q0[2] * q1[1] - q0[3] * q1[0];
+        if (w < 0.0) { w = -w; x = -x; y = -y; z = -z; }
+        const double n = sqrt(x * x + y * y + z * z);
+        const double k = n < 1e-12 ? 1.0 : atan2(n, w) / n;
+        h[0] = k * x; h[1] = k * y; h[2] = k * z;
+    }
+    const float hx = (float)h[0], hy = (float)h[1], hz = (float)h[2];
+    row[3 + 2 * j] = make_float4(hx, hy, hz, hx * hx + hy * hy + hz * hz);
 }
 
 // Keyframe row and blend factor at `time` (step a1): f = fl32(time * fps),
@@ -76,61 +130,33 @@ __device__ __forceinline__ float asin2_over_u(float u)
     return fmaf(p, u, 1.0f);               // n = 1
 }
 
-// sin(sqrt y) / sqrt y for small y (error below 1e-10 for y <= 0.07).
-__device__ __forceinline__ float sinc_sqrt(float y)
-{
-    float p = -1.9841270e-4f;
-    p = fmaf(p, y, 8.3333333e-3f);
-    p = fmaf(p, y, -1.6666667e-1f);
-    return fmaf(p, y, 1.0f);
-}
-
-// Shortest-arc slerp of one joint plus, if asked, the joint's angular velocity
-// in the child frame, 2 log(q0* q1) fps.  The vector part of q0* q1 is formed
-// from q1 - q0, which avoids the cancellation of the direct product when the
-// keyframes are close and keeps the velocity accurate to ~1e-6 rad/s.
-// Keyframes of a motion clip are close together, so the usual case (angle
-// between the two quaternions below 0.25 rad) is evaluated without
-// trigonometric calls: theta^2 from sin^2 theta by the arcsine series, and
-// sin(a theta)/sin(theta) = a sinc(a theta)/sinc(theta) by short polynomials.
-// Everything is normalised by |q0||q1|, so slightly non-unit keyframes give
-// the same rotation as their normalised versions.
+// Shortest-arc slerp of one joint from the table's (keyframe, half-angle log) pair: q0 exp(alpha h), with
+// exp(alpha h) = (cos(alpha theta), sin(alpha theta) / theta h), theta = |h| <= pi / 2.  Keyframes of a motion
+// clip are close together, so the usual case (theta <= 0.5) takes cos and sin(x)/x from their Taylor
+// polynomials in (alpha theta)^2 (truncation below 2e-8).  If asked, also the joint's angular velocity in the
+// child frame, which is constant over the interval: 2 fps h.
 template <bool VEL>
-__device__ __forceinline__ void slerp_joint(Quat q0, Quat q1, float alpha, float fps, Quat &q, Vec3 &wl)
+__device__ __forceinline__ void slerp_joint(float4 k0, float4 lg, float alpha, float fps2, Quat &q, Vec3 &wl)
 {
-    float d = q0.w * q1.w + q0.x * q1.x + q0.y * q1.y + q0.z * q1.z;
-    if (d < 0.0f) { d = -d; q1 = {-q1.w, -q1.x, -q1.y, -q1.z}; }
-    const Quat diff = {q1.w - q0.w, q1.x - q0.x, q1.y - q0.y, q1.z - q0.z};
-    const Quat c = qmul(qconj(q0), diff);
-    const float n2 = c.x * c.x + c.y * c.y + c.z * c.z;
-    const float m2 = fmaf(d, d, n2);                       // (|q0||q1|)^2
-    const float u = __fdividef(n2, m2);                    // sin^2 theta
-    float s0, s1, vel_scale = 0.0f;
-    if (u <= 0.0625f) {
-        const float x = u * asin2_over_u(u);               // theta^2
-        const float sc = sinc_sqrt(x);
-        float inv = __fdividef(1.0f, sc);                  // theta / sin theta ...
-        inv = inv * fmaf(-sc, inv, 2.0f);                  // ... refined to full precision (Newton step)
-        const float a0 = 1.0f - alpha;
-        s0 = a0 * sinc_sqrt(a0 * a0 * x) * inv;
-        s1 = alpha * sinc_sqrt(alpha * alpha * x) * inv;
-        if (VEL) {
-            float rs = rsqrtf(m2);                         // 1 / (|q0||q1|), one Newton step as well:
-            rs = rs * fmaf(-0.5f * m2, rs * rs, 1.5f);     // the velocity is summed down the chain
-            vel_scale = 2.0f * fps * inv * rs;
-        }
+    float c, s;
+    if (lg.w <= 0.25f) {
+        const float x = alpha * alpha * lg.w;
+        float p = fmaf(x, -1.9841270e-4f, 8.3333333e-3f);
+        p = fmaf(p, x, -1.6666667e-1f);
+        s = alpha * fmaf(p, x, 1.0f);
+        float g = fmaf(x, 2.4801587e-5f, -1.3888889e-3f);
+        g = fmaf(g, x, 4.1666667e-2f);
+        g = fmaf(g, x, -0.5f);
+        c = fmaf(g, x, 1.0f);
     } else {
-        const float n = sqrtf(n2);
-        const float theta = atan2f(n, d);
-        const float inv = 1.0f / n;
-        s0 = sinf((1.0f - alpha) * theta) * inv;
-        s1 = sinf(alpha * theta) * inv;
-        vel_scale = 2.0f * theta * fps * inv;
+        const float th = sqrtf(lg.w);
+        float sn;
+        sincosf(alpha * th, &sn, &c);
+        s = sn / th;
     }
-    const Quat r = {s0 * q0.w + s1 * q1.w, s0 * q0.x + s1 * q1.x, s0 * q0.y + s1 * q1.y, s0 * q0.z + s1 * q1.z};
-    const float rn = rsqrtf(r.w * r.w + r.x * r.x + r.y * r.y + r.z * r.z);
-    q = {r.w * rn, r.x * rn, r.y * rn, r.z * rn};
-    if (VEL) wl = {vel_scale * c.x, vel_scale * c.y, vel_scale * c.z};
+    const Quat rel = {c, s * lg.x, s * lg.y, s * lg.z};
+    q = qmul(Quat{k0.x, k0.y, k0.z, k0.w}, rel);
+    if (VEL) wl = {fps2 * lg.x, fps2 * lg.y, fps2 * lg.z};
 }
 
 // Squared rotation angle, in [0, pi^2], of the rotation taking frame a to frame b.  Small
@@ -151,22 +177,35 @@ struct Walk {
     Vec3 p, v, w;
 };
 
-// One link of the chain: interpolate joint b between keyframe rows r0/r1 and
-// compose it onto the running transform.  k == 0 is the root.
+// One link of the chain as read from shared memory.
+struct LinkRec {
+    Vec3 off;
+    float mass_frac;
+    int b, flags;
+};
+__device__ __forceinline__ LinkRec ld_link(const float4 *links, int k)
+{
+    const float4 a = links[2 * k];
+    const int4 i = *reinterpret_cast<const int4 *>(links + 2 * k + 1);
+    return {{a.x, a.y, a.z}, a.w, i.x, i.y};
+}
+
+// Compose the interpolated joint onto the running transform.  k == 0 is the root, whose position is the
+// lerp of the row's root position along its displacement.
 template <bool VEL>
-__device__ __forceinline__ void joint_compose(const SkelDev &sk, const float4 *r0, const float4 *r1, float alpha,
-                                              float fps, int b, int k, Walk &s, Quat ql, Vec3 wl)
+__device__ __forceinline__ void joint_compose(const float4 *r0, float alpha, float fps, Vec3 off, int k, Walk &s,
+                                              Quat ql, Vec3 wl)
 {
     if (k == 0) {
-        const float4 a = __ldg(r0), c = __ldg(r1);
+        const float4 a = __ldg(r0), d = __ldg(r0 + 1);
         s.q = ql;
-        s.p = {a.x + alpha * (c.x - a.x), a.y + alpha * (c.y - a.y), a.z + alpha * (c.z - a.z)};
+        s.p = {fmaf(alpha, d.x, a.x), fmaf(alpha, d.y, a.y), fmaf(alpha, d.z, a.z)};
         if (VEL) {
-            s.v = {(c.x - a.x) * fps, (c.y - a.y) * fps, (c.z - a.z) * fps};
+            s.v = {d.x * fps, d.y * fps, d.z * fps};
             s.w = qrot(ql, wl);
         }
     } else {
-        const Vec3 arm = qrot(s.q, Vec3{sk.off[b][0], sk.off[b][1], sk.off[b][2]});
+        const Vec3 arm = qrot(s.q, off);
         if (VEL) s.v = s.v + cross(s.w, arm);
         s.p = s.p + arm;
         s.q = qmul(s.q, ql);
@@ -174,12 +213,21 @@ __device__ __forceinline__ void joint_compose(const SkelDev &sk, const float4 *r
     }
 }
 
-template <bool VEL>
-__device__ __forceinline__ void joint_step(const SkelDev &sk, const float4 *r0, const float4 *r1, Quat k0, Quat k1,
-                                           float alpha, float fps, int b, int k, Walk &s, Quat &ql, Vec3 &wl)
+// Keyframe words of joint b in row r0: the rotation and the log of the step to the next keyframe.
+struct KeyPair {
+    float4 a, b;
+};
+__device__ __forceinline__ KeyPair ld_keys(const float4 *r0, int b)
 {
-    slerp_joint<VEL>(k0, k1, alpha, fps, ql, wl);
-    joint_compose<VEL>(sk, r0, r1, alpha, fps, b, k, s, ql, wl);
+    return {__ldg(r0 + 2 + 2 * b), __ldg(r0 + 3 + 2 * b)};
+}
+
+template <bool VEL>
+__device__ __forceinline__ void joint_step(const float4 *r0, const KeyPair &key, float alpha, float fps, Vec3 off, int k,
+                                           Walk &s, Quat &ql, Vec3 &wl)
+{
+    slerp_joint<VEL>(key.a, key.b, alpha, 2.0f * fps, ql, wl);
+    joint_compose<VEL>(r0, alpha, fps, off, k, s, ql, wl);
 }
 
 // Motion randomisation of a reset state: three standard normals of Philox counter
@@ -289,28 +337,17 @@ __device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
     return q;
 }
 
-// Body-state loads: `col` points at this thread's env in row 0 of the array, so a component is
-// one per-thread pointer plus a warp-uniform row offset.
-__device__ __forceinline__ Quat ld_sim_quat(const float *col, size_t st, int b)
+// Body-state loads.  Element (row, env) of an array lies at row * stride + env; the offsets are 32-bit
+// (the launcher checks that the arrays are smaller than 2^31 elements), `o` is the offset of the body's
+// first row at this thread's env.
+__device__ __forceinline__ Quat ld_sim_quat(const float *base, uint32_t o, uint32_t st)
 {
-    const float *p = col + (size_t)(4 * b) * st;
-    return {p[0], p[st], p[2 * st], p[3 * st]};
+    return {base[o], base[o + st], base[o + 2 * st], base[o + 3 * st]};
 }
-__device__ __forceinline__ Vec3 ld_sim_vec(const float *col, size_t st, int b)
+__device__ __forceinline__ Vec3 ld_sim_vec(const float *base, uint32_t o, uint32_t st)
 {
-    const float *p = col + (size_t)(3 * b) * st;
-    return {p[0], p[st], p[2 * st]};
+    return {base[o], base[o + st], base[o + 2 * st]};
 }
-
-// Keyframe quaternions of joint b in the two bracketing rows.
-struct KeyPair {
-    float4 a, b;
-};
-__device__ __forceinline__ KeyPair ld_keys(const float4 *r0, const float4 *r1, int b)
-{
-    return {__ldg(r0 + 1 + b), __ldg(r1 + 1 + b)};
-}
-__device__ __forceinline__ Quat as_quat(float4 v) { return {v.x, v.y, v.z, v.w}; }
 
 // Kernel body.  The observation row is assembled in two halves that reuse the same shared
 // memory: columns [0, c1) -- the body blocks and, if 15 J is not a multiple of 4, the phase and
@@ -344,7 +381,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     float *row2 = tile + (size_t)lane * S2;
     const int len = sk.chain_len[c];
     const int first_own = sk.chain_first_own[c];
-    const int RS = J + 1;
+    const int RS = 2 + 2 * J;
+
+    // this chain's link records: global -> shared, private to the warp
+    float4 *links = reinterpret_cast<float4 *>(part + (size_t)kPartials * C * kTile) + 2 * sk.link_start[c];
+    for (int i = lane; i < 2 * len; i += 32) links[i] = __ldg(P.links + 2 * sk.link_start[c] + i);
+    __syncwarp();
 
     if (c == 0)
         for (int i = 15 * J; i < S1; ++i) row1[i] = 0.0f;   // columns between the body blocks and the stride
@@ -354,6 +396,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     ClipMeta cm = {2, 1.0f, 1.0f, 0};
     Heading H = {0.0f, 0.0f, 1.0f, 0.0f};
     float root_z = 0.0f;
+    const uint32_t st = (uint32_t)P.stride, e32 = (uint32_t)envc;
 
     // ---- pass A: reference at the advanced time, errors against the simulated state,
     //      observation entries of the simulated bodies
@@ -368,13 +411,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         int frame;
         float alpha;
         lookup(cm, t1, frame, alpha);
-        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
-        KeyPair keys = ld_keys(r0, r1, sk.chain[c][0]);
+        const float4 *r0 = P.frames + (size_t)frame * RS;
+        LinkRec L = ld_link(links, 0);
+        KeyPair keys = ld_keys(r0, L.b);
 
-        const size_t st = (size_t)P.stride;
-        const float *pos_e = P.pos + envc, *quat_e = P.quat + envc, *lin_e = P.lin + envc, *ang_e = P.ang + envc;
-        const Quat q_root = sanitize(ld_sim_quat(quat_e, st, 0), P.status);
-        const Vec3 p_root = ld_sim_vec(pos_e, st, 0);
+        const Quat q_root = sanitize(ld_sim_quat(P.quat, e32, st), P.status);
+        const Vec3 p_root = ld_sim_vec(P.pos, e32, st);
         H = make_heading(q_root, p_root);
         root_z = p_root.z;
 
@@ -385,25 +427,32 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         Quat qa = {1, 0, 0, 0};                      // simulated state of the previous body of the chain
         Vec3 wa = {0, 0, 0};
         if (first_own > 0) {
-            const int a = sk.chain[c][first_own - 1];
-            qa = sanitize(ld_sim_quat(quat_e, st, a), P.status);
-            wa = ld_sim_vec(ang_e, st, a);
+            const uint32_t a = (uint32_t)ld_link(links, first_own - 1).b;
+            qa = sanitize(ld_sim_quat(P.quat, 4 * a * st + e32, st), P.status);
+            wa = ld_sim_vec(P.ang, 3 * a * st + e32, st);
         }
         for (int k = 0; k < len; ++k) {
-            const int b = sk.chain[c][k];
-            const bool own = k >= first_own;
+            const int b = L.b;
+            const bool own = L.flags & LINK_OWN;
+            const bool ee = L.flags & LINK_EE;
+            const Vec3 off = L.off;
+            const float mf = L.mass_frac;
             SimBody sim;
             if (own) {                                // issue the loads before the interpolation math
-                sim.q = ld_sim_quat(quat_e, st, b);
-                sim.p = ld_sim_vec(pos_e, st, b);
-                sim.v = ld_sim_vec(lin_e, st, b);
-                sim.w = ld_sim_vec(ang_e, st, b);
+                const uint32_t o3 = 3 * (uint32_t)b * st + e32;
+                sim.q = ld_sim_quat(P.quat, 4 * (uint32_t)b * st + e32, st);
+                sim.p = ld_sim_vec(P.pos, o3, st);
+                sim.v = ld_sim_vec(P.lin, o3, st);
+                sim.w = ld_sim_vec(P.ang, o3, st);
             }
             const KeyPair cur = keys;
-            if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);     // next joint's keyframes in flight
+            if (k + 1 < len) {                        // next joint's link and keyframe words in flight
+                L = ld_link(links, k + 1);
+                keys = ld_keys(r0, L.b);
+            }
             Quat ql;
             Vec3 wl;
-            joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cm.fps, b, k, s, ql, wl);
+            joint_step<true>(r0, cur, alpha, cm.fps, off, k, s, ql, wl);
             if (own) {
                 sim.q = sanitize(sim.q, P.status);
                 Quat ql_sim = sim.q;
@@ -420,13 +469,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                 const float dp2 = dot(dp, dp);
                 acc[0] += th_sq;
                 acc[1] += dot(dwl, dwl);
-                if ((sk.ee_mask >> b) & 1u) {
+                if (ee) {
                     acc[2] += dp2;
                     acc[3] += rel_angle_sq(s.q, sim.q);
                 }
                 acc[4] += dp2;
                 acc[5] += dot(dv, dv);
-                const float mf = sk.mass_frac[b];
                 acc[6] += mf * dp.x;
                 acc[7] += mf * dp.y;
                 acc[8] += mf * dp.z;
@@ -522,36 +570,41 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         int frame;
         float alpha;
         lookup(cmc, t_cur, frame, alpha);
-        const float4 *r0 = P.frames + (size_t)frame * RS, *r1 = r0 + RS;
-        KeyPair keys = ld_keys(r0, r1, sk.chain[c][0]);
+        const float4 *r0 = P.frames + (size_t)frame * RS;
+        LinkRec L = ld_link(links, 0);
+        KeyPair keys = ld_keys(r0, L.b);
         Walk s;
         Heading Hn = H;
         for (int k = 0; k < len; ++k) {
-            const int b = sk.chain[c][k];
+            const int b = L.b;
+            const bool own = L.flags & LINK_OWN;
+            const Vec3 off = L.off;
             const KeyPair cur = keys;
-            if (k + 1 < len) keys = ld_keys(r0, r1, sk.chain[c][k + 1]);
+            if (k + 1 < len) {
+                L = ld_link(links, k + 1);
+                keys = ld_keys(r0, L.b);
+            }
             Quat ql;
             Vec3 wl;
             if (OPT && P.reset_noise_std > 0.0f) {
                 // motion randomisation: the joint turns by a small random rotation in its own frame and
                 // the root is shifted; every chain that walks a shared body draws the same numbers
-                slerp_joint<true>(as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, ql, wl);
+                slerp_joint<true>(cur.a, cur.b, alpha, 2.0f * cmc.fps, ql, wl);
                 ql = qmul(ql, reset_noise_quat(P, envc, b));
-                joint_compose<true>(sk, r0, r1, alpha, cmc.fps, b, k, s, ql, wl);
+                joint_compose<true>(r0, alpha, cmc.fps, off, k, s, ql, wl);
                 if (k == 0) s.p = s.p + reset_noise_shift(P, envc, sk.J);
             } else {
-                joint_step<true>(sk, r0, r1, as_quat(cur.a), as_quat(cur.b), alpha, cmc.fps, b, k, s, ql, wl);
+                joint_step<true>(r0, cur, alpha, cmc.fps, off, k, s, ql, wl);
             }
             if (k == 0) Hn = make_heading(s.q, s.p);
-            if (k >= first_own && reset) {
+            if (own && reset) {
                 body_obs(Hn, s.q, s.p, s.v, s.w, row1, b);
                 if (!RESET_ALL && P.write_back && valid) {
-                    const size_t st = (size_t)P.stride;
-                    P.pos[(3 * b + 0) * st + env] = s.p.x; P.pos[(3 * b + 1) * st + env] = s.p.y; P.pos[(3 * b + 2) * st + env] = s.p.z;
-                    P.quat[(4 * b + 0) * st + env] = s.q.w; P.quat[(4 * b + 1) * st + env] = s.q.x;
-                    P.quat[(4 * b + 2) * st + env] = s.q.y; P.quat[(4 * b + 3) * st + env] = s.q.z;
-                    P.lin[(3 * b + 0) * st + env] = s.v.x; P.lin[(3 * b + 1) * st + env] = s.v.y; P.lin[(3 * b + 2) * st + env] = s.v.z;
-                    P.ang[(3 * b + 0) * st + env] = s.w.x; P.ang[(3 * b + 1) * st + env] = s.w.y; P.ang[(3 * b + 2) * st + env] = s.w.z;
+                    const uint32_t o3 = 3 * (uint32_t)b * st + e32, o4 = 4 * (uint32_t)b * st + e32;
+                    P.pos[o3] = s.p.x; P.pos[o3 + st] = s.p.y; P.pos[o3 + 2 * st] = s.p.z;
+                    P.quat[o4] = s.q.w; P.quat[o4 + st] = s.q.x; P.quat[o4 + 2 * st] = s.q.y; P.quat[o4 + 3 * st] = s.q.z;
+                    P.lin[o3] = s.v.x; P.lin[o3 + st] = s.v.y; P.lin[o3 + 2 * st] = s.v.z;
+                    P.ang[o3] = s.w.x; P.ang[o3 + st] = s.w.y; P.ang[o3 + 2 * st] = s.w.z;
                 }
             }
         }
@@ -564,15 +617,11 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     int frame_t;
     float alpha_t;
     lookup(cmc, t_tgt, frame_t, alpha_t);
-    const float4 *rt0 = P.frames + (size_t)frame_t * RS, *rt1 = rt0 + RS;
+    const float4 *rt0 = P.frames + (size_t)frame_t * RS;
     const float phase = t_cur / cmc.dur;
     if (c == 0 && 15 * J < c1) {
-        Walk s;
-        Quat ql;
-        Vec3 wl;
-        const KeyPair kp = ld_keys(rt0, rt1, 0);
-        joint_step<false>(sk, rt0, rt1, as_quat(kp.a), as_quat(kp.b), alpha_t, cmc.fps, 0, 0, s, ql, wl);
-        const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
+        const float4 a = __ldg(rt0), d = __ldg(rt0 + 1);
+        const Vec3 tp = H.turn(Vec3{fmaf(alpha_t, d.x, a.x) - H.ox, fmaf(alpha_t, d.y, a.y) - H.oy, fmaf(alpha_t, d.z, a.z)});
         row1[15 * J] = phase;
         if (15 * J + 1 < c1) row1[15 * J + 1] = tp.x;
         if (15 * J + 2 < c1) row1[15 * J + 2] = tp.y;
@@ -605,16 +654,22 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             for (int i = D_ext - c1; i < S2; ++i) row2[i] = 0.0f;
             if (15 * J >= c1) row2[15 * J - c1] = phase;
         }
-        KeyPair keys = ld_keys(rt0, rt1, sk.chain[c][0]);
+        LinkRec L = ld_link(links, 0);
+        KeyPair keys = ld_keys(rt0, L.b);
         Walk s;
         for (int k = 0; k < len; ++k) {
-            const int b = sk.chain[c][k];
+            const int b = L.b;
+            const bool own = L.flags & LINK_OWN;
+            const Vec3 off = L.off;
             const KeyPair cur = keys;
-            if (k + 1 < len) keys = ld_keys(rt0, rt1, sk.chain[c][k + 1]);
+            if (k + 1 < len) {
+                L = ld_link(links, k + 1);
+                keys = ld_keys(rt0, L.b);
+            }
             Quat ql;
             Vec3 wl;
-            joint_step<false>(sk, rt0, rt1, as_quat(cur.a), as_quat(cur.b), alpha_t, cmc.fps, b, k, s, ql, wl);
-            if (k >= first_own) {
+            joint_step<false>(rt0, cur, alpha_t, cmc.fps, off, k, s, ql, wl);
+            if (own) {
                 const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
                 const Vec3 tt = H.turn(qcol_x(s.q)), tm = H.turn(qcol_z(s.q));
                 const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
@@ -636,15 +691,16 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                 int frame_f;
                 float alpha_f;
                 lookup(cmc, t_f, frame_f, alpha_f);
-                const float4 *rf0 = P.frames + (size_t)frame_f * RS, *rf1 = rf0 + RS;
+                const float4 *rf0 = P.frames + (size_t)frame_f * RS;
                 Walk sf;
                 for (int k = 0; k < len; ++k) {
-                    const int b = sk.chain[c][k];
-                    const KeyPair kp = ld_keys(rf0, rf1, b);
+                    const LinkRec Lf = ld_link(links, k);
+                    const int b = Lf.b;
+                    const KeyPair kp = ld_keys(rf0, b);
                     Quat ql;
                     Vec3 wl;
-                    joint_step<false>(sk, rf0, rf1, as_quat(kp.a), as_quat(kp.b), alpha_f, cmc.fps, b, k, sf, ql, wl);
-                    if (k >= first_own && ((sk.ee_mask >> b) & 1u)) {
+                    joint_step<false>(rf0, kp, alpha_f, cmc.fps, Lf.off, k, sf, ql, wl);
+                    if ((Lf.flags & LINK_OWN) && (Lf.flags & LINK_EE)) {
                         const Vec3 tp = H.turn(Vec3{sf.p.x - H.ox, sf.p.y - H.oy, sf.p.z});
                         const Vec3 tt = H.turn(qcol_x(sf.q)), tm = H.turn(qcol_z(sf.q));
                         const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
@@ -712,18 +768,30 @@ void launch_one(const EnvKernelParams &p, dim3 grid, dim3 block, size_t smem, cu
 
 }  // namespace
 
-size_t env_kernel_smem_bytes(int J, int n_chains, int extra_cols) { return smem_floats(J, n_chains, extra_cols) * sizeof(float); }
+size_t env_kernel_smem_bytes(int J, int n_chains, int n_links, int extra_cols)
+{
+    return smem_floats(J, n_chains, n_links, extra_cols) * sizeof(float);
+}
 
 cudaError_t env_kernel_prepare(size_t smem)
 {
-    static bool done = false;
-    if (done) return cudaSuccess;
-    cudaError_t e = prepare_one<false, false>(smem);
-    if (e == cudaSuccess) e = prepare_one<true, false>(smem);
-    if (e == cudaSuccess) e = prepare_one<false, true>(smem);
-    if (e == cudaSuccess) e = prepare_one<true, true>(smem);
-    done = e == cudaSuccess;
-    return e;
+    static DeviceOnce once;
+    return once.run([&] {
+        cudaError_t e = prepare_one<false, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<true, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<false, true>(smem);
+        if (e == cudaSuccess) e = prepare_one<true, true>(smem);
+        return e;
+    });
+}
+
+cudaError_t launch_clip_table(const float *root_pos, const float *local_quat, const uint8_t *last, int64_t rows, int J,
+                              float4 *frames, cudaStream_t stream)
+{
+    const long long n = (long long)rows * (J + 1);
+    clip_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(root_pos, local_quat, last, (long long)rows, J, frames);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)

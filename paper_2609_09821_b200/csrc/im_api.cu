@@ -9,6 +9,22 @@
 
 namespace im {
 std::atomic<uint64_t> g_launches{0};
+
+int device_sm_count()
+{
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        int cc_major = 0;
+        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (cc_major != 10) n = -1;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n > 0 ? n : 0;
+}
 }
 
 using namespace im;
@@ -63,12 +79,8 @@ im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *off
     std::memset(s, 0, sizeof(*s));
     SkelDev &d = s->dev;
     d.J = J;
-    for (int j = 0; j < J; ++j) {
-        d.parent[j] = parents[j];
-        for (int c = 0; c < 3; ++c) d.off[j][c] = j == 0 ? 0.0f : offsets[3 * j + c];
-        d.mass_frac[j] = (float)((masses ? (double)masses[j] : 1.0) / msum);
-    }
     // one root-to-leaf path per leaf; a shared body belongs to the first path that contains it
+    uint8_t chain[IM_MAX_BODIES][IM_MAX_BODIES];
     {
         bool has_child[IM_MAX_BODIES] = {false}, owned[IM_MAX_BODIES] = {false};
         for (int j = 1; j < J; ++j) has_child[parents[j]] = true;
@@ -79,11 +91,11 @@ im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *off
             for (int a = leaf; a > 0; a = parents[a]) ++depth;
             d.chain_len[c] = (uint8_t)(depth + 1);
             int a = leaf;
-            for (int k = depth; k >= 0; --k) { d.chain[c][k] = (uint8_t)a; a = a > 0 ? parents[a] : 0; }
+            for (int k = depth; k >= 0; --k) { chain[c][k] = (uint8_t)a; a = a > 0 ? parents[a] : 0; }
             int first = 0;
-            while (first <= depth && owned[d.chain[c][first]]) ++first;
+            while (first <= depth && owned[chain[c][first]]) ++first;
             d.chain_first_own[c] = (uint8_t)first;
-            for (int k = first; k <= depth; ++k) owned[d.chain[c][k]] = true;
+            for (int k = first; k <= depth; ++k) owned[chain[c][k]] = true;
         }
     }
     if (ee_ids && n_ee > 0) {
@@ -94,6 +106,18 @@ im_status im_create_skeleton(int32_t J, const int32_t *parents, const float *off
         d.ee_mask = ~has_child & (J == 32 ? 0xffffffffu : ((1u << J) - 1u));
     }
     s->n_ee = __builtin_popcount(d.ee_mask);
+    // the chains' links in the order the env kernel walks them
+    for (int c = 0; c < d.n_chains; ++c) {
+        d.link_start[c] = (uint16_t)d.n_links;
+        for (int k = 0; k < d.chain_len[c]; ++k) {
+            const int b = chain[c][k];
+            ChainLink &L = s->links[d.n_links++];
+            for (int i = 0; i < 3; ++i) L.off[i] = b == 0 ? 0.0f : offsets[3 * b + i];
+            L.mass_frac = (float)((masses ? (double)masses[b] : 1.0) / msum);
+            L.b = b;
+            L.flags = (k >= d.chain_first_own[c] ? LINK_OWN : 0) | (((d.ee_mask >> b) & 1u) ? LINK_EE : 0);
+        }
+    }
     *out = s;
     return IM_OK;
 }
@@ -131,27 +155,33 @@ im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_fra
         cl->min_dur = std::fmin(cl->min_dur, cl->meta[c].dur);
         start += n_frames[c];
     }
-    // Packed rows of (1 + J) float4: (x, y, z, 0), q_0 .. q_{J-1}.  Quaternions are stored as
-    // given: every formula that consumes them is invariant to their (<= 1e-3) scale error.
-    const size_t RS = (size_t)J + 1;
-    std::vector<float4> host((size_t)rows * RS);
-    for (int64_t r = 0; r < rows; ++r) {
-        host[r * RS] = make_float4(root_pos[3 * r], root_pos[3 * r + 1], root_pos[3 * r + 2], 0.0f);
-        for (int j = 0; j < J; ++j) {
-            const float *q = local_quat + 4 * (r * J + j);
-            host[r * RS + 1 + j] = make_float4(q[0], q[1], q[2], q[3]);
-        }
-    }
+    // The table rows (see clip_table_kernel) are built on the device from copies of the caller's arrays.
+    std::vector<uint8_t> last((size_t)rows, 0);
+    for (int c = 0; c < C; ++c) last[(size_t)cl->meta[c].start + n_frames[c] - 1] = 1;
+    const size_t RS = (size_t)clip_row_stride(J);
+    float *d_root = nullptr, *d_quat = nullptr;
+    uint8_t *d_last = nullptr;
     cudaGetDevice(&cl->device);
-    if (cudaMalloc(&cl->d_frames, host.size() * sizeof(float4)) != cudaSuccess ||
-        cudaMalloc(&cl->d_meta, C * sizeof(ClipMeta)) != cudaSuccess) {
-        im_destroy_clips(cl);
-        return IM_ERR_ALLOC;
+    // (one extra row of zeros so that the last frame's "next" reads stay inside the buffers)
+    const size_t root_b = (size_t)(rows + 1) * 3 * sizeof(float), quat_b = (size_t)(rows + 1) * J * 4 * sizeof(float);
+    bool ok = cudaMalloc(&cl->d_frames, (size_t)rows * RS * sizeof(float4)) == cudaSuccess &&
+              cudaMalloc(&cl->d_meta, C * sizeof(ClipMeta)) == cudaSuccess && cudaMalloc(&d_root, root_b) == cudaSuccess &&
+              cudaMalloc(&d_quat, quat_b) == cudaSuccess && cudaMalloc(&d_last, (size_t)rows) == cudaSuccess;
+    im_status st = ok ? IM_OK : IM_ERR_ALLOC;
+    if (ok) {
+        ok = cudaMemset(d_root, 0, root_b) == cudaSuccess && cudaMemset(d_quat, 0, quat_b) == cudaSuccess &&
+             cudaMemcpy(d_root, root_pos, (size_t)rows * 3 * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(d_quat, local_quat, (size_t)rows * J * 4 * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(d_last, last.data(), (size_t)rows, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(cl->d_meta, cl->meta.data(), C * sizeof(ClipMeta), cudaMemcpyHostToDevice) == cudaSuccess &&
+             launch_clip_table(d_root, d_quat, d_last, rows, J, cl->d_frames, nullptr) == cudaSuccess &&
+             cudaDeviceSynchronize() == cudaSuccess;
+        if (!ok) st = IM_ERR_CUDA;
     }
-    if (cudaMemcpy(cl->d_frames, host.data(), host.size() * sizeof(float4), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(cl->d_meta, cl->meta.data(), C * sizeof(ClipMeta), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(d_root); cudaFree(d_quat); cudaFree(d_last);
+    if (st != IM_OK) {
         im_destroy_clips(cl);
-        return IM_ERR_CUDA;
+        return st;
     }
     *out = cl;
     return IM_OK;
@@ -188,7 +218,7 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     if (!e) return IM_ERR_ALLOC;
     std::memset(e, 0, sizeof(*e));
     e->skel = skel; e->clips = clips; e->cfg = *cfg; e->stream = (cudaStream_t)cuda_stream; e->D = D;
-    e->smem_bytes = env_kernel_smem_bytes(J, skel->dev.n_chains, 0);
+    e->smem_bytes = env_kernel_smem_bytes(J, skel->dev.n_chains, skel->dev.n_links, 0);
     e->n_future = 1;
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
@@ -198,9 +228,14 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     if (env_kernel_prepare((size_t)max_smem) != cudaSuccess) { delete e; return IM_ERR_CUDA; }
     const size_t n = (size_t)cfg->n_envs;
     if (cudaMalloc(&e->d_clip_id, n * 4) != cudaSuccess || cudaMalloc(&e->d_t, n * 4) != cudaSuccess ||
-        cudaMalloc(&e->d_ep_len, n * 4) != cudaSuccess || cudaMalloc(&e->d_status, 4) != cudaSuccess) {
+        cudaMalloc(&e->d_ep_len, n * 4) != cudaSuccess || cudaMalloc(&e->d_status, 4) != cudaSuccess ||
+        cudaMalloc(&e->d_links, (size_t)skel->dev.n_links * sizeof(ChainLink)) != cudaSuccess) {
         im_env_destroy(e);
         return IM_ERR_ALLOC;
+    }
+    if (cudaMemcpy(e->d_links, skel->links, (size_t)skel->dev.n_links * sizeof(ChainLink), cudaMemcpyHostToDevice) != cudaSuccess) {
+        im_env_destroy(e);
+        return IM_ERR_CUDA;
     }
     cudaMemsetAsync(e->d_clip_id, 0, n * 4, e->stream);
     cudaMemsetAsync(e->d_t, 0, n * 4, e->stream);
@@ -213,7 +248,7 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
 void im_env_destroy(im_env *e)
 {
     if (!e) return;
-    cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status);
+    cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status); cudaFree(e->d_links);
     cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
     cudaFree(e->d_action); cudaFree(e->d_flags);
     cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
@@ -231,6 +266,7 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     std::memset(&p, 0, sizeof(p));
     p.sk = e->skel->dev;
     p.frames = e->clips->d_frames;
+    p.links = e->d_links;
     p.meta = e->clips->d_meta;
     p.C = e->clips->C;
     p.N = e->cfg.n_envs;
@@ -280,6 +316,7 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim, float 
     if (!aligned16(obs_out) || !aligned16(sim->pos) || !aligned16(sim->quat) || !aligned16(sim->linvel) ||
         !aligned16(sim->angvel) || (sim->comp_stride & 3))
         return IM_ERR_INVALID_ARG;
+    if (sim->comp_stride * 4 * (int64_t)e->skel->dev.J >= (int64_t)1 << 31) return IM_ERR_UNSUPPORTED;   // the kernel indexes with 32 bits
     EnvKernelParams p;
     fill_params(e, step, p);
     p.pos = sim->pos; p.quat = sim->quat; p.lin = sim->linvel; p.ang = sim->angvel;
@@ -506,7 +543,7 @@ im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim,
     const int extra = (n_future - 1) * 9 * e->skel->n_ee + act_dim;
     const int D = 24 * J + 1 + extra;
     if (e->cfg.ld_obs < D) return IM_ERR_INVALID_ARG;
-    const size_t smem = env_kernel_smem_bytes(J, e->skel->dev.n_chains, extra);
+    const size_t smem = env_kernel_smem_bytes(J, e->skel->dev.n_chains, e->skel->dev.n_links, extra);
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);

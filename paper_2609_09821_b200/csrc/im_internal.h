@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "../../include/im.h"
@@ -19,25 +20,57 @@ struct ClipMeta {
     int32_t start;    // first row of the clip in the packed keyframe table
 };
 
+// One link of a kinematic chain as the env kernel reads it from shared memory (two 16-byte words).
+struct ChainLink {
+    float off[3];        // origin of the body in its parent's frame
+    float mass_frac;     // m_b / sum m
+    int32_t b;           // body index
+    int32_t flags;       // LINK_OWN: this chain scores the body and writes its observation entries; LINK_EE: end effector
+    int32_t pad[2];
+};
+constexpr int LINK_OWN = 1, LINK_EE = 2;
+constexpr int IM_MAX_LINKS = 288;          // sum of chain lengths for any tree of up to 32 bodies (<= 16 x 17)
+
 // Skeleton as the kernels see it (passed by value inside the kernel parameters).
+// Kinematic chains: one root-to-leaf path per leaf.  A body shared by several paths is owned by the first of
+// them; within a path the owned bodies are a suffix starting at chain_first_own.  The links of all chains lie
+// in one device array, chain c at [link_start[c], link_start[c] + chain_len[c]).
 struct SkelDev {
     int32_t J;
     uint32_t ee_mask;
-    int32_t parent[IM_MAX_BODIES];
-    float off[IM_MAX_BODIES][3];
-    float mass_frac[IM_MAX_BODIES];                    // m_j / sum m
-    // Kinematic chains: one root-to-leaf path per leaf.  A body shared by several paths is owned
-    // by the first of them; within a path the owned bodies are a suffix starting at chain_first_own.
     int32_t n_chains;
+    int32_t n_links;
     uint8_t chain_len[IM_MAX_BODIES];
     uint8_t chain_first_own[IM_MAX_BODIES];
-    uint8_t chain[IM_MAX_BODIES][IM_MAX_BODIES];       // chain[c][0..chain_len[c]) = root .. leaf
+    uint16_t link_start[IM_MAX_BODIES];
 };
+
+// One-time kernel set-up (shared-memory opt-in, SM count) is per device: run `fn` once for the current device.
+constexpr int kMaxDevices = 64;
+struct DeviceOnce {
+    std::mutex m;
+    bool done[kMaxDevices] = {};
+    template <typename F> cudaError_t run(F fn)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(m);
+        if (done[dev]) return cudaSuccess;
+        e = fn();
+        done[dev] = e == cudaSuccess;
+        return e;
+    }
+};
+// Number of SMs of the current device (cached per device).
+int device_sm_count();
 
 struct EnvKernelParams {
     SkelDev sk;
     // clip library
-    const float4 *frames;     // [rows][1+J] float4: (x,y,z,0), q_0 .. q_{J-1}
+    const float4 *frames;     // [rows][2+2J] float4, see clip_table_kernel
+    const float4 *links;      // [n_links][2]: the chains' ChainLink records
     const ClipMeta *meta;     // [C]
     int32_t C;
     // configuration
@@ -79,6 +112,7 @@ struct EnvKernelParams {
 struct im_skeleton {
     im::SkelDev dev;
     int32_t n_ee;
+    im::ChainLink links[im::IM_MAX_LINKS];
 };
 
 struct im_clips {
@@ -102,6 +136,7 @@ struct im_env {
     float *d_t;
     int32_t *d_ep_len;
     uint32_t *d_status;
+    float4 *d_links;       // the skeleton's chain links on the env's device
     int D;                 // observation width: 24J + 1 plus the extension columns
     size_t smem_bytes;
     uint16_t *d_obs_bf16;  // attached policy's bf16 input rows (null when detached)
@@ -121,7 +156,11 @@ struct im_env {
 
 // Launchers implemented in the kernel translation units.
 namespace im {
-size_t env_kernel_smem_bytes(int J, int n_chains, int extra_cols);
+size_t env_kernel_smem_bytes(int J, int n_chains, int n_links, int extra_cols);
+// clip table rows from the caller's keyframes (device copies of the host arrays); last[r] marks a clip's final frame
+cudaError_t launch_clip_table(const float *root_pos, const float *local_quat, const uint8_t *last, int64_t rows, int J,
+                              float4 *frames, cudaStream_t stream);
+inline int clip_row_stride(int J) { return 2 + 2 * J; }
 cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
 // simulator-native (array of structures) body states <-> component rows [13 J][stride]

@@ -1170,12 +1170,11 @@ template <int BLOCK_N, bool BWD = false>
 cudaError_t launch_hidden(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
-    static bool prepared = false;
-    if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, false, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemLimit);
+    static DeviceOnce once;                      // the attribute is per device
+    {
+        const cudaError_t e = once.run([] { return cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, false, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit); });
         if (e != cudaSuccess) return e;
-        prepared = true;
     }
     GemmParams gp = gp_in;
     gp.stages = Plan::stages_for(Plan::hidden_epi_bytes(BWD));
@@ -1194,12 +1193,11 @@ template <int BLOCK_N>
 cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
-    static bool prepared = false;
-    if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemLimit);
+    static DeviceOnce once;                      // the attribute is per device
+    {
+        const cudaError_t e = once.run([] { return cudaFuncSetAttribute(linear_tc_hidden_kernel<BLOCK_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit); });
         if (e != cudaSuccess) return e;
-        prepared = true;
     }
     GemmParams gp = gp_in;
     gp.stages = Plan::stages_for(Plan::hidden_epi_bytes());
@@ -1215,12 +1213,11 @@ cudaError_t launch_hidden_mn(const TcLayer &L, const GemmParams &gp_in, int n_sm
 template <bool BWD, bool MN = false>
 cudaError_t launch_hidden_pair(const TcLayer &L, const GemmParams &gp, int n_sm, cudaStream_t stream)
 {
-    static bool prepared = false;
-    if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD, MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)pair_smem_bytes(BWD));
+    static DeviceOnce once;                      // the attribute is per device
+    {
+        const cudaError_t e = once.run([] { return cudaFuncSetAttribute(linear_tc_hidden_pair_kernel<BWD, MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)pair_smem_bytes(BWD)); });
         if (e != cudaSuccess) return e;
-        prepared = true;
     }
     const int tiles = ((gp.M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * gp.n_tiles_n * (MN ? gp.n_batches : 1);
     const int pairs = tiles < n_sm / 2 ? tiles : n_sm / 2;
@@ -1234,12 +1231,11 @@ template <int BLOCK_N>
 cudaError_t launch_head(const TcLayer &L, const GemmParams &gp_in, int n_sm, cudaStream_t stream)
 {
     using Plan = SmemPlan<BLOCK_N>;
-    static bool prepared = false;
-    if (!prepared) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_head_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemLimit);
+    static DeviceOnce once;                      // the attribute is per device
+    {
+        const cudaError_t e = once.run([] { return cudaFuncSetAttribute(linear_tc_head_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemLimit); });
         if (e != cudaSuccess) return e;
-        prepared = true;
     }
     GemmParams gp = gp_in;
     const int epi = Plan::head_epi_bytes(gp.N);
@@ -1432,14 +1428,8 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
                   const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches, const void *mask,
                   int64_t ld_mask, float *colsum_partial, int ld_partial)
 {
-    static int n_sm = 0;
-    if (!n_sm) {
-        int dev = 0, cc_major = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    }
+    const int n_sm = device_sm_count();          // 0 unless the current device is an sm_100 part
+    if (n_sm <= 0 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
     TcLayer L;
     L.N = N; L.K = K; L.Kpad = K;
     L.block_n = pick_block_n(N, false);
@@ -1473,14 +1463,8 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
 im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int R, int Mo, int No,
                      int slices, int c_pitch, const float *bias, uint32_t *status, cudaStream_t stream)
 {
-    static int n_sm = 0;
-    if (!n_sm) {
-        int dev = 0, cc_major = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    }
+    const int n_sm = device_sm_count();          // 0 unless the current device is an sm_100 part
+    if (n_sm <= 0 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
     TcLayer L;
     L.N = No; L.K = R / slices; L.Kpad = L.K;
     // wide outputs take 256-column tiles even when that leaves a ragged last tile (640 columns: three tiles,
@@ -1521,14 +1505,8 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
 im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, int M, int N, int K, const float *bias,
                        float *mean_out, uint32_t *status, cudaStream_t stream)
 {
-    static int n_sm = 0;
-    if (!n_sm) {
-        int dev = 0, cc_major = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-        if (cc_major != 10 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    }
+    const int n_sm = device_sm_count();          // 0 unless the current device is an sm_100 part
+    if (n_sm <= 0 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
     TcLayer L;
     L.N = N; L.K = K; L.Kpad = K;
     L.block_n = pick_block_n(N, true);

@@ -561,24 +561,20 @@ im_status im_ppo_loss(const im_ppo_config *cfg, int64_t M, int32_t A, const im_p
     const long long n_tiles = bulk_ok ? M / T : 0;
     int grid_bulk = 0;
     if (n_tiles > 0) {
-        static int n_sm = 0, max_smem = 0;
-        if (!n_sm) {
-            int dev = 0;
-            cudaGetDevice(&dev);
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-            cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        }
+        int dev = 0, n_sm = 0, max_smem = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
         const size_t smem = 2 * (size_t)stage_floats(A, T) * sizeof(float);
         p.row_begin = 0; p.partial_begin = 0;
 #define IM_PPO_BULK(LPR, NI)                                                                                        \
         do {                                                                                                        \
-            static bool prepared = false;                                                                           \
-            if (!prepared) {                                                                                        \
-                if (cudaFuncSetAttribute(ppo_loss_bulk_kernel<LPR, NI>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                         max_smem - 8192) != cudaSuccess)   /* static part: 4.3 KB */       \
-                    return IM_ERR_CUDA;                                                                             \
-                prepared = true;                                                                                    \
-            }                                                                                                       \
+            static DeviceOnce once;   /* the attribute is per device */                                           \
+            if (once.run([&] {                                                                                      \
+                    return cudaFuncSetAttribute(ppo_loss_bulk_kernel<LPR, NI>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                max_smem - 8192);   /* static part: 4.3 KB */                     \
+                }) != cudaSuccess)                                                                                  \
+                return IM_ERR_CUDA;                                                                                 \
             int per_sm = 1;   /* persistent grid: as many CTAs as are resident at once */                         \
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ppo_loss_bulk_kernel<LPR, NI>,                   \
                                                           32 * bulk_warps(LPR), smem);                              \
