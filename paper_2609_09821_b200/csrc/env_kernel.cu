@@ -120,8 +120,7 @@ __device__ __forceinline__ void lookup(const ClipMeta &m, float time, int &row, 
 // Eight terms: relative truncation error below 1e-8 for u <= 0.15.
 __device__ __forceinline__ float asin2_over_u(float u)
 {
-    float p = 0.03978244f;                 // n = 8
-    p = fmaf(p, u, 0.04871319f);           // n = 7
+    float p = fmaf(0.03978244f, u, 0.04871319f);     // n = 8, 7
     p = fmaf(p, u, 0.06156806f);           // n = 6
     p = fmaf(p, u, 0.08126984f);           // n = 5
     p = fmaf(p, u, 0.11428571f);           // n = 4
@@ -130,45 +129,63 @@ __device__ __forceinline__ float asin2_over_u(float u)
     return fmaf(p, u, 1.0f);               // n = 1
 }
 
+// Keyframe words of one joint: the rotation and the log of the step to the next keyframe.  The two
+// 16-byte words are one aligned 32-byte sector, fetched with a single 256-bit load: every lane gathers from a
+// row of its own, so each load instruction costs the load pipe one pass per lane.
+struct KeyPair {
+    float4 a, b;
+};
+__device__ __forceinline__ KeyPair ld_pair(const float4 *p)
+{
+    KeyPair k;
+    asm("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=f"(k.a.x), "=f"(k.a.y), "=f"(k.a.z), "=f"(k.a.w), "=f"(k.b.x), "=f"(k.b.y), "=f"(k.b.z), "=f"(k.b.w)
+        : "l"(p));
+    return k;
+}
+__device__ __forceinline__ KeyPair ld_keys(const float4 *r0, int b) { return ld_pair(r0 + 2 + 2 * b); }
+
 // Shortest-arc slerp of one joint from the table's (keyframe, half-angle log) pair: q0 exp(alpha h), with
 // exp(alpha h) = (cos(alpha theta), sin(alpha theta) / theta h), theta = |h| <= pi / 2.  Keyframes of a motion
 // clip are close together, so the usual case (theta <= 0.5) takes cos and sin(x)/x from their Taylor
-// polynomials in (alpha theta)^2 (truncation below 2e-8).  If asked, also the joint's angular velocity in the
-// child frame, which is constant over the interval: 2 fps h.
+// polynomials in (alpha theta)^2 (truncation below 2e-8); a larger step goes through sincosf.  If asked, also
+// the joint's angular velocity in the child frame, which is constant over the interval: 2 fps h.
 template <bool VEL>
-__device__ __forceinline__ void slerp_joint(float4 k0, float4 lg, float alpha, float fps2, Quat &q, Vec3 &wl)
+__device__ __forceinline__ void slerp_joint(const KeyPair &key, float alpha, float fps2, Quat &q, Vec3 &wl)
 {
-    float c, s;
-    if (lg.w <= 0.25f) {
-        const float x = alpha * alpha * lg.w;
-        float p = fmaf(x, -1.9841270e-4f, 8.3333333e-3f);
-        p = fmaf(p, x, -1.6666667e-1f);
-        s = alpha * fmaf(p, x, 1.0f);
-        float g = fmaf(x, 2.4801587e-5f, -1.3888889e-3f);
-        g = fmaf(g, x, 4.1666667e-2f);
-        g = fmaf(g, x, -0.5f);
-        c = fmaf(g, x, 1.0f);
-    } else {
-        const float th = sqrtf(lg.w);
+    const Quat k0 = {key.a.x, key.a.y, key.a.z, key.a.w};
+    const Vec3 h = {key.b.x, key.b.y, key.b.z};
+    const float th2 = key.b.w;
+    const float x = alpha * alpha * th2;
+    float p = fmaf(x, -1.9841270e-4f, 8.3333333e-3f);
+    p = fmaf(p, x, -1.6666667e-1f);
+    float s = alpha * fmaf(p, x, 1.0f);
+    float g = fmaf(x, 2.4801587e-5f, -1.3888889e-3f);
+    g = fmaf(g, x, 4.1666667e-2f);
+    g = fmaf(g, x, -0.5f);
+    float c = fmaf(g, x, 1.0f);
+    if (th2 > 0.25f) {
+        const float th = sqrtf(th2);
         float sn;
         sincosf(alpha * th, &sn, &c);
         s = sn / th;
     }
-    const Quat rel = {c, s * lg.x, s * lg.y, s * lg.z};
-    q = qmul(Quat{k0.x, k0.y, k0.z, k0.w}, rel);
-    if (VEL) wl = {fps2 * lg.x, fps2 * lg.y, fps2 * lg.z};
+    q = qmul(k0, Quat{c, s * h.x, s * h.y, s * h.z});
+    if (VEL) wl = {fps2 * h.x, fps2 * h.y, fps2 * h.z};
 }
 
-// Squared rotation angle, in [0, pi^2], of the rotation taking frame a to frame b.  Small
+// Squared rotation angle, in [0, pi^2], of the rotation r (a quaternion of any positive norm).  Small
 // angles (below 0.8 rad, the usual tracking error) use the arcsine series on sin^2(theta/2).
-__device__ __forceinline__ float rel_angle_sq(Quat a, Quat b)
+__device__ __forceinline__ float angle_sq(Quat r)
 {
-    const Quat r = qmul(qconj(a), b);
-    const float n2 = r.x * r.x + r.y * r.y + r.z * r.z;
+    const float n2 = fmaf(r.z, r.z, fmaf(r.y, r.y, r.x * r.x));
     const float u = __fdividef(n2, fmaf(r.w, r.w, n2));    // sin^2(theta / 2)
-    if (u <= 0.15f) return 4.0f * u * asin2_over_u(u);
-    const float th = 2.0f * atan2f(sqrtf(n2), fabsf(r.w));
-    return th * th;
+    float th_sq = 4.0f * u * asin2_over_u(u);
+    if (!(u <= 0.15f)) {
+        const float th = 2.0f * atan2f(sqrtf(n2), fabsf(r.w));
+        th_sq = th * th;
+    }
+    return th_sq;
 }
 
 // World transform (and velocities) carried down a kinematic chain (step a2).
@@ -193,11 +210,12 @@ __device__ __forceinline__ LinkRec ld_link(const float4 *links, int k)
 // Compose the interpolated joint onto the running transform.  k == 0 is the root, whose position is the
 // lerp of the row's root position along its displacement.
 template <bool VEL>
-__device__ __forceinline__ void joint_compose(const float4 *r0, float alpha, float fps, Vec3 off, int k, Walk &s,
+__device__ __forceinline__ void joint_compose(const float4 *r0, float alpha, float fps, const LinkRec &L, int k, Walk &s,
                                               Quat ql, Vec3 wl)
 {
     if (k == 0) {
-        const float4 a = __ldg(r0), d = __ldg(r0 + 1);
+        const KeyPair root = ld_pair(r0);
+        const float4 a = root.a, d = root.b;
         s.q = ql;
         s.p = {fmaf(alpha, d.x, a.x), fmaf(alpha, d.y, a.y), fmaf(alpha, d.z, a.z)};
         if (VEL) {
@@ -205,29 +223,20 @@ __device__ __forceinline__ void joint_compose(const float4 *r0, float alpha, flo
             s.w = qrot(ql, wl);
         }
     } else {
-        const Vec3 arm = qrot(s.q, off);
-        if (VEL) s.v = s.v + cross(s.w, arm);
+        const Vec3 arm = qrot(s.q, L.off);
+        if (VEL) s.v = cross_add(s.w, arm, s.v);
         s.p = s.p + arm;
         s.q = qmul(s.q, ql);
-        if (VEL) s.w = s.w + qrot(s.q, wl);
+        if (VEL) s.w = qrot_add(s.q, wl, s.w);
     }
 }
 
-// Keyframe words of joint b in row r0: the rotation and the log of the step to the next keyframe.
-struct KeyPair {
-    float4 a, b;
-};
-__device__ __forceinline__ KeyPair ld_keys(const float4 *r0, int b)
-{
-    return {__ldg(r0 + 2 + 2 * b), __ldg(r0 + 3 + 2 * b)};
-}
-
 template <bool VEL>
-__device__ __forceinline__ void joint_step(const float4 *r0, const KeyPair &key, float alpha, float fps, Vec3 off, int k,
-                                           Walk &s, Quat &ql, Vec3 &wl)
+__device__ __forceinline__ void joint_step(const float4 *r0, const KeyPair &key, float alpha, float fps, const LinkRec &L,
+                                           int k, Walk &s, Quat &ql, Vec3 &wl)
 {
-    slerp_joint<VEL>(key.a, key.b, alpha, 2.0f * fps, ql, wl);
-    joint_compose<VEL>(r0, alpha, fps, off, k, s, ql, wl);
+    slerp_joint<VEL>(key, alpha, fps + fps, ql, wl);
+    joint_compose<VEL>(r0, alpha, fps, L, k, s, ql, wl);
 }
 
 // Motion randomisation of a reset state: three standard normals of Philox counter
@@ -251,11 +260,6 @@ __device__ __forceinline__ Quat reset_noise_quat(const EnvKernelParams &P, int e
     const float k = th > 1e-12f ? sn / th : 0.5f;
     return {cs, k * n.x, k * n.y, k * n.z};
 }
-// ... and as the shift of the root position (block J).
-__device__ __forceinline__ Vec3 reset_noise_shift(const EnvKernelParams &P, int env, int J)
-{
-    return reset_noise_vec(P, env, J);
-}
 
 // Phase bin of time t in a clip whose start times span [0, span]: floor(t / (span / B)) in single
 // fp32 operations, clamped to B - 1.
@@ -271,16 +275,18 @@ __device__ __forceinline__ int phase_bin(float t, float span, int B)
 // root's (x, y, 0), yaw of the root's rotated x axis (step a6).
 struct Heading {
     float ox, oy, c, s;
-    __device__ __forceinline__ Vec3 turn(Vec3 a) const { return {c * a.x + s * a.y, c * a.y - s * a.x, a.z}; }
+    __device__ __forceinline__ Vec3 turn(Vec3 a) const { return {fmaf(s, a.y, c * a.x), fmaf(-s, a.x, c * a.y), a.z}; }
+    // the same for a position: relative to the origin first
+    __device__ __forceinline__ Vec3 local(Vec3 p) const { return turn(Vec3{p.x - ox, p.y - oy, p.z}); }
 };
 
 __device__ __forceinline__ Heading make_heading(Quat q_root, Vec3 p_root)
 {
     const Vec3 h = qcol_x(q_root);
-    const float n2 = h.x * h.x + h.y * h.y;
-    Heading H = {p_root.x, p_root.y, 1.0f, 0.0f};
-    if (n2 >= 1e-12f) { const float inv = rsqrtf(n2); H.c = h.x * inv; H.s = h.y * inv; }
-    return H;
+    const float n2 = fmaf(h.y, h.y, h.x * h.x);
+    const float inv = rsqrtf(n2);
+    const bool ok = n2 >= 1e-12f;
+    return {p_root.x, p_root.y, ok ? h.x * inv : 1.0f, ok ? h.y * inv : 0.0f};
 }
 
 // Stores N consecutive floats at dst, whose offset from a 16-byte boundary is OFF floats,
@@ -315,11 +321,18 @@ __device__ __forceinline__ void store_run(float *row, int col, const float (&v)[
 // The 15 observation floats of one body seen from the heading frame.
 __device__ __forceinline__ void body_obs(const Heading &H, Quat q, Vec3 p, Vec3 v, Vec3 w, float *row, int b)
 {
-    const Vec3 pl = H.turn(Vec3{p.x - H.ox, p.y - H.oy, p.z});
+    const Vec3 pl = H.local(p);
     const Vec3 tn = H.turn(qcol_x(q)), nm = H.turn(qcol_z(q));
     const Vec3 vl = H.turn(v), wl = H.turn(w);
     const float o[15] = {pl.x, pl.y, pl.z, tn.x, tn.y, tn.z, nm.x, nm.y, nm.z, vl.x, vl.y, vl.z, wl.x, wl.y, wl.z};
     store_run<15>(row, 15 * b, o);
+}
+// The 9 target floats of one body of the reference: position and orientation columns in the heading frame.
+__device__ __forceinline__ void target_obs(const Heading &H, Quat q, Vec3 p, float (&o)[9])
+{
+    const Vec3 tp = H.local(p);
+    const Vec3 tt = H.turn(qcol_x(q)), tm = H.turn(qcol_z(q));
+    o[0] = tp.x; o[1] = tp.y; o[2] = tp.z; o[3] = tt.x; o[4] = tt.y; o[5] = tt.z; o[6] = tm.x; o[7] = tm.y; o[8] = tm.z;
 }
 
 struct SimBody {
@@ -327,9 +340,10 @@ struct SimBody {
     Vec3 p, v, w;
 };
 
+// A simulated quaternion of zero or non-finite norm is replaced by the identity and reported.
 __device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
 {
-    const float n2 = q.w * q.w + q.x * q.x + q.y * q.y + q.z * q.z;
+    const float n2 = fmaf(q.z, q.z, fmaf(q.y, q.y, fmaf(q.x, q.x, q.w * q.w)));
     if (!(n2 > 1e-12f && n2 < 1e12f)) {
         atomicOr(status, IM_DEV_BAD_SIM_QUAT);
         return {1, 0, 0, 0};
@@ -338,7 +352,7 @@ __device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
 }
 
 // Body-state loads.  Element (row, env) of an array lies at row * stride + env; the offsets are 32-bit
-// (the launcher checks that the arrays are smaller than 2^31 elements), `o` is the offset of the body's
+// (the launcher checks that the arrays are smaller than 2^31 elements); `o` is the offset of the body's
 // first row at this thread's env.
 __device__ __forceinline__ Quat ld_sim_quat(const float *base, uint32_t o, uint32_t st)
 {
@@ -349,11 +363,56 @@ __device__ __forceinline__ Vec3 ld_sim_vec(const float *base, uint32_t o, uint32
     return {base[o], base[o + st], base[o + 2 * st]};
 }
 
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// Copies the staged half rows to the observation buffers.  Warp w takes rows w, w + n_warps, ..; a row leaves as
+// 16-byte stores, 512 contiguous bytes per warp store.  `quads` 16-byte words of each staged row (row stride S
+// floats) go to float4 positions [first, first + quads) of the destination row, positions up to `last` are
+// zero-filled (the padding of the row).  F32 / BF16 select the destinations at compile time.
+template <bool F32, bool BF16>
+__device__ __forceinline__ void copy_out(const EnvKernelParams &P, const float *tile, int S, int rows, int quads, int first,
+                                         int last, int warp, int n_warps, int lane)
+{
+    const uint32_t src_lane = (uint32_t)__cvta_generic_to_shared(tile) + 16u * lane;
+    const int e0 = blockIdx.x * kTile;
+    quads = min(quads, last - first);             // the staged stride may be wider than what is left of the row
+    for (int r = warp; r < rows; r += n_warps) {
+        const size_t row_off = (size_t)(e0 + r) * P.ld_obs + 4 * (first + lane);
+        float4 *dst = F32 ? reinterpret_cast<float4 *>(P.obs + row_off) : nullptr;
+        uint2 *dst16 = BF16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + row_off) : nullptr;
+        uint32_t src = src_lane + (uint32_t)(r * S) * 4u;
+        int i = lane;
+        for (; i < quads; i += 32, src += 512u) {
+            const float4 v = lds128(src);
+            if (F32) { *dst = v; dst += 32; }
+            if (BF16) { *dst16 = pack_bf16x4(v); dst16 += 32; }
+        }
+        for (; i < last - first; i += 32) {
+            if (F32) { *dst = make_float4(0.0f, 0.0f, 0.0f, 0.0f); dst += 32; }
+            if (BF16) { *dst16 = make_uint2(0u, 0u); dst16 += 32; }
+        }
+    }
+}
+__device__ __forceinline__ void copy_out_any(const EnvKernelParams &P, const float *tile, int S, int quads, int first, int last,
+                                             int warp, int n_warps, int lane)
+{
+    const int rows = min(kTile, P.N - (int)blockIdx.x * kTile);
+    // (a policy-serving loop may ask for the bf16 rows only: obs null)
+    if (P.obs && P.obs_bf16) copy_out<true, true>(P, tile, S, rows, quads, first, last, warp, n_warps, lane);
+    else if (P.obs) copy_out<true, false>(P, tile, S, rows, quads, first, last, warp, n_warps, lane);
+    else copy_out<false, true>(P, tile, S, rows, quads, first, last, warp, n_warps, lane);
+}
+
 // Kernel body.  The observation row is assembled in two halves that reuse the same shared
 // memory: columns [0, c1) -- the body blocks and, if 15 J is not a multiple of 4, the phase and
 // the first target floats -- and columns [c1, D) -- the targets.
-// OPT compiles in the optional semantics (grace steps, motion randomisation, adaptive initialisation); envs that use none run
-// the instantiation without them.
+// OPT compiles in the optional semantics (grace steps, motion randomisation, adaptive initialisation, extended
+// observation); envs that use none run the instantiation without them.
 template <bool RESET_ALL, bool OPT>
 __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
 {
@@ -389,7 +448,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     __syncwarp();
 
     if (c == 0)
-        for (int i = 15 * J; i < S1; ++i) row1[i] = 0.0f;   // columns between the body blocks and the stride
+        for (int i = 15 * J; i < c1; ++i) row1[i] = 0.0f;   // columns between the body blocks and the split
 
     int clip = 0;
     float t1 = 0.0f;
@@ -432,11 +491,9 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             wa = ld_sim_vec(P.ang, 3 * a * st + e32, st);
         }
         for (int k = 0; k < len; ++k) {
-            const int b = L.b;
-            const bool own = L.flags & LINK_OWN;
-            const bool ee = L.flags & LINK_EE;
-            const Vec3 off = L.off;
-            const float mf = L.mass_frac;
+            const LinkRec Lc = L;
+            const int b = Lc.b;
+            const bool own = Lc.flags & LINK_OWN;
             SimBody sim;
             if (own) {                                // issue the loads before the interpolation math
                 const uint32_t o3 = 3 * (uint32_t)b * st + e32;
@@ -452,32 +509,28 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             }
             Quat ql;
             Vec3 wl;
-            joint_step<true>(r0, cur, alpha, cm.fps, off, k, s, ql, wl);
+            joint_step<true>(r0, cur, alpha, cm.fps, Lc, k, s, ql, wl);
             if (own) {
                 sim.q = sanitize(sim.q, P.status);
-                Quat ql_sim = sim.q;
-                Vec3 dw = sim.w;
-                if (b > 0) {
-                    ql_sim = qmul(qconj(qa), sim.q);
-                    dw = sim.w - wa;
-                }
-                const Vec3 wl_sim = qrot_inv(sim.q, dw);
-                const float th_sq = rel_angle_sq(ql, ql_sim);
+                // the root's "parent" is the identity: qa = (1, 0, 0, 0), wa = 0 on the chain that owns it
+                const Quat ql_sim = qmul_conj(qa, sim.q);
+                const Vec3 wl_sim = qrot_inv(sim.q, sim.w - wa);
+                const float th_sq = angle_sq(qmul_conj(ql, ql_sim));
                 const Vec3 dwl = wl_sim - wl;
                 const Vec3 dp = sim.p - s.p;
                 const Vec3 dv = sim.v - s.v;
                 const float dp2 = dot(dp, dp);
                 acc[0] += th_sq;
                 acc[1] += dot(dwl, dwl);
-                if (ee) {
+                if (Lc.flags & LINK_EE) {
                     acc[2] += dp2;
-                    acc[3] += rel_angle_sq(s.q, sim.q);
+                    acc[3] += angle_sq(qmul_conj(s.q, sim.q));
                 }
                 acc[4] += dp2;
                 acc[5] += dot(dv, dv);
-                acc[6] += mf * dp.x;
-                acc[7] += mf * dp.y;
-                acc[8] += mf * dp.z;
+                acc[6] = fmaf(Lc.mass_frac, dp.x, acc[6]);
+                acc[7] = fmaf(Lc.mass_frac, dp.y, acc[7]);
+                acc[8] = fmaf(Lc.mass_frac, dp.z, acc[8]);
                 body_obs(H, sim.q, sim.p, sim.v, sim.w, row1, b);
                 qa = sim.q;
                 wa = sim.w;
@@ -488,31 +541,42 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     }
     __syncthreads();
 
-    // ---- decision: every thread of an env adds the chains' partial sums in chain order and takes
-    //      the same reward, flags and reset draw; chain 0 writes them out
+    // ---- decision.  Chain 0 adds the chains' partial sums in chain order, forms the reward and writes reward,
+    //      flags and the new per-env state.  Every other thread of the env needs the flags as well: it repeats the
+    //      reward only if the reward can terminate an episode (r_min above -inf), else the root height and the
+    //      clip end decide alone.  The reset draw is a function of (env, step) and is repeated by every thread.
     int flags = 0;
     float t_cur = t1;
     int clip_cur = clip;
     if (!RESET_ALL) {
-        float e[kPartials];
+        float r = 0.0f;
+        const bool need_r = c == 0 || P.reward.r_min > -INFINITY;
+        if (need_r) {
+            float e[kPartials];
 #pragma unroll
-        for (int i = 0; i < kPartials; ++i) {
-            float a = 0.0f;
-            for (int cc = 0; cc < C; ++cc) a += part[(i * C + cc) * kTile + lane];
-            e[i] = a;
-        }
-        // term order of the configuration: pose, vel, ee_pos, ee_rot, com, body_pos, body_vel
-        const float term[IM_N_TERMS] = {e[0], e[1], e[2], e[3], e[6] * e[6] + e[7] * e[7] + e[8] * e[8], e[4], e[5]};
-        float r;
-        if (P.reward.mode == 0) {
-            float sum = 0.0f;
+            for (int i = 0; i < kPartials; ++i) {
+                float a = 0.0f;
+                for (int cc = 0; cc < C; ++cc) a += part[(i * C + cc) * kTile + lane];
+                e[i] = a;
+            }
+            // term order of the configuration: pose, vel, ee_pos, ee_rot, com, body_pos, body_vel
+            const float term[IM_N_TERMS] = {e[0], e[1], e[2], e[3], e[6] * e[6] + e[7] * e[7] + e[8] * e[8], e[4], e[5]};
+            if (P.reward.mode == 0) {
+                float sum = 0.0f;
 #pragma unroll
-            for (int k = 0; k < IM_N_TERMS; ++k) sum += P.reward.w[k] * term[k];
-            r = expf(-sum);
-        } else {
-            r = 0.0f;
+                for (int k = 0; k < IM_N_TERMS; ++k) sum += P.reward.w[k] * term[k];
+                r = expf(-sum);
+            } else {
 #pragma unroll
-            for (int k = 0; k < IM_N_TERMS; ++k) r += P.reward.a[k] * expf(-P.reward.w[k] * term[k]);
+                for (int k = 0; k < IM_N_TERMS; ++k) r += P.reward.a[k] * expf(-P.reward.w[k] * term[k]);
+            }
+            if (c == 0 && valid) {
+                P.reward_out[env] = r;
+                if (P.terms_out) {
+#pragma unroll
+                    for (int k = 0; k < IM_N_TERMS; ++k) P.terms_out[(size_t)k * P.N + env] = term[k];
+                }
+            }
         }
         bool terminated = (root_z < P.reward.h_min) || (r < P.reward.r_min);
         if (OPT && P.ep_len[envc] < P.grace_steps) terminated = false;
@@ -523,14 +587,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
         const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
         flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
-        if (c == 0 && valid) {
-            P.reward_out[env] = r;
-            P.flags_out[env] = (uint8_t)flags;
-            if (P.terms_out) {
-#pragma unroll
-                for (int k = 0; k < IM_N_TERMS; ++k) P.terms_out[(size_t)k * P.N + env] = term[k];
-            }
-        }
+        if (c == 0 && valid) P.flags_out[env] = (uint8_t)flags;
     }
     const bool reset = RESET_ALL || flags != 0;
     if (reset) {
@@ -576,9 +633,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         Walk s;
         Heading Hn = H;
         for (int k = 0; k < len; ++k) {
-            const int b = L.b;
-            const bool own = L.flags & LINK_OWN;
-            const Vec3 off = L.off;
+            const LinkRec Lc = L;
+            const int b = Lc.b;
             const KeyPair cur = keys;
             if (k + 1 < len) {
                 L = ld_link(links, k + 1);
@@ -589,15 +645,15 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             if (OPT && P.reset_noise_std > 0.0f) {
                 // motion randomisation: the joint turns by a small random rotation in its own frame and
                 // the root is shifted; every chain that walks a shared body draws the same numbers
-                slerp_joint<true>(cur.a, cur.b, alpha, 2.0f * cmc.fps, ql, wl);
+                slerp_joint<true>(cur, alpha, cmc.fps + cmc.fps, ql, wl);
                 ql = qmul(ql, reset_noise_quat(P, envc, b));
-                joint_compose<true>(r0, alpha, cmc.fps, off, k, s, ql, wl);
-                if (k == 0) s.p = s.p + reset_noise_shift(P, envc, sk.J);
+                joint_compose<true>(r0, alpha, cmc.fps, Lc, k, s, ql, wl);
+                if (k == 0) s.p = s.p + reset_noise_vec(P, envc, sk.J);
             } else {
-                joint_step<true>(r0, cur, alpha, cmc.fps, off, k, s, ql, wl);
+                joint_step<true>(r0, cur, alpha, cmc.fps, Lc, k, s, ql, wl);
             }
             if (k == 0) Hn = make_heading(s.q, s.p);
-            if (own && reset) {
+            if ((Lc.flags & LINK_OWN) && reset) {
                 body_obs(Hn, s.q, s.p, s.v, s.w, row1, b);
                 if (!RESET_ALL && P.write_back && valid) {
                     const uint32_t o3 = 3 * (uint32_t)b * st + e32, o4 = 4 * (uint32_t)b * st + e32;
@@ -618,33 +674,21 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     float alpha_t;
     lookup(cmc, t_tgt, frame_t, alpha_t);
     const float4 *rt0 = P.frames + (size_t)frame_t * RS;
-    const float phase = t_cur / cmc.dur;
-    if (c == 0 && 15 * J < c1) {
-        const float4 a = __ldg(rt0), d = __ldg(rt0 + 1);
-        const Vec3 tp = H.turn(Vec3{fmaf(alpha_t, d.x, a.x) - H.ox, fmaf(alpha_t, d.y, a.y) - H.oy, fmaf(alpha_t, d.z, a.z)});
-        row1[15 * J] = phase;
-        if (15 * J + 1 < c1) row1[15 * J + 1] = tp.x;
-        if (15 * J + 2 < c1) row1[15 * J + 2] = tp.y;
+    float phase = 0.0f;
+    if (c == 0) {
+        phase = t_cur / cmc.dur;
+        if (15 * J < c1) {
+            const KeyPair root = ld_pair(rt0);
+            const Vec3 tp = H.local(Vec3{fmaf(alpha_t, root.b.x, root.a.x), fmaf(alpha_t, root.b.y, root.a.y), 0.0f});
+            row1[15 * J] = phase;
+            if (15 * J + 1 < c1) row1[15 * J + 1] = tp.x;
+            if (15 * J + 2 < c1) row1[15 * J + 2] = tp.y;
+        }
     }
     __syncthreads();
 
-    // ---- first half of the rows to global memory, 16-byte stores, 512 contiguous bytes per warp store
-    {
-        const int n4 = c1 >> 2, S4 = S1 >> 2;
-        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
-        for (int r = c; r < kTile; r += C) {
-            const int e = blockIdx.x * kTile + r;
-            if (e >= P.N) break;
-            // (a policy-serving loop may ask for the bf16 rows only: obs null)
-            float4 *dst = P.obs ? reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs) : nullptr;
-            uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
-            for (int i = lane; i < n4; i += 32) {
-                const float4 v = tile4[(size_t)r * S4 + i];
-                if (dst) dst[i] = v;
-                if (dst16) dst16[i] = pack_bf16x4(v);
-            }
-        }
-    }
+    // ---- first half of the rows to global memory
+    copy_out_any(P, tile, S1, c1 >> 2, 0, c1 >> 2, c, C, lane);
     __syncthreads();
 
     // ---- pass B: reference pose one control interval ahead, seen from the same heading frame,
@@ -658,9 +702,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         KeyPair keys = ld_keys(rt0, L.b);
         Walk s;
         for (int k = 0; k < len; ++k) {
-            const int b = L.b;
-            const bool own = L.flags & LINK_OWN;
-            const Vec3 off = L.off;
+            const LinkRec Lc = L;
+            const int b = Lc.b;
             const KeyPair cur = keys;
             if (k + 1 < len) {
                 L = ld_link(links, k + 1);
@@ -668,11 +711,10 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             }
             Quat ql;
             Vec3 wl;
-            joint_step<false>(rt0, cur, alpha_t, cmc.fps, off, k, s, ql, wl);
-            if (own) {
-                const Vec3 tp = H.turn(Vec3{s.p.x - H.ox, s.p.y - H.oy, s.p.z});
-                const Vec3 tt = H.turn(qcol_x(s.q)), tm = H.turn(qcol_z(s.q));
-                const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
+            joint_step<false>(rt0, cur, alpha_t, cmc.fps, Lc, k, s, ql, wl);
+            if (Lc.flags & LINK_OWN) {
+                float o[9];
+                target_obs(H, s.q, s.p, o);
                 const int col = 15 * J + 1 + 9 * b;
                 if (col >= c1) {
                     store_run<9>(row2, col - c1, o);
@@ -699,11 +741,10 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                     const KeyPair kp = ld_keys(rf0, b);
                     Quat ql;
                     Vec3 wl;
-                    joint_step<false>(rf0, kp, alpha_f, cmc.fps, Lf.off, k, sf, ql, wl);
+                    joint_step<false>(rf0, kp, alpha_f, cmc.fps, Lf, k, sf, ql, wl);
                     if ((Lf.flags & LINK_OWN) && (Lf.flags & LINK_EE)) {
-                        const Vec3 tp = H.turn(Vec3{sf.p.x - H.ox, sf.p.y - H.oy, sf.p.z});
-                        const Vec3 tt = H.turn(qcol_x(sf.q)), tm = H.turn(qcol_z(sf.q));
-                        const float o[9] = {tp.x, tp.y, tp.z, tt.x, tt.y, tt.z, tm.x, tm.y, tm.z};
+                        float o[9];
+                        target_obs(H, sf.q, sf.p, o);
                         float *dst = row2 + (D - c1) + ((f - 2) * n_ee + __popc(sk.ee_mask & ((1u << b) - 1u))) * 9;
 #pragma unroll
                         for (int i = 0; i < 9; ++i) dst[i] = o[i];
@@ -717,27 +758,16 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
     }
     __syncthreads();
-    {
-        const int n4 = c1 >> 2, S4 = S2 >> 2, ld4 = P.ld_obs >> 2;
-        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
-        for (int r = c; r < kTile; r += C) {
-            const int e = blockIdx.x * kTile + r;
-            if (e >= P.N) break;
-            float4 *dst = P.obs ? reinterpret_cast<float4 *>(P.obs + (size_t)e * P.ld_obs) : nullptr;
-            uint2 *dst16 = P.obs_bf16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + (size_t)e * P.ld_obs) : nullptr;
-            for (int i = n4 + lane; i < ld4; i += 32) {
-                const float4 v = (i - n4 < S4) ? tile4[(size_t)r * S4 + i - n4] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                if (dst) dst[i] = v;
-                if (dst16) dst16[i] = pack_bf16x4(v);
-            }
-        }
-    }
+    copy_out_any(P, tile, S2, S2 >> 2, c1 >> 2, P.ld_obs >> 2, c, C, lane);
 }
 
 // Two instantiations per mode: skeletons with at most 8 leaves (blocks of up to 256 threads) get a
 // register budget that lets four blocks share an SM; wider trees fall back to 64 registers.
+#ifndef IM_ENV_MAXNREG
+#define IM_ENV_MAXNREG 96
+#endif
 template <bool RESET_ALL, bool OPT>
-__global__ void __maxnreg__(96) env_step_kernel_small(const __grid_constant__ EnvKernelParams P)
+__global__ void __maxnreg__(IM_ENV_MAXNREG) env_step_kernel_small(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
     env_step_body<RESET_ALL, OPT>(P, smem_raw);

@@ -16,27 +16,46 @@ struct Vec3 { float x, y, z; };
 __device__ __forceinline__ Vec3 operator+(Vec3 a, Vec3 b) { return {a.x + b.x, a.y + b.y, a.z + b.z}; }
 __device__ __forceinline__ Vec3 operator-(Vec3 a, Vec3 b) { return {a.x - b.x, a.y - b.y, a.z - b.z}; }
 __device__ __forceinline__ Vec3 operator*(float s, Vec3 a) { return {s * a.x, s * a.y, s * a.z}; }
-__device__ __forceinline__ float dot(Vec3 a, Vec3 b) { return a.x * b.x + a.y * b.y + a.z * b.z; }
+__device__ __forceinline__ float dot(Vec3 a, Vec3 b) { return fmaf(a.z, b.z, fmaf(a.y, b.y, a.x * b.x)); }
 __device__ __forceinline__ Vec3 cross(Vec3 a, Vec3 b)
 {
-    return {a.y * b.z - a.z * b.y, a.z * b.x - a.x * b.z, a.x * b.y - a.y * b.x};
+    return {fmaf(a.y, b.z, -(a.z * b.y)), fmaf(a.z, b.x, -(a.x * b.z)), fmaf(a.x, b.y, -(a.y * b.x))};
+}
+// c + a x b
+__device__ __forceinline__ Vec3 cross_add(Vec3 a, Vec3 b, Vec3 c)
+{
+    return {fmaf(a.y, b.z, fmaf(-a.z, b.y, c.x)), fmaf(a.z, b.x, fmaf(-a.x, b.z, c.y)), fmaf(a.x, b.y, fmaf(-a.y, b.x, c.z))};
 }
 
 __device__ __forceinline__ Quat qmul(Quat a, Quat b)
 {
-    return {a.w * b.w - a.x * b.x - a.y * b.y - a.z * b.z,
-            a.w * b.x + a.x * b.w + a.y * b.z - a.z * b.y,
-            a.w * b.y - a.x * b.z + a.y * b.w + a.z * b.x,
-            a.w * b.z + a.x * b.y - a.y * b.x + a.z * b.w};
+    return {fmaf(-a.z, b.z, fmaf(-a.y, b.y, fmaf(-a.x, b.x, a.w * b.w))),
+            fmaf(-a.z, b.y, fmaf(a.y, b.z, fmaf(a.x, b.w, a.w * b.x))),
+            fmaf(a.z, b.x, fmaf(a.y, b.w, fmaf(-a.x, b.z, a.w * b.y))),
+            fmaf(a.z, b.w, fmaf(-a.y, b.x, fmaf(a.x, b.y, a.w * b.z)))};
 }
 __device__ __forceinline__ Quat qconj(Quat a) { return {a.w, -a.x, -a.y, -a.z}; }
+// a* b
+__device__ __forceinline__ Quat qmul_conj(Quat a, Quat b) { return qmul(qconj(a), b); }
 
-// R(q) v for a unit quaternion: v + w t + u x t with t = 2 u x v.
+// add + R(q) v for a unit quaternion: v + 2 w (u x v) + 2 u x (u x v).
+__device__ __forceinline__ Vec3 qrot_add(Quat q, Vec3 v, Vec3 add)
+{
+    const Vec3 u = {q.x, q.y, q.z};
+    const Vec3 t = cross(u, v);
+    const Vec3 u2 = {u.x + u.x, u.y + u.y, u.z + u.z};
+    const float w2 = q.w + q.w;
+    const Vec3 base = {fmaf(w2, t.x, v.x + add.x), fmaf(w2, t.y, v.y + add.y), fmaf(w2, t.z, v.z + add.z)};
+    return cross_add(u2, t, base);
+}
 __device__ __forceinline__ Vec3 qrot(Quat q, Vec3 v)
 {
-    Vec3 u = {q.x, q.y, q.z};
-    Vec3 t = 2.0f * cross(u, v);
-    return v + q.w * t + cross(u, t);
+    const Vec3 u = {q.x, q.y, q.z};
+    const Vec3 t = cross(u, v);
+    const Vec3 u2 = {u.x + u.x, u.y + u.y, u.z + u.z};
+    const float w2 = q.w + q.w;
+    const Vec3 base = {fmaf(w2, t.x, v.x), fmaf(w2, t.y, v.y), fmaf(w2, t.z, v.z)};
+    return cross_add(u2, t, base);
 }
 __device__ __forceinline__ Vec3 qrot_inv(Quat q, Vec3 v) { return qrot(qconj(q), v); }
 
@@ -44,11 +63,13 @@ __device__ __forceinline__ Vec3 qrot_inv(Quat q, Vec3 v) { return qrot(qconj(q),
 // of the 6-float orientation encoding of the observation).
 __device__ __forceinline__ Vec3 qcol_x(Quat q)
 {
-    return {1.0f - 2.0f * (q.y * q.y + q.z * q.z), 2.0f * (q.x * q.y + q.w * q.z), 2.0f * (q.x * q.z - q.w * q.y)};
+    const float y2 = q.y + q.y, z2 = q.z + q.z;
+    return {fmaf(-z2, q.z, fmaf(-y2, q.y, 1.0f)), fmaf(y2, q.x, z2 * q.w), fmaf(z2, q.x, -(y2 * q.w))};
 }
 __device__ __forceinline__ Vec3 qcol_z(Quat q)
 {
-    return {2.0f * (q.x * q.z + q.w * q.y), 2.0f * (q.y * q.z - q.w * q.x), 1.0f - 2.0f * (q.x * q.x + q.y * q.y)};
+    const float x2 = q.x + q.x, y2 = q.y + q.y;
+    return {fmaf(x2, q.z, y2 * q.w), fmaf(y2, q.z, -(x2 * q.w)), fmaf(-y2, q.y, fmaf(-x2, q.x, 1.0f))};
 }
 
 // Rotation angle in [0, pi] of the rotation taking frame a to frame b.
