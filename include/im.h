@@ -549,6 +549,20 @@ im_status im_poll_device_status(im_env *e, im_policy *p, uint32_t *out);
 /* Number of kernel launches the library has enqueued since it was loaded. */
 uint64_t im_launch_count(void);
 
+/* ---- diagnostics: the env kernel's approximations in isolation -----------------
+ * (No counterpart in the paper.)  The env kernel evaluates the interpolation of step (a) and the
+ * geodesic angles of the reward without inverse trigonometry where the angles are small: the squared
+ * rotation angle from an arcsine series on sin^2(theta/2) (up to sin^2 = 0.15, atan2 beyond), and
+ * slerp as q0 exp(alpha h) with cos and sin(x)/x from Taylor polynomials (up to |h| = 0.5, sincos
+ * beyond).  This call runs those two device functions on n items so that a test can sweep them across
+ * both branches against closed forms.
+ *   op = IM_DEBUG_ANGLE_SQ   in DEVICE [n][4] quaternions of any positive norm -> out DEVICE [n] angle^2
+ *   op = IM_DEBUG_SLERP      in DEVICE [n][8] = q0 (w,x,y,z), h (3), alpha       -> out DEVICE [n][7] =
+ *                            q0 exp(alpha h) (4) and 2 h (the joint velocity at 1 frame per second) */
+#define IM_DEBUG_ANGLE_SQ 0
+#define IM_DEBUG_SLERP    1
+im_status im_debug_math(int32_t op, int32_t n, const float *in, float *out, void *cuda_stream);
+
 /* ---- allocation-free policy forward ------------------------------------------
  * (The paper has no counterpart of this call; it exists for deployment.)
  * For callers that may not allocate device memory when they need an action: a
@@ -566,12 +580,14 @@ uint64_t im_launch_count(void);
  *   cuda_stream cudaStream_t the work is enqueued on
  * Limits: n <= IM_NOALLOC_MAX_BATCH and hidden widths <= IM_NOALLOC_MAX_WIDTH; beyond them the call
  * returns IM_ERR_UNSUPPORTED and does nothing.
- * The first call on each device looks up the array's device address (a query, not an allocation);
- * make that first call outside any stream capture, with the device that will run it current.
+ * The first call on each device looks up the array's device address.  The look-up itself requests no
+ * memory, but under CUDA's lazy module loading it can be the moment the driver loads this library's
+ * device code on that GPU and backs the array, which may take a while: make the first call at
+ * start-up, off the latency-critical path, outside any stream capture, with the device that will
+ * run it current.  Later calls only launch kernels.
  * All calls on a device share the one array: it keeps whatever the last call left (nothing in it
  * needs clearing, every value read is written first by the same call), and two calls whose work
- * overlaps on the GPU -- different streams, or replays of graphs containing it -- race on it.
- * Run them on one stream. */
+ * overlaps on the GPU (for example on different streams) race on it.  Run them on one stream. */
 #define IM_NOALLOC_MAX_BATCH  1024
 #define IM_NOALLOC_MAX_WIDTH  1024
 #define IM_NOALLOC_SCRATCH_BYTES (2u * IM_NOALLOC_MAX_BATCH * IM_NOALLOC_MAX_WIDTH * 4u)   /* 8 MiB */

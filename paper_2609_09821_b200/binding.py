@@ -29,7 +29,7 @@ EXPORTS = [
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
     "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
     "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math",
 ]
 
 
@@ -142,6 +142,7 @@ def load():
         L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
         L.im_env_adapt_reset_bins.argtypes = [vp, C.c_float, i32]
+        L.im_debug_math.argtypes = [i32, i32, vp, vp, vp]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp, vp]
         L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
@@ -614,6 +615,17 @@ def colsum(x, out, workspace, stream=None):
 
 NOALLOC_MAX_BATCH = 1024
 NOALLOC_MAX_WIDTH = 1024
+DEBUG_ANGLE_SQ, DEBUG_SLERP = 0, 1
+
+
+def debug_math(op: int, inp):
+    """The env kernel's angle / slerp device functions on rows of `inp` (float32 CUDA tensor, [n, 4] or [n, 8])."""
+    import torch
+    assert inp.is_cuda and inp.dtype == torch.float32 and inp.is_contiguous()
+    n = inp.shape[0]
+    out = torch.empty(n if op == DEBUG_ANGLE_SQ else (n, 7), device=inp.device)
+    _check(load().im_debug_math(op, n, inp.data_ptr(), out.data_ptr(), torch.cuda.current_stream().cuda_stream), "im_debug_math")
+    return out
 
 
 def policy_forward_noalloc(dims: Sequence[int], W_dev, b_dev, sigma: float, seed: int, step: int, obs,

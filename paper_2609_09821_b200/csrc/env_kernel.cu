@@ -761,6 +761,26 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     copy_out_any(P, tile, S2, S2 >> 2, c1 >> 2, P.ld_obs >> 2, c, C, lane);
 }
 
+// Diagnostic kernel: the scalar building blocks of the env kernel on caller-given inputs, one thread per item.
+__global__ void debug_math_kernel(int op, int n, const float *__restrict__ in, float *__restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    if (op == 0) {                                   // squared rotation angle of a quaternion of any norm
+        const float *q = in + 4 * i;
+        out[i] = angle_sq(Quat{q[0], q[1], q[2], q[3]});
+    } else {                                         // slerp from (keyframe, half-angle log, blend factor), fps = 1
+        const float *v = in + 8 * i;
+        const KeyPair key = {make_float4(v[0], v[1], v[2], v[3]),
+                             make_float4(v[4], v[5], v[6], v[4] * v[4] + v[5] * v[5] + v[6] * v[6])};
+        Quat q;
+        Vec3 wl;
+        slerp_joint<true>(key, v[7], 2.0f, q, wl);
+        float *o = out + 7 * i;
+        o[0] = q.w; o[1] = q.x; o[2] = q.y; o[3] = q.z; o[4] = wl.x; o[5] = wl.y; o[6] = wl.z;
+    }
+}
+
 // Two instantiations per mode: skeletons with at most 8 leaves (blocks of up to 256 threads) get a
 // register budget that lets four blocks share an SM; wider trees fall back to 64 registers.
 #ifndef IM_ENV_MAXNREG
@@ -820,6 +840,13 @@ cudaError_t launch_clip_table(const float *root_pos, const float *local_quat, co
 {
     const long long n = (long long)rows * (J + 1);
     clip_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(root_pos, local_quat, last, (long long)rows, J, frames);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_debug_math(int op, int n, const float *in, float *out, cudaStream_t stream)
+{
+    debug_math_kernel<<<(n + 127) / 128, 128, 0, stream>>>(op, n, in, out);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }

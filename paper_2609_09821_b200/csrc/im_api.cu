@@ -728,6 +728,13 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     return IM_OK;
 }
 
+im_status im_debug_math(int32_t op, int32_t n, const float *in, float *out, void *cuda_stream)
+{
+    if ((op != IM_DEBUG_ANGLE_SQ && op != IM_DEBUG_SLERP) || n < 1 || !in || !out) return IM_ERR_INVALID_ARG;
+    IM_CUDA(launch_debug_math(op, n, in, out, (cudaStream_t)cuda_stream));
+    return IM_OK;
+}
+
 im_status im_poll_device_status(im_env *e, im_policy *p, uint32_t *out)
 {
     if (!out || (!e && !p) || (e && p)) return IM_ERR_INVALID_ARG;

@@ -163,6 +163,7 @@ cudaError_t launch_clip_table(const float *root_pos, const float *local_quat, co
 inline int clip_row_stride(int J) { return 2 + 2 * J; }
 cudaError_t env_kernel_prepare(size_t smem);
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream);
+cudaError_t launch_debug_math(int op, int n, const float *in, float *out, cudaStream_t stream);
 // simulator-native (array of structures) body states <-> component rows [13 J][stride]
 cudaError_t aos_adapter_prepare();
 // reset-bin weights from the failure counts (rollout.cu); n <= 12288 entries

@@ -24,20 +24,19 @@ constexpr size_t kScratchFloats = 2ull * IM_NOALLOC_MAX_BATCH * IM_NOALLOC_MAX_W
 
 static __device__ __align__(256) float g_noalloc_scratch[kScratchFloats];
 
-constexpr int kMaxDevices = 64;
-float *g_scratch_ptr[kMaxDevices] = {nullptr};
+std::atomic<float *> g_scratch_ptr[im::kMaxDevices];      // per device; threads racing on the first call store the same value
 
 // Device address of the scratch array on the current device (set-up on first use per device).
 im_status scratch_for_current_device(float **out)
 {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return IM_ERR_CUDA;
-    if (!g_scratch_ptr[dev]) {
-        float *ptr = nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= im::kMaxDevices) return IM_ERR_CUDA;
+    float *ptr = g_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return IM_ERR_CUDA;
-        g_scratch_ptr[dev] = ptr;
+        g_scratch_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_ptr[dev];
+    *out = ptr;
     return IM_OK;
 }
 

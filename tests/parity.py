@@ -22,23 +22,17 @@ from paper_2609_09821_b200 import binding as B
 from paper_2609_09821_b200 import workloads as W
 
 OBS_ATOL, OBS_RTOL = 1e-5, 1e-4
-# fp32 slack of velocity-derived entries.  A body's world velocity is a sum of up to depth+1
-# rotated joint velocities; in fp32 each rotated term and each partial sum carries a rounding
-# error of a few ulp of ITS magnitude, whatever the (possibly cancelled) result is.  With S the
-# largest velocity entry of the env's observation, those entries are allowed an extra
-# 2^-20 S (16 ulp-units of S; 1.9e-5 at S = 20 rad/s).  Positions, orientations, phase,
-# targets and the reward keep the plain tolerance.
-VEL_SLACK = 2.0 ** -20
 
 
-def assert_close(got, want, atol=OBS_ATOL, rtol=OBS_RTOL, what="", slack=None):
+def assert_close(got, want, atol=OBS_ATOL, rtol=OBS_RTOL, what="", extra=None):
+    """extra: optional per-entry addition to the limit (see Pair's vel_ulps)."""
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape, (what, got.shape, want.shape)
     err = np.abs(got - want)
     lim = atol + rtol * np.abs(want)
-    if slack is not None:
-        lim = lim + slack
+    if extra is not None:
+        lim = lim + extra
     bad = ~(err <= lim)                   # NaN counts as bad
     if bad.any():
         i = np.unravel_index(np.argmax(np.where(bad, err - lim, -np.inf)), err.shape)
@@ -88,7 +82,7 @@ class Pair:
     def __init__(self, scene: Scene, n: int, reward=W.REWARD_MULT, seed=None, h_min=None, r_min=-np.inf,
                  write_back=False, env_base=0, ld_obs=None, stride_pad=0, with_policy=True, policy_impl=0,
                  policy_sample=None, want_terms=True, obs_atol=OBS_ATOL, grace_steps=0, reset_noise_std=0.0,
-                 n_future=1, prev_action_dim=0):
+                 n_future=1, prev_action_dim=0, vel_ulps=0):
         wl = scene.wl
         self.scene, self.wl, self.n, self.J = scene, wl, n, scene.J
         self.seed = wl.seed if seed is None else seed
@@ -99,6 +93,12 @@ class Pair:
         self.ld_obs = ld_obs or B.padded_ld(self.D)
         self.stride = (n + stride_pad + 3) // 4 * 4        # rows of the body-state arrays stay 16-byte aligned
         self.obs_atol = obs_atol
+        # Every comparison uses the plain tolerance unless a test states vel_ulps: fp32 rounds each velocity to
+        # 2^-24 of ITS magnitude, so where inputs are far larger than the benchmark's (a 120 frames-per-second
+        # clip has four times its velocities) an entry that is a small difference of large velocities cannot
+        # meet an absolute 1e-5; such a test allows vel_ulps * 2^-24 * (largest velocity of the env) more on
+        # velocity entries only.  The benchmark configurations run with vel_ulps = 0.
+        self.vel_ulps = vel_ulps
         self.write_back = write_back
         self.want_terms = want_terms
         ids = np.arange(env_base, env_base + n, dtype=np.uint32)
@@ -146,17 +146,16 @@ class Pair:
                                       err_msg=what + " time bit patterns")
         np.testing.assert_array_equal(l.cpu().numpy(), self.o_env.ep_len, err_msg=what + " episode lengths")
 
-    def vel_scale(self):
-        """Largest velocity entry of each env's (oracle) observation."""
-        body = self.obs_o[:, :15 * self.J].reshape(self.n, self.J, 15)
-        return np.abs(body[:, :, 9:15]).max(axis=(1, 2))
-
     def check_obs(self, what):
         g = self.obs_g.cpu().numpy()
-        slack = np.zeros((self.n, self.J, 15))
-        slack[:, :, 9:15] = (VEL_SLACK * self.vel_scale())[:, None, None]
-        slack = np.concatenate([slack.reshape(self.n, -1), np.zeros((self.n, self.D - 15 * self.J))], axis=1)
-        assert_close(g[:, :self.D], self.obs_o, atol=self.obs_atol, what=what + " obs", slack=slack)
+        extra = None
+        if self.vel_ulps:
+            body = self.obs_o[:, :15 * self.J].reshape(self.n, self.J, 15)
+            scale = np.abs(body[:, :, 9:15]).max(axis=(1, 2))
+            extra = np.zeros((self.n, self.J, 15))
+            extra[:, :, 9:15] = (self.vel_ulps * 2.0 ** -24 * scale)[:, None, None]
+            extra = np.concatenate([extra.reshape(self.n, -1), np.zeros((self.n, self.D - 15 * self.J))], axis=1)
+        assert_close(g[:, :self.D], self.obs_o, atol=self.obs_atol, what=what + " obs", extra=extra)
         assert np.all(g[:, self.D:] == 0.0), what + " obs padding must be zero"
         self.max_err["obs"] = max(self.max_err["obs"], float(np.abs(g[:, :self.D] - self.obs_o).max()))
 
@@ -181,7 +180,7 @@ class Pair:
             plain = O.policy_forward(pol["dims"], pol["W"], pol["b"], self.wl.sigma_action, self.seed, s,
                                      self.obs_o[idx], env_ids=self.ids[idx])["mean"]
             rel = np.abs(mg - plain) / (np.abs(plain) + mean_scale(plain))
-            frac_ok = np.mean(rel <= 2e-2) >= 0.999 or len(idx) < 64      # a fraction needs a population
+            frac_ok = np.mean(rel <= 2e-2) >= 0.999 or rel.size < 10000    # a 0.1 % fraction needs a population
             assert frac_ok and rel.max() <= 6e-2, \
                 "step %d: vs unrounded oracle: %.4f within 2e-2, max %.3g" % (s, np.mean(rel <= 2e-2), rel.max())
             self.max_err["mean_vs_plain"] = max(self.max_err.get("mean_vs_plain", 0.0), float(rel.max()))
@@ -199,7 +198,6 @@ class Pair:
         sim_g[:, :self.n] = sim.to("cuda")
         if self.stride > self.n:
             sim_g[:, self.n:] = float("nan")
-        sim_vel_scale = np.abs(sim_np[7 * self.J:]).max(axis=0)      # largest simulated velocity per env
         o = self.o_env.step(s, sim_np, want_terms=self.want_terms)
         self.g_env.step(s, sim_g, self.obs_g, self.reward_g, self.flags_g, self.terms_g)
         self.obs_o = o["obs"]
@@ -218,17 +216,21 @@ class Pair:
             np.testing.assert_array_equal(fg, o["flags"], err_msg=what + " flags")
         assert_close(rg, o["reward"], what=what + " reward")
         if self.want_terms:
-            # d(sum of squares) = 2 sqrt(J e) d(velocity) for the two velocity terms
-            slack = np.zeros_like(o["terms"])
-            for k in (1, 6):
-                slack[k] = 2.0 * np.sqrt(self.J * o["terms"][k]) * VEL_SLACK * sim_vel_scale
-            assert_close(self.terms_g.cpu().numpy(), o["terms"], what=what + " error terms", slack=slack)
+            extra = None
+            if self.vel_ulps:           # d(sum of squares) = 2 sqrt(J e) d(velocity) for the two velocity terms
+                scale = np.abs(sim_np[7 * self.J:]).max(axis=0)
+                extra = np.zeros_like(o["terms"])
+                for k in (1, 6):
+                    extra[k] = 2.0 * np.sqrt(self.J * o["terms"][k]) * self.vel_ulps * 2.0 ** -24 * scale
+            assert_close(self.terms_g.cpu().numpy(), o["terms"], what=what + " error terms", extra=extra)
         self.check_state(what)
         self.check_obs(what)
         if self.write_back:
-            wb_slack = np.zeros_like(sim_np, dtype=np.float64)
-            wb_slack[7 * self.J:] = VEL_SLACK * np.abs(sim_np[7 * self.J:]).max(axis=0)
-            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, atol=self.obs_atol, slack=wb_slack,
+            extra = None
+            if self.vel_ulps:
+                extra = np.zeros_like(sim_np, dtype=np.float64)
+                extra[7 * self.J:] = self.vel_ulps * 2.0 ** -24 * np.abs(sim_np[7 * self.J:]).max(axis=0)
+            assert_close(sim_g[:, :self.n].cpu().numpy(), sim_np, atol=self.obs_atol, extra=extra,
                          what=what + " written-back states")
         assert self.g_env.device_status() == 0
         self.max_err["reward"] = max(self.max_err["reward"], float(np.abs(rg - o["reward"]).max()))

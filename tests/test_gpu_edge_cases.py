@@ -69,7 +69,8 @@ def test_control_interval_off_the_keyframe_rate(dt):
 def test_clips_of_different_rates():
     sc = _scene("edge_fps", (361, 64, 28), "f32", n_clips=4, frames=(12, 30), fps=[24.0, 30.0, 60.0, 120.0],
                 dt=1.0 / 120.0)
-    p = Pair(sc, 200, with_policy=False)
+    # the 120 frames-per-second clip carries velocities four times the benchmark's: see Pair.vel_ulps
+    p = Pair(sc, 200, with_policy=False, vel_ulps=4)
     h = p.rollout(steps=8)
     assert any((x["flags"] & 2).any() for x in h)        # the short, fast clips truncate within a few steps
 
@@ -362,3 +363,46 @@ def test_extended_observation_is_validated():
     with pytest.raises(ValueError):
         env.set_obs_extension(1, act[:32])                   # fewer rows than envs
     assert env.set_obs_extension(1, act[:, :20]) == 381
+
+
+# ---------------------------------------------------------------- skeletons with many leaves
+def _custom_scene(name, parents, seed, n_clips=2, frames=(6, 12)):
+    J = len(parents)
+    parents = np.asarray(parents, np.int32)
+    wl = W.Workload(name, 100, "custom", n_clips, frames, 3, (24 * J + 1, 64, 8), "f32")
+    rng = np.random.default_rng(seed)
+    offsets = rng.uniform(-0.3, 0.3, (J, 3)).astype(np.float32)
+    offsets[0] = 0
+    has_child = np.zeros(J, bool)
+    has_child[parents[1:]] = True
+    skel = dict(kind="custom", J=J, parents=parents, offsets=offsets, masses=rng.uniform(1, 3, J).astype(np.float32),
+                ee_ids=np.nonzero(~has_child)[0].astype(np.int32))
+    lib = W.make_clip_library(J, n_clips, frames, 30.0, seed=seed)
+    pol = W.make_policy_weights(wl.mlp_dims, "f32", seed=seed)
+    return Scene(wl, skel, lib, pol)
+
+
+WIDE_TREES = {
+    "star12": [-1] + [0] * 11,                                     # 11 leaves under the root
+    "star32": [-1] + [0] * 31,                                     # 31 leaves: the widest tree there is
+    "broom20": [-1, 0, 1, 2] + [3] * 10 + [0] * 6,                 # a 4-link handle with 10 leaves, 6 more at the root
+}
+
+
+@pytest.mark.parametrize("tree", sorted(WIDE_TREES))
+@pytest.mark.parametrize("options", ["plain", "resets_written_back", "optional_semantics"])
+def test_skeletons_with_more_than_eight_leaves(tree, options):
+    """More than 8 root-to-leaf chains make a block of more than 256 threads, which runs the kernel
+    instantiation with the smaller register budget: the same comparison with the oracle as everywhere else."""
+    sc = _custom_scene("wide_" + tree, WIDE_TREES[tree], seed=len(tree))
+    assert (np.bincount(np.asarray(WIDE_TREES[tree][1:]), minlength=len(WIDE_TREES[tree])) == 0).sum() > 8
+    if options == "plain":
+        p = Pair(sc, 70, with_policy=False)
+    elif options == "resets_written_back":
+        p = Pair(sc, 70, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False)
+    else:
+        p = Pair(sc, 70, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, grace_steps=1, reset_noise_std=0.05,
+                 n_future=2, prev_action_dim=5)
+    h = p.rollout(steps=4)
+    if options != "plain":
+        assert any((x["flags"] != 0).any() for x in h)

@@ -100,16 +100,41 @@ def test_full_size(scenes, name):
     wl = W.WORKLOADS[name]
     p = Pair(scenes(name), wl.n_envs, policy_sample=192, want_terms=False)
     p.rollout(steps=3, device="cuda")
+    print("%s: largest observation error %.2e, largest reward error %.2e" % (name, p.max_err["obs"], p.max_err["reward"]))
+
+
+@pytest.mark.parametrize("name", ["cfg2_4096", "cfg3_16384_lib32", "cfg4_65536_smpl24", "cfg5_reset_heavy"])
+def test_full_batch_policy_step(scenes, name):
+    """One policy step on the whole batch of each bf16 configuration: every mean, noise and log-probability
+    element against the oracle (every row and column tile of the GEMM chain, CTA pairs included)."""
+    wl = W.WORKLOADS[name]
+    p = Pair(scenes(name), wl.n_envs, with_policy=True, want_terms=False)
+    p.reset_all()
+    p.policy_step(1)
+
+
+@pytest.mark.parametrize("name,n", [("cfg2_4096", 96 + 3), ("cfg3_16384_lib32", 128 + 5), ("cfg4_65536_smpl24", 64 + 7),
+                                    ("cfg5_reset_heavy", 256 + 1)])
+def test_rollouts_of_the_stated_length(scenes, name, n):
+    """Every configuration run to the rollout length it states (32 steps, 64 for the reset-heavy one) on a reduced
+    env count: resets, truncations at clip ends and re-draws accumulate over the whole horizon."""
+    wl = W.WORKLOADS[name]
+    p = Pair(scenes(name), n, write_back=name == "cfg5_reset_heavy")
+    h = p.rollout(steps=wl.steps, policy_every=8)
+    assert len(h) == wl.steps == (64 if name == "cfg5_reset_heavy" else 32)
+    if name == "cfg5_reset_heavy":
+        rate = np.mean([(x["flags"] != 0).mean() for x in h])
+        assert 0.08 < rate < 0.4
 
 
 # ---------------------------------------------------------------- edge cases
 def test_reward_threshold_termination(scenes):
     """Figure 5's done rule (root height or reward below a threshold); the reward threshold is set
     near the median reward of this workload so that both outcomes occur."""
-    p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.74, with_policy=False)
+    p = Pair(scenes("cfg1_tiny64"), 64, reward=W.REWARD_FIG5, h_min=0.55, r_min=0.865, with_policy=False)
     h = p.rollout(steps=5)
     frac = np.mean([(x["flags"] & 1).mean() for x in h])
-    assert 0.01 < frac < 0.99
+    assert 0.05 < frac < 0.95
 
 
 def test_all_reset_and_none_reset(scenes):
@@ -139,10 +164,9 @@ def test_single_body_and_max_bodies():
                     masses=rng.uniform(1, 3, J).astype(np.float32), ee_ids=np.nonzero(~has_child)[0].astype(np.int32))
         lib = W.make_clip_library(J, 2, (5, 9), 30.0, seed=J)
         pol = W.make_policy_weights(wl.mlp_dims, "f32", seed=J)
-        # fp32 rounding of the pose itself grows with the chain depth too: a 32-link chain (no
-        # benchmark skeleton is deeper than 9) is allowed 4e-5 on positions and orientations
-        p = Pair(Scene(wl, skel, lib, pol), 40, obs_atol=4e-5 if J == 32 else 1e-5)
+        p = Pair(Scene(wl, skel, lib, pol), 40)
         p.rollout(steps=3)
+        print("J = %d: largest observation error %.2e" % (J, p.max_err["obs"]))
 
 
 def test_sharded_envs_reproduce_the_unsplit_batch(scenes):

@@ -473,6 +473,51 @@ def test_reset_draws_are_uniform():
     assert O.reset_draw(ocl, cfg, 77, 1) != (c, t)
 
 
+def test_reset_draw_from_the_published_philox_words():
+    """Hand case on the first known-answer vector (counter 0, key 0 = env 0, step 0, seed 0): the clip comes from
+    word 0 by the high half of a 32 x 32 multiply, the phase from the top 24 bits of word 1."""
+    with open(os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    assert rows[0][:6] == ["00000000"] * 6
+    x0, x1 = int(rows[0][6], 16), int(rows[0][7], 16)
+    wl, skel, lib, pol, osk, ocl = scene_from_workload("cfg3_16384_lib32")
+    cfg = O.make_env_config(wl.dt, 0, W.REWARD_MULT, wl.h_min)
+    clip = (x0 * ocl.C) >> 32
+    u = np.float32((x1 >> 8) * 2.0 ** -24)
+    span = np.float32(np.float32(ocl.duration(clip)) - np.float32(wl.dt))
+    t = np.float32(u * span)
+    c, tt = O.reset_draw(ocl, cfg, 0, 0)
+    assert c == clip == 12 and tt.view(np.uint32) == t.view(np.uint32)      # 0x6627e8d5 * 32 >> 32 = 12
+    # a draw that took both from word 0, or swapped the words, would give another pair
+    assert (x1 * ocl.C) >> 32 != clip and np.float32((x0 >> 8) * 2.0 ** -24) != u
+
+
+def test_reset_clip_and_phase_are_jointly_uniform():
+    """2-D chi-square over (clip, phase decile) of a million draws: uniform marginals alone would also pass
+    if clip and phase came from the same Philox word; the joint table does not."""
+    J = 1
+    lib = W.make_clip_library(J, 32, (60, 600), 30.0, seed=3)
+    osk = O.Skeleton([-1], np.zeros((1, 3), np.float32))
+    ocl = O.Clips(osk, lib["n_frames"], lib["fps"], lib["root_pos"], lib["local_quat"])
+    dt = 1.0 / 30.0
+    cfg = O.make_env_config(dt, 2024, W.REWARD_MULT, 0.0)
+    n = 1000000
+    env = O.Env(osk, ocl, cfg, n)
+    env.reset_all(0)
+    dur = np.array([ocl.duration(c) for c in range(ocl.C)], np.float32)
+    u = env.t / (dur[env.clip_id] - np.float32(dt))
+    decile = np.minimum((u * 10).astype(np.int64), 9)
+    table = np.bincount(env.clip_id.astype(np.int64) * 10 + decile, minlength=320).reshape(32, 10)
+    assert table.sum() == n
+    assert scipy.stats.chisquare(table.ravel()).pvalue > 1e-4                       # all 320 cells equally likely
+    assert scipy.stats.chi2_contingency(table)[1] > 1e-4                            # clip independent of phase
+    # the test has power: the same statistic on draws that reuse one word for both is hopeless
+    x = np.random.default_rng(0).integers(0, 2 ** 32, n, dtype=np.uint64)
+    fake = np.bincount(((x * 32) >> 32).astype(np.int64) * 10 + np.minimum(((x >> 8) * 10) >> 24, 9).astype(np.int64),
+                       minlength=320).reshape(32, 10)
+    assert scipy.stats.chisquare(fake.ravel()).pvalue < 1e-12
+
+
 def test_forced_all_and_none_reset():
     for h_min, frac in [(10.0, 1.0), (-10.0, None)]:
         wl, skel, lib, pol, osk, ocl = scene_from_workload("cfg1_tiny64")

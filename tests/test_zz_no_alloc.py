@@ -6,13 +6,16 @@ use im_policy_forward_noalloc, whose hidden activations live in a fixed array in
 This test calls it through the C ABI twice in a row and requires the same means, actions and
 log-probabilities as im_policy_forward on the same weights and observations, within the
 tolerance the parity tests use for the fp32 policy; the second call also checks that what the
-first call left in the shared array does no harm.  The file sorts last so that a run that stops
-at the first failure has already run everything else.
+first call left in the shared array does no harm.  Both calls are also compared with the CPU
+oracle directly, and the device's free memory must be the same before and after a call once the
+first call has been made.  The file sorts last so that a run that stops at the first failure has
+already run everything else.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_2609_09821_b200 import binding as B
 from paper_2609_09821_b200 import workloads as W
 from tests.parity import assert_close, assert_mean_close
@@ -50,6 +53,18 @@ def test_noalloc_policy_matches_regular_policy_twice():
         logp = torch.full((n,), float("nan"), device="cuda")
         B.policy_forward_noalloc(pol["dims"], Wd, bd, sigma, seed, step, obs, mean, act, logp)
         torch.cuda.synchronize()
+        # once the first call has run, a call leaves the device's free memory where it was
+        free_before = torch.cuda.mem_get_info()[0]
+        B.policy_forward_noalloc(pol["dims"], Wd, bd, sigma, seed, step, obs, mean, act, logp)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        # the oracle itself, not only the library's other path
+        o = O.policy_forward(pol["dims"], pol["W"], pol["b"], sigma, seed, step,
+                             obs[:, :361].cpu().numpy().astype(np.float64), env_ids=np.arange(n, dtype=np.uint32))
+        assert_mean_close(mean.cpu().numpy(), o["mean"], 1e-4, what="step %d vs oracle" % step)
+        assert_close((act - mean).cpu().numpy().astype(np.float64), sigma * o["z"], atol=1e-5, rtol=1e-4,
+                     what="step %d action noise vs oracle" % step)
+        assert_close(logp.cpu().numpy(), o["logp"], atol=1e-3, rtol=1e-5, what="step %d logp vs oracle" % step)
         assert_mean_close(mean.cpu().numpy(), want_mean.cpu().numpy(), 1e-4, what="step %d" % step)
         noise = (act - mean).cpu().numpy().astype(np.float64)
         want_noise = (want_act - want_mean).cpu().numpy().astype(np.float64)
