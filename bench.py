@@ -8,9 +8,17 @@ forward + Gaussian sampling on the current observations, then the fused env
 step (reference lookup/FK, reward, flags, masked reset, next observation) on
 that step's simulated body states.  Prints one JSON line (rank 0).
 
+The timed region is a CUDA graph of K steps, replayed REPLAYS times; `value` is the median replay
+(`replays` carries the spread), `sustained` a loop of replays at least a second long with the SM
+clock sampled beside it.  With the default workload the other four configurations are measured too
+(`other_configs`, each in a process of its own).
+
 `--impl reference` times the CPU oracle on a bounded sample of the same
 workload on the host cores (a deliberately plain program: a baseline, not a
 target).
+
+`--only env|policy|gae|ppo_loss|update` runs one piece in a plain timing loop and prints its own
+JSON line: the entry point the kernel profiles under profiles/ were captured through.
 """
 from __future__ import annotations
 
@@ -44,11 +52,15 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per step from the committed ncu captures
-# (profiles/*_cfg4_65536_smpl24.md): the four policy kernels, and the env step kernel.
-NCU_TRAFFIC_BYTES = {
-    "cfg4_65536_smpl24": dict(policy=(85.2 + 81.5 + 136.3 + 90.9 + 135.3 + 35.9 + 67.2 + 3.7) * 1e6,
-                              env=(89.3 + 202.1) * 1e6),
+REPLAYS = 21            # replays of the K-step graph; the median is reported
+SUSTAINED_SECONDS = 1.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the kernels named in `capture`
+# (one launch each, 65536 envs); None where the timed path runs another kernel variant than the captured one.
+NCU_TRAFFIC = {
+    "cfg4_65536_smpl24": dict(
+        policy=dict(bytes=None, capture=None),
+        env=dict(bytes=None, capture=None)),
 }
 
 
@@ -149,6 +161,133 @@ def oracle_leg(wl: W.Workload, skel, lib, pol, n_sample: int, steps: int, warmup
                 ms_per_step=1e3 * state["t"] / done, wall_s=time.perf_counter() - t_start)
 
 
+# ----------------------------------------------------------------------------- rollout-side pieces
+# Timed on their own (not part of the metric).
+def time_gae(B, wl, n, dev, stream, reps=20):
+    """The advantage estimator over one rollout of wl.steps steps.  Its 17 B per env-step fit in L2, so a 256 MB
+    buffer is read before every launch (reading leaves clean lines behind: a written buffer's write-back would
+    be charged to the kernel)."""
+    import torch
+    T = wl.steps
+    r_np, v_np, f_np = W.make_rollout_signals(T, n, wl.seed)
+    r_d, v_d, f_d = (torch.from_numpy(a).to(dev) for a in (r_np, v_np, f_np))
+    adv_d, ret_d = torch.empty((T, n), device=dev), torch.empty((T, n), device=dev)
+    flush = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
+    t_gae = []
+    for i in range(3 + reps):
+        flush.sum()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.gae(r_d, v_d, f_d, adv_d, ret_d, 0.99, 0.95, True, stream=stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_gae.append(a.elapsed_time(b) * 1e-3)
+    t_gae = float(np.median(t_gae))
+    gae_bytes = T * n * 17 + n * 4
+    return dict(T=T, seconds_per_launch=t_gae, algorithmic_bytes=gae_bytes, achieved_gbs=gae_bytes / t_gae / 1e9,
+                l2="256 MB read before every launch")
+
+
+def time_ppo_loss(B, wl, n, A, dev, stream, reps=20):
+    """PPO minibatch loss: one of four minibatches of the rollout (T * n / 4 samples), moments + loss + finish."""
+    import torch
+    Mb = wl.steps * n // 4
+    pb = {k: torch.from_numpy(v).to(dev) for k, v in W.make_ppo_batch(min(Mb, 65536), A, wl.seed, drift=0.02).items()}
+    reps_rows = (Mb + pb["mean"].shape[0] - 1) // pb["mean"].shape[0]
+    for k in ("mean", "action", "mean_old"):
+        pb[k] = pb[k].repeat(reps_rows, 1)[:Mb].contiguous()
+    for k in ("logp_old", "advantage", "value", "value_old", "returns"):
+        pb[k] = pb[k].repeat(reps_rows)[:Mb].contiguous()
+    ws, mom = B.ppo_workspace(), torch.empty(2, device=dev)
+    outs = [torch.empty((Mb, A), device=dev), torch.empty(A, device=dev), torch.empty(Mb, device=dev),
+            torch.empty(6, device=dev)]
+    t_ppo = []
+    for i in range(3 + reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.moments(pb["advantage"], mom, ws, stream=stream)
+        B.ppo_loss(pb, *outs, ws, 0.2, 2.0, 2.5e-4, True, adv_moments=mom, stream=stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_ppo.append(a.elapsed_time(b) * 1e-3)
+    t_ppo = float(np.median(t_ppo))
+    ppo_bytes = Mb * ((3 * A + 5) * 4 + (A + 1) * 4 + 4)
+    return dict(rows=Mb, A=A, seconds_per_launch=t_ppo, algorithmic_bytes=ppo_bytes, achieved_gbs=ppo_bytes / t_ppo / 1e9,
+                l2="%.0f MB working set, larger than L2" % (ppo_bytes / 1e6))
+
+
+def time_update(B, wl, pol, n, A, D, dev, stream, graph=True, reps=5):
+    """One whole PPO minibatch update (actor + critic forward, loss, both backward passes, clip, Adam, learning
+    rate) on 2 * n rows, a sixteenth of the rollout, through paper_2609_09821_b200.trainer."""
+    import torch
+    from paper_2609_09821_b200 import trainer as TR
+    Mu = 2 * n
+    adims, cdims_u = tuple(wl.mlp_dims), tuple(wl.mlp_dims[:-1]) + (1,)
+    cwu = W.make_policy_weights(cdims_u, "bf16", wl.seed + 1)
+    with torch.cuda.stream(stream):
+        actor_t = TR.MlpTrainer(adims, pol["W"], pol["b"], Mu, stream=stream)
+        critic_t = TR.MlpTrainer(cdims_u, cwu["W"], cwu["b"], Mu, stream=stream)
+        upd = TR.PpoUpdater(actor_t, critic_t, torch.full((A,), -2.0), lr=5e-4, clip=0.2, value_coef=2.0)
+        gen = torch.Generator(device=dev).manual_seed(wl.seed)
+        for tr_ in (actor_t, critic_t):
+            rows_ = tr_.input_rows(Mu)
+            rows_.zero_()
+            rows_[:, :D] = torch.randn((Mu, D), device=dev, generator=gen).to(torch.bfloat16)
+        rnd = lambda *sh: torch.randn(*sh, device=dev, generator=gen)
+        ub = dict(action=rnd(Mu, A) * 0.2, mean_old=rnd(Mu, A) * 0.2, log_std_old=torch.full((A,), -2.0, device=dev),
+                  logp_old=rnd(Mu) + 60.0, advantage=rnd(Mu), value_old=rnd(Mu), returns=rnd(Mu))
+        for i in range(2):
+            upd.update(Mu, ub)
+        stream.synchronize()
+        up_graph = None
+        if graph:
+            # the update's ~100 launches are replayed from one CUDA graph, as a training loop would run them
+            up_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(up_graph, stream=stream):
+                upd.update(Mu, ub)
+        t_up = []
+        for i in range(1 + reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            if up_graph is not None:
+                up_graph.replay()
+            else:
+                upd.update(Mu, ub)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 1:
+                t_up.append(a.elapsed_time(b) * 1e-3)
+    t_up = float(np.median(t_up))
+    up_flops = 3 * (mlp_flops_per_env(adims) + mlp_flops_per_env(cdims_u)) * Mu      # forward + two backward products
+    return dict(rows=Mu, seconds_per_update=t_up, achieved_tflops=up_flops / t_up / 1e12,
+                status=[actor_t.device_status(), critic_t.device_status()],
+                launch="cuda_graph" if graph else "stream",
+                note="forward + backward + Adam of actor and critic on one minibatch; flops = 3 x forward flops")
+
+
+def only_rollout_piece(args):
+    """`--only gae|ppo_loss|update`: that piece alone, in the loop the profiles of those kernels were taken from."""
+    import torch
+    from paper_2609_09821_b200 import binding as B
+    B.load()
+    wl = W.WORKLOADS[args.workload]
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+    n, A, D = wl.n_envs, wl.act_dim, wl.obs_dim
+    if args.only == "gae":
+        res = time_gae(B, wl, n, dev, stream, reps=args.launches)
+    elif args.only == "ppo_loss":
+        res = time_ppo_loss(B, wl, n, A, dev, stream, reps=args.launches)
+    else:
+        pol = W.make_policy_weights(wl.mlp_dims, wl.mlp_dtype, wl.seed)
+        res = time_update(B, wl, pol, n, A, D, dev, stream, graph=not args.no_graph, reps=args.launches)
+    print(json.dumps(dict(only=args.only, workload=wl.name, **res)))
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -164,7 +303,13 @@ def main():
                     help="skip the separate timing of the value head and the advantage estimator")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short device-resident runs of the other benchmark configurations")
+    ap.add_argument("--replays", type=int, default=REPLAYS, help="replays of the K-step graph (median reported)")
+    ap.add_argument("--only", default=None, choices=["env", "policy", "gae", "ppo_loss", "update"],
+                    help="time one piece in a plain loop and print its own JSON line")
+    ap.add_argument("--launches", type=int, default=40, help="launches of the --only loop")
     args = ap.parse_args()
+    if args.only in ("gae", "ppo_loss", "update"):
+        return only_rollout_piece(args)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -279,25 +424,73 @@ def main():
         env.set_state(c0, t0, l0)
         obs.copy_(obs0)
         torch.cuda.synchronize()
+    if args.only in ("env", "policy"):
+        # plain loop over the step buffers (together larger than L2), the piece alone
+        res = []
+        for rep in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(args.launches):
+                s_ = Wm + 1 + i
+                if args.only == "env":
+                    env.step(s_, sims[i % n_buf], obs, reward, flags)
+                else:
+                    policy_forward(s_)
+            b.record(stream)
+            torch.cuda.synchronize()
+            res.append(a.elapsed_time(b) / args.launches * 1e3)
+        if rank == 0:
+            print(json.dumps(dict(only=args.only, workload=wl.name, us_per_launch=res, launches=args.launches,
+                                  bf16_rows=bool(staged), reset_fraction=float((flags != 0).float().mean()))))
+        return
+
     sampler = ClockSampler(local_rank)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(1, args.replays) if graph is not None else 1
+    evs_r = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
     barrier()
     sampler.start()
     before = B.launch_count()
-    ev0.record(stream)
-    if graph is not None:
-        graph.replay()
-    else:
-        run_steps(Wm + 1, K)
-    ev1.record(stream)
+    for ev0, ev1 in evs_r:
+        ev0.record(stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            run_steps(Wm + 1, K)
+        ev1.record(stream)
     barrier()
     clocks = sampler.stop()
     launches = launches_per_replay if graph is not None else B.launch_count() - before
-    ms = ev0.elapsed_time(ev1)
+    times = np.array([a.elapsed_time(b) for a, b in evs_r])
     if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+        tmax = torch.from_numpy(times).to(dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)        # every replay takes as long as its slowest rank
+        times = tmax.cpu().numpy()
+    ms = float(np.median(times))
+    replays = dict(count=int(reps), ms_median=ms, ms_min=float(times.min()), ms_max=float(times.max()),
+                   note="each replay is the K-step graph; value = n_envs * K / median")
+
+    # ---- the same graph replayed back to back for at least a second: the settled figure under the power cap
+    sustained = None
+    if graph is not None and SUSTAINED_SECONDS > 0:
+        n_rep = max(int(np.ceil(SUSTAINED_SECONDS * 1e3 / ms)), 2)
+        s_sampler = ClockSampler(local_rank)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        s_sampler.start()
+        ev0.record(stream)
+        for _ in range(n_rep):
+            graph.replay()
+        ev1.record(stream)
+        barrier()
+        s_clocks = s_sampler.stop()
+        s_ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            tmax = torch.tensor([s_ms], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            s_ms = float(tmax.item())
+        sustained = dict(value=world * n * K * n_rep / (s_ms * 1e-3), unit=UNIT, seconds=s_ms * 1e-3, replays=n_rep,
+                         ms_per_step=s_ms / (K * n_rep), clocks=s_clocks,
+                         ms_per_step_times_sm_mhz=(s_ms / (K * n_rep)) * s_clocks["sm_mhz"] if s_clocks.get("sm_mhz") else None)
 
     # ---- per-call breakdown (stream launches with events around each call) for the rooflines
     env.reset_all(obs, 0)
@@ -322,95 +515,9 @@ def main():
     extras = None
     if not args.no_rollout_extras and rank == 0:
         reps = 20
-        T = wl.steps
-        r_np, v_np, f_np = W.make_rollout_signals(T, n, wl.seed)
-        r_d, v_d, f_d = (torch.from_numpy(a).to(dev) for a in (r_np, v_np, f_np))
-        adv_d, ret_d = torch.empty((T, n), device=dev), torch.empty((T, n), device=dev)
-        flush = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
-        t_gae = []
-        for i in range(3 + reps):
-            flush.sum()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            B.gae(r_d, v_d, f_d, adv_d, ret_d, 0.99, 0.95, True, stream=stream)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                t_gae.append(a.elapsed_time(b) * 1e-3)
-        t_gae = float(np.median(t_gae))
-        gae_bytes = T * n * 17 + n * 4
-        extras = dict(gae=dict(T=T, seconds_per_launch=t_gae, algorithmic_bytes=gae_bytes,
-                               achieved_gbs=gae_bytes / t_gae / 1e9, l2="256 MB read before every launch"))
-        # PPO minibatch loss: one of four minibatches of the rollout (T * n / 4 samples), moments + loss + finish
-        Mb = T * n // 4
-        pb = {k: torch.from_numpy(v).to(dev) for k, v in W.make_ppo_batch(min(Mb, 65536), A, wl.seed, drift=0.02).items()}
-        reps_rows = (Mb + pb["mean"].shape[0] - 1) // pb["mean"].shape[0]
-        for k in ("mean", "action", "mean_old"):
-            pb[k] = pb[k].repeat(reps_rows, 1)[:Mb].contiguous()
-        for k in ("logp_old", "advantage", "value", "value_old", "returns"):
-            pb[k] = pb[k].repeat(reps_rows)[:Mb].contiguous()
-        ws, mom = B.ppo_workspace(), torch.empty(2, device=dev)
-        outs = [torch.empty((Mb, A), device=dev), torch.empty(A, device=dev), torch.empty(Mb, device=dev),
-                torch.empty(6, device=dev)]
-        t_ppo = []
-        for i in range(3 + reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            B.moments(pb["advantage"], mom, ws, stream=stream)
-            B.ppo_loss(pb, *outs, ws, 0.2, 2.0, 2.5e-4, True, adv_moments=mom, stream=stream)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                t_ppo.append(a.elapsed_time(b) * 1e-3)
-        t_ppo = float(np.median(t_ppo))
-        ppo_bytes = Mb * ((3 * A + 5) * 4 + (A + 1) * 4 + 4)
-        extras["ppo_loss"] = dict(rows=Mb, A=A, seconds_per_launch=t_ppo, algorithmic_bytes=ppo_bytes,
-                                  achieved_gbs=ppo_bytes / t_ppo / 1e9,
-                                  l2="%.0f MB working set, larger than L2" % (ppo_bytes / 1e6))
-        del pb, outs
+        extras = dict(gae=time_gae(B, wl, n, dev, stream, reps), ppo_loss=time_ppo_loss(B, wl, n, A, dev, stream, reps))
         if staged:
-            # one whole PPO minibatch update (actor + critic forward, loss, both backward passes, clip, Adam,
-            # learning rate): 2 * n rows, a sixteenth of the rollout, through paper_2609_09821_b200.trainer
-            from paper_2609_09821_b200 import trainer as TR
-            Mu = 2 * n
-            adims, cdims_u = tuple(wl.mlp_dims), tuple(wl.mlp_dims[:-1]) + (1,)
-            cwu = W.make_policy_weights(cdims_u, "bf16", wl.seed + 1)
-            with torch.cuda.stream(stream):
-                actor_t = TR.MlpTrainer(adims, pol["W"], pol["b"], Mu, stream=stream)
-                critic_t = TR.MlpTrainer(cdims_u, cwu["W"], cwu["b"], Mu, stream=stream)
-                upd = TR.PpoUpdater(actor_t, critic_t, torch.full((A,), -2.0), lr=5e-4, clip=0.2, value_coef=2.0)
-                gen = torch.Generator(device=dev).manual_seed(wl.seed)
-                for tr_ in (actor_t, critic_t):
-                    rows_ = tr_.input_rows(Mu)
-                    rows_.zero_()
-                    rows_[:, :D] = torch.randn((Mu, D), device=dev, generator=gen).to(torch.bfloat16)
-                rnd = lambda *sh: torch.randn(*sh, device=dev, generator=gen)
-                ub = dict(action=rnd(Mu, A) * 0.2, mean_old=rnd(Mu, A) * 0.2, log_std_old=torch.full((A,), -2.0, device=dev),
-                          logp_old=rnd(Mu) + 60.0, advantage=rnd(Mu), value_old=rnd(Mu), returns=rnd(Mu))
-                for i in range(2):
-                    upd.update(Mu, ub)
-                stream.synchronize()
-                # the update's ~100 launches are replayed from one CUDA graph, as a training loop would run them
-                up_graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(up_graph, stream=stream):
-                    upd.update(Mu, ub)
-                t_up = []
-                for i in range(1 + 5):
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record(stream)
-                    up_graph.replay()
-                    b.record(stream)
-                    torch.cuda.synchronize()
-                    if i >= 1:
-                        t_up.append(a.elapsed_time(b) * 1e-3)
-            t_up = float(np.median(t_up))
-            up_flops = 3 * (mlp_flops_per_env(adims) + mlp_flops_per_env(cdims_u)) * Mu      # forward + two backward products
-            extras["ppo_update"] = dict(rows=Mu, seconds_per_update=t_up, achieved_tflops=up_flops / t_up / 1e12,
-                                        status=[actor_t.device_status(), critic_t.device_status()],
-                                        launch="cuda_graph",
-                                        note="forward + backward + Adam of actor and critic on one minibatch; "
-                                             "flops = 3 x forward flops")
-            del up_graph, actor_t, critic_t, upd, ub
+            extras["ppo_update"] = time_update(B, wl, pol, n, A, D, dev, stream)
         if staged:
             cdims = tuple(wl.mlp_dims[:-1]) + (1,)
             cw = W.make_policy_weights(cdims, "bf16", wl.seed + 1)
@@ -443,7 +550,6 @@ def main():
                     t_s.append(a.elapsed_time(b) * 1e-3 / 8)
             extras["env_step_bf16_rows_only"] = dict(seconds_per_launch=float(np.median(t_s)),
                                                      note="im_env_step with obs_out == NULL while attached to the policy")
-        del flush
 
     # ---- end to end through the host-buffer entry point: pinned host inputs, results read back
     e2e = None
@@ -482,12 +588,17 @@ def main():
     tf = flops / t_pol / 1e12
     gbs = env_bytes / t_env / 1e9
     tensor_peak = peaks["bf16_tflops_sustained"]
-    traffic = NCU_TRAFFIC_BYTES.get(wl.name, {})
+    traffic = NCU_TRAFFIC.get(wl.name, dict(policy=dict(bytes=None, capture=None), env=dict(bytes=None, capture=None)))
+    # the K-step replays last milliseconds: the burst peak is the denominator that applies to them; the
+    # fraction of the sustained peak is given beside it (it applies to the `sustained` loop)
     roofline = dict(bound="tensor", kernel="policy forward (GEMM chain + Gaussian head)", achieved=tf,
-                    peak=tensor_peak, unit="TFLOP/s", frac=tf / tensor_peak, traffic=traffic.get("policy"),
-                    peak_source="%s bf16 sustained" % peaks["source"], seconds_per_launch=t_pol)
+                    peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tf / peaks["bf16_tflops"],
+                    frac_burst=tf / peaks["bf16_tflops"], frac_sustained=tf / tensor_peak,
+                    peak_sustained=tensor_peak, traffic=traffic["policy"]["bytes"], traffic_capture=traffic["policy"]["capture"],
+                    peak_source="%s bf16 burst (timed region of milliseconds)" % peaks["source"], seconds_per_launch=t_pol)
     roofline_env = dict(bound="hbm", kernel="env_step_kernel", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=gbs / peaks["hbm_gbs"], traffic=traffic.get("env"), peak_source="%s copy" % peaks["source"],
+                        frac=gbs / peaks["hbm_gbs"], traffic=traffic["env"]["bytes"], traffic_capture=traffic["env"]["capture"],
+                        peak_source="%s copy" % peaks["source"],
                         seconds_per_launch=t_env, algorithmic_bytes=env_bytes)
     if wl.mlp_dtype != "bf16":
         roofline["bound"] = "alu"
@@ -500,7 +611,9 @@ def main():
                 ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16" if wl.mlp_dtype == "bf16" else "f32", data="synthetic", config=config,
                 clocks=clocks, gpu_launches=int(launches), roofline=roofline, roofline_env=roofline_env,
-                breakdown_ms=dict(policy_forward=t_pol * 1e3, env_step=t_env * 1e3))
+                breakdown_ms=dict(policy_forward=t_pol * 1e3, env_step=t_env * 1e3), replays=replays)
+    if sustained is not None:
+        line["sustained"] = sustained
     if e2e is not None:
         line["e2e"] = e2e
     if extras is not None:
@@ -511,7 +624,7 @@ def main():
         if "value_head" in extras:
             extras["value_head"]["frac_of_tensor_peak"] = extras["value_head"]["achieved_tflops"] / tensor_peak
         line["rollout_extras"] = extras
-    if world == 1 and not args.no_other_configs and args.workload == DEFAULT_WORKLOAD and args.steps is None:
+    if world == 1 and not args.no_other_configs and args.workload == DEFAULT_WORKLOAD:
         # the other configurations, device-resident numbers only, each in a process of its own (this one's
         # buffers are released first); the headline stays the default workload's
         import subprocess
@@ -525,12 +638,14 @@ def main():
             cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--warmup", str(max(Wm, 3)),
                    "--no-cpu-baseline", "--no-e2e", "--no-rollout-extras", "--no-other-configs"]
             try:
-                out = subprocess.run(cmd, capture_output=True, text=True, timeout=120)
+                out = subprocess.run(cmd, capture_output=True, text=True, timeout=180)
                 d = json.loads(out.stdout.strip().splitlines()[-1])
                 others[name] = dict(value=d["value"], unit=UNIT, ms_per_step=d["ms_per_step"], steps=d["steps"],
-                                    n_envs=d["config"]["n_envs_per_gpu"], dtype=d["dtype"],
-                                    policy_frac_of_tensor_peak=d["roofline"]["frac"] if d["dtype"] == "bf16" else None,
-                                    env_frac_of_hbm_peak=d["roofline_env"]["frac"], sm_mhz=d["clocks"].get("sm_mhz"))
+                                    n_envs=d["config"]["n_envs_per_gpu"], dtype=d["dtype"], replays=d["replays"],
+                                    sustained=d.get("sustained", {}).get("value"),
+                                    roofline=d["roofline"] if d["dtype"] == "bf16" else None,
+                                    roofline_env=d["roofline_env"], breakdown_ms=d["breakdown_ms"],
+                                    sm_mhz=d["clocks"].get("sm_mhz"))
             except Exception as exc:                     # a side measurement must not take the headline down with it
                 others[name] = dict(error=repr(exc)[:200])
         line["other_configs"] = others
