@@ -459,29 +459,22 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   N and K multiples of 64; lda, ldb, ldc multiples of 8; all pointers 16-byte aligned;
  *   bias float [N] (pass zeros for none); status DEVICE uint32 [1] receives
  *   IM_DEV_WAIT_TIMEOUT if a bounded wait inside the kernel runs out.
- * im_gemm_bf16_batched: `batches` independent products in one launch, stacked along the rows:
- *   batch b multiplies A[bM .. bM+M) with B[bN .. bN+N) into C[bM .. bM+M); M a multiple of 128
- *   when batches > 1.  Used to split the long batch-dimension contraction of dW into slices that
- *   fill the machine; im_sum_slices_bf16_to_f32 then adds the slices (in order, fp32) into a dense
- *   float matrix: out[r][c] = sum_s in[s * slice_stride + r * ld_in + c].
  * im_gemm_bf16_tn: the transposed product of two row-major matrices without transposing either:
  *   C_s[Mo][No] = sum over rows r of slice s of A[r][0..Mo) (x) B[r][0..No), for `slices` equal
  *   ranges of the R rows (R a multiple of 64 * slices), partial results stacked c_pitch rows apart
  *   (c_pitch >= Mo, a multiple of 128; rows Mo..c_pitch of a slice are written as zeros).  The
- *   tensor cores read both operands M/N-major.  No a multiple of 64; zeros: DEVICE, non-NULL, kept for
- *   call compatibility (the product has no bias and the buffer is not read).
+ *   tensor cores read both operands M/N-major.  No a multiple of 64.  The slices split the long
+ *   batch-dimension contraction of dW so that it fills the machine; im_sum_slices_bf16_to_f32 then adds
+ *   them (in order, fp32) into a dense float matrix: out[r][c] = sum_s in[s * slice_stride + r * ld_in + c].
  * im_gemm_bf16_f32out: C[M][N] float, dense = A[M][K] B[N][K]^T + bias, N <= 80; B and bias
  *   must hold ceil(N / 16) * 16 rows / floats (the extra ones zero).
  * im_transpose_bf16: out[c][r] = in[r][c] for a [rows][cols] matrix.
- * im_relu_mask_bf16: dH[r][c] = H[r][c] > 0 ? dH[r][c] : 0 in place; cols, ld_d, ld_h
- *   multiples of 8, 16-byte aligned pointers.
  * im_gemm_bf16_dgrad: the backward product through a linear layer fused with what follows it,
  *   dH[r][c] = (H[r][c] > 0) * sum_k dZ[r][k] Wt[c][k]  as bf16 [M][N] (Wt = the layer's weights transposed,
  *   bf16 [N][K]; H = the forward activations the ReLU produced, bf16 [M][N], or NULL for no mask), and
  *   colsum_partial[(r / 32) * ld_partial + c] = the sum of the fp32 values of dH over the 32-row block
  *   (float [M / 32][ld_partial], or NULL); summing those rows with im_colsum_f32 gives the bias gradient
- *   of the layer below.  M a multiple of 32; zeros: DEVICE, non-NULL, kept for call compatibility (not
- *   read: the product has no bias); the other rules of im_gemm_bf16 apply.
+ *   of the layer below.  M a multiple of 32; the product has no bias; the other rules of im_gemm_bf16 apply.
  * im_f32_to_bf16_padded: out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
  * im_gather_rows_f32: out[i][0..cols) = in[idx[i]][0..cols) for i < rows (shuffled minibatches); idx
  *   DEVICE int32 [rows] with values in [0, n_src); out is float [rows][ld_out], or with to_bf16 != 0
@@ -489,8 +482,7 @@ im_status im_policy_layer_buffers(im_policy *p, int32_t layer, void **W, int32_t
  *   and sets IM_DEV_BAD_STATE in *status (DEVICE uint32).
  * im_copy_f32: dst[0..n) = src[0..n), DEVICE to DEVICE on the stream (e.g. a trained bias vector
  *   into the buffer im_policy_layer_buffers returns).
- * im_bf16_to_f32: out (float, dense [rows][cols]) = in (bf16, row stride ld_in).
- * im_colsum_f32 / im_colsum_bf16: out[c] = sum_r x[r][c], float [cols]; rows are summed in
+ * im_colsum_f32: out[c] = sum_r x[r][c], float [cols]; rows are summed in
  *   fp32 within slices of 256 rows and the slices in a fixed order in fp64 (bit-reproducible);
  *   workspace DEVICE, at least ceil(rows / 256) * cols * 4 bytes. */
 im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
@@ -498,31 +490,137 @@ im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_
                        void *cuda_stream);
 im_status im_gemm_bf16_dgrad(const uint16_t *dZ, int64_t ld_dz, const uint16_t *Wt, int64_t ld_wt, uint16_t *dH, int64_t ld_dh,
                              int32_t M, int32_t N, int32_t K, const uint16_t *H, int64_t ld_h, float *colsum_partial,
-                             int32_t ld_partial, const float *zeros, uint32_t *status, void *cuda_stream);
-im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
-                               int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
-                               uint32_t *status, void *cuda_stream);
+                             int32_t ld_partial, uint32_t *status, void *cuda_stream);
 im_status im_gemm_bf16_tn(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
-                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, const float *zeros,
-                          uint32_t *status, void *cuda_stream);
+                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, uint32_t *status,
+                          void *cuda_stream);
 im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
                                     int32_t cols, float *out, void *cuda_stream);
 im_status im_gemm_bf16_f32out(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, float *C, int32_t M,
                               int32_t N, int32_t K, const float *bias, uint32_t *status, void *cuda_stream);
 im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int64_t ld_out,
                             void *cuda_stream);
-im_status im_relu_mask_bf16(uint16_t *dH, int64_t ld_d, const uint16_t *H, int64_t ld_h, int32_t rows, int32_t cols,
-                            void *cuda_stream);
 im_status im_f32_to_bf16_padded(const float *in, int64_t ld_in, int32_t rows, int32_t cols, uint16_t *out, int32_t ld_out,
                                 void *cuda_stream);
 im_status im_gather_rows_f32(const float *in, int64_t ld_in, const int32_t *idx, int64_t n_src, int32_t rows, int32_t cols,
                              void *out, int32_t ld_out, int32_t to_bf16, uint32_t *status, void *cuda_stream);
 im_status im_copy_f32(float *dst, const float *src, int64_t n, void *cuda_stream);
-im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream);
 im_status im_colsum_f32(const float *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
                         size_t workspace_bytes, void *cuda_stream);
-im_status im_colsum_bf16(const uint16_t *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
-                         size_t workspace_bytes, void *cuda_stream);
+
+/* ---- the update phase as handles ------------------------------------------------
+ * (The paper's training loop, Figure 2: `update_policy(storage)` after every rollout; Section 4.1 runs
+ * the PPO update as one compiled unit, and Section 4.2 keeps the host out of it.  The hyper-parameter
+ * table names what im_ppo_update_config holds: learning rate, ratio clip, value-loss and entropy
+ * coefficients, KL threshold, gradient clipping.)
+ *
+ * im_trainer: one MLP in training form -- fp32 master weights and Adam moments, bf16 working copies of the
+ * weights and of their transposes (padded to the 64-column tiles of the tensor-core kernels), one bf16
+ * activation buffer per layer, gradient buffers, and the scratch of the backward pass -- for minibatches of up
+ * to max_rows rows.  Hidden widths must be multiples of 64, the output width at most 80, max_rows a multiple
+ * of 64.  W, b: HOST arrays of n_layers HOST pointers (W[l] float [dims[l+1]][dims[l]], b[l] float
+ * [dims[l+1]]), copied.  All later calls only enqueue kernels on cuda_stream: no host read, no allocation,
+ * capturable.
+ *   im_trainer_forward   runs the net on the first M rows of the input buffer (IM_TRAINER_H of layer 0: bf16
+ *                        [max_rows][ld], filled by the caller, columns beyond dims[0] zero) and leaves the fp32
+ *                        outputs in IM_TRAINER_OUT; every layer's activation is kept for the backward pass.
+ *   im_trainer_backward  d_out DEVICE float [M][dims[last]] = dL/d(outputs) of that forward; M a multiple of 64.
+ *                        Fills the gradients IM_TRAINER_DW / IM_TRAINER_DB of every layer:
+ *                        dW_l = dZ_l^T H_{l-1} (im_gemm_bf16_tn over row slices + im_sum_slices_bf16_to_f32),
+ *                        dZ_{l-1} = (H_{l-1} > 0) (dZ_l W_l) and its column sums (im_gemm_bf16_dgrad + im_colsum_f32).
+ *   im_trainer_step      one Adam step on every tensor (im_adam_step; lr and grad_scale DEVICE float [1],
+ *                        grad_scale may be NULL); the bf16 copies and their transposes follow.
+ *   im_trainer_push_to_policy  writes the current weights and biases into a loaded im_policy of the same
+ *                        shape and stream, so the next rollout acts with the trained network.
+ *   im_trainer_tensor    DEVICE address and shape of one of the trainer's arrays (IM_TRAINER_*; `layer` is
+ *                        ignored for OUT and STATUS).  *dtype: IM_DTYPE_F32 / IM_DTYPE_BF16 / IM_DTYPE_U32.  The
+ *                        arrays stay owned by the trainer; a caller may read them, and may write the input rows.
+ *   im_trainer_set_step_count  sets the Adam step counter (bias correction) -- 0 restarts the optimiser.
+ *   im_trainer_dw_slices the number of row slices the dW product of a layer with Np x Kp (padded) weights takes
+ *                        on M rows: the power of two that minimises a small time model (waves of output tiles on
+ *                        the SMs x rows per slice, plus the pass that adds the partial products).  Host only. */
+typedef struct im_trainer im_trainer;
+#define IM_TRAINER_W        0   /* float [dims[l+1]][dims[l]]                      */
+#define IM_TRAINER_B        1   /* float [dims[l+1]] (buffer padded to 64 floats)   */
+#define IM_TRAINER_W_BF16   2   /* bf16 [Np][Kp], zero padded                       */
+#define IM_TRAINER_WT_BF16  3   /* bf16 [Kp][Np], its transpose                     */
+#define IM_TRAINER_M_W      4
+#define IM_TRAINER_V_W      5
+#define IM_TRAINER_M_B      6
+#define IM_TRAINER_V_B      7
+#define IM_TRAINER_DW       8
+#define IM_TRAINER_DB       9
+#define IM_TRAINER_H       10   /* bf16 [max_rows][Kp]: input of layer l (layer 0: the observations) */
+#define IM_TRAINER_OUT     11   /* float [max_rows][dims[last]]                     */
+#define IM_TRAINER_STATUS  12   /* uint32 [1]: sticky device status word            */
+#define IM_DTYPE_F32  0
+#define IM_DTYPE_BF16 1
+#define IM_DTYPE_U32  2
+im_status im_trainer_create(int32_t n_layers, const int32_t *dims, const float *const *W, const float *const *b,
+                            int32_t max_rows, void *cuda_stream, im_trainer **out);
+void im_trainer_destroy(im_trainer *tr);
+im_status im_trainer_forward(im_trainer *tr, int32_t M);
+im_status im_trainer_backward(im_trainer *tr, const float *d_out, int32_t M);
+im_status im_trainer_step(im_trainer *tr, const im_adam_config *adam, const float *lr, const float *grad_scale);
+im_status im_trainer_push_to_policy(im_trainer *tr, im_policy *p);
+im_status im_trainer_tensor(im_trainer *tr, int32_t which, int32_t layer, void **ptr, int64_t *rows, int64_t *cols,
+                            int64_t *ld, int32_t *dtype);
+im_status im_trainer_set_step_count(im_trainer *tr, int32_t t);
+int32_t im_trainer_dw_slices(int32_t Np, int32_t Kp, int64_t M, int32_t max_split, int32_t any_rows);
+
+/* im_ppo_updater: one actor, one critic (a trainer with a single output) and the learnable per-dimension
+ * log-std, sharing a stream and max_rows.  log_std: HOST float [A], the initial value (also the first
+ * "old" log-std).
+ *   im_ppo_update  one minibatch update on M rows (a multiple of 64): forward of both nets on their input
+ *     rows, advantage moments (if normalize_advantage), im_ppo_loss, both backward passes, im_grad_scale
+ *     over every gradient tensor (global-norm clip at max_grad_norm), Adam on every tensor and on the
+ *     log-std, im_adaptive_lr from the mean KL.  The minibatch's observations must already sit in both
+ *     trainers' input rows.  mb: DEVICE float arrays -- action, mean_old [M][A]; logp_old, advantage,
+ *     value_old (needed with clip_value_loss), returns [M]; log_std_old [A] or NULL for the updater's own copy.
+ *   im_ppo_update_rollout  the whole update phase over a collected rollout: `epochs` passes over
+ *     `n_minibatches` blocks of the T * N samples (row t * N + e of the time-major arrays of `view`;
+ *     T * N / n_minibatches must be a multiple of 64 within max_rows).  perm NULL: contiguous blocks, the
+ *     observations converted into both nets' input rows by im_f32_to_bf16_padded, everything else read in
+ *     place.  perm: DEVICE int32 [epochs][T * N], a permutation of the sample indices per epoch: every array
+ *     of a block is gathered by im_gather_rows_f32 (the first shuffled call of a given size allocates the
+ *     gather buffers; make it outside a capture).
+ *   im_ppo_updater_tensor  DEVICE address of a state array (IM_PPO_*): the log-std and its Adam moments [A],
+ *     the frozen behaviour log-std [A], the learning rate [1], (clip factor, gradient norm) [2], the loss
+ *     summary of the last minibatch [6] as im_ppo_loss writes it. */
+typedef struct im_ppo_updater im_ppo_updater;
+typedef struct {
+    float lr;                     /* initial learning rate; adapted between lr_min and lr_max            */
+    float clip, value_coef, entropy_coef;
+    int32_t clip_value_loss;
+    float max_grad_norm;
+    float kl_target, lr_min, lr_max;
+    int32_t normalize_advantage;
+    im_adam_config adam;
+} im_ppo_update_config;
+typedef struct {
+    const float *action, *mean_old, *log_std_old, *logp_old, *advantage, *value_old, *returns;
+} im_ppo_minibatch;
+typedef struct {
+    int32_t T, N, A, ld_obs;
+    const float *obs;             /* [T * N][ld_obs]                                                      */
+    const float *action, *mean;   /* [T * N][A]: the behaviour policy's actions and means                 */
+    const float *logp, *advantage, *returns, *value;   /* [T * N]                                          */
+} im_rollout_view;
+#define IM_PPO_LOG_STD      0
+#define IM_PPO_LOG_STD_OLD  1
+#define IM_PPO_M_LOG_STD    2
+#define IM_PPO_V_LOG_STD    3
+#define IM_PPO_LR           4
+#define IM_PPO_GRAD_SCALE   5
+#define IM_PPO_SUMMARY      6
+im_status im_ppo_updater_create(im_trainer *actor, im_trainer *critic, const float *log_std,
+                                const im_ppo_update_config *cfg, im_ppo_updater **out);
+void im_ppo_updater_destroy(im_ppo_updater *u);
+im_status im_ppo_update(im_ppo_updater *u, int32_t M, const im_ppo_minibatch *mb);
+im_status im_ppo_update_rollout(im_ppo_updater *u, const im_rollout_view *view, int32_t epochs, int32_t n_minibatches,
+                                const int32_t *perm);
+im_status im_ppo_updater_tensor(im_ppo_updater *u, int32_t which, float **ptr, int64_t *n);
+im_status im_ppo_updater_set_step_count(im_ppo_updater *u, int32_t t);
 
 /* ---- whole step from host buffers ------------------------------------------
  * Convenience for callers whose simulator lives in host memory: copies one

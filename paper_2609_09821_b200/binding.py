@@ -27,8 +27,12 @@ EXPORTS = [
     "im_value_forward", "im_value_forward_staged", "im_gae", "im_env_set_reset_bins", "im_env_get_reset_stats",
     "im_env_step_aos", "im_policy_set_log_std", "im_ppo_workspace_bytes", "im_moments", "im_ppo_loss",
     "im_adam_step", "im_grad_scale", "im_adaptive_lr", "im_policy_layer_buffers",
-    "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_relu_mask_bf16", "im_f32_to_bf16_padded",
-    "im_colsum_f32", "im_colsum_bf16", "im_bf16_to_f32", "im_gemm_bf16_batched", "im_sum_slices_bf16_to_f32",
+    "im_gemm_bf16", "im_gemm_bf16_f32out", "im_transpose_bf16", "im_f32_to_bf16_padded",
+    "im_colsum_f32", "im_sum_slices_bf16_to_f32",
+    "im_trainer_create", "im_trainer_destroy", "im_trainer_forward", "im_trainer_backward", "im_trainer_step",
+    "im_trainer_push_to_policy", "im_trainer_tensor", "im_trainer_set_step_count", "im_trainer_dw_slices",
+    "im_ppo_updater_create", "im_ppo_updater_destroy", "im_ppo_update", "im_ppo_update_rollout", "im_ppo_updater_tensor",
+    "im_ppo_updater_set_step_count",
     "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math",
 ]
 
@@ -73,6 +77,21 @@ class PpoBatch(C.Structure):
 
 class AdamConfig(C.Structure):
     _fields_ = [("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+class PpoUpdateConfig(C.Structure):
+    _fields_ = [("lr", C.c_float), ("clip", C.c_float), ("value_coef", C.c_float), ("entropy_coef", C.c_float),
+                ("clip_value_loss", C.c_int32), ("max_grad_norm", C.c_float), ("kl_target", C.c_float),
+                ("lr_min", C.c_float), ("lr_max", C.c_float), ("normalize_advantage", C.c_int32), ("adam", AdamConfig)]
+
+
+class PpoMinibatch(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("action", "mean_old", "log_std_old", "logp_old", "advantage", "value_old", "returns")]
+
+
+class RolloutView(C.Structure):
+    _fields_ = [("T", C.c_int32), ("N", C.c_int32), ("A", C.c_int32), ("ld_obs", C.c_int32)] + \
+               [(n, C.c_void_p) for n in ("obs", "action", "mean", "logp", "advantage", "returns", "value")]
 
 
 class PolicyConfig(C.Structure):
@@ -134,22 +153,36 @@ def load():
         L.im_policy_layer_buffers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i32), C.POINTER(vp)]
         i64 = C.c_int64
         L.im_gemm_bf16.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i32, vp, vp]
-        L.im_gemm_bf16_batched.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp, i32, vp, vp]
-        L.im_gemm_bf16_tn.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.im_gemm_bf16_tn.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp]
         L.im_sum_slices_bf16_to_f32.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp]
         L.im_gemm_bf16_f32out.argtypes = [vp, i64, vp, i64, vp, i32, i32, i32, vp, vp, vp]
         L.im_transpose_bf16.argtypes = [vp, i64, i32, i32, vp, i64, vp]
-        L.im_relu_mask_bf16.argtypes = [vp, i64, vp, i64, i32, i32, vp]
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
         L.im_env_adapt_reset_bins.argtypes = [vp, C.c_float, i32]
         L.im_debug_math.argtypes = [i32, i32, vp, vp, vp]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
-        L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp, vp]
+        L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp]
+        L.im_trainer_create.argtypes = [i32, vp, vp, vp, i32, vp, C.POINTER(vp)]
+        L.im_trainer_destroy.argtypes = [vp]
+        L.im_trainer_destroy.restype = None
+        L.im_trainer_forward.argtypes = [vp, i32]
+        L.im_trainer_backward.argtypes = [vp, vp, i32]
+        L.im_trainer_step.argtypes = [vp, C.POINTER(AdamConfig), vp, vp]
+        L.im_trainer_push_to_policy.argtypes = [vp, vp]
+        L.im_trainer_tensor.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+        L.im_trainer_set_step_count.argtypes = [vp, i32]
+        L.im_trainer_dw_slices.argtypes = [i32, i32, i64, i32, i32]
+        L.im_trainer_dw_slices.restype = i32
+        L.im_ppo_updater_create.argtypes = [vp, vp, vp, C.POINTER(PpoUpdateConfig), C.POINTER(vp)]
+        L.im_ppo_updater_destroy.argtypes = [vp]
+        L.im_ppo_updater_destroy.restype = None
+        L.im_ppo_update.argtypes = [vp, i32, C.POINTER(PpoMinibatch)]
+        L.im_ppo_update_rollout.argtypes = [vp, C.POINTER(RolloutView), i32, i32, vp]
+        L.im_ppo_updater_tensor.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
+        L.im_ppo_updater_set_step_count.argtypes = [vp, i32]
         L.im_gather_rows_f32.argtypes = [vp, i64, vp, i64, i32, i32, vp, i32, i32, vp, vp]
         L.im_copy_f32.argtypes = [vp, vp, i64, vp]
-        L.im_bf16_to_f32.argtypes = [vp, i64, i32, i32, vp, vp]
         L.im_colsum_f32.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
-        L.im_colsum_bf16.argtypes = [vp, i64, i64, i32, vp, vp, C.c_size_t, vp]
         L.im_value_forward.argtypes = [vp, i32, vp, i32, vp]
         L.im_value_forward_staged.argtypes = [vp, vp, i32, vp]
         L.im_gae.argtypes = [C.POINTER(GaeConfig), i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
@@ -522,20 +555,12 @@ def gemm_bf16(A, B, Cout, bias, relu: bool, status, stream=None):
                                _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16")
 
 
-def gemm_bf16_batched(A, B, Cout, batches: int, bias, relu: bool, status, stream=None):
-    """`batches` stacked products: A [batches * M, K], B [batches * N, K] -> Cout [batches * M, N] (bf16)."""
-    M, K = A.shape[0] // batches, A.shape[1]
-    N = B.shape[0] // batches
-    _check(load().im_gemm_bf16_batched(_ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(Cout), Cout.stride(0), batches,
-                                       M, N, K, _ptr(bias), int(relu), _ptr(status), _st(stream)), "im_gemm_bf16_batched")
-
-
-def gemm_bf16_tn(A, Bm, Cout, slices: int, c_pitch: int, zeros, status, stream=None):
+def gemm_bf16_tn(A, Bm, Cout, slices: int, c_pitch: int, status, stream=None):
     """Cout (bf16, [slices * c_pitch, No]): slice s holds A[rows of s].T @ Bm[rows of s]; A [R, Mo], Bm [R, No]."""
     R, Mo = A.shape
     No = Bm.shape[1]
     _check(load().im_gemm_bf16_tn(_ptr(A), A.stride(0), _ptr(Bm), Bm.stride(0), _ptr(Cout), Cout.stride(0), R, Mo, No,
-                                  slices, c_pitch, _ptr(zeros), _ptr(status), _st(stream)), "im_gemm_bf16_tn")
+                                  slices, c_pitch, _ptr(status), _st(stream)), "im_gemm_bf16_tn")
 
 
 def sum_slices_bf16_to_f32(x, slices: int, rows: int, cols: int, out, stream=None):
@@ -558,11 +583,6 @@ def transpose_bf16(x, out, stream=None):
            "im_transpose_bf16")
 
 
-def relu_mask_bf16(dH, H, stream=None):
-    _check(load().im_relu_mask_bf16(_ptr(dH), dH.stride(0), _ptr(H), H.stride(0), dH.shape[0], dH.shape[1], _st(stream)),
-           "im_relu_mask_bf16")
-
-
 def f32_to_bf16_padded(x, out, stream=None):
     _check(load().im_f32_to_bf16_padded(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), out.stride(0),
                                         _st(stream)), "im_f32_to_bf16_padded")
@@ -574,7 +594,7 @@ def f32_to_bf16_padded_ptr(x, out_ptr: int, ld_out: int, stream=None):
                                         _st(stream)), "im_f32_to_bf16_padded")
 
 
-def gemm_bf16_dgrad(dZ, Wt, dH, H, colsum_partial, zeros, status, stream=None):
+def gemm_bf16_dgrad(dZ, Wt, dH, H, colsum_partial, status, stream=None):
     """dH [M, N] = (H > 0) * (dZ [M, K] @ Wt [N, K]^T) as bf16, and the fp32 column sums of dH per 32-row block into
     colsum_partial [M / 32, >= N] float32.  H and colsum_partial may be None."""
     M, K = dZ.shape
@@ -582,7 +602,7 @@ def gemm_bf16_dgrad(dZ, Wt, dH, H, colsum_partial, zeros, status, stream=None):
     _check(load().im_gemm_bf16_dgrad(_ptr(dZ), dZ.stride(0), _ptr(Wt), Wt.stride(0), _ptr(dH), dH.stride(0), M, N, K,
                                      _ptr(H) if H is not None else None, H.stride(0) if H is not None else 0,
                                      _ptr(colsum_partial) if colsum_partial is not None else None,
-                                     colsum_partial.stride(0) if colsum_partial is not None else 0, _ptr(zeros), _ptr(status),
+                                     colsum_partial.stride(0) if colsum_partial is not None else 0, _ptr(status),
                                      _st(stream)), "im_gemm_bf16_dgrad")
 
 
@@ -601,16 +621,30 @@ def copy_f32_ptr(dst_ptr: int, src, stream=None):
     _check(load().im_copy_f32(C.c_void_p(dst_ptr), _ptr(src), src.numel(), _st(stream)), "im_copy_f32")
 
 
-def bf16_to_f32(x, out, stream=None):
-    """out (dense float32 [rows, cols]) = x (bf16 view [rows, cols])."""
-    _check(load().im_bf16_to_f32(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), _st(stream)), "im_bf16_to_f32")
-
-
 def colsum(x, out, workspace, stream=None):
+    """out[c] = sum over rows of the float32 matrix x."""
+    _check(load().im_colsum_f32(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _st(stream)), "im_colsum_f32")
+
+
+class _DeviceArray:
+    """A device array owned by a library handle, described the way torch.as_tensor understands."""
+
+    def __init__(self, ptr: int, shape, typestr: str, strides=None):
+        self.__cuda_array_interface__ = dict(shape=tuple(shape), typestr=typestr, data=(int(ptr), False), version=3,
+                                             strides=strides)
+
+
+def device_tensor(ptr: int, shape, dtype: str, row_stride: Optional[int] = None):
+    """torch view (no copy) of `shape` elements at device address ptr; dtype 'f32', 'bf16' or 'u32';
+    row_stride in elements for 2-D arrays whose rows are padded.  The owner of the memory must outlive the view."""
     import torch
-    fn = load().im_colsum_bf16 if x.dtype == torch.bfloat16 else load().im_colsum_f32
-    _check(fn(_ptr(x), x.stride(0), x.shape[0], x.shape[1], _ptr(out), _ptr(workspace),
-              workspace.numel() * workspace.element_size(), _st(stream)), "im_colsum")
+    typestr, esz = {"f32": ("<f4", 4), "bf16": ("<i2", 2), "u32": ("<i4", 4)}[dtype]
+    strides = None
+    if len(shape) == 2 and row_stride is not None and row_stride != shape[1]:
+        strides = (row_stride * esz, esz)
+    t = torch.as_tensor(_DeviceArray(ptr, shape, typestr, strides), device="cuda")
+    return t.view(torch.bfloat16) if dtype == "bf16" else t
 
 
 NOALLOC_MAX_BATCH = 1024

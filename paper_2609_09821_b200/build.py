@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 OUT_DIR = os.path.join(_HERE, "_build")
 LIB_PATH = os.path.join(OUT_DIR, "libim_b200.so")
-SOURCES = ["im_api.cu", "env_kernel.cu", "mlp_simt.cu", "mlp_tc.cu", "policy_noalloc.cu", "rollout.cu", "aos_adapter.cu", "ppo.cu", "optim.cu", "train.cu"]
+SOURCES = ["im_api.cu", "env_kernel.cu", "mlp_simt.cu", "mlp_tc.cu", "policy_noalloc.cu", "rollout.cu", "aos_adapter.cu", "ppo.cu", "optim.cu", "train.cu", "trainer.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

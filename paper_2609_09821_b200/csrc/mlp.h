@@ -36,7 +36,7 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
                   const float *bias, bool relu, uint32_t *status, cudaStream_t stream, int batches = 1,
                   const void *mask = nullptr, int64_t ld_mask = 0, float *colsum_partial = nullptr, int ld_partial = 0);
 im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int R, int Mo, int No,
-                     int slices, int c_pitch, const float *bias, uint32_t *status, cudaStream_t stream);
+                     int slices, int c_pitch, uint32_t *status, cudaStream_t stream);
 im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, int M, int N, int K, const float *bias,
                        float *mean_out, uint32_t *status, cudaStream_t stream);
 }  // namespace im

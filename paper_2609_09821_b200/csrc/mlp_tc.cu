@@ -1461,7 +1461,7 @@ im_status tc_gemm(const void *A, int64_t lda, const void *B, int64_t ldb, void *
 // results stacked with a pitch of `c_pitch` rows.  Operands are read M/N-major, so no transposed copy
 // of either matrix is needed.
 im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, void *C, int64_t ldc, int R, int Mo, int No,
-                     int slices, int c_pitch, const float *bias, uint32_t *status, cudaStream_t stream)
+                     int slices, int c_pitch, uint32_t *status, cudaStream_t stream)
 {
     const int n_sm = device_sm_count();          // 0 unless the current device is an sm_100 part
     if (n_sm <= 0 || !encode_tiled_fn()) return IM_ERR_UNSUPPORTED;
@@ -1480,7 +1480,6 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
     GemmParams gp;
     std::memset(&gp, 0, sizeof(gp));
     gp.M = Mo; gp.N = No; gp.K_blocks = (R / slices) / BLOCK_K; gp.n_tiles_n = L.n_tiles_n; gp.bias = nullptr;    // no bias in this product
-    (void)bias;
     gp.act_floor = -INFINITY;
     gp.n_batches = slices; gp.a_batch_rows = R / slices; gp.b_batch_rows = 0; gp.c_batch_rows = c_pitch;
     gp.status = status;

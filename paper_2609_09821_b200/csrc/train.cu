@@ -80,30 +80,6 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
     }
 }
 
-// dH <- dH where H > 0, else 0 (eight bf16 per thread; ld and cols multiples of 8).
-__global__ void __launch_bounds__(256) relu_mask_kernel(__nv_bfloat16 *__restrict__ dH, const __nv_bfloat16 *__restrict__ H,
-                                                        long long ld_d, long long ld_h, int rows, int cols)
-{
-    const int chunks = cols >> 3;
-    const long long total = (long long)rows * chunks;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long r = i / chunks;
-        const int c = (int)(i - r * chunks) << 3;
-        uint4 d = *reinterpret_cast<const uint4 *>(dH + r * ld_d + c);
-        const uint4 h = __ldg(reinterpret_cast<const uint4 *>(H + r * ld_h + c));
-        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
-        uint32_t dw[4] = {d.x, d.y, d.z, d.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            // a bf16 is positive when its sign bit is clear and it is not zero
-            const uint32_t lo = hw[k] & 0xffffu, hi = hw[k] >> 16;
-            const bool plo = lo != 0u && !(lo & 0x8000u), phi = hi != 0u && !(hi & 0x8000u);
-            dw[k] = (plo ? dw[k] & 0x0000ffffu : 0u) | (phi ? dw[k] & 0xffff0000u : 0u);
-        }
-        *reinterpret_cast<uint4 *>(dH + r * ld_d + c) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
-    }
-}
-
 // out[r][c] = bf16(in[r][c]) for c < cols, 0 for cols <= c < ld_out.
 __global__ void __launch_bounds__(256) to_bf16_padded_kernel(const float *__restrict__ in, long long ld_in, int rows, int cols,
                                                              __nv_bfloat16 *__restrict__ out, int ld_out)
@@ -139,18 +115,6 @@ __global__ void __launch_bounds__(256) to_bf16_padded_vec_kernel(const float *__
         h = __floats2bfloat162_rn(v[4], v[5]); o.z = *reinterpret_cast<const uint32_t *>(&h);
         h = __floats2bfloat162_rn(v[6], v[7]); o.w = *reinterpret_cast<const uint32_t *>(&h);
         *reinterpret_cast<uint4 *>(out + r * ld_out + c) = o;
-    }
-}
-
-// out[r][c] (float, dense [rows][cols]) = in[r][c] (bf16, row stride ld_in).
-__global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *__restrict__ in, long long ld_in, int rows,
-                                                          int cols, float *__restrict__ out)
-{
-    const long long total = (long long)rows * cols;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long r = i / cols;
-        const int c = (int)(i - r * cols);
-        out[i] = __bfloat162float(in[r * ld_in + c]);
     }
 }
 
@@ -203,8 +167,6 @@ template <typename T>
 __device__ __forceinline__ float ld_as_float(const T *p);
 template <>
 __device__ __forceinline__ float ld_as_float<float>(const float *p) { return __ldg(p); }
-template <>
-__device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
 
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict__ x, long long ld, long long rows, int cols,
@@ -231,7 +193,7 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict
         partial[(long long)blockIdx.y * cols + c] = ((s_part[0][cx] + s_part[1][cx]) + s_part[2][cx]) + s_part[3][cx];
 }
 
-// The same for matrices that allow 16-byte row accesses: a thread owns 8 (bf16) or 4 (float) adjacent
+// The same for matrices that allow 16-byte row accesses: a thread owns 4 adjacent
 // columns and adds every eighth row of the slice; a CTA covers 32 such column groups and 8 row groups.
 template <typename T>
 struct VecOf;
@@ -242,20 +204,6 @@ struct VecOf<float> {
     {
         const float4 x = __ldg(reinterpret_cast<const float4 *>(p));
         v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-    }
-};
-template <>
-struct VecOf<__nv_bfloat16> {
-    static constexpr int kN = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&v)[8])
-    {
-        const uint4 x = __ldg(reinterpret_cast<const uint4 *>(p));
-        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            v[2 * k] = __uint_as_float(w[k] << 16);
-            v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
-        }
     }
 };
 
@@ -357,42 +305,29 @@ im_status im_gemm_bf16(const uint16_t *A, int64_t lda, const uint16_t *B, int64_
 
 im_status im_gemm_bf16_dgrad(const uint16_t *dZ, int64_t ld_dz, const uint16_t *Wt, int64_t ld_wt, uint16_t *dH, int64_t ld_dh,
                              int32_t M, int32_t N, int32_t K, const uint16_t *H, int64_t ld_h, float *colsum_partial,
-                             int32_t ld_partial, const float *zeros, uint32_t *status, void *cuda_stream)
+                             int32_t ld_partial, uint32_t *status, void *cuda_stream)
 {
     using namespace im;
-    if (!dZ || !Wt || !dH || !zeros || !status || M < 32 || (M & 31) || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
+    if (!dZ || !Wt || !dH || !status || M < 32 || (M & 31) || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
     if ((N & 63) || (K & 63) || ld_dz < K || ld_wt < K || ld_dh < N || (ld_dz & 7) || (ld_wt & 7) || (ld_dh & 7)) return IM_ERR_INVALID_ARG;
-    if (!al16(dZ) || !al16(Wt) || !al16(dH) || !al16(zeros)) return IM_ERR_INVALID_ARG;
+    if (!al16(dZ) || !al16(Wt) || !al16(dH)) return IM_ERR_INVALID_ARG;
     if (H && (ld_h < N || (ld_h & 7) || !al16(H))) return IM_ERR_INVALID_ARG;
     if (colsum_partial && (ld_partial < N || (ld_partial & 1) || (reinterpret_cast<uintptr_t>(colsum_partial) & 7u))) return IM_ERR_INVALID_ARG;
-    return tc_gemm(dZ, ld_dz, Wt, ld_wt, dH, ld_dh, M, N, K, zeros, false, status, (cudaStream_t)cuda_stream, 1, H, ld_h,
+    return tc_gemm(dZ, ld_dz, Wt, ld_wt, dH, ld_dh, M, N, K, nullptr, false, status, (cudaStream_t)cuda_stream, 1, H, ld_h,
                    colsum_partial, ld_partial);
 }
 
-im_status im_gemm_bf16_batched(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
-                               int32_t batches, int32_t M, int32_t N, int32_t K, const float *bias, int32_t relu,
-                               uint32_t *status, void *cuda_stream)
-{
-    using namespace im;
-    if (!A || !B || !C || !bias || !status || batches < 1 || M < 1 || N < 64 || K < 64) return IM_ERR_INVALID_ARG;
-    if ((N & 63) || (K & 63) || lda < K || ldb < K || ldc < N || (lda & 7) || (ldb & 7) || (ldc & 7)) return IM_ERR_INVALID_ARG;
-    if (batches > 1 && (M & 127)) return IM_ERR_INVALID_ARG;          // 128-row tiles must not straddle two batches
-    if ((int64_t)batches * M > 0x7fffffff || (int64_t)batches * N > 0x7fffffff) return IM_ERR_INVALID_ARG;
-    if (!al16(A) || !al16(B) || !al16(C) || !al16(bias)) return IM_ERR_INVALID_ARG;
-    return tc_gemm(A, lda, B, ldb, C, ldc, M, N, K, bias, relu != 0, status, (cudaStream_t)cuda_stream, batches);
-}
-
 im_status im_gemm_bf16_tn(const uint16_t *A, int64_t lda, const uint16_t *B, int64_t ldb, uint16_t *C, int64_t ldc,
-                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, const float *zeros,
-                          uint32_t *status, void *cuda_stream)
+                          int32_t R, int32_t Mo, int32_t No, int32_t slices, int32_t c_pitch, uint32_t *status,
+                          void *cuda_stream)
 {
     using namespace im;
-    if (!A || !B || !C || !zeros || !status || R < 64 || Mo < 1 || No < 64 || slices < 1) return IM_ERR_INVALID_ARG;
+    if (!A || !B || !C || !status || R < 64 || Mo < 1 || No < 64 || slices < 1) return IM_ERR_INVALID_ARG;
     if ((No & 63) || R % (64 * slices) || lda < Mo || ldb < No || ldc < No || (lda & 7) || (ldb & 7) || (ldc & 7))
         return IM_ERR_INVALID_ARG;
     if (c_pitch < Mo || (c_pitch & 127)) return IM_ERR_INVALID_ARG;
-    if (!al16(A) || !al16(B) || !al16(C) || !al16(zeros)) return IM_ERR_INVALID_ARG;
-    return tc_gemm_tn(A, lda, B, ldb, C, ldc, R, Mo, No, slices, c_pitch, zeros, status, (cudaStream_t)cuda_stream);
+    if (!al16(A) || !al16(B) || !al16(C)) return IM_ERR_INVALID_ARG;
+    return tc_gemm_tn(A, lda, B, ldb, C, ldc, R, Mo, No, slices, c_pitch, status, (cudaStream_t)cuda_stream);
 }
 
 im_status im_sum_slices_bf16_to_f32(const uint16_t *in, int64_t slice_stride, int64_t ld_in, int32_t slices, int32_t rows,
@@ -431,22 +366,6 @@ im_status im_transpose_bf16(const uint16_t *in, int64_t ld_in, int32_t rows, int
     __nv_bfloat16 *po = reinterpret_cast<__nv_bfloat16 *>(out);
     if (vec) transpose_bf16_kernel<true><<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(pi, ld_in, rows, cols, po, ld_out);
     else transpose_bf16_kernel<false><<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(pi, ld_in, rows, cols, po, ld_out);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
-}
-
-im_status im_relu_mask_bf16(uint16_t *dH, int64_t ld_d, const uint16_t *H, int64_t ld_h, int32_t rows, int32_t cols,
-                            void *cuda_stream)
-{
-    using namespace im;
-    if (!dH || !H || rows < 1 || cols < 8 || (cols & 7) || (ld_d & 7) || (ld_h & 7) || ld_d < cols || ld_h < cols ||
-        !al16(dH) || !al16(H))
-        return IM_ERR_INVALID_ARG;
-    const long long total = (long long)rows * (cols >> 3);
-    long long g = (total + 255) / 256;
-    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
-    relu_mask_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<__nv_bfloat16 *>(dH),
-                                                                  reinterpret_cast<const __nv_bfloat16 *>(H), ld_d, ld_h, rows, cols);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
@@ -492,30 +411,10 @@ im_status im_copy_f32(float *dst, const float *src, int64_t n, void *cuda_stream
                ? IM_OK : IM_ERR_CUDA;
 }
 
-im_status im_bf16_to_f32(const uint16_t *in, int64_t ld_in, int32_t rows, int32_t cols, float *out, void *cuda_stream)
-{
-    using namespace im;
-    if (!in || !out || rows < 1 || cols < 1 || ld_in < cols) return IM_ERR_INVALID_ARG;
-    const long long total = (long long)rows * cols;
-    long long g = (total + 255) / 256;
-    const int grid = (int)(g > 148 * 16 ? 148 * 16 : g);
-    bf16_to_f32_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(reinterpret_cast<const __nv_bfloat16 *>(in), ld_in, rows,
-                                                                    cols, out);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
-}
-
 im_status im_colsum_f32(const float *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
                         size_t workspace_bytes, void *cuda_stream)
 {
     return im::colsum<float>(x, ld, rows, cols, out, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
-}
-
-im_status im_colsum_bf16(const uint16_t *x, int64_t ld, int64_t rows, int32_t cols, float *out, void *workspace,
-                         size_t workspace_bytes, void *cuda_stream)
-{
-    return im::colsum<__nv_bfloat16>(reinterpret_cast<const __nv_bfloat16 *>(x), ld, rows, cols, out, workspace,
-                                     workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
 }  // extern "C"

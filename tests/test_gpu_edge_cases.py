@@ -406,3 +406,45 @@ def test_skeletons_with_more_than_eight_leaves(tree, options):
     h = p.rollout(steps=4)
     if options != "plain":
         assert any((x["flags"] != 0).any() for x in h)
+
+
+def test_handles_created_from_two_threads_at_once():
+    """The one-time kernel set-up (shared-memory opt-in per device) is guarded: two host threads that create their
+    first handles of every kind at the same moment both get working ones."""
+    import threading
+    from paper_2609_09821_b200 import trainer as T
+    sc = _scene("edge_threads", (361, 128, 28), "bf16")
+    barrier = threading.Barrier(2)
+    results, errors = [None, None], []
+
+    def work(i):
+        try:
+            stream = torch.cuda.Stream()
+            barrier.wait()
+            with torch.cuda.stream(stream):
+                env = B.Env(sc.g_skel, sc.g_clips, B.make_env_config(96, sc.wl.dt, 7, W.REWARD_MULT, 0.3, 384), stream=stream)
+                pol = B.Policy(sc.pol["dims"], sc.pol["W_bf16"], sc.pol["b"], "bf16", 0.1, 7, 96, stream=stream)
+                tr = T.MlpTrainer(sc.pol["dims"], sc.pol["W"], sc.pol["b"], 128, stream=stream)
+                obs = env.new_obs()
+                env.reset_all(obs, 0)
+                mean, act = torch.empty((96, 28), device="cuda"), torch.empty((96, 28), device="cuda")
+                pol.forward(1, obs, mean, act)
+                rows = tr.input_rows(128)
+                rows.zero_()
+                rows[:96, :361] = obs[:, :361].to(torch.bfloat16)
+                out = tr.forward(128)[:96].clone()
+                stream.synchronize()
+                assert env.device_status() == 0 and pol.device_status() == 0 and tr.device_status() == 0
+                results[i] = (obs.clone(), mean.clone(), out)
+        except Exception as e:                                   # surfaced in the main thread below
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for a, b in zip(*results):
+        assert torch.equal(a, b)                                 # same seeds, same results from both threads
+    assert torch.equal(results[0][1], results[0][2])             # and the trainer's forward is the policy's

@@ -32,12 +32,6 @@ def test_building_blocks_against_plain_definitions():
     out = torch.zeros((200, 304), dtype=torch.bfloat16, device="cuda")
     B.transpose_bf16(x, out[:, :300])
     assert torch.equal(out[:, :300], x.t())
-    h = torch.randn((128, 64), device="cuda", generator=g).to(torch.bfloat16)
-    h[0, :4] = torch.tensor([0.0, -0.0, 1e-30, -1e-30], device="cuda").to(torch.bfloat16)
-    d = torch.randn((128, 64), device="cuda", generator=g).to(torch.bfloat16)
-    want = torch.where(h > 0, d, torch.zeros_like(d))
-    B.relu_mask_bf16(d, h)
-    assert torch.equal(d, want)
     f = torch.randn((70, 69), device="cuda", generator=g)
     p = torch.full((70, 128), 7.0, dtype=torch.bfloat16, device="cuda")
     B.f32_to_bf16_padded(f, p)
@@ -49,16 +43,11 @@ def test_building_blocks_against_plain_definitions():
     pw = torch.full((3001, 640), 7.0, dtype=torch.bfloat16, device="cuda")
     B.f32_to_bf16_padded(wide, pw)
     assert torch.equal(pw[:, :577], wide.to(torch.bfloat16)) and (pw[:, 577:] == 0).all()
-    back = torch.empty((70, 69), device="cuda")
-    B.bf16_to_f32(p[:, :69], back)
-    assert torch.equal(back, f.to(torch.bfloat16).float())
     big = torch.randn((5000, 300), device="cuda", generator=g)
     ws = torch.empty(20 * 300, device="cuda")
     cs = torch.empty(300, device="cuda")
     B.colsum(big, cs, ws)
     np.testing.assert_allclose(cs.cpu().numpy(), big.double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
-    B.colsum(big.to(torch.bfloat16), cs, ws)
-    np.testing.assert_allclose(cs.cpu().numpy(), big.to(torch.bfloat16).double().sum(0).cpu().numpy(), rtol=1e-5, atol=1e-4)
     with pytest.raises(B.ImError):
         B.colsum(big, cs, ws[:300])                       # workspace too small for twenty slices
 
@@ -84,27 +73,6 @@ def test_generic_gemm_against_exact_products(M, N, K, relu):
     got = C_.float().cpu().numpy()
     assert np.abs(got - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3
     close(got, want, 1e-2, "gemm")
-
-
-def test_batched_gemm_and_slice_sum():
-    g = np.random.default_rng(5)
-    S, M, N, K = 3, 128, 192, 256
-    a = W.round_to_bf16(g.standard_normal((S * M, K)).astype(np.float32))[0]
-    b = W.round_to_bf16((g.standard_normal((S * N, K)) / 16).astype(np.float32))[0]
-    A_, B_ = torch.from_numpy(a).cuda().to(torch.bfloat16), torch.from_numpy(b).cuda().to(torch.bfloat16)
-    C_ = torch.zeros((S * M, N), dtype=torch.bfloat16, device="cuda")
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    B.gemm_bf16_batched(A_, B_, C_, S, torch.zeros(N, device="cuda"), False, status)
-    out = torch.empty((100, 150), device="cuda")
-    B.sum_slices_bf16_to_f32(C_, S, 100, 150, out)
-    torch.cuda.synchronize()
-    assert status.item() == 0
-    want = np.stack([a[s * M:(s + 1) * M].astype(np.float64) @ b[s * N:(s + 1) * N].astype(np.float64).T for s in range(S)])
-    got = C_.float().cpu().numpy().reshape(S, M, N)
-    assert np.abs(got - want).max() <= 2.0 ** -8 * np.abs(want).max() + 1e-3
-    np.testing.assert_allclose(out.cpu().numpy(), got[:, :100, :150].sum(0), rtol=1e-6, atol=1e-6)
-    with pytest.raises(B.ImError):
-        B.gemm_bf16_batched(A_[:S * 64], B_, C_, S, torch.zeros(N, device="cuda"), False, status)   # 64-row batches
 
 
 @pytest.mark.parametrize("dims,M", [((361, 128, 64, 28), 256), ((577, 256, 128, 69), 640), ((361, 64, 1), 128),
@@ -258,8 +226,8 @@ def test_whole_training_iteration_runs_from_one_cuda_graph():
             for tr, saved in zip((actor_t, critic_t), tr0):
                 for dst, src in zip(tr.W + tr.b + tr.mW + tr.vW + tr.mb + tr.vb + tr.Wb + tr.WbT, saved):
                     dst.copy_(src)
-                tr.t = 0
-            upd.t = 0
+                tr.set_step_count(0)
+            upd.set_step_count(0)
             upd.lr.fill_(5e-4); upd.log_std.fill_(-2.0); upd.m_ls.zero_(); upd.v_ls.zero_()
             actor_t.push_to_policy(actor); critic_t.push_to_policy(critic); actor.set_log_std(upd.log_std)
 
@@ -303,7 +271,7 @@ def test_transposed_product_reads_both_operands_in_place(R, Mo, No, slices):
     pitch = (Mo + 127) // 128 * 128
     C_ = torch.full((slices * pitch, No), 5.0, dtype=torch.bfloat16, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    B.gemm_bf16_tn(A_[:, :Mo], B_, C_, slices, pitch, torch.zeros(No, device="cuda"), status)
+    B.gemm_bf16_tn(A_[:, :Mo], B_, C_, slices, pitch, status)
     torch.cuda.synchronize()
     assert status.item() == 0
     Rs = R // slices
@@ -385,13 +353,12 @@ def test_dgrad_product_masks_and_sums_in_its_epilogue(M, N, K):
     wt = torch.randint(-2, 3, (N, K), generator=g).to(torch.bfloat16).cuda()
     h = torch.randint(-1, 3, (M, N), generator=g).clamp(min=0).to(torch.bfloat16).cuda()
     h[0, :] = 0; h[:, 1] = 0; h[3, 5] = -0.0
-    zeros = torch.zeros(N, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     want = (dz.float() @ wt.float().T) * (h > 0)
     for use_mask, use_sum in ((True, True), (True, False), (False, True)):
         out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
         part = torch.full((M // 32, N + 2), 7.0, device="cuda")
-        B.gemm_bf16_dgrad(dz, wt, out, h if use_mask else None, part if use_sum else None, zeros, status)
+        B.gemm_bf16_dgrad(dz, wt, out, h if use_mask else None, part if use_sum else None, status)
         ref = want if use_mask else dz.float() @ wt.float().T
         assert torch.equal(out.float(), ref.to(torch.bfloat16).float())
         if use_sum:
@@ -400,3 +367,81 @@ def test_dgrad_product_masks_and_sums_in_its_epilogue(M, N, K):
         else:
             assert (part == 7.0).all()
     assert int(status.item()) == 0
+
+
+def test_whole_ppo_update_through_the_raw_c_abi():
+    """One PPO minibatch update driven by lib.im_* calls alone (no Python wrapper classes in between): trainers
+    and updater created, input rows filled, im_ppo_update enqueued, gradients and the loss summary read back
+    through im_trainer_tensor / im_ppo_updater_tensor and compared with the pipeline assembled from oracle
+    functions, as test_ppo_update_matches_the_oracle_pipeline_and_improves_the_objective does through the wrappers."""
+    import ctypes as C
+    lib = B.load()
+    A, D, M = 28, 361, 256
+    adims, cdims = (D, 128, 64, A), (D, 128, 64, 1)
+    aw, cw = W.make_policy_weights(adims, "bf16", 31), W.make_policy_weights(cdims, "bf16", 32)
+    g = np.random.default_rng(33)
+    obs = g.standard_normal((M, D)).astype(np.float32)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def create(dims, w):
+        nl = len(dims) - 1
+        Wc = [np.ascontiguousarray(x, np.float32) for x in w["W"]]
+        bc = [np.ascontiguousarray(x, np.float32) for x in w["b"]]
+        Wp = (C.c_void_p * nl)(*[x.ctypes.data for x in Wc])
+        bp = (C.c_void_p * nl)(*[x.ctypes.data for x in bc])
+        d = np.asarray(dims, np.int32)
+        h = C.c_void_p()
+        assert lib.im_trainer_create(nl, d.ctypes.data, C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), M, stream, C.byref(h)) == 0
+        return h
+
+    def tensor(h, which, layer):
+        ptr, rows, cols, ld, dt = C.c_void_p(), C.c_int64(), C.c_int64(), C.c_int64(), C.c_int32()
+        assert lib.im_trainer_tensor(h, which, layer, C.byref(ptr), C.byref(rows), C.byref(cols), C.byref(ld), C.byref(dt)) == 0
+        vector = which in (1, 6, 7, 9, 12)
+        shape = (cols.value,) if vector else (rows.value, cols.value)
+        return B.device_tensor(ptr.value, shape, {0: "f32", 1: "bf16", 2: "u32"}[dt.value], None if vector else ld.value)
+
+    actor, critic = create(adims, aw), create(cdims, cw)
+    log_std0 = np.full(A, -1.0, np.float32)
+    cfg = B.PpoUpdateConfig(5e-4, 0.2, 2.0, 2.5e-4, 1, 1.0, 0.008, 1e-5, 1e-2, 1, B.AdamConfig(0.9, 0.999, 1e-8))
+    upd = C.c_void_p()
+    assert lib.im_ppo_updater_create(actor, critic, log_std0.ctypes.data, C.byref(cfg), C.byref(upd)) == 0
+    for h in (actor, critic):
+        rows = tensor(h, 10, 0)                                   # IM_TRAINER_H of layer 0: the input rows
+        rows.zero_()
+        rows[:M, :D] = torch.from_numpy(obs).cuda().to(torch.bfloat16)
+    mean_old = O.policy_forward(adims, aw["W"], aw["b"], 1.0, 0, 0, obs.astype(np.float64), bf16_operands=True)["mean"]
+    value_old = O.policy_forward(cdims, cw["W"], cw["b"], 1.0, 0, 0, obs.astype(np.float64), bf16_operands=True)["mean"][:, 0]
+    z = g.standard_normal((M, A))
+    batch_np = dict(action=(mean_old + np.exp(-1.0) * z).astype(np.float32), mean_old=mean_old.astype(np.float32),
+                    logp_old=(-0.5 * (z ** 2).sum(1) + A - 0.5 * A * np.log(2 * np.pi)).astype(np.float32),
+                    advantage=(g.standard_normal(M) * 2 + 0.5).astype(np.float32), value_old=value_old.astype(np.float32),
+                    returns=(value_old + g.standard_normal(M)).astype(np.float32))
+    dev = {k: torch.from_numpy(v).cuda() for k, v in batch_np.items()}
+    mb = B.PpoMinibatch(dev["action"].data_ptr(), dev["mean_old"].data_ptr(), None, dev["logp_old"].data_ptr(),
+                        dev["advantage"].data_ptr(), dev["value_old"].data_ptr(), dev["returns"].data_ptr())
+    assert lib.im_ppo_update(upd, M, C.byref(mb)) == 0
+    assert lib.im_ppo_update(upd, M + 1, C.byref(mb)) == -1                    # rows not a multiple of 64
+    torch.cuda.synchronize()
+    assert int(tensor(actor, 12, 0).item()) == 0 and int(tensor(critic, 12, 0).item()) == 0
+    am, ar = O.moments(batch_np["advantage"])
+    ob = dict(batch_np, mean=mean_old.astype(np.float32), log_std=log_std0, log_std_old=log_std0, value=value_old.astype(np.float32))
+    loss = O.ppo_loss(ob, 0.2, 2.0, 2.5e-4, True, am, ar)
+    ptr, n = C.c_void_p(), C.c_int64()
+    assert lib.im_ppo_updater_tensor(upd, 6, C.byref(ptr), C.byref(n)) == 0 and n.value == 6     # IM_PPO_SUMMARY
+    summary = B.device_tensor(ptr.value, (6,), "f32").cpu().numpy()
+    np.testing.assert_allclose(summary[:4], loss["summary"][:4], rtol=2e-2, atol=2e-3)
+    dWa, dba = O.mlp_backward(adims, aw["W"], aw["b"], obs.astype(np.float64), loss["d_mean"], bf16_operands=True)
+    dWc, dbc = O.mlp_backward(cdims, cw["W"], cw["b"], obs.astype(np.float64), loss["d_value"][:, None], bf16_operands=True)
+    for l in range(3):
+        close(tensor(actor, 8, l).cpu().numpy(), dWa[l], 5e-2, "actor dW[%d]" % l)                 # IM_TRAINER_DW
+        close(tensor(actor, 9, l).cpu().numpy(), dba[l], 5e-2, "actor db[%d]" % l)                 # IM_TRAINER_DB
+        close(tensor(critic, 8, l).cpu().numpy(), dWc[l], 5e-2, "critic dW[%d]" % l)
+    # the step moved the weights and the bf16 copies follow the fp32 masters
+    for l in range(3):
+        w, wb = tensor(actor, 0, l), tensor(actor, 2, l)
+        assert not torch.equal(w.cpu(), torch.from_numpy(np.ascontiguousarray(aw["W"][l], np.float32)))
+        assert torch.equal(wb[:adims[l + 1], :adims[l]], w.to(torch.bfloat16))
+    lib.im_ppo_updater_destroy(upd)
+    lib.im_trainer_destroy(actor)
+    lib.im_trainer_destroy(critic)
