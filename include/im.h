@@ -657,6 +657,14 @@ uint64_t im_launch_count(void);
  *   op = IM_DEBUG_ANGLE_SQ   in DEVICE [n][4] quaternions of any positive norm -> out DEVICE [n] angle^2
  *   op = IM_DEBUG_SLERP      in DEVICE [n][8] = q0 (w,x,y,z), h (3), alpha       -> out DEVICE [n][7] =
  *                            q0 exp(alpha h) (4) and 2 h (the joint velocity at 1 frame per second) */
+/* im_debug_set_wait: every wait inside the tensor-core GEMM kernels and the bulk-copy PPO loss kernel (on an
+ * mbarrier that a copy or an MMA completes) is bounded: when limit_ns (2 s by default) runs out the kernel sets
+ * IM_DEV_WAIT_TIMEOUT in the handle's status word (the PPO loss: a NaN summary), stops issuing, lets what is in
+ * flight land, frees its tensor memory and returns, so the context stays usable.  This call sets the limit for
+ * the current device and, with skip_loads != 0, makes the copy-issuing threads of the single-CTA GEMM kernels
+ * and of the PPO loss kernel issue nothing -- the only way to see a wait run out without a fault: nothing is in
+ * flight, the consumers give up after limit_ns.  For tests of the failure path; synchronises the device. */
+im_status im_debug_set_wait(uint64_t limit_ns, int32_t skip_loads);
 #define IM_DEBUG_ANGLE_SQ 0
 #define IM_DEBUG_SLERP    1
 im_status im_debug_math(int32_t op, int32_t n, const float *in, float *out, void *cuda_stream);

@@ -33,7 +33,7 @@ EXPORTS = [
     "im_trainer_push_to_policy", "im_trainer_tensor", "im_trainer_set_step_count", "im_trainer_dw_slices",
     "im_ppo_updater_create", "im_ppo_updater_destroy", "im_ppo_update", "im_ppo_update_rollout", "im_ppo_updater_tensor",
     "im_ppo_updater_set_step_count",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait",
 ]
 
 
@@ -160,6 +160,7 @@ def load():
         L.im_f32_to_bf16_padded.argtypes = [vp, i64, i32, i32, vp, i32, vp]
         L.im_env_adapt_reset_bins.argtypes = [vp, C.c_float, i32]
         L.im_debug_math.argtypes = [i32, i32, vp, vp, vp]
+        L.im_debug_set_wait.argtypes = [u64, i32]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp]
         L.im_trainer_create.argtypes = [i32, vp, vp, vp, i32, vp, C.POINTER(vp)]
@@ -650,6 +651,11 @@ def device_tensor(ptr: int, shape, dtype: str, row_stride: Optional[int] = None)
 NOALLOC_MAX_BATCH = 1024
 NOALLOC_MAX_WIDTH = 1024
 DEBUG_ANGLE_SQ, DEBUG_SLERP = 0, 1
+
+
+def debug_set_wait(limit_ns: int = 2_000_000_000, skip_loads: bool = False):
+    """Limit of the kernels' bounded waits on the current device; skip_loads makes the copy-issuing threads idle."""
+    _check(load().im_debug_set_wait(int(limit_ns), int(skip_loads)), "im_debug_set_wait")
 
 
 def debug_math(op: int, inp):

@@ -728,6 +728,15 @@ im_status im_step_host(im_env *e, im_policy *p, uint32_t step, const float *sim_
     return IM_OK;
 }
 
+im_status im_debug_set_wait(uint64_t limit_ns, int32_t skip_loads)
+{
+    if (limit_ns == 0) return IM_ERR_INVALID_ARG;
+    IM_CUDA(cudaDeviceSynchronize());                   // kernels in flight keep the setting they started with
+    IM_CUDA(tc_set_wait_debug(limit_ns, skip_loads != 0));
+    IM_CUDA(ppo_set_wait_debug(limit_ns, skip_loads != 0));
+    return IM_OK;
+}
+
 im_status im_debug_math(int32_t op, int32_t n, const float *in, float *out, void *cuda_stream)
 {
     if ((op != IM_DEBUG_ANGLE_SQ && op != IM_DEBUG_SLERP) || n < 1 || !in || !out) return IM_ERR_INVALID_ARG;

@@ -39,4 +39,7 @@ im_status tc_gemm_tn(const void *A, int64_t lda, const void *B, int64_t ldb, voi
                      int slices, int c_pitch, uint32_t *status, cudaStream_t stream);
 im_status tc_gemm_head(const void *A, int64_t lda, const void *B, int64_t ldb, int M, int N, int K, const float *bias,
                        float *mean_out, uint32_t *status, cudaStream_t stream);
+// bounded-wait diagnostics of the tensor-core GEMM kernels and of the bulk-copy PPO loss kernel (current device)
+cudaError_t tc_set_wait_debug(unsigned long long limit_ns, int skip_loads);
+cudaError_t ppo_set_wait_debug(unsigned long long limit_ns, int skip_loads);
 }  // namespace im

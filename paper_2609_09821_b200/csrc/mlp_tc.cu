@@ -34,7 +34,10 @@ constexpr int BLOCK_K = 64;               // 64 bf16 = 128 bytes = one swizzle r
 constexpr int UMMA_K = 16;
 constexpr int kThreads = 192;
 constexpr int kEpiWarps = 4;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+// Limit of every bounded wait below (2 s unless im_debug_set_wait changed it), and the diagnostic switch that makes the
+// TMA producers issue nothing, so that a test can watch a wait run out with no copy or MMA in flight.
+__device__ unsigned long long g_wait_limit_ns = 2000000000ull;
+__device__ int g_skip_loads = 0;
 
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -74,7 +77,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 255) == 255) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            if (global_ns() - t0 > g_wait_limit_ns) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -308,6 +311,7 @@ __device__ __forceinline__ void producer_role(const Pipe &p, const CUtensorMap *
     int stage = 0;
     uint32_t phase = 0;
     const int tiles_per_batch = n_tiles / P.n_batches;
+    if (g_skip_loads) return;                        // diagnostic: the consumers' first wait runs out
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int b = tile / tiles_per_batch, t = tile - b * tiles_per_batch;
         if (MN) {
@@ -1421,6 +1425,13 @@ im_status tc_policy_forward(im_policy *p, uint32_t step, int32_t n, const float 
     return IM_OK;
 }
 
+
+cudaError_t tc_set_wait_debug(unsigned long long limit_ns, int skip_loads)
+{
+    cudaError_t e = cudaMemcpyToSymbol(g_wait_limit_ns, &limit_ns, sizeof(limit_ns));
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_skip_loads, &skip_loads, sizeof(skip_loads));
+    return e;
+}
 
 // C[M][N] = act(A[M][K] B[N][K]^T + bias) on the hidden-layer kernels, operands anywhere in device
 // memory: the three tensor maps are encoded for this call and travel as kernel parameters.

@@ -276,7 +276,10 @@ __global__ void __launch_bounds__(32 * kWarps) ppo_loss_kernel(const PpoParams P
 // Warps per CTA: enough that a 32-row tile gives every warp two or more trips (8-lane groups: four
 // rows per warp and trip, so 4 warps; wider groups: 8 warps).
 __host__ __device__ constexpr int bulk_warps(int LPR) { return LPR == 8 ? 4 : 8; }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+// Limit of the bounded waits below (2 s unless im_debug_set_wait changed it) and the diagnostic switch that makes
+// the bulk-copy kernel fetch nothing, so that a test can watch a wait run out with no copy in flight.
+__device__ unsigned long long g_wait_limit_ns = 2000000000ull;
+__device__ int g_skip_loads = 0;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
@@ -309,7 +312,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 255) == 255) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            if (global_ns() - t0 > g_wait_limit_ns) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -359,6 +362,7 @@ __global__ void __launch_bounds__(32 * bulk_warps(LPR)) ppo_loss_bulk_kernel(con
 
     const bool with_vold = P.cfg.clip_value_loss != 0;
     auto fetch = [&](long long tile, int s) {               // thread 0 only
+        if (g_skip_loads) return;                           // diagnostic: the first wait runs out
         float *st = s_stage + (size_t)s * SF;
         const size_t r0 = (size_t)tile * kTileRows, e0 = r0 * (size_t)A;
         const uint32_t tile_bytes = (uint32_t)TA * 4u, col_bytes = (uint32_t)kTileRows * 4u;
@@ -493,6 +497,13 @@ __global__ void __launch_bounds__(32) moments_finish_kernel(const double *__rest
 }
 
 }  // namespace
+
+cudaError_t ppo_set_wait_debug(unsigned long long limit_ns, int skip_loads)
+{
+    cudaError_t e = cudaMemcpyToSymbol(g_wait_limit_ns, &limit_ns, sizeof(limit_ns));
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_skip_loads, &skip_loads, sizeof(skip_loads));
+    return e;
+}
 
 }  // namespace im
 
