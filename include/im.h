@@ -55,6 +55,7 @@ typedef int32_t im_status;
 #define IM_DEV_BAD_SIM_QUAT    1u   /* a simulated quaternion had zero or non-finite norm; identity used */
 #define IM_DEV_WAIT_TIMEOUT    2u   /* a bounded wait inside a kernel ran out; that tile's output is invalid */
 #define IM_DEV_BAD_STATE       4u   /* a per-env clip id was out of range; clamped */
+#define IM_DEV_DEBUG_CHECK     8u   /* bounds-checked build only: an index formed inside the env kernel was out of range */
 
 #define IM_MAX_BODIES   32
 #define IM_N_TERMS       7          /* pose, vel, ee_pos, ee_rot, com, body_pos, body_vel */
@@ -237,6 +238,21 @@ im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, co
  * row, else IM_ERR_INVALID_ARG; a policy attached for another width is detached.  Takes
  * effect with the next launch (host state only).  im_step_host does not support act_dim > 0. */
 im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim, const float *prev_action, int32_t ld_action);
+
+/* ---- training summaries kept on the device ------------------------------------
+ * (Section 4.2 of the paper: logging must not put a host read on the rollout step, so the summaries a
+ * trainer plots stay on the GPU and are read whenever convenient.)  With an accumulator attached every
+ * im_env_step adds, over its N envs:
+ *   acc[0] += sum of round(reward * 2^40)      (a fixed-point sum: exact, the same whatever order the
+ *                                               thread blocks finish in; divide by 2^40 and the step count)
+ *   acc[1] += envs flagged terminated          acc[2] += envs flagged truncated
+ *   acc[3] += sum over envs reset by this step of the length, in steps, of the episode that ended
+ * acc: DEVICE uint64 [4], owned by the caller (who zeroes it when a logging window starts and reads it
+ * stream-ordered, e.g. once per rollout); NULL detaches.  Host state only, takes effect with the next
+ * launch; the additions are integer atomics enqueued with the step (capturable).  im_env_reset_all does
+ * not touch the accumulator. */
+#define IM_SUMMARY_REWARD_SCALE 1099511627776.0    /* 2^40 */
+im_status im_env_set_summary(im_env *e, uint64_t *acc);
 
 /* ---- adaptive episode initialisation --------------------------------------
  * (The paper trains "with early termination and adaptive episode-initialization

@@ -14,7 +14,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "_build", "libim_b200.so")
+# IM_B200_LIB selects another build of the library (e.g. the bounds-checked libim_b200_debug.so)
+LIB_PATH = os.environ.get("IM_B200_LIB") or os.path.join(_HERE, "_build", "libim_b200.so")
 N_TERMS = 7
 MAX_LAYERS = 8
 
@@ -33,7 +34,7 @@ EXPORTS = [
     "im_trainer_push_to_policy", "im_trainer_tensor", "im_trainer_set_step_count", "im_trainer_dw_slices",
     "im_ppo_updater_create", "im_ppo_updater_destroy", "im_ppo_update", "im_ppo_update_rollout", "im_ppo_updater_tensor",
     "im_ppo_updater_set_step_count",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait", "im_env_set_summary",
 ]
 
 
@@ -161,6 +162,7 @@ def load():
         L.im_env_adapt_reset_bins.argtypes = [vp, C.c_float, i32]
         L.im_debug_math.argtypes = [i32, i32, vp, vp, vp]
         L.im_debug_set_wait.argtypes = [u64, i32]
+        L.im_env_set_summary.argtypes = [vp, vp]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp]
         L.im_trainer_create.argtypes = [i32, vp, vp, vp, i32, vp, C.POINTER(vp)]
@@ -355,6 +357,15 @@ class Env:
         self.n_future = int(n_future)
         self.D = 24 * self.J + 1 + (int(n_future) - 1) * 9 * self.skel.n_ee + A
         return self.D
+
+    def set_summary(self, acc=None):
+        """Attaches (None: detaches) a 4-element int64 CUDA tensor every later step adds to: fixed-point reward sum
+        (2^-40 units), terminated count, truncated count, summed lengths of the episodes that ended."""
+        import torch
+        if acc is not None and (acc.dtype != torch.int64 or acc.numel() != 4 or not acc.is_cuda or not acc.is_contiguous()):
+            raise ValueError("acc must be a contiguous int64 CUDA tensor of 4 elements")
+        _check(load().im_env_set_summary(self.h, _ptr(acc)), "im_env_set_summary")
+        self._summary = acc
 
     def reset_stats(self, clear: bool = False):
         """(starts, failures) per (clip, phase bin) as CUDA int32 tensors [C, n_bins] (uint32 counts)."""

@@ -32,6 +32,22 @@ __device__ __forceinline__ uint2 pack_bf16x4(float4 v)
 constexpr int kTile = 32;          // envs per CTA
 constexpr int kPartials = 9;       // pose, vel, ee_pos, ee_rot, body_pos, body_vel, weighted com difference (3)
 
+// The bounds-checked build (-DIM_DEBUG, a second library next to the regular one): every index the kernel forms
+// from its inputs -- keyframe row, body index of a link, body-state offset, staged observation column,
+// destination row -- is tested against its limit; an index out of range sets IM_DEV_DEBUG_CHECK in the env's
+// status word and is replaced by 0, so the launch always completes (no trap, no fault) and a test reads the word.
+#ifdef IM_DEBUG
+__device__ __forceinline__ uint32_t checked(uint32_t idx, uint32_t limit, uint32_t *status)
+{
+    if (idx < limit) return idx;
+    atomicOr(status, IM_DEV_DEBUG_CHECK);
+    return 0u;
+}
+#define IM_CHECKED(idx, limit) checked((uint32_t)(idx), (uint32_t)(limit), P.status)
+#else
+#define IM_CHECKED(idx, limit) (idx)
+#endif
+
 __host__ __device__ inline int tile_stride(int D)
 {
     int s4 = (D + 3) / 4;
@@ -206,6 +222,16 @@ __device__ __forceinline__ LinkRec ld_link(const float4 *links, int k)
     const int4 i = *reinterpret_cast<const int4 *>(links + 2 * k + 1);
     return {{a.x, a.y, a.z}, a.w, i.x, i.y};
 }
+#ifdef IM_DEBUG
+// (checked build: position within the chain and the body index it holds)
+#define ld_link(links, k) ld_link_checked(links, k, len, J, P.status)
+__device__ __forceinline__ LinkRec ld_link_checked(const float4 *links, int k, int len, int J, uint32_t *status)
+{
+    LinkRec L = (ld_link)(links, (int)checked((uint32_t)k, (uint32_t)len, status));
+    L.b = (int)checked((uint32_t)L.b, (uint32_t)J, status);
+    return L;
+}
+#endif
 
 // Compose the interpolated joint onto the running transform.  k == 0 is the root, whose position is the
 // lerp of the row's root position along its displacement.
@@ -382,7 +408,7 @@ __device__ __forceinline__ void copy_out(const EnvKernelParams &P, const float *
     const int e0 = blockIdx.x * kTile;
     quads = min(quads, last - first);             // the staged stride may be wider than what is left of the row
     for (int r = warp; r < rows; r += n_warps) {
-        const size_t row_off = (size_t)(e0 + r) * P.ld_obs + 4 * (first + lane);
+        const size_t row_off = (size_t)IM_CHECKED(e0 + r, P.N) * P.ld_obs + 4 * (first + lane);
         float4 *dst = F32 ? reinterpret_cast<float4 *>(P.obs + row_off) : nullptr;
         uint2 *dst16 = BF16 ? reinterpret_cast<uint2 *>(P.obs_bf16 + row_off) : nullptr;
         uint32_t src = src_lane + (uint32_t)(r * S) * 4u;
@@ -470,7 +496,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         int frame;
         float alpha;
         lookup(cm, t1, frame, alpha);
-        const float4 *r0 = P.frames + (size_t)frame * RS;
+        const float4 *r0 = P.frames + (size_t)IM_CHECKED(frame, P.n_rows) * RS;
         LinkRec L = ld_link(links, 0);
         KeyPair keys = ld_keys(r0, L.b);
 
@@ -497,6 +523,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             SimBody sim;
             if (own) {                                // issue the loads before the interpolation math
                 const uint32_t o3 = 3 * (uint32_t)b * st + e32;
+                (void)IM_CHECKED((4 * (uint32_t)b + 3) * st + e32, 4u * (uint32_t)J * st);
                 sim.q = ld_sim_quat(P.quat, 4 * (uint32_t)b * st + e32, st);
                 sim.p = ld_sim_vec(P.pos, o3, st);
                 sim.v = ld_sim_vec(P.lin, o3, st);
@@ -531,6 +558,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                 acc[6] = fmaf(Lc.mass_frac, dp.x, acc[6]);
                 acc[7] = fmaf(Lc.mass_frac, dp.y, acc[7]);
                 acc[8] = fmaf(Lc.mass_frac, dp.z, acc[8]);
+                (void)IM_CHECKED(15 * b + 14, c1);
                 body_obs(H, sim.q, sim.p, sim.v, sim.w, row1, b);
                 qa = sim.q;
                 wa = sim.w;
@@ -548,6 +576,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     int flags = 0;
     float t_cur = t1;
     int clip_cur = clip;
+    float reward_val = 0.0f;
     if (!RESET_ALL) {
         float r = 0.0f;
         const bool need_r = c == 0 || P.reward.r_min > -INFINITY;
@@ -587,6 +616,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
         const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
         flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
+        reward_val = r;
         if (c == 0 && valid) P.flags_out[env] = (uint8_t)flags;
     }
     const bool reset = RESET_ALL || flags != 0;
@@ -614,10 +644,27 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             t_cur = __fmul_rn(u, span);
         }
     }
-    if (c == 0 && valid) {
-        P.clip_id[env] = clip_cur;
-        P.t[env] = t_cur;
-        P.ep_len[env] = reset ? 0 : P.ep_len[env] + 1;
+    if (c == 0) {
+        int ep_done = 0;                    // steps of the episode this step ended (0 where none ended)
+        if (valid) {
+            const int len_now = P.ep_len[env] + 1;
+            P.clip_id[env] = clip_cur;
+            P.t[env] = t_cur;
+            P.ep_len[env] = reset ? 0 : len_now;
+            ep_done = reset ? len_now : 0;
+        }
+        if (OPT && !RESET_ALL && P.summary) {
+            // training summaries: integer sums over the tile (one warp), then one atomic per quantity
+            unsigned long long v[4] = {valid ? (unsigned long long)__float2ll_rn(reward_val * 1099511627776.0f) : 0ull,
+                                       (unsigned long long)(valid ? (flags & 1) : 0), (unsigned long long)(valid ? (flags >> 1) & 1 : 0),
+                                       (unsigned long long)ep_done};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
+                if (lane == 0 && v[i]) atomicAdd(P.summary + i, v[i]);
+            }
+        }
     }
     const ClipMeta cmc = reset ? P.meta[clip_cur] : cm;
 
@@ -627,7 +674,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         int frame;
         float alpha;
         lookup(cmc, t_cur, frame, alpha);
-        const float4 *r0 = P.frames + (size_t)frame * RS;
+        const float4 *r0 = P.frames + (size_t)IM_CHECKED(frame, P.n_rows) * RS;
         LinkRec L = ld_link(links, 0);
         KeyPair keys = ld_keys(r0, L.b);
         Walk s;
@@ -673,7 +720,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     int frame_t;
     float alpha_t;
     lookup(cmc, t_tgt, frame_t, alpha_t);
-    const float4 *rt0 = P.frames + (size_t)frame_t * RS;
+    const float4 *rt0 = P.frames + (size_t)IM_CHECKED(frame_t, P.n_rows) * RS;
     float phase = 0.0f;
     if (c == 0) {
         phase = t_cur / cmc.dur;
@@ -716,6 +763,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                 float o[9];
                 target_obs(H, s.q, s.p, o);
                 const int col = 15 * J + 1 + 9 * b;
+                (void)IM_CHECKED(col + 8 - c1, S2);
                 if (col >= c1) {
                     store_run<9>(row2, col - c1, o);
                 } else {                          // the root's block straddles the split
@@ -733,7 +781,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                 int frame_f;
                 float alpha_f;
                 lookup(cmc, t_f, frame_f, alpha_f);
-                const float4 *rf0 = P.frames + (size_t)frame_f * RS;
+                const float4 *rf0 = P.frames + (size_t)IM_CHECKED(frame_f, P.n_rows) * RS;
                 Walk sf;
                 for (int k = 0; k < len; ++k) {
                     const LinkRec Lf = ld_link(links, k);
@@ -854,7 +902,8 @@ cudaError_t launch_debug_math(int op, int n, const float *in, float *out, cudaSt
 cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t smem, cudaStream_t stream)
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
-    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0 || p.n_future > 1 || p.act_dim > 0;
+    const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0 || p.n_future > 1 || p.act_dim > 0 ||
+                     p.summary != nullptr;
     if (opt) {
         if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
         else launch_one<false, true>(p, grid, block, smem, stream);

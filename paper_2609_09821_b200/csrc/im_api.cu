@@ -269,6 +269,7 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.links = e->d_links;
     p.meta = e->clips->d_meta;
     p.C = e->clips->C;
+    p.n_rows = (int32_t)e->clips->rows;
     p.N = e->cfg.n_envs;
     p.env_id_base = e->cfg.env_id_base;
     p.dt = e->cfg.dt;
@@ -287,6 +288,7 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.act_dim = e->act_dim;
     p.prev_action = e->prev_action;
     p.ld_action = e->ld_action;
+    p.summary = e->d_summary;
     p.step = step;
     p.clip_id = e->d_clip_id;
     p.t = e->d_t;
@@ -553,6 +555,13 @@ im_status im_env_set_obs_extension(im_env *e, int32_t n_future, int32_t act_dim,
     if (D != e->D) e->d_obs_bf16 = nullptr;            // a policy attached for another width no longer fits
     e->D = D;
     e->smem_bytes = smem;
+    return IM_OK;
+}
+
+im_status im_env_set_summary(im_env *e, uint64_t *acc)
+{
+    if (!e || (reinterpret_cast<uintptr_t>(acc) & 7u)) return IM_ERR_INVALID_ARG;
+    e->d_summary = reinterpret_cast<unsigned long long *>(acc);
     return IM_OK;
 }
 

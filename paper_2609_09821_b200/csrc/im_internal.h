@@ -73,6 +73,7 @@ struct EnvKernelParams {
     const float4 *links;      // [n_links][2]: the chains' ChainLink records
     const ClipMeta *meta;     // [C]
     int32_t C;
+    int32_t n_rows;           // keyframes of all clips together (rows of `frames`)
     // configuration
     int32_t N;
     uint32_t env_id_base;
@@ -91,6 +92,7 @@ struct EnvKernelParams {
     int32_t act_dim;                         // previous-action entries
     const float *prev_action;                // [N][ld_action]
     int32_t ld_action;
+    unsigned long long *summary;             // [4] training summaries (null: none)
     uint32_t step;
     // per-env state
     int32_t *clip_id;
@@ -145,6 +147,7 @@ struct im_env {
     uint32_t *d_stat_starts, *d_stat_failures;
     int32_t n_future, act_dim, ld_action;   // extended observation (im_env_set_obs_extension); D is the extended width
     const float *prev_action;
+    unsigned long long *d_summary;          // caller-owned accumulator of im_env_set_summary (null: none)
     // staging for the *_host entry points (allocated on first use)
     float *d_aos_sim;      // component rows gathered from array-of-structures inputs (allocated on first use)
     float *d_sim, *d_obs, *d_reward, *d_mean, *d_action;

@@ -448,3 +448,44 @@ def test_handles_created_from_two_threads_at_once():
     for a, b in zip(*results):
         assert torch.equal(a, b)                                 # same seeds, same results from both threads
     assert torch.equal(results[0][1], results[0][2])             # and the trainer's forward is the policy's
+
+
+def test_training_summaries_accumulate_on_the_device():
+    """im_env_set_summary: reward sum (fixed point), terminated / truncated counts and finished-episode lengths
+    accumulated by the step kernel itself; counts exact against the oracle's flags and episode lengths, the reward
+    sum exact against the kernel's own reward output and within tolerance of the oracle's rewards."""
+    sc = _scene("edge_summary", (361, 64, 28), "f32", n_clips=3, frames=(8, 20))
+    n = 333
+    p = Pair(sc, n, h_min=W.ROOT_HEIGHT, with_policy=False)
+    acc = torch.zeros(4, dtype=torch.int64, device="cuda")
+    p.g_env.set_summary(acc)
+    want = np.zeros(4, np.float64)
+    exact_reward = 0
+    p.reset_all()
+    assert acc.abs().sum().item() == 0                       # the reset-all launch adds nothing
+    lens = p.o_env.ep_len.copy()
+
+    def consume(s, sim):
+        nonlocal exact_reward, lens
+        out = p.env_step(s, sim)
+        fl = out["oracle"]["flags"]
+        want[0] += out["oracle"]["reward"].sum()
+        want[1] += (fl & 1).sum()
+        want[2] += ((fl >> 1) & 1).sum()
+        want[3] += (lens[fl != 0] + 1).sum()
+        exact_reward += int(np.rint(out["reward"].astype(np.float64) * 2.0 ** 40).astype(np.int64).sum())
+        lens = p.o_env.ep_len.copy()
+
+    W.rollout_inputs(sc.wl, sc.skel, sc.lib, lambda: (p.o_env.clip_id, p.o_env.t), consume, steps=9)
+    got = acc.cpu().numpy()
+    assert got[1] == want[1] and got[2] == want[2] and got[3] == want[3]
+    assert want[1] > 0 and want[2] > 0 and want[3] > want[1]
+    assert int(got[0]) == exact_reward
+    assert abs(got[0] / 2.0 ** 40 - want[0]) <= 9 * n * 2e-5
+    # detached: later steps leave the accumulator alone
+    p.g_env.set_summary(None)
+    before = acc.clone()
+    sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
+                                  torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, 10, sc.wl)
+    p.env_step(10, sim)
+    assert torch.equal(acc, before)
