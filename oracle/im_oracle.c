@@ -166,6 +166,8 @@ typedef struct {
     int64_t *start;    /* first frame of each clip in the packed tables */
     double *root;      /* [sum K][3] */
     double *quat;      /* [sum K][J][4], renormalised */
+    int *cyclic;       /* per clip: the motion repeats (orc_clips_set_cyclic); 0 by default */
+    double *shift;     /* [C][3] root displacement of one cycle, P[K-1] - P[0] */
 } orc_clips;
 
 orc_skeleton *orc_skeleton_create(int J, const int32_t *parents, const float *offsets,
@@ -213,7 +215,12 @@ orc_clips *orc_clips_create(const orc_skeleton *skel, int C, const int32_t *n_fr
     }
     c->root = (double *)malloc(sizeof(double) * total * 3);
     c->quat = (double *)malloc(sizeof(double) * total * J * 4);
+    c->cyclic = (int *)calloc(C, sizeof(int));
+    c->shift = (double *)calloc((size_t)3 * (size_t)C, sizeof(double));
     for (int64_t i = 0; i < total * 3; ++i) c->root[i] = (double)root_pos[i];
+    for (int i = 0; i < C; ++i)
+        for (int k = 0; k < 3; ++k)
+            c->shift[3*i + k] = (double)root_pos[3 * (c->start[i] + n_frames[i] - 1) + k] - (double)root_pos[3 * c->start[i] + k];
     for (int64_t i = 0; i < total * J; ++i) {
         double q[4] = {local_quat[4*i], local_quat[4*i+1], local_quat[4*i+2], local_quat[4*i+3]};
         quat_normalize(q);
@@ -225,7 +232,18 @@ orc_clips *orc_clips_create(const orc_skeleton *skel, int C, const int32_t *n_fr
 void orc_clips_destroy(orc_clips *c)
 {
     if (!c) return;
-    free(c->K); free(c->fps); free(c->dur); free(c->start); free(c->root); free(c->quat); free(c);
+    free(c->K); free(c->fps); free(c->dur); free(c->start); free(c->root); free(c->quat); free(c->cyclic); free(c->shift); free(c);
+}
+
+/* Cyclic clips (periodic motions such as the paper's walk and run): a clip flagged cyclic is played in a loop.
+ * Its last keyframe is the pose of the first one, displaced by the root translation of one cycle,
+ * shift = P[K-1] - P[0].  An env on such a clip never truncates: when its time reaches the clip's duration it
+ * wraps (one fp32 subtraction of the duration) and the env's cycle count goes up by one; the reference at cycle
+ * n is the clip's pose with n * shift added to the root (and so to every body).  flags: [C] bytes, or NULL to
+ * clear all. */
+void orc_clips_set_cyclic(orc_clips *c, const uint8_t *flags)
+{
+    for (int i = 0; i < c->C; ++i) c->cyclic[i] = flags ? (flags[i] != 0) : 0;
 }
 
 float orc_clip_duration(const orc_clips *c, int clip) { return c->dur[clip]; }
@@ -324,6 +342,30 @@ static void forward_kinematics(const orc_skeleton *s, orc_ref *r)
     center_of_mass(s, r->p, r->com);
 }
 
+/* Reference state of a cyclic clip in its cycle `cyc`: the clip's own state with cyc * shift added to every
+ * position (rotations and velocities repeat). */
+static void reference_state_cyc(const orc_skeleton *s, const orc_clips *cl, int clip, float t, int cyc, orc_ref *r)
+{
+    orc_reference_state(s, cl, clip, t, r);
+    if (cyc == 0) return;
+    for (int c = 0; c < 3; ++c) {
+        double d = (double)cyc * cl->shift[3*clip + c];
+        for (int j = 0; j < s->J; ++j) r->p[j][c] += d;
+        r->com[c] += d;
+    }
+}
+
+/* Time `t_in` moved `ahead` seconds on in a clip (fp32: one addition, and for a cyclic clip one subtraction
+ * of the duration per completed cycle): a non-cyclic clip clamps at its end.  *cyc is advanced. */
+static float time_ahead(const orc_clips *cl, int clip, float t_in, float ahead, int *cyc)
+{
+    volatile float t = t_in + ahead;
+    float dur = cl->dur[clip];
+    if (!cl->cyclic[clip]) return t < dur ? t : dur;
+    while (t >= dur) { t = t - dur; *cyc += 1; }
+    return t;
+}
+
 /* Flat export of orc_reference_state for the tests. */
 void orc_reference_state_flat(const orc_skeleton *s, const orc_clips *cl, int clip, float t,
                               double *p, double *q, double *v, double *w,
@@ -373,6 +415,7 @@ typedef struct {
     int32_t act_dim;
     const float *prev_action;       /* [n][ld_action] */
     int64_t ld_action;
+    int32_t *cycle;                 /* [n] per-env cycle count of cyclic clips (state, updated by the step), or NULL */
 } orc_env_config;
 
 /* Cumulative table of a weight table w[n] >= 0 (not all zero): T_i = floor(2^32 (w_0 + .. + w_i) / total)
@@ -570,7 +613,7 @@ static void ref_to_state(const orc_skeleton *s, const orc_ref *r, orc_body_state
 
 /* Step a6: heading-local observation of state x at (clip, t), D = 24J + 1. */
 static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_config *cfg,
-                      const orc_body_state *x, int clip, float t, double *obs, int i, int was_reset)
+                      const orc_body_state *x, int clip, float t, int cyc, double *obs, int i, int was_reset)
 {
     int J = s->J;
     const double ex[3] = {1.0, 0.0, 0.0}, ez[3] = {0.0, 0.0, 1.0};
@@ -593,10 +636,10 @@ static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_
     }
     obs[15 * J] = (double)t / (double)cl->dur[clip];
 
-    volatile float t_next = t + cfg->dt;                 /* one fp32 add */
-    float t_tgt = t_next < cl->dur[clip] ? t_next : cl->dur[clip];
+    int cyc_tgt = cyc;
+    float t_tgt = time_ahead(cl, clip, t, cfg->dt, &cyc_tgt);      /* one fp32 add; clamped, or wrapped on a cyclic clip */
     orc_ref tgt;
-    orc_reference_state(s, cl, clip, t_tgt, &tgt);
+    reference_state_cyc(s, cl, clip, t_tgt, cyc_tgt, &tgt);
     for (int j = 0; j < J; ++j) {
         double *o = obs + 15 * J + 1 + 9 * j, d[3], ql[4];
         for (int c = 0; c < 3; ++c) d[c] = tgt.p[j][c] - origin[c];
@@ -610,10 +653,10 @@ static void build_obs(const orc_skeleton *s, const orc_clips *cl, const orc_env_
     double *o = obs + 24 * J + 1;
     for (int f = 2; f <= cfg->n_future; ++f) {
         volatile float ahead = (float)f * cfg->dt;          /* one fp32 multiplication, */
-        volatile float t_f = t + ahead;                      /* one fp32 addition        */
-        float t_c = t_f < cl->dur[clip] ? t_f : cl->dur[clip];
+        int cyc_f = cyc;
+        float t_c = time_ahead(cl, clip, t, ahead, &cyc_f);  /* one fp32 addition; clamped or wrapped */
         orc_ref fut;
-        orc_reference_state(s, cl, clip, t_c, &fut);
+        reference_state_cyc(s, cl, clip, t_c, cyc_f, &fut);
         for (int j = 0; j < J; ++j) {
             int is_ee = 0;
             for (int k = 0; k < s->n_ee; ++k) is_ee |= (s->ee[k] == j);
@@ -671,10 +714,11 @@ void orc_env_reset_all(const orc_skeleton *s, const orc_clips *cl, const orc_env
         orc_body_state x;
         orc_reset_draw(cl, cfg, env_ids[i], step, &clip_id[i], &t[i]);
         ep_len[i] = 0;
+        if (cfg->cycle) cfg->cycle[i] = 0;
         orc_reference_state(s, cl, clip_id[i], t[i], &r);
         orc_reset_noise(s, cfg, env_ids[i], step, &r);
         ref_to_state(s, &r, &x);
-        build_obs(s, cl, cfg, &x, clip_id[i], t[i], obs + (int64_t)i * ld_obs, i, 1);
+        build_obs(s, cl, cfg, &x, clip_id[i], t[i], 0, obs + (int64_t)i * ld_obs, i, 1);
     }
 }
 
@@ -697,8 +741,15 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
         double e[ORC_N_TERMS];
         int clip = clip_id[i];
 
-        volatile float t1 = t[i] + cfg->dt;                         /* a0 */
-        orc_reference_state(s, cl, clip, t1, &r);                    /* a1, a2 */
+        int cyc = cfg->cycle ? cfg->cycle[i] : 0;
+        volatile float t_adv = t[i] + cfg->dt;                      /* a0: one fp32 add */
+        float t1 = t_adv;
+        if (cl->cyclic[clip] && t1 >= cl->dur[clip]) {              /* a cyclic clip wraps: one fp32 subtract */
+            volatile float t_wrap = t1 - cl->dur[clip];
+            t1 = t_wrap;
+            cyc += 1;
+        }
+        reference_state_cyc(s, cl, clip, t1, cyc, &r);               /* a1, a2 */
         load_sim(s, pos, quat, linvel, angvel, comp_stride, i, &x);
         error_terms(s, &x, &r, e);                                   /* a3 */
         double rew = orc_reward(&cfg->reward, e);
@@ -717,13 +768,14 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
             cfg->stat_failures[clip * cfg->n_bins + b] += 1u;
         }
         volatile float t2 = t1 + cfg->dt;
-        int truncated = t2 > cl->dur[clip];
+        int truncated = !cl->cyclic[clip] && t2 > cl->dur[clip];    /* a cyclic clip has no end */
         flags[i] = (uint8_t)(terminated | (truncated << 1));
 
         float t_cur = t1;
         if (flags[i]) {                                              /* a5 */
             orc_reset_draw(cl, cfg, env_ids[i], step, &clip, &t_cur);
             ep_len[i] = 0;
+            cyc = 0;
             orc_reference_state(s, cl, clip, t_cur, &r);
             orc_reset_noise(s, cfg, env_ids[i], step, &r);
             ref_to_state(s, &r, &x);
@@ -733,7 +785,8 @@ void orc_env_step(const orc_skeleton *s, const orc_clips *cl, const orc_env_conf
         }
         clip_id[i] = clip;
         t[i] = t_cur;
-        build_obs(s, cl, cfg, &x, clip, t_cur, obs + (int64_t)i * ld_obs, i, flags[i] != 0);   /* a6 */
+        if (cfg->cycle) cfg->cycle[i] = cyc;
+        build_obs(s, cl, cfg, &x, clip, t_cur, cyc, obs + (int64_t)i * ld_obs, i, flags[i] != 0);   /* a6 */
     }
 }
 

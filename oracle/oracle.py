@@ -41,7 +41,8 @@ class EnvConfig(C.Structure):
                 ("reward", RewardConfig), ("write_back_reset", C.c_int32), ("grace_steps", C.c_int32),
                 ("reset_noise_std", C.c_float), ("n_bins", C.c_int32), ("reset_cdf", C.c_void_p),
                 ("stat_starts", C.c_void_p), ("stat_failures", C.c_void_p),
-                ("n_future", C.c_int32), ("act_dim", C.c_int32), ("prev_action", C.c_void_p), ("ld_action", C.c_int64)]
+                ("n_future", C.c_int32), ("act_dim", C.c_int32), ("prev_action", C.c_void_p), ("ld_action", C.c_int64),
+                ("cycle", C.c_void_p)]
 
 
 _lib = None
@@ -65,6 +66,7 @@ def lib():
         L.orc_clips_create.argtypes = [vp, i32, vp, vp, vp, vp]
         L.orc_clips_create.restype = vp
         L.orc_clips_destroy.argtypes = [vp]
+        L.orc_clips_set_cyclic.argtypes = [vp, vp]
         L.orc_clip_duration.argtypes = [vp, i32]
         L.orc_clip_duration.restype = f32
         L.orc_lookup_index.argtypes = [f32, f32, i32, vp, vp]
@@ -214,6 +216,13 @@ class Clips:
     def duration(self, clip: int) -> np.float32:
         return np.float32(lib().orc_clip_duration(self.h, int(clip)))
 
+    def set_cyclic(self, flags) -> None:
+        """flags: one byte per clip (non-zero: the clip is played in a loop), or None to clear all."""
+        f = None if flags is None else np.ascontiguousarray(flags, np.uint8)
+        assert f is None or f.shape == (self.C,)
+        self.cyclic = np.zeros(self.C, np.uint8) if f is None else f.copy()
+        lib().orc_clips_set_cyclic(self.h, _p(f))
+
     def __del__(self):
         if getattr(self, "h", None) and _lib is not None:
             _lib.orc_clips_destroy(self.h)
@@ -254,6 +263,8 @@ class Env:
         self.clip_id = np.zeros(self.n, np.int32)
         self.t = np.zeros(self.n, np.float32)
         self.ep_len = np.zeros(self.n, np.int32)
+        self.cycle = np.zeros(self.n, np.int32)          # cycles completed on a cyclic clip (0 elsewhere)
+        self.cfg.cycle = self.cycle.ctypes.data
         self.D = 24 * skel.J + 1
         self.n_threads = int(n_threads or os.cpu_count() or 1)
 
