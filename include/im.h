@@ -103,6 +103,17 @@ im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_fra
                         const float *root_pos, const float *local_quat, im_clips **out);
 void im_destroy_clips(im_clips *c);
 
+/* Looped playback of periodic motions (the paper's Section 6 tracks walk and run cycles among its clips; it does
+ * not say how a clip's end is handled -- this is the library's reading).  flags: HOST [C] bytes, non-zero marks a
+ * clip as cyclic; NULL clears all.  A cyclic clip's last keyframe is taken to be the pose of its first one moved by
+ * the root translation of one cycle, shift_c = P_c[K-1] - P_c[0].  An env on such a clip never truncates: when its
+ * time reaches D_c it wraps, t <- fl32(t - D_c), and the env's cycle count n goes up by one; the reference at
+ * (c, t, n) is the clip's own state at t with n shift_c added to the root position (rotations and velocities
+ * repeat).  Look-ahead times (the target frame, further future frames) wrap the same way instead of clamping
+ * at D_c, each with the cycle count it reaches.  A reset starts a new episode at cycle 0.  The call waits for the
+ * device and takes effect for every env created on these clips, from its next step on. */
+im_status im_clips_set_cyclic(im_clips *c, const uint8_t *flags);
+
 /* ---- environment ----------------------------------------------------------
  * Reward (paper Section 6.1 and Figure 5) from seven error terms e_k between
  * the simulated character and the reference at the env's time:
@@ -222,6 +233,9 @@ im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim
  * rollout bit-exactly.  Any pointer may be NULL to skip that array. */
 im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_len);
 im_status im_env_set_state(im_env *e, const int32_t *clip_id, const float *t, const int32_t *ep_len);
+/* The cycle counts of envs on cyclic clips (0 elsewhere), DEVICE int32 [N]: the fourth piece of per-env state. */
+im_status im_env_get_cycles(im_env *e, int32_t *cycle);
+im_status im_env_set_cycles(im_env *e, const int32_t *cycle);
 
 /* ---- extended observation ---------------------------------------------------
  * (Section 6: observations also hold "future reference end-effector frames, and the

@@ -34,7 +34,8 @@ EXPORTS = [
     "im_trainer_push_to_policy", "im_trainer_tensor", "im_trainer_set_step_count", "im_trainer_dw_slices",
     "im_ppo_updater_create", "im_ppo_updater_destroy", "im_ppo_update", "im_ppo_update_rollout", "im_ppo_updater_tensor",
     "im_ppo_updater_set_step_count",
-    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait", "im_env_set_summary",
+    "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait", "im_env_set_summary", "im_clips_set_cyclic",
+    "im_env_get_cycles", "im_env_set_cycles",
 ]
 
 
@@ -163,6 +164,9 @@ def load():
         L.im_debug_math.argtypes = [i32, i32, vp, vp, vp]
         L.im_debug_set_wait.argtypes = [u64, i32]
         L.im_env_set_summary.argtypes = [vp, vp]
+        L.im_clips_set_cyclic.argtypes = [vp, vp]
+        L.im_env_get_cycles.argtypes = [vp, vp]
+        L.im_env_set_cycles.argtypes = [vp, vp]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp]
         L.im_trainer_create.argtypes = [i32, vp, vp, vp, i32, vp, C.POINTER(vp)]
@@ -255,6 +259,13 @@ class Clips:
         _check(L.im_load_clips(skel.h, self.C, _ptr(nf), _ptr(f), _ptr(rp), _ptr(lq), C.byref(self.h)),
                "im_load_clips")
 
+    def set_cyclic(self, flags=None):
+        """Marks clips as played in a loop (one byte per clip; None clears all)."""
+        f = None if flags is None else _np(flags, np.uint8)
+        if f is not None and f.shape != (self.C,):
+            raise ValueError("one flag per clip")
+        _check(load().im_clips_set_cyclic(self.h, _ptr(f)), "im_clips_set_cyclic")
+
     def __del__(self):
         if getattr(self, "h", None) and _lib is not None:
             _lib.im_destroy_clips(self.h)
@@ -328,6 +339,19 @@ class Env:
             _check(load().im_env_get_state(self.h, _ptr(c), _ptr(t), _ptr(l)), "im_env_get_state")
         self.stream.synchronize()
         return c, t, l
+
+    def get_cycles(self):
+        """Cycles completed by each env on a looped clip (int32 CUDA tensor)."""
+        import torch
+        c = torch.empty(self.n, dtype=torch.int32, device="cuda")
+        with torch.cuda.stream(self.stream):
+            _check(load().im_env_get_cycles(self.h, _ptr(c)), "im_env_get_cycles")
+        self.stream.synchronize()
+        return c
+
+    def set_cycles(self, cycle):
+        _check(load().im_env_set_cycles(self.h, _ptr(cycle)), "im_env_set_cycles")
+        self.stream.synchronize()
 
     def set_state(self, clip_id=None, t=None, ep_len=None):
         _check(load().im_env_set_state(self.h, _ptr(clip_id), _ptr(t), _ptr(ep_len)), "im_env_set_state")

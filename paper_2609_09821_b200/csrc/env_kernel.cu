@@ -297,6 +297,22 @@ __device__ __forceinline__ int phase_bin(float t, float span, int B)
     return min(max(b, 0), B - 1);
 }
 
+// Looped clips: root displacement after `cyc` completed cycles, and a time moved `ahead` seconds on -- clamped to
+// the clip's end, or, on a looped clip, wrapped (one fp32 subtraction per completed cycle, counted in cyc).
+__device__ __forceinline__ Vec3 loop_shift(const ClipLoop &loop, int cyc)
+{
+    const float n = (float)cyc;
+    return {n * loop.sx, n * loop.sy, n * loop.sz};
+}
+template <bool OPT>
+__device__ __forceinline__ float time_ahead(const ClipLoop &loop, float dur, float t, float ahead, int &cyc)
+{
+    float t2 = __fadd_rn(t, ahead);
+    if (!(OPT && loop.on)) return fminf(t2, dur);
+    for (int i = 0; i < 64 && t2 >= dur; ++i) { t2 = __fsub_rn(t2, dur); ++cyc; }
+    return t2;
+}
+
 // Heading frame of the character the observation is taken from: origin at the
 // root's (x, y, 0), yaw of the root's rotated x axis (step a6).
 struct Heading {
@@ -476,9 +492,10 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     if (c == 0)
         for (int i = 15 * J; i < c1; ++i) row1[i] = 0.0f;   // columns between the body blocks and the split
 
-    int clip = 0;
+    int clip = 0, cyc = 0;
     float t1 = 0.0f;
     ClipMeta cm = {2, 1.0f, 1.0f, 0};
+    ClipLoop loop = {0.0f, 0.0f, 0.0f, 0};
     Heading H = {0.0f, 0.0f, 1.0f, 0.0f};
     float root_z = 0.0f;
     const uint32_t st = (uint32_t)P.stride, e32 = (uint32_t)envc;
@@ -493,6 +510,12 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
         t1 = __fadd_rn(P.t[envc], P.dt);
         cm = P.meta[clip];
+        if (OPT && P.loops) {
+            // a clip played in a loop: the time wraps at the clip's end and the env's cycle count goes up
+            loop = P.loops[clip];
+            cyc = P.cycle[envc];
+            if (loop.on && t1 >= cm.dur) { t1 = __fsub_rn(t1, cm.dur); ++cyc; }
+        }
         int frame;
         float alpha;
         lookup(cm, t1, frame, alpha);
@@ -537,6 +560,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             Quat ql;
             Vec3 wl;
             joint_step<true>(r0, cur, alpha, cm.fps, Lc, k, s, ql, wl);
+            if (OPT && k == 0) s.p = s.p + loop_shift(loop, cyc);    // completed cycles of a looped clip move the root
             if (own) {
                 sim.q = sanitize(sim.q, P.status);
                 // the root's "parent" is the identity: qa = (1, 0, 0, 0), wa = 0 on the chain that owns it
@@ -614,7 +638,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             const float span = fmaxf(__fsub_rn(cm.dur, P.dt), 0.0f);
             atomicAdd(P.stat_failures + clip * P.n_bins + phase_bin(t1, span, P.n_bins), 1u);
         }
-        const bool truncated = __fadd_rn(t1, P.dt) > cm.dur;
+        const bool truncated = !(OPT && loop.on) && __fadd_rn(t1, P.dt) > cm.dur;    // a looped clip has no end
         flags = (terminated ? 1 : 0) | (truncated ? 2 : 0);
         reward_val = r;
         if (c == 0 && valid) P.flags_out[env] = (uint8_t)flags;
@@ -644,12 +668,14 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             t_cur = __fmul_rn(u, span);
         }
     }
+    if (reset) cyc = 0;
     if (c == 0) {
         int ep_done = 0;                    // steps of the episode this step ended (0 where none ended)
         if (valid) {
             const int len_now = P.ep_len[env] + 1;
             P.clip_id[env] = clip_cur;
             P.t[env] = t_cur;
+            if (OPT && P.loops) P.cycle[env] = cyc;
             P.ep_len[env] = reset ? 0 : len_now;
             ep_done = reset ? len_now : 0;
         }
@@ -667,6 +693,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         }
     }
     const ClipMeta cmc = reset ? P.meta[clip_cur] : cm;
+    if (OPT && P.loops && reset) loop = P.loops[clip_cur];
 
     // ---- pass C (only where an env of this warp was reset): reference state at the new phase
     //      replaces the simulated one in the observation, and optionally in the caller's arrays
@@ -716,7 +743,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
 
     // ---- the first half also holds the phase and the first floats of the root's target when 15 J
     //      is not a multiple of 4: chain 0 interpolates the root one interval ahead for them
-    const float t_tgt = fminf(__fadd_rn(t_cur, P.dt), cmc.dur);
+    int cyc_t = cyc;
+    const float t_tgt = time_ahead<OPT>(loop, cmc.dur, t_cur, P.dt, cyc_t);
     int frame_t;
     float alpha_t;
     lookup(cmc, t_tgt, frame_t, alpha_t);
@@ -726,7 +754,9 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         phase = t_cur / cmc.dur;
         if (15 * J < c1) {
             const KeyPair root = ld_pair(rt0);
-            const Vec3 tp = H.local(Vec3{fmaf(alpha_t, root.b.x, root.a.x), fmaf(alpha_t, root.b.y, root.a.y), 0.0f});
+            Vec3 rp = {fmaf(alpha_t, root.b.x, root.a.x), fmaf(alpha_t, root.b.y, root.a.y), 0.0f};
+            if (OPT) rp = rp + loop_shift(loop, cyc_t);
+            const Vec3 tp = H.local(rp);
             row1[15 * J] = phase;
             if (15 * J + 1 < c1) row1[15 * J + 1] = tp.x;
             if (15 * J + 2 < c1) row1[15 * J + 2] = tp.y;
@@ -759,6 +789,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             Quat ql;
             Vec3 wl;
             joint_step<false>(rt0, cur, alpha_t, cmc.fps, Lc, k, s, ql, wl);
+            if (OPT && k == 0) s.p = s.p + loop_shift(loop, cyc_t);
             if (Lc.flags & LINK_OWN) {
                 float o[9];
                 target_obs(H, s.q, s.p, o);
@@ -777,7 +808,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             // frames f = 2 .. n_future of the reference, t + f dt (two fp32 operations, clamped to the clip's end):
             // every chain walks them again and the owner of an end effector writes its nine entries
             for (int f = 2; f <= P.n_future; ++f) {
-                const float t_f = fminf(__fadd_rn(t_cur, __fmul_rn((float)f, P.dt)), cmc.dur);
+                int cyc_f = cyc;
+                const float t_f = time_ahead<OPT>(loop, cmc.dur, t_cur, __fmul_rn((float)f, P.dt), cyc_f);
                 int frame_f;
                 float alpha_f;
                 lookup(cmc, t_f, frame_f, alpha_f);
@@ -790,6 +822,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
                     Quat ql;
                     Vec3 wl;
                     joint_step<false>(rf0, kp, alpha_f, cmc.fps, Lf, k, sf, ql, wl);
+                    if (k == 0) sf.p = sf.p + loop_shift(loop, cyc_f);
                     if ((Lf.flags & LINK_OWN) && (Lf.flags & LINK_EE)) {
                         float o[9];
                         target_obs(H, sf.q, sf.p, o);
@@ -903,7 +936,7 @@ cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t s
 {
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
     const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0 || p.n_future > 1 || p.act_dim > 0 ||
-                     p.summary != nullptr;
+                     p.summary != nullptr || p.loops != nullptr;
     if (opt) {
         if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
         else launch_one<false, true>(p, grid, block, smem, stream);

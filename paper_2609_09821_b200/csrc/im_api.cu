@@ -146,13 +146,17 @@ im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_fra
 
     im_clips *cl = new (std::nothrow) im_clips();
     if (!cl) return IM_ERR_ALLOC;
-    cl->C = C; cl->J = J; cl->rows = rows; cl->d_frames = nullptr; cl->d_meta = nullptr;
+    cl->C = C; cl->J = J; cl->rows = rows; cl->d_frames = nullptr; cl->d_meta = nullptr; cl->d_loops = nullptr;
+    cl->any_loop = false;
     cl->meta.resize(C);
+    cl->loops.resize(C);
     cl->min_dur = INFINITY;
     int32_t start = 0;
     for (int c = 0; c < C; ++c) {
         cl->meta[c] = {n_frames[c], fps[c], (float)(n_frames[c] - 1) / fps[c], start};
         cl->min_dur = std::fmin(cl->min_dur, cl->meta[c].dur);
+        const float *p0 = root_pos + 3 * (int64_t)start, *p1 = root_pos + 3 * ((int64_t)start + n_frames[c] - 1);
+        cl->loops[c] = {(float)((double)p1[0] - p0[0]), (float)((double)p1[1] - p0[1]), (float)((double)p1[2] - p0[2]), 0};
         start += n_frames[c];
     }
     // The table rows (see clip_table_kernel) are built on the device from copies of the caller's arrays.
@@ -165,7 +169,8 @@ im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_fra
     // (one extra row of zeros so that the last frame's "next" reads stay inside the buffers)
     const size_t root_b = (size_t)(rows + 1) * 3 * sizeof(float), quat_b = (size_t)(rows + 1) * J * 4 * sizeof(float);
     bool ok = cudaMalloc(&cl->d_frames, (size_t)rows * RS * sizeof(float4)) == cudaSuccess &&
-              cudaMalloc(&cl->d_meta, C * sizeof(ClipMeta)) == cudaSuccess && cudaMalloc(&d_root, root_b) == cudaSuccess &&
+              cudaMalloc(&cl->d_meta, C * sizeof(ClipMeta)) == cudaSuccess && cudaMalloc(&cl->d_loops, C * sizeof(ClipLoop)) == cudaSuccess &&
+              cudaMalloc(&d_root, root_b) == cudaSuccess &&
               cudaMalloc(&d_quat, quat_b) == cudaSuccess && cudaMalloc(&d_last, (size_t)rows) == cudaSuccess;
     im_status st = ok ? IM_OK : IM_ERR_ALLOC;
     if (ok) {
@@ -174,6 +179,7 @@ im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_fra
              cudaMemcpy(d_quat, local_quat, (size_t)rows * J * 4 * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(d_last, last.data(), (size_t)rows, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(cl->d_meta, cl->meta.data(), C * sizeof(ClipMeta), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(cl->d_loops, cl->loops.data(), C * sizeof(ClipLoop), cudaMemcpyHostToDevice) == cudaSuccess &&
              launch_clip_table(d_root, d_quat, d_last, rows, J, cl->d_frames, nullptr) == cudaSuccess &&
              cudaDeviceSynchronize() == cudaSuccess;
         if (!ok) st = IM_ERR_CUDA;
@@ -192,7 +198,21 @@ void im_destroy_clips(im_clips *c)
     if (!c) return;
     cudaFree(c->d_frames);
     cudaFree(c->d_meta);
+    cudaFree(c->d_loops);
     delete c;
+}
+
+im_status im_clips_set_cyclic(im_clips *c, const uint8_t *flags)
+{
+    if (!c) return IM_ERR_INVALID_ARG;
+    c->any_loop = false;
+    for (int i = 0; i < c->C; ++i) {
+        c->loops[i].on = flags && flags[i] ? 1 : 0;
+        c->any_loop = c->any_loop || c->loops[i].on;
+    }
+    IM_CUDA(cudaDeviceSynchronize());           // steps in flight keep the flags they were launched with
+    IM_CUDA(cudaMemcpy(c->d_loops, c->loops.data(), c->C * sizeof(ClipLoop), cudaMemcpyHostToDevice));
+    return IM_OK;
 }
 
 /* ------------------------------------------------------------------ env */
@@ -229,6 +249,7 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     const size_t n = (size_t)cfg->n_envs;
     if (cudaMalloc(&e->d_clip_id, n * 4) != cudaSuccess || cudaMalloc(&e->d_t, n * 4) != cudaSuccess ||
         cudaMalloc(&e->d_ep_len, n * 4) != cudaSuccess || cudaMalloc(&e->d_status, 4) != cudaSuccess ||
+        cudaMalloc(&e->d_cycle, n * 4) != cudaSuccess ||
         cudaMalloc(&e->d_links, (size_t)skel->dev.n_links * sizeof(ChainLink)) != cudaSuccess) {
         im_env_destroy(e);
         return IM_ERR_ALLOC;
@@ -240,6 +261,7 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
     cudaMemsetAsync(e->d_clip_id, 0, n * 4, e->stream);
     cudaMemsetAsync(e->d_t, 0, n * 4, e->stream);
     cudaMemsetAsync(e->d_ep_len, 0, n * 4, e->stream);
+    cudaMemsetAsync(e->d_cycle, 0, n * 4, e->stream);
     cudaMemsetAsync(e->d_status, 0, 4, e->stream);
     *out = e;
     return IM_OK;
@@ -248,7 +270,7 @@ im_status im_env_create(const im_skeleton *skel, const im_clips *clips, const im
 void im_env_destroy(im_env *e)
 {
     if (!e) return;
-    cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status); cudaFree(e->d_links);
+    cudaFree(e->d_clip_id); cudaFree(e->d_t); cudaFree(e->d_ep_len); cudaFree(e->d_status); cudaFree(e->d_links); cudaFree(e->d_cycle);
     cudaFree(e->d_sim); cudaFree(e->d_obs); cudaFree(e->d_reward); cudaFree(e->d_mean);
     cudaFree(e->d_action); cudaFree(e->d_flags);
     cudaFree(e->d_reset_cdf); cudaFree(e->d_stat_starts); cudaFree(e->d_stat_failures);
@@ -289,6 +311,8 @@ static void fill_params(const im_env *e, uint32_t step, EnvKernelParams &p)
     p.prev_action = e->prev_action;
     p.ld_action = e->ld_action;
     p.summary = e->d_summary;
+    p.loops = e->clips->any_loop ? e->clips->d_loops : nullptr;
+    p.cycle = e->d_cycle;
     p.step = step;
     p.clip_id = e->d_clip_id;
     p.t = e->d_t;
@@ -337,7 +361,7 @@ static im_status env_step_range(im_env *e, uint32_t step, const im_body_state *s
     fill_params(e, step, p);
     p.N = count;
     p.env_id_base += (uint32_t)first;
-    p.clip_id += first; p.t += first; p.ep_len += first;
+    p.clip_id += first; p.t += first; p.ep_len += first; p.cycle += first;
     p.pos = sim->pos + first; p.quat = sim->quat + first; p.lin = sim->linvel + first; p.ang = sim->angvel + first;
     p.stride = sim->comp_stride;
     p.obs = obs_out + (size_t)first * e->cfg.ld_obs;
@@ -395,6 +419,20 @@ im_status im_env_get_state(im_env *e, int32_t *clip_id, float *t, int32_t *ep_le
     if (clip_id) IM_CUDA(cudaMemcpyAsync(clip_id, e->d_clip_id, b, cudaMemcpyDeviceToDevice, e->stream));
     if (t) IM_CUDA(cudaMemcpyAsync(t, e->d_t, b, cudaMemcpyDeviceToDevice, e->stream));
     if (ep_len) IM_CUDA(cudaMemcpyAsync(ep_len, e->d_ep_len, b, cudaMemcpyDeviceToDevice, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_get_cycles(im_env *e, int32_t *cycle)
+{
+    if (!e || !cycle) return IM_ERR_INVALID_ARG;
+    IM_CUDA(cudaMemcpyAsync(cycle, e->d_cycle, (size_t)e->cfg.n_envs * 4, cudaMemcpyDeviceToDevice, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_set_cycles(im_env *e, const int32_t *cycle)
+{
+    if (!e || !cycle) return IM_ERR_INVALID_ARG;
+    IM_CUDA(cudaMemcpyAsync(e->d_cycle, cycle, (size_t)e->cfg.n_envs * 4, cudaMemcpyDeviceToDevice, e->stream));
     return IM_OK;
 }
 

@@ -31,6 +31,12 @@ struct ChainLink {
 constexpr int LINK_OWN = 1, LINK_EE = 2;
 constexpr int IM_MAX_LINKS = 288;          // sum of chain lengths for any tree of up to 32 bodies (<= 16 x 17)
 
+// Per-clip record of looped playback (im_clips_set_cyclic): the root displacement of one cycle and the flag.
+struct ClipLoop {
+    float sx, sy, sz;
+    int32_t on;
+};
+
 // Skeleton as the kernels see it (passed by value inside the kernel parameters).
 // Kinematic chains: one root-to-leaf path per leaf.  A body shared by several paths is owned by the first of
 // them; within a path the owned bodies are a suffix starting at chain_first_own.  The links of all chains lie
@@ -93,6 +99,8 @@ struct EnvKernelParams {
     const float *prev_action;                // [N][ld_action]
     int32_t ld_action;
     unsigned long long *summary;             // [4] training summaries (null: none)
+    const ClipLoop *loops;                   // [C] looped clips (null: no clip of the library loops)
+    int32_t *cycle;                          // per-env cycle count on a looped clip
     uint32_t step;
     // per-env state
     int32_t *clip_id;
@@ -123,6 +131,9 @@ struct im_clips {
     float4 *d_frames;
     im::ClipMeta *d_meta;
     std::vector<im::ClipMeta> meta;
+    std::vector<im::ClipLoop> loops;       // root displacement per cycle; `on` set by im_clips_set_cyclic
+    im::ClipLoop *d_loops;
+    bool any_loop;
     float min_dur;
     int device;
 };
@@ -138,6 +149,7 @@ struct im_env {
     float *d_t;
     int32_t *d_ep_len;
     uint32_t *d_status;
+    int32_t *d_cycle;      // cycles completed on a looped clip
     float4 *d_links;       // the skeleton's chain links on the env's device
     int D;                 // observation width: 24J + 1 plus the extension columns
     size_t smem_bytes;

@@ -145,6 +145,7 @@ class Pair:
         np.testing.assert_array_equal(t.cpu().numpy().view(np.uint32), self.o_env.t.view(np.uint32),
                                       err_msg=what + " time bit patterns")
         np.testing.assert_array_equal(l.cpu().numpy(), self.o_env.ep_len, err_msg=what + " episode lengths")
+        np.testing.assert_array_equal(self.g_env.get_cycles().cpu().numpy(), self.o_env.cycle, err_msg=what + " cycle counts")
 
     def check_obs(self, what):
         g = self.obs_g.cpu().numpy()

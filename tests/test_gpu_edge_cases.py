@@ -489,3 +489,41 @@ def test_training_summaries_accumulate_on_the_device():
                                   torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, 10, sc.wl)
     p.env_step(10, sim)
     assert torch.equal(acc, before)
+
+
+# ---------------------------------------------------------------- looped clips
+@pytest.mark.parametrize("skeleton,dims,extras", [("humanoid15", (361, 64, 28), dict()),
+                                                    ("smpl24", (577, 64, 69), dict(n_future=3, prev_action_dim=4)),
+                                                    ("humanoid15", (361, 64, 28), dict(grace_steps=2, write_back=True))])
+def test_looped_clips_wrap_and_carry_the_root_along(skeleton, dims, extras):
+    """A library that mixes looped and plain clips, run for more than two periods of the looped ones: time wraps, the
+    cycle count (a fourth piece of per-env state, compared exactly) goes up, the root displacement of every completed
+    cycle reaches the observation and the error terms, the plain clips truncate as before.  The simulator stand-in
+    follows the continuous motion, so looped envs keep tracking well past the wrap."""
+    sc = _scene("edge_loop_" + skeleton, dims, "f32", skeleton=skeleton, n_clips=4, frames=(61, 61), seed=9)
+    flags = np.array([1, 0, 1, 1], np.uint8)
+    sc.o_clips.set_cyclic(flags)
+    sc.g_clips.set_cyclic(flags)
+    n = 120
+    p = Pair(sc, n, h_min=0.3, with_policy=False, **extras)
+    p.reset_all()
+    dur = np.float32(2.0)
+    hist = []
+
+    def consume(s, sim):
+        if p.prev_o is not None:
+            p.prev_o[:] = np.random.default_rng(1000 + s).standard_normal(p.prev_o.shape).astype(np.float32)
+            p.prev_g.copy_(torch.from_numpy(p.prev_o))
+        hist.append(p.env_step(s, sim))
+
+    # the continuous time of an env = time inside the clip + completed cycles x duration
+    W.rollout_inputs(sc.wl, sc.skel, sc.lib,
+                     lambda: (p.o_env.clip_id, p.o_env.t.astype(np.float64) + p.o_env.cycle * float(dur)), consume, steps=130)
+    looped = flags[p.o_env.clip_id].astype(bool)
+    assert p.o_env.cycle[looped].max() >= 2 and np.all(p.o_env.cycle[~looped] == 0)
+    assert any(((h["flags"] & 2) != 0).any() for h in hist)                  # plain clips truncated
+    early = [h["reward"].mean() for h in hist[:10]]
+    late = [h["reward"][looped].mean() for h in hist[-20:]]
+    assert np.mean(late) > 0.5 * np.mean(early)                              # tracking as well after two wraps as before any
+    sc.g_clips.set_cyclic(None)
+    sc.o_clips.set_cyclic(None)
