@@ -210,11 +210,15 @@ im_status im_env_step(im_env *e, uint32_t step, const im_body_state *sim,
  * six floats per body (point linvel and angvel into the same array, body_stride 6),
  * are described without copying.  pos, linvel, angvel have 3 components, quat 4
  * (w,x,y,z).  DEVICE; no alignment requirement.
- * One gather kernel transposes the records into component rows inside the library
- * (first call allocates that buffer: not capturable), then the env kernel runs as in
- * im_env_step -- results are identical to im_env_step on the transposed data.  With
- * write_back_reset, the states of reset envs are scattered back into the caller's
- * arrays. */
+ * The env kernel reads the records where they lie (every thread walks the record of its env; with
+ * write_back_reset the states of reset envs are stored back the same way): nothing is staged, nothing
+ * allocated, the call is capturable like im_env_step, and the results are those of im_env_step on the
+ * transposed data, bit for bit.  Per-thread record reads are not coalesced, so the step is slower than on
+ * component rows (measured at 65536 envs x 24 bodies: 213 us against 126 us).  im_env_set_aos_staging(e, 1)
+ * trades memory for time: it allocates a [13J][N] buffer once (outside any capture), after which
+ * im_env_step_aos first transposes the records into it with one gather kernel and runs the env kernel on the
+ * rows (168 us in the same measurement), scattering reset envs back; im_env_set_aos_staging(e, 0) frees the
+ * buffer and returns to in-place reading. */
 typedef struct {
     float *base;
     int64_t env_stride;
@@ -227,6 +231,7 @@ typedef struct {
 
 im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim,
                           float *obs_out, float *reward_out, uint8_t *flags_out, float *terms_out);
+im_status im_env_set_aos_staging(im_env *e, int32_t on);
 
 /* Copies the per-env state to / from DEVICE arrays of N elements (stream
  * ordered); with the step number this is all that is needed to resume a

@@ -35,7 +35,7 @@ EXPORTS = [
     "im_ppo_updater_create", "im_ppo_updater_destroy", "im_ppo_update", "im_ppo_update_rollout", "im_ppo_updater_tensor",
     "im_ppo_updater_set_step_count",
     "im_copy_f32", "im_gemm_bf16_tn", "im_gather_rows_f32", "im_gemm_bf16_dgrad", "im_env_set_obs_extension", "im_env_adapt_reset_bins", "im_debug_math", "im_debug_set_wait", "im_env_set_summary", "im_clips_set_cyclic",
-    "im_env_get_cycles", "im_env_set_cycles",
+    "im_env_get_cycles", "im_env_set_cycles", "im_env_set_aos_staging",
 ]
 
 
@@ -166,6 +166,7 @@ def load():
         L.im_env_set_summary.argtypes = [vp, vp]
         L.im_clips_set_cyclic.argtypes = [vp, vp]
         L.im_env_get_cycles.argtypes = [vp, vp]
+        L.im_env_set_aos_staging.argtypes = [vp, i32]
         L.im_env_set_cycles.argtypes = [vp, vp]
         L.im_env_set_obs_extension.argtypes = [vp, i32, i32, vp, i32]
         L.im_gemm_bf16_dgrad.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, i32, vp, vp]
@@ -339,6 +340,10 @@ class Env:
             _check(load().im_env_get_state(self.h, _ptr(c), _ptr(t), _ptr(l)), "im_env_get_state")
         self.stream.synchronize()
         return c, t, l
+
+    def set_aos_staging(self, on: bool = True):
+        """step_aos through a library-owned [13J][N] staging buffer (faster, allocated here) instead of in place."""
+        _check(load().im_env_set_aos_staging(self.h, int(on)), "im_env_set_aos_staging")
 
     def get_cycles(self):
         """Cycles completed by each env on a looped clip (int32 CUDA tensor)."""

@@ -393,17 +393,62 @@ __device__ __forceinline__ Quat sanitize(Quat q, uint32_t *status)
     return q;
 }
 
-// Body-state loads.  Element (row, env) of an array lies at row * stride + env; the offsets are 32-bit
-// (the launcher checks that the arrays are smaller than 2^31 elements); `o` is the offset of the body's
-// first row at this thread's env.
-__device__ __forceinline__ Quat ld_sim_quat(const float *base, uint32_t o, uint32_t st)
-{
-    return {base[o], base[o + st], base[o + 2 * st], base[o + 3 * st]};
-}
-__device__ __forceinline__ Vec3 ld_sim_vec(const float *base, uint32_t o, uint32_t st)
-{
-    return {base[o], base[o + st], base[o + 2 * st]};
-}
+// Body-state access of one thread (one env).  Two layouts:
+//   component rows (AOS = false): element (row, env) of an array lies at row * stride + env, rows 3 b + c (4 b + c for
+//     the quaternions); a warp load is one full line.  Offsets are 32-bit (the launcher checks the array sizes).
+//   simulator records (AOS = true): element (env, body b, component c) lies at base + env * env_stride +
+//     b * body_stride + c, read where the simulator keeps it; every lane walks its own record, the components of a
+//     body are adjacent words.
+template <bool AOS>
+struct SimView {
+    float *pos, *quat, *lin, *ang;        // rows: array bases; records: this env's record in each array
+    uint32_t st, e;                       // rows
+    int bs_pos, bs_quat, bs_lin, bs_ang;  // records: floats between two bodies
+
+    __device__ __forceinline__ SimView(const EnvKernelParams &P, int envc)
+    {
+        if (AOS) {
+            pos = P.pos + (long long)envc * P.aos_env_stride[0];
+            quat = P.quat + (long long)envc * P.aos_env_stride[1];
+            lin = P.lin + (long long)envc * P.aos_env_stride[2];
+            ang = P.ang + (long long)envc * P.aos_env_stride[3];
+            bs_pos = P.aos_body_stride[0]; bs_quat = P.aos_body_stride[1]; bs_lin = P.aos_body_stride[2]; bs_ang = P.aos_body_stride[3];
+            st = 0; e = 0;
+        } else {
+            pos = P.pos; quat = P.quat; lin = P.lin; ang = P.ang;
+            st = (uint32_t)P.stride; e = (uint32_t)envc;
+            bs_pos = bs_quat = bs_lin = bs_ang = 0;
+        }
+    }
+    __device__ __forceinline__ Quat ld_quat(int b) const
+    {
+        if (AOS) { const float *p = quat + (long long)b * bs_quat; return {p[0], p[1], p[2], p[3]}; }
+        const uint32_t o = 4 * (uint32_t)b * st + e;
+        return {quat[o], quat[o + st], quat[o + 2 * st], quat[o + 3 * st]};
+    }
+    __device__ __forceinline__ Vec3 ld_vec(const float *base, int bs, int b) const
+    {
+        if (AOS) { const float *p = base + (long long)b * bs; return {p[0], p[1], p[2]}; }
+        const uint32_t o = 3 * (uint32_t)b * st + e;
+        return {base[o], base[o + st], base[o + 2 * st]};
+    }
+    __device__ __forceinline__ Vec3 ld_pos(int b) const { return ld_vec(pos, bs_pos, b); }
+    __device__ __forceinline__ Vec3 ld_lin(int b) const { return ld_vec(lin, bs_lin, b); }
+    __device__ __forceinline__ Vec3 ld_ang(int b) const { return ld_vec(ang, bs_ang, b); }
+    __device__ __forceinline__ void st_vec(float *base, int bs, int b, Vec3 v) const
+    {
+        if (AOS) { float *p = base + (long long)b * bs; p[0] = v.x; p[1] = v.y; p[2] = v.z; return; }
+        const uint32_t o = 3 * (uint32_t)b * st + e;
+        base[o] = v.x; base[o + st] = v.y; base[o + 2 * st] = v.z;
+    }
+    __device__ __forceinline__ void st_body(int b, Quat q, Vec3 p, Vec3 v, Vec3 w) const
+    {
+        st_vec(pos, bs_pos, b, p); st_vec(lin, bs_lin, b, v); st_vec(ang, bs_ang, b, w);
+        if (AOS) { float *d = quat + (long long)b * bs_quat; d[0] = q.w; d[1] = q.x; d[2] = q.y; d[3] = q.z; return; }
+        const uint32_t o = 4 * (uint32_t)b * st + e;
+        quat[o] = q.w; quat[o + st] = q.x; quat[o + 2 * st] = q.y; quat[o + 3 * st] = q.z;
+    }
+};
 
 __device__ __forceinline__ float4 lds128(uint32_t addr)
 {
@@ -455,7 +500,7 @@ __device__ __forceinline__ void copy_out_any(const EnvKernelParams &P, const flo
 // the first target floats -- and columns [c1, D) -- the targets.
 // OPT compiles in the optional semantics (grace steps, motion randomisation, adaptive initialisation, extended
 // observation); envs that use none run the instantiation without them.
-template <bool RESET_ALL, bool OPT>
+template <bool RESET_ALL, bool OPT, bool AOS>
 __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *smem_raw)
 {
     // a successor launched with programmatic stream serialization (the policy's first GEMM) may be scheduled
@@ -498,7 +543,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
     ClipLoop loop = {0.0f, 0.0f, 0.0f, 0};
     Heading H = {0.0f, 0.0f, 1.0f, 0.0f};
     float root_z = 0.0f;
-    const uint32_t st = (uint32_t)P.stride, e32 = (uint32_t)envc;
+    const SimView<AOS> sv(P, envc);
 
     // ---- pass A: reference at the advanced time, errors against the simulated state,
     //      observation entries of the simulated bodies
@@ -523,8 +568,8 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         LinkRec L = ld_link(links, 0);
         KeyPair keys = ld_keys(r0, L.b);
 
-        const Quat q_root = sanitize(ld_sim_quat(P.quat, e32, st), P.status);
-        const Vec3 p_root = ld_sim_vec(P.pos, e32, st);
+        const Quat q_root = sanitize(sv.ld_quat(0), P.status);
+        const Vec3 p_root = sv.ld_pos(0);
         H = make_heading(q_root, p_root);
         root_z = p_root.z;
 
@@ -535,9 +580,9 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
         Quat qa = {1, 0, 0, 0};                      // simulated state of the previous body of the chain
         Vec3 wa = {0, 0, 0};
         if (first_own > 0) {
-            const uint32_t a = (uint32_t)ld_link(links, first_own - 1).b;
-            qa = sanitize(ld_sim_quat(P.quat, 4 * a * st + e32, st), P.status);
-            wa = ld_sim_vec(P.ang, 3 * a * st + e32, st);
+            const int a = ld_link(links, first_own - 1).b;
+            qa = sanitize(sv.ld_quat(a), P.status);
+            wa = sv.ld_ang(a);
         }
         for (int k = 0; k < len; ++k) {
             const LinkRec Lc = L;
@@ -545,12 +590,11 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             const bool own = Lc.flags & LINK_OWN;
             SimBody sim;
             if (own) {                                // issue the loads before the interpolation math
-                const uint32_t o3 = 3 * (uint32_t)b * st + e32;
-                (void)IM_CHECKED((4 * (uint32_t)b + 3) * st + e32, 4u * (uint32_t)J * st);
-                sim.q = ld_sim_quat(P.quat, 4 * (uint32_t)b * st + e32, st);
-                sim.p = ld_sim_vec(P.pos, o3, st);
-                sim.v = ld_sim_vec(P.lin, o3, st);
-                sim.w = ld_sim_vec(P.ang, o3, st);
+                if (!AOS) (void)IM_CHECKED((4 * (uint32_t)b + 3) * sv.st + sv.e, 4u * (uint32_t)J * sv.st);
+                sim.q = sv.ld_quat(b);
+                sim.p = sv.ld_pos(b);
+                sim.v = sv.ld_lin(b);
+                sim.w = sv.ld_ang(b);
             }
             const KeyPair cur = keys;
             if (k + 1 < len) {                        // next joint's link and keyframe words in flight
@@ -730,11 +774,7 @@ __device__ __forceinline__ void env_step_body(const EnvKernelParams &P, float *s
             if ((Lc.flags & LINK_OWN) && reset) {
                 body_obs(Hn, s.q, s.p, s.v, s.w, row1, b);
                 if (!RESET_ALL && P.write_back && valid) {
-                    const uint32_t o3 = 3 * (uint32_t)b * st + e32, o4 = 4 * (uint32_t)b * st + e32;
-                    P.pos[o3] = s.p.x; P.pos[o3 + st] = s.p.y; P.pos[o3 + 2 * st] = s.p.z;
-                    P.quat[o4] = s.q.w; P.quat[o4 + st] = s.q.x; P.quat[o4 + 2 * st] = s.q.y; P.quat[o4 + 3 * st] = s.q.z;
-                    P.lin[o3] = s.v.x; P.lin[o3 + st] = s.v.y; P.lin[o3 + 2 * st] = s.v.z;
-                    P.ang[o3] = s.w.x; P.ang[o3 + st] = s.w.y; P.ang[o3 + 2 * st] = s.w.z;
+                    sv.st_body(b, s.q, s.p, s.v, s.w);
                 }
             }
         }
@@ -867,34 +907,34 @@ __global__ void debug_math_kernel(int op, int n, const float *__restrict__ in, f
 #ifndef IM_ENV_MAXNREG
 #define IM_ENV_MAXNREG 96
 #endif
-template <bool RESET_ALL, bool OPT>
+template <bool RESET_ALL, bool OPT, bool AOS>
 __global__ void __maxnreg__(IM_ENV_MAXNREG) env_step_kernel_small(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
-    env_step_body<RESET_ALL, OPT>(P, smem_raw);
+    env_step_body<RESET_ALL, OPT, AOS>(P, smem_raw);
 }
 
-template <bool RESET_ALL, bool OPT>
+template <bool RESET_ALL, bool OPT, bool AOS>
 __global__ void __launch_bounds__(1024, 1) env_step_kernel_wide(const __grid_constant__ EnvKernelParams P)
 {
     extern __shared__ __align__(16) float smem_raw[];
-    env_step_body<RESET_ALL, OPT>(P, smem_raw);
+    env_step_body<RESET_ALL, OPT, AOS>(P, smem_raw);
 }
 
-template <bool RESET_ALL, bool OPT>
+template <bool RESET_ALL, bool OPT, bool AOS>
 cudaError_t prepare_one(size_t smem)
 {
     const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(env_step_kernel_small<RESET_ALL, OPT>, attr, (int)smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<RESET_ALL, OPT>, attr, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(env_step_kernel_small<RESET_ALL, OPT, AOS>, attr, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(env_step_kernel_wide<RESET_ALL, OPT, AOS>, attr, (int)smem);
     return e;
 }
 
-template <bool RESET_ALL, bool OPT>
+template <bool RESET_ALL, bool OPT, bool AOS>
 void launch_one(const EnvKernelParams &p, dim3 grid, dim3 block, size_t smem, cudaStream_t stream)
 {
-    if (block.x <= 256) env_step_kernel_small<RESET_ALL, OPT><<<grid, block, smem, stream>>>(p);
-    else env_step_kernel_wide<RESET_ALL, OPT><<<grid, block, smem, stream>>>(p);
+    if (block.x <= 256) env_step_kernel_small<RESET_ALL, OPT, AOS><<<grid, block, smem, stream>>>(p);
+    else env_step_kernel_wide<RESET_ALL, OPT, AOS><<<grid, block, smem, stream>>>(p);
 }
 
 }  // namespace
@@ -908,10 +948,12 @@ cudaError_t env_kernel_prepare(size_t smem)
 {
     static DeviceOnce once;
     return once.run([&] {
-        cudaError_t e = prepare_one<false, false>(smem);
-        if (e == cudaSuccess) e = prepare_one<true, false>(smem);
-        if (e == cudaSuccess) e = prepare_one<false, true>(smem);
-        if (e == cudaSuccess) e = prepare_one<true, true>(smem);
+        cudaError_t e = prepare_one<false, false, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<true, false, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<false, true, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<true, true, false>(smem);
+        if (e == cudaSuccess) e = prepare_one<false, false, true>(smem);
+        if (e == cudaSuccess) e = prepare_one<false, true, true>(smem);
         return e;
     });
 }
@@ -937,12 +979,15 @@ cudaError_t launch_env_kernel(const EnvKernelParams &p, bool reset_all, size_t s
     const dim3 grid((p.N + kTile - 1) / kTile), block(32 * p.sk.n_chains);
     const bool opt = p.grace_steps > 0 || p.reset_noise_std > 0.0f || p.n_bins > 0 || p.n_future > 1 || p.act_dim > 0 ||
                      p.summary != nullptr || p.loops != nullptr;
-    if (opt) {
-        if (reset_all) launch_one<true, true>(p, grid, block, smem, stream);
-        else launch_one<false, true>(p, grid, block, smem, stream);
+    if (p.aos && !reset_all) {               // simulator records read in place (the reset-all launch reads no body states)
+        if (opt) launch_one<false, true, true>(p, grid, block, smem, stream);
+        else launch_one<false, false, true>(p, grid, block, smem, stream);
+    } else if (opt) {
+        if (reset_all) launch_one<true, true, false>(p, grid, block, smem, stream);
+        else launch_one<false, true, false>(p, grid, block, smem, stream);
     } else {
-        if (reset_all) launch_one<true, false>(p, grid, block, smem, stream);
-        else launch_one<false, false>(p, grid, block, smem, stream);
+        if (reset_all) launch_one<true, false, false>(p, grid, block, smem, stream);
+        else launch_one<false, false, false>(p, grid, block, smem, stream);
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();

@@ -375,8 +375,9 @@ static im_status env_step_range(im_env *e, uint32_t step, const im_body_state *s
 im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim, float *obs_out, float *reward_out,
                           uint8_t *flags_out, float *terms_out)
 {
-    if (!e || !sim || !obs_out || !reward_out || !flags_out || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
-    const int J = e->skel->dev.J, N = e->cfg.n_envs;
+    if (!e || !sim || !reward_out || !flags_out || !aligned16(obs_out)) return IM_ERR_INVALID_ARG;
+    if (!obs_out && !e->d_obs_bf16) return IM_ERR_INVALID_ARG;
+    const int J = e->skel->dev.J;
     const im_aos_array *arr[4] = {&sim->pos, &sim->quat, &sim->linvel, &sim->angvel};
     for (int i = 0; i < 4; ++i) {
         const int comps = i == 1 ? 4 : 3;
@@ -384,18 +385,44 @@ im_status im_env_step_aos(im_env *e, uint32_t step, const im_body_state_aos *sim
             arr[i]->env_stride < (int64_t)(J - 1) * arr[i]->body_stride + comps)
             return IM_ERR_INVALID_ARG;
     }
-    const int64_t stride = ((int64_t)N + 3) / 4 * 4;
-    if (!e->d_aos_sim) {
-        if (aos_adapter_prepare() != cudaSuccess) return IM_ERR_CUDA;
-        if (cudaMalloc(&e->d_aos_sim, (size_t)13 * J * stride * sizeof(float)) != cudaSuccess) return IM_ERR_ALLOC;
+    if (e->d_aos_sim) {
+        // staging was asked for (im_env_set_aos_staging): one gather kernel turns the records into component rows,
+        // the env kernel then streams those; reset envs are scattered back
+        const int N = e->cfg.n_envs;
+        const int64_t stride = ((int64_t)N + 3) / 4 * 4;
+        IM_CUDA(launch_aos_gather(*sim, J, N, e->d_aos_sim, stride, e->stream));
+        im_body_state rows = {e->d_aos_sim, e->d_aos_sim + 3 * J * stride, e->d_aos_sim + 7 * J * stride,
+                              e->d_aos_sim + 10 * J * stride, stride};
+        const im_status s = im_env_step(e, step, &rows, obs_out, reward_out, flags_out, terms_out);
+        if (s != IM_OK) return s;
+        if (e->cfg.write_back_reset)
+            IM_CUDA(launch_aos_scatter_reset(*sim, J, N, e->d_aos_sim, stride, flags_out, e->stream));
+        return IM_OK;
     }
-    IM_CUDA(launch_aos_gather(*sim, J, N, e->d_aos_sim, stride, e->stream));
-    im_body_state rows = {e->d_aos_sim, e->d_aos_sim + 3 * J * stride, e->d_aos_sim + 7 * J * stride,
-                          e->d_aos_sim + 10 * J * stride, stride};
-    const im_status s = im_env_step(e, step, &rows, obs_out, reward_out, flags_out, terms_out);
-    if (s != IM_OK) return s;
-    if (e->cfg.write_back_reset)
-        IM_CUDA(launch_aos_scatter_reset(*sim, J, N, e->d_aos_sim, stride, flags_out, e->stream));
+    // the env kernel reads (and, for reset envs with write_back_reset, writes) the simulator's records where they are
+    EnvKernelParams p;
+    fill_params(e, step, p);
+    p.pos = sim->pos.base; p.quat = sim->quat.base; p.lin = sim->linvel.base; p.ang = sim->angvel.base;
+    p.aos = 1;
+    for (int i = 0; i < 4; ++i) { p.aos_env_stride[i] = arr[i]->env_stride; p.aos_body_stride[i] = arr[i]->body_stride; }
+    p.obs = obs_out; p.reward_out = reward_out; p.flags_out = flags_out; p.terms_out = terms_out;
+    IM_CUDA(launch_env_kernel(p, false, e->smem_bytes, e->stream));
+    return IM_OK;
+}
+
+im_status im_env_set_aos_staging(im_env *e, int32_t on)
+{
+    if (!e) return IM_ERR_INVALID_ARG;
+    if (!on) {
+        IM_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_aos_sim);
+        e->d_aos_sim = nullptr;
+        return IM_OK;
+    }
+    if (e->d_aos_sim) return IM_OK;
+    const int64_t stride = ((int64_t)e->cfg.n_envs + 3) / 4 * 4;
+    if (aos_adapter_prepare() != cudaSuccess) return IM_ERR_CUDA;
+    if (cudaMalloc(&e->d_aos_sim, (size_t)13 * e->skel->dev.J * stride * sizeof(float)) != cudaSuccess) return IM_ERR_ALLOC;
     return IM_OK;
 }
 

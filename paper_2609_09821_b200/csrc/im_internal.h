@@ -108,7 +108,10 @@ struct EnvKernelParams {
     int32_t *ep_len;
     // per-step I/O
     float *pos, *quat, *lin, *ang;
-    long long stride;
+    long long stride;                        // component rows: floats between two rows
+    int32_t aos;                             // non-zero: simulator records read in place, described by the two arrays below
+    long long aos_env_stride[4];             // pos, quat, linvel, angvel: floats between two envs
+    int32_t aos_body_stride[4];              //                            floats between two bodies
     float *obs;
     uint16_t *obs_bf16;       // optional bf16 copy of the observation rows (same row stride), or null
     float *reward_out;

@@ -257,11 +257,13 @@ def test_bin_weights_adapted_on_the_device_match_the_oracle():
 
 
 # ---------------------------------------------------------------- simulator-native input arrays
+@pytest.mark.parametrize("staged", [False, True], ids=["in_place", "staged"])
 @pytest.mark.parametrize("skeleton,dims,n", [("humanoid15", (361, 64, 28), 333), ("smpl24", (577, 64, 69), 200)])
-def test_step_on_array_of_structures_inputs(skeleton, dims, n):
+def test_step_on_array_of_structures_inputs(skeleton, dims, n, staged):
     """Body states laid out as a physics engine keeps them -- [env][body][component] with a leading world
     body and angular|linear velocity stored as six floats -- give bit for bit what the component-row
-    layout gives (which the other tests hold against the oracle), and reset envs are written back."""
+    layout gives (which the other tests hold against the oracle), and reset envs are written back: read in place
+    by the env kernel (nothing allocated: the free device memory does not move), or through the staging buffer."""
     sc = _scene("edge_aos_" + skeleton, dims, "f32", skeleton=skeleton, sigma_root=0.05)
     J = sc.J
     p = Pair(sc, n, h_min=W.ROOT_HEIGHT, write_back=True, with_policy=False, seed=9)
@@ -274,6 +276,8 @@ def test_step_on_array_of_structures_inputs(skeleton, dims, n):
     rew2 = torch.empty(n, device="cuda")
     fl2 = torch.empty(n, dtype=torch.uint8, device="cuda")
     terms2 = torch.empty((7, n), device="cuda")
+    if staged:
+        env2.set_aos_staging(True)
     for s in (1, 2, 3):
         sim = W.synth_sim_state_torch(sc.skel, sc.lib, torch.from_numpy(p.o_env.clip_id.astype(np.int64)),
                                       torch.from_numpy(p.o_env.t.astype(np.float64)) + sc.wl.dt, s, sc.wl).cuda()
@@ -284,7 +288,11 @@ def test_step_on_array_of_structures_inputs(skeleton, dims, n):
         xquat[:, 1:] = sim[3 * J:7 * J].reshape(J, 4, n).permute(2, 0, 1)
         cvel[:, 1:, 3:] = sim[7 * J:10 * J].reshape(J, 3, n).permute(2, 0, 1)
         cvel[:, 1:, :3] = sim[10 * J:13 * J].reshape(J, 3, n).permute(2, 0, 1)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         env2.step_aos(s, xpos[:, 1:], xquat[:, 1:], cvel[:, 1:, 3:], cvel[:, 1:, :3], obs2, rew2, fl2, terms2)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before              # the call itself allocates nothing
         out = p.env_step(s, sim)                                       # component rows, checked against the oracle
         torch.cuda.synchronize()
         assert torch.equal(obs2, p.obs_g) and torch.equal(rew2, p.reward_g) and torch.equal(fl2, p.flags_g)
