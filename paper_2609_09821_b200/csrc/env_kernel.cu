@@ -147,16 +147,20 @@ __device__ __forceinline__ float asin2_over_u(float u)
 
 // Keyframe words of one joint: the rotation and the log of the step to the next keyframe.  The two
 // 16-byte words are one aligned 32-byte sector, fetched with a single 256-bit load: every lane gathers from a
-// row of its own, so each load instruction costs the load pipe one pass per lane.
+// row of its own, so each load instruction costs the load pipe one pass per lane.  The loads ask L2 to evict the
+// table last: it is a few MB that every step gathers from, while hundreds of MB of body states and observation
+// rows (and the policy's activations between two steps) stream through the same cache.
 struct KeyPair {
     float4 a, b;
 };
 __device__ __forceinline__ KeyPair ld_pair(const float4 *p)
 {
     KeyPair k;
-    asm("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+    uint64_t keep;
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+    asm("ld.global.nc.L2::cache_hint.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8], %9;"
         : "=f"(k.a.x), "=f"(k.a.y), "=f"(k.a.z), "=f"(k.a.w), "=f"(k.b.x), "=f"(k.b.y), "=f"(k.b.z), "=f"(k.b.w)
-        : "l"(p));
+        : "l"(p), "l"(keep));
     return k;
 }
 __device__ __forceinline__ KeyPair ld_keys(const float4 *r0, int b) { return ld_pair(r0 + 2 + 2 * b); }
@@ -424,13 +428,14 @@ struct SimView {
     {
         if (AOS) { const float *p = quat + (long long)b * bs_quat; return {p[0], p[1], p[2], p[3]}; }
         const uint32_t o = 4 * (uint32_t)b * st + e;
-        return {quat[o], quat[o + st], quat[o + 2 * st], quat[o + 3 * st]};
+        // streaming loads (evict first): the body states are read once, the keyframe table should stay in L2
+        return {__ldcs(quat + o), __ldcs(quat + o + st), __ldcs(quat + o + 2 * st), __ldcs(quat + o + 3 * st)};
     }
     __device__ __forceinline__ Vec3 ld_vec(const float *base, int bs, int b) const
     {
         if (AOS) { const float *p = base + (long long)b * bs; return {p[0], p[1], p[2]}; }
         const uint32_t o = 3 * (uint32_t)b * st + e;
-        return {base[o], base[o + st], base[o + 2 * st]};
+        return {__ldcs(base + o), __ldcs(base + o + st), __ldcs(base + o + 2 * st)};
     }
     __device__ __forceinline__ Vec3 ld_pos(int b) const { return ld_vec(pos, bs_pos, b); }
     __device__ __forceinline__ Vec3 ld_lin(int b) const { return ld_vec(lin, bs_lin, b); }
@@ -476,7 +481,7 @@ __device__ __forceinline__ void copy_out(const EnvKernelParams &P, const float *
         int i = lane;
         for (; i < quads; i += 32, src += 512u) {
             const float4 v = lds128(src);
-            if (F32) { *dst = v; dst += 32; }
+            if (F32) { __stcs(dst, v); dst += 32; }                 // streamed: written once, not read by this kernel
             if (BF16) { *dst16 = pack_bf16x4(v); dst16 += 32; }
         }
         for (; i < last - first; i += 32) {
