@@ -304,7 +304,7 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short device-resident runs of the other benchmark configurations")
     ap.add_argument("--replays", type=int, default=REPLAYS, help="replays of the K-step graph (median reported)")
-    ap.add_argument("--only", default=None, choices=["env", "policy", "gae", "ppo_loss", "update"],
+    ap.add_argument("--only", default=None, choices=["env", "policy", "gae", "ppo_loss", "update", "fusion_probe"],
                     help="time one piece in a plain loop and print its own JSON line")
     ap.add_argument("--launches", type=int, default=40, help="launches of the --only loop")
     args = ap.parse_args()
@@ -442,6 +442,39 @@ def main():
         if rank == 0:
             print(json.dumps(dict(only=args.only, workload=wl.name, us_per_launch=res, launches=args.launches,
                                   bf16_rows=bool(staged), reset_fraction=float((flags != 0).float().mean()))))
+        return
+
+    if args.only == "fusion_probe":
+        # What fusing the env step with the policy's first layer could save in memory traffic: (a) the env step with
+        # and without the bf16 rows it leaves for the policy; (b) the policy forward on rows that are still in L2
+        # (the same launch repeated) against rows that have to come from HBM (256 MB read in between).
+        def loop(fn, n_l=args.launches, between=None):
+            out = []
+            for rep in range(3):
+                tot = 0.0
+                for i in range(n_l):
+                    if between is not None:
+                        between()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    fn(i)
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    tot += a.elapsed_time(b)
+                out.append(tot / n_l * 1e3)
+            return float(np.median(out))
+        res = dict(only="fusion_probe", workload=wl.name)
+        res["env_fp32_and_bf16_rows_us"] = loop(lambda i: env.step(Wm + 1 + i, sims[i % n_buf], obs, reward, flags))
+        if staged:
+            env.attach_policy(None)
+            res["env_fp32_rows_only_us"] = loop(lambda i: env.step(Wm + 1 + i, sims[i % n_buf], obs, reward, flags))
+            env.attach_policy(policy)
+            env.step(Wm + 1, sims[0], obs, reward, flags)
+        flush = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
+        res["policy_rows_in_l2_us"] = loop(lambda i: policy_forward(Wm + 1 + i))
+        res["policy_rows_from_hbm_us"] = loop(lambda i: policy_forward(Wm + 1 + i), between=lambda: flush.sum())
+        if rank == 0:
+            print(json.dumps(res))
         return
 
     sampler = ClockSampler(local_rank)
