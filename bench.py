@@ -163,12 +163,12 @@ def oracle_leg(wl: W.Workload, skel, lib, pol, n_sample: int, steps: int, warmup
 
 # ----------------------------------------------------------------------------- rollout-side pieces
 # Timed on their own (not part of the metric).
-def time_gae(B, wl, n, dev, stream, reps=20):
-    """The advantage estimator over one rollout of wl.steps steps.  Its 17 B per env-step fit in L2, so a 256 MB
+def time_gae(B, wl, n, dev, stream, reps=20, T=None):
+    """The advantage estimator over one rollout of T (default wl.steps) steps.  Its 17 B per env-step fit in L2, so a 256 MB
     buffer is read before every launch (reading leaves clean lines behind: a written buffer's write-back would
     be charged to the kernel)."""
     import torch
-    T = wl.steps
+    T = T or wl.steps
     r_np, v_np, f_np = W.make_rollout_signals(T, n, wl.seed)
     r_d, v_d, f_d = (torch.from_numpy(a).to(dev) for a in (r_np, v_np, f_np))
     adv_d, ret_d = torch.empty((T, n), device=dev), torch.empty((T, n), device=dev)
@@ -267,8 +267,38 @@ def time_update(B, wl, pol, n, A, D, dev, stream, graph=True, reps=5):
                 note="forward + backward + Adam of actor and critic on one minibatch; flops = 3 x forward flops")
 
 
+def time_gemm(B, shape, dev, stream, launches=20, reps=7):
+    """C = relu(A W^T + b) in bf16 through im_gemm_bf16 for one (M, N, K): back-to-back launches, median of `reps`
+    loops, and a comparison of the first 512 rows with a float32 product of the same operands."""
+    import torch
+    M, N, K = (int(x) for x in shape.split(","))
+    gen = torch.Generator(device=dev).manual_seed(1)
+    a = torch.randn((M, K), device=dev, generator=gen).to(torch.bfloat16)
+    w = (torch.randn((N, K), device=dev, generator=gen) * K ** -0.5).to(torch.bfloat16)
+    c = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    bias = torch.zeros(N, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        B.gemm_bf16(a, w, c, bias, True, status, stream=stream)
+    torch.cuda.synchronize()
+    t = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(launches):
+            B.gemm_bf16(a, w, c, bias, True, status, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t.append(e0.elapsed_time(e1) / launches * 1e-3)
+    sec = float(np.median(t))
+    ref = torch.relu(a[:512].float() @ w.float().T)
+    err = float((c[:512].float() - ref).abs().max() / (ref.abs().max() + 1e-9))
+    return dict(M=M, N=N, K=K, seconds_per_launch=sec, achieved_tflops=2.0 * M * N * K / sec / 1e12,
+                max_rel_err_first_512_rows=err, status=int(status.item()))
+
+
 def only_rollout_piece(args):
-    """`--only gae|ppo_loss|update`: that piece alone, in the loop the profiles of those kernels were taken from."""
+    """`--only gae|ppo_loss|update|gemm`: that piece alone, in the loop the profiles of those kernels were taken from."""
     import torch
     from paper_2609_09821_b200 import binding as B
     B.load()
@@ -277,9 +307,11 @@ def only_rollout_piece(args):
     torch.cuda.set_device(dev)
     stream = torch.cuda.Stream()
     torch.cuda.set_stream(stream)
-    n, A, D = wl.n_envs, wl.act_dim, wl.obs_dim
+    n, A, D = args.envs or wl.n_envs, wl.act_dim, wl.obs_dim
     if args.only == "gae":
-        res = time_gae(B, wl, n, dev, stream, reps=args.launches)
+        res = time_gae(B, wl, n, dev, stream, reps=args.launches, T=args.horizon)
+    elif args.only == "gemm":
+        res = time_gemm(B, args.shape, dev, stream, launches=args.launches)
     elif args.only == "ppo_loss":
         res = time_ppo_loss(B, wl, n, A, dev, stream, reps=args.launches)
     else:
@@ -304,11 +336,15 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short device-resident runs of the other benchmark configurations")
     ap.add_argument("--replays", type=int, default=REPLAYS, help="replays of the K-step graph (median reported)")
-    ap.add_argument("--only", default=None, choices=["env", "policy", "gae", "ppo_loss", "update", "fusion_probe"],
+    ap.add_argument("--only", default=None,
+                    choices=["env", "policy", "gae", "ppo_loss", "update", "gemm", "fusion_probe"],
                     help="time one piece in a plain loop and print its own JSON line")
     ap.add_argument("--launches", type=int, default=40, help="launches of the --only loop")
+    ap.add_argument("--envs", type=int, default=None, help="--only gae|ppo_loss|update: envs instead of the workload's")
+    ap.add_argument("--horizon", type=int, default=None, help="--only gae: steps instead of the workload's")
+    ap.add_argument("--shape", default="65536,1024,1024", help="--only gemm: M,N,K of the bf16 product")
     args = ap.parse_args()
-    if args.only in ("gae", "ppo_loss", "update"):
+    if args.only in ("gae", "ppo_loss", "update", "gemm"):
         return only_rollout_piece(args)
 
     rank = int(os.environ.get("RANK", "0"))
