@@ -97,8 +97,10 @@ void im_destroy_skeleton(im_skeleton *s);
  *   root_pos   HOST [sum K][3]
  *   local_quat HOST [sum K][J][4]  w,x,y,z; must be finite with | |q| - 1 | <= 1e-3; used as given (the
  *                                 interpolation and velocity formulas do not depend on the small scale error)
- * The table is copied to the current CUDA device in rows padded to 16 bytes
- * ([x y z 0 | q_0 | q_1 ...]); free with im_destroy_clips. */
+ * The device table is built on the current CUDA device from these arrays (fp64 arithmetic, stored as fp32): per
+ * keyframe one row of 2 + 2J 16-byte words -- root position, root displacement to the next keyframe, and per
+ * joint the normalised quaternion and the half-angle logarithm of the shorter-arc rotation to the next keyframe
+ * -- so that interpolating a joint is one 32-byte read.  Free with im_destroy_clips. */
 im_status im_load_clips(const im_skeleton *skel, int32_t C, const int32_t *n_frames, const float *fps,
                         const float *root_pos, const float *local_quat, im_clips **out);
 void im_destroy_clips(im_clips *c);
