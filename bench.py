@@ -60,9 +60,9 @@ SUSTAINED_SECONDS = 1.0
 NCU_TRAFFIC = {
     "cfg4_65536_smpl24": dict(
         policy=dict(bytes=645075456, capture="linear_tc_hidden_pair_kernel<0, 0> x 3 + linear_tc_head_kernel<80>, one policy "
-                                              "forward, profiles/linear_tc_kernels_cfg4_65536_smpl24.md"),
+                                              "forward at 65536 envs (ncu --set full)"),
         env=dict(bytes=291532288, capture="env_step_kernel_small<0, 0, 0> writing fp32 and bf16 rows, one launch, "
-                                          "profiles/env_step_kernel_cfg4_65536_smpl24.md")),
+                                          "65536 envs (ncu --set full)")),
 }
 
 
