@@ -77,11 +77,26 @@ __global__ void __launch_bounds__(256) adam_kernel(const AdamParams P)
 constexpr int kSqThreads = 256;
 constexpr int kSqMaxGrid = 64;             // partial sums per tensor
 
-__global__ void __launch_bounds__(kSqThreads) sumsq_kernel(const float *__restrict__ x, long long n, double *__restrict__ partial)
+// Sum of squares of up to kSqMaxTensors tensors in one launch.  Tensor k owns blocks [first[k], first[k+1]) of the
+// grid and as many partial sums; a block adds its grid-strided share of the tensor in double precision.
+constexpr int kSqMaxTensors = 64;
+struct SumSqArgs {
+    const float *x[kSqMaxTensors];
+    long long n[kSqMaxTensors];
+    int first[kSqMaxTensors + 1];
+    int n_tensors;
+};
+
+__global__ void __launch_bounds__(kSqThreads) sumsq_kernel(const __grid_constant__ SumSqArgs a, double *__restrict__ partial)
 {
     __shared__ double s[kSqThreads];
+    int k = 0;
+    while (k + 1 < a.n_tensors && (int)blockIdx.x >= a.first[k + 1]) ++k;
+    const float *__restrict__ x = a.x[k];
+    const long long n = a.n[k];
+    const int blocks = a.first[k + 1] - a.first[k], blk = (int)blockIdx.x - a.first[k];
     double q = 0.0;
-    for (long long i = (long long)blockIdx.x * kSqThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kSqThreads) {
+    for (long long i = (long long)blk * kSqThreads + threadIdx.x; i < n; i += (long long)blocks * kSqThreads) {
         const double v = (double)__ldg(x + i);
         q = fma(v, v, q);
     }
@@ -161,16 +176,23 @@ im_status im_grad_scale(int32_t n_tensors, const float *const *grads, const int6
     if (reinterpret_cast<uintptr_t>(workspace) & 7u) return IM_ERR_INVALID_ARG;
     double *partial = static_cast<double *>(workspace);
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    SumSqArgs a;
+    a.n_tensors = n_tensors;
     int count = 0;
     for (int k = 0; k < n_tensors; ++k) {
         if (!grads[k] || sizes[k] < 1) return IM_ERR_INVALID_ARG;
         long long g = (sizes[k] + kSqThreads * 8 - 1) / (kSqThreads * 8);
         const int grid = (int)(g < 1 ? 1 : (g > kSqMaxGrid ? kSqMaxGrid : g));
-        sumsq_kernel<<<grid, kSqThreads, 0, st>>>(grads[k], sizes[k], partial + count);
+        a.x[k] = grads[k];
+        a.n[k] = sizes[k];
+        a.first[k] = count;
         count += grid;
     }
+    for (int k = n_tensors; k <= kSqMaxTensors; ++k) a.first[k] = count;
+    for (int k = n_tensors; k < kSqMaxTensors; ++k) { a.x[k] = nullptr; a.n[k] = 0; }
+    sumsq_kernel<<<count, kSqThreads, 0, st>>>(a, partial);
     grad_scale_finish_kernel<<<1, 32, 0, st>>>(partial, count, max_norm, scale_out);
-    g_launches.fetch_add((uint64_t)n_tensors + 1, std::memory_order_relaxed);
+    g_launches.fetch_add(2, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? IM_OK : IM_ERR_CUDA;
 }
 
