@@ -20,10 +20,12 @@
  * no CPU access on the rollout step; reset is unconditional with a device-side
  * mask), so a sequence of them can be captured in a CUDA graph (Section 2.2).
  *
- * Threads: a handle may be used from one host thread at a time; different
- * handles may be used from different threads once each kind of handle has been
- * created once (the first creation also configures the kernels' shared-memory
- * limits, which is not guarded).
+ * Threads and devices: a handle may be used from one host thread at a time;
+ * different handles may be created and used from different threads.  A handle
+ * belongs to the CUDA device that was current when it was created and must be
+ * used with that device current; the kernels' one-time set-up (shared-memory
+ * limits, SM count) is done once per device, guarded against concurrent first
+ * calls.
  *
  * Errors: a call that returns a negative status has had no effect.  Anomalies
  * found on the device (a non-finite quaternion, a wait that ran out) set bits
